@@ -1,0 +1,283 @@
+// AdaComp oracle: a plain, slow, single-threaded CPU statement of what the
+// worker-side gradient selection and the parameter-server update compute.
+//
+// THIS IS TEST INFRASTRUCTURE.  It exists so that the CUDA library can be
+// checked against something written straight from the paper.  It shares no
+// code, header, table or helper with the CUDA path and must never be called
+// from it.  Everything here is exact (integer work on fp32 bit patterns, and
+// fp32 arithmetic with one rounding per operation), so results are unique.
+//
+// Parity status: every function below is pinned by tests that do not call it
+// to produce their expectation (brute-force set definitions on tiny inputs,
+// the paper's worked staleness example, closed forms, invariants).  The only
+// thing that stays "parity unpinned" is what this file does not compute at
+// all: model accuracy and traffic curves, which need the paper's dataset.
+//
+// Build: g++ -std=c++17 -O2 -ffp-contract=off -fno-fast-math -shared -fPIC
+
+#include <algorithm>
+#include <cstdint>
+#include <cstring>
+#include <numeric>
+#include <vector>
+
+namespace {
+
+// Magnitude key of a gradient entry: the fp32 bit pattern with the sign bit
+// cleared.  For every non-NaN float, unsigned order of this key equals the
+// order of |g| ("largest parameters, in absolute value", Algorithm 1,
+// SELECT_GRAD); +0 and -0 get the same key.
+inline uint32_t magnitude_key(float g) {
+    uint32_t bits;
+    std::memcpy(&bits, &g, sizeof bits);
+    return bits & 0x7FFFFFFFu;
+}
+
+// The total order that makes the selection unique: larger magnitude first,
+// and among equal magnitudes the lower index first.
+struct LargerMagnitudeThenLowerIndex {
+    const float* g;
+    bool operator()(uint32_t a, uint32_t b) const {
+        const uint32_t ka = magnitude_key(g[a]), kb = magnitude_key(g[b]);
+        if (ka != kb) return ka > kb;
+        return a < b;
+    }
+};
+
+void emit_ascending(const float* g, std::vector<uint32_t>& chosen, uint64_t offset,
+                    uint32_t* idx_out, float* val_out) {
+    std::sort(chosen.begin(), chosen.end());
+    for (size_t t = 0; t < chosen.size(); ++t) {
+        idx_out[t] = static_cast<uint32_t>(offset + chosen[t]);
+        val_out[t] = g[chosen[t]];   // the raw gradient entry, bit for bit
+    }
+}
+
+}  // namespace
+
+extern "C" {
+
+// How many entries a fraction c = c_num / c_den keeps of a tensor of n
+// entries: ceil(c * n), at least 1, at most n.  The paper only says "the
+// (100 x c)% largest" (Algorithm 1, SELECT_GRAD); the ceiling keeps every
+// tensor represented, which is the stated purpose of selecting per tensor
+// ("Selection method" paragraph).  n = 0 keeps nothing.
+uint32_t oracle_keep_count(uint64_t n, uint32_t c_num, uint32_t c_den) {
+    if (n == 0 || c_den == 0) return 0;
+    unsigned __int128 prod = static_cast<unsigned __int128>(n) * c_num;
+    unsigned __int128 k = (prod + c_den - 1) / c_den;
+    if (k < 1) k = 1;
+    if (k > n) k = n;
+    return static_cast<uint32_t>(k);
+}
+
+// SELECT_GRAD on one tensor, written as its definition (Algorithm 1,
+// SELECT_GRAD; "Selection method" paragraph): order ALL entries by decreasing
+// |g| (ties: lower index first), keep the first k, report them by ascending
+// index as (offset + e, g[e]).  Returns 0, or -1 on k > n.
+int oracle_select_sort(const float* g, uint32_t n, uint32_t k, uint64_t offset,
+                       uint32_t* idx_out, float* val_out) {
+    if (k > n) return -1;
+    std::vector<uint32_t> order(n);
+    std::iota(order.begin(), order.end(), 0u);
+    std::sort(order.begin(), order.end(), LargerMagnitudeThenLowerIndex{g});
+    std::vector<uint32_t> chosen(order.begin(), order.begin() + k);
+    emit_ascending(g, chosen, offset, idx_out, val_out);
+    return 0;
+}
+
+// The same selection with a partial sort (std::nth_element) under the same
+// total order.  The order is strict and total, so the first k elements after
+// partitioning are the same set as in oracle_select_sort.  This is the variant
+// used on large inputs.
+int oracle_select(const float* g, uint32_t n, uint32_t k, uint64_t offset,
+                  uint32_t* idx_out, float* val_out) {
+    if (k > n) return -1;
+    std::vector<uint32_t> order(n);
+    std::iota(order.begin(), order.end(), 0u);
+    if (k > 0 && k < n)
+        std::nth_element(order.begin(), order.begin() + (k - 1), order.end(),
+                         LargerMagnitudeThenLowerIndex{g});
+    std::vector<uint32_t> chosen(order.begin(), order.begin() + k);
+    emit_ascending(g, chosen, offset, idx_out, val_out);
+    return 0;
+}
+
+// SELECT_GRAD over a whole gradient vector: each tensor (V_l or beta_l) is a
+// contiguous range [offset_l, offset_l + n_l) and is selected independently
+// (the fraction is "per V_l or beta_l", notation table).  Output: the tensors'
+// selections one after the other, sum(k_l) pairs.
+int oracle_select_layers(const float* grad, const uint64_t* offsets, const uint32_t* ns,
+                         const uint32_t* ks, uint32_t n_layers, int use_full_sort,
+                         uint32_t* idx_out, float* val_out) {
+    uint64_t out = 0;
+    for (uint32_t l = 0; l < n_layers; ++l) {
+        int rc = use_full_sort
+            ? oracle_select_sort(grad + offsets[l], ns[l], ks[l], offsets[l], idx_out + out, val_out + out)
+            : oracle_select(grad + offsets[l], ns[l], ks[l], offsets[l], idx_out + out, val_out + out);
+        if (rc != 0) return rc;
+        out += ks[l];
+    }
+    return 0;
+}
+
+// ---------------------------------------------------------------------------
+// Parameter server (Algorithm 2), two statements of the same function.
+// ---------------------------------------------------------------------------
+
+// One fp32 parameter update, Eq. 4 with the learning rate of Eq. 5:
+//   alpha_k = alpha / sigma_k  if sigma_k != 0, else alpha
+//   Theta_k <- Theta_k - alpha_k * dTheta_k
+// Each operation is rounded to fp32 on its own (divide, multiply, subtract);
+// the build forbids fusing the last two.
+static inline float updated_parameter(float theta_k, float alpha, uint32_t sigma_k, float delta_k) {
+    const float alpha_k = (sigma_k != 0) ? alpha / static_cast<float>(sigma_k) : alpha;
+    const float step = alpha_k * delta_k;
+    return theta_k - step;
+}
+
+// --- literal form -----------------------------------------------------------
+// Keeps every past update as the set of parameter indices it changed with a
+// non-zero value, and evaluates Eq. 3 as written: for each entry of the
+// arriving update, test membership of k in every update u = j .. i-1.
+struct LiteralServer {
+    std::vector<float> theta;
+    uint64_t timestamp = 0;                         // i: number of updates applied so far
+    std::vector<std::vector<uint32_t>> nonzero_idx; // nonzero_idx[u] = sorted {k : dTheta_k(u) != 0}
+};
+
+void* oracle_literal_create(uint64_t n_params, const float* theta0) {
+    auto* s = new LiteralServer;
+    s->theta.assign(theta0, theta0 + n_params);
+    return s;
+}
+void oracle_literal_destroy(void* h) { delete static_cast<LiteralServer*>(h); }
+uint64_t oracle_literal_timestamp(void* h) { return static_cast<LiteralServer*>(h)->timestamp; }
+void oracle_literal_theta(void* h, float* out) {
+    auto* s = static_cast<LiteralServer*>(h);
+    std::copy(s->theta.begin(), s->theta.end(), out);
+}
+
+// One iteration of Algorithm 2: Get (update, j), then for every entry of the
+// update compute sigma_k (Eq. 3), alpha_k (Eq. 5), the new Theta_k (Eq. 4);
+// then the timestamp advances.  An entry whose value is +-0 is present but is
+// not a change: it is not recorded for later windows and leaves Theta_k as it
+// is; its sigma is still reported.  Returns 0; -1 if j > i, idx out of range
+// or idx not strictly ascending.
+int oracle_literal_apply(void* h, const uint32_t* idx, const float* val, uint64_t n_pairs,
+                         uint64_t j, float alpha, uint32_t* sigma_out) {
+    auto* s = static_cast<LiteralServer*>(h);
+    const uint64_t i = s->timestamp;
+    if (j > i) return -1;
+    for (uint64_t e = 0; e < n_pairs; ++e) {
+        if (idx[e] >= s->theta.size()) return -1;
+        if (e > 0 && idx[e] <= idx[e - 1]) return -1;
+    }
+    std::vector<uint32_t> changed;
+    for (uint64_t e = 0; e < n_pairs; ++e) {
+        const uint32_t k = idx[e];
+        uint32_t sigma_k = 0;
+        for (uint64_t u = j; u < i; ++u)
+            if (std::binary_search(s->nonzero_idx[u].begin(), s->nonzero_idx[u].end(), k)) ++sigma_k;
+        if (sigma_out) sigma_out[e] = sigma_k;
+        if (val[e] != 0.0f) {
+            s->theta[k] = updated_parameter(s->theta[k], alpha, sigma_k, val[e]);
+            changed.push_back(k);
+        }
+    }
+    s->nonzero_idx.push_back(std::move(changed));
+    s->timestamp = i + 1;
+    return 0;
+}
+
+// --- per-parameter form -----------------------------------------------------
+// "counting the number of updates applied on it since the last pull by the
+// worker" (text under Eq. 3): every parameter keeps the ascending list of
+// timestamps at which a non-zero update touched it; sigma_k is how many of
+// them are >= j.  Same function as the literal form, cost O(sigma_k) per
+// entry, usable on the full-size workloads.
+struct ListServer {
+    std::vector<float> theta;
+    uint64_t timestamp = 0;
+    std::vector<std::vector<uint64_t>> touched_at;  // touched_at[k]: ascending timestamps
+};
+
+void* oracle_server_create(uint64_t n_params, const float* theta0) {
+    auto* s = new ListServer;
+    s->theta.assign(theta0, theta0 + n_params);
+    s->touched_at.resize(n_params);
+    return s;
+}
+void oracle_server_destroy(void* h) { delete static_cast<ListServer*>(h); }
+uint64_t oracle_server_timestamp(void* h) { return static_cast<ListServer*>(h)->timestamp; }
+void oracle_server_theta(void* h, float* out) {
+    auto* s = static_cast<ListServer*>(h);
+    std::copy(s->theta.begin(), s->theta.end(), out);
+}
+
+int oracle_server_apply(void* h, const uint32_t* idx, const float* val, uint64_t n_pairs,
+                        uint64_t j, float alpha, uint32_t* sigma_out) {
+    auto* s = static_cast<ListServer*>(h);
+    const uint64_t i = s->timestamp;
+    if (j > i) return -1;
+    for (uint64_t e = 0; e < n_pairs; ++e) {
+        if (idx[e] >= s->theta.size()) return -1;
+        if (e > 0 && idx[e] <= idx[e - 1]) return -1;
+    }
+    for (uint64_t e = 0; e < n_pairs; ++e) {
+        const uint32_t k = idx[e];
+        const std::vector<uint64_t>& ts = s->touched_at[k];
+        uint32_t sigma_k = 0;
+        for (size_t t = ts.size(); t > 0 && ts[t - 1] >= j; --t) ++sigma_k;
+        if (sigma_out) sigma_out[e] = sigma_k;
+        if (val[e] != 0.0f) {
+            s->theta[k] = updated_parameter(s->theta[k], alpha, sigma_k, val[e]);
+            s->touched_at[k].push_back(i);
+        }
+    }
+    s->timestamp = i + 1;
+    return 0;
+}
+
+// --- one parameter at a time --------------------------------------------------
+// The history of a single parameter k through a whole sequence of updates,
+// computed the way the paper's complexity paragraph describes it: each update
+// keeps its sorted index list, and Eq. 3 is a membership search per update in
+// the window.  Lets a test check sampled parameters of a workload that is too
+// large to replay in full.  pair_begin[u] .. pair_begin[u+1] delimit update u
+// inside idx/val; pull_ts[u] is its j; update u is applied at timestamp
+// first_timestamp + u, and nothing touched k before first_timestamp.
+// Writes the sigma of each update that contains k to sigma_out (in order,
+// at most n_updates values), their number to *n_hits, the final value to
+// *theta_k.  Returns 0, or -1 if some j is out of range.
+int oracle_parameter_trace(uint32_t k, float theta0_k, const uint32_t* idx, const float* val,
+                           const uint64_t* pair_begin, const uint64_t* pull_ts, uint64_t n_updates,
+                           uint64_t first_timestamp, float alpha,
+                           uint32_t* sigma_out, uint64_t* n_hits, float* theta_k) {
+    float theta = theta0_k;
+    uint64_t hits = 0;
+    std::vector<char> changed_k(n_updates, 0);   // did update u change k with a non-zero value
+    for (uint64_t u = 0; u < n_updates; ++u) {
+        const uint64_t i = first_timestamp + u, j = pull_ts[u];
+        if (j > i) return -1;
+        const uint32_t* lo = idx + pair_begin[u];
+        const uint32_t* hi = idx + pair_begin[u + 1];
+        const uint32_t* at = std::lower_bound(lo, hi, k);
+        if (at == hi || *at != k) continue;
+        uint32_t sigma_k = 0;
+        for (uint64_t t = (j > first_timestamp ? j - first_timestamp : 0); t < u; ++t)
+            sigma_k += changed_k[t];
+        if (sigma_out) sigma_out[hits] = sigma_k;
+        ++hits;
+        const float v = val[at - idx];
+        if (v != 0.0f) {
+            theta = updated_parameter(theta, alpha, sigma_k, v);
+            changed_k[u] = 1;
+        }
+    }
+    *n_hits = hits;
+    *theta_k = theta;
+    return 0;
+}
+
+}  // extern "C"
