@@ -1,0 +1,394 @@
+#!/usr/bin/env python
+"""Benchmark of the AdaComp hot path on B200: SELECT_GRAD (select + compact) over resident dense
+gradients, then the parameter-server update of the selected pairs.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload 0..4] [--keep a/b] [--impl reference]
+
+One step = one pass of the whole hot path over one batch of synthetic input: for every keep
+fraction of the workload, select the gradients of all workers, then apply the resulting updates in
+a seeded arrival order.  Default workload: the 100 M-parameter one (25 tensors x 4 M, 16 workers,
+six keep fractions from 0.1 % to 10 %).  Prints ONE JSON line (rank 0).
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import tempfile
+import time
+
+import numpy as np
+import torch
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+from paper_1702_04683_b200 import workloads as wlmod  # noqa: E402
+
+METRIC = "dense-gradient GB/s scanned (select+compact, with the selected pairs applied)"
+UNIT = "GB/s"
+FALLBACK_HBM_GBS = 6650.0
+
+
+def parse_args():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=10)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="native", choices=["native", "reference"])
+    ap.add_argument("--workload", type=int, default=4)
+    ap.add_argument("--keep", default=None, help="one keep fraction a/b instead of the workload's list")
+    ap.add_argument("--workers", type=int, default=None, help="override the number of workers (smaller captures)")
+    ap.add_argument("--e2e-steps", type=int, default=2)
+    ap.add_argument("--apply-mode", type=int, default=0)
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-e2e", action="store_true")
+    return ap.parse_args()
+
+
+def hbm_peak():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    try:
+        with open(path) as f:
+            return float(json.load(f)["hbm_gbs"]), "measured"
+    except Exception:
+        return FALLBACK_HBM_GBS, "fallback"
+
+
+class ClockSampler:
+    """Samples SM clocks and throttle reasons with nvidia-smi while the timed region runs."""
+    QUERY = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,"
+             "clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+             "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, gpu_index: int):
+        self.gpu = gpu_index
+        self.proc = None
+        self.path = None
+
+    def start(self):
+        try:
+            fd, self.path = tempfile.mkstemp(suffix=".csv")
+            os.close(fd)
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", f"--query-gpu={self.QUERY}", "--format=csv,noheader,nounits", "-lms", "100",
+                 "-i", str(self.gpu)], stdout=open(self.path, "w"), stderr=subprocess.DEVNULL)
+        except Exception:
+            self.proc = None
+
+    def stop(self):
+        out = {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "samples": 0}
+        if self.proc is None:
+            return out
+        time.sleep(0.15)
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except Exception:
+            self.proc.kill()
+        sm, mx, reasons = [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        try:
+            for line in open(self.path):
+                f = [x.strip() for x in line.split(",")]
+                if len(f) < 9:
+                    continue
+                try:
+                    sm.append(float(f[1])); mx.append(float(f[2]))
+                except ValueError:
+                    continue
+                for name, v in zip(names, f[5:9]):
+                    if v.lower() == "active":
+                        reasons.add(name)
+            os.unlink(self.path)
+        except Exception:
+            pass
+        if sm:
+            out.update(sm_mhz=statistics.median(sm), sm_max_mhz=max(mx), samples=len(sm))
+        out["reasons"] = sorted(reasons)
+        return out
+
+
+def parse_keep(text):
+    a, b = text.split("/")
+    return int(a), int(b)
+
+
+def setup_dist(args):
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if world > 1:
+        import torch.distributed as dist
+        torch.cuda.set_device(local)
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+    return world, rank, local
+
+
+# ------------------------------------------------------------------------------------------ native arm
+
+class Point:
+    """One keep fraction of the workload: its selector, output buffers and pair count."""
+
+    def __init__(self, binding, wl, keep, dev):
+        self.keep = keep
+        self.segs = binding.make_segments(wl.tensor_sizes, keep)
+        self.sel = binding.Selector(self.segs, wl.n_workers, dev)
+        self.K = self.sel.pairs_per_worker
+        self.idx = torch.empty((wl.n_workers, self.K), dtype=torch.int32, device=dev)
+        self.val = torch.empty((wl.n_workers, self.K), dtype=torch.float32, device=dev)
+        self.count = np.full(wl.n_workers, self.K, dtype=np.uint32)
+
+
+def step_schedule(wl, rng, srv_ts, last_push_ts):
+    """Arrival order and pull timestamps of one round starting at server timestamp srv_ts."""
+    W = wl.n_workers
+    order = rng.permutation(W)
+    if wl.schedule == "rounds":
+        pull = np.where(last_push_ts[order] < 0, srv_ts, last_push_ts[order] + 1)
+        pull = np.maximum(pull, srv_ts - (2 * W - 1)).astype(np.uint64)
+    else:
+        pull = np.full(W, srv_ts, dtype=np.uint64)
+    last_push_ts[order] = srv_ts + np.arange(W)
+    return order, pull
+
+
+def run_native(args):
+    from paper_1702_04683_b200 import binding
+    world, rank, local = setup_dist(args)
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the hot path has no CPU fallback")
+    dev = torch.device("cuda", local)
+    torch.cuda.set_device(dev)
+    wl = wlmod.workload(args.workload, seed=rank)
+    if args.workers:
+        import dataclasses
+        wl = dataclasses.replace(wl, n_workers=args.workers)
+    keeps = [parse_keep(args.keep)] if args.keep else list(wl.keep_fractions)
+    W, P = wl.n_workers, wl.n_params
+    stream = torch.cuda.current_stream()
+
+    grads = wlmod.round_gradients(wl, 0, dev)                       # resident before the timer starts
+    points = [Point(binding, wl, k, dev) for k in keeps]
+    K_max = max(p.K for p in points)
+    theta = wlmod.initial_parameters(wl, dev)
+    srv = binding.Server(theta, history_pairs=2 * W * K_max, max_window_updates=2 * W)
+    srv.set_mode(args.apply_mode)
+    rng = np.random.default_rng(1234 + rank)
+    last_push = np.full(W, -1, dtype=np.int64)
+
+    def ev():
+        return torch.cuda.Event(enable_timing=True)
+
+    def one_step(record):
+        marks = []
+        for p in points:
+            order, pull = step_schedule(wl, rng, srv.timestamp, last_push)
+            e0 = ev(); e0.record(stream)
+            p.sel.select(grads, p.idx, p.val)
+            e1 = ev(); e1.record(stream)
+            srv.apply(p.idx.view(-1), p.val.view(-1), order.astype(np.uint64) * np.uint64(p.K), p.count, pull, wl.lr)
+            e2 = ev(); e2.record(stream)
+            marks.append((e0, e1, e2))
+        if record is not None:
+            record.append(marks)
+
+    def barrier():
+        if world > 1:
+            import torch.distributed as dist
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    for _ in range(args.warmup):
+        one_step(None)
+    barrier()
+    sampler = ClockSampler(local)
+    if rank == 0:
+        sampler.start()
+    launches0 = binding.adacomp_kernel_launches()
+    rec = []
+    t0, t1 = ev(), ev()
+    barrier()
+    t0.record(stream)
+    for _ in range(args.steps):
+        one_step(rec)
+    t1.record(stream)
+    barrier()
+    launches = binding.adacomp_kernel_launches() - launches0
+    clocks = sampler.stop() if rank == 0 else None
+    total_ms = t0.elapsed_time(t1)
+    if world > 1:
+        import torch.distributed as dist
+        t = torch.tensor([total_ms], device=dev, dtype=torch.float64)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        total_ms = float(t.item())
+    status = [p.sel.last_error()[0] for p in points] + [srv.last_error()]
+    if any(status):
+        raise SystemExit(f"device-side error recorded during the benchmark: {status}")
+
+    # per keep fraction: mean select / apply time over the timed steps
+    peak, peak_kind = hbm_peak()
+    pts = []
+    sel_ms_all, sel_bytes_all = 0.0, 0.0
+    for i, p in enumerate(points):
+        sel_ms = statistics.mean(m[i][0].elapsed_time(m[i][1]) for m in rec)
+        app_ms = statistics.mean(m[i][1].elapsed_time(m[i][2]) for m in rec)
+        scanned = W * 4.0 * P
+        sel_alg = W * (4.0 * P + 8.0 * p.K)
+        pairs = W * p.K
+        pts.append({
+            "keep": f"{p.keep[0]}/{p.keep[1]}", "pairs_per_update": p.K,
+            "select_ms": round(sel_ms, 4), "apply_ms": round(app_ms, 4),
+            "select_scanned_gbs": round(scanned / sel_ms / 1e6, 1),
+            "select_frac_of_hbm_peak": round(sel_alg / sel_ms / 1e6 / peak, 4),
+            "selected_elems_per_s": round(pairs / sel_ms * 1e3, 1),
+            "apply_pairs_per_s": round(pairs / app_ms * 1e3, 1),
+            "apply_updates_per_s": round(W / app_ms * 1e3, 1),
+            "apply_alg_gbs_28B_per_pair": round(pairs * 28.0 / app_ms / 1e6, 1),
+            "apply_alg_frac_of_hbm_peak": round(pairs * 28.0 / app_ms / 1e6 / peak, 4),
+        })
+        sel_ms_all += sel_ms
+        sel_bytes_all += sel_alg
+    ms_per_step = total_ms / args.steps
+    scanned_per_step = len(points) * W * 4.0 * P
+    value = world * scanned_per_step / ms_per_step / 1e6
+
+    out = {
+        "metric": METRIC, "value": round(value, 2), "unit": UNIT, "n_gpus": world, "steps": args.steps,
+        "warmup": args.warmup, "ms_per_step": round(ms_per_step, 4), "higher_is_better": True,
+        "scaling": "weak", "vs_baseline": None, "dtype": "u32 keys / f32 update arithmetic", "data": "synthetic",
+        "config": {"workload": wl.name, "tensors": len(wl.tensor_sizes), "params": P, "workers": W,
+                   "keep_fractions": [pt["keep"] for pt in pts], "step": "select + apply for every keep fraction",
+                   "l2": "inputs larger than L2 (%.1f GB of gradients per keep fraction)" % (W * 4.0 * P / 1e9),
+                   "apply_mode": args.apply_mode, "multi_gpu": "independent replicas, one per rank"},
+        "gpu_launches": int(launches),
+        "clocks": clocks,
+        "points": pts,
+        "roofline": {"bound": "hbm", "kernel": "adacomp_select (all kernels of one call)",
+                     "achieved": round(sel_bytes_all / sel_ms_all / 1e6, 1), "peak": peak, "peak_kind": "of " + peak_kind,
+                     "unit": "GB/s", "frac": round(sel_bytes_all / sel_ms_all / 1e6 / peak, 4), "traffic": None},
+    }
+    if world == 1 and not args.no_e2e:
+        out["e2e"] = run_e2e(args, binding, wl, points, srv, grads, rng, last_push, dev, stream)
+    if world == 1 and rank == 0 and not args.no_cpu_baseline:
+        out["cpu_baseline"] = cpu_baseline(wl, keeps, grads)
+    if rank == 0:
+        print(json.dumps(out))
+    if world > 1:
+        import torch.distributed as dist
+        dist.destroy_process_group()
+
+
+def run_e2e(args, binding, wl, points, srv, grads, rng, last_push, dev, stream):
+    """Same step through the host entry point: every step copies the gradients host -> device
+    from pinned memory and reads the selected pairs back."""
+    W, P = wl.n_workers, wl.n_params
+    try:
+        h_grads = torch.empty((W, P), dtype=torch.float32, pin_memory=True)
+    except RuntimeError as e:
+        return {"value": None, "unit": UNIT, "error": "cannot pin %.1f GB of host memory: %s" % (W * P * 4 / 1e9, e)}
+    h_grads.copy_(grads)
+    staging = torch.empty_like(grads)
+    K_max = max(p.K for p in points)
+    h_idx = torch.empty((W, K_max), dtype=torch.int32, pin_memory=True)
+    h_val = torch.empty((W, K_max), dtype=torch.float32, pin_memory=True)
+    h2d = d2h = 0
+
+    def step():
+        nonlocal h2d, d2h
+        for p in points:
+            order, pull = step_schedule(wl, rng, srv.timestamp, last_push)
+            hi, hv = h_idx.view(-1)[: W * p.K].view(W, p.K), h_val.view(-1)[: W * p.K].view(W, p.K)
+            p.sel.select_host(h_grads, staging, p.idx, p.val, hi, hv)
+            srv.apply(p.idx.view(-1), p.val.view(-1), order.astype(np.uint64) * np.uint64(p.K), p.count, pull, wl.lr)
+            h2d += W * P * 4
+            d2h += W * p.K * 8
+
+    step()
+    torch.cuda.synchronize()
+    h2d = d2h = 0
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record(stream)
+    for _ in range(args.e2e_steps):
+        step()
+    e1.record(stream)
+    torch.cuda.synchronize()
+    ms = e0.elapsed_time(e1) / args.e2e_steps
+    return {"value": round(len(points) * W * 4.0 * P / ms / 1e6, 2), "unit": UNIT, "ms_per_step": round(ms, 3),
+            "steps": args.e2e_steps, "h2d_bytes_per_step": h2d // args.e2e_steps,
+            "d2h_bytes_per_step": d2h // args.e2e_steps,
+            "what": "adacomp_select_host (pinned host gradients in, pairs out) + adacomp_apply"}
+
+
+# ------------------------------------------------------------------------------------------ CPU oracle arms
+
+def oracle_sample_pass(wl, keeps, grads_host, sample_workers):
+    """The oracle, as it stands, over `sample_workers` workers' gradients and every keep fraction:
+    select each, then apply the sampled updates.  Returns (seconds, bytes scanned)."""
+    import oracle
+    theta0 = wlmod.initial_parameters(wl, "cpu").numpy()
+    srv = oracle.Server(theta0)
+    t0 = time.perf_counter()
+    scanned = 0
+    for keep in keeps:
+        ks = [oracle.keep_count(n, *keep) for n in wl.tensor_sizes]
+        j = srv.timestamp
+        for w in range(sample_workers):
+            idx, val = oracle.select_layers(grads_host[w], wl.offsets, wl.tensor_sizes, ks)
+            srv.apply(idx, val, j, wl.lr)
+            scanned += grads_host[w].size * 4
+    return time.perf_counter() - t0, scanned
+
+
+def cpu_baseline(wl, keeps, grads_dev):
+    sample_workers = min(2, wl.n_workers)
+    g = grads_dev[:sample_workers].cpu().numpy()
+    secs, scanned = oracle_sample_pass(wl, keeps, g, sample_workers)
+    return {"value": round(scanned / secs / 1e9, 4), "unit": UNIT, "cores": 1, "kind": "oracle",
+            "seconds": round(secs, 2), "host_cores_available": os.cpu_count(),
+            "sample": "%d of %d workers, all %d keep fractions: oracle select (partial sort) + oracle apply, one thread"
+                      % (sample_workers, wl.n_workers, len(keeps))}
+
+
+def run_reference(args):
+    """The CPU oracle timed on the host, each step a bounded sample of the native arm's step."""
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    wl = wlmod.workload(args.workload)
+    keeps = [parse_keep(args.keep)] if args.keep else list(wl.keep_fractions)
+    sample_workers = 1
+    g = wlmod.round_gradients(wl, 0, "cpu", workers=range(sample_workers)).numpy()
+    for _ in range(min(args.warmup, 1)):
+        oracle_sample_pass(wl, keeps[:1], g, sample_workers)
+    steps = max(1, min(args.steps, 3))
+    secs = scanned = 0.0
+    for _ in range(steps):
+        s, b = oracle_sample_pass(wl, keeps, g, sample_workers)
+        secs += s
+        scanned += b
+    value = scanned / secs / 1e9
+    sample = "%d of %d workers per step, all %d keep fractions, %d steps" % (sample_workers, wl.n_workers, len(keeps), steps)
+    out = {
+        "impl": "reference", "metric": METRIC, "value": round(value, 4), "unit": UNIT, "n_gpus": args.gpus,
+        "steps": steps, "warmup": min(args.warmup, 1), "ms_per_step": round(secs / steps * 1e3, 2),
+        "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "u32 keys / f32 update arithmetic",
+        "data": "synthetic",
+        "config": {"workload": wl.name, "tensors": len(wl.tensor_sizes), "params": wl.n_params, "workers": wl.n_workers,
+                   "keep_fractions": ["%d/%d" % k for k in keeps], "step": "select + apply for every keep fraction"},
+        "cpu_baseline": {"value": round(value, 4), "unit": UNIT, "cores": 1, "kind": "oracle", "sample": sample},
+        "e2e": {"value": round(value, 4), "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+    }
+    print(json.dumps(out))
+
+
+if __name__ == "__main__":
+    a = parse_args()
+    if a.impl == "reference":
+        run_reference(a)
+    else:
+        run_native(a)

@@ -34,6 +34,12 @@
 #include <stddef.h>
 #include <stdint.h>
 
+#if defined(__GNUC__)
+#define ADACOMP_API __attribute__((visibility("default")))
+#else
+#define ADACOMP_API
+#endif
+
 #ifdef __cplusplus
 extern "C" {
 #endif
@@ -51,11 +57,13 @@ enum {
 };
 
 /* Static text for a status code ("ok", "invalid argument", ...). Never NULL. */
-const char* adacomp_status_string(int status);
+ADACOMP_API const char* adacomp_status_string(int status);
 /* Library version, major * 10000 + minor * 100 + patch. */
-int adacomp_version(void);
+ADACOMP_API int adacomp_version(void);
 /* The last cudaError_t (as int) a call of this library saw on the calling thread, 0 if none. */
-int adacomp_last_cuda_error(void);
+ADACOMP_API int adacomp_last_cuda_error(void);
+/* How many kernels this library has launched in this process so far (all handles, all threads). */
+ADACOMP_API uint64_t adacomp_kernel_launches(void);
 
 /* ------------------------------------------------------------------------------------------
  * Worker side: SELECT_GRAD (Algorithm 1; "Selection method" paragraph).
@@ -74,14 +82,14 @@ typedef struct {
  * k = min(n, max(1, ceil(n * c_num / c_den))) in exact integer arithmetic; n = 0 gives 0.
  * The paper does not state the rounding; the ceiling keeps every tensor represented.
  * ADACOMP_ERR_INVALID on c_den = 0, c_num > c_den, n >= 2^32 or k_out = NULL. */
-int adacomp_keep_count(uint64_t n, uint32_t c_num, uint32_t c_den, uint32_t* k_out);
+ADACOMP_API int adacomp_keep_count(uint64_t n, uint32_t c_num, uint32_t c_den, uint32_t* k_out);
 
 typedef struct adacomp_select adacomp_select_t;
 
 /* Bytes of device workspace adacomp_select_create needs for this layout and up to max_workers
  * gradient vectors per call.  ADACOMP_ERR_INVALID on a bad layout (k > n, overlap, unsorted,
  * total entries or pairs beyond 2^32 - 2, n_segs = 0, max_workers = 0). */
-int adacomp_select_workspace_bytes(const adacomp_segment_t* h_segs, uint32_t n_segs,
+ADACOMP_API int adacomp_select_workspace_bytes(const adacomp_segment_t* h_segs, uint32_t n_segs,
                                    uint32_t max_workers, size_t* bytes_out);
 
 /* Creates a selector for a fixed layout on CUDA device `device`.  The paper keeps no state on
@@ -89,7 +97,7 @@ int adacomp_select_workspace_bytes(const adacomp_segment_t* h_segs, uint32_t n_s
  * does the handle: it only holds the layout and scratch.  d_workspace: device memory,
  * 256-byte aligned, at least the size reported above.  Synchronous (copies the layout to the
  * device and clears scratch).  On error *h is NULL. */
-int adacomp_select_create(adacomp_select_t** h, const adacomp_segment_t* h_segs, uint32_t n_segs,
+ADACOMP_API int adacomp_select_create(adacomp_select_t** h, const adacomp_segment_t* h_segs, uint32_t n_segs,
                           uint32_t max_workers, void* d_workspace, size_t workspace_bytes, int device);
 
 /* SELECT_GRAD for n_workers gradient vectors at once.
@@ -105,7 +113,7 @@ int adacomp_select_create(adacomp_select_t** h, const adacomp_segment_t* h_segs,
  * +0 and -0 tie.  Entries not kept are dropped; no residual is accumulated.
  * Errors: ADACOMP_ERR_INVALID (null pointer, n_workers = 0 or > max_workers,
  * worker_stride_elems smaller than the layout's extent), ADACOMP_ERR_CUDA. */
-int adacomp_select(adacomp_select_t* h, const float* d_grads, uint64_t worker_stride_elems,
+ADACOMP_API int adacomp_select(adacomp_select_t* h, const float* d_grads, uint64_t worker_stride_elems,
                    uint32_t n_workers, uint32_t* d_idx_out, float* d_val_out, void* cuda_stream);
 
 /* Same operation for callers whose gradients live in host memory: copies h_grads to the
@@ -113,19 +121,19 @@ int adacomp_select(adacomp_select_t* h, const float* d_grads, uint64_t worker_st
  * pinned for the copies to be asynchronous; they must stay untouched until the stream has
  * drained.  d_grads_staging holds n_workers * worker_stride_elems floats; d_idx_staging and
  * d_val_staging hold n_workers * K entries each. */
-int adacomp_select_host(adacomp_select_t* h, const float* h_grads, uint64_t worker_stride_elems,
+ADACOMP_API int adacomp_select_host(adacomp_select_t* h, const float* h_grads, uint64_t worker_stride_elems,
                         uint32_t n_workers, float* d_grads_staging, uint32_t* d_idx_staging,
                         float* d_val_staging, uint32_t* h_idx_out, float* h_val_out,
                         void* cuda_stream);
 
 /* K = sum of k over the layout's segments (pairs per worker). */
-int adacomp_select_pairs_per_worker(const adacomp_select_t* h, uint64_t* pairs_out);
+ADACOMP_API int adacomp_select_pairs_per_worker(const adacomp_select_t* h, uint64_t* pairs_out);
 /* Waits for cuda_stream, then returns the first error the device recorded since the last call
  * of this function (ADACOMP_OK if none) and clears it.  Also reports, if stats_out is not
  * NULL, stats_out[0] = how many (worker, segment) selections of the last adacomp_select call
  * took the general multi-pass route rather than the bracketed single-pass route. */
-int adacomp_select_last_error(adacomp_select_t* h, void* cuda_stream, uint64_t* stats_out);
-int adacomp_select_destroy(adacomp_select_t* h);
+ADACOMP_API int adacomp_select_last_error(adacomp_select_t* h, void* cuda_stream, uint64_t* stats_out);
+ADACOMP_API int adacomp_select_destroy(adacomp_select_t* h);
 
 /* ------------------------------------------------------------------------------------------
  * Server side: Algorithm 2 (Eq. 3, Eq. 4, Eq. 5; "Complexity" paragraph for the history).
@@ -138,14 +146,14 @@ typedef struct adacomp_server adacomp_server_t;
  * the last d updates (d = worst delay, of the order of the number of workers); here the bound
  * is expressed in pairs: an update whose pull timestamp j is so old that update j's pairs have
  * been overwritten is refused with ADACOMP_ERR_WINDOW. */
-int adacomp_server_workspace_bytes(uint64_t n_params, uint64_t history_pairs, size_t* bytes_out);
+ADACOMP_API int adacomp_server_workspace_bytes(uint64_t n_params, uint64_t history_pairs, size_t* bytes_out);
 
 /* Creates the server state on `device`: timestamp, per-parameter history heads and the ring of
  * the last history_pairs pairs.  max_window_updates bounds i - j for any update (and how many
  * updates one adacomp_apply call may carry); it must be < 2^24 so that sigma converts to fp32
  * exactly.  n_params <= 2^32 - 2, history_pairs < 2^31.  Synchronous.  The server is unusable
  * until adacomp_server_reset has given it a parameter vector. */
-int adacomp_server_create(adacomp_server_t** s, uint64_t n_params, uint64_t history_pairs,
+ADACOMP_API int adacomp_server_create(adacomp_server_t** s, uint64_t n_params, uint64_t history_pairs,
                           uint32_t max_window_updates, void* d_workspace, size_t workspace_bytes,
                           int device);
 
@@ -153,18 +161,19 @@ int adacomp_server_create(adacomp_server_t** s, uint64_t n_params, uint64_t hist
  * the initial values) as the parameter vector that adacomp_apply updates in place, sets the
  * timestamp to 0 and forgets all history.  The buffer must outlive the server or the next
  * reset. */
-int adacomp_server_reset(adacomp_server_t* s, float* d_theta, void* cuda_stream);
+ADACOMP_API int adacomp_server_reset(adacomp_server_t* s, float* d_theta, void* cuda_stream);
 
 /* Pull_Theta (Algorithm 1): reports the current timestamp i in *h_timestamp_out and, if
  * d_theta_copy is not NULL, enqueues a copy of the n_params parameters into it. */
-int adacomp_server_pull(adacomp_server_t* s, float* d_theta_copy, uint64_t* h_timestamp_out,
+ADACOMP_API int adacomp_server_pull(adacomp_server_t* s, float* d_theta_copy, uint64_t* h_timestamp_out,
                         void* cuda_stream);
 
 /* Get + loop body of Algorithm 2 for n_updates arriving updates, strictly in array order
- * (= arrival order).  Update b consists of pairs [h_pair_begin[b], h_pair_begin[b+1]) of
- * d_idx / d_val and of the timestamp h_pull_ts[b] that its worker received with its pull
- * (Push(update, j)).  With i the server timestamp when update b is applied, for each of its
- * pairs (k, v):
+ * (= arrival order).  Update b consists of the h_pair_count[b] pairs that start at pair
+ * h_pair_begin[b] of d_idx / d_val (updates may sit anywhere in those arrays, e.g. worker by
+ * worker as adacomp_select wrote them, while arrival order is a permutation of the workers)
+ * and of the timestamp h_pull_ts[b] that its worker received with its pull (Push(update, j)).
+ * With i the server timestamp when update b is applied, for each of its pairs (k, v):
  *     sigma_k = number of updates u in [j, i-1] that changed Theta_k with a non-zero value (Eq. 3)
  *     alpha_k = lr / sigma_k if sigma_k != 0 else lr                                     (Eq. 5)
  *     Theta_k = Theta_k - alpha_k * v                                                    (Eq. 4)
@@ -176,40 +185,46 @@ int adacomp_server_pull(adacomp_server_t* s, float* d_theta_copy, uint64_t* h_ti
  * to one-at-a-time application.
  *   d_idx          indices into Theta, strictly ascending inside one update (what
  *                  adacomp_select emits); d_val the matching values.
- *   h_pair_begin   [n_updates + 1] host, non-decreasing, h_pair_begin[0] is the first pair.
- *   h_pull_ts      [n_updates] host.
+ *   h_pair_begin, h_pair_count, h_pull_ts   [n_updates] host arrays.
  *   d_sigma_out    NULL, or device array addressed like d_idx that receives sigma_k per pair.
  * Host-side checks happen before anything is enqueued and leave the server unchanged:
  * ADACOMP_ERR_WINDOW (j > i, i - j > max_window_updates, or update j's pairs already evicted
  * from the history ring), ADACOMP_ERR_CAPACITY (n_updates > max_window_updates, or one call's
- * pairs exceed history_pairs), ADACOMP_ERR_INVALID.  Index validity is checked on the device
- * only when validation is switched on (adacomp_server_set_validation) and is then reported by
- * adacomp_server_last_error as ADACOMP_ERR_UNSORTED; offending pairs are skipped. */
-int adacomp_apply(adacomp_server_t* s, const uint32_t* d_idx, const float* d_val,
-                  const uint64_t* h_pair_begin, const uint64_t* h_pull_ts, uint32_t n_updates,
-                  float lr, uint32_t* d_sigma_out, void* cuda_stream);
+ * pairs exceed history_pairs), ADACOMP_ERR_INVALID.  On the device an index >= n_params is
+ * skipped and reported by adacomp_server_last_error as ADACOMP_ERR_UNSORTED; with validation
+ * switched on (adacomp_server_set_validation) so is an index that is not larger than its
+ * predecessor in the same update. */
+ADACOMP_API int adacomp_apply(adacomp_server_t* s, const uint32_t* d_idx, const float* d_val,
+                              const uint64_t* h_pair_begin, const uint32_t* h_pair_count,
+                              const uint64_t* h_pull_ts, uint32_t n_updates, float lr,
+                              uint32_t* d_sigma_out, void* cuda_stream);
 
 /* Same operation for updates that arrive in host memory (the server's ingress): copies the
- * pairs [h_pair_begin[0], h_pair_begin[n_updates]) of h_idx / h_val into the caller's device
- * staging buffers (same addressing) and applies them.  h_sigma_out may be NULL; if not, it
- * receives sigma per pair through d_sigma_staging, which must then be given too. */
-int adacomp_apply_host(adacomp_server_t* s, const uint32_t* h_idx, const float* h_val,
-                       const uint64_t* h_pair_begin, const uint64_t* h_pull_ts, uint32_t n_updates,
-                       float lr, uint32_t* d_idx_staging, float* d_val_staging,
-                       uint32_t* d_sigma_staging, uint32_t* h_sigma_out, void* cuda_stream);
+ * range of pairs the updates span from h_idx / h_val into the caller's device staging buffers
+ * (same addressing) and applies them.  h_sigma_out may be NULL; if not, it receives sigma per
+ * pair through d_sigma_staging, which must then be given too. */
+ADACOMP_API int adacomp_apply_host(adacomp_server_t* s, const uint32_t* h_idx, const float* h_val,
+                                   const uint64_t* h_pair_begin, const uint32_t* h_pair_count,
+                                   const uint64_t* h_pull_ts, uint32_t n_updates, float lr,
+                                   uint32_t* d_idx_staging, float* d_val_staging,
+                                   uint32_t* d_sigma_staging, uint32_t* h_sigma_out, void* cuda_stream);
 
 /* Current timestamp i = number of updates applied since the last reset (host-side counter). */
-int adacomp_server_timestamp(const adacomp_server_t* s, uint64_t* h_timestamp_out);
+ADACOMP_API int adacomp_server_timestamp(const adacomp_server_t* s, uint64_t* h_timestamp_out);
 /* on != 0: every apply also checks on the device that indices are in range and strictly
  * ascending inside an update.  Off by default. */
-int adacomp_server_set_validation(adacomp_server_t* s, int on);
+ADACOMP_API int adacomp_server_set_validation(adacomp_server_t* s, int on);
 /* Chooses how adacomp_apply maps work to the GPU; results are identical.
  * 0 = automatic, 1 = one launch per update, 2 = one launch per call in which each warp owns a
  * contiguous range of parameters and walks the updates in order. */
-int adacomp_server_set_mode(adacomp_server_t* s, int mode);
+ADACOMP_API int adacomp_server_set_mode(adacomp_server_t* s, int mode);
+/* Test hook: advances the history position counter as if `count` more pairs had been applied
+ * (their history is empty).  Lets a test reach the 32-bit position re-basing that otherwise
+ * happens once per ~4 * 10^9 applied pairs.  Call right after adacomp_server_reset. */
+ADACOMP_API int adacomp_server_debug_skip_positions(adacomp_server_t* s, uint64_t count);
 /* Waits for cuda_stream, returns and clears the first error recorded on the device. */
-int adacomp_server_last_error(adacomp_server_t* s, void* cuda_stream);
-int adacomp_server_destroy(adacomp_server_t* s);
+ADACOMP_API int adacomp_server_last_error(adacomp_server_t* s, void* cuda_stream);
+ADACOMP_API int adacomp_server_destroy(adacomp_server_t* s);
 
 #ifdef __cplusplus
 }

@@ -1,0 +1,348 @@
+// Server side of libadacomp: Algorithm 2 (Eq. 3, 4, 5) with the update history kept as
+// per-parameter chains through a ring of the most recent pairs.
+//
+// History layout.  Every pair the server ever applies gets a position: pairs are numbered in
+// application order, so update u occupies positions [start(u), start(u) + pairs(u)).  The device
+// holds, relative to a host-side 64-bit base, 32-bit positions:
+//   head[k]           position of the latest pair that changed parameter k (kNone if none),
+//   prev[slot(pos)]   position of the pair that changed the same parameter before `pos`,
+// with slot(pos) = pos mod ring size (a power of two).  For an update that pulled at timestamp
+// j, sigma_k (Eq. 3) is the number of chain entries of k with position >= start(j): the chain is
+// walked from head[k] until it leaves the window, i.e. O(1 + sigma_k) instead of the one search
+// per remembered update of the paper's "Complexity" paragraph.  The host refuses updates whose
+// window start has been overwritten in the ring.
+#include <new>
+#include <vector>
+
+#include "common.cuh"
+
+using namespace adacomp;
+
+namespace {
+
+constexpr uint32_t kNone = 0xFFFFFFFFu;
+constexpr uint64_t kRebaseAt = 0xFFFFFFF0ull;     // positions stay below this
+constexpr int kApplyThreads = 256;
+
+struct ServerParams {
+    float* theta;
+    uint32_t* head;
+    uint32_t* prev;
+    int* status;
+    uint64_t n_params;
+    uint32_t ring_mask;
+    uint32_t ring_shift;     // (position base) mod ring size: slot = (pos32 + ring_shift) & ring_mask
+    uint32_t max_window;
+    int validate;
+};
+
+struct UpdateDesc {
+    uint64_t pair_begin;     // first pair in d_idx / d_val
+    uint32_t n_pairs;
+    uint32_t pos_start;      // 32-bit position of its first pair
+    uint32_t win_start;      // 32-bit position of the first pair of update j (window start)
+    uint32_t pad;
+};
+
+// One pair of one update: Eq. 3 (chain walk), Eq. 5, Eq. 4, then link the pair into the chain.
+__device__ __forceinline__ void apply_pair(const ServerParams& sp, uint32_t k, float v, uint32_t pos,
+                                           uint32_t win_start, float lr, uint32_t* sigma_slot) {
+    const uint32_t latest = sp.head[k];
+    uint32_t q = latest, sigma = 0;
+    while (q != kNone && q >= win_start) {
+        if (++sigma > sp.max_window) { record_error(sp.status, ADACOMP_ERR_WINDOW); break; }
+        q = sp.prev[(q + sp.ring_shift) & sp.ring_mask];
+    }
+    if (sigma_slot) *sigma_slot = sigma;
+    if (v != 0.0f) {                       // Eq. 3 counts changes: a zero entry is not one
+        const float alpha_k = sigma ? __fdiv_rn(lr, static_cast<float>(sigma)) : lr;   // Eq. 5
+        const float step = __fmul_rn(alpha_k, v);
+        sp.theta[k] = __fsub_rn(sp.theta[k], step);                                       // Eq. 4
+        sp.prev[(pos + sp.ring_shift) & sp.ring_mask] = latest;
+        sp.head[k] = pos;
+    }
+}
+
+// One update per launch, one thread per pair.  Indices inside an update are distinct, so threads
+// never touch the same parameter; the stream orders successive updates.
+__global__ void __launch_bounds__(kApplyThreads)
+k_apply_update(ServerParams sp, UpdateDesc u, const uint32_t* __restrict__ idx, const float* __restrict__ val,
+               float lr, uint32_t* sigma_out) {
+    const uint32_t e = blockIdx.x * kApplyThreads + threadIdx.x;
+    if (e >= u.n_pairs) return;
+    const uint64_t at = u.pair_begin + e;
+    const uint32_t k = idx[at];
+    if (k >= sp.n_params) { record_error(sp.status, ADACOMP_ERR_UNSORTED); return; }
+    if (sp.validate && e > 0 && idx[at - 1] >= k) { record_error(sp.status, ADACOMP_ERR_UNSORTED); return; }
+    apply_pair(sp, k, val[at], u.pos_start + e, u.win_start, lr, sigma_out ? sigma_out + at : nullptr);
+}
+
+// Moves every stored position down by `delta` (entries older than that become kNone).
+__global__ void k_rebase(uint32_t* a, uint64_t n, uint32_t delta) {
+    for (uint64_t i = blockIdx.x * static_cast<uint64_t>(blockDim.x) + threadIdx.x; i < n;
+         i += static_cast<uint64_t>(gridDim.x) * blockDim.x) {
+        const uint32_t q = a[i];
+        if (q != kNone) a[i] = (q >= delta) ? q - delta : kNone;
+    }
+}
+
+uint64_t pow2_at_least(uint64_t x) {
+    uint64_t p = 1;
+    while (p < x) p <<= 1;
+    return p;
+}
+
+}  // namespace
+
+struct adacomp_server {
+    int device = 0;
+    int n_sms = 0;
+    uint64_t n_params = 0;
+    uint64_t history_pairs = 0;   // as requested
+    uint64_t ring = 0;            // power of two >= history_pairs
+    uint32_t max_window = 0;
+    float* d_theta = nullptr;     // borrowed
+    uint32_t* d_head = nullptr;
+    uint32_t* d_prev = nullptr;
+    int* d_status = nullptr;
+    // host-side bookkeeping
+    uint64_t timestamp = 0;       // i
+    uint64_t pos_next = 0;        // absolute position of the next pair
+    uint64_t pos_base = 0;        // absolute position that 32-bit position 0 stands for
+    std::vector<uint64_t> start_of;   // start_of[u % size] = absolute start position of update u
+    int validate = 0;
+    int mode = 0;
+};
+
+namespace {
+
+size_t carve_server(adacomp_server_t* s, void* base, uint64_t n_params, uint64_t ring) {
+    Carver c(base);
+    s->d_head = c.take<uint32_t>(n_params);
+    s->d_prev = c.take<uint32_t>(ring);
+    s->d_status = c.take<int>(1);
+    return c.used;
+}
+
+bool sizes_ok(uint64_t n_params, uint64_t history_pairs) {
+    return n_params >= 1 && n_params <= 0xFFFFFFFEull && history_pairs >= 1 && history_pairs < (1ull << 31);
+}
+
+}  // namespace
+
+extern "C" {
+
+int adacomp_server_workspace_bytes(uint64_t n_params, uint64_t history_pairs, size_t* bytes_out) {
+    if (!bytes_out || !sizes_ok(n_params, history_pairs)) return ADACOMP_ERR_INVALID;
+    adacomp_server_t tmp;
+    *bytes_out = carve_server(&tmp, nullptr, n_params, pow2_at_least(history_pairs));
+    return ADACOMP_OK;
+}
+
+int adacomp_server_create(adacomp_server_t** out, uint64_t n_params, uint64_t history_pairs,
+                          uint32_t max_window_updates, void* d_workspace, size_t workspace_bytes,
+                          int device) {
+    if (!out) return ADACOMP_ERR_INVALID;
+    *out = nullptr;
+    if (!sizes_ok(n_params, history_pairs) || max_window_updates == 0 || max_window_updates >= (1u << 24))
+        return ADACOMP_ERR_INVALID;
+    if (!d_workspace || (reinterpret_cast<uintptr_t>(d_workspace) % kAlign) != 0) return ADACOMP_ERR_INVALID;
+    adacomp_server_t* s = new (std::nothrow) adacomp_server_t;
+    if (!s) return ADACOMP_ERR_ALLOC;
+    s->ring = pow2_at_least(history_pairs);
+    const size_t need = carve_server(s, d_workspace, n_params, s->ring);
+    if (need > workspace_bytes) { delete s; return ADACOMP_ERR_ALLOC; }
+    s->device = device;
+    s->n_params = n_params;
+    s->history_pairs = history_pairs;
+    s->max_window = max_window_updates;
+    try {
+        s->start_of.assign(static_cast<size_t>(max_window_updates) + 1, 0);
+    } catch (...) { delete s; return ADACOMP_ERR_ALLOC; }
+    DeviceGuard guard(device);
+    cudaError_t e = guard.err;
+    if (e == cudaSuccess) e = cudaDeviceGetAttribute(&s->n_sms, cudaDevAttrMultiProcessorCount, device);
+    if (e == cudaSuccess) e = cudaMemset(s->d_status, 0, sizeof(int));
+    if (e == cudaSuccess) e = cudaDeviceSynchronize();
+    if (e != cudaSuccess) { delete s; return cuda_fail(e); }
+    *out = s;
+    return ADACOMP_OK;
+}
+
+int adacomp_server_reset(adacomp_server_t* s, float* d_theta, void* cuda_stream) {
+    if (!s || !d_theta) return ADACOMP_ERR_INVALID;
+    DeviceGuard guard(s->device);
+    if (guard.err != cudaSuccess) return cuda_fail(guard.err);
+    cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+    ADACOMP_CUDA(cudaMemsetAsync(s->d_head, 0xFF, s->n_params * sizeof(uint32_t), st));
+    ADACOMP_CUDA(cudaMemsetAsync(s->d_status, 0, sizeof(int), st));
+    s->d_theta = d_theta;
+    s->timestamp = 0;
+    s->pos_next = 0;
+    s->pos_base = 0;
+    std::fill(s->start_of.begin(), s->start_of.end(), 0);
+    return ADACOMP_OK;
+}
+
+int adacomp_server_pull(adacomp_server_t* s, float* d_theta_copy, uint64_t* h_timestamp_out,
+                        void* cuda_stream) {
+    if (!s || !h_timestamp_out || !s->d_theta) return ADACOMP_ERR_INVALID;
+    *h_timestamp_out = s->timestamp;
+    if (d_theta_copy) {
+        DeviceGuard guard(s->device);
+        if (guard.err != cudaSuccess) return cuda_fail(guard.err);
+        ADACOMP_CUDA(cudaMemcpyAsync(d_theta_copy, s->d_theta, s->n_params * sizeof(float),
+                                     cudaMemcpyDeviceToDevice, static_cast<cudaStream_t>(cuda_stream)));
+    }
+    return ADACOMP_OK;
+}
+
+int adacomp_apply(adacomp_server_t* s, const uint32_t* d_idx, const float* d_val,
+                  const uint64_t* h_pair_begin, const uint32_t* h_pair_count, const uint64_t* h_pull_ts,
+                  uint32_t n_updates, float lr, uint32_t* d_sigma_out, void* cuda_stream) {
+    if (!s || !s->d_theta) return ADACOMP_ERR_INVALID;
+    if (n_updates == 0) return ADACOMP_OK;
+    if (!h_pair_begin || !h_pair_count || !h_pull_ts) return ADACOMP_ERR_INVALID;
+    if (n_updates > s->max_window) return ADACOMP_ERR_CAPACITY;
+    uint64_t call_pairs = 0;
+    for (uint32_t b = 0; b < n_updates; ++b) call_pairs += h_pair_count[b];
+    if (call_pairs > s->history_pairs) return ADACOMP_ERR_CAPACITY;
+    if (call_pairs && (!d_idx || !d_val)) return ADACOMP_ERR_INVALID;
+
+    // ---- host-side window checks; nothing is enqueued and nothing changes until all pass
+    const uint64_t i0 = s->timestamp;
+    const size_t cap = s->start_of.size();
+    std::vector<uint64_t> start_abs(n_updates + 1), win_abs(n_updates);
+    start_abs[0] = s->pos_next;
+    for (uint32_t b = 0; b < n_updates; ++b) start_abs[b + 1] = start_abs[b] + h_pair_count[b];
+    for (uint32_t b = 0; b < n_updates; ++b) {
+        const uint64_t i = i0 + b, j = h_pull_ts[b];
+        if (j > i || i - j > s->max_window) return ADACOMP_ERR_WINDOW;
+        const uint64_t ws = (j >= i0) ? start_abs[j - i0] : s->start_of[j % cap];
+        if (start_abs[b + 1] - ws > s->ring) return ADACOMP_ERR_WINDOW;   // update j's pairs would be overwritten
+        win_abs[b] = ws;
+    }
+
+    DeviceGuard guard(s->device);
+    if (guard.err != cudaSuccess) return cuda_fail(guard.err);
+    cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+
+    // ---- keep 32-bit positions in range
+    if (s->pos_next + call_pairs - s->pos_base >= kRebaseAt) {
+        uint64_t oldest = s->pos_next > s->ring ? s->pos_next - s->ring : 0;   // oldest position still in the ring
+        if (oldest < s->pos_base) oldest = s->pos_base;
+        const uint64_t delta = oldest - s->pos_base;
+        if (delta == 0 || s->pos_next + call_pairs - oldest >= kRebaseAt) return ADACOMP_ERR_CAPACITY;
+        const unsigned grid = static_cast<unsigned>(s->n_sms * 8);
+        k_rebase<<<grid, 256, 0, st>>>(s->d_head, s->n_params, static_cast<uint32_t>(delta));
+        ADACOMP_LAUNCH_CHECK();
+        k_rebase<<<grid, 256, 0, st>>>(s->d_prev, s->ring, static_cast<uint32_t>(delta));
+        ADACOMP_LAUNCH_CHECK();
+        s->pos_base = oldest;
+    }
+
+    ServerParams sp;
+    sp.theta = s->d_theta;
+    sp.head = s->d_head;
+    sp.prev = s->d_prev;
+    sp.status = s->d_status;
+    sp.n_params = s->n_params;
+    sp.ring_mask = static_cast<uint32_t>(s->ring - 1);
+    sp.ring_shift = static_cast<uint32_t>(s->pos_base & (s->ring - 1));
+    sp.max_window = s->max_window;
+    sp.validate = s->validate;
+
+    for (uint32_t b = 0; b < n_updates; ++b) {
+        UpdateDesc u;
+        u.pair_begin = h_pair_begin[b];
+        u.n_pairs = h_pair_count[b];
+        u.pos_start = static_cast<uint32_t>(start_abs[b] - s->pos_base);
+        u.win_start = static_cast<uint32_t>(win_abs[b] - s->pos_base);
+        u.pad = 0;
+        if (u.n_pairs) {
+            const unsigned grid = (u.n_pairs + kApplyThreads - 1) / kApplyThreads;
+            k_apply_update<<<grid, kApplyThreads, 0, st>>>(sp, u, d_idx, d_val, lr, d_sigma_out);
+            ADACOMP_LAUNCH_CHECK();
+        }
+        s->start_of[(i0 + b) % cap] = start_abs[b];
+        s->pos_next = start_abs[b + 1];
+        s->timestamp = i0 + b + 1;        // the timestamp advances once per update (Algorithm 2)
+    }
+    return ADACOMP_OK;
+}
+
+int adacomp_apply_host(adacomp_server_t* s, const uint32_t* h_idx, const float* h_val,
+                       const uint64_t* h_pair_begin, const uint32_t* h_pair_count, const uint64_t* h_pull_ts,
+                       uint32_t n_updates, float lr, uint32_t* d_idx_staging, float* d_val_staging,
+                       uint32_t* d_sigma_staging, uint32_t* h_sigma_out, void* cuda_stream) {
+    if (!s) return ADACOMP_ERR_INVALID;
+    if (n_updates == 0) return ADACOMP_OK;
+    if (!h_pair_begin || !h_pair_count) return ADACOMP_ERR_INVALID;
+    // one copy over the range of pairs the updates span
+    uint64_t first = ~0ull, last = 0;
+    for (uint32_t b = 0; b < n_updates; ++b) {
+        if (!h_pair_count[b]) continue;
+        first = h_pair_begin[b] < first ? h_pair_begin[b] : first;
+        const uint64_t end = h_pair_begin[b] + h_pair_count[b];
+        last = end > last ? end : last;
+    }
+    const uint64_t pairs = last > first ? last - first : 0;
+    if (pairs && (!h_idx || !h_val || !d_idx_staging || !d_val_staging)) return ADACOMP_ERR_INVALID;
+    if (h_sigma_out && !d_sigma_staging) return ADACOMP_ERR_INVALID;
+    DeviceGuard guard(s->device);
+    if (guard.err != cudaSuccess) return cuda_fail(guard.err);
+    cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+    if (pairs) {
+        ADACOMP_CUDA(cudaMemcpyAsync(d_idx_staging + first, h_idx + first, pairs * sizeof(uint32_t), cudaMemcpyHostToDevice, st));
+        ADACOMP_CUDA(cudaMemcpyAsync(d_val_staging + first, h_val + first, pairs * sizeof(float), cudaMemcpyHostToDevice, st));
+    }
+    int rc = adacomp_apply(s, d_idx_staging, d_val_staging, h_pair_begin, h_pair_count, h_pull_ts, n_updates, lr,
+                           h_sigma_out ? d_sigma_staging : nullptr, cuda_stream);
+    if (rc != ADACOMP_OK) return rc;
+    if (h_sigma_out && pairs)
+        ADACOMP_CUDA(cudaMemcpyAsync(h_sigma_out + first, d_sigma_staging + first, pairs * sizeof(uint32_t), cudaMemcpyDeviceToHost, st));
+    return ADACOMP_OK;
+}
+
+int adacomp_server_timestamp(const adacomp_server_t* s, uint64_t* h_timestamp_out) {
+    if (!s || !h_timestamp_out) return ADACOMP_ERR_INVALID;
+    *h_timestamp_out = s->timestamp;
+    return ADACOMP_OK;
+}
+
+int adacomp_server_set_validation(adacomp_server_t* s, int on) {
+    if (!s) return ADACOMP_ERR_INVALID;
+    s->validate = on ? 1 : 0;
+    return ADACOMP_OK;
+}
+
+int adacomp_server_set_mode(adacomp_server_t* s, int mode) {
+    if (!s || mode < 0 || mode > 2) return ADACOMP_ERR_INVALID;
+    s->mode = mode;
+    return ADACOMP_OK;
+}
+
+int adacomp_server_debug_skip_positions(adacomp_server_t* s, uint64_t count) {
+    if (!s) return ADACOMP_ERR_INVALID;
+    s->pos_next += count;
+    return ADACOMP_OK;
+}
+
+int adacomp_server_last_error(adacomp_server_t* s, void* cuda_stream) {
+    if (!s) return ADACOMP_ERR_INVALID;
+    DeviceGuard guard(s->device);
+    if (guard.err != cudaSuccess) return cuda_fail(guard.err);
+    cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+    int status = 0;
+    ADACOMP_CUDA(cudaMemcpyAsync(&status, s->d_status, sizeof status, cudaMemcpyDeviceToHost, st));
+    ADACOMP_CUDA(cudaMemsetAsync(s->d_status, 0, sizeof(int), st));
+    ADACOMP_CUDA(cudaStreamSynchronize(st));
+    return status;
+}
+
+int adacomp_server_destroy(adacomp_server_t* s) {
+    delete s;
+    return ADACOMP_OK;
+}
+
+}  // extern "C"

@@ -1,0 +1,226 @@
+// Worker side of libadacomp: handle, workspace layout and launch sequence of SELECT_GRAD
+// (Algorithm 1).
+#include <new>
+#include <vector>
+
+#include "select_general.cuh"
+
+using namespace adacomp;
+
+struct adacomp_select {
+    int device = 0;
+    int n_sms = 0;
+    uint32_t n_layers = 0, max_workers = 0, slots_per_worker = 0;
+    uint64_t extent = 0;   // one past the last entry any segment covers
+    uint64_t K = 0;        // pairs per worker
+    // device (inside the caller's workspace)
+    Layer* d_layers = nullptr;
+    Inst* d_inst = nullptr;
+    uint32_t* d_hist = nullptr;
+    uint32_t* d_list = nullptr;
+    uint32_t* d_list_slot_start = nullptr;
+    uint32_t* d_list_len = nullptr;
+    uint2* d_chunk_cnt = nullptr;
+    int* d_status = nullptr;
+    uint32_t* d_stats = nullptr;
+};
+
+namespace {
+
+struct Layout {
+    std::vector<Layer> layers;
+    uint64_t extent = 0, K = 0;
+    uint32_t slots_per_worker = 0;
+};
+
+int build_layout(const adacomp_segment_t* segs, uint32_t n_segs, uint32_t max_workers, Layout* out) {
+    if (!segs || n_segs == 0 || max_workers == 0) return ADACOMP_ERR_INVALID;
+    constexpr uint64_t kMaxIndex = 0xFFFFFFFEull;
+    uint64_t end_prev = 0, K = 0, slots = 0;
+    out->layers.resize(n_segs);
+    for (uint32_t l = 0; l < n_segs; ++l) {
+        const adacomp_segment_t& s = segs[l];
+        if (s.k > s.n) return ADACOMP_ERR_INVALID;
+        if (s.offset < end_prev) return ADACOMP_ERR_INVALID;             // overlap or not ascending
+        if (s.offset + s.n > kMaxIndex) return ADACOMP_ERR_INVALID;      // indices are uint32
+        Layer& L = out->layers[l];
+        L.offset = s.offset;
+        L.out_offset = K;
+        L.n = s.n;
+        L.k = s.k;
+        L.n_slots = static_cast<uint32_t>((static_cast<uint64_t>(s.n) + 3 + kChunkElems - 1) / kChunkElems);
+        if (L.n_slots == 0) L.n_slots = 1;
+        L.slot_base = static_cast<uint32_t>(slots);
+        slots += L.n_slots;
+        K += s.k;
+        end_prev = s.offset + s.n;
+    }
+    if (K > kMaxIndex || slots * max_workers > 0x7FFFFFFFull ||
+        static_cast<uint64_t>(n_segs) * max_workers > 0x7FFFFFFFull)
+        return ADACOMP_ERR_INVALID;
+    out->extent = end_prev;
+    out->K = K;
+    out->slots_per_worker = static_cast<uint32_t>(slots);
+    return ADACOMP_OK;
+}
+
+// One place that decides the workspace layout; with a null base it only measures.
+size_t carve(adacomp_select_t* h, void* base, const Layout& lay, uint32_t max_workers) {
+    Carver c(base);
+    const size_t n_inst = static_cast<size_t>(lay.layers.size()) * max_workers;
+    h->d_layers = c.take<Layer>(lay.layers.size());
+    h->d_inst = c.take<Inst>(n_inst);
+    h->d_hist = c.take<uint32_t>(n_inst * kBins);
+    h->d_list = c.take<uint32_t>(n_inst);
+    h->d_list_slot_start = c.take<uint32_t>(n_inst);
+    h->d_list_len = c.take<uint32_t>(2);
+    h->d_chunk_cnt = c.take<uint2>(static_cast<size_t>(lay.slots_per_worker) * max_workers);
+    h->d_status = c.take<int>(1);
+    h->d_stats = c.take<uint32_t>(4);
+    return c.used;
+}
+
+}  // namespace
+
+extern "C" {
+
+int adacomp_select_workspace_bytes(const adacomp_segment_t* h_segs, uint32_t n_segs,
+                                   uint32_t max_workers, size_t* bytes_out) {
+    if (!bytes_out) return ADACOMP_ERR_INVALID;
+    Layout lay;
+    int rc = build_layout(h_segs, n_segs, max_workers, &lay);
+    if (rc != ADACOMP_OK) return rc;
+    adacomp_select_t tmp;
+    *bytes_out = carve(&tmp, nullptr, lay, max_workers);
+    return ADACOMP_OK;
+}
+
+int adacomp_select_create(adacomp_select_t** h, const adacomp_segment_t* h_segs, uint32_t n_segs,
+                          uint32_t max_workers, void* d_workspace, size_t workspace_bytes, int device) {
+    if (!h) return ADACOMP_ERR_INVALID;
+    *h = nullptr;
+    if (!d_workspace || (reinterpret_cast<uintptr_t>(d_workspace) % kAlign) != 0) return ADACOMP_ERR_INVALID;
+    Layout lay;
+    int rc = build_layout(h_segs, n_segs, max_workers, &lay);
+    if (rc != ADACOMP_OK) return rc;
+    adacomp_select_t* s = new (std::nothrow) adacomp_select_t;
+    if (!s) return ADACOMP_ERR_ALLOC;
+    const size_t need = carve(s, d_workspace, lay, max_workers);
+    if (need > workspace_bytes) { delete s; return ADACOMP_ERR_ALLOC; }
+    s->device = device;
+    s->n_layers = n_segs;
+    s->max_workers = max_workers;
+    s->slots_per_worker = lay.slots_per_worker;
+    s->extent = lay.extent;
+    s->K = lay.K;
+    DeviceGuard guard(device);
+    cudaError_t e = guard.err;
+    if (e == cudaSuccess) e = cudaDeviceGetAttribute(&s->n_sms, cudaDevAttrMultiProcessorCount, device);
+    if (e == cudaSuccess) e = cudaMemset(d_workspace, 0, need);
+    if (e == cudaSuccess)
+        e = cudaMemcpy(s->d_layers, lay.layers.data(), lay.layers.size() * sizeof(Layer), cudaMemcpyHostToDevice);
+    if (e == cudaSuccess) e = cudaDeviceSynchronize();
+    if (e != cudaSuccess) { delete s; return cuda_fail(e); }
+    *h = s;
+    return ADACOMP_OK;
+}
+
+int adacomp_select(adacomp_select_t* h, const float* d_grads, uint64_t worker_stride_elems,
+                   uint32_t n_workers, uint32_t* d_idx_out, float* d_val_out, void* cuda_stream) {
+    if (!h || !d_grads || n_workers == 0 || n_workers > h->max_workers) return ADACOMP_ERR_INVALID;
+    if (h->K > 0 && (!d_idx_out || !d_val_out)) return ADACOMP_ERR_INVALID;
+    if (n_workers > 1 && worker_stride_elems < h->extent) return ADACOMP_ERR_INVALID;
+    if (reinterpret_cast<uintptr_t>(d_grads) % 4 != 0) return ADACOMP_ERR_INVALID;
+    DeviceGuard guard(h->device);
+    if (guard.err != cudaSuccess) return cuda_fail(guard.err);
+    cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+
+    SelectParams p;
+    p.grads = d_grads;
+    p.stride = worker_stride_elems;
+    p.n_workers = n_workers;
+    p.n_layers = h->n_layers;
+    p.layers = h->d_layers;
+    p.inst = h->d_inst;
+    p.hist = h->d_hist;
+    p.list = h->d_list;
+    p.list_slot_start = h->d_list_slot_start;
+    p.list_len = h->d_list_len;
+    p.chunk_cnt = h->d_chunk_cnt;
+    p.slots_per_worker = h->slots_per_worker;
+    p.idx_out = d_idx_out;
+    p.val_out = d_val_out;
+    p.K = h->K;
+    p.status = h->d_status;
+
+    const uint64_t total_slots = static_cast<uint64_t>(h->slots_per_worker) * n_workers;
+    uint64_t grid64 = static_cast<uint64_t>(h->n_sms) * 8;
+    if (grid64 > total_slots) grid64 = total_slots;
+    if (grid64 == 0) grid64 = 1;
+    const unsigned grid = static_cast<unsigned>(grid64);
+
+    k_general_plan<<<1, kThreads, 0, st>>>(p, 1);
+    ADACOMP_LAUNCH_CHECK();
+    k_general_hist<0><<<grid, kThreads, 0, st>>>(p);
+    ADACOMP_LAUNCH_CHECK();
+    k_general_hist<1><<<grid, kThreads, 0, st>>>(p);
+    ADACOMP_LAUNCH_CHECK();
+    k_general_hist<2><<<grid, kThreads, 0, st>>>(p);
+    ADACOMP_LAUNCH_CHECK();
+    k_general_count<<<grid, kThreads, 0, st>>>(p);
+    ADACOMP_LAUNCH_CHECK();
+    k_general_write<<<grid, kThreads, 0, st>>>(p);
+    ADACOMP_LAUNCH_CHECK();
+    return ADACOMP_OK;
+}
+
+int adacomp_select_host(adacomp_select_t* h, const float* h_grads, uint64_t worker_stride_elems,
+                        uint32_t n_workers, float* d_grads_staging, uint32_t* d_idx_staging,
+                        float* d_val_staging, uint32_t* h_idx_out, float* h_val_out,
+                        void* cuda_stream) {
+    if (!h || !h_grads || !d_grads_staging || n_workers == 0 || n_workers > h->max_workers)
+        return ADACOMP_ERR_INVALID;
+    if (h->K > 0 && (!d_idx_staging || !d_val_staging || !h_idx_out || !h_val_out)) return ADACOMP_ERR_INVALID;
+    if (n_workers > 1 && worker_stride_elems < h->extent) return ADACOMP_ERR_INVALID;
+    DeviceGuard guard(h->device);
+    if (guard.err != cudaSuccess) return cuda_fail(guard.err);
+    cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+    const uint64_t elems = (n_workers - 1) * worker_stride_elems + h->extent;
+    ADACOMP_CUDA(cudaMemcpyAsync(d_grads_staging, h_grads, elems * sizeof(float), cudaMemcpyHostToDevice, st));
+    int rc = adacomp_select(h, d_grads_staging, worker_stride_elems, n_workers, d_idx_staging, d_val_staging, cuda_stream);
+    if (rc != ADACOMP_OK) return rc;
+    const uint64_t pairs = h->K * n_workers;
+    if (pairs) {
+        ADACOMP_CUDA(cudaMemcpyAsync(h_idx_out, d_idx_staging, pairs * sizeof(uint32_t), cudaMemcpyDeviceToHost, st));
+        ADACOMP_CUDA(cudaMemcpyAsync(h_val_out, d_val_staging, pairs * sizeof(float), cudaMemcpyDeviceToHost, st));
+    }
+    return ADACOMP_OK;
+}
+
+int adacomp_select_pairs_per_worker(const adacomp_select_t* h, uint64_t* pairs_out) {
+    if (!h || !pairs_out) return ADACOMP_ERR_INVALID;
+    *pairs_out = h->K;
+    return ADACOMP_OK;
+}
+
+int adacomp_select_last_error(adacomp_select_t* h, void* cuda_stream, uint64_t* stats_out) {
+    if (!h) return ADACOMP_ERR_INVALID;
+    DeviceGuard guard(h->device);
+    if (guard.err != cudaSuccess) return cuda_fail(guard.err);
+    cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+    int status = 0;
+    uint32_t len[2] = {0, 0};
+    ADACOMP_CUDA(cudaMemcpyAsync(&status, h->d_status, sizeof status, cudaMemcpyDeviceToHost, st));
+    ADACOMP_CUDA(cudaMemcpyAsync(len, h->d_list_len, sizeof len, cudaMemcpyDeviceToHost, st));
+    ADACOMP_CUDA(cudaMemsetAsync(h->d_status, 0, sizeof(int), st));
+    ADACOMP_CUDA(cudaStreamSynchronize(st));
+    if (stats_out) stats_out[0] = len[0];
+    return status;
+}
+
+int adacomp_select_destroy(adacomp_select_t* h) {
+    delete h;
+    return ADACOMP_OK;
+}
+
+}  // extern "C"

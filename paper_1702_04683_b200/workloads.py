@@ -222,3 +222,37 @@ def describe(wl: Workload) -> dict:
             "workers": wl.n_workers, "rounds": wl.n_rounds,
             "keep_fractions": [f"{a}/{b}" for a, b in wl.keep_fractions],
             "distribution": wl.distribution, "schedule": wl.schedule, "seed": wl.seed}
+
+
+# --------------------------------------------------------------------------- ready-made updates
+
+def synthetic_updates(wl: Workload, keep_counts: Sequence[int], rnd: int, device="cpu",
+                      zero_fraction: float = 0.0) -> Tuple[torch.Tensor, torch.Tensor]:
+    """Updates for exercising the server alone: for every worker and tensor, ``keep_counts[l]``
+    distinct ascending indices (one drawn uniformly from each of k equal strata of the tensor)
+    with N(0, scale_l) values.  Returns (idx [W, K] int32 holding uint32 bit patterns,
+    val [W, K] fp32).  Two workers name the same parameter with probability about k/n, as
+    independent uniform choices would."""
+    W, K = wl.n_workers, int(sum(keep_counts))
+    idx = torch.empty((W, K), dtype=torch.int64, device=device)
+    val = torch.empty((W, K), dtype=torch.float32, device=device)
+    gen = torch.Generator(device=device)
+    gen.manual_seed(((wl.seed * 1_000_003 + wl.index) * 10_007 + rnd) * 100_003 + 77_777)
+    at = 0
+    for off, n, k, s in zip(wl.offsets, wl.tensor_sizes, keep_counts, wl.scales):
+        if k == 0:
+            continue
+        t = torch.arange(k, dtype=torch.int64, device=device)
+        lo = (t * n) // k
+        width = ((t + 1) * n) // k - lo
+        u = torch.rand((W, k), dtype=torch.float64, device=device, generator=gen)
+        pick = torch.minimum((u * width).to(torch.int64), width - 1)
+        idx[:, at:at + k] = off + lo + pick
+        val[:, at:at + k].normal_(0.0, 1.0, generator=gen).mul_(s)
+        at += k
+    if zero_fraction > 0:
+        mask = torch.rand((W, K), device=device, generator=gen) < zero_fraction
+        val[mask] = 0.0
+    idx32 = (idx & 0xFFFFFFFF).to(torch.int64)
+    idx32 = torch.where(idx32 >= 2**31, idx32 - 2**32, idx32).to(torch.int32)
+    return idx32, val

@@ -1,0 +1,285 @@
+"""Parity of adacomp_apply and of the whole select -> apply path (CUDA, through the C ABI)
+with the CPU oracle: indices, values, staleness counters and parameters bit for bit."""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+from paper_1702_04683_b200 import workloads as wlmod
+
+from helpers import assert_same_pipeline, bits, gpu_pipeline, oracle_keep_counts, oracle_pipeline, u32
+
+pytestmark = pytest.mark.gpu
+DEV = torch.device("cuda", 0)
+MODES = [1, 2]
+
+
+@pytest.fixture(scope="module")
+def binding():
+    from paper_1702_04683_b200 import binding as b
+    return b
+
+
+def i32(a):
+    """uint32 numpy -> int32 torch tensor with the same bits, on the GPU."""
+    return torch.from_numpy(np.ascontiguousarray(a, dtype=np.uint32).view(np.int32)).to(DEV)
+
+
+# ----------------------------------------------------------------------------- whole path
+
+@pytest.mark.parametrize("mode", MODES)
+def test_small_cnn_full_size_pipeline(mode):
+    wl = wlmod.workload(0)
+    assert_same_pipeline(gpu_pipeline(wl, (1, 100), mode), oracle_pipeline(wl, (1, 100), DEV))
+
+
+@pytest.mark.parametrize("mode", MODES)
+def test_small_cnn_uniform_staleness_pipeline(mode):
+    wl = wlmod.small_cnn_uniform_staleness()
+    assert_same_pipeline(gpu_pipeline(wl, (1, 100), mode), oracle_pipeline(wl, (1, 100), DEV))
+
+
+@pytest.mark.parametrize("mode", MODES)
+def test_many_workers_scaled_pipeline(mode):
+    wl = wlmod.workload(1).scaled(64)                  # 200 workers x 10 rounds, 51 k parameters
+    got, want = gpu_pipeline(wl, (1, 100), mode), oracle_pipeline(wl, (1, 100), DEV)
+    assert_same_pipeline(got, want)
+    assert max(int(s.max()) for s in want["sigma"]) >= 3      # the interleaving does produce staleness
+
+
+@pytest.mark.parametrize("mode", MODES)
+@pytest.mark.parametrize("keep", [(1, 1000), (1, 10)])
+def test_tie_stress_scaled_pipeline(mode, keep):
+    wl = wlmod.workload(2).scaled(8, n_workers=16)
+    assert_same_pipeline(gpu_pipeline(wl, keep, mode), oracle_pipeline(wl, keep, DEV))
+
+
+@pytest.mark.parametrize("mode", MODES)
+def test_resnet_scaled_pipeline(mode):
+    wl = wlmod.workload(3).scaled(8, n_workers=8, n_rounds=3)
+    assert_same_pipeline(gpu_pipeline(wl, (5, 1000), mode), oracle_pipeline(wl, (5, 1000), DEV))
+
+
+@pytest.mark.parametrize("mode", MODES)
+def test_literal_form_agrees_on_a_small_case(mode):
+    wl = wlmod.workload(1).scaled(512, n_workers=12, n_rounds=4)
+    assert_same_pipeline(gpu_pipeline(wl, (1, 20), mode), oracle_pipeline(wl, (1, 20), DEV, literal=True))
+
+
+# ----------------------------------------------------------------------------- server alone, full sizes
+
+def run_server_both(binding, wl, ks, mode, zero_fraction=0.0, rounds=None, sample_only=False):
+    K = int(sum(ks))
+    theta = wlmod.initial_parameters(wl, DEV)
+    theta0 = theta.cpu().numpy()
+    srv = binding.Server(theta, history_pairs=2 * wl.n_workers * K, max_window_updates=2 * wl.n_workers)
+    srv.set_mode(mode)
+    ref = None if sample_only else oracle.Server(theta0)
+    sched = wlmod.arrival_schedule(wl)[:rounds]
+    all_idx, all_val, all_sig, begins, pulls = [], [], [], [], []
+    for r, rd in enumerate(sched):
+        idx, val = wlmod.synthetic_updates(wl, ks, r, DEV, zero_fraction)
+        sigma = torch.empty_like(idx)
+        begin = rd.order.astype(np.uint64) * np.uint64(K)
+        srv.apply(idx.view(-1), val.view(-1), begin, np.full(wl.n_workers, K, np.uint32), rd.pull_ts, wl.lr,
+                  sigma_out=sigma.view(-1))
+        h_idx, h_val, h_sig = u32(idx), val.cpu().numpy(), u32(sigma)
+        if ref is not None:
+            for b, w in enumerate(rd.order.tolist()):
+                want = ref.apply(h_idx[w], h_val[w], int(rd.pull_ts[b]), wl.lr)
+                assert np.array_equal(h_sig[w], want), f"round {r} update {b}: staleness differs"
+        else:
+            for b, w in enumerate(rd.order.tolist()):     # arrival order, for the per-parameter trace
+                all_idx.append(h_idx[w]); all_val.append(h_val[w]); all_sig.append(h_sig[w])
+                pulls.append(int(rd.pull_ts[b]))
+    assert srv.last_error() == 0
+    got = theta.cpu().numpy()
+    if ref is not None:
+        assert np.array_equal(bits(got), bits(ref.theta()))
+        assert srv.timestamp == ref.timestamp
+        return
+    # sampled parameters, each traced through every update by searching its index list
+    idx_cat, val_cat = np.concatenate(all_idx), np.concatenate(all_val)
+    pair_begin = (np.arange(len(all_idx) + 1, dtype=np.uint64) * np.uint64(K))
+    rng = np.random.default_rng(5)
+    named = np.unique(np.concatenate([a[rng.integers(0, K, 40)] for a in all_idx]))
+    picks = np.concatenate([named[:400], rng.integers(0, wl.n_params, 50).astype(np.uint32)])
+    for k in picks:
+        sig_k, theta_k = oracle.parameter_trace(int(k), float(theta0[k]), idx_cat, val_cat, pair_begin,
+                                                np.array(pulls, np.uint64), wl.lr)
+        seen = [int(s[np.searchsorted(a, k)]) for a, s in zip(all_idx, all_sig)
+                if np.searchsorted(a, k) < K and a[np.searchsorted(a, k)] == k]
+        assert list(sig_k) == seen
+        assert np.float32(theta_k).view(np.uint32) == got[k].view(np.uint32)
+    # parameters no update named are untouched
+    touched = np.zeros(wl.n_params, dtype=bool)
+    touched[idx_cat] = True
+    assert np.array_equal(bits(got[~touched]), bits(theta0[~touched]))
+
+
+@pytest.mark.parametrize("mode", MODES)
+def test_many_workers_full_size_server(binding, mode):
+    wl = wlmod.workload(1)                               # 200 workers x 10 rounds x 32 748 pairs
+    ks = oracle_keep_counts(wl.tensor_sizes, (1, 100))
+    run_server_both(binding, wl, ks, mode, zero_fraction=0.01)
+
+
+@pytest.mark.parametrize("mode", MODES)
+def test_resnet_full_size_server(binding, mode):
+    wl = wlmod.workload(3)
+    ks = oracle_keep_counts(wl.tensor_sizes, (5, 1000))
+    run_server_both(binding, wl, ks, mode)
+
+
+@pytest.mark.parametrize("mode", MODES)
+@pytest.mark.parametrize("keep", [(1, 1000), (1, 10)])
+def test_large_flat_full_size_server_sampled(binding, mode, keep):
+    wl = wlmod.workload(4)
+    ks = oracle_keep_counts(wl.tensor_sizes, keep)
+    run_server_both(binding, wl, ks, mode, sample_only=True)
+
+
+# ----------------------------------------------------------------------------- semantics and errors
+
+@pytest.mark.parametrize("mode", MODES)
+def test_zero_values_empty_updates_and_scattered_slices(binding, mode):
+    theta = torch.tensor([-0.0, 1.0, 2.0, -0.0, 5.0, 6.0], device=DEV)
+    srv = binding.Server(theta, history_pairs=64, max_window_updates=8)
+    srv.set_mode(mode)
+    ref = oracle.Server(theta.cpu().numpy())
+    # three updates stored out of arrival order inside one buffer, one of them empty
+    idx = i32([9, 9, 0, 1, 3, 1, 4, 5])
+    val = torch.tensor([0, 0, 0.0, 1.0, -0.0, 0.5, 0.25, 0.0], device=DEV)
+    sigma = torch.full((8,), -1, dtype=torch.int32, device=DEV)
+    begin, count, pull = [5, 0, 2, 5], [3, 0, 3, 3], [0, 0, 0, 1]
+    srv.apply(idx, val, begin, count, pull, 0.5, sigma_out=sigma)
+    want = []
+    for b, c, j in zip(begin, count, pull):
+        want.append(ref.apply(u32(idx)[b:b + c], val.cpu().numpy()[b:b + c], j, 0.5))
+    assert srv.last_error() == 0 and srv.timestamp == 4 == ref.timestamp
+    assert np.array_equal(bits(theta), bits(ref.theta()))
+    s = u32(sigma)
+    assert list(s[5:8]) == list(want[3]) and list(s[2:5]) == list(want[2])
+    assert list(want[3]) == [1, 0, 0]      # the last update overwrote the first one's sigma slots
+    assert torch.signbit(theta[0]) and torch.signbit(theta[3])
+
+
+def test_window_and_capacity_errors_leave_the_server_unchanged(binding):
+    theta = torch.zeros(100, device=DEV)
+    srv = binding.Server(theta, history_pairs=40, max_window_updates=8)     # ring of 64 pairs
+    idx = i32(np.arange(10))
+    val = torch.ones(10, device=DEV)
+    one = lambda j: srv.apply(idx, val, [0], [10], [j], 0.1)
+    for _ in range(6):
+        one(0)                                              # positions 0 .. 59
+    assert srv.timestamp == 6
+    for bad_j in (7, 99):                                   # j > i
+        with pytest.raises(binding.AdacompError) as e:
+            one(bad_j)
+        assert e.value.status == binding.ERR_WINDOW
+    with pytest.raises(binding.AdacompError) as e:          # 70 positions back: update 0 would be overwritten
+        one(0)
+    assert e.value.status == binding.ERR_WINDOW
+    with pytest.raises(binding.AdacompError) as e:          # too many updates in one call
+        srv.apply(idx, val, [0] * 9, [1] * 9, [6] * 9, 0.1)
+    assert e.value.status == binding.ERR_CAPACITY
+    big = i32(np.arange(50))
+    with pytest.raises(binding.AdacompError) as e:          # one call's pairs exceed history_pairs
+        srv.apply(big, torch.ones(50, device=DEV), [0], [50], [6], 0.1)
+    assert e.value.status == binding.ERR_CAPACITY
+    assert srv.timestamp == 6 and srv.last_error() == 0
+    sig = torch.empty(10, dtype=torch.int32, device=DEV)
+    srv.apply(idx, val, [0], [10], [1], 0.1, sigma_out=sig)  # still usable; window = updates 1..5
+    assert srv.timestamp == 7 and sig.tolist() == [5] * 10
+    assert np.allclose(theta[:10].cpu().numpy(), -0.1 * (1 + 1 + 1 / 2 + 1 / 3 + 1 / 4 + 1 / 5 + 1 / 5), rtol=1e-6)
+    for far_j in (0,):                                      # window longer than max_window_updates
+        for _ in range(2):
+            one(srv.timestamp)
+        with pytest.raises(binding.AdacompError) as e:
+            one(0)
+        assert e.value.status == binding.ERR_WINDOW
+
+
+@pytest.mark.parametrize("mode", MODES)
+def test_bad_indices_are_reported_not_followed(binding, mode):
+    theta = torch.zeros(10, device=DEV)
+    srv = binding.Server(theta, history_pairs=64, max_window_updates=8)
+    srv.set_mode(mode)
+    srv.apply(i32([1, 2, 4_000_000_000]), torch.ones(3, device=DEV), [0], [3], [0], 0.5)
+    assert srv.last_error() == binding.ERR_UNSORTED         # index >= n_params: skipped and reported
+    assert srv.last_error() == 0                            # reading clears it
+    assert theta.cpu().tolist() == [0, -0.5, -0.5, 0, 0, 0, 0, 0, 0, 0]
+    srv.set_validation(True)
+    srv.apply(i32([3, 3]), torch.ones(2, device=DEV), [0], [2], [1], 0.5)
+    assert srv.last_error() == binding.ERR_UNSORTED
+
+
+@pytest.mark.parametrize("mode", MODES)
+def test_position_rebasing(binding, mode):
+    wl = wlmod.workload(1).scaled(256, n_workers=10, n_rounds=6)
+    ks = oracle_keep_counts(wl.tensor_sizes, (1, 10))
+    K = int(sum(ks))
+    theta = wlmod.initial_parameters(wl, DEV)
+    ref = oracle.Server(theta.cpu().numpy())
+    srv = binding.Server(theta, history_pairs=2 * wl.n_workers * K, max_window_updates=2 * wl.n_workers)
+    srv.set_mode(mode)
+    srv.debug_skip_positions(2**32 - 16 - 2 * wl.n_workers * K - K // 2)   # re-base falls inside round 2
+    for r, rd in enumerate(wlmod.arrival_schedule(wl)):
+        idx, val = wlmod.synthetic_updates(wl, ks, r, DEV)
+        sigma = torch.empty_like(idx)
+        srv.apply(idx.view(-1), val.view(-1), rd.order.astype(np.uint64) * np.uint64(K),
+                  np.full(wl.n_workers, K, np.uint32), rd.pull_ts, wl.lr, sigma_out=sigma.view(-1))
+        for b, w in enumerate(rd.order.tolist()):
+            want = ref.apply(u32(idx)[w], val[w].cpu().numpy(), int(rd.pull_ts[b]), wl.lr)
+            assert np.array_equal(u32(sigma)[w], want), f"round {r}"
+    assert srv.last_error() == 0
+    assert np.array_equal(bits(theta), bits(ref.theta()))
+
+
+def test_pull_returns_timestamp_and_copy(binding):
+    theta = torch.arange(8, dtype=torch.float32, device=DEV)
+    srv = binding.Server(theta, history_pairs=16, max_window_updates=4)
+    assert srv.pull() == 0
+    srv.apply(i32([2]), torch.ones(1, device=DEV), [0], [1], [0], 1.0)
+    copy = torch.empty_like(theta)
+    assert srv.pull(copy) == 1
+    torch.cuda.synchronize()
+    assert copy.tolist() == [0, 1, 1, 3, 4, 5, 6, 7]
+    fresh = torch.zeros(8, device=DEV)
+    srv.reset(fresh)
+    assert srv.pull() == 0
+    srv.apply(i32([2]), torch.ones(1, device=DEV), [0], [1], [0], 1.0, sigma_out=(s := torch.zeros(1, dtype=torch.int32, device=DEV)))
+    assert int(s[0]) == 0 and fresh[2].item() == -1.0 and theta[2].item() == 1.0   # history was forgotten
+
+
+def test_host_entry_points(binding):
+    wl = wlmod.workload(0).scaled(16)
+    keep = (1, 100)
+    segs = binding.make_segments(wl.tensor_sizes, keep)
+    sel = binding.Selector(segs, wl.n_workers, DEV)
+    K, W, P = sel.pairs_per_worker, wl.n_workers, wl.n_params
+    h_g = wlmod.round_gradients(wl, 0, "cpu").pin_memory()
+    d_g = torch.empty((W, P), device=DEV)
+    d_idx = torch.empty((W, K), dtype=torch.int32, device=DEV)
+    d_val = torch.empty((W, K), device=DEV)
+    h_idx = torch.empty((W, K), dtype=torch.int32).pin_memory()
+    h_val = torch.empty((W, K)).pin_memory()
+    sel.select_host(h_g, d_g, d_idx, d_val, h_idx, h_val)
+    torch.cuda.synchronize()
+    ks = oracle_keep_counts(wl.tensor_sizes, keep)
+    for w in range(W):
+        oi, ov = oracle.select_layers(h_g[w].numpy(), wl.offsets, wl.tensor_sizes, ks)
+        assert np.array_equal(h_idx[w].numpy().view(np.uint32), oi) and np.array_equal(bits(h_val[w]), bits(ov))
+    theta = wlmod.initial_parameters(wl, DEV)
+    ref = oracle.Server(theta.cpu().numpy())
+    srv = binding.Server(theta, history_pairs=W * K, max_window_updates=W)
+    (rd,) = wlmod.arrival_schedule(wl)
+    d_sig = torch.empty((W, K), dtype=torch.int32, device=DEV)
+    h_sig = torch.empty((W, K), dtype=torch.int32).pin_memory()
+    srv.apply_host(h_idx.view(-1), h_val.view(-1), rd.order.astype(np.uint64) * np.uint64(K), np.full(W, K, np.uint32),
+                   rd.pull_ts, wl.lr, d_idx.view(-1), d_val.view(-1), d_sig.view(-1), h_sig.view(-1))
+    torch.cuda.synchronize()
+    for b, w in enumerate(rd.order.tolist()):
+        want = ref.apply(h_idx[w].numpy().view(np.uint32), h_val[w].numpy(), int(rd.pull_ts[b]), wl.lr)
+        assert np.array_equal(h_sig[w].numpy().view(np.uint32), want)
+    assert np.array_equal(bits(theta), bits(ref.theta()))

@@ -1,0 +1,165 @@
+"""Parity of adacomp_select (CUDA, through the C ABI) with the CPU oracle: indices and values
+must match bit for bit."""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+from paper_1702_04683_b200 import workloads as wlmod
+
+from helpers import bits, oracle_keep_counts, oracle_select_round, u32
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module")
+def binding():
+    from paper_1702_04683_b200 import binding as b
+    return b
+
+
+def gpu_select(binding, grads, offsets, ns, ks, max_workers=None):
+    segs = binding.segments_from(offsets, ns, ks)
+    sel = binding.Selector(segs, max_workers or (grads.shape[0] if grads.dim() == 2 else 1), grads.device)
+    idx, val = sel.select(grads)
+    status, _ = sel.last_error()
+    assert status == 0
+    return u32(idx), val.cpu().numpy(), sel
+
+
+def check_against_oracle(binding, grads, offsets, ns, ks):
+    idx, val, _ = gpu_select(binding, grads, offsets, ns, ks)
+    g_host = grads.cpu().numpy()
+    if g_host.ndim == 1:
+        g_host = g_host[None]
+    for w in range(g_host.shape[0]):
+        oi, ov = oracle.select_layers(g_host[w], offsets, ns, ks)
+        assert np.array_equal(idx[w], oi), f"worker {w}: indices differ"
+        assert np.array_equal(bits(val[w]), bits(ov)), f"worker {w}: values differ"
+
+
+# ----------------------------------------------------------------------------- edge cases
+
+def test_tiny_and_degenerate_segments(binding):
+    dev = torch.device("cuda", 0)
+    ns = [1, 2, 0, 7, 13, 64, 1001, 4096, 5, 3]
+    ks = [1, 2, 0, 0, 13, 1, 17, 4096, 5, 1]
+    offsets = np.concatenate([[0], np.cumsum(ns)[:-1]]).tolist()
+    g = torch.randn(3, sum(ns), device=dev)
+    check_against_oracle(binding, g, offsets, ns, ks)
+
+
+def test_ties_zeros_and_inf(binding):
+    dev = torch.device("cuda", 0)
+    n = 300_000                              # three chunks with a ragged tail
+    cases = {
+        "all_equal": torch.full((n,), 0.5),
+        "all_zero_mixed_sign": torch.where(torch.arange(n) % 3 == 0, torch.tensor(-0.0), torch.tensor(0.0)),
+        "two_values": torch.where(torch.rand(n) < 0.5, torch.tensor(1.0), torch.tensor(-2.0)),
+        "coarse_grid": torch.round(torch.randn(n) * 3) / 3,
+        "with_inf": torch.cat([torch.randn(n - 4), torch.tensor([float("inf"), -float("inf"), 0.0, -0.0])]),
+        "denormals": torch.randn(n) * 1e-42,
+    }
+    for name, g in cases.items():
+        g = g.to(torch.float32).to(dev)
+        for k in (1, 2, 1000, n // 2, n - 1, n):
+            check_against_oracle(binding, g, [0], [n], [k])
+
+
+def test_gaps_strides_and_unaligned_views(binding):
+    dev = torch.device("cuda", 0)
+    # segments with gaps between them, odd sizes, a worker stride larger than the extent and a
+    # base pointer that is only 4-byte aligned
+    offsets = [3, 1000, 140_001, 400_000]
+    ns = [990, 139_000, 131_073, 262_145]
+    ks = [10, 1390, 1311, 2622]
+    extent = offsets[-1] + ns[-1]
+    buf = torch.randn(4 * (extent + 37) + 1, device=dev)
+    for shift in (0, 1, 2, 3):
+        g = buf[shift:shift + 4 * (extent + 37)].view(4, extent + 37)
+        assert g.data_ptr() % 16 == (buf.data_ptr() + 4 * shift) % 16
+        check_against_oracle(binding, g, offsets, ns, ks)
+
+
+def test_deterministic_and_input_untouched(binding):
+    dev = torch.device("cuda", 0)
+    wl = wlmod.workload(0)
+    g = wlmod.round_gradients(wl, 0, dev)
+    before = g.clone()
+    ks = oracle_keep_counts(wl.tensor_sizes, (1, 100))
+    a_idx, a_val, sel = gpu_select(binding, g, wl.offsets, wl.tensor_sizes, ks)
+    idx2, val2 = sel.select(g)
+    assert np.array_equal(a_idx, u32(idx2)) and np.array_equal(bits(a_val), bits(val2))
+    assert torch.equal(g, before)
+
+
+def test_fewer_workers_than_the_handle_allows(binding):
+    dev = torch.device("cuda", 0)
+    g = torch.randn(5, 50_000, device=dev)
+    segs = binding.segments_from([0, 20_000], [20_000, 30_000], [200, 3000])
+    sel = binding.Selector(segs, 8, dev)
+    idx, val = sel.select(g[:2])
+    for w in range(2):
+        oi, ov = oracle.select_layers(g[w].cpu().numpy(), [0, 20_000], [20_000, 30_000], [200, 3000])
+        assert np.array_equal(u32(idx)[w], oi) and np.array_equal(bits(val[w]), bits(ov))
+    with pytest.raises(binding.AdacompError):
+        sel.select(torch.randn(9, 50_000, device=dev))
+
+
+# ----------------------------------------------------------------------------- the workloads
+
+def test_small_cnn_full_size(binding):
+    wl = wlmod.workload(0)
+    g = wlmod.round_gradients(wl, 0, torch.device("cuda", 0))
+    ks = oracle_keep_counts(wl.tensor_sizes, wl.keep_fractions[0])
+    assert sum(ks) == 32_748
+    check_against_oracle(binding, g, wl.offsets, wl.tensor_sizes, ks)
+
+
+@pytest.mark.parametrize("keep", [(1, 1000), (1, 100), (1, 10)])
+def test_tie_stress_full_tensors(binding, keep):
+    wl = wlmod.workload(2)
+    g = wlmod.round_gradients(wl, 0, torch.device("cuda", 0), workers=range(6))
+    ks = oracle_keep_counts(wl.tensor_sizes, keep)
+    # the data really has ties at the threshold in the big tensor
+    check_against_oracle(binding, g, wl.offsets, wl.tensor_sizes, ks)
+
+
+def test_resnet50_shaped_full_tensors(binding):
+    wl = wlmod.workload(3)
+    g = wlmod.round_gradients(wl, 0, torch.device("cuda", 0), workers=range(3))
+    ks = oracle_keep_counts(wl.tensor_sizes, wl.keep_fractions[0])
+    assert sum(ks) == 127_874
+    check_against_oracle(binding, g, wl.offsets, wl.tensor_sizes, ks)
+
+
+@pytest.mark.parametrize("keep", [(1, 1000), (1, 64), (1, 10)])
+def test_large_flat_full_size_sampled(binding, keep):
+    """100 M parameters x 16 workers in the launch configuration the benchmark times; the oracle
+    checks sampled (worker, tensor) selections one by one, and cheap invariants cover the rest."""
+    dev = torch.device("cuda", 0)
+    wl = wlmod.workload(4)
+    g = wlmod.round_gradients(wl, 0, dev)
+    ks = oracle_keep_counts(wl.tensor_sizes, keep)
+    K = sum(ks)
+    segs = binding.segments_from(wl.offsets, wl.tensor_sizes, ks)
+    sel = binding.Selector(segs, wl.n_workers, dev)
+    idx, val = sel.select(g)
+    assert sel.last_error()[0] == 0
+    # invariants at full size, on the GPU: ascending inside each tensor's slice, values are the
+    # entries they name, indices stay inside their tensor
+    idx64 = idx.view(wl.n_workers, len(ks), ks[0]).to(torch.int64) & 0xFFFFFFFF
+    assert bool((idx64[:, :, 1:] > idx64[:, :, :-1]).all())
+    lo = torch.tensor(wl.offsets, device=dev).view(1, -1, 1)
+    assert bool(((idx64 >= lo) & (idx64 < lo + wl.tensor_sizes[0])).all())
+    gathered = torch.gather(g, 1, idx64.view(wl.n_workers, K))
+    assert torch.equal(gathered.view(torch.int32), val.view(torch.int32))
+    # the oracle on sampled selections
+    rng = np.random.default_rng(keep[1])
+    for _ in range(6):
+        w, l = int(rng.integers(wl.n_workers)), int(rng.integers(len(ks)))
+        off, n = wl.offsets[l], wl.tensor_sizes[l]
+        oi, ov = oracle.select(g[w, off:off + n].cpu().numpy(), ks[l], offset=off)
+        lo_k = sum(ks[:l])
+        assert np.array_equal(u32(idx[w, lo_k:lo_k + ks[l]]), oi)
+        assert np.array_equal(bits(val[w, lo_k:lo_k + ks[l]]), bits(ov))
