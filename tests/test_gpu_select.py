@@ -74,7 +74,7 @@ def test_gaps_strides_and_unaligned_views(binding):
     ns = [990, 139_000, 131_073, 262_145]
     ks = [10, 1390, 1311, 2622]
     extent = offsets[-1] + ns[-1]
-    buf = torch.randn(4 * (extent + 37) + 1, device=dev)
+    buf = torch.randn(4 * (extent + 37) + 3, device=dev)
     for shift in (0, 1, 2, 3):
         g = buf[shift:shift + 4 * (extent + 37)].view(4, extent + 37)
         assert g.data_ptr() % 16 == (buf.data_ptr() + 4 * shift) % 16
