@@ -126,6 +126,13 @@ ADACOMP_API int adacomp_select_host(adacomp_select_t* h, const float* h_grads, u
                         float* d_val_staging, uint32_t* h_idx_out, float* h_val_out,
                         void* cuda_stream);
 
+/* Chooses how selections are computed; the results are identical.
+ * 0 = automatic: tensors of at least 32768 entries with k <= n/4 take the bracketed route (a
+ *     sample brackets the threshold, then the gradient is read once); instances whose bracket
+ *     turns out wrong, and all other tensors, take the general route;
+ * 1 = general route for everything (multi-pass radix select; reads the gradient five times). */
+ADACOMP_API int adacomp_select_set_route(adacomp_select_t* h, int route);
+
 /* K = sum of k over the layout's segments (pairs per worker). */
 ADACOMP_API int adacomp_select_pairs_per_worker(const adacomp_select_t* h, uint64_t* pairs_out);
 /* Waits for cuda_stream, then returns the first error the device recorded since the last call

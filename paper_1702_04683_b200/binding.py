@@ -55,6 +55,7 @@ def _load():
         "adacomp_select_create": (i32, [P(vp), P(Segment), u32, u32, vp, ctypes.c_size_t, i32]),
         "adacomp_select": (i32, [vp, vp, u64, u32, vp, vp, vp]),
         "adacomp_select_host": (i32, [vp, vp, u64, u32, vp, vp, vp, vp, vp, vp]),
+        "adacomp_select_set_route": (i32, [vp, i32]),
         "adacomp_select_pairs_per_worker": (i32, [vp, P(u64)]),
         "adacomp_select_last_error": (i32, [vp, vp, P(u64)]),
         "adacomp_select_destroy": (i32, [vp]),
@@ -201,6 +202,10 @@ class Selector:
                                         _dev(d_val, torch.float32, "d_val"), _host(h_idx, torch.int32, "h_idx"),
                                         _host(h_val, torch.float32, "h_val"), _stream_ptr(stream)),
                "adacomp_select_host")
+
+    def set_route(self, route: int):
+        """0 = automatic (bracketed single pass where eligible), 1 = general route only."""
+        _check(_lib.adacomp_select_set_route(self._h, int(route)), "adacomp_select_set_route")
 
     def last_error(self, stream: Optional[torch.cuda.Stream] = None) -> Tuple[int, int]:
         """(status, selections that took the general route in the last call); waits for the stream."""

@@ -1,18 +1,21 @@
 // Worker side of libadacomp: handle, workspace layout and launch sequence of SELECT_GRAD
 // (Algorithm 1).
+#include <cmath>
 #include <new>
 #include <vector>
 
-#include "select_general.cuh"
+#include "select_bracket.cuh"
 
 using namespace adacomp;
 
 struct adacomp_select {
     int device = 0;
     int n_sms = 0;
-    uint32_t n_layers = 0, max_workers = 0, slots_per_worker = 0;
+    int route = 0;         // 0 = automatic, 1 = general route for everything
+    uint32_t n_layers = 0, max_workers = 0, slots_per_worker = 0, n_items = 0, max_sample = 0;
     uint64_t extent = 0;   // one past the last entry any segment covers
     uint64_t K = 0;        // pairs per worker
+    uint64_t cand_stride = 0, win_stride = 0, span_stride = 0;
     // device (inside the caller's workspace)
     Layer* d_layers = nullptr;
     Inst* d_inst = nullptr;
@@ -22,16 +25,62 @@ struct adacomp_select {
     uint32_t* d_list_len = nullptr;
     uint2* d_chunk_cnt = nullptr;
     int* d_status = nullptr;
-    uint32_t* d_stats = nullptr;
+    uint2* d_items = nullptr;
+    uint32_t* d_cand_idx = nullptr;
+    float* d_cand_val = nullptr;
+    uint32_t* d_win_key = nullptr;
+    uint32_t* d_win_idx = nullptr;
+    uint2* d_span_tab = nullptr;
+    uint32_t* d_span_off = nullptr;
 };
 
 namespace {
 
 struct Layout {
     std::vector<Layer> layers;
+    std::vector<uint2> items;
     uint64_t extent = 0, K = 0;
-    uint32_t slots_per_worker = 0;
+    uint64_t cand_stride = 0, win_stride = 0, span_stride = 0;
+    uint32_t slots_per_worker = 0, max_sample = 0;
 };
+
+// Decides whether a tensor takes the bracketed route and how much room its lists get.  The
+// capacities follow the bracket's expected size plus six standard deviations of the sample
+// quantiles; exceeding them is not an error, it only sends the instance to the general route.
+void plan_bracket(Layer& L, Layout* out) {
+    L.bracket = 0;
+    L.sample = L.n_spans = L.span_base = L.cand_cap = L.win_cap = 0;
+    L.cand_base = L.win_base = 0;
+    if (L.n < kBracketMinN || L.k == 0 || static_cast<uint64_t>(L.k) * 4 > L.n) return;
+    const uint32_t n_spans = static_cast<uint32_t>((static_cast<uint64_t>(L.n) + 3 + kSpanElems - 1) / kSpanElems);
+    if (n_spans > kMaxSpans) return;
+    uint32_t m = L.n / 8;
+    if (m > kSampleMax) m = kSampleMax;
+    if (m < kSampleMin) m = kSampleMin;
+    m &= ~31u;
+    uint32_t r_hi, r_lo;
+    bracket_ranks(L.n, L.k, m, &r_hi, &r_lo);
+    if (r_lo + 1 > m) return;                              // sample cannot bound the threshold from below
+    const double n = L.n;
+    const double lo_frac = static_cast<double>(r_lo + 1) / m;
+    const double win_frac = static_cast<double>(r_lo + 1 - r_hi) / m;
+    double cand = n * lo_frac * (1.0 + 6.0 / std::sqrt(static_cast<double>(r_lo))) + 2048.0;
+    double win = n * win_frac * (1.0 + 6.0 / std::sqrt(static_cast<double>(r_lo + 1 - r_hi))) + 2048.0;
+    if (cand > n) cand = n;
+    if (win > n) win = n;
+    L.bracket = 1;
+    L.sample = m;
+    L.n_spans = n_spans;
+    L.span_base = static_cast<uint32_t>(out->span_stride);
+    L.cand_cap = static_cast<uint32_t>(cand);
+    L.win_cap = static_cast<uint32_t>(win);
+    L.cand_base = out->cand_stride;
+    L.win_base = out->win_stride;
+    out->span_stride += n_spans;
+    out->cand_stride += (L.cand_cap + 63) & ~63ull;
+    out->win_stride += (L.win_cap + 63) & ~63ull;
+    if (m > out->max_sample) out->max_sample = m;
+}
 
 int build_layout(const adacomp_segment_t* segs, uint32_t n_segs, uint32_t max_workers, Layout* out) {
     if (!segs || n_segs == 0 || max_workers == 0) return ADACOMP_ERR_INVALID;
@@ -54,9 +103,13 @@ int build_layout(const adacomp_segment_t* segs, uint32_t n_segs, uint32_t max_wo
         slots += L.n_slots;
         K += s.k;
         end_prev = s.offset + s.n;
+        plan_bracket(L, out);
+        for (uint32_t s0 = 0; L.bracket && s0 < L.n_spans; s0 += kSpansPerBlock)
+            out->items.push_back(make_uint2(l, s0));
     }
     if (K > kMaxIndex || slots * max_workers > 0x7FFFFFFFull ||
-        static_cast<uint64_t>(n_segs) * max_workers > 0x7FFFFFFFull)
+        static_cast<uint64_t>(n_segs) * max_workers > 0x7FFFFFFFull ||
+        out->span_stride * max_workers > 0x7FFFFFFFull || out->items.size() > 0x7FFFFFFFull)
         return ADACOMP_ERR_INVALID;
     out->extent = end_prev;
     out->K = K;
@@ -67,16 +120,23 @@ int build_layout(const adacomp_segment_t* segs, uint32_t n_segs, uint32_t max_wo
 // One place that decides the workspace layout; with a null base it only measures.
 size_t carve(adacomp_select_t* h, void* base, const Layout& lay, uint32_t max_workers) {
     Carver c(base);
-    const size_t n_inst = static_cast<size_t>(lay.layers.size()) * max_workers;
+    const size_t W = max_workers;
+    const size_t n_inst = lay.layers.size() * W;
     h->d_layers = c.take<Layer>(lay.layers.size());
     h->d_inst = c.take<Inst>(n_inst);
     h->d_hist = c.take<uint32_t>(n_inst * kBins);
     h->d_list = c.take<uint32_t>(n_inst);
     h->d_list_slot_start = c.take<uint32_t>(n_inst);
     h->d_list_len = c.take<uint32_t>(2);
-    h->d_chunk_cnt = c.take<uint2>(static_cast<size_t>(lay.slots_per_worker) * max_workers);
+    h->d_chunk_cnt = c.take<uint2>(lay.slots_per_worker * W);
     h->d_status = c.take<int>(1);
-    h->d_stats = c.take<uint32_t>(4);
+    h->d_items = c.take<uint2>(lay.items.size() + 1);
+    h->d_cand_idx = c.take<uint32_t>(lay.cand_stride * W);
+    h->d_cand_val = c.take<float>(lay.cand_stride * W);
+    h->d_win_key = c.take<uint32_t>(lay.win_stride * W);
+    h->d_win_idx = c.take<uint32_t>(lay.win_stride * W);
+    h->d_span_tab = c.take<uint2>(lay.span_stride * W + 1);
+    h->d_span_off = c.take<uint32_t>(lay.span_stride * W + 1);
     return c.used;
 }
 
@@ -113,15 +173,35 @@ int adacomp_select_create(adacomp_select_t** h, const adacomp_segment_t* h_segs,
     s->slots_per_worker = lay.slots_per_worker;
     s->extent = lay.extent;
     s->K = lay.K;
+    s->n_items = static_cast<uint32_t>(lay.items.size());
+    s->max_sample = lay.max_sample;
+    s->cand_stride = lay.cand_stride;
+    s->win_stride = lay.win_stride;
+    s->span_stride = lay.span_stride;
     DeviceGuard guard(device);
     cudaError_t e = guard.err;
     if (e == cudaSuccess) e = cudaDeviceGetAttribute(&s->n_sms, cudaDevAttrMultiProcessorCount, device);
-    if (e == cudaSuccess) e = cudaMemset(d_workspace, 0, need);
+    // only the bookkeeping needs clearing; the candidate / window lists are write-before-read
+    if (e == cudaSuccess) {
+        const size_t head = reinterpret_cast<char*>(s->d_items) - static_cast<char*>(d_workspace);
+        e = cudaMemset(d_workspace, 0, head);
+    }
     if (e == cudaSuccess)
         e = cudaMemcpy(s->d_layers, lay.layers.data(), lay.layers.size() * sizeof(Layer), cudaMemcpyHostToDevice);
+    if (e == cudaSuccess && !lay.items.empty())
+        e = cudaMemcpy(s->d_items, lay.items.data(), lay.items.size() * sizeof(uint2), cudaMemcpyHostToDevice);
+    if (e == cudaSuccess)
+        e = cudaFuncSetAttribute(k_bracket_sample, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                 static_cast<int>(kSampleMax * sizeof(uint32_t)));
     if (e == cudaSuccess) e = cudaDeviceSynchronize();
     if (e != cudaSuccess) { delete s; return cuda_fail(e); }
     *h = s;
+    return ADACOMP_OK;
+}
+
+int adacomp_select_set_route(adacomp_select_t* h, int route) {
+    if (!h || route < 0 || route > 1) return ADACOMP_ERR_INVALID;
+    h->route = route;
     return ADACOMP_OK;
 }
 
@@ -152,14 +232,41 @@ int adacomp_select(adacomp_select_t* h, const float* d_grads, uint64_t worker_st
     p.val_out = d_val_out;
     p.K = h->K;
     p.status = h->d_status;
+    p.items = h->d_items;
+    p.cand_idx = h->d_cand_idx;
+    p.cand_val = h->d_cand_val;
+    p.win_key = h->d_win_key;
+    p.win_idx = h->d_win_idx;
+    p.span_tab = h->d_span_tab;
+    p.span_off = h->d_span_off;
+    p.cand_stride = h->cand_stride;
+    p.win_stride = h->win_stride;
+    p.span_stride = h->span_stride;
 
+    const unsigned n_inst = n_workers * h->n_layers;
+    const bool bracketed = h->route == 0 && h->n_items > 0;
+
+    // bracketed route: sample -> single pass -> resolve -> emit
+    k_bracket_sample<<<n_inst, kThreads, bracketed ? h->max_sample * sizeof(uint32_t) : 0, st>>>(p, bracketed ? 0 : 1);
+    ADACOMP_LAUNCH_CHECK();
+    if (bracketed) {
+        const dim3 grid(h->n_items, n_workers);
+        k_bracket_scan<<<grid, kThreads, 0, st>>>(p);
+        ADACOMP_LAUNCH_CHECK();
+        k_bracket_resolve<<<n_inst, kThreads, 0, st>>>(p);
+        ADACOMP_LAUNCH_CHECK();
+        k_bracket_emit<<<grid, kThreads, 0, st>>>(p);
+        ADACOMP_LAUNCH_CHECK();
+    }
+
+    // general route for whatever is flagged for it (tensors not on the bracketed route, and
+    // instances whose bracket missed); the kernels find an empty list otherwise
     const uint64_t total_slots = static_cast<uint64_t>(h->slots_per_worker) * n_workers;
     uint64_t grid64 = static_cast<uint64_t>(h->n_sms) * 8;
     if (grid64 > total_slots) grid64 = total_slots;
     if (grid64 == 0) grid64 = 1;
     const unsigned grid = static_cast<unsigned>(grid64);
-
-    k_general_plan<<<1, kThreads, 0, st>>>(p, 1);
+    k_general_plan<<<1, kThreads, 0, st>>>(p);
     ADACOMP_LAUNCH_CHECK();
     k_general_hist<0><<<grid, kThreads, 0, st>>>(p);
     ADACOMP_LAUNCH_CHECK();

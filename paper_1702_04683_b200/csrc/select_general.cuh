@@ -30,6 +30,15 @@ struct Layer {            // one tensor V_l / beta_l of the layout
     uint32_t n, k;
     uint32_t n_slots;     // chunk slots reserved for it (covers any 16-byte misalignment)
     uint32_t slot_base;   // first slot inside a worker's slot range
+    // bracketed route (select_bracket.cuh); all zero when the tensor is not on it
+    uint32_t bracket;     // 1: eligible for the bracketed single-pass route
+    uint32_t sample;      // sample size m (multiple of 32)
+    uint32_t n_spans;     // spans of kSpanElems entries (covers any misalignment)
+    uint32_t span_base;   // first span inside a worker's span range
+    uint32_t cand_cap;    // room in the candidate list
+    uint32_t win_cap;     // room in the window list
+    uint64_t cand_base;   // first candidate slot inside a worker's candidate range
+    uint64_t win_base;    // first window slot inside a worker's window range
 };
 
 struct Inst {             // selection state of one (worker, tensor)
@@ -38,8 +47,14 @@ struct Inst {             // selection state of one (worker, tensor)
     uint32_t n_gt;        // entries whose key is above the current bucket; after pass 2: #{key > T}
     uint32_t flags;       // route bookkeeping (kInstGeneral ...)
     uint32_t done[5];     // finished chunks per pass
-    uint32_t pad[3];
+    // bracketed route
+    uint32_t t_lo, t_hi;  // the threshold key lies in [t_lo, t_hi]
+    uint32_t cand_count;  // entries with key >= t_lo appended so far
+    uint32_t win_count;   // of those, entries with key <= t_hi
+    uint32_t n_def;       // entries with key > t_hi
+    uint32_t T, cut;      // exact threshold: keep key > T, and key == T with shifted index < cut
 };
+static_assert(sizeof(Inst) == 64, "Inst is one 64-byte record");
 constexpr uint32_t kInstGeneral = 1u;   // instance is (to be) handled by the general route
 
 struct SelectParams {
@@ -58,6 +73,15 @@ struct SelectParams {
     float* val_out;
     uint64_t K;
     int* status;
+    // bracketed route
+    const uint2* items;         // scan / emit work items: (tensor, first span)
+    uint32_t* cand_idx;         // [worker][cand_stride] shifted index of each candidate
+    float* cand_val;            //                        its value
+    uint32_t* win_key;          // [worker][win_stride] key of each window entry
+    uint32_t* win_idx;          //                       its shifted index
+    uint2* span_tab;            // [worker][span_stride] (first candidate slot, count | above-window count << 16)
+    uint32_t* span_off;         // [worker][span_stride] kept entries before the span
+    uint64_t cand_stride, win_stride, span_stride;
 };
 
 // ---------------------------------------------------------------------------------------------
@@ -131,9 +155,9 @@ __device__ __forceinline__ WorkItem decode_item(const SelectParams& p, uint32_t 
 }
 
 // ---------------------------------------------------------------------------------------------
-// Builds the work list: every instance with k > 0 (all == 1) or only those flagged for the
-// general route (all == 0).  One block.
-__global__ void __launch_bounds__(kThreads) k_general_plan(SelectParams p, int all) {
+// Builds the work list: the instances flagged for the general route (their state was reset at
+// the start of the call).  One block.
+__global__ void __launch_bounds__(kThreads) k_general_plan(SelectParams p) {
     __shared__ uint32_t s_warp[9];
     __shared__ uint32_t s_carry[2];
     if (threadIdx.x == 0) { s_carry[0] = 0; s_carry[1] = 0; }
@@ -144,13 +168,7 @@ __global__ void __launch_bounds__(kThreads) k_general_plan(SelectParams p, int a
         uint32_t take = 0, slots = 0;
         if (i < n_inst) {
             const Layer& L = p.layers[i % p.n_layers];
-            Inst& st = p.inst[i];
-            if (all) {
-                st.prefix = 0; st.k_rem = L.k; st.n_gt = 0; st.flags = (L.k > 0) ? kInstGeneral : 0u;
-#pragma unroll
-                for (int q = 0; q < 5; ++q) st.done[q] = 0;
-            }
-            take = (st.flags & kInstGeneral) ? 1u : 0u;
+            take = (__ldcg(&p.inst[i].flags) & kInstGeneral) ? 1u : 0u;
             slots = take ? L.n_slots : 0u;
         }
         uint32_t tot_take, tot_slots;

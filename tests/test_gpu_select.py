@@ -106,6 +106,58 @@ def test_fewer_workers_than_the_handle_allows(binding):
         sel.select(torch.randn(9, 50_000, device=dev))
 
 
+def test_routes_agree_and_are_taken(binding):
+    dev = torch.device("cuda", 0)
+    wl = wlmod.workload(0)
+    g = wlmod.round_gradients(wl, 0, dev)
+    ks = oracle_keep_counts(wl.tensor_sizes, (1, 100))
+    segs = binding.segments_from(wl.offsets, wl.tensor_sizes, ks)
+    sel = binding.Selector(segs, wl.n_workers, dev)
+    idx_a, val_a = sel.select(g)
+    status, general = sel.last_error()
+    assert status == 0 and general == 8 * 2        # only the 832- and 10 250-entry tensors are too small
+    sel.set_route(1)
+    idx_g, val_g = sel.select(g)
+    status, general = sel.last_error()
+    assert status == 0 and general == 8 * 4
+    assert torch.equal(idx_a, idx_g) and torch.equal(val_a.view(torch.int32), val_g.view(torch.int32))
+    sel.set_route(0)
+    idx_b, _ = sel.select(g)
+    assert torch.equal(idx_a, idx_b) and sel.last_error() == (0, 16)
+
+
+def test_awkward_value_layouts_stay_exact_and_ties_fall_back(binding):
+    dev = torch.device("cuda", 0)
+    n, k = 1_000_000, 10_000
+    g = torch.randn(3, n, device=dev) * 1e-6
+    # worker 0: every large entry sits in one contiguous block
+    g[0, 500_000:510_000] = (1.0 + torch.rand(10_000, device=dev)) * torch.where(torch.rand(10_000, device=dev) < 0.5, -1.0, 1.0)
+    # worker 1: sorted by magnitude
+    g[1] = torch.sort(g[1].abs())[0]
+    # worker 2: two magnitudes only, so the threshold value is shared by half a million entries and
+    # no bracket can isolate it: the instance must be handed to the general route
+    g[2] = torch.where(torch.rand(n, device=dev) < 0.5, 1.0, -2.0)
+    idx, val, sel = gpu_select(binding, g, [0], [n], [k])
+    for w in range(3):
+        oi, ov = oracle.select(g[w].cpu().numpy(), k)
+        assert np.array_equal(idx[w], oi) and np.array_equal(bits(val[w]), bits(ov))
+    sel.select(g)
+    assert sel.last_error() == (0, 1)
+
+
+@pytest.mark.parametrize("n,k", [(32_768, 1), (32_768, 8192), (40_000, 400), (65_537, 700), (1 << 20, 1), (3_000_001, 30_001)])
+def test_bracket_route_sizes(binding, n, k):
+    dev = torch.device("cuda", 0)
+    g = torch.randn(3, n + 5, device=dev)[:, 2:n + 2]          # rows start at odd alignments
+    segs = binding.segments_from([0], [n], [k])
+    sel = binding.Selector(segs, 3, dev)
+    idx, val = sel.select(g)
+    assert sel.last_error()[0] == 0
+    for w in range(3):
+        oi, ov = oracle.select(g[w].cpu().numpy(), k)
+        assert np.array_equal(u32(idx[w]), oi) and np.array_equal(bits(val[w]), bits(ov))
+
+
 # ----------------------------------------------------------------------------- the workloads
 
 def test_small_cnn_full_size(binding):
