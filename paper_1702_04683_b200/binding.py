@@ -56,6 +56,9 @@ def _load():
         "adacomp_select": (i32, [vp, vp, u64, u32, vp, vp, vp]),
         "adacomp_select_host": (i32, [vp, vp, u64, u32, vp, vp, vp, vp, vp, vp]),
         "adacomp_select_set_route": (i32, [vp, i32]),
+        "adacomp_select_set_profiling": (i32, [vp, i32]),
+        "adacomp_select_profile": (i32, [vp, P(f32), u32]),
+        "adacomp_select_stage_name": (ctypes.c_char_p, [u32]),
         "adacomp_select_pairs_per_worker": (i32, [vp, P(u64)]),
         "adacomp_select_last_error": (i32, [vp, vp, P(u64)]),
         "adacomp_select_destroy": (i32, [vp]),
@@ -206,6 +209,15 @@ class Selector:
     def set_route(self, route: int):
         """0 = automatic (bracketed single pass where eligible), 1 = general route only."""
         _check(_lib.adacomp_select_set_route(self._h, int(route)), "adacomp_select_set_route")
+
+    def set_profiling(self, on: bool):
+        _check(_lib.adacomp_select_set_profiling(self._h, int(on)), "adacomp_select_set_profiling")
+
+    def profile(self) -> dict:
+        """Device milliseconds per kernel of the last select call (profiling must be on)."""
+        ms = (ctypes.c_float * 10)()
+        _check(_lib.adacomp_select_profile(self._h, ms, 10), "adacomp_select_profile")
+        return {_lib.adacomp_select_stage_name(i).decode(): float(ms[i]) for i in range(10)}
 
     def last_error(self, stream: Optional[torch.cuda.Stream] = None) -> Tuple[int, int]:
         """(status, selections that took the general route in the last call); waits for the stream."""

@@ -8,6 +8,13 @@
 
 using namespace adacomp;
 
+namespace {
+constexpr int kSelectStages = 10;
+const char* const kStageNames[kSelectStages] = {
+    "bracket_sample", "bracket_scan", "bracket_resolve", "bracket_emit", "general_plan",
+    "general_hist0", "general_hist1", "general_hist2", "general_count", "general_write"};
+}  // namespace
+
 struct adacomp_select {
     int device = 0;
     int n_sms = 0;
@@ -30,8 +37,12 @@ struct adacomp_select {
     float* d_cand_val = nullptr;
     uint32_t* d_win_key = nullptr;
     uint32_t* d_win_idx = nullptr;
-    uint2* d_span_tab = nullptr;
+    uint2* d_sub_tab = nullptr;
     uint32_t* d_span_off = nullptr;
+    // optional stage timing: events around every kernel of the last call
+    bool profiling = false;
+    cudaEvent_t ev[kSelectStages + 1] = {};
+    bool ev_recorded[kSelectStages + 1] = {};
 };
 
 namespace {
@@ -135,7 +146,7 @@ size_t carve(adacomp_select_t* h, void* base, const Layout& lay, uint32_t max_wo
     h->d_cand_val = c.take<float>(lay.cand_stride * W);
     h->d_win_key = c.take<uint32_t>(lay.win_stride * W);
     h->d_win_idx = c.take<uint32_t>(lay.win_stride * W);
-    h->d_span_tab = c.take<uint2>(lay.span_stride * W + 1);
+    h->d_sub_tab = c.take<uint2>(lay.span_stride * W * kSubsPerSpan + 1);
     h->d_span_off = c.take<uint32_t>(lay.span_stride * W + 1);
     return c.used;
 }
@@ -193,6 +204,9 @@ int adacomp_select_create(adacomp_select_t** h, const adacomp_segment_t* h_segs,
     if (e == cudaSuccess)
         e = cudaFuncSetAttribute(k_bracket_sample, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                  static_cast<int>(kSampleMax * sizeof(uint32_t)));
+    if (e == cudaSuccess)
+        e = cudaFuncSetAttribute(k_bracket_scan, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                 static_cast<int>(kScanSmemPerWarp * (kThreads / 32)));
     if (e == cudaSuccess) e = cudaDeviceSynchronize();
     if (e != cudaSuccess) { delete s; return cuda_fail(e); }
     *h = s;
@@ -237,7 +251,7 @@ int adacomp_select(adacomp_select_t* h, const float* d_grads, uint64_t worker_st
     p.cand_val = h->d_cand_val;
     p.win_key = h->d_win_key;
     p.win_idx = h->d_win_idx;
-    p.span_tab = h->d_span_tab;
+    p.sub_tab = h->d_sub_tab;
     p.span_off = h->d_span_off;
     p.cand_stride = h->cand_stride;
     p.win_stride = h->win_stride;
@@ -245,19 +259,31 @@ int adacomp_select(adacomp_select_t* h, const float* d_grads, uint64_t worker_st
 
     const unsigned n_inst = n_workers * h->n_layers;
     const bool bracketed = h->route == 0 && h->n_items > 0;
+    for (int i = 0; i <= kSelectStages; ++i) h->ev_recorded[i] = false;
+    // mark(i): the boundary before stage i (and after stage i - 1)
+    auto mark = [&](int i) -> cudaError_t {
+        if (!h->profiling) return cudaSuccess;
+        h->ev_recorded[i] = true;
+        return cudaEventRecord(h->ev[i], st);
+    };
+    ADACOMP_CUDA(mark(0));
 
     // bracketed route: sample -> single pass -> resolve -> emit
-    k_bracket_sample<<<n_inst, kThreads, bracketed ? h->max_sample * sizeof(uint32_t) : 0, st>>>(p, bracketed ? 0 : 1);
+    k_bracket_sample<<<n_inst, kBig, bracketed ? h->max_sample * sizeof(uint32_t) : 0, st>>>(p, bracketed ? 0 : 1);
     ADACOMP_LAUNCH_CHECK();
+    ADACOMP_CUDA(mark(1));
     if (bracketed) {
         const dim3 grid(h->n_items, n_workers);
-        k_bracket_scan<<<grid, kThreads, 0, st>>>(p);
+        k_bracket_scan<<<grid, kThreads, kScanSmemPerWarp * (kThreads / 32), st>>>(p);
         ADACOMP_LAUNCH_CHECK();
-        k_bracket_resolve<<<n_inst, kThreads, 0, st>>>(p);
+        ADACOMP_CUDA(mark(2));
+        k_bracket_resolve<<<n_inst, kBig, 0, st>>>(p);
         ADACOMP_LAUNCH_CHECK();
+        ADACOMP_CUDA(mark(3));
         k_bracket_emit<<<grid, kThreads, 0, st>>>(p);
         ADACOMP_LAUNCH_CHECK();
     }
+    ADACOMP_CUDA(mark(4));
 
     // general route for whatever is flagged for it (tensors not on the bracketed route, and
     // instances whose bracket missed); the kernels find an empty list otherwise
@@ -268,17 +294,50 @@ int adacomp_select(adacomp_select_t* h, const float* d_grads, uint64_t worker_st
     const unsigned grid = static_cast<unsigned>(grid64);
     k_general_plan<<<1, kThreads, 0, st>>>(p);
     ADACOMP_LAUNCH_CHECK();
+    ADACOMP_CUDA(mark(5));
     k_general_hist<0><<<grid, kThreads, 0, st>>>(p);
     ADACOMP_LAUNCH_CHECK();
+    ADACOMP_CUDA(mark(6));
     k_general_hist<1><<<grid, kThreads, 0, st>>>(p);
     ADACOMP_LAUNCH_CHECK();
+    ADACOMP_CUDA(mark(7));
     k_general_hist<2><<<grid, kThreads, 0, st>>>(p);
     ADACOMP_LAUNCH_CHECK();
+    ADACOMP_CUDA(mark(8));
     k_general_count<<<grid, kThreads, 0, st>>>(p);
     ADACOMP_LAUNCH_CHECK();
+    ADACOMP_CUDA(mark(9));
     k_general_write<<<grid, kThreads, 0, st>>>(p);
     ADACOMP_LAUNCH_CHECK();
+    ADACOMP_CUDA(mark(10));
     return ADACOMP_OK;
+}
+
+int adacomp_select_set_profiling(adacomp_select_t* h, int on) {
+    if (!h) return ADACOMP_ERR_INVALID;
+    DeviceGuard guard(h->device);
+    if (guard.err != cudaSuccess) return cuda_fail(guard.err);
+    if (on && !h->ev[0])
+        for (int i = 0; i <= kSelectStages; ++i) ADACOMP_CUDA(cudaEventCreate(&h->ev[i]));
+    h->profiling = on != 0;
+    return ADACOMP_OK;
+}
+
+int adacomp_select_profile(adacomp_select_t* h, float* h_ms_out, uint32_t n_stages) {
+    if (!h || !h_ms_out || n_stages != kSelectStages || !h->ev[0]) return ADACOMP_ERR_INVALID;
+    DeviceGuard guard(h->device);
+    if (guard.err != cudaSuccess) return cuda_fail(guard.err);
+    for (int i = 0; i < kSelectStages; ++i) {
+        h_ms_out[i] = 0.0f;
+        if (!h->ev_recorded[i] || !h->ev_recorded[i + 1]) continue;
+        ADACOMP_CUDA(cudaEventSynchronize(h->ev[i + 1]));
+        ADACOMP_CUDA(cudaEventElapsedTime(&h_ms_out[i], h->ev[i], h->ev[i + 1]));
+    }
+    return ADACOMP_OK;
+}
+
+const char* adacomp_select_stage_name(uint32_t stage) {
+    return stage < kSelectStages ? kStageNames[stage] : "";
 }
 
 int adacomp_select_host(adacomp_select_t* h, const float* h_grads, uint64_t worker_stride_elems,
@@ -326,6 +385,10 @@ int adacomp_select_last_error(adacomp_select_t* h, void* cuda_stream, uint64_t* 
 }
 
 int adacomp_select_destroy(adacomp_select_t* h) {
+    if (h && h->ev[0]) {
+        DeviceGuard guard(h->device);
+        for (int i = 0; i <= kSelectStages; ++i) cudaEventDestroy(h->ev[i]);
+    }
     delete h;
     return ADACOMP_OK;
 }

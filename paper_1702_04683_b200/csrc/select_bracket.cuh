@@ -5,18 +5,19 @@
 //   k_bracket_sample   per (worker, tensor): read a stratified sample, take two of its order
 //                      statistics t_lo <= t_hi chosen so that, with overwhelming probability,
 //                      #{key > t_hi} <= k <= #{key >= t_lo};
-//   k_bracket_scan     the single pass over the gradient: every entry with key >= t_lo (a
-//                      "candidate", about 1.1-2.5 k of them) is appended, in index order span by
-//                      span, to the instance's candidate list; candidates with key <= t_hi (the
-//                      "window", where the threshold must lie) are also appended to a small
-//                      unordered list; per span the pass records where its candidates went and
-//                      how many entries are above the window;
+//   k_bracket_scan     the single pass over the gradient.  Every warp works on its own: it
+//                      classifies 1024 consecutive entries, reserves room with one 64-bit atomic
+//                      and appends, in index order, the entries with key >= t_lo ("candidates",
+//                      about 1.1-2.5 k of them per tensor) to the instance's candidate list;
+//                      candidates with key <= t_hi (the "window", where the threshold must lie)
+//                      also go to a small unordered list; a table records where each 1024-entry
+//                      piece put its candidates and how many of them are above the window;
 //   k_bracket_resolve  per instance: verify the bracket with the exact counts, find the exact
 //                      threshold inside the window (radix select on (key, index) composites,
 //                      finished by brute force once few entries remain), count the kept window
 //                      entries per span and turn the per-span kept counts into output offsets;
-//   k_bracket_emit     per span: read its candidates, keep those at or above the exact threshold,
-//                      write them to the output in index order.
+//   k_bracket_emit     per span (8 pieces), one warp: read its candidates, keep those at or above
+//                      the exact threshold, write them to the output in index order.
 // The result is exact whatever the sample looked like: if the exact counts contradict the
 // bracket, or a list overflows its capacity, the instance is handed to the general route.
 // No kernel waits on another block; all cross-block traffic is atomics plus kernel boundaries.
@@ -26,15 +27,17 @@
 
 namespace adacomp {
 
-constexpr uint32_t kSpanElems = 8192;                 // entries per span (one block iteration)
-constexpr uint32_t kSpanVecs = kSpanElems / 4;
+constexpr uint32_t kSubElems = 1024;                  // entries one warp classifies at a time
+constexpr uint32_t kSubsPerSpan = 8;
+constexpr uint32_t kSpanElems = kSubElems * kSubsPerSpan;   // 8192: unit of the output-offset prefix
 constexpr uint32_t kSpansPerBlock = 8;                // scan: consecutive spans per block; emit: one per warp
 constexpr uint32_t kMaxSpans = 4096;                  // per tensor on this route (n <= 33.5 M)
 constexpr uint32_t kBracketMinN = 32768;
 constexpr uint32_t kSampleMax = 16384;
 constexpr uint32_t kSampleMin = 2048;
 constexpr float kBracketZ = 5.0f;                     // half-width of the bracket in sample standard deviations
-constexpr uint32_t kGatherMax = 512;
+constexpr uint32_t kGatherMax = 1024;
+constexpr int kBig = 1024;                            // threads of the per-instance kernels
 
 constexpr uint32_t kInstBracket = 2u;                 // bracket valid, scan/emit act on the instance
 constexpr uint32_t kInstOverflow = 4u;                // a candidate or window list ran out of room
@@ -55,19 +58,18 @@ __device__ __forceinline__ uint32_t hash32(uint32_t x) {
     return x;
 }
 
-// Descending walk over a histogram in shared memory: the bucket holding the rem-th largest.
-// All kThreads threads call; results are returned to all.  NB must be a multiple of kThreads.
-template <int NB>
+// Descending walk over a 2048-bin histogram in shared memory: the bucket holding the rem-th
+// largest.  All kBig threads call; results are returned to all.
 __device__ __forceinline__ void block_pick_bucket(const uint32_t* hist, uint32_t rem, uint32_t* bucket,
                                                   uint32_t* above_out, uint32_t* count_out,
-                                                  uint32_t* s_warp, uint32_t* s_bc /*[3]*/) {
-    constexpr int M = NB / kThreads;
-    const int top = NB - 1 - static_cast<int>(threadIdx.x) * M;
+                                                  uint32_t* s_warp /*[33]*/, uint32_t* s_bc /*[3]*/) {
+    constexpr int M = 2048 / kBig;
+    const int top = 2047 - static_cast<int>(threadIdx.x) * M;
     uint32_t h[M], sum = 0;
 #pragma unroll
     for (int q = 0; q < M; ++q) { h[q] = hist[top - q]; sum += h[q]; }
     uint32_t total;
-    uint32_t above = block_exclusive_scan(sum, &total, s_warp);
+    uint32_t above = block_exclusive_scan_t<kBig>(sum, &total, s_warp);
 #pragma unroll
     for (int q = 0; q < M; ++q) {
         if (above < rem && rem <= above + h[q]) { s_bc[0] = top - q; s_bc[1] = above; s_bc[2] = h[q]; }
@@ -86,16 +88,16 @@ __device__ uint32_t smem_kth_largest(const uint32_t* keys, uint32_t m, uint32_t 
     for (int pass = 0; pass < 3; ++pass) {
         const int shift = pass == 0 ? 20 : (pass == 1 ? 10 : 0);
         const int nb = pass == 0 ? 2048 : 1024;
-        for (int b = threadIdx.x; b < 2048; b += kThreads) hist[b] = 0;
+        for (int b = threadIdx.x; b < 2048; b += kBig) hist[b] = 0;
         __syncthreads();
-        for (uint32_t i = threadIdx.x; i < m; i += kThreads) {
+        for (uint32_t i = threadIdx.x; i < m; i += kBig) {
             const uint32_t key = keys[i];
             const bool match = pass == 0 || (key >> (shift + 10)) == (prefix >> (shift + 10));
             if (match) atomicAdd(&hist[(key >> shift) & (nb - 1)], 1u);
         }
         __syncthreads();
         uint32_t b, above, cnt;
-        block_pick_bucket<2048>(hist, rem, &b, &above, &cnt, s_warp, s_bc);   // unused upper bins are zero
+        block_pick_bucket(hist, rem, &b, &above, &cnt, s_warp, s_bc);   // unused upper bins are zero
         prefix |= b << shift;
         rem -= above;
     }
@@ -105,10 +107,10 @@ __device__ uint32_t smem_kth_largest(const uint32_t* keys, uint32_t m, uint32_t 
 // ---------------------------------------------------------------------------------------------
 // One block per (worker, tensor): reset the instance, and bracket its threshold if it is on
 // this route.  Dynamic shared memory: the sample keys.
-__global__ void __launch_bounds__(kThreads) k_bracket_sample(SelectParams p, int general_only) {
+__global__ void __launch_bounds__(kBig) k_bracket_sample(SelectParams p, int general_only) {
     extern __shared__ uint32_t s_keys[];
     __shared__ uint32_t s_hist[2048];
-    __shared__ uint32_t s_warp[9];
+    __shared__ uint32_t s_warp[33];
     __shared__ uint32_t s_bc[3];
     const uint32_t inst = blockIdx.x;
     const uint32_t w = inst / p.n_layers, l = inst - w * p.n_layers;
@@ -120,9 +122,13 @@ __global__ void __launch_bounds__(kThreads) k_bracket_sample(SelectParams p, int
         st->flags = bracket ? 0u : (L.k > 0 ? kInstGeneral : 0u);
 #pragma unroll
         for (int q = 0; q < 5; ++q) st->done[q] = 0;
-        st->cand_count = 0; st->win_count = 0; st->n_def = 0; st->T = 0; st->cut = 0;
+        st->cand_count = 0; st->win_count = 0; st->T = 0; st->cut = 0;
     }
     if (!bracket) return;
+    {   // the scan only writes the table entries of pieces that hold candidates
+        uint2* sub_tab = p.sub_tab + (static_cast<uint64_t>(w) * p.span_stride + L.span_base) * kSubsPerSpan;
+        for (uint32_t t = threadIdx.x; t < L.n_spans * kSubsPerSpan; t += kBig) sub_tab[t] = make_uint2(0u, 0u);
+    }
 
     const float* first = p.grads + static_cast<uint64_t>(w) * p.stride + L.offset;
     const uint32_t mis = static_cast<uint32_t>((reinterpret_cast<uintptr_t>(first) >> 2) & 3u);
@@ -130,7 +136,7 @@ __global__ void __launch_bounds__(kThreads) k_bracket_sample(SelectParams p, int
     const uint32_t m = L.sample, n_chunks = m / 32, stratum = L.n / n_chunks;   // stratum >= 128
     // chunk j: 32 consecutive entries starting at a hashed position inside stratum j, moved up to
     // the next 32-byte boundary; always inside the tensor
-    for (uint32_t t = threadIdx.x; t < n_chunks * 8; t += kThreads) {
+    for (uint32_t t = threadIdx.x; t < n_chunks * 8; t += kBig) {
         const uint32_t j = t >> 3, part = t & 7;
         const uint32_t e = j * stratum + hash32(j * 2654435761u + l * 40503u + 977u) % (stratum - 40);
         const uint32_t s = (e + mis + 7) & ~7u;                  // shifted coordinate, multiple of 8
@@ -147,140 +153,219 @@ __global__ void __launch_bounds__(kThreads) k_bracket_sample(SelectParams p, int
         return;
     }
     const uint32_t t_lo = smem_kth_largest(s_keys, m, r_lo, s_hist, s_warp, s_bc);
-    const uint32_t t_hi = r_hi ? smem_kth_largest(s_keys, m, r_hi, s_hist, s_warp, s_bc) : 0x7FFFFFFFu;
-    if (threadIdx.x == 0) { st->t_lo = t_lo; st->t_hi = t_hi; st->flags = kInstBracket; }
+    uint32_t t_hi = r_hi ? smem_kth_largest(s_keys, m, r_hi, s_hist, s_warp, s_bc) : 0x7FFFFFFFu;
+    if (t_hi > 0x7F800000u) t_hi = 0x7FFFFFFFu;       // "no upper bound" (as a float: unordered)
+    // the scan compares magnitudes as floats and blanks padding with zeros: it needs a positive,
+    // non-NaN lower bound
+    const bool usable = t_lo != 0 && t_lo <= 0x7F800000u;
+    if (threadIdx.x == 0) { st->t_lo = t_lo; st->t_hi = t_hi; st->flags = usable ? kInstBracket : kInstGeneral; }
 }
 
 // ---------------------------------------------------------------------------------------------
+// max(a, b) that returns NaN if either input is NaN (fmaxf would drop the NaN).
+__device__ __forceinline__ float max_nan(float a, float b) {
+    float r;
+    asm("max.NaN.f32 %0, %1, %2;" : "=f"(r) : "f"(a), "f"(b));
+    return r;
+}
+
 // The single pass over the gradient.  grid = (scan items, workers); an item is up to
-// kSpansPerBlock consecutive spans of one tensor.  Each warp holds 1024 consecutive entries of a
-// span in registers (8 coalesced float4 loads), so candidates come out in index order.
-__global__ void __launch_bounds__(kThreads) k_bracket_scan(SelectParams p) {
-    __shared__ uint32_t s_tot[kThreads / 32];
-    __shared__ uint32_t s_base[2];
-    __shared__ uint32_t s_over;
+// kSpansPerBlock consecutive spans of one tensor = 64 pieces of 1024 entries, and each of the 8
+// warps of a block takes 8 of them (round robin), entirely on its own: no block-level barrier.
+// A warp reads a piece with 8 coalesced float4 loads per lane, so index order is (piece, load,
+// lane, component).
+//   Streaming phase (small, branch-light code).  The four magnitudes of a load are reduced to
+//   their maximum and compared once with t_lo (for non-NaN data |x| >= t as floats is the integer
+//   test on the key; a NaN propagates through the maximum and counts as a hit).  Loads that hit
+//   are queued, in index order, in the warp's slice of shared memory (one ballot per load).  As
+//   soon as a load has been tested its registers are refilled with the same load of the warp's
+//   next piece, so a warp always has 4 KB in flight.
+//   Tail, once per 8 pieces, with work proportional to the queued loads.  Pass A fetches the
+//   queued loads again (an L1 / L2 hit), classifies their entries with bounds checks and counts
+//   candidates and window entries per piece; one 64-bit atomic then reserves room for all 8
+//   pieces; pass B ranks the queue with warp scans and writes candidates (in index order) and
+//   window entries.  The first and last piece of a tensor are not streamed: all their loads are
+//   queued.  A NaN hands the instance to the general route, which works on bit patterns only.
+constexpr uint32_t kScanQueue = 2048;                          // queued loads per warp: 8 pieces x 256
+constexpr size_t kScanSmemPerWarp = kScanQueue * 3 + 64;       // u16 queue + u8 info + 8 piece counters
+
+__device__ __forceinline__ bool load_hits(const float4& x, float tlo_f) {
+    const float m4 = max_nan(max_nan(fabsf(x.x), fabsf(x.y)), max_nan(fabsf(x.z), fabsf(x.w)));
+    return !(m4 < tlo_f);
+}
+
+__global__ void __launch_bounds__(kThreads, 4) k_bracket_scan(SelectParams p) {
+    extern __shared__ __align__(16) unsigned char s_scan[];
     const uint2 item = p.items[blockIdx.x];
     const uint32_t l = item.x, w = blockIdx.y;
     const Layer L = p.layers[l];
     Inst* st = &p.inst[w * p.n_layers + l];
     if (!(__ldcg(&st->flags) & kInstBracket)) return;
-    const uint32_t t_lo = __ldcg(&st->t_lo), t_hi = __ldcg(&st->t_hi);
+    const uint32_t t_hi = __ldcg(&st->t_hi);
+    const float tlo_f = __uint_as_float(__ldcg(&st->t_lo)), thi_f = __uint_as_float(t_hi);
     const float* first = p.grads + static_cast<uint64_t>(w) * p.stride + L.offset;
     const uint32_t mis = static_cast<uint32_t>((reinterpret_cast<uintptr_t>(first) >> 2) & 3u);
     const float4* vec = reinterpret_cast<const float4*>(first - mis);
-    const uint32_t n_shift = L.n + mis;                        // n <= 2^31 on this route
+    const uint32_t n_shift = L.n + mis;                        // n <= 33.5 M on this route
     const uint32_t nvec = (n_shift + 3) >> 2;
+    const uint32_t lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const uint32_t lt = (1u << lane) - 1u;
+    constexpr uint32_t kStep = kThreads / 32;                  // pieces between two pieces of one warp
+    constexpr uint32_t kBatch = kSpansPerBlock * kSubsPerSpan / kStep;   // pieces per warp: 8
+    const uint32_t ss_end = min(item.y + kSpansPerBlock, L.n_spans) * kSubsPerSpan;
+    const uint32_t ss0 = item.y * kSubsPerSpan + warp;         // this warp's pieces: ss0 + kStep * j
+    if (ss0 >= ss_end) return;
+    // pieces [in_lo, in_hi) lie entirely inside the tensor: no bounds checks needed
+    const uint32_t in_lo = mis ? 1u : 0u, in_hi = n_shift / kSubElems;
+    unsigned char* mine = s_scan + warp * kScanSmemPerWarp;
+    uint16_t* q = reinterpret_cast<uint16_t*>(mine);           // queued load: j * 256 + i * 32 + lane
+    unsigned char* info = mine + kScanQueue * 2;               // its candidate nibble | window nibble << 4
+    uint32_t* s_cnt = reinterpret_cast<uint32_t*>(mine + kScanQueue * 3);   // per piece: candidates | window << 16
+    if (lane < kBatch) s_cnt[lane] = 0;
+
+    // ---- streaming phase
+    uint32_t qn = 0;                                           // queued loads (warp-uniform)
+    float4 x[8];
+    bool loaded = false;
+    if (ss0 >= in_lo && ss0 < in_hi) {
+        const float4* ptr = vec + ss0 * (kSubElems / 4) + lane;
+#pragma unroll
+        for (int i = 0; i < 8; ++i) x[i] = __ldg(ptr + i * 32);
+        loaded = true;
+    }
+#pragma unroll 1
+    for (uint32_t j = 0; j < kBatch; ++j) {
+        const uint32_t ss = ss0 + kStep * j, next = ss + kStep;
+        if (ss >= ss_end) break;
+        const bool next_inside = (j + 1 < kBatch) && next < ss_end && next >= in_lo && next < in_hi;
+        const float4* nptr = vec + (next_inside ? next : ss0) * (kSubElems / 4) + lane;   // ss0: any valid address
+        if (loaded) {
+#pragma unroll
+            for (int i = 0; i < 8; ++i) {
+                const bool h = load_hits(x[i], tlo_f);
+                const uint32_t b = __ballot_sync(0xFFFFFFFFu, h);
+                if (b) {
+                    if (h) q[qn + __popc(b & lt)] = static_cast<uint16_t>(j * 256 + i * 32 + lane);
+                    qn += __popc(b);
+                }
+                if (next_inside) x[i] = __ldg(nptr + i * 32);
+            }
+        } else {                                               // a piece at the tensor's ends: queue every load
+#pragma unroll
+            for (int i = 0; i < 8; ++i) {
+                q[qn + i * 32 + lane] = static_cast<uint16_t>(j * 256 + i * 32 + lane);
+                if (next_inside) x[i] = __ldg(nptr + i * 32);
+            }
+            qn += 256;
+        }
+        loaded = next_inside;
+    }
+    __syncwarp();
+    if (!qn) return;                                           // the table entries stay (0, 0)
+
+    // ---- tail, pass A: classify the queued loads, count per piece
+    bool saw_nan = false;
+    for (uint32_t t = lane; t < qn; t += 32) {
+        const uint32_t ent = q[t];
+        const uint32_t j = ent >> 8;
+        const uint32_t v = (ss0 + kStep * j) * (kSubElems / 4) + (ent & 255u);
+        const float4 y = (v < nvec) ? __ldg(&vec[v]) : make_float4(0.f, 0.f, 0.f, 0.f);
+        const float ys[4] = {y.x, y.y, y.z, y.w};
+        uint32_t nc = 0, nw = 0;
+#pragma unroll
+        for (int c4 = 0; c4 < 4; ++c4) {
+            const uint32_t e = v * 4 + c4;
+            const float a = fabsf(ys[c4]);
+            const bool cand = (e >= mis && e < n_shift) && !(a < tlo_f);
+            saw_nan |= cand && (a != a);
+            if (cand) nc |= 1u << c4;
+            if (cand && !(a > thi_f)) nw |= 1u << c4;
+        }
+        info[t] = static_cast<unsigned char>(nc | (nw << 4));
+        if (nc) atomicAdd(&s_cnt[j], __popc(nc) | (__popc(nw) << 16));
+    }
+    if (saw_nan) atomicOr(&st->flags, kInstOverflow);
+    __syncwarp();
+    // totals and per-piece first slots (lanes 0..7 hold one piece each)
+    const uint32_t mycnt = lane < kBatch ? s_cnt[lane] : 0u;
+    uint32_t inc = mycnt;
+#pragma unroll
+    for (int d = 1; d < static_cast<int>(kBatch); d <<= 1) {
+        const uint32_t y = __shfl_up_sync(0xFFFFFFFFu, inc, d);
+        if (lane >= static_cast<uint32_t>(d)) inc += y;
+    }
+    const uint32_t tot = __shfl_sync(0xFFFFFFFFu, inc, kBatch - 1);
+    const uint32_t total_c = tot & 0xFFFFu, total_w = tot >> 16;
+    if (!total_c) return;
+    unsigned long long old = 0;
+    if (lane == 0)                                             // one reservation for the 8 pieces
+        old = atomicAdd(reinterpret_cast<unsigned long long*>(&st->cand_count),
+                        static_cast<unsigned long long>(total_c) | (static_cast<unsigned long long>(total_w) << 32));
+    old = __shfl_sync(0xFFFFFFFFu, old, 0);
+    const uint32_t cb = static_cast<uint32_t>(old), wb = static_cast<uint32_t>(old >> 32);
+    if ((static_cast<uint64_t>(cb) + total_c > L.cand_cap) || (static_cast<uint64_t>(wb) + total_w > L.win_cap)) {
+        if (lane == 0) atomicOr(&st->flags, kInstOverflow);
+        return;
+    }
+    if (lane < kBatch && (mycnt & 0xFFFFu)) {
+        const uint32_t tc = mycnt & 0xFFFFu, tw = mycnt >> 16;
+        p.sub_tab[(static_cast<uint64_t>(w) * p.span_stride + L.span_base) * kSubsPerSpan + ss0 + kStep * lane] =
+            make_uint2(cb + ((inc - mycnt) & 0xFFFFu), tc | ((tc - tw) << 16));
+    }
+
+    // ---- tail, pass B: rank the queue, write the lists
     uint32_t* cand_idx = p.cand_idx + static_cast<uint64_t>(w) * p.cand_stride + L.cand_base;
     float* cand_val = p.cand_val + static_cast<uint64_t>(w) * p.cand_stride + L.cand_base;
     uint32_t* win_key = p.win_key + static_cast<uint64_t>(w) * p.win_stride + L.win_base;
     uint32_t* win_idx = p.win_idx + static_cast<uint64_t>(w) * p.win_stride + L.win_base;
-    uint2* span_tab = p.span_tab + static_cast<uint64_t>(w) * p.span_stride + L.span_base;
-    const uint32_t lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-    const uint32_t lt = (1u << lane) - 1u;
-    const uint32_t s_end = min(item.y + kSpansPerBlock, L.n_spans);
-
-    for (uint32_t s = item.y; s < s_end; ++s) {
-        const uint32_t vec0 = s * kSpanVecs + warp * 256;
-        const bool full = (s * kSpanElems >= mis) && ((s + 1) * kSpanElems <= n_shift);
-        float4 x[8];
-#pragma unroll
-        for (int i = 0; i < 8; ++i) {
-            const uint32_t v = vec0 + i * 32 + lane;
-            x[i] = (v < nvec) ? __ldcs(&vec[v]) : make_float4(0.f, 0.f, 0.f, 0.f);
+    uint32_t run = cb | (static_cast<uint32_t>(0) << 0), wrun = wb;
+    for (uint32_t t0 = 0; t0 < qn; t0 += 32) {
+        const uint32_t t = t0 + lane;
+        uint32_t nc = 0, nw = 0, v = 0;
+        if (t < qn) {
+            const uint32_t ent = q[t], inf = info[t];
+            nc = inf & 15u;
+            nw = inf >> 4;
+            v = (ss0 + kStep * (ent >> 8)) * (kSubElems / 4) + (ent & 255u);
         }
-        // pass A: classify; one bit per held entry
-        uint32_t mask_c = 0, mask_w = 0;
+        const uint32_t cnt = __popc(nc) | (__popc(nw) << 16);
+        uint32_t sc = cnt;
 #pragma unroll
-        for (int i = 0; i < 8; ++i) {
-            const float xs[4] = {x[i].x, x[i].y, x[i].z, x[i].w};
-            const uint32_t e0 = (vec0 + i * 32 + lane) * 4;
-#pragma unroll
-            for (int q = 0; q < 4; ++q) {
-                const uint32_t key = magnitude_key(xs[q]);
-                const bool ok = full || (e0 + q >= mis && e0 + q < n_shift);
-                const bool c = ok && key >= t_lo;
-                mask_c |= (c ? 1u : 0u) << (i * 4 + q);
-                mask_w |= ((c && key <= t_hi) ? 1u : 0u) << (i * 4 + q);
-            }
+        for (int d = 1; d < 32; d <<= 1) {
+            const uint32_t y = __shfl_up_sync(0xFFFFFFFFu, sc, d);
+            if (lane >= static_cast<uint32_t>(d)) sc += y;
         }
-        const uint32_t cw = __popc(mask_w);
-        const uint32_t tc = __reduce_add_sync(0xFFFFFFFFu, __popc(mask_c));
-        const uint32_t tw = __reduce_add_sync(0xFFFFFFFFu, cw);
-        if (lane == 0) s_tot[warp] = tc | (tw << 16);
-        __syncthreads();
-        uint32_t pc = 0, pw = 0, totc = 0, totw = 0;
+        const uint32_t tot32 = __shfl_sync(0xFFFFFFFFu, sc, 31);
+        if (nc) {
+            uint32_t pos = run + ((sc - cnt) & 0xFFFFu), wpos = wrun + ((sc - cnt) >> 16);
+            const float4 y = __ldg(&vec[v]);                     // nc != 0 implies v < nvec
+            const float ys[4] = {y.x, y.y, y.z, y.w};
 #pragma unroll
-        for (int ww = 0; ww < kThreads / 32; ++ww) {
-            const uint32_t t = s_tot[ww];
-            if (ww < warp) { pc += t & 0xFFFFu; pw += t >> 16; }
-            totc += t & 0xFFFFu; totw += t >> 16;
-        }
-        if (threadIdx.x == 0) {
-            const uint32_t cb = totc ? atomicAdd(&st->cand_count, totc) : 0u;
-            const uint32_t wb = totw ? atomicAdd(&st->win_count, totw) : 0u;
-            const uint32_t ndef = totc - totw;
-            if (ndef) atomicAdd(&st->n_def, ndef);
-            const bool over = (static_cast<uint64_t>(cb) + totc > L.cand_cap) || (static_cast<uint64_t>(wb) + totw > L.win_cap);
-            if (over) atomicOr(&st->flags, kInstOverflow);
-            s_base[0] = cb; s_base[1] = wb; s_over = over ? 1u : 0u;
-            span_tab[s] = make_uint2(cb, totc | (ndef << 16));
-        }
-        __syncthreads();
-        const uint32_t cb = s_base[0], wb = s_base[1];
-        const bool over = s_over != 0;
-        if (!over && tc > 0) {
-            // pass B: positions.  Candidates in index order = (load i, lane, component q).
-            uint32_t wpos = 0;
-            if (tw > 0) {                                  // window: any order, lane-major
-                uint32_t inc = cw;
-#pragma unroll
-                for (int d = 1; d < 32; d <<= 1) {
-                    const uint32_t y = __shfl_up_sync(0xFFFFFFFFu, inc, d);
-                    if (lane >= d) inc += y;
-                }
-                wpos = wb + pw + inc - cw;
-            }
-            uint32_t running = cb + pc;
-#pragma unroll
-            for (int i = 0; i < 8; ++i) {
-                const uint32_t m4 = (mask_c >> (i * 4)) & 15u;
-                if (!__any_sync(0xFFFFFFFFu, m4 != 0)) continue;
-                const uint32_t c4 = __popc(m4);
-                const uint32_t b0 = __ballot_sync(0xFFFFFFFFu, c4 & 1u);
-                const uint32_t b1 = __ballot_sync(0xFFFFFFFFu, c4 & 2u);
-                const uint32_t b2 = __ballot_sync(0xFFFFFFFFu, c4 & 4u);
-                uint32_t pos = running + __popc(b0 & lt) + 2 * __popc(b1 & lt) + 4 * __popc(b2 & lt);
-                running += __popc(b0) + 2 * __popc(b1) + 4 * __popc(b2);
-                if (m4) {
-                    const float xs[4] = {x[i].x, x[i].y, x[i].z, x[i].w};
-                    const uint32_t e0 = (vec0 + i * 32 + lane) * 4;
-                    const uint32_t w4 = (mask_w >> (i * 4)) & 15u;
-#pragma unroll
-                    for (int q = 0; q < 4; ++q) {
-                        if ((m4 >> q) & 1u) {
-                            cand_idx[pos] = e0 + q;            // shifted coordinate inside the tensor
-                            cand_val[pos] = xs[q];
-                            ++pos;
-                            if ((w4 >> q) & 1u) {
-                                win_key[wpos] = magnitude_key(xs[q]);
-                                win_idx[wpos] = e0 + q;
-                                ++wpos;
-                            }
-                        }
+            for (int c4 = 0; c4 < 4; ++c4) {
+                if ((nc >> c4) & 1u) {
+                    cand_idx[pos] = v * 4 + c4;                  // shifted coordinate inside the tensor
+                    cand_val[pos] = ys[c4];
+                    ++pos;
+                    if ((nw >> c4) & 1u) {
+                        win_key[wpos] = magnitude_key(ys[c4]);
+                        win_idx[wpos] = v * 4 + c4;
+                        ++wpos;
                     }
                 }
             }
         }
+        run += tot32 & 0xFFFFu;
+        wrun += tot32 >> 16;
     }
 }
 
 // ---------------------------------------------------------------------------------------------
 // One block per instance: exact threshold inside the window, per-span output offsets.
-__global__ void __launch_bounds__(kThreads) k_bracket_resolve(SelectParams p) {
+__global__ void __launch_bounds__(kBig) k_bracket_resolve(SelectParams p) {
     __shared__ uint32_t s_hist[2048];
     __shared__ uint32_t s_sel[kMaxSpans];
     __shared__ unsigned long long s_g[kGatherMax];
-    __shared__ uint32_t s_warp[9];
+    __shared__ uint32_t s_warp[33];
     __shared__ uint32_t s_bc[3];
     __shared__ uint32_t s_cnt;
     __shared__ unsigned long long s_cstar;
@@ -291,7 +376,8 @@ __global__ void __launch_bounds__(kThreads) k_bracket_resolve(SelectParams p) {
     Inst* st = &p.inst[inst];
     const uint32_t flags = __ldcg(&st->flags);
     if (!(flags & kInstBracket)) return;
-    const uint32_t n_cand = __ldcg(&st->cand_count), n_win = __ldcg(&st->win_count), n_def = __ldcg(&st->n_def);
+    const uint32_t n_cand = __ldcg(&st->cand_count), n_win = __ldcg(&st->win_count);
+    const uint32_t n_def = n_cand - n_win;            // entries above the window
     const uint32_t t_lo = __ldcg(&st->t_lo), t_hi = __ldcg(&st->t_hi);
     const bool bad = (flags & kInstOverflow) || n_cand > L.cand_cap || n_win > L.win_cap || n_def > L.k ||
                      L.k - n_def > n_win;
@@ -301,7 +387,7 @@ __global__ void __launch_bounds__(kThreads) k_bracket_resolve(SelectParams p) {
     }
     const uint32_t* win_key = p.win_key + static_cast<uint64_t>(w) * p.win_stride + L.win_base;
     const uint32_t* win_idx = p.win_idx + static_cast<uint64_t>(w) * p.win_stride + L.win_base;
-    uint2* span_tab = p.span_tab + static_cast<uint64_t>(w) * p.span_stride + L.span_base;
+    const uint2* sub_tab = p.sub_tab + (static_cast<uint64_t>(w) * p.span_stride + L.span_base) * kSubsPerSpan;
     uint32_t* span_off = p.span_off + static_cast<uint64_t>(w) * p.span_stride + L.span_base;
     const uint32_t need = L.k - n_def;
 
@@ -314,20 +400,20 @@ __global__ void __launch_bounds__(kThreads) k_bracket_resolve(SelectParams p) {
     unsigned long long cstar = ~0ull;                 // keep window entries with composite >= cstar
     if (need > 0) {
         const uint32_t range = t_hi - t_lo;
-        int hi_shift = (range ? 32 - __clz(range) : 0) + 32;   // undecided low bits of the composite
+        int hi_shift = (range ? 32 - __clz(range) : 0) + 32;   // undecided low bits of the composite (<= 63)
         unsigned long long prefix = 0;
         uint32_t rem = need, count = n_win;
         while (true) {
             if (count <= kGatherMax) {                // few left: gather them and rank by brute force
                 if (threadIdx.x == 0) s_cnt = 0;
                 __syncthreads();
-                for (uint32_t i = threadIdx.x; i < n_win; i += kThreads) {
+                for (uint32_t i = threadIdx.x; i < n_win; i += kBig) {
                     const unsigned long long c = composite(i);
-                    if (hi_shift >= 64 || (c >> hi_shift) == prefix) s_g[atomicAdd(&s_cnt, 1u)] = c;
+                    if ((c >> hi_shift) == prefix) s_g[atomicAdd(&s_cnt, 1u)] = c;
                 }
                 __syncthreads();
-                for (uint32_t t = threadIdx.x; t < count; t += kThreads) {
-                    const unsigned long long mine = s_g[t];
+                if (threadIdx.x < count) {
+                    const unsigned long long mine = s_g[threadIdx.x];
                     uint32_t larger = 0;
                     for (uint32_t u = 0; u < count; ++u) larger += s_g[u] > mine ? 1u : 0u;
                     if (larger == rem - 1) s_cstar = mine;
@@ -339,16 +425,16 @@ __global__ void __launch_bounds__(kThreads) k_bracket_resolve(SelectParams p) {
             if (hi_shift == 0) { cstar = prefix; break; }     // cannot happen: composites are distinct
             const int bits = hi_shift < 11 ? hi_shift : 11;
             const int new_shift = hi_shift - bits;
-            for (int b = threadIdx.x; b < 2048; b += kThreads) s_hist[b] = 0;
+            for (int b = threadIdx.x; b < 2048; b += kBig) s_hist[b] = 0;
             __syncthreads();
-            for (uint32_t i = threadIdx.x; i < n_win; i += kThreads) {
+            for (uint32_t i = threadIdx.x; i < n_win; i += kBig) {
                 const unsigned long long c = composite(i);
-                if (hi_shift >= 64 || (c >> hi_shift) == prefix)
+                if ((c >> hi_shift) == prefix)
                     atomicAdd(&s_hist[static_cast<uint32_t>(c >> new_shift) & ((1u << bits) - 1u)], 1u);
             }
             __syncthreads();
             uint32_t b, above, cnt;
-            block_pick_bucket<2048>(s_hist, rem, &b, &above, &cnt, s_warp, s_bc);
+            block_pick_bucket(s_hist, rem, &b, &above, &cnt, s_warp, s_bc);
             prefix = (prefix << bits) | b;
             rem -= above;
             count = cnt;
@@ -356,21 +442,25 @@ __global__ void __launch_bounds__(kThreads) k_bracket_resolve(SelectParams p) {
         }
     }
     // kept window entries per span
-    for (uint32_t s = threadIdx.x; s < L.n_spans; s += kThreads) s_sel[s] = 0;
+    for (uint32_t s = threadIdx.x; s < L.n_spans; s += kBig) s_sel[s] = 0;
     if (threadIdx.x == 0) s_carry = 0;
     __syncthreads();
     if (need > 0) {
-        for (uint32_t i = threadIdx.x; i < n_win; i += kThreads)
+        for (uint32_t i = threadIdx.x; i < n_win; i += kBig)
             if (composite(i) >= cstar) atomicAdd(&s_sel[__ldcg(&win_idx[i]) / kSpanElems], 1u);
     }
     __syncthreads();
     // exclusive prefix of kept entries over the spans
-    for (uint32_t base = 0; base < L.n_spans; base += kThreads) {
+    for (uint32_t base = 0; base < L.n_spans; base += kBig) {
         const uint32_t s = base + threadIdx.x;
         uint32_t kept = 0;
-        if (s < L.n_spans) kept = (__ldcg(&span_tab[s]).y >> 16) + s_sel[s];
+        if (s < L.n_spans) {
+            kept = s_sel[s];
+#pragma unroll
+            for (uint32_t j = 0; j < kSubsPerSpan; ++j) kept += __ldcg(&sub_tab[s * kSubsPerSpan + j]).y >> 16;
+        }
         uint32_t tot;
-        const uint32_t ex = block_exclusive_scan(kept, &tot, s_warp);
+        const uint32_t ex = block_exclusive_scan_t<kBig>(kept, &tot, s_warp);
         const uint32_t carry = s_carry;
         if (s < L.n_spans) span_off[s] = carry + ex;
         __syncthreads();
@@ -391,7 +481,8 @@ __global__ void __launch_bounds__(kThreads) k_bracket_resolve(SelectParams p) {
 }
 
 // ---------------------------------------------------------------------------------------------
-// grid = (scan items, workers); one warp per span: filter its candidates, write in order.
+// grid = (scan items, workers); one warp per span: walk the candidates of its 8 pieces in index
+// order, keep those at or above the exact threshold, write them out contiguously.
 __global__ void __launch_bounds__(kThreads) k_bracket_emit(SelectParams p) {
     const uint2 item = p.items[blockIdx.x];
     const uint32_t l = item.x, w = blockIdx.y;
@@ -406,20 +497,38 @@ __global__ void __launch_bounds__(kThreads) k_bracket_emit(SelectParams p) {
     const uint32_t mis = static_cast<uint32_t>((reinterpret_cast<uintptr_t>(first) >> 2) & 3u);
     const uint32_t* cand_idx = p.cand_idx + static_cast<uint64_t>(w) * p.cand_stride + L.cand_base;
     const float* cand_val = p.cand_val + static_cast<uint64_t>(w) * p.cand_stride + L.cand_base;
-    const uint2 tab = __ldcg(&p.span_tab[static_cast<uint64_t>(w) * p.span_stride + L.span_base + s]);
+    const uint64_t span_at = static_cast<uint64_t>(w) * p.span_stride + L.span_base + s;
+    uint2 tab = make_uint2(0, 0);
+    if (lane < kSubsPerSpan) tab = __ldcg(&p.sub_tab[span_at * kSubsPerSpan + lane]);
     const uint32_t cnt = tab.y & 0xFFFFu;
-    uint32_t off = __ldcg(&p.span_off[static_cast<uint64_t>(w) * p.span_stride + L.span_base + s]);
+    uint32_t inc = cnt;                                        // inclusive prefix over the 8 pieces
+#pragma unroll
+    for (int d = 1; d < 8; d <<= 1) {
+        const uint32_t y = __shfl_up_sync(0xFFFFFFFFu, inc, d);
+        if (lane >= d) inc += y;
+    }
+    const uint32_t pre = inc - cnt;
+    const uint32_t total = __shfl_sync(0xFFFFFFFFu, inc, kSubsPerSpan - 1);
+    uint32_t off = __ldcg(&p.span_off[span_at]);
     uint32_t* idx_out = p.idx_out + static_cast<uint64_t>(w) * p.K + L.out_offset;
     float* val_out = p.val_out + static_cast<uint64_t>(w) * p.K + L.out_offset;
     const uint32_t lt = (1u << lane) - 1u;
     const uint32_t glob = static_cast<uint32_t>(L.offset) - mis;        // shifted coordinate -> vector index
-    for (uint32_t c = lane; c < ((cnt + 31) & ~31u); c += 32) {
+    for (uint32_t f = lane; f < ((total + 31) & ~31u); f += 32) {
+        uint32_t at = 0;
+#pragma unroll
+        for (int j = 0; j < static_cast<int>(kSubsPerSpan); ++j) {
+            const uint32_t pj = __shfl_sync(0xFFFFFFFFu, pre, j);
+            const uint32_t cj = __shfl_sync(0xFFFFFFFFu, cnt, j);
+            const uint32_t bj = __shfl_sync(0xFFFFFFFFu, tab.x, j);
+            if (f >= pj && f < pj + cj) at = bj + (f - pj);
+        }
         bool keep = false;
         uint32_t e = 0;
         float v = 0.f;
-        if (c < cnt) {
-            e = __ldcs(&cand_idx[tab.x + c]);
-            v = __ldcs(&cand_val[tab.x + c]);
+        if (f < total) {
+            e = __ldcs(&cand_idx[at]);
+            v = __ldcs(&cand_val[at]);
             const uint32_t key = magnitude_key(v);
             keep = key > T || (key == T && e < cut);
         }

@@ -14,6 +14,8 @@
 // serve "all instances" and "only the instances another route gave up on".
 #pragma once
 
+#include <cstddef>
+
 #include "common.cuh"
 
 namespace adacomp {
@@ -48,13 +50,16 @@ struct Inst {             // selection state of one (worker, tensor)
     uint32_t flags;       // route bookkeeping (kInstGeneral ...)
     uint32_t done[5];     // finished chunks per pass
     // bracketed route
-    uint32_t t_lo, t_hi;  // the threshold key lies in [t_lo, t_hi]
-    uint32_t cand_count;  // entries with key >= t_lo appended so far
-    uint32_t win_count;   // of those, entries with key <= t_hi
-    uint32_t n_def;       // entries with key > t_hi
+    uint32_t t_lo;        // the threshold key lies in [t_lo, t_hi]
+    uint32_t cand_count;  // entries with key >= t_lo appended so far   } one 8-byte word, advanced
+    uint32_t win_count;   // of those, entries with key <= t_hi         } by a single 64-bit atomic
+    uint32_t t_hi;
+    uint32_t spare;
     uint32_t T, cut;      // exact threshold: keep key > T, and key == T with shifted index < cut
 };
 static_assert(sizeof(Inst) == 64, "Inst is one 64-byte record");
+static_assert(offsetof(Inst, cand_count) % 8 == 0 && offsetof(Inst, win_count) == offsetof(Inst, cand_count) + 4,
+              "cand_count / win_count form one aligned 64-bit word");
 constexpr uint32_t kInstGeneral = 1u;   // instance is (to be) handled by the general route
 
 struct SelectParams {
@@ -79,7 +84,7 @@ struct SelectParams {
     float* cand_val;            //                        its value
     uint32_t* win_key;          // [worker][win_stride] key of each window entry
     uint32_t* win_idx;          //                       its shifted index
-    uint2* span_tab;            // [worker][span_stride] (first candidate slot, count | above-window count << 16)
+    uint2* sub_tab;             // [worker][span_stride * 8] per 1024-entry piece: (first candidate slot, count | above-window count << 16)
     uint32_t* span_off;         // [worker][span_stride] kept entries before the span
     uint64_t cand_stride, win_stride, span_stride;
 };
@@ -107,6 +112,37 @@ __device__ __forceinline__ uint32_t block_exclusive_scan(uint32_t v, uint32_t* t
     }
     *total = tot;
     return base + inc - v;
+}
+
+// The same for any block size that is a multiple of 32 (up to 1024): warp scans, then a scan of
+// the warp totals by the first warp.  s_warp needs 33 entries.
+template <int THREADS>
+__device__ __forceinline__ uint32_t block_exclusive_scan_t(uint32_t v, uint32_t* total, uint32_t* s_warp /*[33]*/) {
+    constexpr int WARPS = THREADS / 32;
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    uint32_t inc = v;
+#pragma unroll
+    for (int d = 1; d < 32; d <<= 1) {
+        uint32_t y = __shfl_up_sync(0xFFFFFFFFu, inc, d);
+        if (lane >= d) inc += y;
+    }
+    __syncthreads();
+    if (lane == 31) s_warp[warp] = inc;
+    __syncthreads();
+    if (warp == 0) {
+        const uint32_t t = lane < WARPS ? s_warp[lane] : 0u;
+        uint32_t winc = t;
+#pragma unroll
+        for (int d = 1; d < 32; d <<= 1) {
+            uint32_t y = __shfl_up_sync(0xFFFFFFFFu, winc, d);
+            if (lane >= d) winc += y;
+        }
+        if (lane < WARPS) s_warp[lane] = winc - t;       // exclusive prefix of the warp totals
+        if (lane == 31) s_warp[32] = winc;               // block total
+    }
+    __syncthreads();
+    *total = s_warp[32];
+    return s_warp[warp] + inc - v;
 }
 
 // Geometry of one work item: a chunk of an instance, in "shifted" coordinates that start at the
