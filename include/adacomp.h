@@ -134,12 +134,15 @@ ADACOMP_API int adacomp_select_host(adacomp_select_t* h, const float* h_grads, u
 ADACOMP_API int adacomp_select_set_route(adacomp_select_t* h, int route);
 
 /* Stage timing.  With profiling on, every adacomp_select call records CUDA events on its stream
- * around each of its kernels (a few microseconds of overhead per call).  adacomp_select_profile
- * waits for the last call and writes the device time of each stage in milliseconds to
- * h_ms_out[0 .. n_stages), n_stages = 10 (0 for a stage the call did not run);
+ * around each of its kernels (a few microseconds of host work per call, no synchronisation).
+ * adacomp_select_profile waits for the calls made since profiling was switched on and writes
+ * the mean device time per call of each stage, in milliseconds, to h_ms_out[0 .. n_stages),
+ * n_stages = 10 (0 for a stage that never ran), and the number of calls to *h_calls_out (may be
+ * NULL).  Switching profiling on (again) starts a fresh measurement.
  * adacomp_select_stage_name names a stage ("bracket_scan", ...; "" beyond the last). */
 ADACOMP_API int adacomp_select_set_profiling(adacomp_select_t* h, int on);
-ADACOMP_API int adacomp_select_profile(adacomp_select_t* h, float* h_ms_out, uint32_t n_stages);
+ADACOMP_API int adacomp_select_profile(adacomp_select_t* h, float* h_ms_out, uint32_t n_stages,
+                                       uint64_t* h_calls_out);
 ADACOMP_API const char* adacomp_select_stage_name(uint32_t stage);
 
 /* K = sum of k over the layout's segments (pairs per worker). */

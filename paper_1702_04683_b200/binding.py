@@ -57,7 +57,7 @@ def _load():
         "adacomp_select_host": (i32, [vp, vp, u64, u32, vp, vp, vp, vp, vp, vp]),
         "adacomp_select_set_route": (i32, [vp, i32]),
         "adacomp_select_set_profiling": (i32, [vp, i32]),
-        "adacomp_select_profile": (i32, [vp, P(f32), u32]),
+        "adacomp_select_profile": (i32, [vp, P(f32), u32, P(u64)]),
         "adacomp_select_stage_name": (ctypes.c_char_p, [u32]),
         "adacomp_select_pairs_per_worker": (i32, [vp, P(u64)]),
         "adacomp_select_last_error": (i32, [vp, vp, P(u64)]),
@@ -214,10 +214,13 @@ class Selector:
         _check(_lib.adacomp_select_set_profiling(self._h, int(on)), "adacomp_select_set_profiling")
 
     def profile(self) -> dict:
-        """Device milliseconds per kernel of the last select call (profiling must be on)."""
+        """Mean device milliseconds per kernel and call since profiling was switched on."""
         ms = (ctypes.c_float * 10)()
-        _check(_lib.adacomp_select_profile(self._h, ms, 10), "adacomp_select_profile")
-        return {_lib.adacomp_select_stage_name(i).decode(): float(ms[i]) for i in range(10)}
+        calls = ctypes.c_uint64(0)
+        _check(_lib.adacomp_select_profile(self._h, ms, 10, ctypes.byref(calls)), "adacomp_select_profile")
+        out = {_lib.adacomp_select_stage_name(i).decode(): float(ms[i]) for i in range(10)}
+        out["calls"] = int(calls.value)
+        return out
 
     def last_error(self, stream: Optional[torch.cuda.Stream] = None) -> Tuple[int, int]:
         """(status, selections that took the general route in the last call); waits for the stream."""

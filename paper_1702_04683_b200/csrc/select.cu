@@ -10,6 +10,7 @@ using namespace adacomp;
 
 namespace {
 constexpr int kSelectStages = 10;
+constexpr int kProfileRing = 32;
 const char* const kStageNames[kSelectStages] = {
     "bracket_sample", "bracket_scan", "bracket_resolve", "bracket_emit", "general_plan",
     "general_hist0", "general_hist1", "general_hist2", "general_count", "general_write"};
@@ -19,6 +20,7 @@ struct adacomp_select {
     int device = 0;
     int n_sms = 0;
     int route = 0;         // 0 = automatic, 1 = general route for everything
+    bool all_bracketed = false;   // every tensor with k > 0 is eligible for the bracketed route
     uint32_t n_layers = 0, max_workers = 0, slots_per_worker = 0, n_items = 0, max_sample = 0;
     uint64_t extent = 0;   // one past the last entry any segment covers
     uint64_t K = 0;        // pairs per worker
@@ -40,9 +42,14 @@ struct adacomp_select {
     uint2* d_sub_tab = nullptr;
     uint32_t* d_span_off = nullptr;
     // optional stage timing: events around every kernel of the last call
+    // optional stage timing: a ring of event sets, one per call, folded into sums when reused or read
     bool profiling = false;
-    cudaEvent_t ev[kSelectStages + 1] = {};
-    bool ev_recorded[kSelectStages + 1] = {};
+    cudaEvent_t ev[kProfileRing][kSelectStages + 1] = {};
+    bool ev_recorded[kProfileRing][kSelectStages + 1] = {};
+    bool ring_used[kProfileRing] = {};
+    int ring_next = 0;
+    double stage_ms_sum[kSelectStages] = {};
+    uint64_t profiled_calls = 0;
 };
 
 namespace {
@@ -151,6 +158,23 @@ size_t carve(adacomp_select_t* h, void* base, const Layout& lay, uint32_t max_wo
     return c.used;
 }
 
+// Adds the stage times of one finished (or finishing: waits for it) event set to the sums.
+cudaError_t fold_profile_slot(adacomp_select_t* h, int slot) {
+    if (!h->ring_used[slot]) return cudaSuccess;
+    for (int i = 0; i < kSelectStages; ++i) {
+        if (!h->ev_recorded[slot][i] || !h->ev_recorded[slot][i + 1]) continue;
+        cudaError_t e = cudaEventSynchronize(h->ev[slot][i + 1]);
+        if (e != cudaSuccess) return e;
+        float ms = 0.f;
+        e = cudaEventElapsedTime(&ms, h->ev[slot][i], h->ev[slot][i + 1]);
+        if (e != cudaSuccess) return e;
+        h->stage_ms_sum[i] += ms;
+    }
+    h->ring_used[slot] = false;
+    h->profiled_calls += 1;
+    return cudaSuccess;
+}
+
 }  // namespace
 
 extern "C" {
@@ -185,6 +209,9 @@ int adacomp_select_create(adacomp_select_t** h, const adacomp_segment_t* h_segs,
     s->extent = lay.extent;
     s->K = lay.K;
     s->n_items = static_cast<uint32_t>(lay.items.size());
+    s->all_bracketed = true;
+    for (const Layer& L : lay.layers)
+        if (L.k > 0 && !L.bracket) s->all_bracketed = false;
     s->max_sample = lay.max_sample;
     s->cand_stride = lay.cand_stride;
     s->win_stride = lay.win_stride;
@@ -259,12 +286,19 @@ int adacomp_select(adacomp_select_t* h, const float* d_grads, uint64_t worker_st
 
     const unsigned n_inst = n_workers * h->n_layers;
     const bool bracketed = h->route == 0 && h->n_items > 0;
-    for (int i = 0; i <= kSelectStages; ++i) h->ev_recorded[i] = false;
+    int slot = 0;
+    if (h->profiling) {                                   // take the next event set of the ring
+        slot = h->ring_next;
+        h->ring_next = (h->ring_next + 1) % kProfileRing;
+        ADACOMP_CUDA(fold_profile_slot(h, slot));         // its previous user finished long ago
+        for (int i = 0; i <= kSelectStages; ++i) h->ev_recorded[slot][i] = false;
+        h->ring_used[slot] = true;
+    }
     // mark(i): the boundary before stage i (and after stage i - 1)
     auto mark = [&](int i) -> cudaError_t {
         if (!h->profiling) return cudaSuccess;
-        h->ev_recorded[i] = true;
-        return cudaEventRecord(h->ev[i], st);
+        h->ev_recorded[slot][i] = true;
+        return cudaEventRecord(h->ev[slot][i], st);
     };
     ADACOMP_CUDA(mark(0));
 
@@ -288,7 +322,9 @@ int adacomp_select(adacomp_select_t* h, const float* d_grads, uint64_t worker_st
     // general route for whatever is flagged for it (tensors not on the bracketed route, and
     // instances whose bracket missed); the kernels find an empty list otherwise
     const uint64_t total_slots = static_cast<uint64_t>(h->slots_per_worker) * n_workers;
-    uint64_t grid64 = static_cast<uint64_t>(h->n_sms) * 8;
+    // when every tensor is on the bracketed route the general kernels almost always find an empty
+    // list: keep their grid small then (a rare miss still gets one block per SM and chunk)
+    uint64_t grid64 = static_cast<uint64_t>(h->n_sms) * (bracketed && h->all_bracketed ? 1 : 8);
     if (grid64 > total_slots) grid64 = total_slots;
     if (grid64 == 0) grid64 = 1;
     const unsigned grid = static_cast<unsigned>(grid64);
@@ -317,22 +353,24 @@ int adacomp_select_set_profiling(adacomp_select_t* h, int on) {
     if (!h) return ADACOMP_ERR_INVALID;
     DeviceGuard guard(h->device);
     if (guard.err != cudaSuccess) return cuda_fail(guard.err);
-    if (on && !h->ev[0])
-        for (int i = 0; i <= kSelectStages; ++i) ADACOMP_CUDA(cudaEventCreate(&h->ev[i]));
+    if (on && !h->ev[0][0])
+        for (int r = 0; r < kProfileRing; ++r)
+            for (int i = 0; i <= kSelectStages; ++i) ADACOMP_CUDA(cudaEventCreate(&h->ev[r][i]));
+    for (int r = 0; r < kProfileRing; ++r) ADACOMP_CUDA(fold_profile_slot(h, r));
+    for (int i = 0; i < kSelectStages; ++i) h->stage_ms_sum[i] = 0.0;      // a fresh measurement starts here
+    h->profiled_calls = 0;
     h->profiling = on != 0;
     return ADACOMP_OK;
 }
 
-int adacomp_select_profile(adacomp_select_t* h, float* h_ms_out, uint32_t n_stages) {
-    if (!h || !h_ms_out || n_stages != kSelectStages || !h->ev[0]) return ADACOMP_ERR_INVALID;
+int adacomp_select_profile(adacomp_select_t* h, float* h_ms_out, uint32_t n_stages, uint64_t* h_calls_out) {
+    if (!h || !h_ms_out || n_stages != kSelectStages || !h->ev[0][0]) return ADACOMP_ERR_INVALID;
     DeviceGuard guard(h->device);
     if (guard.err != cudaSuccess) return cuda_fail(guard.err);
-    for (int i = 0; i < kSelectStages; ++i) {
-        h_ms_out[i] = 0.0f;
-        if (!h->ev_recorded[i] || !h->ev_recorded[i + 1]) continue;
-        ADACOMP_CUDA(cudaEventSynchronize(h->ev[i + 1]));
-        ADACOMP_CUDA(cudaEventElapsedTime(&h_ms_out[i], h->ev[i], h->ev[i + 1]));
-    }
+    for (int r = 0; r < kProfileRing; ++r) ADACOMP_CUDA(fold_profile_slot(h, r));
+    for (int i = 0; i < kSelectStages; ++i)
+        h_ms_out[i] = h->profiled_calls ? static_cast<float>(h->stage_ms_sum[i] / static_cast<double>(h->profiled_calls)) : 0.0f;
+    if (h_calls_out) *h_calls_out = h->profiled_calls;
     return ADACOMP_OK;
 }
 
@@ -385,9 +423,10 @@ int adacomp_select_last_error(adacomp_select_t* h, void* cuda_stream, uint64_t* 
 }
 
 int adacomp_select_destroy(adacomp_select_t* h) {
-    if (h && h->ev[0]) {
+    if (h && h->ev[0][0]) {
         DeviceGuard guard(h->device);
-        for (int i = 0; i <= kSelectStages; ++i) cudaEventDestroy(h->ev[i]);
+        for (int r = 0; r < kProfileRing; ++r)
+            for (int i = 0; i <= kSelectStages; ++i) cudaEventDestroy(h->ev[r][i]);
     }
     delete h;
     return ADACOMP_OK;

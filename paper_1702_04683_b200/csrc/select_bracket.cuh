@@ -174,20 +174,23 @@ __device__ __forceinline__ float max_nan(float a, float b) {
 // warps of a block takes 8 of them (round robin), entirely on its own: no block-level barrier.
 // A warp reads a piece with 8 coalesced float4 loads per lane, so index order is (piece, load,
 // lane, component).
-//   Streaming phase (small, branch-light code).  The four magnitudes of a load are reduced to
-//   their maximum and compared once with t_lo (for non-NaN data |x| >= t as floats is the integer
-//   test on the key; a NaN propagates through the maximum and counts as a hit).  Loads that hit
-//   are queued, in index order, in the warp's slice of shared memory (one ballot per load).  As
-//   soon as a load has been tested its registers are refilled with the same load of the warp's
-//   next piece, so a warp always has 4 KB in flight.
-//   Tail, once per 8 pieces, with work proportional to the queued loads.  Pass A fetches the
-//   queued loads again (an L1 / L2 hit), classifies their entries with bounds checks and counts
-//   candidates and window entries per piece; one 64-bit atomic then reserves room for all 8
-//   pieces; pass B ranks the queue with warp scans and writes candidates (in index order) and
-//   window entries.  The first and last piece of a tensor are not streamed: all their loads are
-//   queued.  A NaN hands the instance to the general route, which works on bit patterns only.
-constexpr uint32_t kScanQueue = 2048;                          // queued loads per warp: 8 pieces x 256
-constexpr size_t kScanSmemPerWarp = kScanQueue * 3 + 64;       // u16 queue + u8 info + 8 piece counters
+//   Streaming.  The four magnitudes of a load are reduced to their maximum and compared once
+//   with t_lo (for non-NaN data |x| >= t as floats is the integer test on the key; a NaN
+//   propagates through the maximum and counts as a hit).  One ballot per load tells the warp
+//   whether any lane hit; only then do the hitting lanes classify their four entries and queue
+//   the load (its position and two 4-bit masks: candidates, window) in the warp's slice of
+//   shared memory, in index order.  As soon as a load has been tested its registers are refilled
+//   with the same load of the warp's next piece, so a warp always has 4 KB in flight.
+//   Tail, once per round (up to 8 pieces, fewer when the queue fills), with work proportional to
+//   the queued loads.  One 64-bit atomic reserves room in both lists for the whole round; the
+//   queue is then ranked with warp scans, the queued loads are fetched again (an L1 / L2 hit),
+//   and candidates and window entries are staged in shared memory and copied out with coalesced
+//   stores.
+// The first and last piece of a tensor use checked loads.  A NaN hands the instance to the
+// general route, which works on bit patterns only.
+constexpr uint32_t kScanQueue = 768;                           // queued loads per warp and round
+constexpr uint32_t kScanStage = 128;                           // entries staged per copy step (32 loads x 4)
+constexpr size_t kScanSmemPerWarp = kScanQueue * 3 + 32 + kScanStage * 16;
 
 __device__ __forceinline__ bool load_hits(const float4& x, float tlo_f) {
     const float m4 = max_nan(max_nan(fabsf(x.x), fabsf(x.y)), max_nan(fabsf(x.z), fabsf(x.w)));
@@ -218,145 +221,163 @@ __global__ void __launch_bounds__(kThreads, 4) k_bracket_scan(SelectParams p) {
     // pieces [in_lo, in_hi) lie entirely inside the tensor: no bounds checks needed
     const uint32_t in_lo = mis ? 1u : 0u, in_hi = n_shift / kSubElems;
     unsigned char* mine = s_scan + warp * kScanSmemPerWarp;
-    uint16_t* q = reinterpret_cast<uint16_t*>(mine);           // queued load: j * 256 + i * 32 + lane
-    unsigned char* info = mine + kScanQueue * 2;               // its candidate nibble | window nibble << 4
-    uint32_t* s_cnt = reinterpret_cast<uint32_t*>(mine + kScanQueue * 3);   // per piece: candidates | window << 16
-    if (lane < kBatch) s_cnt[lane] = 0;
+    uint32_t* stage_idx = reinterpret_cast<uint32_t*>(mine);                        // [kScanStage]
+    float* stage_val = reinterpret_cast<float*>(mine + kScanStage * 4);             // [kScanStage]
+    uint32_t* stage_widx = reinterpret_cast<uint32_t*>(mine + kScanStage * 8);      // [kScanStage]
+    uint32_t* stage_wkey = reinterpret_cast<uint32_t*>(mine + kScanStage * 12);     // [kScanStage]
+    uint32_t* s_cnt = reinterpret_cast<uint32_t*>(mine + kScanStage * 16);          // [8] per piece: cand | win << 16
+    uint16_t* q = reinterpret_cast<uint16_t*>(mine + kScanStage * 16 + 32);         // queued load: j * 256 + i * 32 + lane
+    unsigned char* info = mine + kScanStage * 16 + 32 + kScanQueue * 2;             // candidate nibble | window nibble << 4
+    uint32_t* cand_idx = p.cand_idx + static_cast<uint64_t>(w) * p.cand_stride + L.cand_base;
+    float* cand_val = p.cand_val + static_cast<uint64_t>(w) * p.cand_stride + L.cand_base;
+    uint32_t* win_key = p.win_key + static_cast<uint64_t>(w) * p.win_stride + L.win_base;
+    uint32_t* win_idx = p.win_idx + static_cast<uint64_t>(w) * p.win_stride + L.win_base;
 
-    // ---- streaming phase
-    uint32_t qn = 0;                                           // queued loads (warp-uniform)
     float4 x[8];
-    bool loaded = false;
+    bool loaded = false;                                       // x holds the piece about to be tested
     if (ss0 >= in_lo && ss0 < in_hi) {
         const float4* ptr = vec + ss0 * (kSubElems / 4) + lane;
 #pragma unroll
         for (int i = 0; i < 8; ++i) x[i] = __ldg(ptr + i * 32);
         loaded = true;
     }
+    bool saw_nan = false;
+    uint32_t j = 0;
+    while (j < kBatch && ss0 + kStep * j < ss_end) {
+        // ================= one round: stream pieces until the queue could overflow
+        uint32_t qn = 0;                                       // queued loads (warp-uniform)
+        if (lane < kBatch) s_cnt[lane] = 0;
+        __syncwarp();
 #pragma unroll 1
-    for (uint32_t j = 0; j < kBatch; ++j) {
-        const uint32_t ss = ss0 + kStep * j, next = ss + kStep;
-        if (ss >= ss_end) break;
-        const bool next_inside = (j + 1 < kBatch) && next < ss_end && next >= in_lo && next < in_hi;
-        const float4* nptr = vec + (next_inside ? next : ss0) * (kSubElems / 4) + lane;   // ss0: any valid address
-        if (loaded) {
+        for (; j < kBatch && qn + 256 <= kScanQueue; ++j) {
+            const uint32_t ss = ss0 + kStep * j, next = ss + kStep;
+            if (ss >= ss_end) break;
+            const bool next_inside = (j + 1 < kBatch) && next < ss_end && next >= in_lo && next < in_hi;
+            const float4* nptr = vec + (next_inside ? next : ss0) * (kSubElems / 4) + lane;   // ss0: any valid address
+            uint32_t pcnt = 0;                                 // this lane's candidates | window << 16 in the piece
 #pragma unroll
             for (int i = 0; i < 8; ++i) {
-                const bool h = load_hits(x[i], tlo_f);
+                float4 y;
+                bool h;
+                if (loaded) {
+                    y = x[i];
+                    h = load_hits(y, tlo_f);
+                } else {                                       // a piece at the tensor's ends: checked load, blank outside
+                    const uint32_t v = ss * (kSubElems / 4) + i * 32 + lane;
+                    y = (v < nvec) ? __ldg(&vec[v]) : make_float4(0.f, 0.f, 0.f, 0.f);
+                    float* ys = reinterpret_cast<float*>(&y);
+#pragma unroll
+                    for (int c4 = 0; c4 < 4; ++c4)
+                        if (v * 4 + c4 < mis || v * 4 + c4 >= n_shift) ys[c4] = 0.f;    // t_lo > 0: never a candidate
+                    h = load_hits(y, tlo_f);
+                }
                 const uint32_t b = __ballot_sync(0xFFFFFFFFu, h);
                 if (b) {
-                    if (h) q[qn + __popc(b & lt)] = static_cast<uint16_t>(j * 256 + i * 32 + lane);
+                    if (h) {
+                        const float ys[4] = {y.x, y.y, y.z, y.w};
+                        uint32_t nc = 0, nw = 0;
+#pragma unroll
+                        for (int c4 = 0; c4 < 4; ++c4) {
+                            const float a = fabsf(ys[c4]);
+                            const bool cand = !(a < tlo_f);
+                            saw_nan |= a != a;
+                            if (cand) nc |= 1u << c4;
+                            if (cand && !(a > thi_f)) nw |= 1u << c4;
+                        }
+                        const uint32_t slot = qn + __popc(b & lt);
+                        q[slot] = static_cast<uint16_t>(j * 256 + i * 32 + lane);
+                        info[slot] = static_cast<unsigned char>(nc | (nw << 4));
+                        pcnt += __popc(nc) | (__popc(nw) << 16);
+                    }
                     qn += __popc(b);
                 }
                 if (next_inside) x[i] = __ldg(nptr + i * 32);
             }
-        } else {                                               // a piece at the tensor's ends: queue every load
+            loaded = next_inside;
+            const uint32_t ptot = __reduce_add_sync(0xFFFFFFFFu, pcnt);
+            if (lane == 0) s_cnt[j] = ptot;
+        }
+        __syncwarp();
+        if (!qn) continue;                                     // the table entries stay (0, 0)
+
+        // ================= tail: reserve once for the round, then rank and write
+        const uint32_t mycnt = lane < kBatch ? s_cnt[lane] : 0u;
+        uint32_t inc = mycnt;
 #pragma unroll
-            for (int i = 0; i < 8; ++i) {
-                q[qn + i * 32 + lane] = static_cast<uint16_t>(j * 256 + i * 32 + lane);
-                if (next_inside) x[i] = __ldg(nptr + i * 32);
+        for (int d = 1; d < static_cast<int>(kBatch); d <<= 1) {
+            const uint32_t y = __shfl_up_sync(0xFFFFFFFFu, inc, d);
+            if (lane >= static_cast<uint32_t>(d)) inc += y;
+        }
+        const uint32_t tot = __shfl_sync(0xFFFFFFFFu, inc, kBatch - 1);
+        const uint32_t total_c = tot & 0xFFFFu, total_w = tot >> 16;
+        if (!total_c) continue;
+        unsigned long long old = 0;
+        if (lane == 0)
+            old = atomicAdd(reinterpret_cast<unsigned long long*>(&st->cand_count),
+                            static_cast<unsigned long long>(total_c) | (static_cast<unsigned long long>(total_w) << 32));
+        old = __shfl_sync(0xFFFFFFFFu, old, 0);
+        const uint32_t cb = static_cast<uint32_t>(old), wb = static_cast<uint32_t>(old >> 32);
+        if ((static_cast<uint64_t>(cb) + total_c > L.cand_cap) || (static_cast<uint64_t>(wb) + total_w > L.win_cap)) {
+            if (lane == 0) atomicOr(&st->flags, kInstOverflow);
+            continue;
+        }
+        if (lane < kBatch && (mycnt & 0xFFFFu)) {
+            const uint32_t tc = mycnt & 0xFFFFu, tw = mycnt >> 16;
+            p.sub_tab[(static_cast<uint64_t>(w) * p.span_stride + L.span_base) * kSubsPerSpan + ss0 + kStep * lane] =
+                make_uint2(cb + ((inc - mycnt) & 0xFFFFu), tc | ((tc - tw) << 16));
+        }
+        uint32_t run = cb, wrun = wb;
+        for (uint32_t t0 = 0; t0 < qn; t0 += 32) {
+            const uint32_t t = t0 + lane;
+            uint32_t nc = 0, nw = 0, v = 0;
+            if (t < qn) {
+                const uint32_t ent = q[t], inf = info[t];
+                nc = inf & 15u;
+                nw = inf >> 4;
+                v = (ss0 + kStep * (ent >> 8)) * (kSubElems / 4) + (ent & 255u);
             }
-            qn += 256;
-        }
-        loaded = next_inside;
-    }
-    __syncwarp();
-    if (!qn) return;                                           // the table entries stay (0, 0)
-
-    // ---- tail, pass A: classify the queued loads, count per piece
-    bool saw_nan = false;
-    for (uint32_t t = lane; t < qn; t += 32) {
-        const uint32_t ent = q[t];
-        const uint32_t j = ent >> 8;
-        const uint32_t v = (ss0 + kStep * j) * (kSubElems / 4) + (ent & 255u);
-        const float4 y = (v < nvec) ? __ldg(&vec[v]) : make_float4(0.f, 0.f, 0.f, 0.f);
-        const float ys[4] = {y.x, y.y, y.z, y.w};
-        uint32_t nc = 0, nw = 0;
+            const uint32_t cnt = __popc(nc) | (__popc(nw) << 16);
+            uint32_t sc = cnt;
 #pragma unroll
-        for (int c4 = 0; c4 < 4; ++c4) {
-            const uint32_t e = v * 4 + c4;
-            const float a = fabsf(ys[c4]);
-            const bool cand = (e >= mis && e < n_shift) && !(a < tlo_f);
-            saw_nan |= cand && (a != a);
-            if (cand) nc |= 1u << c4;
-            if (cand && !(a > thi_f)) nw |= 1u << c4;
-        }
-        info[t] = static_cast<unsigned char>(nc | (nw << 4));
-        if (nc) atomicAdd(&s_cnt[j], __popc(nc) | (__popc(nw) << 16));
-    }
-    if (saw_nan) atomicOr(&st->flags, kInstOverflow);
-    __syncwarp();
-    // totals and per-piece first slots (lanes 0..7 hold one piece each)
-    const uint32_t mycnt = lane < kBatch ? s_cnt[lane] : 0u;
-    uint32_t inc = mycnt;
+            for (int d = 1; d < 32; d <<= 1) {
+                const uint32_t y = __shfl_up_sync(0xFFFFFFFFu, sc, d);
+                if (lane >= static_cast<uint32_t>(d)) sc += y;
+            }
+            const uint32_t tot32 = __shfl_sync(0xFFFFFFFFu, sc, 31);
+            if (nc) {
+                uint32_t r = (sc - cnt) & 0xFFFFu, wr = (sc - cnt) >> 16;
+                const float4 y = __ldg(&vec[v]);                 // queued loads lie inside the vector range
+                const float ys[4] = {y.x, y.y, y.z, y.w};
 #pragma unroll
-    for (int d = 1; d < static_cast<int>(kBatch); d <<= 1) {
-        const uint32_t y = __shfl_up_sync(0xFFFFFFFFu, inc, d);
-        if (lane >= static_cast<uint32_t>(d)) inc += y;
-    }
-    const uint32_t tot = __shfl_sync(0xFFFFFFFFu, inc, kBatch - 1);
-    const uint32_t total_c = tot & 0xFFFFu, total_w = tot >> 16;
-    if (!total_c) return;
-    unsigned long long old = 0;
-    if (lane == 0)                                             // one reservation for the 8 pieces
-        old = atomicAdd(reinterpret_cast<unsigned long long*>(&st->cand_count),
-                        static_cast<unsigned long long>(total_c) | (static_cast<unsigned long long>(total_w) << 32));
-    old = __shfl_sync(0xFFFFFFFFu, old, 0);
-    const uint32_t cb = static_cast<uint32_t>(old), wb = static_cast<uint32_t>(old >> 32);
-    if ((static_cast<uint64_t>(cb) + total_c > L.cand_cap) || (static_cast<uint64_t>(wb) + total_w > L.win_cap)) {
-        if (lane == 0) atomicOr(&st->flags, kInstOverflow);
-        return;
-    }
-    if (lane < kBatch && (mycnt & 0xFFFFu)) {
-        const uint32_t tc = mycnt & 0xFFFFu, tw = mycnt >> 16;
-        p.sub_tab[(static_cast<uint64_t>(w) * p.span_stride + L.span_base) * kSubsPerSpan + ss0 + kStep * lane] =
-            make_uint2(cb + ((inc - mycnt) & 0xFFFFu), tc | ((tc - tw) << 16));
-    }
-
-    // ---- tail, pass B: rank the queue, write the lists
-    uint32_t* cand_idx = p.cand_idx + static_cast<uint64_t>(w) * p.cand_stride + L.cand_base;
-    float* cand_val = p.cand_val + static_cast<uint64_t>(w) * p.cand_stride + L.cand_base;
-    uint32_t* win_key = p.win_key + static_cast<uint64_t>(w) * p.win_stride + L.win_base;
-    uint32_t* win_idx = p.win_idx + static_cast<uint64_t>(w) * p.win_stride + L.win_base;
-    uint32_t run = cb | (static_cast<uint32_t>(0) << 0), wrun = wb;
-    for (uint32_t t0 = 0; t0 < qn; t0 += 32) {
-        const uint32_t t = t0 + lane;
-        uint32_t nc = 0, nw = 0, v = 0;
-        if (t < qn) {
-            const uint32_t ent = q[t], inf = info[t];
-            nc = inf & 15u;
-            nw = inf >> 4;
-            v = (ss0 + kStep * (ent >> 8)) * (kSubElems / 4) + (ent & 255u);
-        }
-        const uint32_t cnt = __popc(nc) | (__popc(nw) << 16);
-        uint32_t sc = cnt;
-#pragma unroll
-        for (int d = 1; d < 32; d <<= 1) {
-            const uint32_t y = __shfl_up_sync(0xFFFFFFFFu, sc, d);
-            if (lane >= static_cast<uint32_t>(d)) sc += y;
-        }
-        const uint32_t tot32 = __shfl_sync(0xFFFFFFFFu, sc, 31);
-        if (nc) {
-            uint32_t pos = run + ((sc - cnt) & 0xFFFFu), wpos = wrun + ((sc - cnt) >> 16);
-            const float4 y = __ldg(&vec[v]);                     // nc != 0 implies v < nvec
-            const float ys[4] = {y.x, y.y, y.z, y.w};
-#pragma unroll
-            for (int c4 = 0; c4 < 4; ++c4) {
-                if ((nc >> c4) & 1u) {
-                    cand_idx[pos] = v * 4 + c4;                  // shifted coordinate inside the tensor
-                    cand_val[pos] = ys[c4];
-                    ++pos;
-                    if ((nw >> c4) & 1u) {
-                        win_key[wpos] = magnitude_key(ys[c4]);
-                        win_idx[wpos] = v * 4 + c4;
-                        ++wpos;
+                for (int c4 = 0; c4 < 4; ++c4) {
+                    if ((nc >> c4) & 1u) {
+                        stage_idx[r] = v * 4 + c4;               // shifted coordinate inside the tensor
+                        stage_val[r] = ys[c4];
+                        ++r;
+                        if ((nw >> c4) & 1u) {
+                            stage_widx[wr] = v * 4 + c4;
+                            stage_wkey[wr] = magnitude_key(ys[c4]);
+                            ++wr;
+                        }
                     }
                 }
             }
+            __syncwarp();
+            const uint32_t n_c = tot32 & 0xFFFFu, n_w = tot32 >> 16;
+            for (uint32_t r = lane; r < n_c; r += 32) {
+                cand_idx[run + r] = stage_idx[r];
+                cand_val[run + r] = stage_val[r];
+            }
+            for (uint32_t r = lane; r < n_w; r += 32) {
+                win_idx[wrun + r] = stage_widx[r];
+                win_key[wrun + r] = stage_wkey[r];
+            }
+            __syncwarp();
+            run += n_c;
+            wrun += n_w;
         }
-        run += tot32 & 0xFFFFu;
-        wrun += tot32 >> 16;
     }
+    if (saw_nan) atomicOr(&st->flags, kInstOverflow);
 }
 
 // ---------------------------------------------------------------------------------------------
@@ -391,10 +412,26 @@ __global__ void __launch_bounds__(kBig) k_bracket_resolve(SelectParams p) {
     uint32_t* span_off = p.span_off + static_cast<uint64_t>(w) * p.span_stride + L.span_base;
     const uint32_t need = L.k - n_def;
 
-    // composite of a window entry: larger = kept first (larger key, then lower index)
-    auto composite = [&](uint32_t i) -> unsigned long long {
-        return (static_cast<unsigned long long>(__ldcg(&win_key[i]) - t_lo) << 32) |
-               static_cast<unsigned long long>(0xFFFFFFFFu - __ldcg(&win_idx[i]));
+    // composite of a window entry = (key - t_lo) << 32 | ~index: larger = kept first (larger key,
+    // then lower index)
+    // calls fn(composite, shifted index) for every window entry; four entries per thread are
+    // fetched before any is used, so their loads overlap
+    auto for_each_window = [&](auto fn) {
+        for (uint32_t i0 = threadIdx.x; i0 < n_win; i0 += kBig * 4) {
+            uint32_t key[4], idx[4];
+#pragma unroll
+            for (int u = 0; u < 4; ++u) {
+                const uint32_t i = i0 + u * kBig;
+                key[u] = i < n_win ? __ldcg(&win_key[i]) : 0u;
+                idx[u] = i < n_win ? __ldcg(&win_idx[i]) : 0u;
+            }
+#pragma unroll
+            for (int u = 0; u < 4; ++u)
+                if (i0 + u * kBig < n_win)
+                    fn((static_cast<unsigned long long>(key[u] - t_lo) << 32) |
+                           static_cast<unsigned long long>(0xFFFFFFFFu - idx[u]),
+                       idx[u]);
+        }
     };
 
     unsigned long long cstar = ~0ull;                 // keep window entries with composite >= cstar
@@ -407,10 +444,9 @@ __global__ void __launch_bounds__(kBig) k_bracket_resolve(SelectParams p) {
             if (count <= kGatherMax) {                // few left: gather them and rank by brute force
                 if (threadIdx.x == 0) s_cnt = 0;
                 __syncthreads();
-                for (uint32_t i = threadIdx.x; i < n_win; i += kBig) {
-                    const unsigned long long c = composite(i);
+                for_each_window([&](unsigned long long c, uint32_t) {
                     if ((c >> hi_shift) == prefix) s_g[atomicAdd(&s_cnt, 1u)] = c;
-                }
+                });
                 __syncthreads();
                 if (threadIdx.x < count) {
                     const unsigned long long mine = s_g[threadIdx.x];
@@ -427,11 +463,10 @@ __global__ void __launch_bounds__(kBig) k_bracket_resolve(SelectParams p) {
             const int new_shift = hi_shift - bits;
             for (int b = threadIdx.x; b < 2048; b += kBig) s_hist[b] = 0;
             __syncthreads();
-            for (uint32_t i = threadIdx.x; i < n_win; i += kBig) {
-                const unsigned long long c = composite(i);
+            for_each_window([&](unsigned long long c, uint32_t) {
                 if ((c >> hi_shift) == prefix)
                     atomicAdd(&s_hist[static_cast<uint32_t>(c >> new_shift) & ((1u << bits) - 1u)], 1u);
-            }
+            });
             __syncthreads();
             uint32_t b, above, cnt;
             block_pick_bucket(s_hist, rem, &b, &above, &cnt, s_warp, s_bc);
@@ -446,8 +481,9 @@ __global__ void __launch_bounds__(kBig) k_bracket_resolve(SelectParams p) {
     if (threadIdx.x == 0) s_carry = 0;
     __syncthreads();
     if (need > 0) {
-        for (uint32_t i = threadIdx.x; i < n_win; i += kBig)
-            if (composite(i) >= cstar) atomicAdd(&s_sel[__ldcg(&win_idx[i]) / kSpanElems], 1u);
+        for_each_window([&](unsigned long long c, uint32_t idx) {
+            if (c >= cstar) atomicAdd(&s_sel[idx / kSpanElems], 1u);
+        });
     }
     __syncthreads();
     // exclusive prefix of kept entries over the spans
@@ -514,31 +550,44 @@ __global__ void __launch_bounds__(kThreads) k_bracket_emit(SelectParams p) {
     float* val_out = p.val_out + static_cast<uint64_t>(w) * p.K + L.out_offset;
     const uint32_t lt = (1u << lane) - 1u;
     const uint32_t glob = static_cast<uint32_t>(L.offset) - mis;        // shifted coordinate -> vector index
-    for (uint32_t f = lane; f < ((total + 31) & ~31u); f += 32) {
-        uint32_t at = 0;
+    // where each piece's candidates start in the span's flattened order (warp-uniform registers):
+    // flattened position f of piece j lives at slot f + delta[j]
+    uint32_t start[kSubsPerSpan], delta[kSubsPerSpan];
 #pragma unroll
-        for (int j = 0; j < static_cast<int>(kSubsPerSpan); ++j) {
-            const uint32_t pj = __shfl_sync(0xFFFFFFFFu, pre, j);
-            const uint32_t cj = __shfl_sync(0xFFFFFFFFu, cnt, j);
-            const uint32_t bj = __shfl_sync(0xFFFFFFFFu, tab.x, j);
-            if (f >= pj && f < pj + cj) at = bj + (f - pj);
+    for (int j = 0; j < static_cast<int>(kSubsPerSpan); ++j) {
+        start[j] = __shfl_sync(0xFFFFFFFFu, pre, j);
+        delta[j] = __shfl_sync(0xFFFFFFFFu, tab.x, j) - start[j];
+    }
+    constexpr int kUnroll = 4;                                 // 128 candidates in flight per warp
+    for (uint32_t f0 = 0; f0 < total; f0 += 32 * kUnroll) {
+        uint32_t e[kUnroll];
+        float v[kUnroll];
+#pragma unroll
+        for (int u = 0; u < kUnroll; ++u) {
+            const uint32_t f = f0 + u * 32 + lane;
+            uint32_t d = delta[0];
+#pragma unroll
+            for (int j = 1; j < static_cast<int>(kSubsPerSpan); ++j)
+                if (f >= start[j]) d = delta[j];               // starts never decrease: the last match wins
+            e[u] = 0;
+            v[u] = 0.f;
+            if (f < total) {
+                e[u] = __ldcs(&cand_idx[f + d]);
+                v[u] = __ldcs(&cand_val[f + d]);
+            }
         }
-        bool keep = false;
-        uint32_t e = 0;
-        float v = 0.f;
-        if (f < total) {
-            e = __ldcs(&cand_idx[at]);
-            v = __ldcs(&cand_val[at]);
-            const uint32_t key = magnitude_key(v);
-            keep = key > T || (key == T && e < cut);
+#pragma unroll
+        for (int u = 0; u < kUnroll; ++u) {
+            const uint32_t key = magnitude_key(v[u]);
+            const bool keep = (f0 + u * 32 + lane < total) && (key > T || (key == T && e[u] < cut));
+            const uint32_t b = __ballot_sync(0xFFFFFFFFu, keep);
+            if (keep) {
+                const uint32_t pos = off + __popc(b & lt);
+                idx_out[pos] = glob + e[u];
+                val_out[pos] = v[u];
+            }
+            off += __popc(b);
         }
-        const uint32_t b = __ballot_sync(0xFFFFFFFFu, keep);
-        if (keep) {
-            const uint32_t pos = off + __popc(b & lt);
-            idx_out[pos] = glob + e;
-            val_out[pos] = v;
-        }
-        off += __popc(b);
     }
 }
 
