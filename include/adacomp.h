@@ -154,6 +154,28 @@ ADACOMP_API int adacomp_select_pairs_per_worker(const adacomp_select_t* h, uint6
 ADACOMP_API int adacomp_select_last_error(adacomp_select_t* h, void* cuda_stream, uint64_t* stats_out);
 ADACOMP_API int adacomp_select_destroy(adacomp_select_t* h);
 
+/* Selection of ONE tensor for callers that cannot allocate device memory.  (The paper has no
+ * counterpart: this is a convenience of this library.)  Same rule and same output as
+ * adacomp_select for a single segment {offset 0, n, k} and a single worker: the k entries of
+ * largest magnitude of d_grad[0 .. n), lower index first among equals, written by ascending
+ * index to d_idx_out[0 .. k) / d_val_out[0 .. k).  No handle and no workspace: the scratch the
+ * selection needs (about 11 KB) is a fixed array inside the library, present on every GPU that
+ * loads it for as long as the process lives; the call allocates nothing, on the host or on the
+ * device, and frees nothing.  Meant for code that runs where an allocation is not an option:
+ * inside another framework's step whose memory pool it cannot reach, in a loop whose memory was
+ * budgeted at start-up, or while an allocation would stall or fail.
+ *   n <= 16 777 216 (2^24) entries; a larger n is refused with ADACOMP_ERR_CAPACITY and nothing
+ *   is enqueued.  k <= n; k = 0 does nothing.  d_grad must be 4-byte aligned.
+ *   The first call on a device looks up the array's device address (a CUDA runtime query, done
+ *   once per device with that device current); make that first call before any stream capture.
+ *   All calls on a device share the one array, which keeps whatever the previous call left
+ *   (every call clears what it needs zeroed): two calls whose device work overlaps, on two
+ *   streams or from two threads, race on it.  Keep calls on a device in one stream, or order
+ *   them with events.
+ * Work is enqueued on cuda_stream; the call returns without waiting. */
+ADACOMP_API int adacomp_select_static(const float* d_grad, uint32_t n, uint32_t k, uint32_t* d_idx_out,
+                                      float* d_val_out, int device, void* cuda_stream);
+
 /* ------------------------------------------------------------------------------------------
  * Server side: Algorithm 2 (Eq. 3, Eq. 4, Eq. 5; "Complexity" paragraph for the history).
  * ---------------------------------------------------------------------------------------- */

@@ -59,6 +59,7 @@ def _load():
         "adacomp_select_set_profiling": (i32, [vp, i32]),
         "adacomp_select_profile": (i32, [vp, P(f32), u32, P(u64)]),
         "adacomp_select_stage_name": (ctypes.c_char_p, [u32]),
+        "adacomp_select_static": (i32, [vp, u32, u32, vp, vp, i32, vp]),
         "adacomp_select_pairs_per_worker": (i32, [vp, P(u64)]),
         "adacomp_select_last_error": (i32, [vp, vp, P(u64)]),
         "adacomp_select_destroy": (i32, [vp]),
@@ -149,6 +150,17 @@ def segments_from(offsets: Sequence[int], ns: Sequence[int], ks: Sequence[int]):
     for l in range(len(ns)):
         segs[l].offset, segs[l].n, segs[l].k = int(offsets[l]), int(ns[l]), int(ks[l])
     return segs
+
+
+def adacomp_select_static(grad: torch.Tensor, k: int, idx_out: torch.Tensor, val_out: torch.Tensor,
+                          stream: Optional[torch.cuda.Stream] = None) -> None:
+    """Top-k-by-magnitude of one tensor through the entry point that allocates nothing: the caller
+    brings the input and both outputs, the scratch is a fixed array inside the library."""
+    if not (grad.is_cuda and grad.dtype == torch.float32 and grad.dim() == 1 and grad.stride(0) == 1):
+        raise TypeError("grad: need a 1-D contiguous CUDA fp32 tensor")
+    _check(_lib.adacomp_select_static(grad.data_ptr(), grad.numel(), int(k), _dev(idx_out, torch.int32, "idx_out"),
+                                      _dev(val_out, torch.float32, "val_out"), grad.device.index,
+                                      _stream_ptr(stream)), "adacomp_select_static")
 
 
 # ----------------------------------------------------------------------------- worker side

@@ -1,6 +1,7 @@
 // Worker side of libadacomp: handle, workspace layout and launch sequence of SELECT_GRAD
 // (Algorithm 1).
 #include <cmath>
+#include <mutex>
 #include <new>
 #include <vector>
 
@@ -433,3 +434,119 @@ int adacomp_select_destroy(adacomp_select_t* h) {
 }
 
 }  // extern "C"
+
+// ---------------------------------------------------------------------------------------------
+// Selection of one tensor with no workspace from the caller and no allocation by the library:
+// the scratch of the general route (one layout record, one instance record, the digit
+// histogram, the work list and the per-chunk counters) lives in a fixed array that is part of
+// the library image on every GPU that loads it.
+namespace {
+
+constexpr uint32_t kStaticMaxN = 1u << 24;                                   // entries per call
+constexpr uint32_t kStaticMaxSlots = (kStaticMaxN + 3 + kChunkElems - 1) / kChunkElems;   // 129 chunks
+// byte offsets inside the array (each 256-byte aligned)
+constexpr size_t kStOffLayer = 0;
+constexpr size_t kStOffInst = 256;
+constexpr size_t kStOffList = 512;
+constexpr size_t kStOffSlotStart = 768;
+constexpr size_t kStOffListLen = 1024;
+constexpr size_t kStOffStatus = 1280;
+constexpr size_t kStOffHist = 1536;
+constexpr size_t kStOffChunk = kStOffHist + kBins * sizeof(uint32_t);
+constexpr size_t kStaticScratchBytes = kStOffChunk + ((kStaticMaxSlots * sizeof(uint2) + 255) / 256) * 256;
+static_assert(sizeof(Layer) <= 256 && sizeof(Inst) <= 256, "records fit their 256-byte cells");
+static_assert(kStaticScratchBytes <= 16 * 1024, "the built-in scratch stays small");
+
+static __device__ __align__(256) unsigned char g_static_scratch[kStaticScratchBytes];
+
+// Writes the layout record and clears what a selection expects to find zeroed.  Names the array
+// directly: device code may.
+__global__ void k_static_setup(Layer L) {
+    *reinterpret_cast<Layer*>(g_static_scratch + kStOffLayer) = L;
+    uint32_t* hist = reinterpret_cast<uint32_t*>(g_static_scratch + kStOffHist);
+    for (int b = threadIdx.x; b < kBins; b += blockDim.x) hist[b] = 0;
+    if (threadIdx.x < 2) reinterpret_cast<uint32_t*>(g_static_scratch + kStOffListLen)[threadIdx.x] = 0;
+    if (threadIdx.x == 0) *reinterpret_cast<int*>(g_static_scratch + kStOffStatus) = 0;
+}
+
+// Device address of the array on each device, looked up once per device.  In host code the
+// array's name is only a handle for this lookup, never an address a kernel could use.
+constexpr int kMaxDevices = 64;
+unsigned char* g_static_ptr[kMaxDevices] = {};
+std::mutex g_static_mutex;
+
+int static_scratch_for(int device, unsigned char** out) {      // `device` must be current
+    if (device < 0 || device >= kMaxDevices) return ADACOMP_ERR_INVALID;
+    std::lock_guard<std::mutex> lock(g_static_mutex);
+    if (!g_static_ptr[device]) {
+        void* ptr = nullptr;
+        ADACOMP_CUDA(cudaGetSymbolAddress(&ptr, g_static_scratch));
+        g_static_ptr[device] = static_cast<unsigned char*>(ptr);
+    }
+    *out = g_static_ptr[device];
+    return ADACOMP_OK;
+}
+
+}  // namespace
+
+extern "C" int adacomp_select_static(const float* d_grad, uint32_t n, uint32_t k, uint32_t* d_idx_out,
+                                     float* d_val_out, int device, void* cuda_stream) {
+    if (n > kStaticMaxN) return ADACOMP_ERR_CAPACITY;          // beyond the built-in scratch
+    if (k > n || !d_grad || (k > 0 && (!d_idx_out || !d_val_out))) return ADACOMP_ERR_INVALID;
+    if (reinterpret_cast<uintptr_t>(d_grad) % 4 != 0) return ADACOMP_ERR_INVALID;
+    if (k == 0) return ADACOMP_OK;
+    DeviceGuard guard(device);
+    if (guard.err != cudaSuccess) return cuda_fail(guard.err);
+    unsigned char* base = nullptr;
+    int rc = static_scratch_for(device, &base);
+    if (rc != ADACOMP_OK) return rc;
+    int n_sms = 0;
+    ADACOMP_CUDA(cudaDeviceGetAttribute(&n_sms, cudaDevAttrMultiProcessorCount, device));
+    cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+
+    Layer L = {};
+    L.offset = 0;
+    L.out_offset = 0;
+    L.n = n;
+    L.k = k;
+    L.n_slots = static_cast<uint32_t>((static_cast<uint64_t>(n) + 3 + kChunkElems - 1) / kChunkElems);
+    L.slot_base = 0;
+
+    SelectParams p = {};
+    p.grads = d_grad;
+    p.stride = n;
+    p.n_workers = 1;
+    p.n_layers = 1;
+    p.layers = reinterpret_cast<const Layer*>(base + kStOffLayer);
+    p.inst = reinterpret_cast<Inst*>(base + kStOffInst);
+    p.hist = reinterpret_cast<uint32_t*>(base + kStOffHist);
+    p.list = reinterpret_cast<uint32_t*>(base + kStOffList);
+    p.list_slot_start = reinterpret_cast<uint32_t*>(base + kStOffSlotStart);
+    p.list_len = reinterpret_cast<uint32_t*>(base + kStOffListLen);
+    p.chunk_cnt = reinterpret_cast<uint2*>(base + kStOffChunk);
+    p.slots_per_worker = L.n_slots;
+    p.idx_out = d_idx_out;
+    p.val_out = d_val_out;
+    p.K = k;
+    p.status = reinterpret_cast<int*>(base + kStOffStatus);
+
+    unsigned grid = static_cast<unsigned>(n_sms) * 8;
+    if (grid > L.n_slots) grid = L.n_slots;
+    k_static_setup<<<1, kThreads, 0, st>>>(L);
+    ADACOMP_LAUNCH_CHECK();
+    k_bracket_sample<<<1, kBig, 0, st>>>(p, 1);                 // general route only: resets the instance record
+    ADACOMP_LAUNCH_CHECK();
+    k_general_plan<<<1, kThreads, 0, st>>>(p);
+    ADACOMP_LAUNCH_CHECK();
+    k_general_hist<0><<<grid, kThreads, 0, st>>>(p);
+    ADACOMP_LAUNCH_CHECK();
+    k_general_hist<1><<<grid, kThreads, 0, st>>>(p);
+    ADACOMP_LAUNCH_CHECK();
+    k_general_hist<2><<<grid, kThreads, 0, st>>>(p);
+    ADACOMP_LAUNCH_CHECK();
+    k_general_count<<<grid, kThreads, 0, st>>>(p);
+    ADACOMP_LAUNCH_CHECK();
+    k_general_write<<<grid, kThreads, 0, st>>>(p);
+    ADACOMP_LAUNCH_CHECK();
+    return ADACOMP_OK;
+}
