@@ -22,7 +22,7 @@ struct adacomp_select {
     int n_sms = 0;
     int route = 0;         // 0 = automatic, 1 = general route for everything
     bool all_bracketed = false;   // every tensor with k > 0 is eligible for the bracketed route
-    uint32_t n_layers = 0, max_workers = 0, slots_per_worker = 0, n_items = 0, max_sample = 0;
+    uint32_t n_layers = 0, max_workers = 0, slots_per_worker = 0, n_items = 0, n_items_sparse = 0, max_sample = 0;
     uint64_t extent = 0;   // one past the last entry any segment covers
     uint64_t K = 0;        // pairs per worker
     uint64_t cand_stride = 0, win_stride = 0, span_stride = 0;
@@ -57,10 +57,11 @@ namespace {
 
 struct Layout {
     std::vector<Layer> layers;
-    std::vector<uint2> items;
+    std::vector<uint2> items;          // scan / emit work items: sparse-scan tensors first, then dense-scan ones
+    std::vector<uint2> dense_items;
     uint64_t extent = 0, K = 0;
     uint64_t cand_stride = 0, win_stride = 0, span_stride = 0;
-    uint32_t slots_per_worker = 0, max_sample = 0;
+    uint32_t slots_per_worker = 0, max_sample = 0, n_items_sparse = 0;
 };
 
 // Decides whether a tensor takes the bracketed route and how much room its lists get.  The
@@ -87,7 +88,8 @@ void plan_bracket(Layer& L, Layout* out) {
     double win = n * win_frac * (1.0 + 6.0 / std::sqrt(static_cast<double>(r_lo + 1 - r_hi))) + 2048.0;
     if (cand > n) cand = n;
     if (win > n) win = n;
-    L.bracket = 1;
+    // tensors whose candidates will be about a tenth of the entries or more take the dense scan kernel
+    L.bracket = lo_frac >= 0.08 ? 2 : 1;
     L.sample = m;
     L.n_spans = n_spans;
     L.span_base = static_cast<uint32_t>(out->span_stride);
@@ -124,8 +126,10 @@ int build_layout(const adacomp_segment_t* segs, uint32_t n_segs, uint32_t max_wo
         end_prev = s.offset + s.n;
         plan_bracket(L, out);
         for (uint32_t s0 = 0; L.bracket && s0 < L.n_spans; s0 += kSpansPerBlock)
-            out->items.push_back(make_uint2(l, s0));
+            (L.bracket == 2 ? out->dense_items : out->items).push_back(make_uint2(l, s0));
     }
+    out->n_items_sparse = static_cast<uint32_t>(out->items.size());
+    out->items.insert(out->items.end(), out->dense_items.begin(), out->dense_items.end());
     if (K > kMaxIndex || slots * max_workers > 0x7FFFFFFFull ||
         static_cast<uint64_t>(n_segs) * max_workers > 0x7FFFFFFFull ||
         out->span_stride * max_workers > 0x7FFFFFFFull || out->items.size() > 0x7FFFFFFFull)
@@ -210,6 +214,7 @@ int adacomp_select_create(adacomp_select_t** h, const adacomp_segment_t* h_segs,
     s->extent = lay.extent;
     s->K = lay.K;
     s->n_items = static_cast<uint32_t>(lay.items.size());
+    s->n_items_sparse = lay.n_items_sparse;
     s->all_bracketed = true;
     for (const Layer& L : lay.layers)
         if (L.k > 0 && !L.bracket) s->all_bracketed = false;
@@ -235,6 +240,9 @@ int adacomp_select_create(adacomp_select_t** h, const adacomp_segment_t* h_segs,
     if (e == cudaSuccess)
         e = cudaFuncSetAttribute(k_bracket_scan, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                  static_cast<int>(kScanSmemPerWarp * (kThreads / 32)));
+    if (e == cudaSuccess)
+        e = cudaFuncSetAttribute(k_bracket_scan_dense, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                 static_cast<int>(kDenseSmemPerWarp * (kThreads / 32)));
     if (e == cudaSuccess) e = cudaDeviceSynchronize();
     if (e != cudaSuccess) { delete s; return cuda_fail(e); }
     *h = s;
@@ -309,8 +317,15 @@ int adacomp_select(adacomp_select_t* h, const float* d_grads, uint64_t worker_st
     ADACOMP_CUDA(mark(1));
     if (bracketed) {
         const dim3 grid(h->n_items, n_workers);
-        k_bracket_scan<<<grid, kThreads, kScanSmemPerWarp * (kThreads / 32), st>>>(p);
-        ADACOMP_LAUNCH_CHECK();
+        if (h->n_items_sparse) {
+            k_bracket_scan<<<dim3(h->n_items_sparse, n_workers), kThreads, kScanSmemPerWarp * (kThreads / 32), st>>>(p, 0u);
+            ADACOMP_LAUNCH_CHECK();
+        }
+        if (h->n_items > h->n_items_sparse) {
+            k_bracket_scan_dense<<<dim3(h->n_items - h->n_items_sparse, n_workers), kThreads,
+                                   kDenseSmemPerWarp * (kThreads / 32), st>>>(p, h->n_items_sparse);
+            ADACOMP_LAUNCH_CHECK();
+        }
         ADACOMP_CUDA(mark(2));
         k_bracket_resolve<<<n_inst, kBig, 0, st>>>(p);
         ADACOMP_LAUNCH_CHECK();

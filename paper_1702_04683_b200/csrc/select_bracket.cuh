@@ -197,9 +197,9 @@ __device__ __forceinline__ bool load_hits(const float4& x, float tlo_f) {
     return !(m4 < tlo_f);
 }
 
-__global__ void __launch_bounds__(kThreads, 4) k_bracket_scan(SelectParams p) {
+__global__ void __launch_bounds__(kThreads, 4) k_bracket_scan(SelectParams p, uint32_t item_base) {
     extern __shared__ __align__(16) unsigned char s_scan[];
-    const uint2 item = p.items[blockIdx.x];
+    const uint2 item = p.items[item_base + blockIdx.x];
     const uint32_t l = item.x, w = blockIdx.y;
     const Layer L = p.layers[l];
     Inst* st = &p.inst[w * p.n_layers + l];
@@ -376,6 +376,172 @@ __global__ void __launch_bounds__(kThreads, 4) k_bracket_scan(SelectParams p) {
             run += n_c;
             wrun += n_w;
         }
+    }
+    if (saw_nan) atomicOr(&st->flags, kInstOverflow);
+}
+
+// ---------------------------------------------------------------------------------------------
+// The same pass for tensors whose candidates are dense (a few percent of the entries or more),
+// where nearly every load holds a candidate and queueing loads would only add work.  Same
+// decomposition (8 warps x 8 pieces of 1024 entries per block, warps on their own), but a piece
+// is classified entirely in registers: two bit masks per lane (candidate, window), one 64-bit
+// atomic per piece to reserve room, and while it is in flight the warp ranks its candidates in
+// index order (two byte-packed warp scans: candidates per load and lane) and stages index and
+// value of each in shared memory straight from the registers, so nothing is read twice.  The
+// next piece's loads are issued as soon as the registers are free, before the reservation is
+// consumed; the staged lists then leave with coalesced stores.
+constexpr uint32_t kDenseStage = 640;                          // candidates staged per piece (of 1024 entries)
+constexpr uint32_t kDenseWinStage = 384;                       // window entries staged per piece
+constexpr size_t kDenseSmemPerWarp = (kDenseStage + kDenseWinStage) * 8;
+
+__global__ void __launch_bounds__(kThreads, 3) k_bracket_scan_dense(SelectParams p, uint32_t item_base) {
+    extern __shared__ __align__(16) unsigned char s_scan[];
+    const uint2 item = p.items[item_base + blockIdx.x];
+    const uint32_t l = item.x, w = blockIdx.y;
+    const Layer L = p.layers[l];
+    Inst* st = &p.inst[w * p.n_layers + l];
+    if (!(__ldcg(&st->flags) & kInstBracket)) return;
+    const float tlo_f = __uint_as_float(__ldcg(&st->t_lo)), thi_f = __uint_as_float(__ldcg(&st->t_hi));
+    const float* first = p.grads + static_cast<uint64_t>(w) * p.stride + L.offset;
+    const uint32_t mis = static_cast<uint32_t>((reinterpret_cast<uintptr_t>(first) >> 2) & 3u);
+    const float4* vec = reinterpret_cast<const float4*>(first - mis);
+    const uint32_t n_shift = L.n + mis;                        // n <= 33.5 M on this route
+    const uint32_t nvec = (n_shift + 3) >> 2;
+    const uint32_t lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    constexpr uint32_t kStep = kThreads / 32;
+    constexpr uint32_t kBatch = kSpansPerBlock * kSubsPerSpan / kStep;
+    const uint32_t ss_end = min(item.y + kSpansPerBlock, L.n_spans) * kSubsPerSpan;
+    const uint32_t ss0 = item.y * kSubsPerSpan + warp;
+    if (ss0 >= ss_end) return;
+    const uint32_t in_lo = mis ? 1u : 0u, in_hi = n_shift / kSubElems;
+    unsigned char* mine = s_scan + warp * kDenseSmemPerWarp;
+    uint32_t* stage_idx = reinterpret_cast<uint32_t*>(mine);
+    float* stage_val = reinterpret_cast<float*>(mine + kDenseStage * 4);
+    uint32_t* stage_widx = reinterpret_cast<uint32_t*>(mine + kDenseStage * 8);
+    uint32_t* stage_wkey = reinterpret_cast<uint32_t*>(mine + kDenseStage * 8 + kDenseWinStage * 4);
+    uint32_t* cand_idx = p.cand_idx + static_cast<uint64_t>(w) * p.cand_stride + L.cand_base;
+    float* cand_val = p.cand_val + static_cast<uint64_t>(w) * p.cand_stride + L.cand_base;
+    uint32_t* win_key = p.win_key + static_cast<uint64_t>(w) * p.win_stride + L.win_base;
+    uint32_t* win_idx = p.win_idx + static_cast<uint64_t>(w) * p.win_stride + L.win_base;
+    uint2* sub_tab = p.sub_tab + (static_cast<uint64_t>(w) * p.span_stride + L.span_base) * kSubsPerSpan;
+
+    float4 x[8];
+    bool have_x = false;                                       // x already holds the piece about to be classified
+    bool saw_nan = false;
+#pragma unroll 1
+    for (uint32_t j = 0; j < kBatch; ++j) {
+        const uint32_t ss = ss0 + kStep * j, next = ss + kStep;
+        if (ss >= ss_end) break;
+        const bool inside = ss >= in_lo && ss < in_hi;
+        const uint32_t vec0 = ss * (kSubElems / 4);
+        if (!have_x) {
+#pragma unroll
+            for (int i = 0; i < 8; ++i) {
+                const uint32_t v = vec0 + i * 32 + lane;
+                x[i] = (inside || v < nvec) ? __ldg(&vec[v]) : make_float4(0.f, 0.f, 0.f, 0.f);
+            }
+        }
+        // classify every entry: bit 4 i + q = component q of this lane's load i
+        uint32_t mask_c = 0, mask_w = 0;
+#pragma unroll
+        for (int i = 0; i < 8; ++i) {
+            float xs[4] = {x[i].x, x[i].y, x[i].z, x[i].w};
+            if (!inside) {                                     // first / last piece: blank what lies outside (t_lo > 0)
+                const uint32_t e0 = (vec0 + i * 32 + lane) * 4;
+#pragma unroll
+                for (int q = 0; q < 4; ++q)
+                    if (e0 + q < mis || e0 + q >= n_shift) xs[q] = 0.f;
+                x[i] = make_float4(xs[0], xs[1], xs[2], xs[3]);
+            }
+            const float m4 = max_nan(max_nan(fabsf(xs[0]), fabsf(xs[1])), max_nan(fabsf(xs[2]), fabsf(xs[3])));
+            saw_nan |= m4 != m4;
+#pragma unroll
+            for (int q = 0; q < 4; ++q) {
+                const float a = fabsf(xs[q]);
+                const bool cand = !(a < tlo_f);
+                if (cand) mask_c |= 1u << (i * 4 + q);
+                if (cand && !(a > thi_f)) mask_w |= 1u << (i * 4 + q);
+            }
+        }
+        const uint32_t cw = __popc(mask_w);
+        const uint32_t tc = __reduce_add_sync(0xFFFFFFFFu, __popc(mask_c));
+        const uint32_t tw = __reduce_add_sync(0xFFFFFFFFu, cw);
+        unsigned long long old = 0;
+        if (tc && lane == 0)                                  // reserve room: one atomic per piece
+            old = atomicAdd(reinterpret_cast<unsigned long long*>(&st->cand_count),
+                            static_cast<unsigned long long>(tc) | (static_cast<unsigned long long>(tw) << 32));
+        const bool fits = tc <= kDenseStage && tw <= kDenseWinStage;
+        if (tc && fits) {
+            // rank in index order = (load, lane, component): per-load counts of this lane, one byte
+            // each (a load holds at most 128 candidates across the warp), scanned over the lanes
+            const uint32_t cnt_a = __popc(mask_c & 0xFu) | (__popc(mask_c & 0xF0u) << 8) |
+                                   (__popc(mask_c & 0xF00u) << 16) | (__popc(mask_c & 0xF000u) << 24);
+            const uint32_t cnt_b = __popc(mask_c & 0xF0000u) | (__popc(mask_c & 0xF00000u) << 8) |
+                                   (__popc(mask_c & 0xF000000u) << 16) | (__popc(mask_c & 0xF0000000u) << 24);
+            uint32_t inc_a = cnt_a, inc_b = cnt_b, inc_w = cw;
+#pragma unroll
+            for (int d = 1; d < 32; d <<= 1) {
+                const uint32_t ya = __shfl_up_sync(0xFFFFFFFFu, inc_a, d);
+                const uint32_t yb = __shfl_up_sync(0xFFFFFFFFu, inc_b, d);
+                const uint32_t yw = __shfl_up_sync(0xFFFFFFFFu, inc_w, d);
+                if (lane >= static_cast<uint32_t>(d)) { inc_a += ya; inc_b += yb; inc_w += yw; }
+            }
+            const uint32_t tot_a = __shfl_sync(0xFFFFFFFFu, inc_a, 31), tot_b = __shfl_sync(0xFFFFFFFFu, inc_b, 31);
+            const uint32_t pre_a = inc_a - cnt_a, pre_b = inc_b - cnt_b;
+            uint32_t wr = inc_w - cw;                             // window entries: any order (lane-major)
+            uint32_t load_off = 0;
+#pragma unroll
+            for (int i = 0; i < 8; ++i) {
+                const uint32_t pre_i = ((i < 4 ? pre_a : pre_b) >> ((i & 3) * 8)) & 255u;
+                const uint32_t tot_i = ((i < 4 ? tot_a : tot_b) >> ((i & 3) * 8)) & 255u;
+                const float xs[4] = {x[i].x, x[i].y, x[i].z, x[i].w};
+                const uint32_t e0 = (vec0 + i * 32 + lane) * 4;
+                uint32_t r = load_off + pre_i;
+#pragma unroll
+                for (int q = 0; q < 4; ++q) {
+                    if ((mask_c >> (i * 4 + q)) & 1u) {
+                        stage_idx[r] = e0 + q;                    // shifted coordinate inside the tensor
+                        stage_val[r] = xs[q];
+                        ++r;
+                        if ((mask_w >> (i * 4 + q)) & 1u) {
+                            stage_widx[wr] = e0 + q;
+                            stage_wkey[wr] = magnitude_key(xs[q]);
+                            ++wr;
+                        }
+                    }
+                }
+                load_off += tot_i;
+            }
+        }
+        __syncwarp();
+        // the registers are free: start the next piece's loads before consuming the reservation
+        have_x = (j + 1 < kBatch) && next < ss_end && next >= in_lo && next < in_hi;
+        if (have_x) {
+            const float4* nptr = vec + next * (kSubElems / 4) + lane;
+#pragma unroll
+            for (int i = 0; i < 8; ++i) x[i] = __ldg(nptr + i * 32);
+        }
+        if (tc) {
+            old = __shfl_sync(0xFFFFFFFFu, old, 0);
+            const uint32_t cb = static_cast<uint32_t>(old), wb = static_cast<uint32_t>(old >> 32);
+            const bool over = !fits || (static_cast<uint64_t>(cb) + tc > L.cand_cap) ||
+                              (static_cast<uint64_t>(wb) + tw > L.win_cap);
+            if (lane == 0) {
+                sub_tab[ss] = make_uint2(cb, tc | ((tc - tw) << 16));
+                if (over) atomicOr(&st->flags, kInstOverflow);
+            }
+            if (!over) {
+                for (uint32_t r = lane; r < tc; r += 32) {
+                    cand_idx[cb + r] = stage_idx[r];
+                    cand_val[cb + r] = stage_val[r];
+                }
+                for (uint32_t r = lane; r < tw; r += 32) {
+                    win_idx[wb + r] = stage_widx[r];
+                    win_key[wb + r] = stage_wkey[r];
+                }
+            }
+        }
+        __syncwarp();                                         // the stage is reused by the next piece
     }
     if (saw_nan) atomicOr(&st->flags, kInstOverflow);
 }
