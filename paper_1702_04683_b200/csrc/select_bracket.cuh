@@ -249,7 +249,7 @@ __global__ void __launch_bounds__(kThreads, 4) k_bracket_scan(SelectParams p, ui
         if (lane < kBatch) s_cnt[lane] = 0;
         __syncwarp();
 #pragma unroll 1
-        for (; j < kBatch && qn + 256 <= kScanQueue; ++j) {
+        for (; j < kBatch && qn + 256 <= kScanQueue && qn < 96; ++j) {
             const uint32_t ss = ss0 + kStep * j, next = ss + kStep;
             if (ss >= ss_end) break;
             const bool next_inside = (j + 1 < kBatch) && next < ss_end && next >= in_lo && next < in_hi;
