@@ -254,7 +254,6 @@ __global__ void __launch_bounds__(kThreads, 4) k_bracket_scan(SelectParams p, ui
             if (ss >= ss_end) break;
             const bool next_inside = (j + 1 < kBatch) && next < ss_end && next >= in_lo && next < in_hi;
             const float4* nptr = vec + (next_inside ? next : ss0) * (kSubElems / 4) + lane;   // ss0: any valid address
-            uint32_t pcnt = 0;                                 // this lane's candidates | window << 16 in the piece
 #pragma unroll
             for (int i = 0; i < 8; ++i) {
                 float4 y;
@@ -272,33 +271,39 @@ __global__ void __launch_bounds__(kThreads, 4) k_bracket_scan(SelectParams p, ui
                     h = load_hits(y, tlo_f);
                 }
                 const uint32_t b = __ballot_sync(0xFFFFFFFFu, h);
-                if (b) {
-                    if (h) {
-                        const float ys[4] = {y.x, y.y, y.z, y.w};
-                        uint32_t nc = 0, nw = 0;
-#pragma unroll
-                        for (int c4 = 0; c4 < 4; ++c4) {
-                            const float a = fabsf(ys[c4]);
-                            const bool cand = !(a < tlo_f);
-                            saw_nan |= a != a;
-                            if (cand) nc |= 1u << c4;
-                            if (cand && !(a > thi_f)) nw |= 1u << c4;
-                        }
-                        const uint32_t slot = qn + __popc(b & lt);
-                        q[slot] = static_cast<uint16_t>(j * 256 + i * 32 + lane);
-                        info[slot] = static_cast<unsigned char>(nc | (nw << 4));
-                        pcnt += __popc(nc) | (__popc(nw) << 16);
-                    }
+                if (b) {                                       // queue the loads that hit; they are classified in the tail
+                    if (h) q[qn + __popc(b & lt)] = static_cast<uint16_t>(j * 256 + i * 32 + lane);
                     qn += __popc(b);
                 }
                 if (next_inside) x[i] = __ldg(nptr + i * 32);
             }
             loaded = next_inside;
-            const uint32_t ptot = __reduce_add_sync(0xFFFFFFFFu, pcnt);
-            if (lane == 0) s_cnt[j] = ptot;
         }
         __syncwarp();
         if (!qn) continue;                                     // the table entries stay (0, 0)
+
+        // ================= tail, pass A: fetch the queued loads again (an L1 / L2 hit: the round is
+        // short), classify their entries with every lane busy, count per piece
+        for (uint32_t t = lane; t < qn; t += 32) {
+            const uint32_t ent = q[t];
+            const uint32_t pj = ent >> 8;
+            const uint32_t v = (ss0 + kStep * pj) * (kSubElems / 4) + (ent & 255u);
+            const float4 y = (v < nvec) ? __ldg(&vec[v]) : make_float4(0.f, 0.f, 0.f, 0.f);
+            const float ys[4] = {y.x, y.y, y.z, y.w};
+            uint32_t nc = 0, nw = 0;
+#pragma unroll
+            for (int c4 = 0; c4 < 4; ++c4) {
+                const uint32_t e = v * 4 + c4;
+                const float a = fabsf(ys[c4]);
+                const bool cand = (e >= mis && e < n_shift) && !(a < tlo_f);
+                saw_nan |= cand && (a != a);
+                if (cand) nc |= 1u << c4;
+                if (cand && !(a > thi_f)) nw |= 1u << c4;
+            }
+            info[t] = static_cast<unsigned char>(nc | (nw << 4));
+            if (nc) atomicAdd(&s_cnt[pj], __popc(nc) | (__popc(nw) << 16));
+        }
+        __syncwarp();
 
         // ================= tail: reserve once for the round, then rank and write
         const uint32_t mycnt = lane < kBatch ? s_cnt[lane] : 0u;
