@@ -155,6 +155,157 @@ k_apply_batch(ServerParams sp, BatchDesc d, const uint32_t* __restrict__ idx, co
     if (r_hi == n_ranges && lane < B && cursor < my_n) record_error(sp.status, ADACOMP_ERR_UNSORTED);
 }
 
+// ---------------------------------------------------------------------------------------------
+// Several updates per launch, block-level owner ("owner block"), for batches that touch a good
+// part of the parameters.  A block owns a run of kOwnRange-parameter ranges.  Per range it loads
+// Theta and the history heads into shared memory (coalesced), then works in rounds: all warps
+// together stage, for every update of the batch at once, the next pairs of the range (so the
+// global loads of all updates overlap); the updates are then applied IN ARRIVAL ORDER out of
+// shared memory, one block barrier per update.  Only parameters below a limit are applied in a
+// round: the smallest index some update could not stage any more, so every update's pairs below
+// the limit are on chip.  Staleness inside the batch comes from a per-parameter bit mask of the
+// batch's updates that changed it (Eq. 3 restricted to the batch is a population count); the
+// part of a window that lies before the batch is counted by walking the chain from the head the
+// parameter had when the batch began.  Theta and heads of the range are written back once.
+// Same results, bit for bit, as one launch per update.
+constexpr uint32_t kOwnRange = 1024;
+constexpr uint32_t kOwnStage = 128;            // pairs staged per update and round
+constexpr int kOwnThreads = 256;
+
+struct OwnDesc {
+    BatchDesc b;
+    uint32_t win_bits[kMaxBatch];              // updates of this batch inside update b's window (bits below b)
+    uint32_t pre_mask;                         // bit b: update b's window starts before the batch
+};
+
+constexpr size_t kOwnSmemBytes = kOwnRange * 16 + kMaxBatch * kOwnStage * 6 + kMaxBatch * 8 + 16;
+
+__global__ void __launch_bounds__(kOwnThreads)
+k_apply_owner(ServerParams sp, OwnDesc d, const uint32_t* __restrict__ idx, const float* __restrict__ val,
+              float lr, uint32_t* sigma_out, uint32_t n_ranges) {
+    extern __shared__ __align__(16) unsigned char s_own[];
+    float* s_theta = reinterpret_cast<float*>(s_own);
+    uint32_t* s_head = reinterpret_cast<uint32_t*>(s_own + kOwnRange * 4);       // head when the batch began
+    uint32_t* s_last = reinterpret_cast<uint32_t*>(s_own + kOwnRange * 8);       // latest position set by the batch
+    uint32_t* s_mask = reinterpret_cast<uint32_t*>(s_own + kOwnRange * 12);      // updates of the batch that changed it
+    float* s_v = reinterpret_cast<float*>(s_own + kOwnRange * 16);                                    // [B][kOwnStage]
+    uint16_t* s_k = reinterpret_cast<uint16_t*>(s_own + kOwnRange * 16 + kMaxBatch * kOwnStage * 4);   // [B][kOwnStage]
+    uint32_t* s_cnt = reinterpret_cast<uint32_t*>(s_own + kOwnRange * 16 + kMaxBatch * kOwnStage * 6);
+    uint32_t* s_cur = s_cnt + kMaxBatch;
+    uint32_t* s_limit = s_cur + kMaxBatch;
+
+    const uint32_t tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const uint32_t B = d.b.n_updates;
+    const uint32_t r_lo = static_cast<uint32_t>(static_cast<uint64_t>(n_ranges) * blockIdx.x / gridDim.x);
+    const uint32_t r_hi = static_cast<uint32_t>(static_cast<uint64_t>(n_ranges) * (blockIdx.x + 1) / gridDim.x);
+    if (r_lo == r_hi) return;
+    if (tid < B) {                                              // cursor: first pair at or above the first owned parameter
+        const uint64_t first_param = static_cast<uint64_t>(r_lo) * kOwnRange;
+        const uint64_t begin = d.b.pair_begin[tid];
+        uint32_t lo = 0, hi = d.b.n_pairs[tid];
+        while (lo < hi) {
+            const uint32_t mid = lo + ((hi - lo) >> 1);
+            if (idx[begin + mid] < first_param) lo = mid + 1; else hi = mid;
+        }
+        s_cur[tid] = lo;
+    }
+    __syncthreads();
+
+    for (uint32_t r = r_lo; r < r_hi; ++r) {
+        const uint32_t lo = r * kOwnRange;
+        const uint64_t hi64 = static_cast<uint64_t>(lo) + kOwnRange;
+        const uint32_t hi = hi64 < sp.n_params ? static_cast<uint32_t>(hi64) : static_cast<uint32_t>(sp.n_params);
+        for (uint32_t t = tid; t < kOwnRange; t += kOwnThreads) {
+            const bool in = lo + t < hi;
+            s_theta[t] = in ? sp.theta[lo + t] : 0.f;
+            s_head[t] = in ? sp.head[lo + t] : kNone;
+            s_last[t] = kNone;
+            s_mask[t] = 0;
+        }
+        while (true) {
+            if (tid == 0) *s_limit = hi;
+            __syncthreads();
+            // ---- stage: warp w takes updates w, w + 8, ...; 4 x 32 pairs each
+            for (uint32_t b = warp; b < B; b += kOwnThreads / 32) {
+                const uint64_t begin = d.b.pair_begin[b];
+                const uint32_t n_b = d.b.n_pairs[b], cur = s_cur[b];
+                uint32_t cnt = 0, last_k = 0;
+#pragma unroll
+                for (uint32_t c = 0; c < kOwnStage / 32; ++c) {
+                    const uint32_t t = c * 32 + lane, e = cur + t;
+                    uint32_t k = kNone;
+                    float v = 0.f;
+                    if (e < n_b) {                              // both loads at once: the value does not wait for the index
+                        k = idx[begin + e];
+                        v = val[begin + e];
+                    }
+                    const bool mine = k < hi;                   // ascending list: matching slots form a prefix
+                    if (mine) {
+                        if (sp.validate && e > 0 && idx[begin + e - 1] >= k) record_error(sp.status, ADACOMP_ERR_UNSORTED);
+                        s_k[b * kOwnStage + t] = static_cast<uint16_t>(k - lo);
+                        s_v[b * kOwnStage + t] = v;
+                    }
+                    cnt += __popc(__ballot_sync(0xFFFFFFFFu, mine));
+                    if (c == kOwnStage / 32 - 1) last_k = __shfl_sync(0xFFFFFFFFu, k, 31);
+                }
+                if (lane == 0) {
+                    s_cnt[b] = cnt;
+                    if (cnt == kOwnStage) atomicMin(s_limit, last_k + 1);   // more of this update may follow in the range
+                }
+            }
+            __syncthreads();
+            const uint32_t limit = *s_limit;
+            // ---- apply, update after update
+            for (uint32_t b = 0; b < B; ++b) {
+                const uint32_t cnt = s_cnt[b];
+                if (cnt == 0) continue;                         // nothing of update b in this round (same for all threads)
+                bool take = false;
+                if (tid < cnt) {
+                    const uint32_t kl = s_k[b * kOwnStage + tid];
+                    take = lo + kl < limit;
+                    if (take) {
+                        const float v = s_v[b * kOwnStage + tid];
+                        const uint32_t e = s_cur[b] + tid;
+                        const uint32_t m = s_mask[kl], ho = s_head[kl];
+                        uint32_t sigma = __popc(m & d.win_bits[b]);
+                        if ((d.pre_mask >> b) & 1u) {           // the part of the window before the batch
+                            uint32_t q = ho, hops = 0;
+                            const uint32_t ws = d.b.win_start[b];
+                            while (q != kNone && q >= ws) {
+                                if (++hops > sp.max_window) { record_error(sp.status, ADACOMP_ERR_WINDOW); break; }
+                                q = sp.prev[(q + sp.ring_shift) & sp.ring_mask];
+                            }
+                            sigma += hops;
+                        }
+                        if (sigma_out) sigma_out[d.b.pair_begin[b] + e] = sigma;
+                        if (v != 0.0f) {                        // Eq. 3 counts changes: a zero entry is not one
+                            const float alpha_k = sigma ? __fdiv_rn(lr, static_cast<float>(sigma)) : lr;      // Eq. 5
+                            s_theta[kl] = __fsub_rn(s_theta[kl], __fmul_rn(alpha_k, v));                       // Eq. 4
+                            const uint32_t pos = d.b.pos_start[b] + e;
+                            sp.prev[(pos + sp.ring_shift) & sp.ring_mask] = m ? s_last[kl] : ho;
+                            s_last[kl] = pos;
+                            s_mask[kl] = m | (1u << b);
+                        }
+                    }
+                }
+                const uint32_t took = __syncthreads_count(take);   // also orders update b before update b + 1
+                if (tid == 0) s_cur[b] += took;
+            }
+            __syncthreads();
+            if (limit >= hi) break;                             // every update's pairs of the range are done
+        }
+        for (uint32_t t = tid; t < kOwnRange; t += kOwnThreads) {
+            if (lo + t < hi && s_mask[t]) {
+                sp.theta[lo + t] = s_theta[t];
+                sp.head[lo + t] = s_last[t];
+            }
+        }
+        __syncthreads();
+    }
+    // whoever owns the last range sees what no range claimed: indices >= n_params
+    if (r_hi == n_ranges && tid < B && s_cur[tid] < d.b.n_pairs[tid]) record_error(sp.status, ADACOMP_ERR_UNSORTED);
+}
+
 // Moves every stored position down by `delta` (entries older than that become kNone).
 __global__ void k_rebase(uint32_t* a, uint64_t n, uint32_t delta) {
     for (uint64_t i = blockIdx.x * static_cast<uint64_t>(blockDim.x) + threadIdx.x; i < n;
@@ -241,6 +392,8 @@ int adacomp_server_create(adacomp_server_t** out, uint64_t n_params, uint64_t hi
     cudaError_t e = guard.err;
     if (e == cudaSuccess) e = cudaDeviceGetAttribute(&s->n_sms, cudaDevAttrMultiProcessorCount, device);
     if (e == cudaSuccess) e = cudaMemset(s->d_status, 0, sizeof(int));
+    if (e == cudaSuccess)
+        e = cudaFuncSetAttribute(k_apply_owner, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(kOwnSmemBytes));
     if (e == cudaSuccess) e = cudaDeviceSynchronize();
     if (e != cudaSuccess) { delete s; return cuda_fail(e); }
     *out = s;
@@ -334,16 +487,24 @@ int adacomp_apply(adacomp_server_t* s, const uint32_t* d_idx, const float* d_val
     // (automatic: the batched kernel pays off when an update names between about 0.2 % and 6 % of
     // the parameters; sparser updates are launch-bound either way, denser ones keep DRAM busy alone)
     const double density = static_cast<double>(call_pairs) / n_updates / static_cast<double>(s->n_params);
-    const bool batched = s->mode == 2 || (s->mode == 0 && n_updates >= 2 && density >= 0.002 && density <= 0.06);
-    if (batched) {
-        const uint64_t n_ranges64 = (s->n_params + kRangeParams - 1) / kRangeParams;
-        const uint32_t n_ranges = static_cast<uint32_t>(n_ranges64);
+    // (automatic: when the updates of a launch (up to 32) together name about half as many pairs as
+    // there are parameters, the block owner kernel, which sweeps Theta once per launch; else the warp
+    // owner kernel for updates that name 0.2 % - 6 % of the parameters; else one launch per update)
+    const uint32_t per_launch = n_updates < kMaxBatch ? n_updates : kMaxBatch;
+    const bool owner = s->mode == 3 || (s->mode == 0 && n_updates >= 2 && density * per_launch >= 0.4);
+    const bool batched = !owner && (s->mode == 2 || (s->mode == 0 && n_updates >= 2 && density >= 0.002 && density <= 0.06));
+    if (owner || batched) {
+        const uint32_t n_ranges = static_cast<uint32_t>((s->n_params + kRangeParams - 1) / kRangeParams);   // kOwnRange == kRangeParams
         uint64_t want_warps = static_cast<uint64_t>(s->n_sms) * 64;            // 64 resident warps per SM
         if (want_warps > n_ranges) want_warps = n_ranges;
         const unsigned grid = static_cast<unsigned>((want_warps + kApplyThreads / 32 - 1) / (kApplyThreads / 32));
+        unsigned own_grid = static_cast<unsigned>(s->n_sms) * 5;
+        if (own_grid > n_ranges) own_grid = n_ranges;
         for (uint32_t b0 = 0; b0 < n_updates; b0 += kMaxBatch) {
-            BatchDesc d;
+            OwnDesc od;
+            BatchDesc& d = od.b;
             d.n_updates = (n_updates - b0 < kMaxBatch) ? n_updates - b0 : kMaxBatch;
+            od.pre_mask = 0;
             uint64_t pairs = 0;
             for (uint32_t b = 0; b < d.n_updates; ++b) {
                 d.pair_begin[b] = h_pair_begin[b0 + b];
@@ -351,11 +512,20 @@ int adacomp_apply(adacomp_server_t* s, const uint32_t* d_idx, const float* d_val
                 d.pos_start[b] = static_cast<uint32_t>(start_abs[b0 + b] - s->pos_base);
                 d.win_start[b] = static_cast<uint32_t>(win_abs[b0 + b] - s->pos_base);
                 pairs += h_pair_count[b0 + b];
+                // which updates of this launch lie in update b's window [j, i - 1]
+                const uint64_t ts0 = i0 + b0, j = h_pull_ts[b0 + b];
+                const uint32_t first_in = j > ts0 ? static_cast<uint32_t>(j - ts0) : 0u;     // <= b
+                od.win_bits[b] = ((1u << b) - 1u) & ~((1u << first_in) - 1u);
+                if (j < ts0) od.pre_mask |= 1u << b;
             }
-            if (pairs) {
+            for (uint32_t b = d.n_updates; b < kMaxBatch; ++b) od.win_bits[b] = 0;
+            if (!pairs) continue;
+            if (owner) {
+                k_apply_owner<<<own_grid, kOwnThreads, kOwnSmemBytes, st>>>(sp, od, d_idx, d_val, lr, d_sigma_out, n_ranges);
+            } else {
                 k_apply_batch<<<grid, kApplyThreads, 0, st>>>(sp, d, d_idx, d_val, lr, d_sigma_out, n_ranges);
-                ADACOMP_LAUNCH_CHECK();
             }
+            ADACOMP_LAUNCH_CHECK();
         }
     } else {
         for (uint32_t b = 0; b < n_updates; ++b) {
@@ -424,7 +594,7 @@ int adacomp_server_set_validation(adacomp_server_t* s, int on) {
 }
 
 int adacomp_server_set_mode(adacomp_server_t* s, int mode) {
-    if (!s || mode < 0 || mode > 2) return ADACOMP_ERR_INVALID;
+    if (!s || mode < 0 || mode > 3) return ADACOMP_ERR_INVALID;
     s->mode = mode;
     return ADACOMP_OK;
 }
