@@ -18,8 +18,8 @@
  *     All device memory is owned by the caller.  The library never allocates
  *     device memory: handles carve their scratch out of the caller's workspace
  *     (size from the *_workspace_bytes calls, base aligned to 256 bytes), which
- *     must stay valid until the handle is destroyed.  Handles themselves and one
- *     small pinned staging area per server are host allocations of the library.
+ *     must stay valid until the handle is destroyed.  Handles themselves are small host
+ *     allocations of the library.
  *   - cuda_stream is a cudaStream_t passed as void* (NULL = the legacy default
  *     stream).  Device work is enqueued on it and the call returns without
  *     waiting.  Argument errors are returned at once, before anything is
@@ -127,9 +127,9 @@ ADACOMP_API int adacomp_select_host(adacomp_select_t* h, const float* h_grads, u
                         void* cuda_stream);
 
 /* Chooses how selections are computed; the results are identical.
- * 0 = automatic: tensors of at least 32768 entries with k <= n/4 take the bracketed route (a
+ * 0 = automatic: tensors of 32768 to 33.5 M entries with k <= n/4 take the bracketed route (a
  *     sample brackets the threshold, then the gradient is read once); instances whose bracket
- *     turns out wrong, and all other tensors, take the general route;
+ *     turns out wrong (or that hold a NaN), and all other tensors, take the general route;
  * 1 = general route for everything (multi-pass radix select; reads the gradient five times). */
 ADACOMP_API int adacomp_select_set_route(adacomp_select_t* h, int route);
 
@@ -256,8 +256,12 @@ ADACOMP_API int adacomp_server_timestamp(const adacomp_server_t* s, uint64_t* h_
  * ascending inside an update.  Off by default. */
 ADACOMP_API int adacomp_server_set_validation(adacomp_server_t* s, int on);
 /* Chooses how adacomp_apply maps work to the GPU; results are identical.
- * 0 = automatic, 1 = one launch per update, 2 = one launch per call in which each warp owns a
- * contiguous range of parameters and walks the updates in order. */
+ * 0 = automatic (by how many parameters the updates name);
+ * 1 = one launch per update, one thread per pair;
+ * 2 = up to 32 updates per launch, each warp owning a run of 1024-parameter ranges and walking
+ *     the updates in arrival order;
+ * 3 = up to 32 updates per launch, each block owning a run of ranges whose Theta and history
+ *     heads it keeps in shared memory while it applies the updates in arrival order. */
 ADACOMP_API int adacomp_server_set_mode(adacomp_server_t* s, int mode);
 /* Test hook: advances the history position counter as if `count` more pairs had been applied
  * (their history is empty).  Lets a test reach the 32-bit position re-basing that otherwise

@@ -5,13 +5,15 @@
 //   k_bracket_sample   per (worker, tensor): read a stratified sample, take two of its order
 //                      statistics t_lo <= t_hi chosen so that, with overwhelming probability,
 //                      #{key > t_hi} <= k <= #{key >= t_lo};
-//   k_bracket_scan     the single pass over the gradient.  Every warp works on its own: it
-//                      classifies 1024 consecutive entries, reserves room with one 64-bit atomic
-//                      and appends, in index order, the entries with key >= t_lo ("candidates",
-//                      about 1.1-2.5 k of them per tensor) to the instance's candidate list;
-//                      candidates with key <= t_hi (the "window", where the threshold must lie)
-//                      also go to a small unordered list; a table records where each 1024-entry
-//                      piece put its candidates and how many of them are above the window;
+//   k_bracket_scan     the single pass over the gradient (k_bracket_scan_dense for tensors where
+//                      a tenth or more of the entries are candidates).  Every warp works on its
+//                      own: it streams 1024-entry pieces, reserves room with one 64-bit atomic
+//                      per round of up to 8 pieces and appends, in index order, the entries with
+//                      key >= t_lo ("candidates", about 1.1-2.5 k of them per tensor) to the
+//                      instance's candidate list; candidates with key <= t_hi (the "window",
+//                      where the threshold must lie) also go to a small unordered list; a table
+//                      records where each piece put its candidates and how many of them are
+//                      above the window;
 //   k_bracket_resolve  per instance: verify the bracket with the exact counts, find the exact
 //                      threshold inside the window (radix select on (key, index) composites,
 //                      finished by brute force once few entries remain), count the kept window
@@ -177,15 +179,17 @@ __device__ __forceinline__ float max_nan(float a, float b) {
 //   Streaming.  The four magnitudes of a load are reduced to their maximum and compared once
 //   with t_lo (for non-NaN data |x| >= t as floats is the integer test on the key; a NaN
 //   propagates through the maximum and counts as a hit).  One ballot per load tells the warp
-//   whether any lane hit; only then do the hitting lanes classify their four entries and queue
-//   the load (its position and two 4-bit masks: candidates, window) in the warp's slice of
-//   shared memory, in index order.  As soon as a load has been tested its registers are refilled
-//   with the same load of the warp's next piece, so a warp always has 4 KB in flight.
-//   Tail, once per round (up to 8 pieces, fewer when the queue fills), with work proportional to
-//   the queued loads.  One 64-bit atomic reserves room in both lists for the whole round; the
-//   queue is then ranked with warp scans, the queued loads are fetched again (an L1 / L2 hit),
-//   and candidates and window entries are staged in shared memory and copied out with coalesced
-//   stores.
+//   whether any lane hit; the loads that hit are queued (their position only, 2 bytes) in the
+//   warp's slice of shared memory, in index order.  As soon as a load has been tested its
+//   registers are refilled with the same load of the warp's next piece, so a warp always has
+//   4 KB in flight.
+//   Tail, once per round (a round ends after 8 pieces, or earlier once ~100 loads are queued, so
+//   that what the tail fetches again is still in L1 / L2), with work proportional to the queued
+//   loads and every lane busy.  Pass A fetches the queued loads again, classifies their entries
+//   (candidate: key >= t_lo; window: also key <= t_hi; bounds-checked) and counts per piece.  One
+//   64-bit atomic then reserves room in both lists for the whole round.  Pass B ranks the queue
+//   with warp scans, stages candidates and window entries in shared memory and copies them out
+//   with coalesced stores; 8 lanes write the pieces' table entries.
 // The first and last piece of a tensor use checked loads.  A NaN hands the instance to the
 // general route, which works on bit patterns only.
 constexpr uint32_t kScanQueue = 768;                           // queued loads per warp and round
