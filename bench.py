@@ -33,6 +33,29 @@ METRIC = "dense-gradient GB/s scanned (select+compact, with the selected pairs a
 UNIT = "GB/s"
 FALLBACK_HBM_GBS = 6650.0
 
+# DRAM bytes (read + write) of ONE scan-kernel launch, from the ncu capture summarised in
+# profiles/dram_traffic_large_flat_w4.md: workload 4 with 4 workers, MB per keep fraction (1/10 is
+# the dense scan kernel).  A launch over W workers moves W / 4 times as much.  Only valid while
+# the kernel source is the one that was profiled.
+SCAN_TRAFFIC_W4_MB = {"1/1000": 1647.5, "1/400": 1686.0, "1/160": 1797.2, "1/64": 1789.0, "1/25": 1865.3, "1/10": 2013.6}
+SCAN_SOURCE_SHA256_16 = "58db70353905ced6"
+
+
+def scan_traffic_bytes(workload_index, keeps, workers):
+    """Mean DRAM bytes per scan launch over the given keep fractions, or None if unknown."""
+    import hashlib
+    try:
+        src = open(os.path.join(ROOT, "paper_1702_04683_b200", "csrc", "select_bracket.cuh"), "rb").read()
+    except OSError:
+        return None
+    if hashlib.sha256(src).hexdigest()[:16] != SCAN_SOURCE_SHA256_16 or workload_index != 4:
+        return None
+    try:
+        per = [SCAN_TRAFFIC_W4_MB["%d/%d" % k] * 1e6 * workers / 4.0 for k in keeps]
+    except KeyError:
+        return None
+    return sum(per) / len(per)
+
 
 def parse_args():
     ap = argparse.ArgumentParser()
@@ -284,7 +307,8 @@ def run_native(args):
                      "achieved": round(scan_bytes_all / scan_ms_all / 1e6, 1) if scan_ms_all else None,
                      "peak": peak, "peak_kind": "of " + peak_kind, "unit": "GB/s",
                      "frac": round(scan_bytes_all / scan_ms_all / 1e6 / peak, 4) if scan_ms_all else None,
-                     "traffic": None,
+                     "traffic": (lambda t: round(t / 1e9, 3) if t else None)(scan_traffic_bytes(args.workload, keeps, W)),
+                     "traffic_unit": "GB per launch (ncu dram read + write, mean over the keep fractions; algorithmic: %.1f GB)" % (W * 4.0 * P / 1e9),
                      "select_call": {"what": "all kernels of adacomp_select, read 4P + write 8K per worker",
                                      "achieved": round(sel_bytes_all / sel_ms_all / 1e6, 1),
                                      "frac": round(sel_bytes_all / sel_ms_all / 1e6 / peak, 4)}},
