@@ -256,12 +256,16 @@ ADACOMP_API int adacomp_server_timestamp(const adacomp_server_t* s, uint64_t* h_
  * ascending inside an update.  Off by default. */
 ADACOMP_API int adacomp_server_set_validation(adacomp_server_t* s, int on);
 /* Chooses how adacomp_apply maps work to the GPU; results are identical.
- * 0 = automatic (by how many parameters the updates name);
+ * 0 = automatic: per launch of up to 32 updates, 3 when the launch's pairs number a fifth of
+ *     the parameters or more, else 2; a single update goes as 1;
  * 1 = one launch per update, one thread per pair;
- * 2 = up to 32 updates per launch, each warp owning a run of 1024-parameter ranges and walking
- *     the updates in arrival order;
- * 3 = up to 32 updates per launch, each block owning a run of ranges whose Theta and history
- *     heads it keeps in shared memory while it applies the updates in arrival order. */
+ * 2 = up to 32 updates per launch; a block owns a run of parameter ranges sized to the updates'
+ *     density, sees all pairs of a range at once (one thread per pair) and keeps the order of
+ *     the updates per parameter;
+ * 3 = the same over a dense sweep: Theta and the history heads of every 1024-parameter range
+ *     are read and written back whole (needs Theta on a 16-byte boundary, else 2 is used).
+ * Updates whose pair slices overlap in memory, with d_sigma_out given, always go as 1: their
+ * staleness slots are shared and the later update's count must be the one that stays. */
 ADACOMP_API int adacomp_server_set_mode(adacomp_server_t* s, int mode);
 /* Test hook: advances the history position counter as if `count` more pairs had been applied
  * (their history is empty).  Lets a test reach the 32-bit position re-basing that otherwise

@@ -325,7 +325,7 @@ class Server:
         _check(_lib.adacomp_server_set_validation(self._h, int(on)), "adacomp_server_set_validation")
 
     def set_mode(self, mode: int):
-        """0 automatic, 1 one launch per update, 2 warp-owner batches, 3 block-owner batches."""
+        """0 automatic, 1 one launch per update, 2 batches by parameter ranges, 3 batches over a dense sweep."""
         _check(_lib.adacomp_server_set_mode(self._h, int(mode)), "adacomp_server_set_mode")
 
     def debug_skip_positions(self, count: int):

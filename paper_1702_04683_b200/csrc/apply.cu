@@ -11,7 +11,10 @@
 // walked from head[k] until it leaves the window, i.e. O(1 + sigma_k) instead of the one search
 // per remembered update of the paper's "Complexity" paragraph.  The host refuses updates whose
 // window start has been overwritten in the ring.
+#include <algorithm>
+#include <cmath>
 #include <new>
+#include <utility>
 #include <vector>
 
 #include "common.cuh"
@@ -78,232 +81,540 @@ k_apply_update(ServerParams sp, UpdateDesc u, const uint32_t* __restrict__ idx, 
 }
 
 // ---------------------------------------------------------------------------------------------
-// Several updates per launch ("owner computes").  The parameter vector is cut into ranges of
-// kRangeParams consecutive parameters; every warp owns a run of consecutive ranges and, range by
-// range, walks the updates of the batch IN ARRIVAL ORDER, applying the pairs that fall into the
-// range.  Every update's index list is ascending, so its pairs for a range are one contiguous
-// slice; lane b of the warp keeps update b's cursor, which only ever moves forward, so nothing
-// is searched except each cursor's starting point.  A parameter is only ever touched by the
-// warp that owns its range and sees its updates in arrival order, so the result is bit-identical
-// to one-launch-per-update application, with no synchronisation between warps.  The owner's
-// range of Theta / head stays in L1 / L2 across the updates of the batch, so DRAM sees each
-// touched sector once per batch instead of once per update.
-constexpr int kMaxBatch = 32;                  // updates per launch: one cursor per lane
-constexpr uint32_t kRangeParams = 1024;
+// Several updates per launch: what the kernels below are told about them.
+constexpr int kMaxBatch = 32;                  // updates per launch: one bit each in a parameter's mask
 
 struct BatchDesc {
     uint64_t pair_begin[kMaxBatch];
     uint32_t n_pairs[kMaxBatch];
     uint32_t pos_start[kMaxBatch];
     uint32_t win_start[kMaxBatch];
+    uint32_t win_bits[kMaxBatch];              // updates of this launch inside update b's window (bits below b)
+    uint32_t pre_mask;                         // bit b: update b's window starts before the launch
     uint32_t n_updates;
 };
 
-__global__ void __launch_bounds__(kApplyThreads)
-k_apply_batch(ServerParams sp, BatchDesc d, const uint32_t* __restrict__ idx, const float* __restrict__ val,
-              float lr, uint32_t* sigma_out, uint32_t n_ranges) {
-    const uint32_t lane = threadIdx.x & 31;
-    const uint32_t warp_global = blockIdx.x * (kApplyThreads / 32) + (threadIdx.x >> 5);
-    const uint32_t n_warps = gridDim.x * (kApplyThreads / 32);
-    const uint32_t r_lo = static_cast<uint32_t>(static_cast<uint64_t>(n_ranges) * warp_global / n_warps);
-    const uint32_t r_hi = static_cast<uint32_t>(static_cast<uint64_t>(n_ranges) * (warp_global + 1) / n_warps);
-    if (r_lo == r_hi) return;
-    const uint32_t B = d.n_updates;
-    // lane b: update b's description and its cursor = first pair with index >= the first owned parameter
-    const uint64_t my_begin = lane < B ? d.pair_begin[lane] : 0;
-    const uint32_t my_n = lane < B ? d.n_pairs[lane] : 0;
-    const uint32_t my_pos = lane < B ? d.pos_start[lane] : 0;
-    const uint32_t my_win = lane < B ? d.win_start[lane] : 0;
-    uint32_t cursor = 0;
-    {
-        const uint64_t first_param = static_cast<uint64_t>(r_lo) * kRangeParams;
-        uint32_t lo = 0, hi = my_n;                       // lower bound by bisection: at most 32 steps
-        while (lo < hi) {
-            const uint32_t mid = lo + ((hi - lo) >> 1);
-            if (idx[my_begin + mid] < first_param) lo = mid + 1; else hi = mid;
-        }
-        cursor = lo;
-    }
-    for (uint32_t r = r_lo; r < r_hi; ++r) {
-        const uint64_t range_end64 = static_cast<uint64_t>(r + 1) * kRangeParams;
-        const uint32_t range_end = range_end64 < sp.n_params ? static_cast<uint32_t>(range_end64)
-                                                             : static_cast<uint32_t>(sp.n_params);
-        for (uint32_t b = 0; b < B; ++b) {
-            const uint64_t begin = __shfl_sync(0xFFFFFFFFu, my_begin, b);
-            const uint32_t n_b = __shfl_sync(0xFFFFFFFFu, my_n, b);
-            const uint32_t pos_b = __shfl_sync(0xFFFFFFFFu, my_pos, b);
-            const uint32_t win_b = __shfl_sync(0xFFFFFFFFu, my_win, b);
-            uint32_t cur = __shfl_sync(0xFFFFFFFFu, cursor, b);
-            while (true) {
-                const uint32_t e = cur + lane;
-                uint32_t k = kNone;
-                if (e < n_b) k = idx[begin + e];
-                const bool mine = k < range_end;              // ascending list: the lanes that match form a prefix
-                if (mine) {
-                    if (sp.validate && e > 0 && idx[begin + e - 1] >= k) record_error(sp.status, ADACOMP_ERR_UNSORTED);
-                    apply_pair(sp, k, val[begin + e], pos_b + e, win_b, lr, sigma_out ? sigma_out + begin + e : nullptr);
-                }
-                const uint32_t took = __popc(__ballot_sync(0xFFFFFFFFu, mine));
-                cur += took;
-                if (took < 32) break;
-            }
-            if (lane == b) cursor = cur;
-            __syncwarp();                                     // update b's writes are visible before update b + 1 reads
-        }
-    }
-    // whoever owns the last range sees what no range claimed: indices >= n_params
-    if (r_hi == n_ranges && lane < B && cursor < my_n) record_error(sp.status, ADACOMP_ERR_UNSORTED);
-}
-
 // ---------------------------------------------------------------------------------------------
-// Several updates per launch, block-level owner ("owner block"), for batches that touch a good
-// part of the parameters.  A block owns a run of kOwnRange-parameter ranges.  Per range it loads
-// Theta and the history heads into shared memory (coalesced), then works in rounds: all warps
-// together stage, for every update of the batch at once, the next pairs of the range (so the
-// global loads of all updates overlap); the updates are then applied IN ARRIVAL ORDER out of
-// shared memory, one block barrier per update.  Only parameters below a limit are applied in a
-// round: the smallest index some update could not stage any more, so every update's pairs below
-// the limit are on chip.  Staleness inside the batch comes from a per-parameter bit mask of the
-// batch's updates that changed it (Eq. 3 restricted to the batch is a population count); the
-// part of a window that lies before the batch is counted by walking the chain from the head the
-// parameter had when the batch began.  Theta and heads of the range are written back once.
-// Same results, bit for bit, as one launch per update.
-constexpr uint32_t kOwnRange = 1024;
-constexpr uint32_t kOwnStage = 128;            // pairs staged per update and round
-constexpr int kOwnThreads = 256;
+// Several updates per launch, the block that owns a range of parameters sees all of its pairs at
+// once.  A block owns a run of ranges of `range` consecutive parameters.  Per range:
+//   stage    warp w loads, for updates w, w + 8, ..., the next <= 128 pairs from the update's
+//            cursor into shared memory (the loads of all updates are in flight together);
+//   scatter  every staged pair with a non-zero value sets bit b in the mask of its parameter
+//            (shared memory) and, if the table fits, records its slot under [b][parameter];
+//   pairs    ONE THREAD PER STAGED PAIR: Eq. 3 inside the batch is a population count of the mask
+//            under the update's window bits, the part of a window before the batch is a chain walk
+//            from the head the parameter had when the batch began; Eq. 5; the pair is linked behind
+//            the pair of the next lower bit (or the old head).  A pair that is its parameter's only
+//            change in the batch applies Eq. 4 at once (unless zero-valued pairs, which only read,
+//            are around); the others leave their step in shared memory and the pair of the
+//            highest bit lists the parameter;
+//   sums     one thread per listed parameter subtracts its steps in arrival order (Eq. 4 keeps its
+//            rounding order) and writes Theta and the head once.
+// No barrier separates the updates: the order is kept per parameter, which is all Algorithm 2
+// needs.  The limit of a round is the smallest index some update could not stage any more, so
+// every update's pairs below it are on chip; the range is finished in further rounds.  Same
+// results, bit for bit, as one launch per update.
+constexpr int kRgThreads = 256;
+constexpr uint32_t kRgStage = 128;             // pairs staged per update and round, at most
+constexpr uint32_t kRgChunks = kRgStage / 32;
+constexpr uint32_t kRgMinRange = 256, kRgMaxRange = 8192;
+constexpr uint32_t kRgLate = 0xFFFFu;          // staged slot that is not applied in this round
+constexpr uint32_t kRgAlphas = 33;             // alpha / sigma kept ready for sigma < 33
 
-struct OwnDesc {
-    BatchDesc b;
-    uint32_t win_bits[kMaxBatch];              // updates of this batch inside update b's window (bits below b)
-    uint32_t pre_mask;                         // bit b: update b's window starts before the batch
+struct RangeDesc {
+    BatchDesc o;
+    uint32_t range;                            // parameters per range, a multiple of 32
+    uint32_t chunks;                           // 32-pair chunks staged per update and round, 1..kRgChunks
+    uint32_t use_table;
 };
 
-constexpr size_t kOwnSmemBytes = kOwnRange * 16 + kMaxBatch * kOwnStage * 6 + kMaxBatch * 8 + 16;
+struct RgMeta {                                // per-update state in shared memory
+    uint64_t begin[kMaxBatch];
+    uint32_t n[kMaxBatch], pos[kMaxBatch], win[kMaxBatch], bits[kMaxBatch];
+    uint32_t cur[kMaxBatch], cnt[kMaxBatch], adv[kMaxBatch];
+    float alpha[kRgAlphas];
+    uint32_t limit, n_listed, any_zero;
+};
 
-__global__ void __launch_bounds__(kOwnThreads)
-k_apply_owner(ServerParams sp, OwnDesc d, const uint32_t* __restrict__ idx, const float* __restrict__ val,
-              float lr, uint32_t* sigma_out, uint32_t n_ranges) {
-    extern __shared__ __align__(16) unsigned char s_own[];
-    float* s_theta = reinterpret_cast<float*>(s_own);
-    uint32_t* s_head = reinterpret_cast<uint32_t*>(s_own + kOwnRange * 4);       // head when the batch began
-    uint32_t* s_last = reinterpret_cast<uint32_t*>(s_own + kOwnRange * 8);       // latest position set by the batch
-    uint32_t* s_mask = reinterpret_cast<uint32_t*>(s_own + kOwnRange * 12);      // updates of the batch that changed it
-    float* s_v = reinterpret_cast<float*>(s_own + kOwnRange * 16);                                    // [B][kOwnStage]
-    uint16_t* s_k = reinterpret_cast<uint16_t*>(s_own + kOwnRange * 16 + kMaxBatch * kOwnStage * 4);   // [B][kOwnStage]
-    uint32_t* s_cnt = reinterpret_cast<uint32_t*>(s_own + kOwnRange * 16 + kMaxBatch * kOwnStage * 6);
-    uint32_t* s_cur = s_cnt + kMaxBatch;
-    uint32_t* s_limit = s_cur + kMaxBatch;
+__host__ __device__ inline size_t rg_smem_bytes(uint32_t range, uint32_t n_updates, bool table) {
+    size_t b = static_cast<size_t>(range) * 4 + static_cast<size_t>(n_updates) * kRgStage * 4 + sizeof(RgMeta) +
+               static_cast<size_t>(n_updates) * kRgStage * 2 + static_cast<size_t>(range) * 2;
+    if (table) b += static_cast<size_t>(n_updates) * range;
+    return (b + 15) & ~static_cast<size_t>(15);
+}
+
+__global__ void __launch_bounds__(kRgThreads)
+k_apply_ranges(ServerParams sp, RangeDesc d, const uint32_t* __restrict__ idx, const float* __restrict__ val,
+               float lr, uint32_t* sigma_out, uint32_t n_ranges) {
+    extern __shared__ __align__(16) unsigned char s_rg[];
+    const uint32_t R = d.range, B = d.o.n_updates;
+    uint32_t* s_mask = reinterpret_cast<uint32_t*>(s_rg);                       // [R] updates that change the parameter
+    float* s_v = reinterpret_cast<float*>(s_mask + R);                          // [B][kRgStage] value, later the step
+    RgMeta* s_m = reinterpret_cast<RgMeta*>(s_v + B * kRgStage);
+    uint16_t* s_k = reinterpret_cast<uint16_t*>(s_m + 1);                       // [B][kRgStage] index - range start
+    uint16_t* s_list = s_k + B * kRgStage;                                      // [R] parameters changed more than once
+    uint8_t* s_tab = reinterpret_cast<uint8_t*>(s_list + R);                    // [B][R] slot of (update, parameter)
 
     const uint32_t tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-    const uint32_t B = d.b.n_updates;
     const uint32_t r_lo = static_cast<uint32_t>(static_cast<uint64_t>(n_ranges) * blockIdx.x / gridDim.x);
     const uint32_t r_hi = static_cast<uint32_t>(static_cast<uint64_t>(n_ranges) * (blockIdx.x + 1) / gridDim.x);
     if (r_lo == r_hi) return;
-    if (tid < B) {                                              // cursor: first pair at or above the first owned parameter
-        const uint64_t first_param = static_cast<uint64_t>(r_lo) * kOwnRange;
-        const uint64_t begin = d.b.pair_begin[tid];
-        uint32_t lo = 0, hi = d.b.n_pairs[tid];
+    if (tid < B) {
+        const uint64_t first_param = static_cast<uint64_t>(r_lo) * R;
+        const uint64_t begin = d.o.pair_begin[tid];
+        uint32_t lo = 0, hi = d.o.n_pairs[tid];               // cursor: first pair at or above the first owned parameter
         while (lo < hi) {
             const uint32_t mid = lo + ((hi - lo) >> 1);
             if (idx[begin + mid] < first_param) lo = mid + 1; else hi = mid;
         }
-        s_cur[tid] = lo;
+        s_m->cur[tid] = lo;
+        s_m->adv[tid] = 0;
+        s_m->begin[tid] = begin;
+        s_m->n[tid] = d.o.n_pairs[tid];
+        s_m->pos[tid] = d.o.pos_start[tid];
+        s_m->win[tid] = d.o.win_start[tid];
+        s_m->bits[tid] = d.o.win_bits[tid];
     }
+    if (tid >= 64 && tid < 64 + kRgAlphas) {                    // Eq. 5 for the small counts, once
+        const uint32_t sigma = tid - 64;
+        s_m->alpha[sigma] = sigma ? __fdiv_rn(lr, static_cast<float>(sigma)) : lr;
+    }
+    auto range_end = [&](uint32_t r) -> uint32_t {
+        const uint64_t e = (static_cast<uint64_t>(r) + 1) * R;
+        return e < sp.n_params ? static_cast<uint32_t>(e) : static_cast<uint32_t>(sp.n_params);
+    };
+    // the slot of update b's pair on parameter kl of the range
+    auto slot_of = [&](uint32_t b, uint32_t kl) -> uint32_t {
+        if (d.use_table) return s_tab[b * R + kl];
+        const uint32_t cnt = s_m->cnt[b];                       // update b's stage is ascending: bisection
+        uint32_t t = 0;
+#pragma unroll
+        for (uint32_t step = kRgStage / 2; step; step >>= 1)
+            if (t + step < cnt && s_k[b * kRgStage + t + step] <= kl) t += step;
+        return t;
+    };
+    if (tid == 0) s_m->limit = range_end(r_lo);
     __syncthreads();
 
-    for (uint32_t r = r_lo; r < r_hi; ++r) {
-        const uint32_t lo = r * kOwnRange;
-        const uint64_t hi64 = static_cast<uint64_t>(lo) + kOwnRange;
-        const uint32_t hi = hi64 < sp.n_params ? static_cast<uint32_t>(hi64) : static_cast<uint32_t>(sp.n_params);
-        for (uint32_t t = tid; t < kOwnRange; t += kOwnThreads) {
-            const bool in = lo + t < hi;
-            s_theta[t] = in ? sp.theta[lo + t] : 0.f;
-            s_head[t] = in ? sp.head[lo + t] : kNone;
-            s_last[t] = kNone;
-            s_mask[t] = 0;
-        }
-        while (true) {
-            if (tid == 0) *s_limit = hi;
-            __syncthreads();
-            // ---- stage: warp w takes updates w, w + 8, ...; 4 x 32 pairs each
-            for (uint32_t b = warp; b < B; b += kOwnThreads / 32) {
-                const uint64_t begin = d.b.pair_begin[b];
-                const uint32_t n_b = d.b.n_pairs[b], cur = s_cur[b];
-                uint32_t cnt = 0, last_k = 0;
+    uint32_t r = r_lo;
+    while (r < r_hi) {
+        const uint32_t lo = r * R, hi = range_end(r);
+        for (uint32_t t = tid; t < R / 4; t += kRgThreads) reinterpret_cast<uint4*>(s_mask)[t] = make_uint4(0, 0, 0, 0);
+        if (tid == 0) { s_m->n_listed = 0; s_m->any_zero = 0; }
+        // ---- stage
+        for (uint32_t b = warp; b < B; b += kRgThreads / 32) {
+            const uint64_t begin = s_m->begin[b];
+            const uint32_t n_b = s_m->n[b], cur = s_m->cur[b] + s_m->adv[b];     // past what the last round consumed
+            __syncwarp();
+            if (lane == 0) s_m->cur[b] = cur;
+            const uint32_t* ip = idx + begin + cur;
+            const float* vp = val + begin + cur;
+            const uint32_t left = n_b - cur;
+            uint32_t kk[kRgChunks];
+            float vv[kRgChunks];
 #pragma unroll
-                for (uint32_t c = 0; c < kOwnStage / 32; ++c) {
-                    const uint32_t t = c * 32 + lane, e = cur + t;
-                    uint32_t k = kNone;
-                    float v = 0.f;
-                    if (e < n_b) {                              // both loads at once: the value does not wait for the index
-                        k = idx[begin + e];
-                        v = val[begin + e];
-                    }
-                    const bool mine = k < hi;                   // ascending list: matching slots form a prefix
-                    if (mine) {
-                        if (sp.validate && e > 0 && idx[begin + e - 1] >= k) record_error(sp.status, ADACOMP_ERR_UNSORTED);
-                        s_k[b * kOwnStage + t] = static_cast<uint16_t>(k - lo);
-                        s_v[b * kOwnStage + t] = v;
-                    }
-                    cnt += __popc(__ballot_sync(0xFFFFFFFFu, mine));
-                    if (c == kOwnStage / 32 - 1) last_k = __shfl_sync(0xFFFFFFFFu, k, 31);
-                }
-                if (lane == 0) {
-                    s_cnt[b] = cnt;
-                    if (cnt == kOwnStage) atomicMin(s_limit, last_k + 1);   // more of this update may follow in the range
+            for (uint32_t c = 0; c < kRgChunks; ++c) {          // every load first: none waits for another
+                const uint32_t t = c * 32 + lane;
+                kk[c] = kNone;
+                vv[c] = 0.f;
+                if (c < d.chunks && t < left) {
+                    kk[c] = ip[t];
+                    vv[c] = vp[t];
                 }
             }
-            __syncthreads();
-            const uint32_t limit = *s_limit;
-            // ---- apply, update after update
-            for (uint32_t b = 0; b < B; ++b) {
-                const uint32_t cnt = s_cnt[b];
-                if (cnt == 0) continue;                         // nothing of update b in this round (same for all threads)
+            uint32_t cnt = 0, last_k = 0;
+            bool run = true;                                    // staged = the leading slots below the range's end
+#pragma unroll
+            for (uint32_t c = 0; c < kRgChunks; ++c) {
+                const uint32_t t = c * 32 + lane, k = kk[c];
+                const bool in = k < hi;
+                if (in) {
+                    if (sp.validate && cur + t > 0 && ip[static_cast<int64_t>(t) - 1] >= k) record_error(sp.status, ADACOMP_ERR_UNSORTED);
+                    s_k[b * kRgStage + t] = k >= lo ? static_cast<uint16_t>(k - lo) : static_cast<uint16_t>(kRgLate);
+                    s_v[b * kRgStage + t] = vv[c];
+                }
+                const uint32_t bal = __ballot_sync(0xFFFFFFFFu, in);
+                if (run) {
+                    if (bal == 0xFFFFFFFFu) cnt += 32; else { cnt += __ffs(~bal) - 1; run = false; }
+                }
+                if (c + 1 == d.chunks) last_k = __shfl_sync(0xFFFFFFFFu, k, 31);
+            }
+            if (lane == 0) {
+                s_m->cnt[b] = cnt;
+                if (cnt == d.chunks * 32) atomicMin(&s_m->limit, last_k + 1);   // more of this update may follow in the range
+            }
+        }
+        __syncthreads();
+        const uint32_t limit = s_m->limit;
+        // ---- scatter: bit b on every parameter update b changes below the limit
+        for (uint32_t b = warp; b < B; b += kRgThreads / 32) {
+            const uint32_t cnt = s_m->cnt[b];
+            uint32_t adv = 0;
+            for (uint32_t t = lane; t < ((cnt + 31) & ~31u); t += 32) {
                 bool take = false;
-                if (tid < cnt) {
-                    const uint32_t kl = s_k[b * kOwnStage + tid];
-                    take = lo + kl < limit;
-                    if (take) {
-                        const float v = s_v[b * kOwnStage + tid];
-                        const uint32_t e = s_cur[b] + tid;
-                        const uint32_t m = s_mask[kl], ho = s_head[kl];
-                        uint32_t sigma = __popc(m & d.win_bits[b]);
-                        if ((d.pre_mask >> b) & 1u) {           // the part of the window before the batch
-                            uint32_t q = ho, hops = 0;
-                            const uint32_t ws = d.b.win_start[b];
+                if (t < cnt) {
+                    const uint32_t kl = s_k[b * kRgStage + t];
+                    if (kl == kRgLate) {                        // an index before the range: the list was not ascending
+                        record_error(sp.status, ADACOMP_ERR_UNSORTED);
+                        take = true;                            // consumed, not applied
+                    } else if (lo + kl < limit) {
+                        take = true;
+                        if (s_v[b * kRgStage + t] != 0.0f) {    // Eq. 3 counts changes: a zero entry is not one
+                            atomicOr(&s_mask[kl], 1u << b);
+                            if (d.use_table) s_tab[b * R + kl] = static_cast<uint8_t>(t);
+                        } else {
+                            s_m->any_zero = 1;                  // somebody may only read a parameter another pair changes
+                        }
+                    } else {
+                        s_k[b * kRgStage + t] = static_cast<uint16_t>(kRgLate);   // a later round's
+                    }
+                }
+                adv += __popc(__ballot_sync(0xFFFFFFFFu, take));
+            }
+            if (lane == 0) s_m->adv[b] = adv;
+        }
+        __syncthreads();
+        if (tid == 0) s_m->limit = limit < hi ? hi : (r + 1 < r_hi ? range_end(r + 1) : hi);   // for the next round
+        // ---- pairs: one thread per staged pair.  Heads and Theta are only written at once where no other
+        // pair of the round looks at the parameter: never while a zero-valued pair is around
+        const bool at_once = s_m->any_zero == 0;
+        for (uint32_t b = warp; b < B; b += kRgThreads / 32) {
+            const uint32_t cnt = s_m->adv[b];                   // ascending list: the pairs below the limit lead
+            const uint32_t cur_b = s_m->cur[b], pos_b = s_m->pos[b] + cur_b, bits_b = s_m->bits[b];
+            const uint32_t below_b = (1u << b) - 1u, ws = s_m->win[b];
+            const bool pre_b = (d.o.pre_mask >> b) & 1u;
+            uint32_t* sig = sigma_out ? sigma_out + s_m->begin[b] + cur_b : nullptr;
+            uint32_t kl[kRgChunks], m[kRgChunks], h0[kRgChunks];
+            float th[kRgChunks];
+#pragma unroll
+            for (uint32_t c = 0; c < kRgChunks; ++c) {          // every load first
+                const uint32_t t = c * 32 + lane;
+                kl[c] = kRgLate;
+                m[c] = 0;
+                h0[c] = kNone;
+                th[c] = 0.f;
+                if (t < cnt) kl[c] = s_k[b * kRgStage + t];
+                if (kl[c] != kRgLate) {
+                    m[c] = s_mask[kl[c]];
+                    h0[c] = sp.head[lo + kl[c]];
+                    th[c] = sp.theta[lo + kl[c]];
+                }
+            }
+#pragma unroll
+            for (uint32_t c = 0; c < kRgChunks; ++c) {
+                const uint32_t t = c * 32 + lane;
+                bool top = false;                               // this pair is the last of several changes of its parameter
+                if (kl[c] != kRgLate) {
+                    const float v = s_v[b * kRgStage + t];
+                    uint32_t sigma = __popc(m[c] & bits_b);                                            // Eq. 3, inside the batch
+                    if (pre_b) {                                                                       // Eq. 3, before the batch
+                        uint32_t q = h0[c], hops = 0;
+                        while (q != kNone && q >= ws) {
+                            if (++hops > sp.max_window) { record_error(sp.status, ADACOMP_ERR_WINDOW); break; }
+                            q = sp.prev[(q + sp.ring_shift) & sp.ring_mask];
+                        }
+                        sigma += hops;
+                    }
+                    if (sig) sig[t] = sigma;
+                    if (v != 0.0f) {
+                        const float alpha_k = sigma < kRgAlphas ? s_m->alpha[sigma] : __fdiv_rn(lr, static_cast<float>(sigma));   // Eq. 5
+                        const float step = __fmul_rn(alpha_k, v);
+                        const uint32_t pos = pos_b + t, low = m[c] & below_b;
+                        uint32_t before = h0[c];                // the pair that changed the parameter last
+                        if (low) {
+                            const uint32_t b2 = 31 - __clz(low);
+                            before = s_m->pos[b2] + s_m->cur[b2] + slot_of(b2, kl[c]);
+                        }
+                        sp.prev[(pos + sp.ring_shift) & sp.ring_mask] = before;
+                        if (at_once && m[c] == (1u << b)) {     // the parameter's only change in this batch
+                            sp.theta[lo + kl[c]] = __fsub_rn(th[c], step);                             // Eq. 4
+                            sp.head[lo + kl[c]] = pos;
+                        } else {
+                            s_v[b * kRgStage + t] = step;
+                            top = (m[c] >> b) == 1u;
+                        }
+                    }
+                }
+                const uint32_t bal = __ballot_sync(0xFFFFFFFFu, top);
+                if (bal) {
+                    uint32_t base = 0;
+                    if (lane == 0) base = atomicAdd(&s_m->n_listed, __popc(bal));
+                    base = __shfl_sync(0xFFFFFFFFu, base, 0);
+                    if (top) s_list[base + __popc(bal & ((1u << lane) - 1u))] = static_cast<uint16_t>(kl[c]);
+                }
+            }
+        }
+        __syncthreads();
+        // ---- sums: one thread per parameter changed more than once, its steps in arrival order
+        const uint32_t n_listed = s_m->n_listed;
+        for (uint32_t j = tid; j < n_listed; j += kRgThreads) {
+            const uint32_t kl = s_list[j];
+            uint32_t m = s_mask[kl], t = 0, b = 0;
+            float theta = sp.theta[lo + kl];
+            while (m) {
+                b = __ffs(m) - 1;
+                m &= m - 1;
+                t = slot_of(b, kl);
+                theta = __fsub_rn(theta, s_v[b * kRgStage + t]);                                       // Eq. 4
+            }
+            sp.theta[lo + kl] = theta;
+            sp.head[lo + kl] = s_m->pos[b] + s_m->cur[b] + t;
+        }
+        __syncthreads();
+        if (limit >= hi) ++r;                                   // else: the rest of the range in another round
+    }
+    // whoever owns the last range sees what no range claimed: indices >= n_params
+    if (r_hi == n_ranges && tid < B && s_m->cur[tid] + s_m->adv[tid] < s_m->n[tid]) record_error(sp.status, ADACOMP_ERR_UNSORTED);
+}
+
+// ---------------------------------------------------------------------------------------------
+// Several updates per launch over a dense sweep of the parameters, for batches that touch a good
+// part of every 32-byte sector of Theta anyway.  A block owns a run of ranges of kSwRange
+// consecutive parameters, thread t the four parameters 4t .. 4t + 3 of the range.  Per range:
+//   sweep    Theta of the range goes into registers and its heads into shared memory with one
+//            16-byte load each per thread;
+//   stage    warp w loads, for updates w, w + 8, ..., the next <= 128 pairs from the update's
+//            cursor (the loads of all updates and of the sweep are in flight together), keeps
+//            them in shared memory and sets, for every non-zero pair, bit b in the mask of its
+//            parameter and its slot in a table under [b][parameter];
+//   pairs    ONE THREAD PER STAGED PAIR below the round's limit: Eq. 3 inside the batch is a
+//            population count of the mask under the update's window bits, the part of a window
+//            before the batch a chain walk from the head the parameter had when the batch began;
+//            Eq. 5; the pair leaves its step alpha_k * value in shared memory and is linked behind
+//            the pair of the next lower bit (or the old head);
+//   sums     every thread subtracts, for its four parameters, the steps in arrival order (Eq. 4
+//            keeps its rounding order) and remembers the new head;
+//   finally Theta and the heads of the range are written back, 16 bytes per thread, where changed.
+// No barrier separates the updates: the order is kept per parameter, which is all Algorithm 2
+// needs.  The limit of a round is the smallest index some update could not stage any more, so
+// every update's pairs below it are on chip; the range is finished in further rounds.  Same
+// results, bit for bit, as one launch per update.
+constexpr uint32_t kSwRange = 1024;
+constexpr int kSwThreads = kSwRange / 4;
+
+struct SweepDesc {
+    BatchDesc o;
+    uint32_t chunks;                           // 32-pair chunks staged per update and round, 1..kRgChunks
+};
+
+__host__ __device__ inline size_t sw_smem_bytes(uint32_t n_updates) {
+    return kSwRange * 8 + static_cast<size_t>(n_updates) * kRgStage * 6 + sizeof(RgMeta) +
+           static_cast<size_t>(n_updates) * kSwRange;
+}
+
+__global__ void __launch_bounds__(kSwThreads)
+k_apply_sweep(ServerParams sp, SweepDesc d, const uint32_t* __restrict__ idx, const float* __restrict__ val,
+              float lr, uint32_t* sigma_out, uint32_t n_ranges) {
+    extern __shared__ __align__(16) unsigned char s_sw[];
+    const uint32_t B = d.o.n_updates;
+    uint32_t* s_mask = reinterpret_cast<uint32_t*>(s_sw);                       // [range] updates that change the parameter
+    uint32_t* s_head = s_mask + kSwRange;                                       // [range] head when the batch began
+    float* s_v = reinterpret_cast<float*>(s_head + kSwRange);                   // [B][kRgStage] value, later the step
+    RgMeta* s_m = reinterpret_cast<RgMeta*>(s_v + B * kRgStage);
+    uint16_t* s_k = reinterpret_cast<uint16_t*>(s_m + 1);                       // [B][kRgStage] index - range start
+    uint8_t* s_tab = reinterpret_cast<uint8_t*>(s_k + B * kRgStage);            // [B][range] slot of (update, parameter)
+
+    const uint32_t tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const uint32_t r_lo = static_cast<uint32_t>(static_cast<uint64_t>(n_ranges) * blockIdx.x / gridDim.x);
+    const uint32_t r_hi = static_cast<uint32_t>(static_cast<uint64_t>(n_ranges) * (blockIdx.x + 1) / gridDim.x);
+    if (r_lo == r_hi) return;
+    if (tid < B) {
+        const uint64_t first_param = static_cast<uint64_t>(r_lo) * kSwRange;
+        const uint64_t begin = d.o.pair_begin[tid];
+        uint32_t lo = 0, hi = d.o.n_pairs[tid];               // cursor: first pair at or above the first owned parameter
+        while (lo < hi) {
+            const uint32_t mid = lo + ((hi - lo) >> 1);
+            if (idx[begin + mid] < first_param) lo = mid + 1; else hi = mid;
+        }
+        s_m->cur[tid] = lo;
+        s_m->adv[tid] = 0;
+        s_m->begin[tid] = begin;
+        s_m->n[tid] = d.o.n_pairs[tid];
+        s_m->win[tid] = d.o.win_start[tid];
+        s_m->bits[tid] = d.o.win_bits[tid];
+    }
+    if (tid >= 64 && tid < 64 + kRgAlphas) {                    // Eq. 5 for the small counts, once
+        const uint32_t sigma = tid - 64;
+        s_m->alpha[sigma] = sigma ? __fdiv_rn(lr, static_cast<float>(sigma)) : lr;
+    }
+    auto range_end = [&](uint32_t r) -> uint32_t {
+        const uint64_t e = (static_cast<uint64_t>(r) + 1) * kSwRange;
+        return e < sp.n_params ? static_cast<uint32_t>(e) : static_cast<uint32_t>(sp.n_params);
+    };
+    if (tid == 0) s_m->limit = range_end(r_lo);
+    reinterpret_cast<uint4*>(s_mask)[tid] = make_uint4(0, 0, 0, 0);
+    __syncthreads();
+
+    uint32_t r = r_lo, changed = 0;                             // bit j: parameter 4 tid + j of the range got a new head
+    bool fresh = true;                                          // first round of the range
+    float th[4] = {0.f, 0.f, 0.f, 0.f};
+    uint32_t nh[4] = {kNone, kNone, kNone, kNone};
+    while (r < r_hi) {
+        const uint32_t lo = r * kSwRange, hi = range_end(r);
+        const uint32_t mine = lo + 4 * tid;
+        const bool whole = mine + 4 <= hi;                      // all four parameters exist
+        uint4 h4 = make_uint4(kNone, kNone, kNone, kNone);
+        if (fresh) {                                            // ---- sweep
+            changed = 0;
+            if (whole) {
+                h4 = *reinterpret_cast<const uint4*>(sp.head + mine);
+                const float4 t4 = *reinterpret_cast<const float4*>(sp.theta + mine);
+                th[0] = t4.x; th[1] = t4.y; th[2] = t4.z; th[3] = t4.w;
+            } else {
+                uint32_t hh[4] = {kNone, kNone, kNone, kNone};
+#pragma unroll
+                for (uint32_t j = 0; j < 4; ++j)
+                    if (mine + j < hi) { hh[j] = sp.head[mine + j]; th[j] = sp.theta[mine + j]; }
+                h4 = make_uint4(hh[0], hh[1], hh[2], hh[3]);
+            }
+        }
+        // ---- stage
+        for (uint32_t b = warp; b < B; b += kSwThreads / 32) {
+            const uint64_t begin = s_m->begin[b];
+            const uint32_t n_b = s_m->n[b], cur = s_m->cur[b] + s_m->adv[b];     // past what the last round consumed
+            __syncwarp();
+            if (lane == 0) {
+                s_m->cur[b] = cur;
+                s_m->pos[b] = d.o.pos_start[b] + cur;         // position of the pair in slot 0
+            }
+            const uint32_t* ip = idx + begin + cur;
+            const float* vp = val + begin + cur;
+            const uint32_t left = n_b - cur;
+            uint32_t kk[kRgChunks];
+            float vv[kRgChunks];
+#pragma unroll
+            for (uint32_t c = 0; c < kRgChunks; ++c) {          // every load first: none waits for another
+                const uint32_t t = c * 32 + lane;
+                kk[c] = kNone;
+                vv[c] = 0.f;
+                if (c < d.chunks && t < left) {
+                    kk[c] = ip[t];
+                    vv[c] = vp[t];
+                }
+            }
+            uint32_t cnt = 0, last_k = 0;
+            bool run = true;                                    // staged = the leading slots below the range's end
+#pragma unroll
+            for (uint32_t c = 0; c < kRgChunks; ++c) {
+                const uint32_t t = c * 32 + lane, k = kk[c];
+                const bool in = k < hi;
+                if (in) {
+                    if (sp.validate && cur + t > 0 && ip[static_cast<int64_t>(t) - 1] >= k) record_error(sp.status, ADACOMP_ERR_UNSORTED);
+                    const uint32_t kl = k - lo;
+                    s_v[b * kRgStage + t] = vv[c];
+                    if (k >= lo) {
+                        s_k[b * kRgStage + t] = static_cast<uint16_t>(kl);
+                        if (vv[c] != 0.0f) {                    // Eq. 3 counts changes: a zero entry is not one
+                            atomicOr(&s_mask[kl], 1u << b);
+                            s_tab[b * kSwRange + kl] = static_cast<uint8_t>(t);
+                        }
+                    } else {                                    // an index before the range: the list was not ascending
+                        s_k[b * kRgStage + t] = static_cast<uint16_t>(kRgLate);
+                        record_error(sp.status, ADACOMP_ERR_UNSORTED);
+                    }
+                }
+                const uint32_t bal = __ballot_sync(0xFFFFFFFFu, in);
+                if (run) {
+                    if (bal == 0xFFFFFFFFu) cnt += 32; else { cnt += __ffs(~bal) - 1; run = false; }
+                }
+                if (c + 1 == d.chunks) last_k = __shfl_sync(0xFFFFFFFFu, k, 31);
+            }
+            if (lane == 0) {
+                s_m->cnt[b] = cnt;
+                if (cnt == d.chunks * 32) atomicMin(&s_m->limit, last_k + 1);   // more of this update may follow in the range
+            }
+        }
+        if (fresh) reinterpret_cast<uint4*>(s_head)[tid] = h4;
+        __syncthreads();
+        const uint32_t limit = s_m->limit;
+        // ---- pairs: one thread per staged pair below the limit
+        for (uint32_t b = warp; b < B; b += kSwThreads / 32) {
+            const uint32_t cnt = s_m->cnt[b], pos_b = s_m->pos[b], bits_b = s_m->bits[b];
+            const uint32_t below_b = (1u << b) - 1u, ws = s_m->win[b];
+            const bool pre_b = (d.o.pre_mask >> b) & 1u;
+            uint32_t* sig = sigma_out ? sigma_out + s_m->begin[b] + s_m->cur[b] : nullptr;
+            uint32_t adv = 0;
+            for (uint32_t t = lane; t < ((cnt + 31) & ~31u); t += 32) {
+                bool take = false;
+                if (t < cnt) {
+                    const uint32_t kl = s_k[b * kRgStage + t];
+                    take = kl == kRgLate || lo + kl < limit;    // consumed in this round (ascending list: these lead)
+                    if (take && kl != kRgLate) {
+                        const float v = s_v[b * kRgStage + t];
+                        const uint32_t m = s_mask[kl], h0 = s_head[kl];
+                        uint32_t sigma = __popc(m & bits_b);                                           // Eq. 3, inside the batch
+                        if (pre_b) {                                                                   // Eq. 3, before the batch
+                            uint32_t q = h0, hops = 0;
                             while (q != kNone && q >= ws) {
                                 if (++hops > sp.max_window) { record_error(sp.status, ADACOMP_ERR_WINDOW); break; }
                                 q = sp.prev[(q + sp.ring_shift) & sp.ring_mask];
                             }
                             sigma += hops;
                         }
-                        if (sigma_out) sigma_out[d.b.pair_begin[b] + e] = sigma;
-                        if (v != 0.0f) {                        // Eq. 3 counts changes: a zero entry is not one
-                            const float alpha_k = sigma ? __fdiv_rn(lr, static_cast<float>(sigma)) : lr;      // Eq. 5
-                            s_theta[kl] = __fsub_rn(s_theta[kl], __fmul_rn(alpha_k, v));                       // Eq. 4
-                            const uint32_t pos = d.b.pos_start[b] + e;
-                            sp.prev[(pos + sp.ring_shift) & sp.ring_mask] = m ? s_last[kl] : ho;
-                            s_last[kl] = pos;
-                            s_mask[kl] = m | (1u << b);
+                        if (sig) sig[t] = sigma;
+                        if (v != 0.0f) {
+                            const float alpha_k = sigma < kRgAlphas ? s_m->alpha[sigma] : __fdiv_rn(lr, static_cast<float>(sigma));   // Eq. 5
+                            s_v[b * kRgStage + t] = __fmul_rn(alpha_k, v);
+                            const uint32_t low = m & below_b;
+                            uint32_t before = h0;               // the pair that changed the parameter last
+                            if (low) {
+                                const uint32_t b2 = 31 - __clz(low);
+                                before = s_m->pos[b2] + s_tab[b2 * kSwRange + kl];
+                            }
+                            sp.prev[(pos_b + t + sp.ring_shift) & sp.ring_mask] = before;
                         }
                     }
                 }
-                const uint32_t took = __syncthreads_count(take);   // also orders update b before update b + 1
-                if (tid == 0) s_cur[b] += took;
+                adv += __popc(__ballot_sync(0xFFFFFFFFu, take));
             }
-            __syncthreads();
-            if (limit >= hi) break;                             // every update's pairs of the range are done
+            if (lane == 0) s_m->adv[b] = adv;
         }
-        for (uint32_t t = tid; t < kOwnRange; t += kOwnThreads) {
-            if (lo + t < hi && s_mask[t]) {
-                sp.theta[lo + t] = s_theta[t];
-                sp.head[lo + t] = s_last[t];
+        __syncthreads();
+        const bool done = limit >= hi;                          // else: the rest of the range in another round
+        if (tid == 0) s_m->limit = !done ? hi : (r + 1 < r_hi ? range_end(r + 1) : hi);   // for the next round
+        // ---- sums: the steps of each parameter in arrival order
+        {
+            const uint4 m4 = reinterpret_cast<const uint4*>(s_mask)[tid];
+            reinterpret_cast<uint4*>(s_mask)[tid] = make_uint4(0, 0, 0, 0);     // empty for the next round's stage
+            const uint32_t mm[4] = {m4.x, m4.y, m4.z, m4.w};
+#pragma unroll
+            for (uint32_t j = 0; j < 4; ++j) {
+                uint32_t m = mm[j];
+                const uint32_t kl = 4 * tid + j;
+                if (m && lo + kl < limit) {
+                    uint32_t b = 0, t = 0;
+                    do {
+                        b = __ffs(m) - 1;
+                        m &= m - 1;
+                        t = s_tab[b * kSwRange + kl];
+                        th[j] = __fsub_rn(th[j], s_v[b * kRgStage + t]);                               // Eq. 4
+                    } while (m);
+                    nh[j] = s_m->pos[b] + t;
+                    changed |= 1u << j;
+                }
+            }
+        }
+        if (done && changed) {                                  // ---- write back
+            const uint4 o4 = reinterpret_cast<const uint4*>(s_head)[tid];
+            const uint32_t oh[4] = {o4.x, o4.y, o4.z, o4.w};
+            uint32_t wh[4];
+#pragma unroll
+            for (uint32_t j = 0; j < 4; ++j) wh[j] = (changed >> j) & 1u ? nh[j] : oh[j];
+            if (whole) {
+                *reinterpret_cast<uint4*>(sp.head + mine) = make_uint4(wh[0], wh[1], wh[2], wh[3]);
+                *reinterpret_cast<float4*>(sp.theta + mine) = make_float4(th[0], th[1], th[2], th[3]);
+            } else {
+#pragma unroll
+                for (uint32_t j = 0; j < 4; ++j)
+                    if ((changed >> j) & 1u) { sp.head[mine + j] = wh[j]; sp.theta[mine + j] = th[j]; }
             }
         }
         __syncthreads();
+        fresh = done;
+        if (done) ++r;
     }
     // whoever owns the last range sees what no range claimed: indices >= n_params
-    if (r_hi == n_ranges && tid < B && s_cur[tid] < d.b.n_pairs[tid]) record_error(sp.status, ADACOMP_ERR_UNSORTED);
+    if (r_hi == n_ranges && tid < B && s_m->cur[tid] + s_m->adv[tid] < s_m->n[tid]) record_error(sp.status, ADACOMP_ERR_UNSORTED);
 }
 
 // Moves every stored position down by `delta` (entries older than that become kNone).
@@ -393,7 +704,11 @@ int adacomp_server_create(adacomp_server_t** out, uint64_t n_params, uint64_t hi
     if (e == cudaSuccess) e = cudaDeviceGetAttribute(&s->n_sms, cudaDevAttrMultiProcessorCount, device);
     if (e == cudaSuccess) e = cudaMemset(s->d_status, 0, sizeof(int));
     if (e == cudaSuccess)
-        e = cudaFuncSetAttribute(k_apply_owner, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(kOwnSmemBytes));
+        e = cudaFuncSetAttribute(k_apply_ranges, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                 static_cast<int>(rg_smem_bytes(kRgMaxRange, kMaxBatch, false) + 32768));   // + the largest slot table
+    if (e == cudaSuccess)
+        e = cudaFuncSetAttribute(k_apply_sweep, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                 static_cast<int>(sw_smem_bytes(kMaxBatch)));
     if (e == cudaSuccess) e = cudaDeviceSynchronize();
     if (e != cudaSuccess) { delete s; return cuda_fail(e); }
     *out = s;
@@ -483,63 +798,95 @@ int adacomp_apply(adacomp_server_t* s, const uint32_t* d_idx, const float* d_val
     sp.max_window = s->max_window;
     sp.validate = s->validate;
 
-    // one launch per update, or owner-computes launches of up to kMaxBatch updates: same results
-    // (automatic: the batched kernel pays off when an update names between about 0.2 % and 6 % of
-    // the parameters; sparser updates are launch-bound either way, denser ones keep DRAM busy alone)
-    const double density = static_cast<double>(call_pairs) / n_updates / static_cast<double>(s->n_params);
-    // (automatic: when the updates of a launch (up to 32) together name about half as many pairs as
-    // there are parameters, the block owner kernel, which sweeps Theta once per launch; else the warp
-    // owner kernel for updates that name 0.2 % - 6 % of the parameters; else one launch per update)
-    const uint32_t per_launch = n_updates < kMaxBatch ? n_updates : kMaxBatch;
-    const bool owner = s->mode == 3 || (s->mode == 0 && n_updates >= 2 && density * per_launch >= 0.4);
-    const bool batched = !owner && (s->mode == 2 || (s->mode == 0 && n_updates >= 2 && density >= 0.002 && density <= 0.06));
-    if (owner || batched) {
-        const uint32_t n_ranges = static_cast<uint32_t>((s->n_params + kRangeParams - 1) / kRangeParams);   // kOwnRange == kRangeParams
-        uint64_t want_warps = static_cast<uint64_t>(s->n_sms) * 64;            // 64 resident warps per SM
-        if (want_warps > n_ranges) want_warps = n_ranges;
-        const unsigned grid = static_cast<unsigned>((want_warps + kApplyThreads / 32 - 1) / (kApplyThreads / 32));
-        unsigned own_grid = static_cast<unsigned>(s->n_sms) * 5;
-        if (own_grid > n_ranges) own_grid = n_ranges;
-        for (uint32_t b0 = 0; b0 < n_updates; b0 += kMaxBatch) {
-            OwnDesc od;
-            BatchDesc& d = od.b;
-            d.n_updates = (n_updates - b0 < kMaxBatch) ? n_updates - b0 : kMaxBatch;
-            od.pre_mask = 0;
-            uint64_t pairs = 0;
-            for (uint32_t b = 0; b < d.n_updates; ++b) {
-                d.pair_begin[b] = h_pair_begin[b0 + b];
-                d.n_pairs[b] = h_pair_count[b0 + b];
-                d.pos_start[b] = static_cast<uint32_t>(start_abs[b0 + b] - s->pos_base);
-                d.win_start[b] = static_cast<uint32_t>(win_abs[b0 + b] - s->pos_base);
-                pairs += h_pair_count[b0 + b];
-                // which updates of this launch lie in update b's window [j, i - 1]
-                const uint64_t ts0 = i0 + b0, j = h_pull_ts[b0 + b];
-                const uint32_t first_in = j > ts0 ? static_cast<uint32_t>(j - ts0) : 0u;     // <= b
-                od.win_bits[b] = ((1u << b) - 1u) & ~((1u << first_in) - 1u);
-                if (j < ts0) od.pre_mask |= 1u << b;
-            }
-            for (uint32_t b = d.n_updates; b < kMaxBatch; ++b) od.win_bits[b] = 0;
-            if (!pairs) continue;
-            if (owner) {
-                k_apply_owner<<<own_grid, kOwnThreads, kOwnSmemBytes, st>>>(sp, od, d_idx, d_val, lr, d_sigma_out, n_ranges);
-            } else {
-                k_apply_batch<<<grid, kApplyThreads, 0, st>>>(sp, d, d_idx, d_val, lr, d_sigma_out, n_ranges);
-            }
-            ADACOMP_LAUNCH_CHECK();
+    // ---- launches.  One launch per update, or launches of up to kMaxBatch updates each: same results.
+    // Automatic choice per launch: the sweep kernel when the launch's pairs number a fifth of the parameters or
+    // more (nearly every 32-byte sector of Theta is touched anyway), else the ranges kernel; a single update,
+    // and updates whose staleness slots overlap in memory, go one per launch.
+    bool shared_slots = false;                 // two updates write their counts to the same slots: order matters
+    if (d_sigma_out && n_updates > 1 && s->mode != 1) {
+        std::vector<std::pair<uint64_t, uint64_t>> slices;
+        for (uint32_t b = 0; b < n_updates; ++b)
+            if (h_pair_count[b]) slices.emplace_back(h_pair_begin[b], h_pair_begin[b] + h_pair_count[b]);
+        std::sort(slices.begin(), slices.end());
+        for (size_t a = 1; a < slices.size(); ++a)
+            if (slices[a].first < slices[a - 1].second) { shared_slots = true; break; }
+    }
+    const bool one_by_one = s->mode == 1 || shared_slots || (s->mode == 0 && n_updates == 1);
+    const bool theta_aligned = reinterpret_cast<uintptr_t>(s->d_theta) % 16 == 0;
+    for (uint32_t b0 = 0; b0 < n_updates && !one_by_one; b0 += kMaxBatch) {
+        BatchDesc d;
+        d.n_updates = (n_updates - b0 < kMaxBatch) ? n_updates - b0 : kMaxBatch;
+        d.pre_mask = 0;
+        uint64_t pairs = 0;
+        uint32_t most = 0;
+        const uint64_t ts0 = i0 + b0;
+        for (uint32_t b = 0; b < kMaxBatch; ++b) {
+            const bool live = b < d.n_updates;
+            d.pair_begin[b] = live ? h_pair_begin[b0 + b] : 0;
+            d.n_pairs[b] = live ? h_pair_count[b0 + b] : 0;
+            d.pos_start[b] = live ? static_cast<uint32_t>(start_abs[b0 + b] - s->pos_base) : 0;
+            d.win_start[b] = live ? static_cast<uint32_t>(win_abs[b0 + b] - s->pos_base) : 0;
+            d.win_bits[b] = 0;
+            if (!live) continue;
+            pairs += d.n_pairs[b];
+            most = d.n_pairs[b] > most ? d.n_pairs[b] : most;
+            const uint64_t j = h_pull_ts[b0 + b];           // which updates of this launch lie in the window [j, i - 1]
+            const uint32_t first_in = j > ts0 ? static_cast<uint32_t>(j - ts0) : 0u;     // <= b
+            d.win_bits[b] = ((1u << b) - 1u) & ~((1u << first_in) - 1u);
+            if (j < ts0) d.pre_mask |= 1u << b;
         }
-    } else {
-        for (uint32_t b = 0; b < n_updates; ++b) {
-            UpdateDesc u;
-            u.pair_begin = h_pair_begin[b];
-            u.n_pairs = h_pair_count[b];
-            u.pos_start = static_cast<uint32_t>(start_abs[b] - s->pos_base);
-            u.win_start = static_cast<uint32_t>(win_abs[b] - s->pos_base);
-            u.pad = 0;
-            if (u.n_pairs) {
-                const unsigned grid = (u.n_pairs + kApplyThreads - 1) / kApplyThreads;
-                k_apply_update<<<grid, kApplyThreads, 0, st>>>(sp, u, d_idx, d_val, lr, d_sigma_out);
-                ADACOMP_LAUNCH_CHECK();
-            }
+        if (!pairs) continue;
+        const double dens = static_cast<double>(most) / static_cast<double>(s->n_params);   // of the densest update
+        const bool sweep = theta_aligned &&
+                           (s->mode == 3 || (s->mode == 0 && static_cast<double>(pairs) >= 0.2 * static_cast<double>(s->n_params)));
+        if (sweep) {
+            SweepDesc sd;
+            sd.o = d;
+            // stage what a uniformly spread update brings per range, plus three standard deviations
+            const double mean = dens * kSwRange;
+            const uint32_t chunks = static_cast<uint32_t>((mean + 3.0 * std::sqrt(mean) + 2.0) / 32.0) + 1;
+            sd.chunks = chunks > kRgChunks ? kRgChunks : chunks;
+            const size_t smem = sw_smem_bytes(d.n_updates);
+            const uint32_t n_ranges = static_cast<uint32_t>((s->n_params + kSwRange - 1) / kSwRange);
+            int per_sm = 1;
+            ADACOMP_CUDA(cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, k_apply_sweep, kSwThreads, smem));
+            unsigned grid = static_cast<unsigned>(s->n_sms) * static_cast<unsigned>(per_sm > 0 ? per_sm : 1);
+            if (grid > n_ranges) grid = n_ranges;
+            k_apply_sweep<<<grid, kSwThreads, smem, st>>>(sp, sd, d_idx, d_val, lr, d_sigma_out, n_ranges);
+        } else {
+            RangeDesc rd;
+            rd.o = d;
+            // range size: the densest update should bring about 96 pairs per range, so that mean + 3 standard
+            // deviations of a uniformly spread update still fit the stage of 128
+            const double want = 96.0 / dens;
+            uint32_t range = want >= kRgMaxRange ? kRgMaxRange : static_cast<uint32_t>(want) & ~31u;
+            if (range < kRgMinRange) range = kRgMinRange;
+            const double mean = dens * range;
+            const uint32_t chunks = static_cast<uint32_t>((mean + 3.0 * std::sqrt(mean) + 2.0) / 32.0) + 1;
+            rd.range = range;
+            rd.chunks = chunks > kRgChunks ? kRgChunks : chunks;
+            rd.use_table = static_cast<uint64_t>(d.n_updates) * range <= 32768 ? 1u : 0u;
+            const size_t smem = rg_smem_bytes(range, d.n_updates, rd.use_table != 0);
+            const uint32_t n_ranges = static_cast<uint32_t>((s->n_params + range - 1) / range);
+            int per_sm = 1;
+            ADACOMP_CUDA(cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, k_apply_ranges, kRgThreads, smem));
+            unsigned grid = static_cast<unsigned>(s->n_sms) * static_cast<unsigned>(per_sm > 0 ? per_sm : 1);
+            if (grid > n_ranges) grid = n_ranges;
+            k_apply_ranges<<<grid, kRgThreads, smem, st>>>(sp, rd, d_idx, d_val, lr, d_sigma_out, n_ranges);
+        }
+        ADACOMP_LAUNCH_CHECK();
+    }
+    for (uint32_t b = 0; b < n_updates && one_by_one; ++b) {
+        UpdateDesc u;
+        u.pair_begin = h_pair_begin[b];
+        u.n_pairs = h_pair_count[b];
+        u.pos_start = static_cast<uint32_t>(start_abs[b] - s->pos_base);
+        u.win_start = static_cast<uint32_t>(win_abs[b] - s->pos_base);
+        u.pad = 0;
+        if (u.n_pairs) {
+            const unsigned grid = (u.n_pairs + kApplyThreads - 1) / kApplyThreads;
+            k_apply_update<<<grid, kApplyThreads, 0, st>>>(sp, u, d_idx, d_val, lr, d_sigma_out);
+            ADACOMP_LAUNCH_CHECK();
         }
     }
     for (uint32_t b = 0; b < n_updates; ++b) s->start_of[(i0 + b) % cap] = start_abs[b];

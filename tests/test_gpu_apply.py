@@ -164,6 +164,43 @@ def test_zero_values_empty_updates_and_scattered_slices(binding, mode):
     assert torch.signbit(theta[0]) and torch.signbit(theta[3])
 
 
+@pytest.mark.parametrize("mode", MODES)
+def test_clustered_and_uneven_updates(binding, mode):
+    """Updates whose indices crowd into a few stretches of the parameter vector (far more pairs per
+    stretch than any kernel stages at once), next to thin and empty ones, over three calls."""
+    P = 300_000
+    rng = np.random.default_rng(11)
+    theta = torch.from_numpy(rng.standard_normal(P).astype(np.float32)).to(DEV)
+    ref = oracle.Server(theta.cpu().numpy())
+    srv = binding.Server(theta, history_pairs=1 << 20, max_window_updates=32)
+    srv.set_mode(mode)
+    def updates():
+        out = [np.arange(50_000, 60_000), np.arange(0, P, 7), np.sort(rng.choice(P, 3000, replace=False)),
+               np.arange(55_000, 75_000), np.array([], dtype=np.int64), np.arange(P - 700, P),
+               np.sort(rng.choice(np.arange(100_000, 101_000), 900, replace=False)), np.arange(58_000, 58_100)]
+        return [a.astype(np.uint32) for a in out]
+    ts = 0
+    for call in range(3):
+        ups = updates()
+        vals = [rng.standard_normal(a.size).astype(np.float32) for a in ups]
+        vals[3][::5] = 0.0                                   # present, but not a change
+        begin = np.concatenate([[0], np.cumsum([a.size for a in ups])[:-1]]).astype(np.uint64)
+        count = np.array([a.size for a in ups], np.uint32)
+        pull = np.array([max(0, ts + b - int(rng.integers(0, 6))) for b in range(len(ups))], np.uint64)
+        idx, val = i32(np.concatenate(ups)), torch.from_numpy(np.concatenate(vals)).to(DEV)
+        sigma = torch.full_like(idx, -1)
+        order = rng.permutation(len(ups))                    # arrival order differs from memory order
+        srv.apply(idx, val, begin[order], count[order], pull, 0.05, sigma_out=sigma)
+        s = u32(sigma)
+        for b, w in enumerate(order.tolist()):
+            want = ref.apply(ups[w], vals[w], int(pull[b]), 0.05)
+            lo = int(begin[w])
+            assert np.array_equal(s[lo:lo + ups[w].size], want), f"call {call} update {b}"
+        ts += len(ups)
+    assert srv.last_error() == 0 and srv.timestamp == ts == ref.timestamp
+    assert np.array_equal(bits(theta), bits(ref.theta()))
+
+
 def test_window_and_capacity_errors_leave_the_server_unchanged(binding):
     theta = torch.zeros(100, device=DEV)
     srv = binding.Server(theta, history_pairs=40, max_window_updates=8)     # ring of 64 pairs
