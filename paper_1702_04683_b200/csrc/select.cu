@@ -89,7 +89,7 @@ void plan_bracket(Layer& L, Layout* out) {
     if (cand > n) cand = n;
     if (win > n) win = n;
     // tensors whose candidates will be about a tenth of the entries or more take the dense scan kernel
-    L.bracket = lo_frac >= 0.08 ? 2 : 1;
+    L.bracket = lo_frac >= 0.03 ? 2 : 1;
     L.sample = m;
     L.n_spans = n_spans;
     L.span_base = static_cast<uint32_t>(out->span_stride);

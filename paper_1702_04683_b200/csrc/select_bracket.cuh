@@ -390,20 +390,48 @@ __global__ void __launch_bounds__(kThreads, 4) k_bracket_scan(SelectParams p, ui
 }
 
 // ---------------------------------------------------------------------------------------------
-// The same pass for tensors whose candidates are dense (a few percent of the entries or more),
-// where nearly every load holds a candidate and queueing loads would only add work.  Same
-// decomposition (8 warps x 8 pieces of 1024 entries per block, warps on their own), but a piece
-// is classified entirely in registers: two bit masks per lane (candidate, window), one 64-bit
-// atomic per piece to reserve room, and while it is in flight the warp ranks its candidates in
-// index order (two byte-packed warp scans: candidates per load and lane) and stages index and
-// value of each in shared memory straight from the registers, so nothing is read twice.  The
-// next piece's loads are issued as soon as the registers are free, before the reservation is
-// consumed; the staged lists then leave with coalesced stores.
-constexpr uint32_t kDenseStage = 640;                          // candidates staged per piece (of 1024 entries)
-constexpr uint32_t kDenseWinStage = 384;                       // window entries staged per piece
-constexpr size_t kDenseSmemPerWarp = (kDenseStage + kDenseWinStage) * 8;
+// The same pass for tensors whose candidates are dense (a percent of the entries or more), where
+// nearly every load holds a candidate and queueing loads would only add work.  Same
+// decomposition (8 warps x 8 pieces of 1024 entries per block, warps on their own), per piece:
+//   count    the four components of each of the lane's 8 loads are tested and counted (one byte
+//            per load; population counts and ballots are slow instructions, sums of predicates
+//            are not) and two byte-packed warp scans turn the counts into every candidate's place
+//            in index order (load, lane, component).  The piece's total is known now: one atomic
+//            reserves its room in the candidate list and stays in flight during what follows;
+//   place    a second sweep over the registers stores every candidate's position and value at
+//            its place on a shared-memory stage, with predicated stores (no branch per entry);
+//            the next piece's loads follow at once;
+//   window   with every lane busy: one lane per staged candidate tests it against t_hi (and for
+//            NaN) and stages window entries, ranked by ballot; a second atomic reserves their
+//            room, and they are copied out one piece later, when that atomic has long returned;
+//   copy     the staged candidates leave with coalesced stores.
+constexpr uint32_t kDenseStage = 512;                          // candidates staged per piece (of 1024 entries)
+constexpr uint32_t kDenseWinStage = 256;                       // window entries staged per piece
+constexpr size_t kDenseSmemPerWarp = kDenseStage * 6 + kDenseWinStage * 8;
 
-__global__ void __launch_bounds__(kThreads, 3) k_bracket_scan_dense(SelectParams p, uint32_t item_base) {
+// if (|x| >= t or unordered) { pos[r] = place; val[r] = x; ++r; } with predicated instructions;
+// pos_base and val_base are the shared-memory addresses of the two stage arrays
+__device__ __forceinline__ void dense_place(float x, float t, uint32_t& r, uint32_t pos_base, uint32_t val_base,
+                                            uint32_t place) {
+    asm volatile(
+        "{\n\t"
+        ".reg .pred p;\n\t"
+        ".reg .f32 a;\n\t"
+        ".reg .u32 ap, av;\n\t"
+        "abs.f32 a, %1;\n\t"
+        "setp.geu.f32 p, a, %2;\n\t"
+        "mad.lo.u32 ap, %0, 2, %3;\n\t"
+        "mad.lo.u32 av, %0, 4, %4;\n\t"
+        "@p st.shared.u16 [ap], %5;\n\t"
+        "@p st.shared.f32 [av], %1;\n\t"
+        "@p add.u32 %0, %0, 1;\n\t"
+        "}"
+        : "+r"(r)
+        : "f"(x), "f"(t), "r"(pos_base), "r"(val_base), "h"(static_cast<unsigned short>(place))
+        : "memory");
+}
+
+__global__ void __launch_bounds__(kThreads, 4) k_bracket_scan_dense(SelectParams p, uint32_t item_base) {
     extern __shared__ __align__(16) unsigned char s_scan[];
     const uint2 item = p.items[item_base + blockIdx.x];
     const uint32_t l = item.x, w = blockIdx.y;
@@ -417,6 +445,7 @@ __global__ void __launch_bounds__(kThreads, 3) k_bracket_scan_dense(SelectParams
     const uint32_t n_shift = L.n + mis;                        // n <= 33.5 M on this route
     const uint32_t nvec = (n_shift + 3) >> 2;
     const uint32_t lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const uint32_t lt = (1u << lane) - 1u;
     constexpr uint32_t kStep = kThreads / 32;
     constexpr uint32_t kBatch = kSpansPerBlock * kSubsPerSpan / kStep;
     const uint32_t ss_end = min(item.y + kSpansPerBlock, L.n_spans) * kSubsPerSpan;
@@ -424,10 +453,12 @@ __global__ void __launch_bounds__(kThreads, 3) k_bracket_scan_dense(SelectParams
     if (ss0 >= ss_end) return;
     const uint32_t in_lo = mis ? 1u : 0u, in_hi = n_shift / kSubElems;
     unsigned char* mine = s_scan + warp * kDenseSmemPerWarp;
-    uint32_t* stage_idx = reinterpret_cast<uint32_t*>(mine);
-    float* stage_val = reinterpret_cast<float*>(mine + kDenseStage * 4);
-    uint32_t* stage_widx = reinterpret_cast<uint32_t*>(mine + kDenseStage * 8);
-    uint32_t* stage_wkey = reinterpret_cast<uint32_t*>(mine + kDenseStage * 8 + kDenseWinStage * 4);
+    float* stage_val = reinterpret_cast<float*>(mine);                                        // [kDenseStage]
+    uint32_t* stage_widx = reinterpret_cast<uint32_t*>(mine + kDenseStage * 4);                // [kDenseWinStage]
+    uint32_t* stage_wkey = stage_widx + kDenseWinStage;
+    uint16_t* stage_pos = reinterpret_cast<uint16_t*>(mine + kDenseStage * 4 + kDenseWinStage * 8);   // [kDenseStage] place inside the piece
+    const uint32_t val_base = static_cast<uint32_t>(__cvta_generic_to_shared(stage_val));
+    const uint32_t pos_base = static_cast<uint32_t>(__cvta_generic_to_shared(stage_pos));
     uint32_t* cand_idx = p.cand_idx + static_cast<uint64_t>(w) * p.cand_stride + L.cand_base;
     float* cand_val = p.cand_val + static_cast<uint64_t>(w) * p.cand_stride + L.cand_base;
     uint32_t* win_key = p.win_key + static_cast<uint64_t>(w) * p.win_stride + L.win_base;
@@ -435,8 +466,25 @@ __global__ void __launch_bounds__(kThreads, 3) k_bracket_scan_dense(SelectParams
     uint2* sub_tab = p.sub_tab + (static_cast<uint64_t>(w) * p.span_stride + L.span_base) * kSubsPerSpan;
 
     float4 x[8];
-    bool have_x = false;                                       // x already holds the piece about to be classified
-    bool saw_nan = false;
+    bool have_x = false;                                       // x already holds the piece about to be compacted
+    bool saw_nan = false, lost = false;                        // lost: something did not fit
+    uint32_t tw_prev = 0, old_w = 0;                           // the window entries still on the stage, and their reservation
+    // the previous piece's window entries leave the stage (its reservation has had a whole piece's time to return)
+    auto copy_window = [&]() {
+        if (tw_prev) {
+            const uint32_t wb = __shfl_sync(0xFFFFFFFFu, old_w, 0);
+            if (static_cast<uint64_t>(wb) + tw_prev > L.win_cap) {
+                lost = true;
+            } else {
+                for (uint32_t r = lane; r < tw_prev; r += 32) {
+                    win_idx[wb + r] = stage_widx[r];
+                    win_key[wb + r] = stage_wkey[r];
+                }
+            }
+            __syncwarp();
+            tw_prev = 0;
+        }
+    };
 #pragma unroll 1
     for (uint32_t j = 0; j < kBatch; ++j) {
         const uint32_t ss = ss0 + kStep * j, next = ss + kStep;
@@ -450,109 +498,98 @@ __global__ void __launch_bounds__(kThreads, 3) k_bracket_scan_dense(SelectParams
                 x[i] = (inside || v < nvec) ? __ldg(&vec[v]) : make_float4(0.f, 0.f, 0.f, 0.f);
             }
         }
-        // classify every entry: bit 4 i + q = component q of this lane's load i
-        uint32_t mask_c = 0, mask_w = 0;
+        // ---- count
+        uint32_t cnt_a = 0, cnt_b = 0;                         // loads 0-3, loads 4-7
 #pragma unroll
         for (int i = 0; i < 8; ++i) {
-            float xs[4] = {x[i].x, x[i].y, x[i].z, x[i].w};
             if (!inside) {                                     // first / last piece: blank what lies outside (t_lo > 0)
+                float xs[4] = {x[i].x, x[i].y, x[i].z, x[i].w};
                 const uint32_t e0 = (vec0 + i * 32 + lane) * 4;
 #pragma unroll
                 for (int q = 0; q < 4; ++q)
                     if (e0 + q < mis || e0 + q >= n_shift) xs[q] = 0.f;
                 x[i] = make_float4(xs[0], xs[1], xs[2], xs[3]);
             }
-            const float m4 = max_nan(max_nan(fabsf(xs[0]), fabsf(xs[1])), max_nan(fabsf(xs[2]), fabsf(xs[3])));
-            saw_nan |= m4 != m4;
-#pragma unroll
-            for (int q = 0; q < 4; ++q) {
-                const float a = fabsf(xs[q]);
-                const bool cand = !(a < tlo_f);
-                if (cand) mask_c |= 1u << (i * 4 + q);
-                if (cand && !(a > thi_f)) mask_w |= 1u << (i * 4 + q);
-            }
+            const uint32_t n = (!(fabsf(x[i].x) < tlo_f) ? 1u : 0u) + (!(fabsf(x[i].y) < tlo_f) ? 1u : 0u) +
+                               (!(fabsf(x[i].z) < tlo_f) ? 1u : 0u) + (!(fabsf(x[i].w) < tlo_f) ? 1u : 0u);
+            if (i < 4) cnt_a += n << (8 * i); else cnt_b += n << (8 * (i - 4));
         }
-        const uint32_t cw = __popc(mask_w);
-        const uint32_t tc = __reduce_add_sync(0xFFFFFFFFu, __popc(mask_c));
-        const uint32_t tw = __reduce_add_sync(0xFFFFFFFFu, cw);
-        unsigned long long old = 0;
-        if (tc && lane == 0)                                  // reserve room: one atomic per piece
-            old = atomicAdd(reinterpret_cast<unsigned long long*>(&st->cand_count),
-                            static_cast<unsigned long long>(tc) | (static_cast<unsigned long long>(tw) << 32));
-        const bool fits = tc <= kDenseStage && tw <= kDenseWinStage;
-        if (tc && fits) {
-            // rank in index order = (load, lane, component): per-load counts of this lane, one byte
-            // each (a load holds at most 128 candidates across the warp), scanned over the lanes
-            const uint32_t cnt_a = __popc(mask_c & 0xFu) | (__popc(mask_c & 0xF0u) << 8) |
-                                   (__popc(mask_c & 0xF00u) << 16) | (__popc(mask_c & 0xF000u) << 24);
-            const uint32_t cnt_b = __popc(mask_c & 0xF0000u) | (__popc(mask_c & 0xF00000u) << 8) |
-                                   (__popc(mask_c & 0xF000000u) << 16) | (__popc(mask_c & 0xF0000000u) << 24);
-            uint32_t inc_a = cnt_a, inc_b = cnt_b, inc_w = cw;
+        uint32_t inc_a = cnt_a, inc_b = cnt_b;                 // a load holds at most 128 candidates: no byte overflows
 #pragma unroll
-            for (int d = 1; d < 32; d <<= 1) {
-                const uint32_t ya = __shfl_up_sync(0xFFFFFFFFu, inc_a, d);
-                const uint32_t yb = __shfl_up_sync(0xFFFFFFFFu, inc_b, d);
-                const uint32_t yw = __shfl_up_sync(0xFFFFFFFFu, inc_w, d);
-                if (lane >= static_cast<uint32_t>(d)) { inc_a += ya; inc_b += yb; inc_w += yw; }
-            }
-            const uint32_t tot_a = __shfl_sync(0xFFFFFFFFu, inc_a, 31), tot_b = __shfl_sync(0xFFFFFFFFu, inc_b, 31);
-            const uint32_t pre_a = inc_a - cnt_a, pre_b = inc_b - cnt_b;
-            uint32_t wr = inc_w - cw;                             // window entries: any order (lane-major)
+        for (int d = 1; d < 32; d <<= 1) {
+            const uint32_t ya = __shfl_up_sync(0xFFFFFFFFu, inc_a, d);
+            const uint32_t yb = __shfl_up_sync(0xFFFFFFFFu, inc_b, d);
+            if (lane >= static_cast<uint32_t>(d)) { inc_a += ya; inc_b += yb; }
+        }
+        const uint32_t tot_a = __shfl_sync(0xFFFFFFFFu, inc_a, 31), tot_b = __shfl_sync(0xFFFFFFFFu, inc_b, 31);
+        const uint32_t pre_a = inc_a - cnt_a, pre_b = inc_b - cnt_b;
+        const uint32_t sum_a = (tot_a & 0x00FF00FFu) + ((tot_a >> 8) & 0x00FF00FFu);
+        const uint32_t sum_b = (tot_b & 0x00FF00FFu) + ((tot_b >> 8) & 0x00FF00FFu);
+        const uint32_t tc = (sum_a & 0xFFFFu) + (sum_a >> 16) + (sum_b & 0xFFFFu) + (sum_b >> 16);
+        uint32_t old_c = 0;
+        if (tc && lane == 0) old_c = atomicAdd(&st->cand_count, tc);     // room in the candidate list
+        const bool crowded = tc > kDenseStage;                 // more candidates than the stage holds
+        // ---- place
+        if (tc && !crowded) {
             uint32_t load_off = 0;
 #pragma unroll
             for (int i = 0; i < 8; ++i) {
                 const uint32_t pre_i = ((i < 4 ? pre_a : pre_b) >> ((i & 3) * 8)) & 255u;
                 const uint32_t tot_i = ((i < 4 ? tot_a : tot_b) >> ((i & 3) * 8)) & 255u;
-                const float xs[4] = {x[i].x, x[i].y, x[i].z, x[i].w};
-                const uint32_t e0 = (vec0 + i * 32 + lane) * 4;
                 uint32_t r = load_off + pre_i;
-#pragma unroll
-                for (int q = 0; q < 4; ++q) {
-                    if ((mask_c >> (i * 4 + q)) & 1u) {
-                        stage_idx[r] = e0 + q;                    // shifted coordinate inside the tensor
-                        stage_val[r] = xs[q];
-                        ++r;
-                        if ((mask_w >> (i * 4 + q)) & 1u) {
-                            stage_widx[wr] = e0 + q;
-                            stage_wkey[wr] = magnitude_key(xs[q]);
-                            ++wr;
-                        }
-                    }
-                }
+                const uint32_t place = i * 128 + lane * 4;
+                dense_place(x[i].x, tlo_f, r, pos_base, val_base, place);
+                dense_place(x[i].y, tlo_f, r, pos_base, val_base, place + 1);
+                dense_place(x[i].z, tlo_f, r, pos_base, val_base, place + 2);
+                dense_place(x[i].w, tlo_f, r, pos_base, val_base, place + 3);
                 load_off += tot_i;
             }
         }
         __syncwarp();
-        // the registers are free: start the next piece's loads before consuming the reservation
+        // the registers are free: start the next piece's loads
         have_x = (j + 1 < kBatch) && next < ss_end && next >= in_lo && next < in_hi;
         if (have_x) {
             const float4* nptr = vec + next * (kSubElems / 4) + lane;
 #pragma unroll
             for (int i = 0; i < 8; ++i) x[i] = __ldg(nptr + i * 32);
         }
-        if (tc) {
-            old = __shfl_sync(0xFFFFFFFFu, old, 0);
-            const uint32_t cb = static_cast<uint32_t>(old), wb = static_cast<uint32_t>(old >> 32);
-            const bool over = !fits || (static_cast<uint64_t>(cb) + tc > L.cand_cap) ||
-                              (static_cast<uint64_t>(wb) + tw > L.win_cap);
-            if (lane == 0) {
-                sub_tab[ss] = make_uint2(cb, tc | ((tc - tw) << 16));
-                if (over) atomicOr(&st->flags, kInstOverflow);
+        if (!tc) continue;
+        copy_window();                                         // the window stage is about to be reused
+        // ---- window: one lane per staged candidate
+        uint32_t tw = 0;
+        if (!crowded) {
+            for (uint32_t r0 = 0; r0 < tc; r0 += 32) {
+                const uint32_t r = r0 + lane;
+                const float a = r < tc ? fabsf(stage_val[r]) : 0.f;
+                const bool isw = r < tc && !(a > thi_f);
+                saw_nan |= a != a;
+                const uint32_t bw = __ballot_sync(0xFFFFFFFFu, isw);
+                if (bw) {
+                    const uint32_t wr = tw + __popc(bw & lt);
+                    if (isw && wr < kDenseWinStage) {
+                        stage_widx[wr] = vec0 * 4 + stage_pos[r];        // shifted coordinate inside the tensor
+                        stage_wkey[wr] = __float_as_uint(a);             // the magnitude key
+                    }
+                    tw += __popc(bw);
+                }
             }
-            if (!over) {
-                for (uint32_t r = lane; r < tc; r += 32) {
-                    cand_idx[cb + r] = stage_idx[r];
-                    cand_val[cb + r] = stage_val[r];
-                }
-                for (uint32_t r = lane; r < tw; r += 32) {
-                    win_idx[wb + r] = stage_widx[r];
-                    win_key[wb + r] = stage_wkey[r];
-                }
+        }
+        if (tw && lane == 0) old_w = atomicAdd(&st->win_count, tw);       // room in the window list
+        const uint32_t cb = __shfl_sync(0xFFFFFFFFu, old_c, 0);
+        if (lane == 0) sub_tab[ss] = make_uint2(cb, tc | ((tc - tw) << 16));
+        if (crowded || tw > kDenseWinStage || static_cast<uint64_t>(cb) + tc > L.cand_cap) {
+            lost = true;
+        } else {
+            tw_prev = tw;
+            for (uint32_t r = lane; r < tc; r += 32) {         // ---- copy
+                cand_idx[cb + r] = vec0 * 4 + stage_pos[r];
+                cand_val[cb + r] = stage_val[r];
             }
         }
         __syncwarp();                                         // the stage is reused by the next piece
     }
-    if (saw_nan) atomicOr(&st->flags, kInstOverflow);
+    copy_window();
+    if (saw_nan || lost) atomicOr(&st->flags, kInstOverflow);
 }
 
 // ---------------------------------------------------------------------------------------------
