@@ -392,22 +392,25 @@ __global__ void __launch_bounds__(kThreads, 4) k_bracket_scan(SelectParams p, ui
 // ---------------------------------------------------------------------------------------------
 // The same pass for tensors whose candidates are dense (a percent of the entries or more), where
 // nearly every load holds a candidate and queueing loads would only add work.  Same
-// decomposition (8 warps x 8 pieces of 1024 entries per block, warps on their own), per piece:
-//   count    the four components of each of the lane's 8 loads are tested and counted (one byte
+// decomposition (8 warps x 8 pieces of 1024 entries per block, warps on their own).  Per piece:
+//   count    the four components of each of the lane's loads are tested and counted (one byte
 //            per load; population counts and ballots are slow instructions, sums of predicates
-//            are not) and two byte-packed warp scans turn the counts into every candidate's place
-//            in index order (load, lane, component).  The piece's total is known now: one atomic
-//            reserves its room in the candidate list and stays in flight during what follows;
+//            are not) and a byte-packed warp scan turns the counts into every candidate's place
+//            in index order (load, lane, component);
 //   place    a second sweep over the registers stores every candidate's position and value at
-//            its place on a shared-memory stage, with predicated stores (no branch per entry);
-//            the next piece's loads follow at once;
-//   window   with every lane busy: one lane per staged candidate tests it against t_hi (and for
-//            NaN) and stages window entries, ranked by ballot; a second atomic reserves their
-//            room, and they are copied out one piece later, when that atomic has long returned;
-//   copy     the staged candidates leave with coalesced stores.
-constexpr uint32_t kDenseStage = 512;                          // candidates staged per piece (of 1024 entries)
-constexpr uint32_t kDenseWinStage = 256;                       // window entries staged per piece
-constexpr size_t kDenseSmemPerWarp = kDenseStage * 6 + kDenseWinStage * 8;
+//            its place on a shared-memory stage, behind the candidates of the pieces staged
+//            before, with predicated stores (no branch per entry).
+//   Both run for the lane's loads 0-3, whose registers are then refilled with the next piece,
+//   and again for loads 4-7.
+// Flush, once the stage could not take another piece and after the last one, while the next
+// piece's loads are in flight: an atomic reserves room in the candidate list for all staged
+// pieces; with every lane busy, one lane per staged candidate tests it against t_hi (and for
+// NaN) and stages window entries, ranked by ballot; a second atomic reserves their room; the
+// table entries of the pieces are written and the lists leave with coalesced stores.
+constexpr uint32_t kDenseStage = 768;                          // candidates the stage holds
+constexpr uint32_t kDensePiece = 512;                          // most candidates one piece (of 1024 entries) may bring
+constexpr uint32_t kDenseWinStage = 256;                       // window entries staged per flush
+constexpr size_t kDenseSmemPerWarp = kDenseStage * 6 + kDenseWinStage * 8 + 64;
 
 // if (|x| >= t or unordered) { pos[r] = place; val[r] = x; ++r; } with predicated instructions;
 // pos_base and val_base are the shared-memory addresses of the two stage arrays
@@ -456,7 +459,9 @@ __global__ void __launch_bounds__(kThreads, 4) k_bracket_scan_dense(SelectParams
     float* stage_val = reinterpret_cast<float*>(mine);                                        // [kDenseStage]
     uint32_t* stage_widx = reinterpret_cast<uint32_t*>(mine + kDenseStage * 4);                // [kDenseWinStage]
     uint32_t* stage_wkey = stage_widx + kDenseWinStage;
-    uint16_t* stage_pos = reinterpret_cast<uint16_t*>(mine + kDenseStage * 4 + kDenseWinStage * 8);   // [kDenseStage] place inside the piece
+    uint32_t* s_tc = stage_wkey + kDenseWinStage;                                             // [8] candidates per piece
+    uint32_t* s_tw = s_tc + kBatch;                                                           // [8] window entries per piece
+    uint16_t* stage_pos = reinterpret_cast<uint16_t*>(s_tw + kBatch);                         // [kDenseStage] piece * 1024 + place
     const uint32_t val_base = static_cast<uint32_t>(__cvta_generic_to_shared(stage_val));
     const uint32_t pos_base = static_cast<uint32_t>(__cvta_generic_to_shared(stage_pos));
     uint32_t* cand_idx = p.cand_idx + static_cast<uint64_t>(w) * p.cand_stride + L.cand_base;
@@ -465,26 +470,77 @@ __global__ void __launch_bounds__(kThreads, 4) k_bracket_scan_dense(SelectParams
     uint32_t* win_idx = p.win_idx + static_cast<uint64_t>(w) * p.win_stride + L.win_base;
     uint2* sub_tab = p.sub_tab + (static_cast<uint64_t>(w) * p.span_stride + L.span_base) * kSubsPerSpan;
 
-    float4 x[8];
-    bool have_x = false;                                       // x already holds the piece about to be compacted
     bool saw_nan = false, lost = false;                        // lost: something did not fit
-    uint32_t tw_prev = 0, old_w = 0;                           // the window entries still on the stage, and their reservation
-    // the previous piece's window entries leave the stage (its reservation has had a whole piece's time to return)
-    auto copy_window = [&]() {
-        if (tw_prev) {
-            const uint32_t wb = __shfl_sync(0xFFFFFFFFu, old_w, 0);
-            if (static_cast<uint64_t>(wb) + tw_prev > L.win_cap) {
-                lost = true;
-            } else {
-                for (uint32_t r = lane; r < tw_prev; r += 32) {
-                    win_idx[wb + r] = stage_widx[r];
-                    win_key[wb + r] = stage_wkey[r];
+    uint32_t staged = 0, j_first = 0;                          // candidates on the stage; first piece they belong to
+    // shifted coordinate inside the tensor of a staged position
+    auto entry_of = [&](uint32_t pos) -> uint32_t { return (ss0 + kStep * (pos >> 10)) * kSubElems + (pos & 1023u); };
+    // everything staged since the last flush (pieces j_first .. j_end - 1) goes to the lists
+    auto flush = [&](uint32_t j_end) {
+        if (staged) {
+            uint32_t old_c = 0, old_w = 0;
+            if (lane == 0) old_c = atomicAdd(&st->cand_count, staged);   // room in the candidate list
+            if (lane < kBatch) s_tw[lane] = 0;
+            __syncwarp();
+            uint32_t tw = 0;
+#pragma unroll 1
+            for (uint32_t r0 = 0; r0 < staged; r0 += 32) {         // window: one lane per staged candidate
+                const uint32_t r = r0 + lane;
+                const float a = r < staged ? fabsf(stage_val[r]) : 0.f;
+                const bool isw = r < staged && !(a > thi_f);
+                saw_nan |= a != a;
+                const uint32_t bw = __ballot_sync(0xFFFFFFFFu, isw);
+                if (bw) {
+                    if (isw) {
+                        const uint32_t wr = tw + __popc(bw & lt), pos = stage_pos[r];
+                        if (wr < kDenseWinStage) {
+                            stage_widx[wr] = entry_of(pos);
+                            stage_wkey[wr] = __float_as_uint(a);     // the magnitude key
+                        }
+                        atomicAdd(&s_tw[pos >> 10], 1u);
+                    }
+                    tw += __popc(bw);
                 }
             }
+            if (tw && lane == 0) old_w = atomicAdd(&st->win_count, tw);   // room in the window list
             __syncwarp();
-            tw_prev = 0;
+            // where each piece's candidates begin
+            const bool mine_in = lane >= j_first && lane < j_end;
+            const uint32_t tcj = mine_in ? s_tc[lane] : 0u, twj = mine_in ? s_tw[lane] : 0u;
+            uint32_t inc = tcj;
+#pragma unroll
+            for (int d = 1; d < static_cast<int>(kBatch); d <<= 1) {
+                const uint32_t y = __shfl_up_sync(0xFFFFFFFFu, inc, d);
+                if (lane >= static_cast<uint32_t>(d)) inc += y;
+            }
+            const uint32_t cb = __shfl_sync(0xFFFFFFFFu, old_c, 0);
+            if (tcj) sub_tab[ss0 + kStep * lane] = make_uint2(cb + inc - tcj, tcj | ((tcj - twj) << 16));
+            if (tw > kDenseWinStage || static_cast<uint64_t>(cb) + staged > L.cand_cap) {
+                lost = true;
+            } else {
+#pragma unroll 1
+                for (uint32_t r = lane; r < staged; r += 32) {
+                    cand_idx[cb + r] = entry_of(stage_pos[r]);
+                    cand_val[cb + r] = stage_val[r];
+                }
+                const uint32_t wb = __shfl_sync(0xFFFFFFFFu, old_w, 0);
+                if (static_cast<uint64_t>(wb) + tw > L.win_cap) {
+                    lost = true;
+                } else {
+#pragma unroll 1
+                    for (uint32_t r = lane; r < tw; r += 32) {
+                        win_idx[wb + r] = stage_widx[r];
+                        win_key[wb + r] = stage_wkey[r];
+                    }
+                }
+            }
+            __syncwarp();                                     // the stage is reused
         }
+        staged = 0;
+        j_first = j_end;
     };
+
+    float4 x[8];
+    bool have_x = false;                                       // x already holds the piece about to be compacted
 #pragma unroll 1
     for (uint32_t j = 0; j < kBatch; ++j) {
         const uint32_t ss = ss0 + kStep * j, next = ss + kStep;
@@ -498,97 +554,64 @@ __global__ void __launch_bounds__(kThreads, 4) k_bracket_scan_dense(SelectParams
                 x[i] = (inside || v < nvec) ? __ldg(&vec[v]) : make_float4(0.f, 0.f, 0.f, 0.f);
             }
         }
-        // ---- count
-        uint32_t cnt_a = 0, cnt_b = 0;                         // loads 0-3, loads 4-7
+        // ---- count and place, the lane's loads 0-3 first, then 4-7: the first half of the registers
+        // is refilled with the next piece while the second half is still being worked on
+        const bool next_inside = (j + 1 < kBatch) && next < ss_end && next >= in_lo && next < in_hi;
+        const float4* nptr = vec + (next_inside ? next : ss) * (kSubElems / 4) + lane;
+        uint32_t tc = 0;
+        bool crowded = false;                                  // more candidates than a piece may bring
 #pragma unroll
-        for (int i = 0; i < 8; ++i) {
-            if (!inside) {                                     // first / last piece: blank what lies outside (t_lo > 0)
-                float xs[4] = {x[i].x, x[i].y, x[i].z, x[i].w};
-                const uint32_t e0 = (vec0 + i * 32 + lane) * 4;
+        for (int h = 0; h < 2; ++h) {
+            uint32_t cnt = 0;                                  // candidates per load of this lane, one byte each
 #pragma unroll
-                for (int q = 0; q < 4; ++q)
-                    if (e0 + q < mis || e0 + q >= n_shift) xs[q] = 0.f;
-                x[i] = make_float4(xs[0], xs[1], xs[2], xs[3]);
+            for (int i = 4 * h; i < 4 * h + 4; ++i) {
+                if (!inside) {                                 // first / last piece: blank what lies outside (t_lo > 0)
+                    float xs[4] = {x[i].x, x[i].y, x[i].z, x[i].w};
+                    const uint32_t e0 = (vec0 + i * 32 + lane) * 4;
+#pragma unroll
+                    for (int q = 0; q < 4; ++q)
+                        if (e0 + q < mis || e0 + q >= n_shift) xs[q] = 0.f;
+                    x[i] = make_float4(xs[0], xs[1], xs[2], xs[3]);
+                }
+                const uint32_t n = (!(fabsf(x[i].x) < tlo_f) ? 1u : 0u) + (!(fabsf(x[i].y) < tlo_f) ? 1u : 0u) +
+                                   (!(fabsf(x[i].z) < tlo_f) ? 1u : 0u) + (!(fabsf(x[i].w) < tlo_f) ? 1u : 0u);
+                cnt += n << (8 * (i & 3));
             }
-            const uint32_t n = (!(fabsf(x[i].x) < tlo_f) ? 1u : 0u) + (!(fabsf(x[i].y) < tlo_f) ? 1u : 0u) +
-                               (!(fabsf(x[i].z) < tlo_f) ? 1u : 0u) + (!(fabsf(x[i].w) < tlo_f) ? 1u : 0u);
-            if (i < 4) cnt_a += n << (8 * i); else cnt_b += n << (8 * (i - 4));
-        }
-        uint32_t inc_a = cnt_a, inc_b = cnt_b;                 // a load holds at most 128 candidates: no byte overflows
+            uint32_t inc = cnt;                                // a load holds at most 128 candidates: no byte overflows
 #pragma unroll
-        for (int d = 1; d < 32; d <<= 1) {
-            const uint32_t ya = __shfl_up_sync(0xFFFFFFFFu, inc_a, d);
-            const uint32_t yb = __shfl_up_sync(0xFFFFFFFFu, inc_b, d);
-            if (lane >= static_cast<uint32_t>(d)) { inc_a += ya; inc_b += yb; }
-        }
-        const uint32_t tot_a = __shfl_sync(0xFFFFFFFFu, inc_a, 31), tot_b = __shfl_sync(0xFFFFFFFFu, inc_b, 31);
-        const uint32_t pre_a = inc_a - cnt_a, pre_b = inc_b - cnt_b;
-        const uint32_t sum_a = (tot_a & 0x00FF00FFu) + ((tot_a >> 8) & 0x00FF00FFu);
-        const uint32_t sum_b = (tot_b & 0x00FF00FFu) + ((tot_b >> 8) & 0x00FF00FFu);
-        const uint32_t tc = (sum_a & 0xFFFFu) + (sum_a >> 16) + (sum_b & 0xFFFFu) + (sum_b >> 16);
-        uint32_t old_c = 0;
-        if (tc && lane == 0) old_c = atomicAdd(&st->cand_count, tc);     // room in the candidate list
-        const bool crowded = tc > kDenseStage;                 // more candidates than the stage holds
-        // ---- place
-        if (tc && !crowded) {
-            uint32_t load_off = 0;
-#pragma unroll
-            for (int i = 0; i < 8; ++i) {
-                const uint32_t pre_i = ((i < 4 ? pre_a : pre_b) >> ((i & 3) * 8)) & 255u;
-                const uint32_t tot_i = ((i < 4 ? tot_a : tot_b) >> ((i & 3) * 8)) & 255u;
-                uint32_t r = load_off + pre_i;
-                const uint32_t place = i * 128 + lane * 4;
-                dense_place(x[i].x, tlo_f, r, pos_base, val_base, place);
-                dense_place(x[i].y, tlo_f, r, pos_base, val_base, place + 1);
-                dense_place(x[i].z, tlo_f, r, pos_base, val_base, place + 2);
-                dense_place(x[i].w, tlo_f, r, pos_base, val_base, place + 3);
-                load_off += tot_i;
+            for (int d = 1; d < 32; d <<= 1) {
+                const uint32_t y = __shfl_up_sync(0xFFFFFFFFu, inc, d);
+                if (lane >= static_cast<uint32_t>(d)) inc += y;
             }
-        }
-        __syncwarp();
-        // the registers are free: start the next piece's loads
-        have_x = (j + 1 < kBatch) && next < ss_end && next >= in_lo && next < in_hi;
-        if (have_x) {
-            const float4* nptr = vec + next * (kSubElems / 4) + lane;
+            const uint32_t tot = __shfl_sync(0xFFFFFFFFu, inc, 31), pre = inc - cnt;
+            const uint32_t sum = (tot & 0x00FF00FFu) + ((tot >> 8) & 0x00FF00FFu);
+            uint32_t load_off = staged + tc;                   // behind what is staged, the first half's candidates first
+            tc += (sum & 0xFFFFu) + (sum >> 16);
+            crowded = tc > kDensePiece;                        // (a half brings at most 512: the first one always fits)
+            if (!crowded) {
 #pragma unroll
-            for (int i = 0; i < 8; ++i) x[i] = __ldg(nptr + i * 32);
-        }
-        if (!tc) continue;
-        copy_window();                                         // the window stage is about to be reused
-        // ---- window: one lane per staged candidate
-        uint32_t tw = 0;
-        if (!crowded) {
-            for (uint32_t r0 = 0; r0 < tc; r0 += 32) {
-                const uint32_t r = r0 + lane;
-                const float a = r < tc ? fabsf(stage_val[r]) : 0.f;
-                const bool isw = r < tc && !(a > thi_f);
-                saw_nan |= a != a;
-                const uint32_t bw = __ballot_sync(0xFFFFFFFFu, isw);
-                if (bw) {
-                    const uint32_t wr = tw + __popc(bw & lt);
-                    if (isw && wr < kDenseWinStage) {
-                        stage_widx[wr] = vec0 * 4 + stage_pos[r];        // shifted coordinate inside the tensor
-                        stage_wkey[wr] = __float_as_uint(a);             // the magnitude key
-                    }
-                    tw += __popc(bw);
+                for (int i = 4 * h; i < 4 * h + 4; ++i) {
+                    uint32_t r = load_off + ((pre >> ((i & 3) * 8)) & 255u);
+                    const uint32_t place = j * 1024 + i * 128 + lane * 4;
+                    dense_place(x[i].x, tlo_f, r, pos_base, val_base, place);
+                    dense_place(x[i].y, tlo_f, r, pos_base, val_base, place + 1);
+                    dense_place(x[i].z, tlo_f, r, pos_base, val_base, place + 2);
+                    dense_place(x[i].w, tlo_f, r, pos_base, val_base, place + 3);
+                    load_off += (tot >> ((i & 3) * 8)) & 255u;
                 }
             }
-        }
-        if (tw && lane == 0) old_w = atomicAdd(&st->win_count, tw);       // room in the window list
-        const uint32_t cb = __shfl_sync(0xFFFFFFFFu, old_c, 0);
-        if (lane == 0) sub_tab[ss] = make_uint2(cb, tc | ((tc - tw) << 16));
-        if (crowded || tw > kDenseWinStage || static_cast<uint64_t>(cb) + tc > L.cand_cap) {
-            lost = true;
-        } else {
-            tw_prev = tw;
-            for (uint32_t r = lane; r < tc; r += 32) {         // ---- copy
-                cand_idx[cb + r] = vec0 * 4 + stage_pos[r];
-                cand_val[cb + r] = stage_val[r];
+            if (next_inside) {                                 // these registers are free: the next piece's loads
+#pragma unroll
+                for (int i = 4 * h; i < 4 * h + 4; ++i) x[i] = __ldg(nptr + i * 32);
             }
         }
-        __syncwarp();                                         // the stage is reused by the next piece
+        have_x = next_inside;
+        if (crowded) { lost = true; tc = 0; }
+        if (lane == 0) s_tc[j] = tc;
+        staged += tc;
+        __syncwarp();
+        if (staged + kDensePiece > kDenseStage || j + 1 == kBatch || next >= ss_end) flush(j + 1);
     }
-    copy_window();
     if (saw_nan || lost) atomicOr(&st->flags, kInstOverflow);
 }
 
