@@ -202,6 +202,7 @@ k_apply_ranges(ServerParams sp, RangeDesc d, const uint32_t* __restrict__ idx, c
         for (uint32_t t = tid; t < R / 4; t += kRgThreads) reinterpret_cast<uint4*>(s_mask)[t] = make_uint4(0, 0, 0, 0);
         if (tid == 0) { s_m->n_listed = 0; s_m->any_zero = 0; }
         // ---- stage
+        #pragma unroll 1
         for (uint32_t b = warp; b < B; b += kRgThreads / 32) {
             const uint64_t begin = s_m->begin[b];
             const uint32_t n_b = s_m->n[b], cur = s_m->cur[b] + s_m->adv[b];     // past what the last round consumed
@@ -247,9 +248,11 @@ k_apply_ranges(ServerParams sp, RangeDesc d, const uint32_t* __restrict__ idx, c
         __syncthreads();
         const uint32_t limit = s_m->limit;
         // ---- scatter: bit b on every parameter update b changes below the limit
+        #pragma unroll 1
         for (uint32_t b = warp; b < B; b += kRgThreads / 32) {
             const uint32_t cnt = s_m->cnt[b];
             uint32_t adv = 0;
+            #pragma unroll 1
             for (uint32_t t = lane; t < ((cnt + 31) & ~31u); t += 32) {
                 bool take = false;
                 if (t < cnt) {
@@ -278,6 +281,7 @@ k_apply_ranges(ServerParams sp, RangeDesc d, const uint32_t* __restrict__ idx, c
         // ---- pairs: one thread per staged pair.  Heads and Theta are only written at once where no other
         // pair of the round looks at the parameter: never while a zero-valued pair is around
         const bool at_once = s_m->any_zero == 0;
+        #pragma unroll 1
         for (uint32_t b = warp; b < B; b += kRgThreads / 32) {
             const uint32_t cnt = s_m->adv[b];                   // ascending list: the pairs below the limit lead
             const uint32_t cur_b = s_m->cur[b], pos_b = s_m->pos[b] + cur_b, bits_b = s_m->bits[b];
@@ -347,6 +351,7 @@ k_apply_ranges(ServerParams sp, RangeDesc d, const uint32_t* __restrict__ idx, c
         __syncthreads();
         // ---- sums: one thread per parameter changed more than once, its steps in arrival order
         const uint32_t n_listed = s_m->n_listed;
+        #pragma unroll 1
         for (uint32_t j = tid; j < n_listed; j += kRgThreads) {
             const uint32_t kl = s_list[j];
             uint32_t m = s_mask[kl], t = 0, b = 0;
@@ -469,6 +474,7 @@ k_apply_sweep(ServerParams sp, SweepDesc d, const uint32_t* __restrict__ idx, co
             }
         }
         // ---- stage
+        #pragma unroll 1
         for (uint32_t b = warp; b < B; b += kSwThreads / 32) {
             const uint64_t begin = s_m->begin[b];
             const uint32_t n_b = s_m->n[b], cur = s_m->cur[b] + s_m->adv[b];     // past what the last round consumed
@@ -528,12 +534,14 @@ k_apply_sweep(ServerParams sp, SweepDesc d, const uint32_t* __restrict__ idx, co
         __syncthreads();
         const uint32_t limit = s_m->limit;
         // ---- pairs: one thread per staged pair below the limit
+        #pragma unroll 1
         for (uint32_t b = warp; b < B; b += kSwThreads / 32) {
             const uint32_t cnt = s_m->cnt[b], pos_b = s_m->pos[b], bits_b = s_m->bits[b];
             const uint32_t below_b = (1u << b) - 1u, ws = s_m->win[b];
             const bool pre_b = (d.o.pre_mask >> b) & 1u;
             uint32_t* sig = sigma_out ? sigma_out + s_m->begin[b] + s_m->cur[b] : nullptr;
             uint32_t adv = 0;
+            #pragma unroll 1
             for (uint32_t t = lane; t < ((cnt + 31) & ~31u); t += 32) {
                 bool take = false;
                 if (t < cnt) {

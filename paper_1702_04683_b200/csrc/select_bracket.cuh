@@ -288,6 +288,7 @@ __global__ void __launch_bounds__(kThreads, 4) k_bracket_scan(SelectParams p, ui
 
         // ================= tail, pass A: fetch the queued loads again (an L1 / L2 hit: the round is
         // short), classify their entries with every lane busy, count per piece
+        #pragma unroll 1
         for (uint32_t t = lane; t < qn; t += 32) {
             const uint32_t ent = q[t];
             const uint32_t pj = ent >> 8;
@@ -336,6 +337,7 @@ __global__ void __launch_bounds__(kThreads, 4) k_bracket_scan(SelectParams p, ui
                 make_uint2(cb + ((inc - mycnt) & 0xFFFFu), tc | ((tc - tw) << 16));
         }
         uint32_t run = cb, wrun = wb;
+        #pragma unroll 1
         for (uint32_t t0 = 0; t0 < qn; t0 += 32) {
             const uint32_t t = t0 + lane;
             uint32_t nc = 0, nw = 0, v = 0;
@@ -373,10 +375,12 @@ __global__ void __launch_bounds__(kThreads, 4) k_bracket_scan(SelectParams p, ui
             }
             __syncwarp();
             const uint32_t n_c = tot32 & 0xFFFFu, n_w = tot32 >> 16;
+            #pragma unroll 1
             for (uint32_t r = lane; r < n_c; r += 32) {
                 cand_idx[run + r] = stage_idx[r];
                 cand_val[run + r] = stage_val[r];
             }
+            #pragma unroll 1
             for (uint32_t r = lane; r < n_w; r += 32) {
                 win_idx[wrun + r] = stage_widx[r];
                 win_key[wrun + r] = stage_wkey[r];
