@@ -34,11 +34,11 @@ UNIT = "GB/s"
 FALLBACK_HBM_GBS = 6650.0
 
 # DRAM bytes (read + write) of ONE scan-kernel launch, from the ncu capture summarised in
-# profiles/dram_traffic_large_flat_w4.md: workload 4 with 4 workers, MB per keep fraction (1/10 is
-# the dense scan kernel).  A launch over W workers moves W / 4 times as much.  Only valid while
+# profiles/dram_traffic_large_flat_w4.md: workload 4 with 4 workers, MB per keep fraction (1/25 and
+# 1/10 are the dense scan kernel).  A launch over W workers moves W / 4 times as much.  Only valid while
 # the kernel source is the one that was profiled.
-SCAN_TRAFFIC_W4_MB = {"1/1000": 1647.5, "1/400": 1686.0, "1/160": 1797.2, "1/64": 1789.0, "1/25": 1865.3, "1/10": 2013.6}
-SCAN_SOURCE_SHA256_16 = "58db70353905ced6"
+SCAN_TRAFFIC_W4_MB = {"1/1000": 1647.3, "1/400": 1685.3, "1/160": 1798.1, "1/64": 1791.7, "1/25": 1789.3, "1/10": 2007.4}
+SCAN_SOURCE_SHA256_16 = "fafde59f6b7c9c48"
 
 
 def scan_traffic_bytes(workload_index, keeps, workers):
@@ -303,7 +303,7 @@ def run_native(args):
         # dominant kernel: the single streaming pass over the dense gradients.  Algorithmic bytes per
         # launch = workers x 4 bytes x parameters; duration = mean over its launches in the timed
         # region, from CUDA events recorded on the launching stream around the kernel.
-        "roofline": {"bound": "hbm", "kernel": "k_bracket_scan", "launches_timed": int(scan_launches),
+        "roofline": {"bound": "hbm", "kernel": "k_bracket_scan (k_bracket_scan_dense where 3 % of the entries or more are candidates)", "launches_timed": int(scan_launches),
                      "achieved": round(scan_bytes_all / scan_ms_all / 1e6, 1) if scan_ms_all else None,
                      "peak": peak, "peak_kind": "of " + peak_kind, "unit": "GB/s",
                      "frac": round(scan_bytes_all / scan_ms_all / 1e6 / peak, 4) if scan_ms_all else None,
