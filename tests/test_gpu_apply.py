@@ -201,6 +201,39 @@ def test_clustered_and_uneven_updates(binding, mode):
     assert np.array_equal(bits(theta), bits(ref.theta()))
 
 
+@pytest.mark.parametrize("mode", MODES)
+def test_parameters_on_an_odd_address_and_odd_count(binding, mode):
+    """Theta as a view that starts 4 bytes past a 16-byte boundary, with a parameter count that is
+    no multiple of 4: vector accesses must not be assumed."""
+    P = 70_001
+    rng = np.random.default_rng(3)
+    buf = torch.from_numpy(rng.standard_normal(P + 8).astype(np.float32)).to(DEV)
+    theta = buf[1:P + 1]
+    assert theta.data_ptr() % 16 == 4
+    guard_lo, guard_hi = buf[0].item(), buf[P + 1:].clone()
+    ref = oracle.Server(theta.cpu().numpy())
+    srv = binding.Server(theta, history_pairs=1 << 18, max_window_updates=16)
+    srv.set_mode(mode)
+    ts = 0
+    for call in range(2):
+        ups = [np.sort(rng.choice(P, size, replace=False)).astype(np.uint32) for size in (30_000, 9_000, 50_000, 700, P)]
+        vals = [rng.standard_normal(a.size).astype(np.float32) for a in ups]
+        begin = np.concatenate([[0], np.cumsum([a.size for a in ups])[:-1]]).astype(np.uint64)
+        count = np.array([a.size for a in ups], np.uint32)
+        pull = np.array([max(0, ts + b - 2) for b in range(len(ups))], np.uint64)
+        idx, val = i32(np.concatenate(ups)), torch.from_numpy(np.concatenate(vals)).to(DEV)
+        sigma = torch.full_like(idx, -1)
+        srv.apply(idx, val, begin, count, pull, 0.1, sigma_out=sigma)
+        s = u32(sigma)
+        for b in range(len(ups)):
+            want = ref.apply(ups[b], vals[b], int(pull[b]), 0.1)
+            assert np.array_equal(s[int(begin[b]):int(begin[b]) + ups[b].size], want), f"call {call} update {b}"
+        ts += len(ups)
+    assert srv.last_error() == 0
+    assert np.array_equal(bits(theta), bits(ref.theta()))
+    assert buf[0].item() == guard_lo and torch.equal(buf[P + 1:], guard_hi)      # nothing written outside Theta
+
+
 def test_window_and_capacity_errors_leave_the_server_unchanged(binding):
     theta = torch.zeros(100, device=DEV)
     srv = binding.Server(theta, history_pairs=40, max_window_updates=8)     # ring of 64 pairs

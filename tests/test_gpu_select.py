@@ -145,6 +145,30 @@ def test_awkward_value_layouts_stay_exact_and_ties_fall_back(binding):
     assert sel.last_error() == (0, 1)
 
 
+def test_dense_candidates_crowded_and_spread(binding):
+    """Keep fractions of 5-20 %, where the compacting scan kernel runs: spread-out data stays on the
+    single-pass route; a stretch in which every entry is large cannot be staged and the tensor is
+    handed to the general route.  Either way the answer is exact."""
+    dev = torch.device("cuda", 0)
+    n = 1_500_001
+    g = torch.randn(4, n + 3, device=dev)[:, 1:n + 1]
+    g[1] = g[1] * torch.rand(n, device=dev) ** 4                       # heavy concentration near zero
+    g[2, 200_000:420_000] *= 1000.0                                    # 220 000 large entries in one stretch
+    g[3] = torch.round(g[3] * 8) / 8                                   # coarse grid: many ties at every level
+    for k, general_expected in ((75_000, None), (150_000, None), (300_000, None)):
+        segs = binding.segments_from([0], [n], [k])
+        sel = binding.Selector(segs, 4, dev)
+        idx, val = sel.select(g)
+        status, general = sel.last_error()
+        assert status == 0
+        for w in range(4):
+            oi, ov = oracle.select(g[w].cpu().numpy(), k)
+            assert np.array_equal(u32(idx[w]), oi), (k, w)
+            assert np.array_equal(bits(val[w]), bits(ov)), (k, w)
+        assert general >= 1                                            # the crowded worker (and the tied one) fell back
+        assert general <= 2
+
+
 @pytest.mark.parametrize("n,k", [(32_768, 1), (32_768, 8192), (40_000, 400), (65_537, 700), (1 << 20, 1), (3_000_001, 30_001)])
 def test_bracket_route_sizes(binding, n, k):
     dev = torch.device("cuda", 0)
