@@ -52,7 +52,7 @@ def lib():
                 f.argtypes = [f32p, ctypes.c_uint32, ctypes.c_uint32, ctypes.c_uint64, u32p, f32p]
             L.oracle_select_layers.restype = ctypes.c_int
             L.oracle_select_layers.argtypes = [f32p, u64p, u32p, u32p, ctypes.c_uint32, ctypes.c_int, u32p, f32p]
-            for kind in ("literal", "server"):
+            for kind in ("literal", "server", "global"):
                 getattr(L, f"oracle_{kind}_create").restype = ctypes.c_void_p
                 getattr(L, f"oracle_{kind}_create").argtypes = [ctypes.c_uint64, f32p]
                 getattr(L, f"oracle_{kind}_destroy").restype = None
@@ -64,6 +64,10 @@ def lib():
                 getattr(L, f"oracle_{kind}_apply").restype = ctypes.c_int
                 getattr(L, f"oracle_{kind}_apply").argtypes = [
                     ctypes.c_void_p, u32p, f32p, ctypes.c_uint64, ctypes.c_uint64, ctypes.c_float, u32p]
+            L.oracle_global_apply_dense.restype = ctypes.c_int
+            L.oracle_global_apply_dense.argtypes = [ctypes.c_void_p, f32p, ctypes.c_uint64, ctypes.c_float]
+            L.oracle_gather.restype = ctypes.c_int
+            L.oracle_gather.argtypes = [f32p, ctypes.c_uint64, u32p, ctypes.c_uint64, f32p]
             L.oracle_parameter_trace.restype = ctypes.c_int
             L.oracle_parameter_trace.argtypes = [
                 ctypes.c_uint32, ctypes.c_float, u32p, f32p, u64p, u64p, ctypes.c_uint64, ctypes.c_uint64,
@@ -112,10 +116,14 @@ def select_layers(grad, offsets, ns, ks, full_sort: bool = False):
 
 class Server:
     """Algorithm 2 on the CPU. ``literal=True`` evaluates Eq. 3 by membership tests
-    over every update of the window; the default keeps per-parameter timestamp lists."""
+    over every update of the window; the default keeps per-parameter timestamp lists.
+    ``rule="global"`` is the competitors' rule instead (ASGD, Comp-ASGD): one staleness
+    i - j for the whole update."""
 
-    def __init__(self, theta0, literal: bool = False):
-        self._kind = "literal" if literal else "server"
+    def __init__(self, theta0, literal: bool = False, rule: str = "adacomp"):
+        if rule not in ("adacomp", "global"):
+            raise ValueError("rule must be 'adacomp' or 'global'")
+        self._kind = "global" if rule == "global" else ("literal" if literal else "server")
         theta0 = _f32(theta0).ravel()
         self.n_params = theta0.size
         self._h = getattr(lib(), f"oracle_{self._kind}_create")(self.n_params, _p(theta0, ctypes.c_float))
@@ -131,6 +139,16 @@ class Server:
         if rc != 0:
             raise ValueError("oracle apply: bad push (j > i, index out of range or not ascending)")
         return sigma
+
+    def apply_dense(self, delta, pull_ts: int, alpha: float):
+        """One dense push (the whole gradient, ASGD); only under rule="global"."""
+        if self._kind != "global":
+            raise ValueError("dense pushes belong to the global-staleness rule")
+        delta = _f32(delta).ravel()
+        if delta.size != self.n_params:
+            raise ValueError("a dense push has one entry per parameter")
+        if lib().oracle_global_apply_dense(self._h, _p(delta, ctypes.c_float), int(pull_ts), float(alpha)) != 0:
+            raise ValueError("oracle apply_dense: bad push (j > i)")
 
     @property
     def timestamp(self) -> int:
@@ -151,6 +169,16 @@ class Server:
             self.close()
         except Exception:
             pass
+
+
+def gather(g, idx):
+    """val[e] = g[idx[e]]."""
+    g = _f32(g).ravel()
+    idx = np.ascontiguousarray(idx, dtype=np.uint32)
+    out = np.empty(idx.size, dtype=np.float32)
+    if lib().oracle_gather(_p(g, ctypes.c_float), g.size, _p(idx, ctypes.c_uint32), idx.size, _p(out, ctypes.c_float)) != 0:
+        raise ValueError("oracle gather: index out of range")
+    return out
 
 
 def parameter_trace(k: int, theta0_k: float, idx, val, pair_begin, pull_ts, alpha: float,

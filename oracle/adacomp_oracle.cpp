@@ -9,7 +9,9 @@
 //
 // Parity status: every function below is pinned by tests that do not call it
 // to produce their expectation (brute-force set definitions on tiny inputs,
-// the paper's worked staleness example, closed forms, invariants).  The only
+// the paper's worked staleness example, closed forms, invariants; for the
+// competitors' global-staleness rule also its agreement with the per-parameter
+// rule on full updates, where the two must coincide).  The only
 // thing that stays "parity unpinned" is what this file does not compute at
 // all: model accuracy and traffic curves, which need the paper's dataset.
 //
@@ -236,6 +238,70 @@ int oracle_server_apply(void* h, const uint32_t* idx, const float* val, uint64_t
         }
     }
     s->timestamp = i + 1;
+    return 0;
+}
+
+// --- the competitors' rule ------------------------------------------------------
+// ASGD and Comp-ASGD ("Experimental setup"): "the learning rate is divided by
+// staleness and is global to each update".  The staleness of an update is the
+// number of times Theta has evolved between the fetch at timestamp j and the push
+// at timestamp i ("The parameter server model": w2's update on Figure 2 has
+// staleness 2), i.e. sigma = i - j, the same for every entry of the update.  The
+// update itself is Eq. 4 with alpha / sigma (alpha when sigma = 0, as in Eq. 5),
+// applied to every entry as written: no history is needed and none is kept.
+struct GlobalServer {
+    std::vector<float> theta;
+    uint64_t timestamp = 0;
+};
+
+void* oracle_global_create(uint64_t n_params, const float* theta0) {
+    auto* s = new GlobalServer;
+    s->theta.assign(theta0, theta0 + n_params);
+    return s;
+}
+void oracle_global_destroy(void* h) { delete static_cast<GlobalServer*>(h); }
+uint64_t oracle_global_timestamp(void* h) { return static_cast<GlobalServer*>(h)->timestamp; }
+void oracle_global_theta(void* h, float* out) {
+    auto* s = static_cast<GlobalServer*>(h);
+    std::copy(s->theta.begin(), s->theta.end(), out);
+}
+
+// A sparse update (Comp-ASGD: a selection of the gradient entries).
+int oracle_global_apply(void* h, const uint32_t* idx, const float* val, uint64_t n_pairs,
+                        uint64_t j, float alpha, uint32_t* sigma_out) {
+    auto* s = static_cast<GlobalServer*>(h);
+    const uint64_t i = s->timestamp;
+    if (j > i || i - j > 0xFFFFFFFFull) return -1;
+    for (uint64_t e = 0; e < n_pairs; ++e) {
+        if (idx[e] >= s->theta.size()) return -1;
+        if (e > 0 && idx[e] <= idx[e - 1]) return -1;
+    }
+    const uint32_t sigma = static_cast<uint32_t>(i - j);
+    for (uint64_t e = 0; e < n_pairs; ++e) {
+        if (sigma_out) sigma_out[e] = sigma;
+        s->theta[idx[e]] = updated_parameter(s->theta[idx[e]], alpha, sigma, val[e]);
+    }
+    s->timestamp = i + 1;
+    return 0;
+}
+
+// A dense update (ASGD: the whole gradient).
+int oracle_global_apply_dense(void* h, const float* delta, uint64_t j, float alpha) {
+    auto* s = static_cast<GlobalServer*>(h);
+    const uint64_t i = s->timestamp;
+    if (j > i || i - j > 0xFFFFFFFFull) return -1;
+    const uint32_t sigma = static_cast<uint32_t>(i - j);
+    for (size_t k = 0; k < s->theta.size(); ++k) s->theta[k] = updated_parameter(s->theta[k], alpha, sigma, delta[k]);
+    s->timestamp = i + 1;
+    return 0;
+}
+
+// Values of chosen entries: val[e] = g[idx[e]] (a selection made elsewhere, e.g. at random).
+int oracle_gather(const float* g, uint64_t n, const uint32_t* idx, uint64_t n_pairs, float* val_out) {
+    for (uint64_t e = 0; e < n_pairs; ++e) {
+        if (idx[e] >= n) return -1;
+        val_out[e] = g[idx[e]];
+    }
     return 0;
 }
 
