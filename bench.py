@@ -57,6 +57,69 @@ def scan_traffic_bytes(workload_index, keeps, workers):
     return sum(per) / len(per)
 
 
+def run_competitors(binding, wl, grads, dev, peak, keep=(1, 100), reps=5, warmup=3):
+    """The paper's two competitors on the same inputs, next to AdaComp at the same keep fraction:
+    ASGD (dense updates) and Comp-ASGD (whole-model top-k), both with the learning rate divided by the
+    update's staleness.  Every worker pulls at the start of a round; a round = W updates.  Ingress
+    bytes per update follow the paper's accounting (size of what the server receives)."""
+    W, P = grads.shape[0], wl.n_params
+    stream = torch.cuda.current_stream()
+
+    def timed(fn):
+        for _ in range(warmup):
+            fn()
+        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        a.record(stream)
+        for _ in range(reps):
+            fn()
+        b.record(stream)
+        torch.cuda.synchronize()
+        return a.elapsed_time(b) / reps
+
+    out = {"keep": "%d/%d" % keep, "workers": W, "round": "W updates, all pulled at the start of the round"}
+    begin = lambda K: np.arange(W, dtype=np.uint64) * np.uint64(K)
+    # ASGD: W dense updates
+    theta = wlmod.initial_parameters(wl, dev)
+    srv = binding.Server(theta, history_pairs=1, max_window_updates=2 * W)
+    srv.set_rule(1)
+    def asgd_round():
+        ts = srv.timestamp
+        for w in range(W):
+            srv.apply_dense(grads[w, :P], ts, wl.lr)
+    ms = timed(asgd_round)
+    out["asgd"] = {"apply_ms_per_round": round(ms, 4), "updates_per_s": round(W / ms * 1e3, 1),
+                   "apply_gbs_12B_per_param": round(W * 12.0 * P / ms / 1e6, 1),
+                   "apply_frac_of_hbm_peak": round(W * 12.0 * P / ms / 1e6 / peak, 4),
+                   "ingress_bytes_per_update": 4 * P}
+    assert srv.last_error() == 0
+    # Comp-ASGD: whole-model top-k (one segment), sparse updates under the global rule
+    k = binding.adacomp_keep_count(P, keep[0], keep[1])
+    sel = binding.Selector(binding.segments_from([0], [P], [k]), W, dev)
+    idx, val = sel.select(grads)
+    sel_ms = timed(lambda: sel.select(grads, idx, val))
+    count = np.full(W, k, np.uint32)
+    app_ms = timed(lambda: srv.apply(idx.view(-1), val.view(-1), begin(k), count, np.full(W, srv.timestamp, np.uint64), wl.lr))
+    out["comp_asgd"] = {"select": "one segment over all %d parameters (larger than the single-pass route takes: five reads)" % P,
+                        "select_ms_per_round": round(sel_ms, 4), "select_scanned_gbs": round(W * 4.0 * P / sel_ms / 1e6, 1),
+                        "apply_ms_per_round": round(app_ms, 4), "apply_pairs_per_s": round(W * k / app_ms * 1e3, 1),
+                        "ingress_bytes_per_update": 8 * k}
+    assert sel.last_error()[0] == 0 and srv.last_error() == 0
+    del sel, srv
+    # AdaComp at the same keep fraction: per-tensor top-k, per-parameter staleness
+    sel = binding.Selector(binding.make_segments(wl.tensor_sizes, keep), W, dev)
+    K = sel.pairs_per_worker
+    idx, val = sel.select(grads)
+    sel_ms = timed(lambda: sel.select(grads, idx, val))
+    srv = binding.Server(theta, history_pairs=2 * W * K, max_window_updates=2 * W)
+    count = np.full(W, K, np.uint32)
+    app_ms = timed(lambda: srv.apply(idx.view(-1), val.view(-1), begin(K), count, np.full(W, srv.timestamp, np.uint64), wl.lr))
+    out["adacomp"] = {"select_ms_per_round": round(sel_ms, 4), "select_scanned_gbs": round(W * 4.0 * P / sel_ms / 1e6, 1),
+                      "apply_ms_per_round": round(app_ms, 4), "apply_pairs_per_s": round(W * K / app_ms * 1e3, 1),
+                      "ingress_bytes_per_update": 8 * K}
+    assert sel.last_error()[0] == 0 and srv.last_error() == 0
+    return out
+
+
 def parse_args():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -70,6 +133,7 @@ def parse_args():
     ap.add_argument("--apply-mode", type=int, default=0)
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--no-competitors", action="store_true")
     return ap.parse_args()
 
 
@@ -313,6 +377,8 @@ def run_native(args):
                                      "achieved": round(sel_bytes_all / sel_ms_all / 1e6, 1),
                                      "frac": round(sel_bytes_all / sel_ms_all / 1e6 / peak, 4)}},
     }
+    if world == 1 and not args.no_competitors and args.keep is None:
+        out["competitors"] = run_competitors(binding, wl, grads, dev, peak)
     if world == 1 and not args.no_e2e:
         out["e2e"] = run_e2e(args, binding, wl, points, srv, grads, rng, last_push, dev, stream)
     if world == 1 and rank == 0 and not args.no_cpu_baseline:

@@ -147,6 +147,16 @@ ADACOMP_API const char* adacomp_select_stage_name(uint32_t stage);
 
 /* K = sum of k over the layout's segments (pairs per worker). */
 ADACOMP_API int adacomp_select_pairs_per_worker(const adacomp_select_t* h, uint64_t* pairs_out);
+/* Values of entries chosen elsewhere: d_val_out[w][e] = d_grads[w][d_idx[w][e]] for the handle's
+ * K = pairs_per_worker entries of each of n_workers workers (same layouts as adacomp_select).
+ * Serves selections the library does not make itself, e.g. the random selection that one variant
+ * of Comp-ASGD uses ("Compression" paragraph: the subset is chosen "randomly, or by keeping only
+ * the largest gradients"); the random draw is the caller's.  An index outside the layout's extent
+ * reads as 0 and is reported by adacomp_select_last_error as ADACOMP_ERR_INVALID. */
+ADACOMP_API int adacomp_select_gather(adacomp_select_t* h, const float* d_grads, uint64_t worker_stride_elems,
+                                      uint32_t n_workers, const uint32_t* d_idx, float* d_val_out,
+                                      void* cuda_stream);
+
 /* Waits for cuda_stream, then returns the first error the device recorded since the last call
  * of this function (ADACOMP_OK if none) and clears it.  Also reports, if stats_out is not
  * NULL, stats_out[0] = how many (worker, segment) selections of the last adacomp_select call
@@ -267,6 +277,21 @@ ADACOMP_API int adacomp_server_set_validation(adacomp_server_t* s, int on);
  * Updates whose pair slices overlap in memory, with d_sigma_out given, always go as 1: their
  * staleness slots are shared and the later update's count must be the one that stays. */
 ADACOMP_API int adacomp_server_set_mode(adacomp_server_t* s, int mode);
+/* Which rule adacomp_apply follows.
+ * 0 = AdaComp (default): per-parameter staleness sigma_k of Eq. 3, learning rate of Eq. 5.
+ * 1 = the competitors' rule of the "Experimental setup" (ASGD, Comp-ASGD: "the learning rate is
+ *     divided by staleness and is global to each update"): every entry of an update that pulled
+ *     at j and is applied at timestamp i gets alpha / (i - j) (alpha if i = j), Eq. 4 is applied
+ *     to every entry as written (zero-valued ones too), d_sigma_out receives i - j, and no history
+ *     is read or kept.  ADACOMP_ERR_WINDOW if j > i or i - j >= 2^24.
+ * The rule can only be changed while the timestamp is 0 (after create or reset): ADACOMP_ERR_INVALID
+ * otherwise. */
+ADACOMP_API int adacomp_server_set_rule(adacomp_server_t* s, int rule);
+/* A dense update under rule 1 (ASGD pushes the whole gradient): Theta <- Theta - alpha / (i - j) *
+ * d_delta, d_delta[n_params] in device memory; the timestamp advances by one.
+ * ADACOMP_ERR_INVALID under rule 0 (a dense AdaComp update is adacomp_apply with every index). */
+ADACOMP_API int adacomp_apply_dense(adacomp_server_t* s, const float* d_delta, uint64_t pull_ts, float lr,
+                                    void* cuda_stream);
 /* Test hook: advances the history position counter as if `count` more pairs had been applied
  * (their history is empty).  Lets a test reach the 32-bit position re-basing that otherwise
  * happens once per ~4 * 10^9 applied pairs.  Call right after adacomp_server_reset. */

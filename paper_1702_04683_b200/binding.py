@@ -72,6 +72,9 @@ def _load():
         "adacomp_server_timestamp": (i32, [vp, P(u64)]),
         "adacomp_server_set_validation": (i32, [vp, i32]),
         "adacomp_server_set_mode": (i32, [vp, i32]),
+        "adacomp_server_set_rule": (i32, [vp, i32]),
+        "adacomp_apply_dense": (i32, [vp, vp, u64, f32, vp]),
+        "adacomp_select_gather": (i32, [vp, vp, u64, u32, vp, vp, vp]),
         "adacomp_server_debug_skip_positions": (i32, [vp, u64]),
         "adacomp_server_last_error": (i32, [vp, vp]),
         "adacomp_server_destroy": (i32, [vp]),
@@ -218,6 +221,22 @@ class Selector:
                                         _host(h_val, torch.float32, "h_val"), _stream_ptr(stream)),
                "adacomp_select_host")
 
+    def gather(self, grads: torch.Tensor, idx: torch.Tensor, val_out: Optional[torch.Tensor] = None,
+               stream: Optional[torch.cuda.Stream] = None) -> torch.Tensor:
+        """val[w][e] = grads[w][idx[w][e]] for idx of shape [W, pairs_per_worker]."""
+        g = grads if grads.dim() == 2 else grads.unsqueeze(0)
+        W = g.shape[0]
+        if idx.numel() != W * self.pairs_per_worker:
+            raise ValueError("idx needs pairs_per_worker entries per worker")
+        if val_out is None:
+            val_out = torch.empty((W, self.pairs_per_worker), dtype=torch.float32, device=g.device)
+        if g.stride(1) != 1 or not (g.is_cuda and g.dtype == torch.float32):
+            raise TypeError("grads: need a CUDA fp32 tensor whose innermost dimension is contiguous")
+        _check(_lib.adacomp_select_gather(self._h, g.data_ptr(), g.stride(0) if W > 1 else g.shape[1],
+                                          W, _dev(idx, torch.int32, "idx"), _dev(val_out, torch.float32, "val_out"),
+                                          _stream_ptr(stream)), "adacomp_select_gather")
+        return val_out
+
     def set_route(self, route: int):
         """0 = automatic (bracketed single pass where eligible), 1 = general route only."""
         _check(_lib.adacomp_select_set_route(self._h, int(route)), "adacomp_select_set_route")
@@ -327,6 +346,17 @@ class Server:
     def set_mode(self, mode: int):
         """0 automatic, 1 one launch per update, 2 batches by parameter ranges, 3 batches over a dense sweep."""
         _check(_lib.adacomp_server_set_mode(self._h, int(mode)), "adacomp_server_set_mode")
+
+    def set_rule(self, rule: int):
+        """0 AdaComp (per-parameter staleness), 1 the competitors' rule (the update's staleness i - j)."""
+        _check(_lib.adacomp_server_set_rule(self._h, int(rule)), "adacomp_server_set_rule")
+
+    def apply_dense(self, delta: torch.Tensor, pull_ts: int, lr: float, stream: Optional[torch.cuda.Stream] = None):
+        """One dense update under rule 1: Theta <- Theta - lr / (i - pull_ts) * delta."""
+        if delta.numel() != self.n_params:
+            raise ValueError("a dense update has one entry per parameter")
+        _check(_lib.adacomp_apply_dense(self._h, _dev(delta, torch.float32, "delta"), int(pull_ts), float(lr),
+                                        _stream_ptr(stream)), "adacomp_apply_dense")
 
     def debug_skip_positions(self, count: int):
         _check(_lib.adacomp_server_debug_skip_positions(self._h, int(count)), "adacomp_server_debug_skip_positions")

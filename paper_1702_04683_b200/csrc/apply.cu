@@ -625,6 +625,43 @@ k_apply_sweep(ServerParams sp, SweepDesc d, const uint32_t* __restrict__ idx, co
     if (r_hi == n_ranges && tid < B && s_m->cur[tid] + s_m->adv[tid] < s_m->n[tid]) record_error(sp.status, ADACOMP_ERR_UNSORTED);
 }
 
+// ---------------------------------------------------------------------------------------------
+// The competitors' rule ("Experimental setup": for ASGD and Comp-ASGD the learning rate is divided
+// by staleness and is global to each update): every entry of an update gets the same learning
+// rate alpha / (i - j), which the host has already computed (one fp32 division); Eq. 4 is applied
+// to every entry as written.  No history is read or kept.  One launch per update, the stream
+// orders updates.
+__global__ void __launch_bounds__(kApplyThreads)
+k_apply_global(ServerParams sp, UpdateDesc u, const uint32_t* __restrict__ idx, const float* __restrict__ val,
+               float alpha_u, uint32_t sigma_u, uint32_t* sigma_out) {
+    const uint32_t e = blockIdx.x * kApplyThreads + threadIdx.x;
+    if (e >= u.n_pairs) return;
+    const uint64_t at = u.pair_begin + e;
+    const uint32_t k = idx[at];
+    if (k >= sp.n_params) { record_error(sp.status, ADACOMP_ERR_UNSORTED); return; }
+    if (sp.validate && e > 0 && idx[at - 1] >= k) { record_error(sp.status, ADACOMP_ERR_UNSORTED); return; }
+    if (sigma_out) sigma_out[at] = sigma_u;
+    sp.theta[k] = __fsub_rn(sp.theta[k], __fmul_rn(alpha_u, val[at]));                             // Eq. 4
+}
+
+// A dense update (ASGD pushes the whole gradient): Theta <- Theta - alpha_u * delta, 16 bytes per
+// thread and step where both arrays allow it (`vec` = number of leading float4 groups).
+__global__ void __launch_bounds__(kApplyThreads)
+k_apply_dense(float* __restrict__ theta, const float* __restrict__ delta, uint64_t n, uint64_t vec, float alpha_u) {
+    const uint64_t stride = static_cast<uint64_t>(gridDim.x) * kApplyThreads;
+    const uint64_t t0 = static_cast<uint64_t>(blockIdx.x) * kApplyThreads + threadIdx.x;
+    for (uint64_t v = t0; v < vec; v += stride) {
+        float4 th = reinterpret_cast<float4*>(theta)[v];
+        const float4 d = __ldg(reinterpret_cast<const float4*>(delta) + v);
+        th.x = __fsub_rn(th.x, __fmul_rn(alpha_u, d.x));
+        th.y = __fsub_rn(th.y, __fmul_rn(alpha_u, d.y));
+        th.z = __fsub_rn(th.z, __fmul_rn(alpha_u, d.z));
+        th.w = __fsub_rn(th.w, __fmul_rn(alpha_u, d.w));
+        reinterpret_cast<float4*>(theta)[v] = th;
+    }
+    for (uint64_t k = vec * 4 + t0; k < n; k += stride) theta[k] = __fsub_rn(theta[k], __fmul_rn(alpha_u, delta[k]));
+}
+
 // Moves every stored position down by `delta` (entries older than that become kNone).
 __global__ void k_rebase(uint32_t* a, uint64_t n, uint32_t delta) {
     for (uint64_t i = blockIdx.x * static_cast<uint64_t>(blockDim.x) + threadIdx.x; i < n;
@@ -660,6 +697,7 @@ struct adacomp_server {
     std::vector<uint64_t> start_of;   // start_of[u % size] = absolute start position of update u
     int validate = 0;
     int mode = 0;
+    int rule = 0;                 // 0: per-parameter staleness (Eq. 3); 1: the update's staleness i - j for every entry
 };
 
 namespace {
@@ -757,11 +795,46 @@ int adacomp_apply(adacomp_server_t* s, const uint32_t* d_idx, const float* d_val
     if (!s || !s->d_theta) return ADACOMP_ERR_INVALID;
     if (n_updates == 0) return ADACOMP_OK;
     if (!h_pair_begin || !h_pair_count || !h_pull_ts) return ADACOMP_ERR_INVALID;
-    if (n_updates > s->max_window) return ADACOMP_ERR_CAPACITY;
     uint64_t call_pairs = 0;
     for (uint32_t b = 0; b < n_updates; ++b) call_pairs += h_pair_count[b];
-    if (call_pairs > s->history_pairs) return ADACOMP_ERR_CAPACITY;
     if (call_pairs && (!d_idx || !d_val)) return ADACOMP_ERR_INVALID;
+    if (s->rule == 0 && (n_updates > s->max_window || call_pairs > s->history_pairs)) return ADACOMP_ERR_CAPACITY;
+
+    if (s->rule == 1) {
+        // ---- the competitors' rule: one learning rate per update, no history
+        const uint64_t i0 = s->timestamp;
+        for (uint32_t b = 0; b < n_updates; ++b) {
+            const uint64_t i = i0 + b, j = h_pull_ts[b];
+            if (j > i || i - j >= (1ull << 24)) return ADACOMP_ERR_WINDOW;     // the staleness must be exact as a float
+        }
+        DeviceGuard guard(s->device);
+        if (guard.err != cudaSuccess) return cuda_fail(guard.err);
+        cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+        ServerParams sp;
+        sp.theta = s->d_theta;
+        sp.head = nullptr;
+        sp.prev = nullptr;
+        sp.status = s->d_status;
+        sp.n_params = s->n_params;
+        sp.ring_mask = sp.ring_shift = 0;
+        sp.max_window = s->max_window;
+        sp.validate = s->validate;
+        for (uint32_t b = 0; b < n_updates; ++b) {
+            UpdateDesc u;
+            u.pair_begin = h_pair_begin[b];
+            u.n_pairs = h_pair_count[b];
+            u.pos_start = u.win_start = u.pad = 0;
+            const uint32_t sigma_u = static_cast<uint32_t>(i0 + b - h_pull_ts[b]);
+            const float alpha_u = sigma_u ? lr / static_cast<float>(sigma_u) : lr;   // Eq. 5 with the update's staleness
+            if (u.n_pairs) {
+                const unsigned grid = (u.n_pairs + kApplyThreads - 1) / kApplyThreads;
+                k_apply_global<<<grid, kApplyThreads, 0, st>>>(sp, u, d_idx, d_val, alpha_u, sigma_u, d_sigma_out);
+                ADACOMP_LAUNCH_CHECK();
+            }
+        }
+        s->timestamp = i0 + n_updates;
+        return ADACOMP_OK;
+    }
 
     // ---- host-side window checks; nothing is enqueued and nothing changes until all pass
     const uint64_t i0 = s->timestamp;
@@ -951,6 +1024,32 @@ int adacomp_server_set_validation(adacomp_server_t* s, int on) {
 int adacomp_server_set_mode(adacomp_server_t* s, int mode) {
     if (!s || mode < 0 || mode > 3) return ADACOMP_ERR_INVALID;
     s->mode = mode;
+    return ADACOMP_OK;
+}
+
+int adacomp_server_set_rule(adacomp_server_t* s, int rule) {
+    if (!s || rule < 0 || rule > 1) return ADACOMP_ERR_INVALID;
+    if (rule != s->rule && s->timestamp != 0) return ADACOMP_ERR_INVALID;   // the history of the other rule is missing
+    s->rule = rule;
+    return ADACOMP_OK;
+}
+
+int adacomp_apply_dense(adacomp_server_t* s, const float* d_delta, uint64_t pull_ts, float lr, void* cuda_stream) {
+    if (!s || !s->d_theta || !d_delta || s->rule != 1) return ADACOMP_ERR_INVALID;
+    const uint64_t i = s->timestamp;
+    if (pull_ts > i || i - pull_ts >= (1ull << 24)) return ADACOMP_ERR_WINDOW;
+    DeviceGuard guard(s->device);
+    if (guard.err != cudaSuccess) return cuda_fail(guard.err);
+    const uint32_t sigma_u = static_cast<uint32_t>(i - pull_ts);
+    const float alpha_u = sigma_u ? lr / static_cast<float>(sigma_u) : lr;       // Eq. 5 with the update's staleness
+    const bool aligned = reinterpret_cast<uintptr_t>(s->d_theta) % 16 == 0 && reinterpret_cast<uintptr_t>(d_delta) % 16 == 0;
+    const uint64_t vec = aligned ? s->n_params / 4 : 0;
+    uint64_t want = (s->n_params / 4 + kApplyThreads - 1) / kApplyThreads;
+    const uint64_t cap = static_cast<uint64_t>(s->n_sms) * 16;
+    const unsigned grid = static_cast<unsigned>(want < 1 ? 1 : (want > cap ? cap : want));
+    k_apply_dense<<<grid, kApplyThreads, 0, static_cast<cudaStream_t>(cuda_stream)>>>(s->d_theta, d_delta, s->n_params, vec, alpha_u);
+    ADACOMP_LAUNCH_CHECK();
+    s->timestamp = i + 1;
     return ADACOMP_OK;
 }
 

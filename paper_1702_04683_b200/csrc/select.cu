@@ -438,6 +438,24 @@ int adacomp_select_last_error(adacomp_select_t* h, void* cuda_stream, uint64_t* 
     return status;
 }
 
+int adacomp_select_gather(adacomp_select_t* h, const float* d_grads, uint64_t worker_stride_elems, uint32_t n_workers,
+                          const uint32_t* d_idx, float* d_val_out, void* cuda_stream) {
+    if (!h || !d_grads || n_workers == 0 || n_workers > h->max_workers) return ADACOMP_ERR_INVALID;
+    if (worker_stride_elems < h->extent) return ADACOMP_ERR_INVALID;
+    if (h->K == 0) return ADACOMP_OK;
+    if (!d_idx || !d_val_out) return ADACOMP_ERR_INVALID;
+    DeviceGuard guard(h->device);
+    if (guard.err != cudaSuccess) return cuda_fail(guard.err);
+    const uint64_t total = static_cast<uint64_t>(h->K) * n_workers;
+    uint64_t grid = (total + kThreads - 1) / kThreads;
+    const uint64_t cap = static_cast<uint64_t>(h->n_sms) * 32;
+    if (grid > cap) grid = cap;
+    k_gather<<<static_cast<unsigned>(grid), kThreads, 0, static_cast<cudaStream_t>(cuda_stream)>>>(
+        d_grads, worker_stride_elems, h->extent, d_idx, d_val_out, h->K, total, h->d_status);
+    ADACOMP_LAUNCH_CHECK();
+    return ADACOMP_OK;
+}
+
 int adacomp_select_destroy(adacomp_select_t* h) {
     if (h && h->ev[0][0]) {
         DeviceGuard guard(h->device);

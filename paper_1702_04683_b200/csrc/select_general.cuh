@@ -422,4 +422,21 @@ __global__ void __launch_bounds__(kThreads) k_general_write(SelectParams p) {
     }
 }
 
+// ---------------------------------------------------------------------------------------------
+// Values of entries chosen elsewhere (e.g. a random selection, as one of the Comp-ASGD variants
+// makes): val[w][e] = g[w][idx[w][e]].  An index outside the layout is reported and reads as 0.
+__global__ void __launch_bounds__(kThreads)
+k_gather(const float* __restrict__ grads, uint64_t stride, uint64_t extent, const uint32_t* __restrict__ idx,
+         float* __restrict__ val_out, uint64_t pairs_per_worker, uint64_t total, int* status) {
+    for (uint64_t t = static_cast<uint64_t>(blockIdx.x) * kThreads + threadIdx.x; t < total;
+         t += static_cast<uint64_t>(gridDim.x) * kThreads) {
+        const uint64_t w = t / pairs_per_worker;
+        const uint32_t k = idx[t];
+        float v = 0.f;
+        if (k < extent) v = __ldg(grads + w * stride + k);
+        else record_error(status, ADACOMP_ERR_INVALID);
+        val_out[t] = v;
+    }
+}
+
 }  // namespace adacomp
