@@ -217,6 +217,56 @@ def arrival_schedule(wl: Workload) -> List[Round]:
     return rounds
 
 
+@dataclasses.dataclass
+class ClosedLoop:
+    """A sequence of pushes as an emulated platform would produce it: ``worker[u]`` pushes update u
+    (u = the server's timestamp when it is applied) computed from the parameters it pulled at
+    ``pull_ts[u]``.  ``klass[w]`` is the speed class of worker w, ``crashed_after[w]`` the number of
+    pushes after which worker w stopped for good (-1: still alive at the end)."""
+    worker: np.ndarray
+    pull_ts: np.ndarray
+    klass: np.ndarray
+    crashed_after: np.ndarray
+
+
+def closed_loop_schedule(n_workers: int, n_updates: int, seed: int = 0,
+                         class_fractions: Sequence[float] = (1.0,), class_rates: Sequence[float] = (1.0,),
+                         crash_probability: float = 0.0) -> ClosedLoop:
+    """Event-driven emulation of the workers' loop (Algorithm 1: pull, compute, push, pull again at
+    once).  A worker of class c needs an exponentially distributed time with mean 1 / class_rates[c]
+    per update, so classes send updates in the ratio of their rates; the first
+    round(class_fractions[0] * n_workers) workers are in class 0, and so on (the heterogeneity
+    experiment: fractions 0.3 / 0.4 / 0.3 with rates 100 : 10 : 1).  After each of its pushes a worker
+    stops for good with probability ``crash_probability`` (the fail-stop experiment: 0.004).  The
+    sequence ends after ``n_updates`` pushes, or earlier if every worker has stopped."""
+    import heapq
+    if len(class_fractions) != len(class_rates) or abs(sum(class_fractions) - 1.0) > 1e-9:
+        raise ValueError("one rate per class, fractions summing to 1")
+    rng = np.random.default_rng(seed * 7919 + 13)
+    bounds = np.round(np.cumsum(class_fractions) * n_workers).astype(np.int64)
+    klass = np.searchsorted(bounds, np.arange(n_workers), side="right").astype(np.int64)
+    klass = np.minimum(klass, len(class_rates) - 1)
+    rate = np.asarray(class_rates, dtype=np.float64)[klass]
+    heap = [(float(rng.exponential(1.0 / rate[w])), w) for w in range(n_workers)]
+    heapq.heapify(heap)
+    pulled_at = np.zeros(n_workers, dtype=np.int64)
+    pushes = np.zeros(n_workers, dtype=np.int64)
+    crashed_after = np.full(n_workers, -1, dtype=np.int64)
+    worker, pull_ts = [], []
+    while heap and len(worker) < n_updates:
+        t, w = heapq.heappop(heap)
+        worker.append(w)
+        pull_ts.append(pulled_at[w])
+        pushes[w] += 1
+        pulled_at[w] = len(worker)                        # pulls again right after its own push
+        if crash_probability > 0.0 and rng.random() < crash_probability:
+            crashed_after[w] = pushes[w]
+        else:
+            heapq.heappush(heap, (t + float(rng.exponential(1.0 / rate[w])), w))
+    return ClosedLoop(worker=np.asarray(worker, dtype=np.int64), pull_ts=np.asarray(pull_ts, dtype=np.uint64),
+                      klass=klass, crashed_after=crashed_after)
+
+
 def describe(wl: Workload) -> dict:
     return {"workload": wl.name, "tensors": len(wl.tensor_sizes), "params": wl.n_params,
             "workers": wl.n_workers, "rounds": wl.n_rounds,

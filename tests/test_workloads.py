@@ -1,5 +1,6 @@
 """The synthetic input generators: shapes, determinism, schedule structure."""
 import numpy as np
+import pytest
 import torch
 
 from paper_1702_04683_b200 import workloads as wlmod
@@ -77,3 +78,45 @@ def test_schedule_uniform_staleness():
     assert np.all(lag >= 0) and np.all(lag <= 7) and np.all(rd.pull_ts.astype(np.int64) >= 0)
     (rd0,) = wlmod.arrival_schedule(wlmod.workload(0))
     assert not rd0.pull_ts.any()
+
+
+def test_closed_loop_heterogeneous_classes():
+    """Three classes in proportions 30 / 40 / 30 % whose workers send updates in the ratio 100 : 10 : 1
+    (the heterogeneity experiment); pulls follow the worker's own push."""
+    n, N = 200, 60_000
+    cl = wlmod.closed_loop_schedule(n, N, seed=3, class_fractions=(0.3, 0.4, 0.3), class_rates=(100, 10, 1))
+    assert np.bincount(cl.klass).tolist() == [60, 80, 60]
+    assert cl.worker.size == N and (cl.crashed_after == -1).all()
+    per_worker = np.bincount(cl.worker, minlength=n).astype(np.float64)
+    mean = [per_worker[cl.klass == c].mean() for c in range(3)]
+    assert 8.5 < mean[0] / mean[1] < 11.5 and 7.0 < mean[1] / mean[2] < 14.0
+    last = {}
+    for u, (w, j) in enumerate(zip(cl.worker.tolist(), cl.pull_ts.tolist())):
+        assert j == (last[w] + 1 if w in last else 0) and j <= u
+        last[w] = u
+    lag = np.arange(N) - cl.pull_ts.astype(np.int64)
+    slow = np.isin(cl.worker, np.where(cl.klass == 2)[0])
+    assert lag[slow].mean() > 20 * lag[~slow].mean()            # slow workers' updates are far staler
+    again = wlmod.closed_loop_schedule(n, N, seed=3, class_fractions=(0.3, 0.4, 0.3), class_rates=(100, 10, 1))
+    assert np.array_equal(cl.worker, again.worker) and np.array_equal(cl.pull_ts, again.pull_ts)
+    other = wlmod.closed_loop_schedule(n, N, seed=4, class_fractions=(0.3, 0.4, 0.3), class_rates=(100, 10, 1))
+    assert not np.array_equal(cl.worker, other.worker)
+
+
+def test_closed_loop_fail_stop_crashes():
+    """After each push a worker stops for good with probability p: it never pushes again, and the number
+    of pushes a worker manages is geometric with mean 1 / p."""
+    n, p = 400, 0.02
+    cl = wlmod.closed_loop_schedule(n, 10**6, seed=5, crash_probability=p)
+    assert (cl.crashed_after >= 1).all() and cl.worker.size == int(cl.crashed_after.sum())   # everybody stops in the end
+    per_worker = np.bincount(cl.worker, minlength=n)
+    assert np.array_equal(per_worker, cl.crashed_after)
+    assert abs(per_worker.mean() * p - 1.0) < 0.15                                          # mean of a geometric law
+    assert abs((per_worker > 35).mean() - (1 - p) ** 35) < 0.08                             # its tail
+    few = wlmod.closed_loop_schedule(200, 5000, seed=6, crash_probability=0.004)
+    gone = few.crashed_after >= 0
+    assert 5 <= gone.sum() <= 40                                                             # about 5000 * 0.004 = 20
+    for w in np.where(gone)[0]:
+        assert (few.worker == w).sum() == few.crashed_after[w]
+    with pytest.raises(ValueError):
+        wlmod.closed_loop_schedule(10, 10, class_fractions=(0.5, 0.4), class_rates=(1, 2))
