@@ -117,6 +117,22 @@ def run_competitors(binding, wl, grads, dev, peak, keep=(1, 100), reps=5, warmup
                       "apply_ms_per_round": round(app_ms, 4), "apply_pairs_per_s": round(W * K / app_ms * 1e3, 1),
                       "ingress_bytes_per_update": 8 * K}
     assert sel.last_error()[0] == 0 and srv.last_error() == 0
+    # the two history structures on the same updates: chains (automatic mode) against the paper's sorted
+    # lists with one search per update of the window; "fresh" = all pulled at the start of the round
+    # (windows of 0 .. W - 1 updates), "stale" = every update pulled 2 W updates before it is applied
+    hist = {}
+    for name, mode in (("chains", 0), ("sorted_lists", 4)):
+        srv = binding.Server(theta, history_pairs=4 * W * K, max_window_updates=4 * W)
+        srv.set_mode(mode)
+        fresh = lambda: srv.apply(idx.view(-1), val.view(-1), begin(K), count, np.full(W, srv.timestamp, np.uint64), wl.lr)
+        stale = lambda: srv.apply(idx.view(-1), val.view(-1), begin(K), count,
+                                  srv.timestamp + np.arange(W, dtype=np.uint64) - np.uint64(2 * W), wl.lr)
+        f_ms = timed(fresh)
+        s_ms = timed(stale)
+        hist[name] = {"fresh_apply_ms_per_round": round(f_ms, 4), "stale_apply_ms_per_round": round(s_ms, 4)}
+        assert srv.last_error() == 0
+        del srv
+    out["history_structures"] = hist
     return out
 
 

@@ -274,6 +274,12 @@ ADACOMP_API int adacomp_server_set_validation(adacomp_server_t* s, int on);
  *     the updates per parameter;
  * 3 = the same over a dense sweep: Theta and the history heads of every 1024-parameter range
  *     are read and written back whole (needs Theta on a 16-byte boundary, else 2 is used).
+ * 4 = the paper's own history structure ("Complexity" paragraph) instead of the chains: the ring
+ *     keeps the sorted index lists of the recent updates and sigma_k is found with one dichotomous
+ *     search per update of the window; one launch per update.  Windows are bounded to 448 updates
+ *     (ADACOMP_ERR_WINDOW beyond).  Same results; O((i - j) log K) probes per pair.  Because the
+ *     ring then holds another kind of history, mode 4 can only be entered or left while the
+ *     timestamp is 0 (ADACOMP_ERR_INVALID otherwise).
  * Updates whose pair slices overlap in memory, with d_sigma_out given, always go as 1: their
  * staleness slots are shared and the later update's count must be the one that stays. */
 ADACOMP_API int adacomp_server_set_mode(adacomp_server_t* s, int mode);

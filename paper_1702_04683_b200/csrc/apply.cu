@@ -662,6 +662,60 @@ k_apply_dense(float* __restrict__ theta, const float* __restrict__ delta, uint64
     for (uint64_t k = vec * 4 + t0; k < n; k += stride) theta[k] = __fsub_rn(theta[k], __fmul_rn(alpha_u, delta[k]));
 }
 
+// ---------------------------------------------------------------------------------------------
+// The paper's own history structure ("Complexity" paragraph): the server keeps the sorted index
+// lists of the last d updates and finds sigma_k of Eq. 3 with one dichotomous search per list of
+// the window.  Here the ring that otherwise holds the chains holds copies of the lists (positions
+// are the same: update u owns ring slots start(u) .. start(u) + pairs(u) - 1), one byte per slot
+// says whether the entry was a change (non-zero), and the window's lists come as a table in the
+// kernel's arguments, which bounds d to kListWindow.  One launch per update, one thread per pair:
+// O((i - j) log K) probes per pair, against O(1 + sigma_k) for the chains.
+constexpr uint32_t kListWindow = 448;          // most updates a window may span with this structure
+
+struct ListWindow {
+    uint32_t slot[kListWindow];                // ring slot of the first pair of update j + t
+    uint32_t count[kListWindow];               // its number of pairs
+    uint32_t n;                                // i - j
+};
+
+__global__ void __launch_bounds__(kApplyThreads)
+k_apply_lists(ServerParams sp, UpdateDesc u, ListWindow win, uint8_t* __restrict__ changed,
+              const uint32_t* __restrict__ idx, const float* __restrict__ val, float lr, uint32_t* sigma_out) {
+    const uint32_t e = blockIdx.x * kApplyThreads + threadIdx.x;
+    if (e >= u.n_pairs) return;
+    const uint64_t at = u.pair_begin + e;
+    const uint32_t k = idx[at];
+    const float v = val[at];
+    const uint32_t own = (u.pos_start + e) & sp.ring_mask;      // this pair's slot (pos_start: slot of the first pair)
+    if (k >= sp.n_params) {                                     // skipped and reported; its slot must not match anything
+        record_error(sp.status, ADACOMP_ERR_UNSORTED);
+        sp.prev[own] = kNone;
+        changed[own] = 0;
+        return;
+    }
+    if (sp.validate && e > 0 && idx[at - 1] >= k) record_error(sp.status, ADACOMP_ERR_UNSORTED);
+    uint32_t sigma = 0;
+    for (uint32_t t = 0; t < win.n; ++t) {                      // Eq. 3: one search per update of the window
+        uint32_t lo = 0, hi = win.count[t];
+        const uint32_t first = win.slot[t];
+        while (lo < hi) {
+            const uint32_t mid = lo + ((hi - lo) >> 1);
+            if (sp.prev[(first + mid) & sp.ring_mask] < k) lo = mid + 1; else hi = mid;
+        }
+        if (lo < win.count[t]) {
+            const uint32_t slot = (first + lo) & sp.ring_mask;
+            sigma += (sp.prev[slot] == k && changed[slot]) ? 1u : 0u;
+        }
+    }
+    if (sigma_out) sigma_out[at] = sigma;
+    sp.prev[own] = k;
+    changed[own] = v != 0.0f ? 1 : 0;                           // Eq. 3 counts changes: a zero entry is not one
+    if (v != 0.0f) {
+        const float alpha_k = sigma ? __fdiv_rn(lr, static_cast<float>(sigma)) : lr;    // Eq. 5
+        sp.theta[k] = __fsub_rn(sp.theta[k], __fmul_rn(alpha_k, v));                     // Eq. 4
+    }
+}
+
 // Moves every stored position down by `delta` (entries older than that become kNone).
 __global__ void k_rebase(uint32_t* a, uint64_t n, uint32_t delta) {
     for (uint64_t i = blockIdx.x * static_cast<uint64_t>(blockDim.x) + threadIdx.x; i < n;
@@ -689,6 +743,7 @@ struct adacomp_server {
     float* d_theta = nullptr;     // borrowed
     uint32_t* d_head = nullptr;
     uint32_t* d_prev = nullptr;
+    uint8_t* d_changed = nullptr; // one byte per ring slot, used by the list structure only
     int* d_status = nullptr;
     // host-side bookkeeping
     uint64_t timestamp = 0;       // i
@@ -706,6 +761,7 @@ size_t carve_server(adacomp_server_t* s, void* base, uint64_t n_params, uint64_t
     Carver c(base);
     s->d_head = c.take<uint32_t>(n_params);
     s->d_prev = c.take<uint32_t>(ring);
+    s->d_changed = c.take<uint8_t>(ring);
     s->d_status = c.take<int>(1);
     return c.used;
 }
@@ -853,6 +909,48 @@ int adacomp_apply(adacomp_server_t* s, const uint32_t* d_idx, const float* d_val
     DeviceGuard guard(s->device);
     if (guard.err != cudaSuccess) return cuda_fail(guard.err);
     cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+
+    if (s->mode == 4) {
+        // ---- the paper's list structure: windows are bounded, positions are only ring slots (no re-basing)
+        for (uint32_t b = 0; b < n_updates; ++b)
+            if (i0 + b - h_pull_ts[b] > kListWindow) return ADACOMP_ERR_WINDOW;
+        ServerParams sp;
+        sp.theta = s->d_theta;
+        sp.head = s->d_head;
+        sp.prev = s->d_prev;
+        sp.status = s->d_status;
+        sp.n_params = s->n_params;
+        sp.ring_mask = static_cast<uint32_t>(s->ring - 1);
+        sp.ring_shift = 0;
+        sp.max_window = s->max_window;
+        sp.validate = s->validate;
+        const uint64_t mask = s->ring - 1;
+        for (uint32_t b = 0; b < n_updates; ++b) {
+            const uint64_t i = i0 + b, j = h_pull_ts[b];
+            ListWindow win;
+            win.n = static_cast<uint32_t>(i - j);
+            for (uint64_t t = j; t < i; ++t) {                  // start and size of update t, from this call or before
+                const uint64_t st_t = t >= i0 ? start_abs[t - i0] : s->start_of[t % cap];
+                const uint64_t en_t = t + 1 >= i0 ? start_abs[t + 1 - i0] : s->start_of[(t + 1) % cap];
+                win.slot[t - j] = static_cast<uint32_t>(st_t & mask);
+                win.count[t - j] = static_cast<uint32_t>(en_t - st_t);
+            }
+            UpdateDesc u;
+            u.pair_begin = h_pair_begin[b];
+            u.n_pairs = h_pair_count[b];
+            u.pos_start = static_cast<uint32_t>(start_abs[b] & mask);
+            u.win_start = u.pad = 0;
+            if (u.n_pairs) {
+                const unsigned grid = (u.n_pairs + kApplyThreads - 1) / kApplyThreads;
+                k_apply_lists<<<grid, kApplyThreads, 0, st>>>(sp, u, win, s->d_changed, d_idx, d_val, lr, d_sigma_out);
+                ADACOMP_LAUNCH_CHECK();
+            }
+        }
+        for (uint32_t b = 0; b < n_updates; ++b) s->start_of[(i0 + b) % cap] = start_abs[b];
+        s->pos_next = start_abs[n_updates];
+        s->timestamp = i0 + n_updates;
+        return ADACOMP_OK;
+    }
 
     // ---- keep 32-bit positions in range
     if (s->pos_next + call_pairs - s->pos_base >= kRebaseAt) {
@@ -1022,7 +1120,9 @@ int adacomp_server_set_validation(adacomp_server_t* s, int on) {
 }
 
 int adacomp_server_set_mode(adacomp_server_t* s, int mode) {
-    if (!s || mode < 0 || mode > 3) return ADACOMP_ERR_INVALID;
+    if (!s || mode < 0 || mode > 4) return ADACOMP_ERR_INVALID;
+    // the list structure keeps another history in the same ring: no switching once updates were applied
+    if ((mode == 4) != (s->mode == 4) && s->timestamp != 0) return ADACOMP_ERR_INVALID;
     s->mode = mode;
     return ADACOMP_OK;
 }
