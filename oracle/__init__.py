@@ -68,6 +68,10 @@ def lib():
             L.oracle_global_apply_dense.argtypes = [ctypes.c_void_p, f32p, ctypes.c_uint64, ctypes.c_float]
             L.oracle_gather.restype = ctypes.c_int
             L.oracle_gather.argtypes = [f32p, ctypes.c_uint64, u32p, ctypes.c_uint64, f32p]
+            L.oracle_encode_indices.restype = ctypes.c_uint64
+            L.oracle_encode_indices.argtypes = [u32p, ctypes.c_uint64, u32p, u64p]
+            L.oracle_decode_indices.restype = ctypes.c_int
+            L.oracle_decode_indices.argtypes = [u32p, u64p, ctypes.c_uint64, u32p]
             L.oracle_parameter_trace.restype = ctypes.c_int
             L.oracle_parameter_trace.argtypes = [
                 ctypes.c_uint32, ctypes.c_float, u32p, f32p, u64p, u64p, ctypes.c_uint64, ctypes.c_uint64,
@@ -178,6 +182,25 @@ def gather(g, idx):
     out = np.empty(idx.size, dtype=np.float32)
     if lib().oracle_gather(_p(g, ctypes.c_float), g.size, _p(idx, ctypes.c_uint32), idx.size, _p(out, ctypes.c_float)) != 0:
         raise ValueError("oracle gather: index out of range")
+    return out
+
+
+def encode_indices(idx):
+    """Block-wise gap coding of an ascending index list -> (words uint32, block_off uint64[n_blocks + 1])."""
+    idx = np.ascontiguousarray(idx, dtype=np.uint32)
+    n_blocks = (idx.size + 255) // 256
+    words = np.empty(idx.size + 2 * n_blocks, dtype=np.uint32)          # the most the format can take
+    off = np.empty(n_blocks + 1, dtype=np.uint64)
+    total = lib().oracle_encode_indices(_p(idx, ctypes.c_uint32), idx.size, _p(words, ctypes.c_uint32), _p(off, ctypes.c_uint64))
+    return words[:int(total)].copy(), off
+
+
+def decode_indices(words, block_off, n_pairs: int):
+    words = np.ascontiguousarray(words, dtype=np.uint32)
+    block_off = np.ascontiguousarray(block_off, dtype=np.uint64)
+    out = np.empty(n_pairs, dtype=np.uint32)
+    if lib().oracle_decode_indices(_p(words, ctypes.c_uint32), _p(block_off, ctypes.c_uint64), n_pairs, _p(out, ctypes.c_uint32)) != 0:
+        raise ValueError("oracle decode: bad stream")
     return out
 
 

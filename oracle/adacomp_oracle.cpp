@@ -305,6 +305,69 @@ int oracle_gather(const float* g, uint64_t n, const uint32_t* idx, uint64_t n_pa
     return 0;
 }
 
+// --- index coding -------------------------------------------------------------------
+// The paper leaves the encoding of the (index, value) pairs open (footnote of
+// "Algorithm details").  This is the format the library offers for the index half,
+// stated entry by entry; values travel as they are.  An update's ascending index
+// list is cut into blocks of 256 entries.  A block is stored as
+//   word 0      the first index of the block,
+//   word 1      w = the number of bits of the largest gap in the block, where the gap
+//               of an entry is (index - previous index - 1), modulo 2^32,
+//   then        the gaps of entries 1 .. n-1 of the block, w bits each, entry e at bit
+//               (e - 1) * w of a little-endian bit string held in 32-bit words
+//               (ceil((n - 1) * w / 32) words; none if w = 0).
+// block_off[b] is the word at which block b starts; block_off[n_blocks] the total.
+static inline uint32_t bits_needed(uint32_t x) {
+    uint32_t n = 0;
+    while (x) { ++n; x >>= 1; }
+    return n;
+}
+
+uint64_t oracle_encode_indices(const uint32_t* idx, uint64_t n_pairs, uint32_t* words_out, uint64_t* block_off_out) {
+    uint64_t at = 0, n_blocks = (n_pairs + 255) / 256;
+    for (uint64_t b = 0; b < n_blocks; ++b) {
+        const uint64_t first = b * 256, n = std::min<uint64_t>(256, n_pairs - first);
+        block_off_out[b] = at;
+        uint32_t widest = 0;
+        for (uint64_t e = 1; e < n; ++e) widest = std::max(widest, bits_needed(idx[first + e] - idx[first + e - 1] - 1u));
+        words_out[at++] = idx[first];
+        words_out[at++] = widest;
+        const uint64_t payload = ((n - 1) * widest + 31) / 32;
+        for (uint64_t i = 0; i < payload; ++i) words_out[at + i] = 0;
+        for (uint64_t e = 1; e < n; ++e) {
+            const uint64_t gap = idx[first + e] - idx[first + e - 1] - 1u;      // 32 bits, zero-extended
+            for (uint32_t bit = 0; bit < widest; ++bit) {                        // bit by bit, as the format is defined
+                const uint64_t pos = (e - 1) * widest + bit;
+                if ((gap >> bit) & 1u) words_out[at + pos / 32] |= 1u << (pos % 32);
+            }
+        }
+        at += payload;
+    }
+    block_off_out[n_blocks] = at;
+    return at;
+}
+
+int oracle_decode_indices(const uint32_t* words, const uint64_t* block_off, uint64_t n_pairs, uint32_t* idx_out) {
+    const uint64_t n_blocks = (n_pairs + 255) / 256;
+    for (uint64_t b = 0; b < n_blocks; ++b) {
+        const uint64_t first = b * 256, n = std::min<uint64_t>(256, n_pairs - first), at = block_off[b];
+        const uint32_t widest = words[at + 1];
+        if (widest > 32) return -1;
+        uint32_t k = words[at];
+        idx_out[first] = k;
+        for (uint64_t e = 1; e < n; ++e) {
+            uint32_t gap = 0;
+            for (uint32_t bit = 0; bit < widest; ++bit) {
+                const uint64_t pos = (e - 1) * widest + bit;
+                gap |= ((words[at + 2 + pos / 32] >> (pos % 32)) & 1u) << bit;
+            }
+            k = k + gap + 1u;
+            idx_out[first + e] = k;
+        }
+    }
+    return 0;
+}
+
 // --- one parameter at a time --------------------------------------------------
 // The history of a single parameter k through a whole sequence of updates,
 // computed the way the paper's complexity paragraph describes it: each update
