@@ -136,6 +136,42 @@ def run_competitors(binding, wl, grads, dev, peak, keep=(1, 100), reps=5, warmup
     return out
 
 
+def run_encoding(binding, points, W, peak, reps=5, warmup=3):
+    """The index coding on what the last step selected, per keep fraction: bytes per pair on the wire
+    (coded index + 4-byte value, against 8 plain) and the time to code and decode W updates."""
+    stream = torch.cuda.current_stream()
+    out = []
+    for p in points:
+        words, off = binding.adacomp_encode_indices(p.idx)
+        cap = words.shape[1]
+
+        def timed(fn):
+            for _ in range(warmup):
+                fn()
+            a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            a.record(stream)
+            for _ in range(reps):
+                fn()
+            b.record(stream)
+            torch.cuda.synchronize()
+            return a.elapsed_time(b) / reps
+        raw = binding.raw()
+        dev_index = p.idx.device.index or 0
+        back = torch.empty_like(p.idx)
+        enc_ms = timed(lambda: binding._check(raw.adacomp_encode_indices(p.idx.data_ptr(), p.K, W, words.data_ptr(), cap, off.data_ptr(),
+                                                                         dev_index, int(stream.cuda_stream)), "encode"))
+        dec_ms = timed(lambda: binding._check(raw.adacomp_decode_indices(words.data_ptr(), cap, off.data_ptr(), p.K, W, back.data_ptr(),
+                                                                         dev_index, int(stream.cuda_stream)), "decode"))
+        if not torch.equal(back, p.idx):
+            raise SystemExit("index coding: the round trip changed an index")
+        coded_words = float(off[:, -1].sum().item())
+        out.append({"keep": f"{p.keep[0]}/{p.keep[1]}", "bytes_per_pair": round(4.0 + 4.0 * coded_words / (W * p.K), 3),
+                    "plain_bytes_per_pair": 8.0, "encode_ms": round(enc_ms, 4), "decode_ms": round(dec_ms, 4),
+                    "encode_pairs_per_s": round(W * p.K / enc_ms * 1e3, 1), "decode_pairs_per_s": round(W * p.K / dec_ms * 1e3, 1)})
+        del words, off, back
+    return out
+
+
 def parse_args():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -393,6 +429,8 @@ def run_native(args):
                                      "achieved": round(sel_bytes_all / sel_ms_all / 1e6, 1),
                                      "frac": round(sel_bytes_all / sel_ms_all / 1e6 / peak, 4)}},
     }
+    if world == 1 and not args.no_competitors:
+        out["encoding"] = run_encoding(binding, points, W, peak)
     if world == 1 and not args.no_competitors and args.keep is None:
         out["competitors"] = run_competitors(binding, wl, grads, dev, peak)
     if world == 1 and not args.no_e2e:

@@ -306,6 +306,26 @@ ADACOMP_API int adacomp_server_debug_skip_positions(adacomp_server_t* s, uint64_
 ADACOMP_API int adacomp_server_last_error(adacomp_server_t* s, void* cuda_stream);
 ADACOMP_API int adacomp_server_destroy(adacomp_server_t* s);
 
+/* ---- index coding -------------------------------------------------------------------------
+ * The paper leaves the encoding of the pairs open (footnote of "Algorithm details"); this is a
+ * lossless coding of the index half (values travel as they are).  A worker's index list of
+ * pairs_per_worker entries, ascending as adacomp_select emits it, is cut into blocks of 256
+ * entries; a block is stored as: the first index; w = the number of bits of the largest gap in
+ * the block (gap of an entry = index - previous index - 1, modulo 2^32, so any list survives the
+ * round trip); the gaps of the block's other entries, w bits each, entry e at bit (e - 1) * w
+ * of a little-endian bit string held in 32-bit words.  d_block_off[w][b] (n_blocks + 1 entries
+ * per worker, n_blocks = ceil(pairs_per_worker / 256)) is the word at which block b starts in
+ * worker w's stream d_words + w * words_per_worker; the last entry is the stream's length.
+ * words_per_worker must be at least adacomp_encode_capacity_words(pairs_per_worker)
+ * (ADACOMP_ERR_CAPACITY otherwise).  All arrays are the caller's device memory. */
+ADACOMP_API uint64_t adacomp_encode_capacity_words(uint64_t pairs_per_worker);
+ADACOMP_API int adacomp_encode_indices(const uint32_t* d_idx, uint64_t pairs_per_worker, uint32_t n_workers,
+                                       uint32_t* d_words, uint64_t words_per_worker, uint64_t* d_block_off,
+                                       int device, void* cuda_stream);
+ADACOMP_API int adacomp_decode_indices(const uint32_t* d_words, uint64_t words_per_worker,
+                                       const uint64_t* d_block_off, uint64_t pairs_per_worker,
+                                       uint32_t n_workers, uint32_t* d_idx_out, int device, void* cuda_stream);
+
 #ifdef __cplusplus
 }
 #endif

@@ -72,6 +72,9 @@ def _load():
         "adacomp_server_timestamp": (i32, [vp, P(u64)]),
         "adacomp_server_set_validation": (i32, [vp, i32]),
         "adacomp_server_set_mode": (i32, [vp, i32]),
+        "adacomp_encode_capacity_words": (u64, [u64]),
+        "adacomp_encode_indices": (i32, [vp, u64, u32, vp, u64, vp, i32, vp]),
+        "adacomp_decode_indices": (i32, [vp, u64, vp, u64, u32, vp, i32, vp]),
         "adacomp_server_set_rule": (i32, [vp, i32]),
         "adacomp_apply_dense": (i32, [vp, vp, u64, f32, vp]),
         "adacomp_select_gather": (i32, [vp, vp, u64, u32, vp, vp, vp]),
@@ -167,6 +170,34 @@ def adacomp_select_static(grad: torch.Tensor, k: int, idx_out: torch.Tensor, val
 
 
 # ----------------------------------------------------------------------------- worker side
+
+def adacomp_encode_capacity_words(pairs_per_worker: int) -> int:
+    return int(_lib.adacomp_encode_capacity_words(int(pairs_per_worker)))
+
+
+def adacomp_encode_indices(idx: torch.Tensor, stream: Optional[torch.cuda.Stream] = None):
+    """idx [W, K] (int32 holding uint32 bit patterns) -> (words [W, capacity] int32, block_off [W, n_blocks + 1]
+    int64): the block-wise gap coding of every worker's index list."""
+    if idx.dim() == 1:
+        idx = idx.unsqueeze(0)
+    W, K = idx.shape
+    cap = adacomp_encode_capacity_words(K)
+    words = torch.empty((W, max(cap, 1)), dtype=torch.int32, device=idx.device)
+    off = torch.empty((W, (K + 255) // 256 + 1), dtype=torch.int64, device=idx.device)
+    _check(_lib.adacomp_encode_indices(_dev(idx, torch.int32, "idx") if K else None, K, W, words.data_ptr(), words.shape[1],
+                                       off.data_ptr(), idx.device.index or 0, _stream_ptr(stream)), "adacomp_encode_indices")
+    return words, off
+
+
+def adacomp_decode_indices(words: torch.Tensor, block_off: torch.Tensor, pairs_per_worker: int,
+                           stream: Optional[torch.cuda.Stream] = None) -> torch.Tensor:
+    W = words.shape[0]
+    out = torch.empty((W, pairs_per_worker), dtype=torch.int32, device=words.device)
+    _check(_lib.adacomp_decode_indices(_dev(words, torch.int32, "words"), words.shape[1], _dev(block_off, torch.int64, "block_off"),
+                                       int(pairs_per_worker), W, out.data_ptr(), words.device.index or 0, _stream_ptr(stream)),
+           "adacomp_decode_indices")
+    return out
+
 
 class Selector:
     """SELECT_GRAD (Algorithm 1) for a fixed tensor layout; owns its device workspace."""
