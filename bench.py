@@ -99,7 +99,7 @@ def run_competitors(binding, wl, grads, dev, peak, keep=(1, 100), reps=5, warmup
     sel_ms = timed(lambda: sel.select(grads, idx, val))
     count = np.full(W, k, np.uint32)
     app_ms = timed(lambda: srv.apply(idx.view(-1), val.view(-1), begin(k), count, np.full(W, srv.timestamp, np.uint64), wl.lr))
-    out["comp_asgd"] = {"select": "one segment over all %d parameters (larger than the single-pass route takes: five reads)" % P,
+    out["comp_asgd"] = {"select": "one segment over all %d parameters" % P,
                         "select_ms_per_round": round(sel_ms, 4), "select_scanned_gbs": round(W * 4.0 * P / sel_ms / 1e6, 1),
                         "apply_ms_per_round": round(app_ms, 4), "apply_pairs_per_s": round(W * k / app_ms * 1e3, 1),
                         "ingress_bytes_per_update": 8 * k}

@@ -127,7 +127,7 @@ ADACOMP_API int adacomp_select_host(adacomp_select_t* h, const float* h_grads, u
                         void* cuda_stream);
 
 /* Chooses how selections are computed; the results are identical.
- * 0 = automatic: tensors of 32768 to 33.5 M entries with k <= n/4 take the bracketed route (a
+ * 0 = automatic: tensors of at least 32768 entries with k <= n/4 take the bracketed route (a
  *     sample brackets the threshold, then the gradient is read once); instances whose bracket
  *     turns out wrong (or that hold a NaN), and all other tensors, take the general route;
  * 1 = general route for everything (multi-pass radix select; reads the gradient five times). */

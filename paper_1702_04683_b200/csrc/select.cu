@@ -71,9 +71,8 @@ void plan_bracket(Layer& L, Layout* out) {
     L.bracket = 0;
     L.sample = L.n_spans = L.span_base = L.cand_cap = L.win_cap = 0;
     L.cand_base = L.win_base = 0;
-    if (L.n < kBracketMinN || L.k == 0 || static_cast<uint64_t>(L.k) * 4 > L.n) return;
+    if (L.n < kBracketMinN || L.n > kBracketMaxN || L.k == 0 || static_cast<uint64_t>(L.k) * 4 > L.n) return;
     const uint32_t n_spans = static_cast<uint32_t>((static_cast<uint64_t>(L.n) + 3 + kSpanElems - 1) / kSpanElems);
-    if (n_spans > kMaxSpans) return;
     uint32_t m = L.n / 8;
     if (m > kSampleMax) m = kSampleMax;
     if (m < kSampleMin) m = kSampleMin;

@@ -33,7 +33,8 @@ constexpr uint32_t kSubElems = 1024;                  // entries one warp classi
 constexpr uint32_t kSubsPerSpan = 8;
 constexpr uint32_t kSpanElems = kSubElems * kSubsPerSpan;   // 8192: unit of the output-offset prefix
 constexpr uint32_t kSpansPerBlock = 8;                // scan: consecutive spans per block; emit: one per warp
-constexpr uint32_t kMaxSpans = 4096;                  // per tensor on this route (n <= 33.5 M)
+constexpr uint32_t kMaxSpans = 4096;                  // spans whose counters the resolve kernel keeps in shared memory
+constexpr uint32_t kBracketMaxN = 0xFFFF0000u;        // shifted 32-bit coordinates must not wrap
 constexpr uint32_t kBracketMinN = 32768;
 constexpr uint32_t kSampleMax = 16384;
 constexpr uint32_t kSampleMin = 2048;
@@ -213,7 +214,7 @@ __global__ void __launch_bounds__(kThreads, 4) k_bracket_scan(SelectParams p, ui
     const float* first = p.grads + static_cast<uint64_t>(w) * p.stride + L.offset;
     const uint32_t mis = static_cast<uint32_t>((reinterpret_cast<uintptr_t>(first) >> 2) & 3u);
     const float4* vec = reinterpret_cast<const float4*>(first - mis);
-    const uint32_t n_shift = L.n + mis;                        // n <= 33.5 M on this route
+    const uint32_t n_shift = L.n + mis;                        // n <= kBracketMaxN on this route
     const uint32_t nvec = (n_shift + 3) >> 2;
     const uint32_t lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     const uint32_t lt = (1u << lane) - 1u;
@@ -449,7 +450,7 @@ __global__ void __launch_bounds__(kThreads, 4) k_bracket_scan_dense(SelectParams
     const float* first = p.grads + static_cast<uint64_t>(w) * p.stride + L.offset;
     const uint32_t mis = static_cast<uint32_t>((reinterpret_cast<uintptr_t>(first) >> 2) & 3u);
     const float4* vec = reinterpret_cast<const float4*>(first - mis);
-    const uint32_t n_shift = L.n + mis;                        // n <= 33.5 M on this route
+    const uint32_t n_shift = L.n + mis;                        // n <= kBracketMaxN on this route
     const uint32_t nvec = (n_shift + 3) >> 2;
     const uint32_t lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     const uint32_t lt = (1u << lane) - 1u;
@@ -715,13 +716,15 @@ __global__ void __launch_bounds__(kBig) k_bracket_resolve(SelectParams p) {
             hi_shift = new_shift;
         }
     }
-    // kept window entries per span
-    for (uint32_t s = threadIdx.x; s < L.n_spans; s += kBig) s_sel[s] = 0;
+    // kept window entries per span: counted in shared memory, or for very long tensors in the table
+    // that receives the spans' output offsets anyway
+    uint32_t* sel = L.n_spans <= kMaxSpans ? s_sel : span_off;
+    for (uint32_t s = threadIdx.x; s < L.n_spans; s += kBig) sel[s] = 0;
     if (threadIdx.x == 0) s_carry = 0;
     __syncthreads();
     if (need > 0) {
         for_each_window([&](unsigned long long c, uint32_t idx) {
-            if (c >= cstar) atomicAdd(&s_sel[idx / kSpanElems], 1u);
+            if (c >= cstar) atomicAdd(&sel[idx / kSpanElems], 1u);
         });
     }
     __syncthreads();
@@ -730,7 +733,7 @@ __global__ void __launch_bounds__(kBig) k_bracket_resolve(SelectParams p) {
         const uint32_t s = base + threadIdx.x;
         uint32_t kept = 0;
         if (s < L.n_spans) {
-            kept = s_sel[s];
+            kept = sel == s_sel ? s_sel[s] : __ldcg(&sel[s]);
 #pragma unroll
             for (uint32_t j = 0; j < kSubsPerSpan; ++j) kept += __ldcg(&sub_tab[s * kSubsPerSpan + j]).y >> 16;
         }

@@ -182,6 +182,24 @@ def test_bracket_route_sizes(binding, n, k):
         assert np.array_equal(u32(idx[w]), oi) and np.array_equal(bits(val[w]), bits(ov))
 
 
+def test_one_segment_over_a_hundred_million_entries(binding):
+    """A tensor far longer than the resolve kernel's shared-memory span table (whole-model selection, an
+    embedding table): still the single-pass route, still exact."""
+    dev = torch.device("cuda", 0)
+    n, k = 100_000_003, 1_000_001
+    g = torch.randn(2, n + 3, device=dev)[:, 1:n + 1]
+    g[1] *= torch.rand(n, device=dev)
+    sel = binding.Selector(binding.segments_from([0], [n], [k]), 2, dev)
+    idx, val = sel.select(g)
+    assert sel.last_error() == (0, 0)                                  # nobody fell back to the general route
+    idx64 = idx.to(torch.int64) & 0xFFFFFFFF
+    assert bool((idx64[:, 1:] > idx64[:, :-1]).all()) and int(idx64.max()) < n
+    assert torch.equal(torch.gather(g, 1, idx64).view(torch.int32), val.view(torch.int32))
+    for w in range(2):
+        oi, ov = oracle.select(g[w].cpu().numpy(), k)
+        assert np.array_equal(u32(idx[w]), oi) and np.array_equal(bits(val[w]), bits(ov))
+
+
 # ----------------------------------------------------------------------------- the workloads
 
 def test_small_cnn_full_size(binding):
