@@ -38,7 +38,7 @@ FALLBACK_HBM_GBS = 6650.0
 # 1/10 are the dense scan kernel).  A launch over W workers moves W / 4 times as much.  Only valid while
 # the kernel source is the one that was profiled.
 SCAN_TRAFFIC_W4_MB = {"1/1000": 1647.3, "1/400": 1685.3, "1/160": 1798.1, "1/64": 1791.7, "1/25": 1789.3, "1/10": 2007.4}
-SCAN_SOURCE_SHA256_16 = "fafde59f6b7c9c48"
+SCAN_SOURCE_SHA256_16 = "357943fb5ed13c1e"
 
 
 def scan_traffic_bytes(workload_index, keeps, workers):
