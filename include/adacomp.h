@@ -272,8 +272,10 @@ ADACOMP_API int adacomp_server_set_validation(adacomp_server_t* s, int on);
  * 2 = up to 32 updates per launch; a block owns a run of parameter ranges sized to the updates'
  *     density, sees all pairs of a range at once (one thread per pair) and keeps the order of
  *     the updates per parameter;
- * 3 = the same over a dense sweep: Theta and the history heads of every 1024-parameter range
- *     are read and written back whole (needs Theta on a 16-byte boundary, else 2 is used).
+ * 3 = up to 32 updates per launch over a dense sweep: a warp owns a run of ranges of 128 to 512
+ *     parameters (sized to the updates' density), brings Theta and the history heads of a range
+ *     into shared memory whole, applies the updates' pairs of the range one update after the
+ *     other, and writes back what changed (needs Theta on a 16-byte boundary, else 2 is used).
  * 4 = the paper's own history structure ("Complexity" paragraph) instead of the chains: the ring
  *     keeps the sorted index lists of the recent updates and sigma_k is found with one dichotomous
  *     search per update of the window; one launch per update.  Windows are bounded to 448 updates

@@ -373,256 +373,229 @@ k_apply_ranges(ServerParams sp, RangeDesc d, const uint32_t* __restrict__ idx, c
 }
 
 // ---------------------------------------------------------------------------------------------
-// Several updates per launch over a dense sweep of the parameters, for batches that touch a good
-// part of every 32-byte sector of Theta anyway.  A block owns a run of ranges of kSwRange
-// consecutive parameters, thread t the four parameters 4t .. 4t + 3 of the range.  Per range:
-//   sweep    Theta of the range goes into registers and its heads into shared memory with one
-//            16-byte load each per thread;
-//   stage    warp w loads, for updates w, w + 8, ..., the next <= 128 pairs from the update's
-//            cursor (the loads of all updates and of the sweep are in flight together), keeps
-//            them in shared memory and sets, for every non-zero pair, bit b in the mask of its
-//            parameter and its slot in a table under [b][parameter];
-//   pairs    ONE THREAD PER STAGED PAIR below the round's limit: Eq. 3 inside the batch is a
-//            population count of the mask under the update's window bits, the part of a window
-//            before the batch a chain walk from the head the parameter had when the batch began;
-//            Eq. 5; the pair leaves its step alpha_k * value in shared memory and is linked behind
-//            the pair of the next lower bit (or the old head);
-//   sums     every thread subtracts, for its four parameters, the steps in arrival order (Eq. 4
-//            keeps its rounding order) and remembers the new head;
-//   finally Theta and the heads of the range are written back, 16 bytes per thread, where changed.
-// No barrier separates the updates: the order is kept per parameter, which is all Algorithm 2
-// needs.  The limit of a round is the smallest index some update could not stage any more, so
-// every update's pairs below it are on chip; the range is finished in further rounds.  Same
-// results, bit for bit, as one launch per update.
-constexpr uint32_t kSwRange = 1024;
-constexpr int kSwThreads = kSwRange / 4;
+// Several updates per launch, one WARP per range of parameters, no block barrier in the loop.  A
+// warp owns a run of ranges of R consecutive parameters and a slice of shared memory: Theta and
+// the heads of the range (two buffers: the next range's arrive while this one is worked on), a
+// mask per parameter (bit b: update b of the launch changed it) and, per update, a stage with
+// the update's next 32 pairs from its cursor.  All of that is brought in by asynchronous copies
+// issued a range ahead, so that no load is waited for in the common case.
+// Per range the warp takes the updates ONE AFTER THE OTHER in arrival order.  The staged pairs
+// below the range's end are the update's pairs of this range (its index list is ascending), and
+// each lane applies one of them against shared memory exactly as Algorithm 2 states it: Eq. 3
+// inside the launch is a population count of the parameter's mask under the update's window bits,
+// the part of a window before the launch a chain walk from the head the parameter had when the
+// launch began; Eq. 5; Eq. 4; the pair is linked behind the head (one coalesced store to the ring
+// per update) and becomes the head.  The stage of an update that consumed pairs is refilled from
+// its new cursor; updates with no pair in the range are skipped four or eight at a time.  When all
+// 32 staged pairs lay in the range the update may have more there: they are fetched and applied
+// before the next update is looked at (the host sizes R so that this is rare).  At the end of
+// the range Theta and heads go back, 16 bytes per lane, where a parameter changed.  Updates are
+// applied in order per range, which is all Algorithm 2 needs: same results, bit for bit, as one
+// launch per update.  kExtra: staleness counts are written, or the lists are validated.
+constexpr int kWpThreads = 128;
+constexpr uint32_t kWpWarps = kWpThreads / 32;
+constexpr uint32_t kWpGroups = 4;              // groups of asynchronous copies per range
 
-struct SweepDesc {
-    BatchDesc o;
-    uint32_t chunks;                           // 32-pair chunks staged per update and round, 1..kRgChunks
-};
-
-__host__ __device__ inline size_t sw_smem_bytes(uint32_t n_updates) {
-    return kSwRange * 8 + static_cast<size_t>(n_updates) * kRgStage * 6 + sizeof(RgMeta) +
-           static_cast<size_t>(n_updates) * kSwRange;
+__host__ __device__ inline size_t wp_warp_words(uint32_t range, uint32_t n_updates, bool pre) {
+    return 32 + 64 * static_cast<size_t>(n_updates) + (pre ? 6 : 5) * static_cast<size_t>(range);
+}
+__host__ __device__ inline size_t wp_smem_bytes(uint32_t range, uint32_t n_updates, bool pre) {
+    return 64 * 4 + kWpWarps * wp_warp_words(range, n_updates, pre) * 4;
 }
 
-__global__ void __launch_bounds__(kSwThreads)
-k_apply_sweep(ServerParams sp, SweepDesc d, const uint32_t* __restrict__ idx, const float* __restrict__ val,
-              float lr, uint32_t* sigma_out, uint32_t n_ranges) {
-    extern __shared__ __align__(16) unsigned char s_sw[];
-    const uint32_t B = d.o.n_updates;
-    uint32_t* s_mask = reinterpret_cast<uint32_t*>(s_sw);                       // [range] updates that change the parameter
-    uint32_t* s_head = s_mask + kSwRange;                                       // [range] head when the batch began
-    float* s_v = reinterpret_cast<float*>(s_head + kSwRange);                   // [B][kRgStage] value, later the step
-    RgMeta* s_m = reinterpret_cast<RgMeta*>(s_v + B * kRgStage);
-    uint16_t* s_k = reinterpret_cast<uint16_t*>(s_m + 1);                       // [B][kRgStage] index - range start
-    uint8_t* s_tab = reinterpret_cast<uint8_t*>(s_k + B * kRgStage);            // [B][range] slot of (update, parameter)
+__device__ __forceinline__ uint32_t smem_address(const void* p) { return static_cast<uint32_t>(__cvta_generic_to_shared(p)); }
+__device__ __forceinline__ void copy_async_16(uint32_t smem, const void* gmem) {
+    asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(smem), "l"(gmem) : "memory");
+}
+__device__ __forceinline__ void copy_async_4(uint32_t smem, const void* gmem) {
+    asm volatile("cp.async.ca.shared.global [%0], [%1], 4;" ::"r"(smem), "l"(gmem) : "memory");
+}
+__device__ __forceinline__ void prefetch_l2(const void* gmem) { asm volatile("prefetch.global.L2 [%0];" ::"l"(gmem)); }
+__device__ __forceinline__ void copy_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
+template <int kPending>
+__device__ __forceinline__ void copy_async_wait() { asm volatile("cp.async.wait_group %0;" ::"n"(kPending) : "memory"); }
 
+template <uint32_t R, bool kPre, bool kExtra>
+__global__ void __launch_bounds__(kWpThreads)
+k_apply_warps(const ServerParams sp, const BatchDesc d, const uint32_t* __restrict__ idx, const float* __restrict__ val,
+              float lr, uint32_t* sigma_out, uint32_t n_ranges) {
+    extern __shared__ __align__(16) unsigned char s_wp[];
+    static_assert(R % 64 == 0 && R >= 128, "16-byte pieces, whole warps");
+    float* s_alpha = reinterpret_cast<float*>(s_wp);                            // [64] alpha / sigma for the small counts
+    const uint32_t B = d.n_updates;
     const uint32_t tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-    const uint32_t r_lo = static_cast<uint32_t>(static_cast<uint64_t>(n_ranges) * blockIdx.x / gridDim.x);
-    const uint32_t r_hi = static_cast<uint32_t>(static_cast<uint64_t>(n_ranges) * (blockIdx.x + 1) / gridDim.x);
+    uint32_t* s_cur = reinterpret_cast<uint32_t*>(s_wp) + 64 + warp * wp_warp_words(R, B, kPre);   // [32] cursor of every update
+    uint32_t* s_k = s_cur + 32;                                                 // [B][32] staged indices
+    float* s_v = reinterpret_cast<float*>(s_k + 32 * B);                        // [B][32] staged values
+    float* s_theta = s_v + 32 * B;                                              // [2][R] Theta of the range
+    uint32_t* s_head = reinterpret_cast<uint32_t*>(s_theta) + 2 * R;            // [2][R] latest change of the parameter
+    uint32_t* s_mask = s_head + 2 * R;                                          // [R] updates of this launch that changed it
+    uint32_t* s_head0 = s_mask + R;                                             // [R] head when the launch began (kPre)
+
+    if (tid < kRgAlphas) s_alpha[tid] = tid ? __fdiv_rn(lr, static_cast<float>(tid)) : lr;   // Eq. 5 for the small counts, once
+    __syncthreads();                                            // the only block barrier
+    const uint32_t gw = blockIdx.x * kWpWarps + warp, n_gw = gridDim.x * kWpWarps;
+    const uint32_t r_lo = static_cast<uint32_t>(static_cast<uint64_t>(n_ranges) * gw / n_gw);
+    const uint32_t r_hi = static_cast<uint32_t>(static_cast<uint64_t>(n_ranges) * (gw + 1) / n_gw);
     if (r_lo == r_hi) return;
-    if (tid < B) {
-        const uint64_t first_param = static_cast<uint64_t>(r_lo) * kSwRange;
-        const uint64_t begin = d.o.pair_begin[tid];
-        uint32_t lo = 0, hi = d.o.n_pairs[tid];               // cursor: first pair at or above the first owned parameter
+
+    constexpr bool kAhead = R <= 256;                           // dense updates: a stage is often used up within a range
+    const uint32_t a_k = smem_address(s_k + lane), a_v = smem_address(s_v + lane);
+    // the stage of update b takes its next 32 pairs from `cur` (kNone beyond the end of the list)
+    auto refill = [&](uint32_t b, uint32_t cur) {
+        const uint32_t t = cur + lane;
+        if (t < d.n_pairs[b]) {
+            copy_async_4(a_k + b * 128, idx + d.pair_begin[b] + t);
+            copy_async_4(a_v + b * 128, val + d.pair_begin[b] + t);
+            if (kAhead && t + 32 < d.n_pairs[b]) {              // the 32 pairs after these: wanted soon, or at once if all 32 lie in the range
+                prefetch_l2(idx + d.pair_begin[b] + t + 32);
+                prefetch_l2(val + d.pair_begin[b] + t + 32);
+            }
+        } else {
+            s_k[b * 32 + lane] = kNone;
+        }
+    };
+    auto range_end = [&](uint32_t r) -> uint32_t {
+        const uint64_t e = (static_cast<uint64_t>(r) + 1) * R;
+        return e <= sp.n_params ? static_cast<uint32_t>(e) : static_cast<uint32_t>(sp.n_params);
+    };
+    // Theta and heads of range r into buffer p
+    auto sweep_in = [&](uint32_t r, uint32_t p) {
+        const uint32_t lo = r * R, hi = range_end(r);
+        if (hi - lo == R) {
+#pragma unroll
+            for (uint32_t o = lane * 4; o < R; o += 128) {
+                copy_async_16(smem_address(s_theta + p * R + o), sp.theta + lo + o);
+                copy_async_16(smem_address(s_head + p * R + o), sp.head + lo + o);
+            }
+        } else {                                                // the last range may be short: plain loads
+            for (uint32_t o = lane; o < R; o += 32) {
+                s_theta[p * R + o] = lo + o < hi ? sp.theta[lo + o] : 0.f;
+                s_head[p * R + o] = lo + o < hi ? sp.head[lo + o] : kNone;
+            }
+        }
+    };
+
+    if (lane < B) {
+        const uint64_t first_param = static_cast<uint64_t>(r_lo) * R;
+        const uint32_t* list = idx + d.pair_begin[lane];
+        uint32_t lo = 0, hi = d.n_pairs[lane];                 // cursor: first pair at or above the first owned parameter
         while (lo < hi) {
             const uint32_t mid = lo + ((hi - lo) >> 1);
-            if (idx[begin + mid] < first_param) lo = mid + 1; else hi = mid;
+            if (list[mid] < first_param) lo = mid + 1; else hi = mid;
         }
-        s_m->cur[tid] = lo;
-        s_m->adv[tid] = 0;
-        s_m->begin[tid] = begin;
-        s_m->n[tid] = d.o.n_pairs[tid];
-        s_m->win[tid] = d.o.win_start[tid];
-        s_m->bits[tid] = d.o.win_bits[tid];
+        s_cur[lane] = lo;
     }
-    if (tid >= 64 && tid < 64 + kRgAlphas) {                    // Eq. 5 for the small counts, once
-        const uint32_t sigma = tid - 64;
-        s_m->alpha[sigma] = sigma ? __fdiv_rn(lr, static_cast<float>(sigma)) : lr;
-    }
-    auto range_end = [&](uint32_t r) -> uint32_t {
-        const uint64_t e = (static_cast<uint64_t>(r) + 1) * kSwRange;
-        return e < sp.n_params ? static_cast<uint32_t>(e) : static_cast<uint32_t>(sp.n_params);
-    };
-    if (tid == 0) s_m->limit = range_end(r_lo);
-    reinterpret_cast<uint4*>(s_mask)[tid] = make_uint4(0, 0, 0, 0);
-    __syncthreads();
+    __syncwarp();
+    for (uint32_t b = 0; b < B; ++b) refill(b, s_cur[b]);
+    sweep_in(r_lo, 0);
+#pragma unroll
+    for (uint32_t g = 0; g < kWpGroups; ++g) copy_async_commit();   // the first holds everything, the others are empty
 
-    uint32_t r = r_lo, changed = 0;                             // bit j: parameter 4 tid + j of the range got a new head
-    bool fresh = true;                                          // first round of the range
-    float th[4] = {0.f, 0.f, 0.f, 0.f};
-    uint32_t nh[4] = {kNone, kNone, kNone, kNone};
-    while (r < r_hi) {
-        const uint32_t lo = r * kSwRange, hi = range_end(r);
-        const uint32_t mine = lo + 4 * tid;
-        const bool whole = mine + 4 <= hi;                      // all four parameters exist
-        uint4 h4 = make_uint4(kNone, kNone, kNone, kNone);
-        if (fresh) {                                            // ---- sweep
-            changed = 0;
-            if (whole) {
-                h4 = *reinterpret_cast<const uint4*>(sp.head + mine);
-                const float4 t4 = *reinterpret_cast<const float4*>(sp.theta + mine);
-                th[0] = t4.x; th[1] = t4.y; th[2] = t4.z; th[3] = t4.w;
-            } else {
-                uint32_t hh[4] = {kNone, kNone, kNone, kNone};
+    const uint32_t per_group = (B + kWpGroups - 1) / kWpGroups;     // <= 8
+    for (uint32_t r = r_lo; r < r_hi; ++r) {
+        const uint32_t p = (r - r_lo) & 1u;
+        const uint32_t lo = r * R, hi = range_end(r);
+        float* th = s_theta + p * R;
+        uint32_t* hd = s_head + p * R;
+        if (r + 1 < r_hi) sweep_in(r + 1, p ^ 1u);
 #pragma unroll
-                for (uint32_t j = 0; j < 4; ++j)
-                    if (mine + j < hi) { hh[j] = sp.head[mine + j]; th[j] = sp.theta[mine + j]; }
-                h4 = make_uint4(hh[0], hh[1], hh[2], hh[3]);
-            }
-        }
-        // ---- stage
-        #pragma unroll 1
-        for (uint32_t b = warp; b < B; b += kSwThreads / 32) {
-            const uint64_t begin = s_m->begin[b];
-            const uint32_t n_b = s_m->n[b], cur = s_m->cur[b] + s_m->adv[b];     // past what the last round consumed
+        for (uint32_t o = lane * 4; o < R; o += 128) *reinterpret_cast<uint4*>(s_mask + o) = make_uint4(0, 0, 0, 0);
+        // ---- the updates in arrival order
+#pragma unroll 1
+        for (uint32_t g = 0; g < kWpGroups; ++g) {
+            copy_async_wait<kWpGroups - 1>();                   // what was issued a range ago for this group has landed
             __syncwarp();
-            if (lane == 0) {
-                s_m->cur[b] = cur;
-                s_m->pos[b] = d.o.pos_start[b] + cur;         // position of the pair in slot 0
-            }
-            const uint32_t* ip = idx + begin + cur;
-            const float* vp = val + begin + cur;
-            const uint32_t left = n_b - cur;
-            uint32_t kk[kRgChunks];
-            float vv[kRgChunks];
+            if (kPre && g == 0) {
 #pragma unroll
-            for (uint32_t c = 0; c < kRgChunks; ++c) {          // every load first: none waits for another
-                const uint32_t t = c * 32 + lane;
-                kk[c] = kNone;
-                vv[c] = 0.f;
-                if (c < d.chunks && t < left) {
-                    kk[c] = ip[t];
-                    vv[c] = vp[t];
-                }
+                for (uint32_t o = lane * 4; o < R; o += 128)
+                    *reinterpret_cast<uint4*>(s_head0 + o) = *reinterpret_cast<const uint4*>(hd + o);
+                __syncwarp();
             }
-            uint32_t cnt = 0, last_k = 0;
-            bool run = true;                                    // staged = the leading slots below the range's end
-#pragma unroll
-            for (uint32_t c = 0; c < kRgChunks; ++c) {
-                const uint32_t t = c * 32 + lane, k = kk[c];
-                const bool in = k < hi;
-                if (in) {
-                    if (sp.validate && cur + t > 0 && ip[static_cast<int64_t>(t) - 1] >= k) record_error(sp.status, ADACOMP_ERR_UNSORTED);
-                    const uint32_t kl = k - lo;
-                    s_v[b * kRgStage + t] = vv[c];
-                    if (k >= lo) {
-                        s_k[b * kRgStage + t] = static_cast<uint16_t>(kl);
-                        if (vv[c] != 0.0f) {                    // Eq. 3 counts changes: a zero entry is not one
-                            atomicOr(&s_mask[kl], 1u << b);
-                            s_tab[b * kSwRange + kl] = static_cast<uint8_t>(t);
-                        }
-                    } else {                                    // an index before the range: the list was not ascending
-                        s_k[b * kRgStage + t] = static_cast<uint16_t>(kRgLate);
-                        record_error(sp.status, ADACOMP_ERR_UNSORTED);
+            // which updates of the group have a pair in this range: lane t looks at the first staged index of update g * per_group + t
+            const uint32_t b_first = g * per_group;
+            uint32_t first_k = kNone;
+            if (lane < per_group && b_first + lane < B) first_k = s_k[(b_first + lane) * 32];
+            uint32_t live = __ballot_sync(0xFFFFFFFFu, first_k < hi);
+#pragma unroll 1
+            while (live) {
+                const uint32_t b = b_first + __ffs(live) - 1;
+                live &= live - 1;
+                uint32_t k = s_k[b * 32 + lane];
+                float v = s_v[b * 32 + lane];
+                uint32_t cur = s_cur[b];
+                const uint32_t bits_b = d.win_bits[b], bit_b = 1u << b, pos_l = d.pos_start[b] + lane;
+                uint32_t bal = __ballot_sync(0xFFFFFFFFu, k < hi);
+                for (;;) {
+                    if (kExtra && sp.validate) {
+                        uint32_t before = __shfl_up_sync(0xFFFFFFFFu, k, 1);
+                        if (lane == 0) before = cur > 0 ? idx[d.pair_begin[b] + cur - 1] : 0u;
+                        if (k < hi && cur + lane > 0 && before >= k) record_error(sp.status, ADACOMP_ERR_UNSORTED);
                     }
-                }
-                const uint32_t bal = __ballot_sync(0xFFFFFFFFu, in);
-                if (run) {
-                    if (bal == 0xFFFFFFFFu) cnt += 32; else { cnt += __ffs(~bal) - 1; run = false; }
-                }
-                if (c + 1 == d.chunks) last_k = __shfl_sync(0xFFFFFFFFu, k, 31);
-            }
-            if (lane == 0) {
-                s_m->cnt[b] = cnt;
-                if (cnt == d.chunks * 32) atomicMin(&s_m->limit, last_k + 1);   // more of this update may follow in the range
-            }
-        }
-        if (fresh) reinterpret_cast<uint4*>(s_head)[tid] = h4;
-        __syncthreads();
-        const uint32_t limit = s_m->limit;
-        // ---- pairs: one thread per staged pair below the limit
-        #pragma unroll 1
-        for (uint32_t b = warp; b < B; b += kSwThreads / 32) {
-            const uint32_t cnt = s_m->cnt[b], pos_b = s_m->pos[b], bits_b = s_m->bits[b];
-            const uint32_t below_b = (1u << b) - 1u, ws = s_m->win[b];
-            const bool pre_b = (d.o.pre_mask >> b) & 1u;
-            uint32_t* sig = sigma_out ? sigma_out + s_m->begin[b] + s_m->cur[b] : nullptr;
-            uint32_t adv = 0;
-            #pragma unroll 1
-            for (uint32_t t = lane; t < ((cnt + 31) & ~31u); t += 32) {
-                bool take = false;
-                if (t < cnt) {
-                    const uint32_t kl = s_k[b * kRgStage + t];
-                    take = kl == kRgLate || lo + kl < limit;    // consumed in this round (ascending list: these lead)
-                    if (take && kl != kRgLate) {
-                        const float v = s_v[b * kRgStage + t];
-                        const uint32_t m = s_mask[kl], h0 = s_head[kl];
-                        uint32_t sigma = __popc(m & bits_b);                                           // Eq. 3, inside the batch
-                        if (pre_b) {                                                                   // Eq. 3, before the batch
-                            uint32_t q = h0, hops = 0;
-                            while (q != kNone && q >= ws) {
-                                if (++hops > sp.max_window) { record_error(sp.status, ADACOMP_ERR_WINDOW); break; }
-                                q = sp.prev[(q + sp.ring_shift) & sp.ring_mask];
+                    if (k < hi) {
+                        if (k >= lo) {
+                            const uint32_t kl = k - lo;
+                            const bool change = v != 0.0f;      // Eq. 3 counts changes: a zero entry is not one
+                            const uint32_t m = change ? atomicOr(&s_mask[kl], bit_b) : s_mask[kl];
+                            uint32_t sigma = __popc(m & bits_b);                                       // Eq. 3, inside the launch
+                            if (kPre && (d.pre_mask & bit_b)) {                                        // Eq. 3, before the launch
+                                const uint32_t ws = d.win_start[b];
+                                uint32_t q = s_head0[kl], hops = 0;
+                                while (q != kNone && q >= ws) {
+                                    if (++hops > sp.max_window) { record_error(sp.status, ADACOMP_ERR_WINDOW); break; }
+                                    q = sp.prev[(q + sp.ring_shift) & sp.ring_mask];
+                                }
+                                sigma += hops;
                             }
-                            sigma += hops;
-                        }
-                        if (sig) sig[t] = sigma;
-                        if (v != 0.0f) {
-                            const float alpha_k = sigma < kRgAlphas ? s_m->alpha[sigma] : __fdiv_rn(lr, static_cast<float>(sigma));   // Eq. 5
-                            s_v[b * kRgStage + t] = __fmul_rn(alpha_k, v);
-                            const uint32_t low = m & below_b;
-                            uint32_t before = h0;               // the pair that changed the parameter last
-                            if (low) {
-                                const uint32_t b2 = 31 - __clz(low);
-                                before = s_m->pos[b2] + s_tab[b2 * kSwRange + kl];
+                            if (kExtra && sigma_out) sigma_out[d.pair_begin[b] + cur + lane] = sigma;
+                            if (change) {
+                                const float alpha_k = sigma < kRgAlphas ? s_alpha[sigma] : __fdiv_rn(lr, static_cast<float>(sigma));   // Eq. 5
+                                th[kl] = __fsub_rn(th[kl], __fmul_rn(alpha_k, v));                     // Eq. 4
+                                const uint32_t pos = pos_l + cur;
+                                sp.prev[(pos + sp.ring_shift) & sp.ring_mask] = atomicExch(&hd[kl], pos);
                             }
-                            sp.prev[(pos_b + t + sp.ring_shift) & sp.ring_mask] = before;
+                        } else {                                // an index before the range: the list was not ascending
+                            record_error(sp.status, ADACOMP_ERR_UNSORTED);
                         }
                     }
+                    __syncwarp();                               // the next update sees this one's changes
+                    const uint32_t cnt = __popc(bal);
+                    cur += cnt;
+                    if (cnt < 32) break;
+                    const uint32_t t = cur + lane;              // the update may have more pairs in this range
+                    k = kNone;
+                    if (t < d.n_pairs[b]) {
+                        k = idx[d.pair_begin[b] + t];
+                        v = val[d.pair_begin[b] + t];
+                    }
+                    bal = __ballot_sync(0xFFFFFFFFu, k < hi);
+                    if (bal == 0) break;
                 }
-                adv += __popc(__ballot_sync(0xFFFFFFFFu, take));
+                if (lane == 0) s_cur[b] = cur;
+                refill(b, cur);
             }
-            if (lane == 0) s_m->adv[b] = adv;
+            copy_async_commit();
         }
-        __syncthreads();
-        const bool done = limit >= hi;                          // else: the rest of the range in another round
-        if (tid == 0) s_m->limit = !done ? hi : (r + 1 < r_hi ? range_end(r + 1) : hi);   // for the next round
-        // ---- sums: the steps of each parameter in arrival order
-        {
-            const uint4 m4 = reinterpret_cast<const uint4*>(s_mask)[tid];
-            reinterpret_cast<uint4*>(s_mask)[tid] = make_uint4(0, 0, 0, 0);     // empty for the next round's stage
-            const uint32_t mm[4] = {m4.x, m4.y, m4.z, m4.w};
+        // ---- Theta and heads go back where a parameter changed
+        if (hi - lo == R) {
 #pragma unroll
-            for (uint32_t j = 0; j < 4; ++j) {
-                uint32_t m = mm[j];
-                const uint32_t kl = 4 * tid + j;
-                if (m && lo + kl < limit) {
-                    uint32_t b = 0, t = 0;
-                    do {
-                        b = __ffs(m) - 1;
-                        m &= m - 1;
-                        t = s_tab[b * kSwRange + kl];
-                        th[j] = __fsub_rn(th[j], s_v[b * kRgStage + t]);                               // Eq. 4
-                    } while (m);
-                    nh[j] = s_m->pos[b] + t;
-                    changed |= 1u << j;
+            for (uint32_t o = lane * 4; o < R; o += 128) {
+                const uint4 m4 = *reinterpret_cast<const uint4*>(s_mask + o);
+                if (m4.x | m4.y | m4.z | m4.w) {
+                    *reinterpret_cast<float4*>(sp.theta + lo + o) = *reinterpret_cast<const float4*>(th + o);
+                    *reinterpret_cast<uint4*>(sp.head + lo + o) = *reinterpret_cast<const uint4*>(hd + o);
                 }
             }
+        } else {
+            for (uint32_t o = lane; o < R; o += 32)
+                if (lo + o < hi && s_mask[o]) { sp.theta[lo + o] = th[o]; sp.head[lo + o] = hd[o]; }
         }
-        if (done && changed) {                                  // ---- write back
-            const uint4 o4 = reinterpret_cast<const uint4*>(s_head)[tid];
-            const uint32_t oh[4] = {o4.x, o4.y, o4.z, o4.w};
-            uint32_t wh[4];
-#pragma unroll
-            for (uint32_t j = 0; j < 4; ++j) wh[j] = (changed >> j) & 1u ? nh[j] : oh[j];
-            if (whole) {
-                *reinterpret_cast<uint4*>(sp.head + mine) = make_uint4(wh[0], wh[1], wh[2], wh[3]);
-                *reinterpret_cast<float4*>(sp.theta + mine) = make_float4(th[0], th[1], th[2], th[3]);
-            } else {
-#pragma unroll
-                for (uint32_t j = 0; j < 4; ++j)
-                    if ((changed >> j) & 1u) { sp.head[mine + j] = wh[j]; sp.theta[mine + j] = th[j]; }
-            }
-        }
-        __syncthreads();
-        fresh = done;
-        if (done) ++r;
+        __syncwarp();
     }
+    copy_async_wait<0>();
+    __syncwarp();
     // whoever owns the last range sees what no range claimed: indices >= n_params
-    if (r_hi == n_ranges && tid < B && s_m->cur[tid] + s_m->adv[tid] < s_m->n[tid]) record_error(sp.status, ADACOMP_ERR_UNSORTED);
+    if (r_hi == n_ranges && lane < B && s_cur[lane] < d.n_pairs[lane]) record_error(sp.status, ADACOMP_ERR_UNSORTED);
 }
 
 // ---------------------------------------------------------------------------------------------
@@ -766,6 +739,34 @@ size_t carve_server(adacomp_server_t* s, void* base, uint64_t n_params, uint64_t
     return c.used;
 }
 
+// Launches k_apply_warps<R, kPre, kExtra> over all ranges of R parameters with as many blocks as stay resident.
+template <uint32_t R, bool kPre, bool kExtra>
+int launch_apply_warps_as(const adacomp_server_t* s, const ServerParams& sp, const BatchDesc& d, const uint32_t* d_idx,
+                          const float* d_val, float lr, uint32_t* d_sigma_out, cudaStream_t st) {
+    const size_t smem = wp_smem_bytes(R, d.n_updates, kPre);
+    const uint32_t n_ranges = static_cast<uint32_t>((s->n_params + R - 1) / R);
+    ADACOMP_CUDA(cudaFuncSetAttribute(k_apply_warps<R, kPre, kExtra>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                      static_cast<int>(wp_smem_bytes(R, kMaxBatch, kPre))));
+    int per_sm = 1;
+    ADACOMP_CUDA(cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, k_apply_warps<R, kPre, kExtra>, kWpThreads, smem));
+    unsigned grid = static_cast<unsigned>(s->n_sms) * static_cast<unsigned>(per_sm > 0 ? per_sm : 1);
+    const unsigned most_blocks = (n_ranges + kWpWarps - 1) / kWpWarps;
+    if (grid > most_blocks) grid = most_blocks;
+    k_apply_warps<R, kPre, kExtra><<<grid, kWpThreads, smem, st>>>(sp, d, d_idx, d_val, lr, d_sigma_out, n_ranges);
+    ADACOMP_LAUNCH_CHECK();
+    return ADACOMP_OK;
+}
+
+template <uint32_t R>
+int launch_apply_warps(const adacomp_server_t* s, const ServerParams& sp, const BatchDesc& d, const uint32_t* d_idx,
+                       const float* d_val, float lr, uint32_t* d_sigma_out, cudaStream_t st) {
+    const bool pre = d.pre_mask != 0, extra = d_sigma_out != nullptr || sp.validate != 0;
+    if (pre) return extra ? launch_apply_warps_as<R, true, true>(s, sp, d, d_idx, d_val, lr, d_sigma_out, st)
+                          : launch_apply_warps_as<R, true, false>(s, sp, d, d_idx, d_val, lr, d_sigma_out, st);
+    return extra ? launch_apply_warps_as<R, false, true>(s, sp, d, d_idx, d_val, lr, d_sigma_out, st)
+                 : launch_apply_warps_as<R, false, false>(s, sp, d, d_idx, d_val, lr, d_sigma_out, st);
+}
+
 bool sizes_ok(uint64_t n_params, uint64_t history_pairs) {
     return n_params >= 1 && n_params <= 0xFFFFFFFEull && history_pairs >= 1 && history_pairs < (1ull << 31);
 }
@@ -808,9 +809,6 @@ int adacomp_server_create(adacomp_server_t** out, uint64_t n_params, uint64_t hi
     if (e == cudaSuccess)
         e = cudaFuncSetAttribute(k_apply_ranges, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                  static_cast<int>(rg_smem_bytes(kRgMaxRange, kMaxBatch, false) + 32768));   // + the largest slot table
-    if (e == cudaSuccess)
-        e = cudaFuncSetAttribute(k_apply_sweep, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                 static_cast<int>(sw_smem_bytes(kMaxBatch)));
     if (e == cudaSuccess) e = cudaDeviceSynchronize();
     if (e != cudaSuccess) { delete s; return cuda_fail(e); }
     *out = s;
@@ -978,9 +976,9 @@ int adacomp_apply(adacomp_server_t* s, const uint32_t* d_idx, const float* d_val
     sp.validate = s->validate;
 
     // ---- launches.  One launch per update, or launches of up to kMaxBatch updates each: same results.
-    // Automatic choice per launch: the sweep kernel when the launch's pairs number a fifth of the parameters or
-    // more (nearly every 32-byte sector of Theta is touched anyway), else the ranges kernel; a single update,
-    // and updates whose staleness slots overlap in memory, go one per launch.
+    // Automatic choice per launch: the warp-per-range kernel over a dense sweep of Theta when the launch's pairs
+    // number a fifth of the parameters or more (nearly every 32-byte sector of Theta is touched anyway), else the
+    // ranges kernel; a single update, and updates whose staleness slots overlap in memory, go one per launch.
     bool shared_slots = false;                 // two updates write their counts to the same slots: order matters
     if (d_sigma_out && n_updates > 1 && s->mode != 1) {
         std::vector<std::pair<uint64_t, uint64_t>> slices;
@@ -1019,19 +1017,17 @@ int adacomp_apply(adacomp_server_t* s, const uint32_t* d_idx, const float* d_val
         const bool sweep = theta_aligned &&
                            (s->mode == 3 || (s->mode == 0 && static_cast<double>(pairs) >= 0.2 * static_cast<double>(s->n_params)));
         if (sweep) {
-            SweepDesc sd;
-            sd.o = d;
-            // stage what a uniformly spread update brings per range, plus three standard deviations
-            const double mean = dens * kSwRange;
-            const uint32_t chunks = static_cast<uint32_t>((mean + 3.0 * std::sqrt(mean) + 2.0) / 32.0) + 1;
-            sd.chunks = chunks > kRgChunks ? kRgChunks : chunks;
-            const size_t smem = sw_smem_bytes(d.n_updates);
-            const uint32_t n_ranges = static_cast<uint32_t>((s->n_params + kSwRange - 1) / kSwRange);
-            int per_sm = 1;
-            ADACOMP_CUDA(cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, k_apply_sweep, kSwThreads, smem));
-            unsigned grid = static_cast<unsigned>(s->n_sms) * static_cast<unsigned>(per_sm > 0 ? per_sm : 1);
-            if (grid > n_ranges) grid = n_ranges;
-            k_apply_sweep<<<grid, kSwThreads, smem, st>>>(sp, sd, d_idx, d_val, lr, d_sigma_out, n_ranges);
+            // range size: the densest update should bring about 26 pairs per range (mean of a uniformly spread
+            // update), so that one load of 32 pairs per update and range is usually all of them
+            const double want = 26.0 / dens;
+            int rc;
+            if (want >= 512.0) rc = launch_apply_warps<512>(s, sp, d, d_idx, d_val, lr, d_sigma_out, st);
+            else if (want >= 384.0) rc = launch_apply_warps<384>(s, sp, d, d_idx, d_val, lr, d_sigma_out, st);
+            else if (want >= 256.0) rc = launch_apply_warps<256>(s, sp, d, d_idx, d_val, lr, d_sigma_out, st);
+            else if (want >= 192.0) rc = launch_apply_warps<192>(s, sp, d, d_idx, d_val, lr, d_sigma_out, st);
+            else rc = launch_apply_warps<128>(s, sp, d, d_idx, d_val, lr, d_sigma_out, st);
+            if (rc != ADACOMP_OK) return rc;
+            continue;
         } else {
             RangeDesc rd;
             rd.o = d;

@@ -234,6 +234,36 @@ def test_parameters_on_an_odd_address_and_odd_count(binding, mode):
     assert buf[0].item() == guard_lo and torch.equal(buf[P + 1:], guard_hi)      # nothing written outside Theta
 
 
+@pytest.mark.parametrize("mode", MODES)
+@pytest.mark.parametrize("density", [0.002, 0.03, 0.12, 0.3])
+def test_forty_updates_without_staleness_counts(binding, mode, density):
+    """More updates per call than one launch takes (32), windows that reach back before the call,
+    no staleness output asked for (the kernels' plain variants): parameters bit for bit."""
+    P = 200_003
+    rng = np.random.default_rng(int(density * 1000))
+    theta = torch.from_numpy(rng.standard_normal(P).astype(np.float32)).to(DEV)
+    ref = oracle.Server(theta.cpu().numpy())
+    srv = binding.Server(theta, history_pairs=1 << 23, max_window_updates=128)
+    srv.set_mode(mode)
+    ts = 0
+    for call in range(2):
+        n_up = 40
+        ups = [np.sort(rng.choice(P, int(P * density * rng.uniform(0.5, 1.0)), replace=False)).astype(np.uint32)
+               for _ in range(n_up)]
+        vals = [rng.standard_normal(a.size).astype(np.float32) for a in ups]
+        vals[7][::3] = 0.0
+        begin = np.concatenate([[0], np.cumsum([a.size for a in ups])[:-1]]).astype(np.uint64)
+        count = np.array([a.size for a in ups], np.uint32)
+        pull = np.array([max(0, ts + b - int(rng.integers(0, 50))) for b in range(n_up)], np.uint64)
+        idx, val = i32(np.concatenate(ups)), torch.from_numpy(np.concatenate(vals)).to(DEV)
+        srv.apply(idx, val, begin, count, pull, 0.05)
+        for b in range(n_up):
+            ref.apply(ups[b], vals[b], int(pull[b]), 0.05)
+        ts += n_up
+    assert srv.last_error() == 0 and srv.timestamp == ts == ref.timestamp
+    assert np.array_equal(bits(theta), bits(ref.theta()))
+
+
 def test_window_and_capacity_errors_leave_the_server_unchanged(binding):
     theta = torch.zeros(100, device=DEV)
     srv = binding.Server(theta, history_pairs=40, max_window_updates=8)     # ring of 64 pairs
