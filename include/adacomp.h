@@ -269,9 +269,9 @@ ADACOMP_API int adacomp_server_set_validation(adacomp_server_t* s, int on);
  * 0 = automatic: per launch of up to 32 updates, 3 when the launch's pairs number a fifth of
  *     the parameters or more, else 2; a single update goes as 1;
  * 1 = one launch per update, one thread per pair;
- * 2 = up to 32 updates per launch; a block owns a run of parameter ranges sized to the updates'
- *     density, sees all pairs of a range at once (one thread per pair) and keeps the order of
- *     the updates per parameter;
+ * 2 = up to 32 sparse updates per launch; a warp owns a run of parameter ranges, lines up all
+ *     pairs of a range in arrival order and applies them 32 at a time straight on global memory
+ *     (lanes that hold the same parameter take turns); only the named parameters are touched;
  * 3 = up to 32 updates per launch over a dense sweep: a warp owns a run of ranges of 128 to 512
  *     parameters (sized to the updates' density), brings Theta and the history heads of a range
  *     into shared memory whole, applies the updates' pairs of the range one update after the

@@ -94,283 +94,7 @@ struct BatchDesc {
     uint32_t n_updates;
 };
 
-// ---------------------------------------------------------------------------------------------
-// Several updates per launch, the block that owns a range of parameters sees all of its pairs at
-// once.  A block owns a run of ranges of `range` consecutive parameters.  Per range:
-//   stage    warp w loads, for updates w, w + 8, ..., the next <= 128 pairs from the update's
-//            cursor into shared memory (the loads of all updates are in flight together);
-//   scatter  every staged pair with a non-zero value sets bit b in the mask of its parameter
-//            (shared memory) and, if the table fits, records its slot under [b][parameter];
-//   pairs    ONE THREAD PER STAGED PAIR: Eq. 3 inside the batch is a population count of the mask
-//            under the update's window bits, the part of a window before the batch is a chain walk
-//            from the head the parameter had when the batch began; Eq. 5; the pair is linked behind
-//            the pair of the next lower bit (or the old head).  A pair that is its parameter's only
-//            change in the batch applies Eq. 4 at once (unless zero-valued pairs, which only read,
-//            are around); the others leave their step in shared memory and the pair of the
-//            highest bit lists the parameter;
-//   sums     one thread per listed parameter subtracts its steps in arrival order (Eq. 4 keeps its
-//            rounding order) and writes Theta and the head once.
-// No barrier separates the updates: the order is kept per parameter, which is all Algorithm 2
-// needs.  The limit of a round is the smallest index some update could not stage any more, so
-// every update's pairs below it are on chip; the range is finished in further rounds.  Same
-// results, bit for bit, as one launch per update.
-constexpr int kRgThreads = 256;
-constexpr uint32_t kRgStage = 128;             // pairs staged per update and round, at most
-constexpr uint32_t kRgChunks = kRgStage / 32;
-constexpr uint32_t kRgMinRange = 256, kRgMaxRange = 8192;
-constexpr uint32_t kRgLate = 0xFFFFu;          // staged slot that is not applied in this round
 constexpr uint32_t kRgAlphas = 33;             // alpha / sigma kept ready for sigma < 33
-
-struct RangeDesc {
-    BatchDesc o;
-    uint32_t range;                            // parameters per range, a multiple of 32
-    uint32_t chunks;                           // 32-pair chunks staged per update and round, 1..kRgChunks
-    uint32_t use_table;
-};
-
-struct RgMeta {                                // per-update state in shared memory
-    uint64_t begin[kMaxBatch];
-    uint32_t n[kMaxBatch], pos[kMaxBatch], win[kMaxBatch], bits[kMaxBatch];
-    uint32_t cur[kMaxBatch], cnt[kMaxBatch], adv[kMaxBatch];
-    float alpha[kRgAlphas];
-    uint32_t limit, n_listed, any_zero;
-};
-
-__host__ __device__ inline size_t rg_smem_bytes(uint32_t range, uint32_t n_updates, bool table) {
-    size_t b = static_cast<size_t>(range) * 4 + static_cast<size_t>(n_updates) * kRgStage * 4 + sizeof(RgMeta) +
-               static_cast<size_t>(n_updates) * kRgStage * 2 + static_cast<size_t>(range) * 2;
-    if (table) b += static_cast<size_t>(n_updates) * range;
-    return (b + 15) & ~static_cast<size_t>(15);
-}
-
-__global__ void __launch_bounds__(kRgThreads)
-k_apply_ranges(ServerParams sp, RangeDesc d, const uint32_t* __restrict__ idx, const float* __restrict__ val,
-               float lr, uint32_t* sigma_out, uint32_t n_ranges) {
-    extern __shared__ __align__(16) unsigned char s_rg[];
-    const uint32_t R = d.range, B = d.o.n_updates;
-    uint32_t* s_mask = reinterpret_cast<uint32_t*>(s_rg);                       // [R] updates that change the parameter
-    float* s_v = reinterpret_cast<float*>(s_mask + R);                          // [B][kRgStage] value, later the step
-    RgMeta* s_m = reinterpret_cast<RgMeta*>(s_v + B * kRgStage);
-    uint16_t* s_k = reinterpret_cast<uint16_t*>(s_m + 1);                       // [B][kRgStage] index - range start
-    uint16_t* s_list = s_k + B * kRgStage;                                      // [R] parameters changed more than once
-    uint8_t* s_tab = reinterpret_cast<uint8_t*>(s_list + R);                    // [B][R] slot of (update, parameter)
-
-    const uint32_t tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-    const uint32_t r_lo = static_cast<uint32_t>(static_cast<uint64_t>(n_ranges) * blockIdx.x / gridDim.x);
-    const uint32_t r_hi = static_cast<uint32_t>(static_cast<uint64_t>(n_ranges) * (blockIdx.x + 1) / gridDim.x);
-    if (r_lo == r_hi) return;
-    if (tid < B) {
-        const uint64_t first_param = static_cast<uint64_t>(r_lo) * R;
-        const uint64_t begin = d.o.pair_begin[tid];
-        uint32_t lo = 0, hi = d.o.n_pairs[tid];               // cursor: first pair at or above the first owned parameter
-        while (lo < hi) {
-            const uint32_t mid = lo + ((hi - lo) >> 1);
-            if (idx[begin + mid] < first_param) lo = mid + 1; else hi = mid;
-        }
-        s_m->cur[tid] = lo;
-        s_m->adv[tid] = 0;
-        s_m->begin[tid] = begin;
-        s_m->n[tid] = d.o.n_pairs[tid];
-        s_m->pos[tid] = d.o.pos_start[tid];
-        s_m->win[tid] = d.o.win_start[tid];
-        s_m->bits[tid] = d.o.win_bits[tid];
-    }
-    if (tid >= 64 && tid < 64 + kRgAlphas) {                    // Eq. 5 for the small counts, once
-        const uint32_t sigma = tid - 64;
-        s_m->alpha[sigma] = sigma ? __fdiv_rn(lr, static_cast<float>(sigma)) : lr;
-    }
-    auto range_end = [&](uint32_t r) -> uint32_t {
-        const uint64_t e = (static_cast<uint64_t>(r) + 1) * R;
-        return e < sp.n_params ? static_cast<uint32_t>(e) : static_cast<uint32_t>(sp.n_params);
-    };
-    // the slot of update b's pair on parameter kl of the range
-    auto slot_of = [&](uint32_t b, uint32_t kl) -> uint32_t {
-        if (d.use_table) return s_tab[b * R + kl];
-        const uint32_t cnt = s_m->cnt[b];                       // update b's stage is ascending: bisection
-        uint32_t t = 0;
-#pragma unroll
-        for (uint32_t step = kRgStage / 2; step; step >>= 1)
-            if (t + step < cnt && s_k[b * kRgStage + t + step] <= kl) t += step;
-        return t;
-    };
-    if (tid == 0) s_m->limit = range_end(r_lo);
-    __syncthreads();
-
-    uint32_t r = r_lo;
-    while (r < r_hi) {
-        const uint32_t lo = r * R, hi = range_end(r);
-        for (uint32_t t = tid; t < R / 4; t += kRgThreads) reinterpret_cast<uint4*>(s_mask)[t] = make_uint4(0, 0, 0, 0);
-        if (tid == 0) { s_m->n_listed = 0; s_m->any_zero = 0; }
-        // ---- stage
-        #pragma unroll 1
-        for (uint32_t b = warp; b < B; b += kRgThreads / 32) {
-            const uint64_t begin = s_m->begin[b];
-            const uint32_t n_b = s_m->n[b], cur = s_m->cur[b] + s_m->adv[b];     // past what the last round consumed
-            __syncwarp();
-            if (lane == 0) s_m->cur[b] = cur;
-            const uint32_t* ip = idx + begin + cur;
-            const float* vp = val + begin + cur;
-            const uint32_t left = n_b - cur;
-            uint32_t kk[kRgChunks];
-            float vv[kRgChunks];
-#pragma unroll
-            for (uint32_t c = 0; c < kRgChunks; ++c) {          // every load first: none waits for another
-                const uint32_t t = c * 32 + lane;
-                kk[c] = kNone;
-                vv[c] = 0.f;
-                if (c < d.chunks && t < left) {
-                    kk[c] = ip[t];
-                    vv[c] = vp[t];
-                }
-            }
-            uint32_t cnt = 0, last_k = 0;
-            bool run = true;                                    // staged = the leading slots below the range's end
-#pragma unroll
-            for (uint32_t c = 0; c < kRgChunks; ++c) {
-                const uint32_t t = c * 32 + lane, k = kk[c];
-                const bool in = k < hi;
-                if (in) {
-                    if (sp.validate && cur + t > 0 && ip[static_cast<int64_t>(t) - 1] >= k) record_error(sp.status, ADACOMP_ERR_UNSORTED);
-                    s_k[b * kRgStage + t] = k >= lo ? static_cast<uint16_t>(k - lo) : static_cast<uint16_t>(kRgLate);
-                    s_v[b * kRgStage + t] = vv[c];
-                }
-                const uint32_t bal = __ballot_sync(0xFFFFFFFFu, in);
-                if (run) {
-                    if (bal == 0xFFFFFFFFu) cnt += 32; else { cnt += __ffs(~bal) - 1; run = false; }
-                }
-                if (c + 1 == d.chunks) last_k = __shfl_sync(0xFFFFFFFFu, k, 31);
-            }
-            if (lane == 0) {
-                s_m->cnt[b] = cnt;
-                if (cnt == d.chunks * 32) atomicMin(&s_m->limit, last_k + 1);   // more of this update may follow in the range
-            }
-        }
-        __syncthreads();
-        const uint32_t limit = s_m->limit;
-        // ---- scatter: bit b on every parameter update b changes below the limit
-        #pragma unroll 1
-        for (uint32_t b = warp; b < B; b += kRgThreads / 32) {
-            const uint32_t cnt = s_m->cnt[b];
-            uint32_t adv = 0;
-            #pragma unroll 1
-            for (uint32_t t = lane; t < ((cnt + 31) & ~31u); t += 32) {
-                bool take = false;
-                if (t < cnt) {
-                    const uint32_t kl = s_k[b * kRgStage + t];
-                    if (kl == kRgLate) {                        // an index before the range: the list was not ascending
-                        record_error(sp.status, ADACOMP_ERR_UNSORTED);
-                        take = true;                            // consumed, not applied
-                    } else if (lo + kl < limit) {
-                        take = true;
-                        if (s_v[b * kRgStage + t] != 0.0f) {    // Eq. 3 counts changes: a zero entry is not one
-                            atomicOr(&s_mask[kl], 1u << b);
-                            if (d.use_table) s_tab[b * R + kl] = static_cast<uint8_t>(t);
-                        } else {
-                            s_m->any_zero = 1;                  // somebody may only read a parameter another pair changes
-                        }
-                    } else {
-                        s_k[b * kRgStage + t] = static_cast<uint16_t>(kRgLate);   // a later round's
-                    }
-                }
-                adv += __popc(__ballot_sync(0xFFFFFFFFu, take));
-            }
-            if (lane == 0) s_m->adv[b] = adv;
-        }
-        __syncthreads();
-        if (tid == 0) s_m->limit = limit < hi ? hi : (r + 1 < r_hi ? range_end(r + 1) : hi);   // for the next round
-        // ---- pairs: one thread per staged pair.  Heads and Theta are only written at once where no other
-        // pair of the round looks at the parameter: never while a zero-valued pair is around
-        const bool at_once = s_m->any_zero == 0;
-        #pragma unroll 1
-        for (uint32_t b = warp; b < B; b += kRgThreads / 32) {
-            const uint32_t cnt = s_m->adv[b];                   // ascending list: the pairs below the limit lead
-            const uint32_t cur_b = s_m->cur[b], pos_b = s_m->pos[b] + cur_b, bits_b = s_m->bits[b];
-            const uint32_t below_b = (1u << b) - 1u, ws = s_m->win[b];
-            const bool pre_b = (d.o.pre_mask >> b) & 1u;
-            uint32_t* sig = sigma_out ? sigma_out + s_m->begin[b] + cur_b : nullptr;
-            uint32_t kl[kRgChunks], m[kRgChunks], h0[kRgChunks];
-            float th[kRgChunks];
-#pragma unroll
-            for (uint32_t c = 0; c < kRgChunks; ++c) {          // every load first
-                const uint32_t t = c * 32 + lane;
-                kl[c] = kRgLate;
-                m[c] = 0;
-                h0[c] = kNone;
-                th[c] = 0.f;
-                if (t < cnt) kl[c] = s_k[b * kRgStage + t];
-                if (kl[c] != kRgLate) {
-                    m[c] = s_mask[kl[c]];
-                    h0[c] = sp.head[lo + kl[c]];
-                    th[c] = sp.theta[lo + kl[c]];
-                }
-            }
-#pragma unroll
-            for (uint32_t c = 0; c < kRgChunks; ++c) {
-                const uint32_t t = c * 32 + lane;
-                bool top = false;                               // this pair is the last of several changes of its parameter
-                if (kl[c] != kRgLate) {
-                    const float v = s_v[b * kRgStage + t];
-                    uint32_t sigma = __popc(m[c] & bits_b);                                            // Eq. 3, inside the batch
-                    if (pre_b) {                                                                       // Eq. 3, before the batch
-                        uint32_t q = h0[c], hops = 0;
-                        while (q != kNone && q >= ws) {
-                            if (++hops > sp.max_window) { record_error(sp.status, ADACOMP_ERR_WINDOW); break; }
-                            q = sp.prev[(q + sp.ring_shift) & sp.ring_mask];
-                        }
-                        sigma += hops;
-                    }
-                    if (sig) sig[t] = sigma;
-                    if (v != 0.0f) {
-                        const float alpha_k = sigma < kRgAlphas ? s_m->alpha[sigma] : __fdiv_rn(lr, static_cast<float>(sigma));   // Eq. 5
-                        const float step = __fmul_rn(alpha_k, v);
-                        const uint32_t pos = pos_b + t, low = m[c] & below_b;
-                        uint32_t before = h0[c];                // the pair that changed the parameter last
-                        if (low) {
-                            const uint32_t b2 = 31 - __clz(low);
-                            before = s_m->pos[b2] + s_m->cur[b2] + slot_of(b2, kl[c]);
-                        }
-                        sp.prev[(pos + sp.ring_shift) & sp.ring_mask] = before;
-                        if (at_once && m[c] == (1u << b)) {     // the parameter's only change in this batch
-                            sp.theta[lo + kl[c]] = __fsub_rn(th[c], step);                             // Eq. 4
-                            sp.head[lo + kl[c]] = pos;
-                        } else {
-                            s_v[b * kRgStage + t] = step;
-                            top = (m[c] >> b) == 1u;
-                        }
-                    }
-                }
-                const uint32_t bal = __ballot_sync(0xFFFFFFFFu, top);
-                if (bal) {
-                    uint32_t base = 0;
-                    if (lane == 0) base = atomicAdd(&s_m->n_listed, __popc(bal));
-                    base = __shfl_sync(0xFFFFFFFFu, base, 0);
-                    if (top) s_list[base + __popc(bal & ((1u << lane) - 1u))] = static_cast<uint16_t>(kl[c]);
-                }
-            }
-        }
-        __syncthreads();
-        // ---- sums: one thread per parameter changed more than once, its steps in arrival order
-        const uint32_t n_listed = s_m->n_listed;
-        #pragma unroll 1
-        for (uint32_t j = tid; j < n_listed; j += kRgThreads) {
-            const uint32_t kl = s_list[j];
-            uint32_t m = s_mask[kl], t = 0, b = 0;
-            float theta = sp.theta[lo + kl];
-            while (m) {
-                b = __ffs(m) - 1;
-                m &= m - 1;
-                t = slot_of(b, kl);
-                theta = __fsub_rn(theta, s_v[b * kRgStage + t]);                                       // Eq. 4
-            }
-            sp.theta[lo + kl] = theta;
-            sp.head[lo + kl] = s_m->pos[b] + s_m->cur[b] + t;
-        }
-        __syncthreads();
-        if (limit >= hi) ++r;                                   // else: the rest of the range in another round
-    }
-    // whoever owns the last range sees what no range claimed: indices >= n_params
-    if (r_hi == n_ranges && tid < B && s_m->cur[tid] + s_m->adv[tid] < s_m->n[tid]) record_error(sp.status, ADACOMP_ERR_UNSORTED);
-}
 
 // ---------------------------------------------------------------------------------------------
 // Several updates per launch, one WARP per range of parameters, no block barrier in the loop.  A
@@ -598,6 +322,239 @@ k_apply_warps(const ServerParams sp, const BatchDesc d, const uint32_t* __restri
     if (r_hi == n_ranges && lane < B && s_cur[lane] < d.n_pairs[lane]) record_error(sp.status, ADACOMP_ERR_UNSORTED);
 }
 
+// First position of an ascending index list whose entry is >= target.  The lists of an update are spread
+// over [0, n_params) more or less evenly, so a few interpolation steps narrow the search before the
+// bisection that finishes it: far fewer dependent loads than bisection alone on a long list.
+__device__ __forceinline__ uint32_t first_at_or_above(const uint32_t* __restrict__ list, uint32_t n, uint64_t target,
+                                                      uint64_t n_params) {
+    uint32_t lo = 0, hi = n;                                    // answer in [lo, hi]
+    uint64_t v_lo = 0, v_hi = n_params;                         // list[lo - 1] < target <= list[hi], bounds on those values
+#pragma unroll 1
+    for (int step = 0; step < 4 && hi - lo > 64; ++step) {
+        if (target <= v_lo || target >= v_hi) break;
+        const uint64_t span = hi - lo;
+        uint64_t guess = lo + (target - v_lo) * span / (v_hi - v_lo);
+        // two probes a little either side of the guess: both outcomes shrink the range a lot
+        const uint64_t slack = 8 + (span >> 7);
+        const uint32_t p0 = static_cast<uint32_t>(guess > lo + slack ? guess - slack : lo);
+        const uint32_t p1 = static_cast<uint32_t>(guess + slack < hi - 1 ? guess + slack : hi - 1);
+        const uint32_t x0 = list[p0], x1 = list[p1];
+        if (x0 >= target) { hi = p0; v_hi = x0; }
+        else if (x1 < target) { lo = p1 + 1; v_lo = x1; }
+        else { lo = p0 + 1; v_lo = x0; hi = p1; v_hi = x1; }
+    }
+    while (lo < hi) {
+        const uint32_t mid = lo + ((hi - lo) >> 1);
+        if (list[mid] < target) lo = mid + 1; else hi = mid;
+    }
+    return lo;
+}
+
+// ---------------------------------------------------------------------------------------------
+// Several sparse updates per launch, one WARP per range of parameters, no block barrier, nothing
+// swept: only the parameters that are named are touched.  A warp owns a run of ranges and keeps,
+// per update, a stage with the update's next 32 pairs from its cursor (lane b looks after update
+// b).  Per range: lane b counts the staged pairs of update b below the range's end (a bisection:
+// the list is ascending); a warp scan lines all of them up in arrival order (update after update);
+// then they are applied 32 at a time, one pair per lane, straight on global memory and exactly as
+// Algorithm 2 states it: Eq. 3 is the walk along the parameter's chain while it stays inside the
+// window (pairs of this launch applied earlier are on the chain already), Eq. 5, Eq. 4, and the
+// pair becomes the head.  Pairs of one update name distinct parameters; two lanes that hold the
+// same parameter (different updates) are found with a match and take turns in arrival order.
+// Loads of Theta, heads and links go to L2 (no L1 line survives a change by another lane), and a
+// warp-level barrier orders one group of 32 before the next.  A stage that runs low is refilled
+// from the update's new cursor; one that ran dry inside the range is refilled at once and the
+// range is looked at again (later updates wait until that update is through with the range).  Same results, bit for bit, as one launch per update.
+constexpr int kMgThreads = 128;
+constexpr uint32_t kMgWarps = kMgThreads / 32;
+constexpr uint32_t kMgPitch = 33;              // words per staged update: lanes that probe, and lanes that fill, hit distinct banks
+constexpr uint32_t kMgLow = 10;                // refill a stage with fewer pairs left
+
+__host__ __device__ inline size_t mg_smem_bytes(uint32_t n_updates) {
+    return static_cast<size_t>(kMgWarps) * n_updates * kMgPitch * 8;
+}
+
+template <bool kExtra>
+__global__ void __launch_bounds__(kMgThreads)
+k_apply_merged(const ServerParams sp, const BatchDesc d, uint32_t range, const uint32_t* __restrict__ idx,
+               const float* __restrict__ val, float lr, uint32_t* sigma_out, uint32_t n_ranges) {
+    extern __shared__ __align__(16) unsigned char s_mg[];
+    const uint32_t B = d.n_updates;
+    const uint32_t lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const uint32_t lt = (1u << lane) - 1u;
+    uint32_t* s_k = reinterpret_cast<uint32_t*>(s_mg) + warp * B * kMgPitch * 2;   // [B][33] staged indices
+    float* s_v = reinterpret_cast<float*>(s_k + B * kMgPitch);                  // [B][33] staged values
+    const uint32_t gw = blockIdx.x * kMgWarps + warp, n_gw = gridDim.x * kMgWarps;
+    const uint32_t r_lo = static_cast<uint32_t>(static_cast<uint64_t>(n_ranges) * gw / n_gw);
+    const uint32_t r_hi = static_cast<uint32_t>(static_cast<uint64_t>(n_ranges) * (gw + 1) / n_gw);
+    if (r_lo == r_hi) return;
+
+    // lane b's view of update b
+    const bool has = lane < B;
+    const uint32_t n_b = has ? d.n_pairs[lane] : 0u, pos0_b = has ? d.pos_start[lane] : 0u, ws_b = has ? d.win_start[lane] : 0u;
+    const uint64_t begin_b = has ? d.pair_begin[lane] : 0ull;
+    uint32_t cur = 0, sb = 0;                                   // cursor; cursor of the stage's slot 0
+    if (has) cur = first_at_or_above(idx + begin_b, n_b, static_cast<uint64_t>(r_lo) * range, sp.n_params);
+    // the stage of update b takes its next 32 pairs from cursor c (kNone beyond the end of the list); all lanes;
+    // the copies are asynchronous: copy_async_wait<0>() and a warp barrier before the stage is read
+    const uint32_t a_k = smem_address(s_k + lane), a_v = smem_address(s_v + lane);
+    auto fill = [&](uint32_t b, uint32_t c) {
+        const uint32_t t = c + lane;
+        if (t < d.n_pairs[b]) {
+            copy_async_4(a_k + b * (kMgPitch * 4), idx + d.pair_begin[b] + t);
+            copy_async_4(a_v + b * (kMgPitch * 4), val + d.pair_begin[b] + t);
+        } else {
+            s_k[b * kMgPitch + lane] = kNone;
+        }
+    };
+    for (uint32_t b = 0; b < B; ++b) fill(b, __shfl_sync(0xFFFFFFFFu, cur, b));
+    sb = cur;
+    copy_async_commit();
+    copy_async_wait<0>();
+    __syncwarp();
+
+    for (uint32_t r = r_lo; r < r_hi; ++r) {
+        const uint64_t end64 = (static_cast<uint64_t>(r) + 1) * range;
+        const uint32_t hi = end64 <= sp.n_params ? static_cast<uint32_t>(end64) : static_cast<uint32_t>(sp.n_params);
+        const uint32_t lo = r * range;
+        for (;;) {
+            // ---- how many staged pairs of update b lie below the range's end
+            const uint32_t c0 = cur - sb;                       // first staged slot not yet applied, 0..32
+            uint32_t cnt = 0;
+            bool dry = false;
+            if (has) {
+                uint32_t a = c0, z = 32;                        // first slot in [c0, 32) whose index is >= hi
+                while (a < z) {
+                    const uint32_t mid = (a + z) >> 1;
+                    if (s_k[lane * kMgPitch + mid] < hi) a = mid + 1; else z = mid;
+                }
+                cnt = a - c0;
+                dry = a == 32 && sb + 32 < n_b;                 // every staged pair lies in the range: more may follow
+            }
+            // a stage that ran dry: its update may have more pairs in the range, and they come before those of
+            // every later update, so the later updates wait for the next turn
+            const uint32_t dry_mask = __ballot_sync(0xFFFFFFFFu, dry);
+            if (dry_mask) {
+                const uint32_t first_dry = __ffs(dry_mask) - 1;
+                if (lane > first_dry) cnt = 0;
+                dry = lane == first_dry;
+            }
+            uint32_t incl = cnt;
+#pragma unroll
+            for (int s = 1; s < 32; s <<= 1) {
+                const uint32_t y = __shfl_up_sync(0xFFFFFFFFu, incl, s);
+                if (lane >= static_cast<uint32_t>(s)) incl += y;
+            }
+            const uint32_t total = __shfl_sync(0xFFFFFFFFu, incl, 31), off = incl - cnt;
+            // stages that run low are refilled from the cursor the update will have after this turn
+            const uint32_t cur_next = cur + cnt;
+            const bool low = has && sb + 32 < n_b && (dry || sb + 32 - cur_next < kMgLow);
+            const uint32_t low_mask = __ballot_sync(0xFFFFFFFFu, low);
+            auto refill = [&]() {
+                __syncwarp();                                   // every lane has what it wanted from the stages
+                uint32_t m = low_mask;
+                while (m) {
+                    const uint32_t b = __ffs(m) - 1;
+                    m &= m - 1;
+                    fill(b, __shfl_sync(0xFFFFFFFFu, cur_next, b));
+                }
+                copy_async_commit();
+            };
+            // ---- up to 128 pairs at a time, four per lane, in arrival order
+            const bool early = total <= 128;                    // one turn of the loop below: refill while it works
+            bool refilled = false;
+#pragma unroll 1
+            for (uint32_t c = 0; c < total; c += 128) {
+                uint32_t kq[4], posq[4], wsq[4];
+                uint64_t sq[4];                                 // kExtra: where the pair's staleness count goes
+                float vq[4];
+#pragma unroll
+                for (uint32_t u = 0; u < 4; ++u) {
+                    const uint32_t e = c + 32 * u + lane;
+                    const bool valid = e < total;
+                    uint32_t b = 0;                             // the update of pair e: how many updates end at or before e
+#pragma unroll
+                    for (uint32_t s = 16; s; s >>= 1) {
+                        const uint32_t t = __shfl_sync(0xFFFFFFFFu, incl, (b + s - 1) & 31u);
+                        if (t <= e) b += s;
+                    }
+                    b &= 31u;
+                    const uint32_t jj = e - __shfl_sync(0xFFFFFFFFu, off, b);    // its place among the update's pairs of this turn
+                    const uint32_t slot = __shfl_sync(0xFFFFFFFFu, c0, b) + jj;
+                    const uint32_t at = __shfl_sync(0xFFFFFFFFu, cur, b) + jj;  // its place in the update's list
+                    posq[u] = __shfl_sync(0xFFFFFFFFu, pos0_b, b) + at;
+                    wsq[u] = __shfl_sync(0xFFFFFFFFu, ws_b, b);
+                    sq[u] = 0;
+                    if (kExtra) {
+                        const uint32_t blo = __shfl_sync(0xFFFFFFFFu, static_cast<uint32_t>(begin_b), b);
+                        const uint32_t bhi = __shfl_sync(0xFFFFFFFFu, static_cast<uint32_t>(begin_b >> 32), b);
+                        sq[u] = ((static_cast<uint64_t>(bhi) << 32) | blo) + at;
+                    }
+                    kq[u] = kNone;
+                    vq[u] = 0.f;
+                    if (valid) {
+                        kq[u] = s_k[b * kMgPitch + slot];
+                        vq[u] = s_v[b * kMgPitch + slot];
+                        prefetch_l2(sp.head + kq[u]);           // wanted in a moment, by a load that must see the latest value
+                        prefetch_l2(sp.theta + kq[u]);
+                        if (kq[u] < lo) record_error(sp.status, ADACOMP_ERR_UNSORTED);   // the list was not ascending
+                        if (kExtra && sp.validate && at > 0) {
+                            const uint32_t before = slot > 0 ? s_k[b * kMgPitch + slot - 1] : idx[sq[u] - 1];
+                            if (before >= kq[u]) record_error(sp.status, ADACOMP_ERR_UNSORTED);
+                        }
+                    }
+                }
+                if (early && low_mask) { refill(); refilled = true; }
+#pragma unroll
+                for (uint32_t u = 0; u < 4; ++u) {
+                    if (c + 32 * u >= total) break;
+                    const uint32_t k = kq[u], ws = wsq[u], pos = posq[u];
+                    const float v = vq[u];
+                    // lanes that hold the same parameter take turns, lower lane (earlier update) first
+                    const uint32_t vmask = __ballot_sync(0xFFFFFFFFu, k != kNone);
+                    const uint32_t peers = __match_any_sync(0xFFFFFFFFu, k) & vmask;
+                    uint32_t pending = vmask;
+                    bool waiting = k != kNone;
+                    while (pending) {
+                        const bool go = waiting && (peers & pending & lt) == 0;
+                        if (go) {
+                            const uint32_t latest = __ldcg(sp.head + k);
+                            const float theta = __ldcg(sp.theta + k);
+                            uint32_t q = latest, sigma = 0;                                            // Eq. 3
+                            while (q != kNone && q >= ws) {
+                                if (++sigma > sp.max_window) { record_error(sp.status, ADACOMP_ERR_WINDOW); break; }
+                                q = __ldcg(sp.prev + ((q + sp.ring_shift) & sp.ring_mask));
+                            }
+                            if (kExtra && sigma_out) sigma_out[sq[u]] = sigma;
+                            if (v != 0.0f) {                    // Eq. 3 counts changes: a zero entry is not one
+                                const float alpha_k = sigma ? __fdiv_rn(lr, static_cast<float>(sigma)) : lr;   // Eq. 5
+                                __stcg(sp.theta + k, __fsub_rn(theta, __fmul_rn(alpha_k, v)));         // Eq. 4
+                                __stcg(sp.prev + ((pos + sp.ring_shift) & sp.ring_mask), latest);
+                                __stcg(sp.head + k, pos);
+                            }
+                            waiting = false;
+                        }
+                        __syncwarp();                           // what this turn wrote is seen by the next
+                        pending &= ~__ballot_sync(0xFFFFFFFFu, go);
+                    }
+                }
+            }
+            if (low_mask && !refilled) refill();
+            // ---- cursors move on
+            cur = cur_next;
+            if (low) sb = cur;
+            if (low_mask) {
+                copy_async_wait<0>();
+                __syncwarp();
+            }
+            const bool again = dry_mask != 0;
+            if (!again) break;
+        }
+    }
+    // whoever owns the last range sees what no range claimed: indices >= n_params
+    if (r_hi == n_ranges && has && cur < n_b) record_error(sp.status, ADACOMP_ERR_UNSORTED);
+}
+
 // ---------------------------------------------------------------------------------------------
 // The competitors' rule ("Experimental setup": for ASGD and Comp-ASGD the learning rate is divided
 // by staleness and is global to each update): every entry of an update gets the same learning
@@ -767,6 +724,38 @@ int launch_apply_warps(const adacomp_server_t* s, const ServerParams& sp, const 
                  : launch_apply_warps_as<R, false, false>(s, sp, d, d_idx, d_val, lr, d_sigma_out, st);
 }
 
+// Launches k_apply_merged with ranges sized so that a range holds about 128 pairs of the launch.
+int launch_apply_merged(const adacomp_server_t* s, const ServerParams& sp, const BatchDesc& d, uint64_t pairs,
+                        const uint32_t* d_idx, const float* d_val, float lr, uint32_t* d_sigma_out, cudaStream_t st) {
+    const bool extra = d_sigma_out != nullptr || sp.validate != 0;
+    const size_t smem = mg_smem_bytes(d.n_updates);
+    int per_sm = 1;
+    if (extra) {
+        ADACOMP_CUDA(cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, k_apply_merged<true>, kMgThreads, smem));
+    } else {
+        ADACOMP_CUDA(cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, k_apply_merged<false>, kMgThreads, smem));
+    }
+    const uint64_t warps = static_cast<uint64_t>(s->n_sms) * static_cast<uint64_t>(per_sm > 0 ? per_sm : 1) * kMgWarps;
+    // a range should hold about 128 pairs (at most ~8 per update, so that a stage of 32 lasts), and every warp
+    // should get several ranges
+    double want = 128.0 * static_cast<double>(s->n_params) / static_cast<double>(pairs);
+    const double balance = static_cast<double>(s->n_params) / (2.0 * static_cast<double>(warps));
+    if (want > balance) want = balance;
+    uint64_t range = want < 32.0 ? 32 : static_cast<uint64_t>(want) / 32 * 32;
+    if (range > (1u << 30)) range = 1u << 30;
+    const uint64_t n_ranges64 = (s->n_params + range - 1) / range;
+    const uint32_t n_ranges = static_cast<uint32_t>(n_ranges64);
+    uint64_t grid = warps / kMgWarps;
+    const uint64_t most_blocks = (n_ranges64 + kMgWarps - 1) / kMgWarps;
+    if (grid > most_blocks) grid = most_blocks;
+    if (extra)
+        k_apply_merged<true><<<static_cast<unsigned>(grid), kMgThreads, smem, st>>>(sp, d, static_cast<uint32_t>(range), d_idx, d_val, lr, d_sigma_out, n_ranges);
+    else
+        k_apply_merged<false><<<static_cast<unsigned>(grid), kMgThreads, smem, st>>>(sp, d, static_cast<uint32_t>(range), d_idx, d_val, lr, d_sigma_out, n_ranges);
+    ADACOMP_LAUNCH_CHECK();
+    return ADACOMP_OK;
+}
+
 bool sizes_ok(uint64_t n_params, uint64_t history_pairs) {
     return n_params >= 1 && n_params <= 0xFFFFFFFEull && history_pairs >= 1 && history_pairs < (1ull << 31);
 }
@@ -806,9 +795,6 @@ int adacomp_server_create(adacomp_server_t** out, uint64_t n_params, uint64_t hi
     cudaError_t e = guard.err;
     if (e == cudaSuccess) e = cudaDeviceGetAttribute(&s->n_sms, cudaDevAttrMultiProcessorCount, device);
     if (e == cudaSuccess) e = cudaMemset(s->d_status, 0, sizeof(int));
-    if (e == cudaSuccess)
-        e = cudaFuncSetAttribute(k_apply_ranges, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                 static_cast<int>(rg_smem_bytes(kRgMaxRange, kMaxBatch, false) + 32768));   // + the largest slot table
     if (e == cudaSuccess) e = cudaDeviceSynchronize();
     if (e != cudaSuccess) { delete s; return cuda_fail(e); }
     *out = s;
@@ -978,7 +964,8 @@ int adacomp_apply(adacomp_server_t* s, const uint32_t* d_idx, const float* d_val
     // ---- launches.  One launch per update, or launches of up to kMaxBatch updates each: same results.
     // Automatic choice per launch: the warp-per-range kernel over a dense sweep of Theta when the launch's pairs
     // number a fifth of the parameters or more (nearly every 32-byte sector of Theta is touched anyway), else the
-    // ranges kernel; a single update, and updates whose staleness slots overlap in memory, go one per launch.
+    // kernel that touches only the named parameters; a single update, and updates whose staleness slots overlap in
+    // memory, go one per launch.
     bool shared_slots = false;                 // two updates write their counts to the same slots: order matters
     if (d_sigma_out && n_updates > 1 && s->mode != 1) {
         std::vector<std::pair<uint64_t, uint64_t>> slices;
@@ -1016,40 +1003,20 @@ int adacomp_apply(adacomp_server_t* s, const uint32_t* d_idx, const float* d_val
         const double dens = static_cast<double>(most) / static_cast<double>(s->n_params);   // of the densest update
         const bool sweep = theta_aligned &&
                            (s->mode == 3 || (s->mode == 0 && static_cast<double>(pairs) >= 0.2 * static_cast<double>(s->n_params)));
+        int rc;
         if (sweep) {
             // range size: the densest update should bring about 26 pairs per range (mean of a uniformly spread
             // update), so that one load of 32 pairs per update and range is usually all of them
             const double want = 26.0 / dens;
-            int rc;
             if (want >= 512.0) rc = launch_apply_warps<512>(s, sp, d, d_idx, d_val, lr, d_sigma_out, st);
             else if (want >= 384.0) rc = launch_apply_warps<384>(s, sp, d, d_idx, d_val, lr, d_sigma_out, st);
             else if (want >= 256.0) rc = launch_apply_warps<256>(s, sp, d, d_idx, d_val, lr, d_sigma_out, st);
             else if (want >= 192.0) rc = launch_apply_warps<192>(s, sp, d, d_idx, d_val, lr, d_sigma_out, st);
             else rc = launch_apply_warps<128>(s, sp, d, d_idx, d_val, lr, d_sigma_out, st);
-            if (rc != ADACOMP_OK) return rc;
-            continue;
         } else {
-            RangeDesc rd;
-            rd.o = d;
-            // range size: the densest update should bring about 96 pairs per range, so that mean + 3 standard
-            // deviations of a uniformly spread update still fit the stage of 128
-            const double want = 96.0 / dens;
-            uint32_t range = want >= kRgMaxRange ? kRgMaxRange : static_cast<uint32_t>(want) & ~31u;
-            if (range < kRgMinRange) range = kRgMinRange;
-            const double mean = dens * range;
-            const uint32_t chunks = static_cast<uint32_t>((mean + 3.0 * std::sqrt(mean) + 2.0) / 32.0) + 1;
-            rd.range = range;
-            rd.chunks = chunks > kRgChunks ? kRgChunks : chunks;
-            rd.use_table = static_cast<uint64_t>(d.n_updates) * range <= 32768 ? 1u : 0u;
-            const size_t smem = rg_smem_bytes(range, d.n_updates, rd.use_table != 0);
-            const uint32_t n_ranges = static_cast<uint32_t>((s->n_params + range - 1) / range);
-            int per_sm = 1;
-            ADACOMP_CUDA(cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, k_apply_ranges, kRgThreads, smem));
-            unsigned grid = static_cast<unsigned>(s->n_sms) * static_cast<unsigned>(per_sm > 0 ? per_sm : 1);
-            if (grid > n_ranges) grid = n_ranges;
-            k_apply_ranges<<<grid, kRgThreads, smem, st>>>(sp, rd, d_idx, d_val, lr, d_sigma_out, n_ranges);
+            rc = launch_apply_merged(s, sp, d, pairs, d_idx, d_val, lr, d_sigma_out, st);
         }
-        ADACOMP_LAUNCH_CHECK();
+        if (rc != ADACOMP_OK) return rc;
     }
     for (uint32_t b = 0; b < n_updates && one_by_one; ++b) {
         UpdateDesc u;

@@ -398,44 +398,81 @@ __global__ void __launch_bounds__(kThreads, 4) k_bracket_scan(SelectParams p, ui
 // The same pass for tensors whose candidates are dense (a percent of the entries or more), where
 // nearly every load holds a candidate and queueing loads would only add work.  Same
 // decomposition (8 warps x 8 pieces of 1024 entries per block, warps on their own).  Per piece:
-//   count    the four components of each of the lane's loads are tested and counted (one byte
-//            per load; population counts and ballots are slow instructions, sums of predicates
-//            are not) and a byte-packed warp scan turns the counts into every candidate's place
-//            in index order (load, lane, component);
-//   place    a second sweep over the registers stores every candidate's position and value at
-//            its place on a shared-memory stage, behind the candidates of the pieces staged
-//            before, with predicated stores (no branch per entry).
+//   count    the four components of each of the lane's loads are tested and counted, one byte per
+//            load (a compare and a predicated add per entry), and a byte-packed warp scan turns
+//            the counts into every candidate's place in index order (load, lane, component);
+//   place    a second sweep over the registers stores every candidate, value and position in one
+//            8-byte entry, at its place on a shared-memory stage behind the candidates of the
+//            pieces staged before (a compare, a predicated store and a predicated step of the
+//            address per entry: no branch).
 //   Both run for the lane's loads 0-3, whose registers are then refilled with the next piece,
 //   and again for loads 4-7.
 // Flush, once the stage could not take another piece and after the last one, while the next
-// piece's loads are in flight: an atomic reserves room in the candidate list for all staged
-// pieces; with every lane busy, one lane per staged candidate tests it against t_hi (and for
-// NaN) and stages window entries, ranked by ballot; a second atomic reserves their room; the
-// table entries of the pieces are written and the lists leave with coalesced stores.
+// piece's loads are in flight: a first pass with one lane per staged candidate counts the window
+// entries (those not above t_hi; also per piece, for the table) and looks for NaN; two atomics
+// reserve room in the candidate and the window list; a second pass writes both lists with
+// coalesced stores, window entries ranked by ballot.
 constexpr uint32_t kDenseStage = 768;                          // candidates the stage holds
 constexpr uint32_t kDensePiece = 512;                          // most candidates one piece (of 1024 entries) may bring
-constexpr uint32_t kDenseWinStage = 256;                       // window entries staged per flush
-constexpr size_t kDenseSmemPerWarp = kDenseStage * 6 + kDenseWinStage * 8 + 64;
+constexpr size_t kDenseSmemPerWarp = kDenseStage * 8 + 64;
 
-// if (|x| >= t or unordered) { pos[r] = place; val[r] = x; ++r; } with predicated instructions;
-// pos_base and val_base are the shared-memory addresses of the two stage arrays
-__device__ __forceinline__ void dense_place(float x, float t, uint32_t& r, uint32_t pos_base, uint32_t val_base,
-                                            uint32_t place) {
+// cnt += kUnit for each of the four components with |x| >= t or unordered
+template <uint32_t kUnit>
+__device__ __forceinline__ void dense_count(const float4& x, float t, uint32_t& cnt) {
+    asm("{\n\t"
+        ".reg .pred p;\n\t"
+        ".reg .f32 a;\n\t"
+        "abs.f32 a, %1;\n\t"
+        "setp.geu.f32 p, a, %5;\n\t"
+        "@p add.u32 %0, %0, %6;\n\t"
+        "abs.f32 a, %2;\n\t"
+        "setp.geu.f32 p, a, %5;\n\t"
+        "@p add.u32 %0, %0, %6;\n\t"
+        "abs.f32 a, %3;\n\t"
+        "setp.geu.f32 p, a, %5;\n\t"
+        "@p add.u32 %0, %0, %6;\n\t"
+        "abs.f32 a, %4;\n\t"
+        "setp.geu.f32 p, a, %5;\n\t"
+        "@p add.u32 %0, %0, %6;\n\t"
+        "}"
+        : "+r"(cnt)
+        : "f"(x.x), "f"(x.y), "f"(x.z), "f"(x.w), "f"(t), "n"(kUnit));
+}
+
+// for each of the four components with |x| >= t or unordered: { stage[a] = (x, e); a += 8; ++e regardless }
+// a: shared-memory byte address of the next free stage entry of this lane's run; e0: position of x.x
+__device__ __forceinline__ void dense_place(const float4& x, float t, uint32_t& a, uint32_t e0) {
     asm volatile(
         "{\n\t"
         ".reg .pred p;\n\t"
-        ".reg .f32 a;\n\t"
-        ".reg .u32 ap, av;\n\t"
-        "abs.f32 a, %1;\n\t"
-        "setp.geu.f32 p, a, %2;\n\t"
-        "mad.lo.u32 ap, %0, 2, %3;\n\t"
-        "mad.lo.u32 av, %0, 4, %4;\n\t"
-        "@p st.shared.u16 [ap], %5;\n\t"
-        "@p st.shared.f32 [av], %1;\n\t"
-        "@p add.u32 %0, %0, 1;\n\t"
+        ".reg .f32 m;\n\t"
+        ".reg .b32 v, e;\n\t"
+        "abs.f32 m, %1;\n\t"
+        "setp.geu.f32 p, m, %5;\n\t"
+        "mov.b32 v, %1;\n\t"
+        "@p st.shared.v2.b32 [%0], {v, %6};\n\t"
+        "@p add.u32 %0, %0, 8;\n\t"
+        "abs.f32 m, %2;\n\t"
+        "setp.geu.f32 p, m, %5;\n\t"
+        "mov.b32 v, %2;\n\t"
+        "add.u32 e, %6, 1;\n\t"
+        "@p st.shared.v2.b32 [%0], {v, e};\n\t"
+        "@p add.u32 %0, %0, 8;\n\t"
+        "abs.f32 m, %3;\n\t"
+        "setp.geu.f32 p, m, %5;\n\t"
+        "mov.b32 v, %3;\n\t"
+        "add.u32 e, %6, 2;\n\t"
+        "@p st.shared.v2.b32 [%0], {v, e};\n\t"
+        "@p add.u32 %0, %0, 8;\n\t"
+        "abs.f32 m, %4;\n\t"
+        "setp.geu.f32 p, m, %5;\n\t"
+        "mov.b32 v, %4;\n\t"
+        "add.u32 e, %6, 3;\n\t"
+        "@p st.shared.v2.b32 [%0], {v, e};\n\t"
+        "@p add.u32 %0, %0, 8;\n\t"
         "}"
-        : "+r"(r)
-        : "f"(x), "f"(t), "r"(pos_base), "r"(val_base), "h"(static_cast<unsigned short>(place))
+        : "+r"(a)
+        : "f"(x.x), "f"(x.y), "f"(x.z), "f"(x.w), "f"(t), "r"(e0)
         : "memory");
 }
 
@@ -456,19 +493,16 @@ __global__ void __launch_bounds__(kThreads, 4) k_bracket_scan_dense(SelectParams
     const uint32_t lt = (1u << lane) - 1u;
     constexpr uint32_t kStep = kThreads / 32;
     constexpr uint32_t kBatch = kSpansPerBlock * kSubsPerSpan / kStep;
+    static_assert(kStep == 8, "the piece of a staged position is found with a shift");
     const uint32_t ss_end = min(item.y + kSpansPerBlock, L.n_spans) * kSubsPerSpan;
     const uint32_t ss0 = item.y * kSubsPerSpan + warp;
     if (ss0 >= ss_end) return;
     const uint32_t in_lo = mis ? 1u : 0u, in_hi = n_shift / kSubElems;
     unsigned char* mine = s_scan + warp * kDenseSmemPerWarp;
-    float* stage_val = reinterpret_cast<float*>(mine);                                        // [kDenseStage]
-    uint32_t* stage_widx = reinterpret_cast<uint32_t*>(mine + kDenseStage * 4);                // [kDenseWinStage]
-    uint32_t* stage_wkey = stage_widx + kDenseWinStage;
-    uint32_t* s_tc = stage_wkey + kDenseWinStage;                                             // [8] candidates per piece
+    uint2* stage = reinterpret_cast<uint2*>(mine);                                            // [kDenseStage] (value bits, shifted position)
+    uint32_t* s_tc = reinterpret_cast<uint32_t*>(mine + kDenseStage * 8);                      // [8] candidates per piece
     uint32_t* s_tw = s_tc + kBatch;                                                           // [8] window entries per piece
-    uint16_t* stage_pos = reinterpret_cast<uint16_t*>(s_tw + kBatch);                         // [kDenseStage] piece * 1024 + place
-    const uint32_t val_base = static_cast<uint32_t>(__cvta_generic_to_shared(stage_val));
-    const uint32_t pos_base = static_cast<uint32_t>(__cvta_generic_to_shared(stage_pos));
+    const uint32_t stage_base = static_cast<uint32_t>(__cvta_generic_to_shared(stage));
     uint32_t* cand_idx = p.cand_idx + static_cast<uint64_t>(w) * p.cand_stride + L.cand_base;
     float* cand_val = p.cand_val + static_cast<uint64_t>(w) * p.cand_stride + L.cand_base;
     uint32_t* win_key = p.win_key + static_cast<uint64_t>(w) * p.win_stride + L.win_base;
@@ -477,36 +511,30 @@ __global__ void __launch_bounds__(kThreads, 4) k_bracket_scan_dense(SelectParams
 
     bool saw_nan = false, lost = false;                        // lost: something did not fit
     uint32_t staged = 0, j_first = 0;                          // candidates on the stage; first piece they belong to
-    // shifted coordinate inside the tensor of a staged position
-    auto entry_of = [&](uint32_t pos) -> uint32_t { return (ss0 + kStep * (pos >> 10)) * kSubElems + (pos & 1023u); };
     // everything staged since the last flush (pieces j_first .. j_end - 1) goes to the lists
     auto flush = [&](uint32_t j_end) {
         if (staged) {
-            uint32_t old_c = 0, old_w = 0;
-            if (lane == 0) old_c = atomicAdd(&st->cand_count, staged);   // room in the candidate list
             if (lane < kBatch) s_tw[lane] = 0;
             __syncwarp();
             uint32_t tw = 0;
 #pragma unroll 1
-            for (uint32_t r0 = 0; r0 < staged; r0 += 32) {         // window: one lane per staged candidate
+            for (uint32_t r0 = 0; r0 < staged; r0 += 32) {         // window entries: how many, and per piece
                 const uint32_t r = r0 + lane;
-                const float a = r < staged ? fabsf(stage_val[r]) : 0.f;
-                const bool isw = r < staged && !(a > thi_f);
-                saw_nan |= a != a;
-                const uint32_t bw = __ballot_sync(0xFFFFFFFFu, isw);
-                if (bw) {
-                    if (isw) {
-                        const uint32_t wr = tw + __popc(bw & lt), pos = stage_pos[r];
-                        if (wr < kDenseWinStage) {
-                            stage_widx[wr] = entry_of(pos);
-                            stage_wkey[wr] = __float_as_uint(a);     // the magnitude key
-                        }
-                        atomicAdd(&s_tw[pos >> 10], 1u);
-                    }
-                    tw += __popc(bw);
+                bool isw = false;
+                if (r < staged) {
+                    const uint2 c = stage[r];
+                    const float a = fabsf(__uint_as_float(c.x));
+                    saw_nan |= a != a;
+                    isw = !(a > thi_f);
+                    if (isw) atomicAdd(&s_tw[((c.y >> 10) - ss0) >> 3], 1u);
                 }
+                tw += __popc(__ballot_sync(0xFFFFFFFFu, isw));
             }
-            if (tw && lane == 0) old_w = atomicAdd(&st->win_count, tw);   // room in the window list
+            uint32_t old_c = 0, old_w = 0;
+            if (lane == 0) {
+                old_c = atomicAdd(&st->cand_count, staged);    // room in the candidate list
+                if (tw) old_w = atomicAdd(&st->win_count, tw); // room in the window list
+            }
             __syncwarp();
             // where each piece's candidates begin
             const bool mine_in = lane >= j_first && lane < j_end;
@@ -517,25 +545,30 @@ __global__ void __launch_bounds__(kThreads, 4) k_bracket_scan_dense(SelectParams
                 const uint32_t y = __shfl_up_sync(0xFFFFFFFFu, inc, d);
                 if (lane >= static_cast<uint32_t>(d)) inc += y;
             }
-            const uint32_t cb = __shfl_sync(0xFFFFFFFFu, old_c, 0);
+            const uint32_t cb = __shfl_sync(0xFFFFFFFFu, old_c, 0), wb = __shfl_sync(0xFFFFFFFFu, old_w, 0);
             if (tcj) sub_tab[ss0 + kStep * lane] = make_uint2(cb + inc - tcj, tcj | ((tcj - twj) << 16));
-            if (tw > kDenseWinStage || static_cast<uint64_t>(cb) + staged > L.cand_cap) {
+            if (static_cast<uint64_t>(cb) + staged > L.cand_cap || static_cast<uint64_t>(wb) + tw > L.win_cap) {
                 lost = true;
             } else {
+                uint32_t wr = wb;
 #pragma unroll 1
-                for (uint32_t r = lane; r < staged; r += 32) {
-                    cand_idx[cb + r] = entry_of(stage_pos[r]);
-                    cand_val[cb + r] = stage_val[r];
-                }
-                const uint32_t wb = __shfl_sync(0xFFFFFFFFu, old_w, 0);
-                if (static_cast<uint64_t>(wb) + tw > L.win_cap) {
-                    lost = true;
-                } else {
-#pragma unroll 1
-                    for (uint32_t r = lane; r < tw; r += 32) {
-                        win_idx[wb + r] = stage_widx[r];
-                        win_key[wb + r] = stage_wkey[r];
+                for (uint32_t r0 = 0; r0 < staged; r0 += 32) {
+                    const uint32_t r = r0 + lane;
+                    bool isw = false;
+                    uint2 c = make_uint2(0u, 0u);
+                    if (r < staged) {
+                        c = stage[r];
+                        cand_idx[cb + r] = c.y;
+                        cand_val[cb + r] = __uint_as_float(c.x);
+                        isw = !(fabsf(__uint_as_float(c.x)) > thi_f);
                     }
+                    const uint32_t bw = __ballot_sync(0xFFFFFFFFu, isw);
+                    if (isw) {
+                        const uint32_t o = wr + __popc(bw & lt);
+                        win_idx[o] = c.y;
+                        win_key[o] = c.x & 0x7FFFFFFFu;          // the magnitude key
+                    }
+                    wr += __popc(bw);
                 }
             }
             __syncwarp();                                     // the stage is reused
@@ -563,14 +596,14 @@ __global__ void __launch_bounds__(kThreads, 4) k_bracket_scan_dense(SelectParams
         // is refilled with the next piece while the second half is still being worked on
         const bool next_inside = (j + 1 < kBatch) && next < ss_end && next >= in_lo && next < in_hi;
         const float4* nptr = vec + (next_inside ? next : ss) * (kSubElems / 4) + lane;
+        const uint32_t e_lane = ss * kSubElems + lane * 4;    // shifted position of the lane's first entry of load 0
         uint32_t tc = 0;
         bool crowded = false;                                  // more candidates than a piece may bring
 #pragma unroll
         for (int h = 0; h < 2; ++h) {
-            uint32_t cnt = 0;                                  // candidates per load of this lane, one byte each
+            if (!inside) {                                     // first / last piece: blank what lies outside (t_lo > 0)
 #pragma unroll
-            for (int i = 4 * h; i < 4 * h + 4; ++i) {
-                if (!inside) {                                 // first / last piece: blank what lies outside (t_lo > 0)
+                for (int i = 4 * h; i < 4 * h + 4; ++i) {
                     float xs[4] = {x[i].x, x[i].y, x[i].z, x[i].w};
                     const uint32_t e0 = (vec0 + i * 32 + lane) * 4;
 #pragma unroll
@@ -578,10 +611,12 @@ __global__ void __launch_bounds__(kThreads, 4) k_bracket_scan_dense(SelectParams
                         if (e0 + q < mis || e0 + q >= n_shift) xs[q] = 0.f;
                     x[i] = make_float4(xs[0], xs[1], xs[2], xs[3]);
                 }
-                const uint32_t n = (!(fabsf(x[i].x) < tlo_f) ? 1u : 0u) + (!(fabsf(x[i].y) < tlo_f) ? 1u : 0u) +
-                                   (!(fabsf(x[i].z) < tlo_f) ? 1u : 0u) + (!(fabsf(x[i].w) < tlo_f) ? 1u : 0u);
-                cnt += n << (8 * (i & 3));
             }
+            uint32_t cnt = 0;                                  // candidates per load of this lane, one byte each
+            dense_count<1u>(x[4 * h], tlo_f, cnt);
+            dense_count<1u << 8>(x[4 * h + 1], tlo_f, cnt);
+            dense_count<1u << 16>(x[4 * h + 2], tlo_f, cnt);
+            dense_count<1u << 24>(x[4 * h + 3], tlo_f, cnt);
             uint32_t inc = cnt;                                // a load holds at most 128 candidates: no byte overflows
 #pragma unroll
             for (int d = 1; d < 32; d <<= 1) {
@@ -596,12 +631,8 @@ __global__ void __launch_bounds__(kThreads, 4) k_bracket_scan_dense(SelectParams
             if (!crowded) {
 #pragma unroll
                 for (int i = 4 * h; i < 4 * h + 4; ++i) {
-                    uint32_t r = load_off + ((pre >> ((i & 3) * 8)) & 255u);
-                    const uint32_t place = j * 1024 + i * 128 + lane * 4;
-                    dense_place(x[i].x, tlo_f, r, pos_base, val_base, place);
-                    dense_place(x[i].y, tlo_f, r, pos_base, val_base, place + 1);
-                    dense_place(x[i].z, tlo_f, r, pos_base, val_base, place + 2);
-                    dense_place(x[i].w, tlo_f, r, pos_base, val_base, place + 3);
+                    uint32_t a = stage_base + 8u * (load_off + ((pre >> ((i & 3) * 8)) & 255u));
+                    dense_place(x[i], tlo_f, a, e_lane + i * 128);
                     load_off += (tot >> ((i & 3) * 8)) & 255u;
                 }
             }
