@@ -266,16 +266,17 @@ ADACOMP_API int adacomp_server_timestamp(const adacomp_server_t* s, uint64_t* h_
  * ascending inside an update.  Off by default. */
 ADACOMP_API int adacomp_server_set_validation(adacomp_server_t* s, int on);
 /* Chooses how adacomp_apply maps work to the GPU; results are identical.
- * 0 = automatic: per launch of up to 32 updates, 3 when the launch's pairs number a fifth of
- *     the parameters or more, else 2; a single update goes as 1;
+ * 0 = automatic: per launch of up to 32 updates, 3 when the launch's pairs number 8 % of the
+ *     parameters or more, else 2; a single update goes as 1;
  * 1 = one launch per update, one thread per pair;
- * 2 = up to 32 sparse updates per launch; a warp owns a run of parameter ranges, lines up all
- *     pairs of a range in arrival order and applies them 32 at a time straight on global memory
- *     (lanes that hold the same parameter take turns); only the named parameters are touched;
+ * 2 = up to 32 updates per launch; a warp owns a run of parameter ranges, lines up all pairs of
+ *     a range in arrival order and applies them 32 at a time straight on global memory (lanes
+ *     that hold the same parameter take turns); only the named parameters are touched;
  * 3 = up to 32 updates per launch over a dense sweep: a warp owns a run of ranges of 128 to 512
  *     parameters (sized to the updates' density), brings Theta and the history heads of a range
- *     into shared memory whole, applies the updates' pairs of the range one update after the
- *     other, and writes back what changed (needs Theta on a 16-byte boundary, else 2 is used).
+ *     into shared memory whole, applies the updates' pairs of the range there (thin updates: all
+ *     lined up in arrival order, 32 at a time; dense updates: one update after the other) and
+ *     writes back what changed (needs Theta on a 16-byte boundary, else 2 is used).
  * 4 = the paper's own history structure ("Complexity" paragraph) instead of the chains: the ring
  *     keeps the sorted index lists of the recent updates and sigma_k is found with one dichotomous
  *     search per update of the window; one launch per update.  Windows are bounded to 448 updates

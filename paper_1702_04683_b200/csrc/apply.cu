@@ -370,20 +370,36 @@ constexpr uint32_t kMgWarps = kMgThreads / 32;
 constexpr uint32_t kMgPitch = 33;              // words per staged update: lanes that probe, and lanes that fill, hit distinct banks
 constexpr uint32_t kMgLow = 10;                // refill a stage with fewer pairs left
 
-__host__ __device__ inline size_t mg_smem_bytes(uint32_t n_updates) {
-    return static_cast<size_t>(kMgWarps) * n_updates * kMgPitch * 8;
+__host__ __device__ inline size_t mg_warp_words(uint32_t range, uint32_t n_updates, bool pre) {
+    return (range ? (pre ? 6 : 5) * static_cast<size_t>(range) : 0) + ((static_cast<size_t>(n_updates) * kMgPitch * 2 + 3) & ~static_cast<size_t>(3));
+}
+__host__ __device__ inline size_t mg_smem_bytes(uint32_t range, uint32_t n_updates, bool pre) {
+    return (range ? 256 : 0) + kMgWarps * mg_warp_words(range, n_updates, pre) * 4;
 }
 
-template <bool kExtra>
+template <uint32_t R, bool kPre, bool kExtra>
 __global__ void __launch_bounds__(kMgThreads)
 k_apply_merged(const ServerParams sp, const BatchDesc d, uint32_t range, const uint32_t* __restrict__ idx,
                const float* __restrict__ val, float lr, uint32_t* sigma_out, uint32_t n_ranges) {
     extern __shared__ __align__(16) unsigned char s_mg[];
+    static_assert(R % 128 == 0, "16-byte pieces, whole warps");
+    constexpr bool kSlices = R != 0;                            // Theta, heads and masks of the range in shared memory
+    if (kSlices) range = R;
     const uint32_t B = d.n_updates;
     const uint32_t lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     const uint32_t lt = (1u << lane) - 1u;
-    uint32_t* s_k = reinterpret_cast<uint32_t*>(s_mg) + warp * B * kMgPitch * 2;   // [B][33] staged indices
+    float* s_alpha = reinterpret_cast<float*>(s_mg);                            // [64] alpha / sigma for the small counts (slices only)
+    uint32_t* mine = reinterpret_cast<uint32_t*>(s_mg) + (kSlices ? 64 : 0) + warp * mg_warp_words(R, B, kPre);
+    float* s_theta = reinterpret_cast<float*>(mine);                            // [2][R] Theta of the range
+    uint32_t* s_head = mine + 2 * R;                                            // [2][R] latest change of the parameter
+    uint32_t* s_mask = s_head + 2 * R;                                          // [R] updates of this launch that changed it
+    uint32_t* s_head0 = s_mask + R;                                             // [R] head when the launch began (kPre)
+    uint32_t* s_k = mine + (kPre ? 6 : 5) * R;                                  // [B][33] staged indices
     float* s_v = reinterpret_cast<float*>(s_k + B * kMgPitch);                  // [B][33] staged values
+    if (kSlices) {
+        if (threadIdx.x < kRgAlphas) s_alpha[threadIdx.x] = threadIdx.x ? __fdiv_rn(lr, static_cast<float>(threadIdx.x)) : lr;   // Eq. 5, once
+        __syncthreads();                                        // the only block barrier
+    }
     const uint32_t gw = blockIdx.x * kMgWarps + warp, n_gw = gridDim.x * kMgWarps;
     const uint32_t r_lo = static_cast<uint32_t>(static_cast<uint64_t>(n_ranges) * gw / n_gw);
     const uint32_t r_hi = static_cast<uint32_t>(static_cast<uint64_t>(n_ranges) * (gw + 1) / n_gw);
@@ -392,6 +408,7 @@ k_apply_merged(const ServerParams sp, const BatchDesc d, uint32_t range, const u
     // lane b's view of update b
     const bool has = lane < B;
     const uint32_t n_b = has ? d.n_pairs[lane] : 0u, pos0_b = has ? d.pos_start[lane] : 0u, ws_b = has ? d.win_start[lane] : 0u;
+    const uint32_t bits_b = has ? d.win_bits[lane] : 0u;
     const uint64_t begin_b = has ? d.pair_begin[lane] : 0ull;
     uint32_t cur = 0, sb = 0;                                   // cursor; cursor of the stage's slot 0
     if (has) cur = first_at_or_above(idx + begin_b, n_b, static_cast<uint64_t>(r_lo) * range, sp.n_params);
@@ -407,16 +424,48 @@ k_apply_merged(const ServerParams sp, const BatchDesc d, uint32_t range, const u
             s_k[b * kMgPitch + lane] = kNone;
         }
     };
+    auto range_end = [&](uint32_t r) -> uint32_t {
+        const uint64_t e = (static_cast<uint64_t>(r) + 1) * range;
+        return e <= sp.n_params ? static_cast<uint32_t>(e) : static_cast<uint32_t>(sp.n_params);
+    };
+    // Theta and heads of range r into buffer p (slices only)
+    auto sweep_in = [&](uint32_t r, uint32_t p) {
+        const uint32_t lo = r * R, hi = range_end(r);
+        if (hi - lo == R) {
+#pragma unroll
+            for (uint32_t o = lane * 4; o < R; o += 128) {
+                copy_async_16(smem_address(s_theta + p * R + o), sp.theta + lo + o);
+                copy_async_16(smem_address(s_head + p * R + o), sp.head + lo + o);
+            }
+        } else {                                                // the last range may be short: plain loads
+            for (uint32_t o = lane; o < R; o += 32) {
+                s_theta[p * R + o] = lo + o < hi ? sp.theta[lo + o] : 0.f;
+                s_head[p * R + o] = lo + o < hi ? sp.head[lo + o] : kNone;
+            }
+        }
+    };
     for (uint32_t b = 0; b < B; ++b) fill(b, __shfl_sync(0xFFFFFFFFu, cur, b));
     sb = cur;
+    if (kSlices) sweep_in(r_lo, 0);
     copy_async_commit();
     copy_async_wait<0>();
     __syncwarp();
 
     for (uint32_t r = r_lo; r < r_hi; ++r) {
-        const uint64_t end64 = (static_cast<uint64_t>(r) + 1) * range;
-        const uint32_t hi = end64 <= sp.n_params ? static_cast<uint32_t>(end64) : static_cast<uint32_t>(sp.n_params);
+        const uint32_t hi = range_end(r);
         const uint32_t lo = r * range;
+        const uint32_t p = (r - r_lo) & 1u;
+        float* th = s_theta + p * R;
+        uint32_t* hd = s_head + p * R;
+        if (kSlices) {
+            if (r + 1 < r_hi) sweep_in(r + 1, p ^ 1u);          // lands while this range is worked on
+#pragma unroll
+            for (uint32_t o = lane * 4; o < R; o += 128) {
+                *reinterpret_cast<uint4*>(s_mask + o) = make_uint4(0, 0, 0, 0);
+                if (kPre) *reinterpret_cast<uint4*>(s_head0 + o) = *reinterpret_cast<const uint4*>(hd + o);
+            }
+            __syncwarp();
+        }
         for (;;) {
             // ---- how many staged pairs of update b lie below the range's end
             const uint32_t c0 = cur - sb;                       // first staged slot not yet applied, 0..32
@@ -465,7 +514,7 @@ k_apply_merged(const ServerParams sp, const BatchDesc d, uint32_t range, const u
             bool refilled = false;
 #pragma unroll 1
             for (uint32_t c = 0; c < total; c += 128) {
-                uint32_t kq[4], posq[4], wsq[4];
+                uint32_t kq[4], posq[4], wsq[4], bq[4], bitsq[4];
                 uint64_t sq[4];                                 // kExtra: where the pair's staleness count goes
                 float vq[4];
 #pragma unroll
@@ -484,6 +533,8 @@ k_apply_merged(const ServerParams sp, const BatchDesc d, uint32_t range, const u
                     const uint32_t at = __shfl_sync(0xFFFFFFFFu, cur, b) + jj;  // its place in the update's list
                     posq[u] = __shfl_sync(0xFFFFFFFFu, pos0_b, b) + at;
                     wsq[u] = __shfl_sync(0xFFFFFFFFu, ws_b, b);
+                    bitsq[u] = kSlices ? __shfl_sync(0xFFFFFFFFu, bits_b, b) : 0u;
+                    bq[u] = b;
                     sq[u] = 0;
                     if (kExtra) {
                         const uint32_t blo = __shfl_sync(0xFFFFFFFFu, static_cast<uint32_t>(begin_b), b);
@@ -495,12 +546,17 @@ k_apply_merged(const ServerParams sp, const BatchDesc d, uint32_t range, const u
                     if (valid) {
                         kq[u] = s_k[b * kMgPitch + slot];
                         vq[u] = s_v[b * kMgPitch + slot];
-                        prefetch_l2(sp.head + kq[u]);           // wanted in a moment, by a load that must see the latest value
-                        prefetch_l2(sp.theta + kq[u]);
-                        if (kq[u] < lo) record_error(sp.status, ADACOMP_ERR_UNSORTED);   // the list was not ascending
+                        if (!kSlices) {
+                            prefetch_l2(sp.head + kq[u]);       // wanted in a moment, by a load that must see the latest value
+                            prefetch_l2(sp.theta + kq[u]);
+                        }
                         if (kExtra && sp.validate && at > 0) {
                             const uint32_t before = slot > 0 ? s_k[b * kMgPitch + slot - 1] : idx[sq[u] - 1];
                             if (before >= kq[u]) record_error(sp.status, ADACOMP_ERR_UNSORTED);
+                        }
+                        if (kq[u] < lo) {                       // the list was not ascending: consumed, not applied
+                            record_error(sp.status, ADACOMP_ERR_UNSORTED);
+                            kq[u] = kNone;
                         }
                     }
                 }
@@ -517,7 +573,28 @@ k_apply_merged(const ServerParams sp, const BatchDesc d, uint32_t range, const u
                     bool waiting = k != kNone;
                     while (pending) {
                         const bool go = waiting && (peers & pending & lt) == 0;
-                        if (go) {
+                        if (go && kSlices) {
+                            const uint32_t kl = k - lo, bit = 1u << bq[u];
+                            const bool change = v != 0.0f;      // Eq. 3 counts changes: a zero entry is not one
+                            const uint32_t m = change ? atomicOr(&s_mask[kl], bit) : s_mask[kl];
+                            uint32_t sigma = __popc(m & bitsq[u]);                                     // Eq. 3, inside the launch
+                            if (kPre && (d.pre_mask & bit)) {                                          // Eq. 3, before the launch
+                                uint32_t q = s_head0[kl], hops = 0;
+                                while (q != kNone && q >= ws) {
+                                    if (++hops > sp.max_window) { record_error(sp.status, ADACOMP_ERR_WINDOW); break; }
+                                    q = sp.prev[(q + sp.ring_shift) & sp.ring_mask];
+                                }
+                                sigma += hops;
+                            }
+                            if (kExtra && sigma_out) sigma_out[sq[u]] = sigma;
+                            if (change) {
+                                const float alpha_k = sigma < kRgAlphas ? s_alpha[sigma] : __fdiv_rn(lr, static_cast<float>(sigma));   // Eq. 5
+                                th[kl] = __fsub_rn(th[kl], __fmul_rn(alpha_k, v));                     // Eq. 4
+                                sp.prev[(pos + sp.ring_shift) & sp.ring_mask] = atomicExch(&hd[kl], pos);
+                            }
+                            waiting = false;
+                        }
+                        if (go && !kSlices) {
                             const uint32_t latest = __ldcg(sp.head + k);
                             const float theta = __ldcg(sp.theta + k);
                             uint32_t q = latest, sigma = 0;                                            // Eq. 3
@@ -549,6 +626,24 @@ k_apply_merged(const ServerParams sp, const BatchDesc d, uint32_t range, const u
             }
             const bool again = dry_mask != 0;
             if (!again) break;
+        }
+        if (kSlices) {                                          // ---- Theta and heads go back where a parameter changed
+            if (hi - lo == R) {
+#pragma unroll
+                for (uint32_t o = lane * 4; o < R; o += 128) {
+                    const uint4 m4 = *reinterpret_cast<const uint4*>(s_mask + o);
+                    if (m4.x | m4.y | m4.z | m4.w) {
+                        *reinterpret_cast<float4*>(sp.theta + lo + o) = *reinterpret_cast<const float4*>(th + o);
+                        *reinterpret_cast<uint4*>(sp.head + lo + o) = *reinterpret_cast<const uint4*>(hd + o);
+                    }
+                }
+            } else {
+                for (uint32_t o = lane; o < R; o += 32)
+                    if (lo + o < hi && s_mask[o]) { sp.theta[lo + o] = th[o]; sp.head[lo + o] = hd[o]; }
+            }
+            copy_async_commit();                                // the next range's Theta and heads
+            copy_async_wait<0>();
+            __syncwarp();
         }
     }
     // whoever owns the last range sees what no range claimed: indices >= n_params
@@ -724,36 +819,45 @@ int launch_apply_warps(const adacomp_server_t* s, const ServerParams& sp, const 
                  : launch_apply_warps_as<R, false, false>(s, sp, d, d_idx, d_val, lr, d_sigma_out, st);
 }
 
-// Launches k_apply_merged with ranges sized so that a range holds about 128 pairs of the launch.
-int launch_apply_merged(const adacomp_server_t* s, const ServerParams& sp, const BatchDesc& d, uint64_t pairs,
-                        const uint32_t* d_idx, const float* d_val, float lr, uint32_t* d_sigma_out, cudaStream_t st) {
-    const bool extra = d_sigma_out != nullptr || sp.validate != 0;
-    const size_t smem = mg_smem_bytes(d.n_updates);
+// Launches k_apply_merged<R, kPre, kExtra>.  R = 0: only the named parameters are touched, ranges sized so that
+// one holds about 128 pairs of the launch; R > 0: ranges of R parameters, swept through shared memory.
+template <uint32_t R, bool kPre, bool kExtra>
+int launch_apply_merged_as(const adacomp_server_t* s, const ServerParams& sp, const BatchDesc& d, uint64_t pairs,
+                           const uint32_t* d_idx, const float* d_val, float lr, uint32_t* d_sigma_out, cudaStream_t st) {
+    const size_t smem = mg_smem_bytes(R, d.n_updates, kPre);
+    ADACOMP_CUDA(cudaFuncSetAttribute(k_apply_merged<R, kPre, kExtra>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                      static_cast<int>(mg_smem_bytes(R, kMaxBatch, kPre))));
     int per_sm = 1;
-    if (extra) {
-        ADACOMP_CUDA(cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, k_apply_merged<true>, kMgThreads, smem));
-    } else {
-        ADACOMP_CUDA(cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, k_apply_merged<false>, kMgThreads, smem));
-    }
+    ADACOMP_CUDA(cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, k_apply_merged<R, kPre, kExtra>, kMgThreads, smem));
     const uint64_t warps = static_cast<uint64_t>(s->n_sms) * static_cast<uint64_t>(per_sm > 0 ? per_sm : 1) * kMgWarps;
-    // a range should hold about 128 pairs (at most ~8 per update, so that a stage of 32 lasts), and every warp
-    // should get several ranges
-    double want = 128.0 * static_cast<double>(s->n_params) / static_cast<double>(pairs);
-    const double balance = static_cast<double>(s->n_params) / (2.0 * static_cast<double>(warps));
-    if (want > balance) want = balance;
-    uint64_t range = want < 32.0 ? 32 : static_cast<uint64_t>(want) / 32 * 32;
-    if (range > (1u << 30)) range = 1u << 30;
-    const uint64_t n_ranges64 = (s->n_params + range - 1) / range;
-    const uint32_t n_ranges = static_cast<uint32_t>(n_ranges64);
+    uint64_t range = R;
+    if (R == 0) {
+        // a range should hold about 128 pairs (some 8 per update, so that a stage of 32 lasts a few ranges), and
+        // every warp should get at least two ranges
+        double want = 128.0 * static_cast<double>(s->n_params) / static_cast<double>(pairs);
+        const double balance = static_cast<double>(s->n_params) / (2.0 * static_cast<double>(warps));
+        if (want > balance) want = balance;
+        range = want < 32.0 ? 32 : static_cast<uint64_t>(want) / 32 * 32;
+        if (range > (1u << 30)) range = 1u << 30;
+    }
+    const uint64_t n_ranges = (s->n_params + range - 1) / range;
     uint64_t grid = warps / kMgWarps;
-    const uint64_t most_blocks = (n_ranges64 + kMgWarps - 1) / kMgWarps;
+    const uint64_t most_blocks = (n_ranges + kMgWarps - 1) / kMgWarps;
     if (grid > most_blocks) grid = most_blocks;
-    if (extra)
-        k_apply_merged<true><<<static_cast<unsigned>(grid), kMgThreads, smem, st>>>(sp, d, static_cast<uint32_t>(range), d_idx, d_val, lr, d_sigma_out, n_ranges);
-    else
-        k_apply_merged<false><<<static_cast<unsigned>(grid), kMgThreads, smem, st>>>(sp, d, static_cast<uint32_t>(range), d_idx, d_val, lr, d_sigma_out, n_ranges);
+    k_apply_merged<R, kPre, kExtra><<<static_cast<unsigned>(grid), kMgThreads, smem, st>>>(
+        sp, d, static_cast<uint32_t>(range), d_idx, d_val, lr, d_sigma_out, static_cast<uint32_t>(n_ranges));
     ADACOMP_LAUNCH_CHECK();
     return ADACOMP_OK;
+}
+
+template <uint32_t R>
+int launch_apply_merged(const adacomp_server_t* s, const ServerParams& sp, const BatchDesc& d, uint64_t pairs,
+                        const uint32_t* d_idx, const float* d_val, float lr, uint32_t* d_sigma_out, cudaStream_t st) {
+    const bool pre = R != 0 && d.pre_mask != 0, extra = d_sigma_out != nullptr || sp.validate != 0;
+    if (pre) return extra ? launch_apply_merged_as<R, R != 0, true>(s, sp, d, pairs, d_idx, d_val, lr, d_sigma_out, st)
+                          : launch_apply_merged_as<R, R != 0, false>(s, sp, d, pairs, d_idx, d_val, lr, d_sigma_out, st);
+    return extra ? launch_apply_merged_as<R, false, true>(s, sp, d, pairs, d_idx, d_val, lr, d_sigma_out, st)
+                 : launch_apply_merged_as<R, false, false>(s, sp, d, pairs, d_idx, d_val, lr, d_sigma_out, st);
 }
 
 bool sizes_ok(uint64_t n_params, uint64_t history_pairs) {
@@ -962,10 +1066,10 @@ int adacomp_apply(adacomp_server_t* s, const uint32_t* d_idx, const float* d_val
     sp.validate = s->validate;
 
     // ---- launches.  One launch per update, or launches of up to kMaxBatch updates each: same results.
-    // Automatic choice per launch: the warp-per-range kernel over a dense sweep of Theta when the launch's pairs
-    // number a fifth of the parameters or more (nearly every 32-byte sector of Theta is touched anyway), else the
-    // kernel that touches only the named parameters; a single update, and updates whose staleness slots overlap in
-    // memory, go one per launch.
+    // Automatic choice per launch: a dense sweep of Theta through shared memory when the launch's pairs number
+    // 8 % of the parameters or more (most 32-byte sectors of Theta are touched anyway), else the kernel that
+    // touches only the named parameters; a single update, and updates whose staleness slots overlap in memory, go
+    // one per launch.
     bool shared_slots = false;                 // two updates write their counts to the same slots: order matters
     if (d_sigma_out && n_updates > 1 && s->mode != 1) {
         std::vector<std::pair<uint64_t, uint64_t>> slices;
@@ -1002,9 +1106,14 @@ int adacomp_apply(adacomp_server_t* s, const uint32_t* d_idx, const float* d_val
         if (!pairs) continue;
         const double dens = static_cast<double>(most) / static_cast<double>(s->n_params);   // of the densest update
         const bool sweep = theta_aligned &&
-                           (s->mode == 3 || (s->mode == 0 && static_cast<double>(pairs) >= 0.2 * static_cast<double>(s->n_params)));
+                           (s->mode == 3 || (s->mode == 0 && static_cast<double>(pairs) >= 0.08 * static_cast<double>(s->n_params)));
         int rc;
-        if (sweep) {
+        if (sweep && dens * 256.0 <= 5.0) {
+            // thin updates (a handful of pairs per update and range): all updates' pairs of a range lined up and
+            // applied 32 at a time against the range's slices in shared memory
+            if (dens * 512.0 <= 4.0) rc = launch_apply_merged<512>(s, sp, d, pairs, d_idx, d_val, lr, d_sigma_out, st);
+            else rc = launch_apply_merged<256>(s, sp, d, pairs, d_idx, d_val, lr, d_sigma_out, st);
+        } else if (sweep) {
             // range size: the densest update should bring about 26 pairs per range (mean of a uniformly spread
             // update), so that one load of 32 pairs per update and range is usually all of them
             const double want = 26.0 / dens;
@@ -1014,7 +1123,7 @@ int adacomp_apply(adacomp_server_t* s, const uint32_t* d_idx, const float* d_val
             else if (want >= 192.0) rc = launch_apply_warps<192>(s, sp, d, d_idx, d_val, lr, d_sigma_out, st);
             else rc = launch_apply_warps<128>(s, sp, d, d_idx, d_val, lr, d_sigma_out, st);
         } else {
-            rc = launch_apply_merged(s, sp, d, pairs, d_idx, d_val, lr, d_sigma_out, st);
+            rc = launch_apply_merged<0>(s, sp, d, pairs, d_idx, d_val, lr, d_sigma_out, st);
         }
         if (rc != ADACOMP_OK) return rc;
     }

@@ -235,7 +235,7 @@ def test_parameters_on_an_odd_address_and_odd_count(binding, mode):
 
 
 @pytest.mark.parametrize("mode", MODES)
-@pytest.mark.parametrize("density", [0.002, 0.03, 0.12, 0.3])
+@pytest.mark.parametrize("density", [0.002, 0.012, 0.03, 0.12, 0.3])
 def test_forty_updates_without_staleness_counts(binding, mode, density):
     """More updates per call than one launch takes (32), windows that reach back before the call,
     no staleness output asked for (the kernels' plain variants): parameters bit for bit."""
