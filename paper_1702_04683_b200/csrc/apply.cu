@@ -96,6 +96,34 @@ struct BatchDesc {
 
 constexpr uint32_t kRgAlphas = 33;             // alpha / sigma kept ready for sigma < 33
 
+// First position of an ascending index list whose entry is >= target.  The lists of an update are spread
+// over [0, n_params) more or less evenly, so a few interpolation steps narrow the search before the
+// bisection that finishes it: far fewer dependent loads than bisection alone on a long list.
+__device__ __forceinline__ uint32_t first_at_or_above(const uint32_t* __restrict__ list, uint32_t n, uint64_t target,
+                                                      uint64_t n_params) {
+    uint32_t lo = 0, hi = n;                                    // answer in [lo, hi]
+    uint64_t v_lo = 0, v_hi = n_params;                         // list[lo - 1] < target <= list[hi], bounds on those values
+#pragma unroll 1
+    for (int step = 0; step < 4 && hi - lo > 64; ++step) {
+        if (target <= v_lo || target >= v_hi) break;
+        const uint64_t span = hi - lo;
+        uint64_t guess = lo + (target - v_lo) * span / (v_hi - v_lo);
+        // two probes a little either side of the guess: both outcomes shrink the range a lot
+        const uint64_t slack = 8 + (span >> 7);
+        const uint32_t p0 = static_cast<uint32_t>(guess > lo + slack ? guess - slack : lo);
+        const uint32_t p1 = static_cast<uint32_t>(guess + slack < hi - 1 ? guess + slack : hi - 1);
+        const uint32_t x0 = list[p0], x1 = list[p1];
+        if (x0 >= target) { hi = p0; v_hi = x0; }
+        else if (x1 < target) { lo = p1 + 1; v_lo = x1; }
+        else { lo = p0 + 1; v_lo = x0; hi = p1; v_hi = x1; }
+    }
+    while (lo < hi) {
+        const uint32_t mid = lo + ((hi - lo) >> 1);
+        if (list[mid] < target) lo = mid + 1; else hi = mid;
+    }
+    return lo;
+}
+
 // ---------------------------------------------------------------------------------------------
 // Several updates per launch, one WARP per range of parameters, no block barrier in the loop.  A
 // warp owns a run of ranges of R consecutive parameters and a slice of shared memory: Theta and
@@ -200,16 +228,8 @@ k_apply_warps(const ServerParams sp, const BatchDesc d, const uint32_t* __restri
         }
     };
 
-    if (lane < B) {
-        const uint64_t first_param = static_cast<uint64_t>(r_lo) * R;
-        const uint32_t* list = idx + d.pair_begin[lane];
-        uint32_t lo = 0, hi = d.n_pairs[lane];                 // cursor: first pair at or above the first owned parameter
-        while (lo < hi) {
-            const uint32_t mid = lo + ((hi - lo) >> 1);
-            if (list[mid] < first_param) lo = mid + 1; else hi = mid;
-        }
-        s_cur[lane] = lo;
-    }
+    if (lane < B)                                               // cursor: first pair at or above the first owned parameter
+        s_cur[lane] = first_at_or_above(idx + d.pair_begin[lane], d.n_pairs[lane], static_cast<uint64_t>(r_lo) * R, sp.n_params);
     __syncwarp();
     for (uint32_t b = 0; b < B; ++b) refill(b, s_cur[b]);
     sweep_in(r_lo, 0);
@@ -322,49 +342,27 @@ k_apply_warps(const ServerParams sp, const BatchDesc d, const uint32_t* __restri
     if (r_hi == n_ranges && lane < B && s_cur[lane] < d.n_pairs[lane]) record_error(sp.status, ADACOMP_ERR_UNSORTED);
 }
 
-// First position of an ascending index list whose entry is >= target.  The lists of an update are spread
-// over [0, n_params) more or less evenly, so a few interpolation steps narrow the search before the
-// bisection that finishes it: far fewer dependent loads than bisection alone on a long list.
-__device__ __forceinline__ uint32_t first_at_or_above(const uint32_t* __restrict__ list, uint32_t n, uint64_t target,
-                                                      uint64_t n_params) {
-    uint32_t lo = 0, hi = n;                                    // answer in [lo, hi]
-    uint64_t v_lo = 0, v_hi = n_params;                         // list[lo - 1] < target <= list[hi], bounds on those values
-#pragma unroll 1
-    for (int step = 0; step < 4 && hi - lo > 64; ++step) {
-        if (target <= v_lo || target >= v_hi) break;
-        const uint64_t span = hi - lo;
-        uint64_t guess = lo + (target - v_lo) * span / (v_hi - v_lo);
-        // two probes a little either side of the guess: both outcomes shrink the range a lot
-        const uint64_t slack = 8 + (span >> 7);
-        const uint32_t p0 = static_cast<uint32_t>(guess > lo + slack ? guess - slack : lo);
-        const uint32_t p1 = static_cast<uint32_t>(guess + slack < hi - 1 ? guess + slack : hi - 1);
-        const uint32_t x0 = list[p0], x1 = list[p1];
-        if (x0 >= target) { hi = p0; v_hi = x0; }
-        else if (x1 < target) { lo = p1 + 1; v_lo = x1; }
-        else { lo = p0 + 1; v_lo = x0; hi = p1; v_hi = x1; }
-    }
-    while (lo < hi) {
-        const uint32_t mid = lo + ((hi - lo) >> 1);
-        if (list[mid] < target) lo = mid + 1; else hi = mid;
-    }
-    return lo;
-}
-
 // ---------------------------------------------------------------------------------------------
-// Several sparse updates per launch, one WARP per range of parameters, no block barrier, nothing
-// swept: only the parameters that are named are touched.  A warp owns a run of ranges and keeps,
-// per update, a stage with the update's next 32 pairs from its cursor (lane b looks after update
-// b).  Per range: lane b counts the staged pairs of update b below the range's end (a bisection:
-// the list is ascending); a warp scan lines all of them up in arrival order (update after update);
-// then they are applied 32 at a time, one pair per lane, straight on global memory and exactly as
-// Algorithm 2 states it: Eq. 3 is the walk along the parameter's chain while it stays inside the
-// window (pairs of this launch applied earlier are on the chain already), Eq. 5, Eq. 4, and the
-// pair becomes the head.  Pairs of one update name distinct parameters; two lanes that hold the
-// same parameter (different updates) are found with a match and take turns in arrival order.
-// Loads of Theta, heads and links go to L2 (no L1 line survives a change by another lane), and a
-// warp-level barrier orders one group of 32 before the next.  A stage that runs low is refilled
-// from the update's new cursor; one that ran dry inside the range is refilled at once and the
-// range is looked at again (later updates wait until that update is through with the range).  Same results, bit for bit, as one launch per update.
+// Several thin updates per launch, one WARP per range of parameters, no block barrier in the loop.
+// A warp owns a run of ranges and keeps, per update, a stage with the update's next 32 pairs from
+// its cursor (lane b looks after update b).  Per range: lane b counts the staged pairs of update b
+// below the range's end (a bisection: the list is ascending); a warp scan lines all of them up in
+// arrival order (update after update); then they are applied 32 at a time, one pair per lane,
+// exactly as Algorithm 2 states it.  Pairs of one update name distinct parameters; two lanes that
+// hold the same parameter (different updates) are found with a match and take turns in arrival
+// order, a warp-level barrier between turns.  A stage that runs low is refilled from the update's
+// new cursor while the pairs are worked on; one that ran dry inside the range is refilled at once
+// and the range is looked at again (later updates wait until that update is through with it).
+// Same results, bit for bit, as one launch per update.  Two forms:
+//   R = 0   nothing is swept, only the parameters that are named are touched, straight on global
+//           memory: Eq. 3 is the walk along the parameter's chain while it stays inside the window
+//           (pairs of this launch applied earlier are on the chain already), Eq. 5, Eq. 4, and the
+//           pair becomes the head.  Loads of Theta, heads and links go to L2 (no L1 line survives
+//           a change by another lane).  The host sizes the ranges to about 128 pairs.
+//   R > 0   ranges of R parameters whose Theta, heads and change masks live in the warp's shared
+//           memory, as in k_apply_warps (asynchronous copies a range ahead, Eq. 3 inside the launch
+//           from the mask, written back where changed): for launches that touch most 32-byte
+//           sectors of Theta anyway with updates too thin to fill a warp one at a time.
 constexpr int kMgThreads = 128;
 constexpr uint32_t kMgWarps = kMgThreads / 32;
 constexpr uint32_t kMgPitch = 33;              // words per staged update: lanes that probe, and lanes that fill, hit distinct banks
@@ -384,7 +382,7 @@ k_apply_merged(const ServerParams sp, const BatchDesc d, uint32_t range, const u
     extern __shared__ __align__(16) unsigned char s_mg[];
     static_assert(R % 128 == 0, "16-byte pieces, whole warps");
     constexpr bool kSlices = R != 0;                            // Theta, heads and masks of the range in shared memory
-    if (kSlices) range = R;
+    if constexpr (kSlices) range = R;
     const uint32_t B = d.n_updates;
     const uint32_t lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     const uint32_t lt = (1u << lane) - 1u;
@@ -396,7 +394,7 @@ k_apply_merged(const ServerParams sp, const BatchDesc d, uint32_t range, const u
     uint32_t* s_head0 = s_mask + R;                                             // [R] head when the launch began (kPre)
     uint32_t* s_k = mine + (kPre ? 6 : 5) * R;                                  // [B][33] staged indices
     float* s_v = reinterpret_cast<float*>(s_k + B * kMgPitch);                  // [B][33] staged values
-    if (kSlices) {
+    if constexpr (kSlices) {
         if (threadIdx.x < kRgAlphas) s_alpha[threadIdx.x] = threadIdx.x ? __fdiv_rn(lr, static_cast<float>(threadIdx.x)) : lr;   // Eq. 5, once
         __syncthreads();                                        // the only block barrier
     }
@@ -430,23 +428,25 @@ k_apply_merged(const ServerParams sp, const BatchDesc d, uint32_t range, const u
     };
     // Theta and heads of range r into buffer p (slices only)
     auto sweep_in = [&](uint32_t r, uint32_t p) {
-        const uint32_t lo = r * R, hi = range_end(r);
-        if (hi - lo == R) {
+        if constexpr (kSlices) {
+            const uint32_t lo = r * R, hi = range_end(r);
+            if (hi - lo == R) {
 #pragma unroll
-            for (uint32_t o = lane * 4; o < R; o += 128) {
-                copy_async_16(smem_address(s_theta + p * R + o), sp.theta + lo + o);
-                copy_async_16(smem_address(s_head + p * R + o), sp.head + lo + o);
-            }
-        } else {                                                // the last range may be short: plain loads
-            for (uint32_t o = lane; o < R; o += 32) {
-                s_theta[p * R + o] = lo + o < hi ? sp.theta[lo + o] : 0.f;
-                s_head[p * R + o] = lo + o < hi ? sp.head[lo + o] : kNone;
+                for (uint32_t o = lane * 4; o < R; o += 128) {
+                    copy_async_16(smem_address(s_theta + p * R + o), sp.theta + lo + o);
+                    copy_async_16(smem_address(s_head + p * R + o), sp.head + lo + o);
+                }
+            } else {                                            // the last range may be short: plain loads
+                for (uint32_t o = lane; o < R; o += 32) {
+                    s_theta[p * R + o] = lo + o < hi ? sp.theta[lo + o] : 0.f;
+                    s_head[p * R + o] = lo + o < hi ? sp.head[lo + o] : kNone;
+                }
             }
         }
     };
     for (uint32_t b = 0; b < B; ++b) fill(b, __shfl_sync(0xFFFFFFFFu, cur, b));
     sb = cur;
-    if (kSlices) sweep_in(r_lo, 0);
+    if constexpr (kSlices) sweep_in(r_lo, 0);
     copy_async_commit();
     copy_async_wait<0>();
     __syncwarp();
@@ -457,7 +457,7 @@ k_apply_merged(const ServerParams sp, const BatchDesc d, uint32_t range, const u
         const uint32_t p = (r - r_lo) & 1u;
         float* th = s_theta + p * R;
         uint32_t* hd = s_head + p * R;
-        if (kSlices) {
+        if constexpr (kSlices) {
             if (r + 1 < r_hi) sweep_in(r + 1, p ^ 1u);          // lands while this range is worked on
 #pragma unroll
             for (uint32_t o = lane * 4; o < R; o += 128) {
@@ -627,7 +627,7 @@ k_apply_merged(const ServerParams sp, const BatchDesc d, uint32_t range, const u
             const bool again = dry_mask != 0;
             if (!again) break;
         }
-        if (kSlices) {                                          // ---- Theta and heads go back where a parameter changed
+        if constexpr (kSlices) {                                // ---- Theta and heads go back where a parameter changed
             if (hi - lo == R) {
 #pragma unroll
                 for (uint32_t o = lane * 4; o < R; o += 128) {
