@@ -37,8 +37,8 @@ FALLBACK_HBM_GBS = 6650.0
 # profiles/dram_traffic_large_flat_w4.md: workload 4 with 4 workers, MB per keep fraction (1/25 and
 # 1/10 are the dense scan kernel).  A launch over W workers moves W / 4 times as much.  Only valid while
 # the kernel source is the one that was profiled.
-SCAN_TRAFFIC_W4_MB = {"1/1000": 1647.3, "1/400": 1685.3, "1/160": 1798.1, "1/64": 1791.7, "1/25": 1789.3, "1/10": 2007.4}
-SCAN_SOURCE_SHA256_16 = "357943fb5ed13c1e"
+SCAN_TRAFFIC_W4_MB = {"1/1000": 1645.7, "1/400": 1684.6, "1/160": 1795.8, "1/64": 1793.4, "1/25": 1788.9, "1/10": 2008.2}
+SCAN_SOURCE_SHA256_16 = "75377b76aac8d2eb"
 
 
 def scan_traffic_bytes(workload_index, keeps, workers):
