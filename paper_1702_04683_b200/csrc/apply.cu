@@ -560,6 +560,27 @@ k_apply_merged(const ServerParams sp, const BatchDesc d, uint32_t range, const u
                         }
                     }
                 }
+                // Eq. 3 before the launch: the walk from the head the parameter had when the launch began does not
+                // depend on the order inside the launch, so the walks of a lane's four pairs run side by side here
+                uint32_t hops[4] = {0u, 0u, 0u, 0u};
+                if (kSlices && kPre) {
+                    uint32_t q[4];
+#pragma unroll
+                    for (uint32_t u = 0; u < 4; ++u)
+                        q[u] = (kq[u] != kNone && ((d.pre_mask >> bq[u]) & 1u)) ? s_head0[kq[u] - lo] : kNone;
+                    bool walking = true;
+                    while (walking) {
+                        walking = false;
+#pragma unroll
+                        for (uint32_t u = 0; u < 4; ++u) {
+                            if (q[u] != kNone && q[u] >= wsq[u]) {
+                                if (++hops[u] > sp.max_window) { record_error(sp.status, ADACOMP_ERR_WINDOW); q[u] = kNone; }
+                                else q[u] = sp.prev[(q[u] + sp.ring_shift) & sp.ring_mask];
+                                walking = true;
+                            }
+                        }
+                    }
+                }
                 if (early && low_mask) { refill(); refilled = true; }
 #pragma unroll
                 for (uint32_t u = 0; u < 4; ++u) {
@@ -578,14 +599,7 @@ k_apply_merged(const ServerParams sp, const BatchDesc d, uint32_t range, const u
                             const bool change = v != 0.0f;      // Eq. 3 counts changes: a zero entry is not one
                             const uint32_t m = change ? atomicOr(&s_mask[kl], bit) : s_mask[kl];
                             uint32_t sigma = __popc(m & bitsq[u]);                                     // Eq. 3, inside the launch
-                            if (kPre && (d.pre_mask & bit)) {                                          // Eq. 3, before the launch
-                                uint32_t q = s_head0[kl], hops = 0;
-                                while (q != kNone && q >= ws) {
-                                    if (++hops > sp.max_window) { record_error(sp.status, ADACOMP_ERR_WINDOW); break; }
-                                    q = sp.prev[(q + sp.ring_shift) & sp.ring_mask];
-                                }
-                                sigma += hops;
-                            }
+                            if (kPre) sigma += hops[u];                                                // Eq. 3, before the launch
                             if (kExtra && sigma_out) sigma_out[sq[u]] = sigma;
                             if (change) {
                                 const float alpha_k = sigma < kRgAlphas ? s_alpha[sigma] : __fdiv_rn(lr, static_cast<float>(sigma));   // Eq. 5
