@@ -375,7 +375,7 @@ class Server:
         _check(_lib.adacomp_server_set_validation(self._h, int(on)), "adacomp_server_set_validation")
 
     def set_mode(self, mode: int):
-        """0 automatic, 1 one launch per update, 2 batches by parameter ranges, 3 batches over a dense sweep,
+        """0 automatic, 1 one launch per update, 2 batches that touch only the named parameters, 3 batches over a dense sweep,
         4 the paper's sorted lists with one search per update of the window (only switchable at timestamp 0)."""
         _check(_lib.adacomp_server_set_mode(self._h, int(mode)), "adacomp_server_set_mode")
 
