@@ -149,7 +149,7 @@ constexpr uint32_t kWpWarps = kWpThreads / 32;
 constexpr uint32_t kWpGroups = 4;              // groups of asynchronous copies per range
 
 __host__ __device__ inline size_t wp_warp_words(uint32_t range, uint32_t n_updates, bool pre) {
-    return 32 + 64 * static_cast<size_t>(n_updates) + (pre ? 6 : 5) * static_cast<size_t>(range);
+    return 32 + (pre ? 96 : 64) * static_cast<size_t>(n_updates) + (pre ? 6 : 5) * static_cast<size_t>(range);
 }
 __host__ __device__ inline size_t wp_smem_bytes(uint32_t range, uint32_t n_updates, bool pre) {
     return 64 * 4 + kWpWarps * wp_warp_words(range, n_updates, pre) * 4;
@@ -183,6 +183,7 @@ k_apply_warps(const ServerParams sp, const BatchDesc d, const uint32_t* __restri
     uint32_t* s_head = reinterpret_cast<uint32_t*>(s_theta) + 2 * R;            // [2][R] latest change of the parameter
     uint32_t* s_mask = s_head + 2 * R;                                          // [R] updates of this launch that changed it
     uint32_t* s_head0 = s_mask + R;                                             // [R] head when the launch began (kPre)
+    uint32_t* s_hops = s_head0 + R;                                             // [B][32] chain entries inside the window before the launch (kPre)
 
     if (tid < kRgAlphas) s_alpha[tid] = tid ? __fdiv_rn(lr, static_cast<float>(tid)) : lr;   // Eq. 5 for the small counts, once
     __syncthreads();                                            // the only block barrier
@@ -256,8 +257,47 @@ k_apply_warps(const ServerParams sp, const BatchDesc d, const uint32_t* __restri
                     *reinterpret_cast<uint4*>(s_head0 + o) = *reinterpret_cast<const uint4*>(hd + o);
                 __syncwarp();
             }
-            // which updates of the group have a pair in this range: lane t looks at the first staged index of update g * per_group + t
             const uint32_t b_first = g * per_group;
+            if (kPre) {
+                // Eq. 3 before the launch for the staged pairs of the group's updates: the walk from the head the
+                // parameter had when the launch began does not depend on the order inside the launch, so four
+                // updates' walks run side by side here instead of one after the other in the loop below
+                const uint32_t b_last = b_first + per_group < B ? b_first + per_group : B;
+#pragma unroll 1
+                for (uint32_t b0 = b_first; b0 < b_last; b0 += 4) {
+                    uint32_t q[4], ws[4], hp[4];
+#pragma unroll
+                    for (uint32_t u = 0; u < 4; ++u) {
+                        q[u] = kNone;
+                        ws[u] = 0;
+                        hp[u] = 0;
+                        if (b0 + u < b_last && ((d.pre_mask >> (b0 + u)) & 1u)) {
+                            const uint32_t k = s_k[(b0 + u) * 32 + lane];
+                            if (k >= lo && k < hi) {
+                                q[u] = s_head0[k - lo];
+                                ws[u] = d.win_start[b0 + u];
+                            }
+                        }
+                    }
+                    bool walking = true;
+                    while (walking) {
+                        walking = false;
+#pragma unroll
+                        for (uint32_t u = 0; u < 4; ++u) {
+                            if (q[u] != kNone && q[u] >= ws[u]) {
+                                if (++hp[u] > sp.max_window) { record_error(sp.status, ADACOMP_ERR_WINDOW); q[u] = kNone; }
+                                else q[u] = sp.prev[(q[u] + sp.ring_shift) & sp.ring_mask];
+                                walking = true;
+                            }
+                        }
+                    }
+#pragma unroll
+                    for (uint32_t u = 0; u < 4; ++u)
+                        if (b0 + u < b_last) s_hops[(b0 + u) * 32 + lane] = hp[u];
+                }
+                __syncwarp();
+            }
+            // which updates of the group have a pair in this range: lane t looks at the first staged index of update g * per_group + t
             uint32_t first_k = kNone;
             if (lane < per_group && b_first + lane < B) first_k = s_k[(b_first + lane) * 32];
             uint32_t live = __ballot_sync(0xFFFFFFFFu, first_k < hi);
@@ -270,6 +310,7 @@ k_apply_warps(const ServerParams sp, const BatchDesc d, const uint32_t* __restri
                 uint32_t cur = s_cur[b];
                 const uint32_t bits_b = d.win_bits[b], bit_b = 1u << b, pos_l = d.pos_start[b] + lane;
                 uint32_t bal = __ballot_sync(0xFFFFFFFFu, k < hi);
+                bool staged = true;                             // these 32 pairs come from the stage: their walks are done
                 for (;;) {
                     if (kExtra && sp.validate) {
                         uint32_t before = __shfl_up_sync(0xFFFFFFFFu, k, 1);
@@ -283,13 +324,17 @@ k_apply_warps(const ServerParams sp, const BatchDesc d, const uint32_t* __restri
                             const uint32_t m = change ? atomicOr(&s_mask[kl], bit_b) : s_mask[kl];
                             uint32_t sigma = __popc(m & bits_b);                                       // Eq. 3, inside the launch
                             if (kPre && (d.pre_mask & bit_b)) {                                        // Eq. 3, before the launch
-                                const uint32_t ws = d.win_start[b];
-                                uint32_t q = s_head0[kl], hops = 0;
-                                while (q != kNone && q >= ws) {
-                                    if (++hops > sp.max_window) { record_error(sp.status, ADACOMP_ERR_WINDOW); break; }
-                                    q = sp.prev[(q + sp.ring_shift) & sp.ring_mask];
+                                if (staged) {
+                                    sigma += s_hops[b * 32 + lane];
+                                } else {
+                                    const uint32_t ws = d.win_start[b];
+                                    uint32_t q = s_head0[kl], hops = 0;
+                                    while (q != kNone && q >= ws) {
+                                        if (++hops > sp.max_window) { record_error(sp.status, ADACOMP_ERR_WINDOW); break; }
+                                        q = sp.prev[(q + sp.ring_shift) & sp.ring_mask];
+                                    }
+                                    sigma += hops;
                                 }
-                                sigma += hops;
                             }
                             if (kExtra && sigma_out) sigma_out[d.pair_begin[b] + cur + lane] = sigma;
                             if (change) {
@@ -307,6 +352,7 @@ k_apply_warps(const ServerParams sp, const BatchDesc d, const uint32_t* __restri
                     cur += cnt;
                     if (cnt < 32) break;
                     const uint32_t t = cur + lane;              // the update may have more pairs in this range
+                    staged = false;
                     k = kNone;
                     if (t < d.n_pairs[b]) {
                         k = idx[d.pair_begin[b] + t];
