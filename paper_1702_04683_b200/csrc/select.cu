@@ -22,6 +22,7 @@ struct adacomp_select {
     int n_sms = 0;
     int route = 0;         // 0 = automatic, 1 = general route for everything
     bool all_bracketed = false;   // every tensor with k > 0 is eligible for the bracketed route
+    bool any_small = false;       // some tensor is selected whole in shared memory by the sample kernel
     uint32_t n_layers = 0, max_workers = 0, slots_per_worker = 0, n_items = 0, n_items_sparse = 0, max_sample = 0;
     uint64_t extent = 0;   // one past the last entry any segment covers
     uint64_t K = 0;        // pairs per worker
@@ -62,6 +63,7 @@ struct Layout {
     uint64_t extent = 0, K = 0;
     uint64_t cand_stride = 0, win_stride = 0, span_stride = 0;
     uint32_t slots_per_worker = 0, max_sample = 0, n_items_sparse = 0;
+    bool any_small = false;            // some tensor is selected whole in shared memory by the sample kernel
 };
 
 // Decides whether a tensor takes the bracketed route and how much room its lists get.  The
@@ -71,7 +73,13 @@ void plan_bracket(Layer& L, Layout* out) {
     L.bracket = 0;
     L.sample = L.n_spans = L.span_base = L.cand_cap = L.win_cap = 0;
     L.cand_base = L.win_base = 0;
-    if (L.n < kBracketMinN || L.n > kBracketMaxN || L.k == 0 || static_cast<uint64_t>(L.k) * 4 > L.n) return;
+    if (L.n < kBracketMinN || L.n > kBracketMaxN || L.k == 0 || static_cast<uint64_t>(L.k) * 4 > L.n) {
+        if (L.k > 0 && L.n <= kSampleMax) {                    // small enough for the keys to sit in shared memory whole
+            L.bracket = kRouteSmall;
+            if (L.n > out->max_sample) out->max_sample = L.n;
+        }
+        return;
+    }
     const uint32_t n_spans = static_cast<uint32_t>((static_cast<uint64_t>(L.n) + 3 + kSpanElems - 1) / kSpanElems);
     uint32_t m = L.n / 8;
     if (m > kSampleMax) m = kSampleMax;
@@ -124,6 +132,7 @@ int build_layout(const adacomp_segment_t* segs, uint32_t n_segs, uint32_t max_wo
         K += s.k;
         end_prev = s.offset + s.n;
         plan_bracket(L, out);
+        if (L.bracket == kRouteSmall) out->any_small = true;
         for (uint32_t s0 = 0; L.bracket && s0 < L.n_spans; s0 += kSpansPerBlock)
             (L.bracket == 2 ? out->dense_items : out->items).push_back(make_uint2(l, s0));
     }
@@ -218,6 +227,7 @@ int adacomp_select_create(adacomp_select_t** h, const adacomp_segment_t* h_segs,
     for (const Layer& L : lay.layers)
         if (L.k > 0 && !L.bracket) s->all_bracketed = false;
     s->max_sample = lay.max_sample;
+    s->any_small = lay.any_small;
     s->cand_stride = lay.cand_stride;
     s->win_stride = lay.win_stride;
     s->span_stride = lay.span_stride;
@@ -293,7 +303,7 @@ int adacomp_select(adacomp_select_t* h, const float* d_grads, uint64_t worker_st
     p.span_stride = h->span_stride;
 
     const unsigned n_inst = n_workers * h->n_layers;
-    const bool bracketed = h->route == 0 && h->n_items > 0;
+    const bool bracketed = h->route == 0 && (h->n_items > 0 || h->any_small);
     int slot = 0;
     if (h->profiling) {                                   // take the next event set of the ring
         slot = h->ring_next;
@@ -314,7 +324,7 @@ int adacomp_select(adacomp_select_t* h, const float* d_grads, uint64_t worker_st
     k_bracket_sample<<<n_inst, kBig, bracketed ? h->max_sample * sizeof(uint32_t) : 0, st>>>(p, bracketed ? 0 : 1);
     ADACOMP_LAUNCH_CHECK();
     ADACOMP_CUDA(mark(1));
-    if (bracketed) {
+    if (bracketed && h->n_items > 0) {
         const dim3 grid(h->n_items, n_workers);
         if (h->n_items_sparse) {
             k_bracket_scan<<<dim3(h->n_items_sparse, n_workers), kThreads, kScanSmemPerWarp * (kThreads / 32), st>>>(p, 0u);

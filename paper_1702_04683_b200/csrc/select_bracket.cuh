@@ -42,6 +42,7 @@ constexpr float kBracketZ = 5.0f;                     // half-width of the brack
 constexpr uint32_t kGatherMax = 1024;
 constexpr int kBig = 1024;                            // threads of the per-instance kernels
 
+constexpr uint32_t kRouteSmall = 3u;                  // Layer::bracket of a tensor that is selected whole in shared memory
 constexpr uint32_t kInstBracket = 2u;                 // bracket valid, scan/emit act on the instance
 constexpr uint32_t kInstOverflow = 4u;                // a candidate or window list ran out of room
 
@@ -128,6 +129,74 @@ __global__ void __launch_bounds__(kBig) k_bracket_sample(SelectParams p, int gen
         st->cand_count = 0; st->win_count = 0; st->T = 0; st->cut = 0;
     }
     if (!bracket) return;
+    if (L.bracket == kRouteSmall) {
+        // ---- a tensor that fits into shared memory whole is selected right here: the exact threshold by
+        // digit passes over the keys on chip, then an ordered write (a warp per stretch of the tensor)
+        const float* first = p.grads + static_cast<uint64_t>(w) * p.stride + L.offset;
+        const uint32_t n = L.n, k = L.k;
+        for (uint32_t i = threadIdx.x; i < n; i += kBig) s_keys[i] = magnitude_key(first[i]);
+        __syncthreads();
+        // k-th largest key; with k = n every entry is kept (T = 0: all keys are above or equal)
+        const uint32_t T = k < n ? smem_kth_largest(s_keys, n, k, s_hist, s_warp, s_bc) : 0u;
+        const uint32_t lane = threadIdx.x & 31, warp = threadIdx.x >> 5, lt = (1u << lane) - 1u;
+        const uint32_t seg = (((n + 31) / 32) + 31) & ~31u;    // entries per warp, a multiple of 32
+        const uint32_t e0 = warp * seg < n ? warp * seg : n, e1 = e0 + seg < n ? e0 + seg : n;
+        uint32_t gt = 0, eq = 0;
+        for (uint32_t e = e0 + lane; e < e1; e += 32) {
+            const uint32_t key = s_keys[e];
+            gt += key > T ? 1u : 0u;
+            eq += key == T ? 1u : 0u;
+        }
+#pragma unroll
+        for (int d = 16; d; d >>= 1) {
+            gt += __shfl_xor_sync(0xFFFFFFFFu, gt, d);
+            eq += __shfl_xor_sync(0xFFFFFFFFu, eq, d);
+        }
+        if (lane == 0) { s_hist[warp] = gt; s_hist[32 + warp] = eq; }
+        __syncthreads();
+        // every warp works out where all stretches begin: lane j stands for warp j's stretch
+        const uint32_t gt_j = s_hist[lane], eq_j = s_hist[32 + lane];
+        uint32_t n_gt = gt_j, eq_inc = eq_j;
+#pragma unroll
+        for (int d = 16; d; d >>= 1) n_gt += __shfl_xor_sync(0xFFFFFFFFu, n_gt, d);
+#pragma unroll
+        for (int d = 1; d < 32; d <<= 1) {
+            const uint32_t y = __shfl_up_sync(0xFFFFFFFFu, eq_inc, d);
+            if (lane >= static_cast<uint32_t>(d)) eq_inc += y;
+        }
+        const uint32_t r = k - n_gt;                            // entries equal to T to keep: the lowest indices
+        const uint32_t eq_before_j = eq_inc - eq_j;
+        const uint32_t eq_kept_j = r > eq_before_j ? (r - eq_before_j < eq_j ? r - eq_before_j : eq_j) : 0u;
+        uint32_t out_inc = gt_j + eq_kept_j;
+        const uint32_t kept_j = out_inc;
+#pragma unroll
+        for (int d = 1; d < 32; d <<= 1) {
+            const uint32_t y = __shfl_up_sync(0xFFFFFFFFu, out_inc, d);
+            if (lane >= static_cast<uint32_t>(d)) out_inc += y;
+        }
+        uint32_t run_eq = __shfl_sync(0xFFFFFFFFu, eq_before_j, warp);
+        uint32_t run_out = __shfl_sync(0xFFFFFFFFu, out_inc - kept_j, warp);
+        uint32_t* idx_out = p.idx_out + static_cast<uint64_t>(w) * p.K + L.out_offset;
+        float* val_out = p.val_out + static_cast<uint64_t>(w) * p.K + L.out_offset;
+        const uint32_t glob = static_cast<uint32_t>(L.offset);
+        for (uint32_t base = e0; base < e1; base += 32) {
+            const uint32_t e = base + lane;
+            const bool valid = e < e1;
+            const uint32_t key = valid ? s_keys[e] : 0u;
+            const bool is_eq = valid && key == T;
+            const uint32_t b_eq = __ballot_sync(0xFFFFFFFFu, is_eq);
+            const bool keep = valid && (key > T || (is_eq && run_eq + __popc(b_eq & lt) < r));
+            const uint32_t b_keep = __ballot_sync(0xFFFFFFFFu, keep);
+            if (keep) {
+                const uint32_t pos = run_out + __popc(b_keep & lt);
+                idx_out[pos] = glob + e;
+                val_out[pos] = first[e];
+            }
+            run_eq += __popc(b_eq);
+            run_out += __popc(b_keep);
+        }
+        return;
+    }
     {   // the scan only writes the table entries of pieces that hold candidates
         uint2* sub_tab = p.sub_tab + (static_cast<uint64_t>(w) * p.span_stride + L.span_base) * kSubsPerSpan;
         for (uint32_t t = threadIdx.x; t < L.n_spans * kSubsPerSpan; t += kBig) sub_tab[t] = make_uint2(0u, 0u);

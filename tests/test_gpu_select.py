@@ -115,7 +115,7 @@ def test_routes_agree_and_are_taken(binding):
     sel = binding.Selector(segs, wl.n_workers, dev)
     idx_a, val_a = sel.select(g)
     status, general = sel.last_error()
-    assert status == 0 and general == 8 * 2        # only the 832- and 10 250-entry tensors are too small
+    assert status == 0 and general == 0            # the 832- and 10 250-entry tensors are selected on chip, the others bracketed
     sel.set_route(1)
     idx_g, val_g = sel.select(g)
     status, general = sel.last_error()
@@ -123,7 +123,32 @@ def test_routes_agree_and_are_taken(binding):
     assert torch.equal(idx_a, idx_g) and torch.equal(val_a.view(torch.int32), val_g.view(torch.int32))
     sel.set_route(0)
     idx_b, _ = sel.select(g)
-    assert torch.equal(idx_a, idx_b) and sel.last_error() == (0, 16)
+    assert torch.equal(idx_a, idx_b) and sel.last_error() == (0, 0)
+
+
+def test_three_routes_by_size_and_keep_fraction(binding):
+    """Tensors up to 16 384 entries are selected whole in shared memory, tensors between that and
+    32 768 entries and tensors that keep more than a quarter take the general route, the rest the
+    single-pass route: all against the oracle, with ties and every keep count at the edges."""
+    dev = torch.device("cuda", 0)
+    rng = np.random.default_rng(21)
+    sizes = [1, 2, 31, 32, 33, 1000, 1024, 4097, 16_383, 16_384, 16_385, 20_000, 32_767, 40_000, 70_000]
+    ks = [1, 2, 31, 1, 33, 999, 7, 4097, 5, 16_384, 100, 19_999, 300, 30_000, 700]
+    offsets = np.concatenate([[0], np.cumsum(np.array(sizes) + 3)[:-1]]).tolist()   # odd gaps: unaligned tensors
+    W = 3
+    stride = offsets[-1] + sizes[-1] + 5
+    g = rng.standard_normal((W, stride)).astype(np.float32)
+    g[:, ::7] = np.round(g[:, ::7], 1)                     # ties
+    g[1, ::5] = 0.0
+    gt = torch.from_numpy(g).to(dev)
+    sel = binding.Selector(binding.segments_from(offsets, sizes, ks), W, dev)
+    idx, val = sel.select(gt)
+    status, general = sel.last_error()
+    assert status == 0 and general == W * 4                # 16 385, 20 000, 32 767 (size) and 30 000 of 40 000 (fraction); k = n of 16 384 is on chip
+    h_idx, h_val = idx.cpu().numpy().view(np.uint32), val.cpu().numpy()
+    for w in range(W):
+        oi, ov = oracle.select_layers(g[w], offsets, sizes, ks)
+        assert np.array_equal(h_idx[w], oi) and np.array_equal(h_val[w].view(np.uint32), ov.view(np.uint32))
 
 
 def test_awkward_value_layouts_stay_exact_and_ties_fall_back(binding):
