@@ -94,7 +94,7 @@ struct BatchDesc {
     uint32_t n_updates;
 };
 
-constexpr uint32_t kRgAlphas = 33;             // alpha / sigma kept ready for sigma < 33
+constexpr uint32_t kAlphaTable = 33;             // alpha / sigma kept ready for sigma < 33
 
 // First position of an ascending index list whose entry is >= target.  The lists of an update are spread
 // over [0, n_params) more or less evenly, so a few interpolation steps narrow the search before the
@@ -185,7 +185,7 @@ k_apply_warps(const ServerParams sp, const BatchDesc d, const uint32_t* __restri
     uint32_t* s_head0 = s_mask + R;                                             // [R] head when the launch began (kPre)
     uint32_t* s_hops = s_head0 + R;                                             // [B][32] chain entries inside the window before the launch (kPre)
 
-    if (tid < kRgAlphas) s_alpha[tid] = tid ? __fdiv_rn(lr, static_cast<float>(tid)) : lr;   // Eq. 5 for the small counts, once
+    if (tid < kAlphaTable) s_alpha[tid] = tid ? __fdiv_rn(lr, static_cast<float>(tid)) : lr;   // Eq. 5 for the small counts, once
     __syncthreads();                                            // the only block barrier
     const uint32_t gw = blockIdx.x * kWpWarps + warp, n_gw = gridDim.x * kWpWarps;
     const uint32_t r_lo = static_cast<uint32_t>(static_cast<uint64_t>(n_ranges) * gw / n_gw);
@@ -338,7 +338,7 @@ k_apply_warps(const ServerParams sp, const BatchDesc d, const uint32_t* __restri
                             }
                             if (kExtra && sigma_out) sigma_out[d.pair_begin[b] + cur + lane] = sigma;
                             if (change) {
-                                const float alpha_k = sigma < kRgAlphas ? s_alpha[sigma] : __fdiv_rn(lr, static_cast<float>(sigma));   // Eq. 5
+                                const float alpha_k = sigma < kAlphaTable ? s_alpha[sigma] : __fdiv_rn(lr, static_cast<float>(sigma));   // Eq. 5
                                 th[kl] = __fsub_rn(th[kl], __fmul_rn(alpha_k, v));                     // Eq. 4
                                 const uint32_t pos = pos_l + cur;
                                 sp.prev[(pos + sp.ring_shift) & sp.ring_mask] = atomicExch(&hd[kl], pos);
@@ -441,7 +441,7 @@ k_apply_merged(const ServerParams sp, const BatchDesc d, uint32_t range, const u
     uint32_t* s_k = mine + (kPre ? 6 : 5) * R;                                  // [B][33] staged indices
     float* s_v = reinterpret_cast<float*>(s_k + B * kMgPitch);                  // [B][33] staged values
     if constexpr (kSlices) {
-        if (threadIdx.x < kRgAlphas) s_alpha[threadIdx.x] = threadIdx.x ? __fdiv_rn(lr, static_cast<float>(threadIdx.x)) : lr;   // Eq. 5, once
+        if (threadIdx.x < kAlphaTable) s_alpha[threadIdx.x] = threadIdx.x ? __fdiv_rn(lr, static_cast<float>(threadIdx.x)) : lr;   // Eq. 5, once
         __syncthreads();                                        // the only block barrier
     }
     const uint32_t gw = blockIdx.x * kMgWarps + warp, n_gw = gridDim.x * kMgWarps;
@@ -648,7 +648,7 @@ k_apply_merged(const ServerParams sp, const BatchDesc d, uint32_t range, const u
                             if (kPre) sigma += hops[u];                                                // Eq. 3, before the launch
                             if (kExtra && sigma_out) sigma_out[sq[u]] = sigma;
                             if (change) {
-                                const float alpha_k = sigma < kRgAlphas ? s_alpha[sigma] : __fdiv_rn(lr, static_cast<float>(sigma));   // Eq. 5
+                                const float alpha_k = sigma < kAlphaTable ? s_alpha[sigma] : __fdiv_rn(lr, static_cast<float>(sigma));   // Eq. 5
                                 th[kl] = __fsub_rn(th[kl], __fmul_rn(alpha_k, v));                     // Eq. 4
                                 sp.prev[(pos + sp.ring_shift) & sp.ring_mask] = atomicExch(&hd[kl], pos);
                             }
