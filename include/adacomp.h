@@ -128,8 +128,9 @@ ADACOMP_API int adacomp_select_host(adacomp_select_t* h, const float* h_grads, u
 
 /* Chooses how selections are computed; the results are identical.
  * 0 = automatic: tensors of at least 32768 entries with k <= n/4 take the bracketed route (a
- *     sample brackets the threshold, then the gradient is read once); instances whose bracket
- *     turns out wrong (or that hold a NaN), and all other tensors, take the general route;
+ *     sample brackets the threshold, then the gradient is read once); tensors of up to 16384
+ *     entries are selected whole in shared memory (read once); instances whose bracket turns out
+ *     wrong (or that hold a NaN), and all other tensors, take the general route;
  * 1 = general route for everything (multi-pass radix select; reads the gradient five times). */
 ADACOMP_API int adacomp_select_set_route(adacomp_select_t* h, int route);
 
@@ -160,7 +161,7 @@ ADACOMP_API int adacomp_select_gather(adacomp_select_t* h, const float* d_grads,
 /* Waits for cuda_stream, then returns the first error the device recorded since the last call
  * of this function (ADACOMP_OK if none) and clears it.  Also reports, if stats_out is not
  * NULL, stats_out[0] = how many (worker, segment) selections of the last adacomp_select call
- * took the general multi-pass route rather than the bracketed single-pass route. */
+ * took the general multi-pass route rather than one of the two single-pass routes. */
 ADACOMP_API int adacomp_select_last_error(adacomp_select_t* h, void* cuda_stream, uint64_t* stats_out);
 ADACOMP_API int adacomp_select_destroy(adacomp_select_t* h);
 
