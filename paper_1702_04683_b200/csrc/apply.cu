@@ -13,6 +13,7 @@
 // window start has been overwritten in the ring.
 #include <algorithm>
 #include <cmath>
+#include <map>
 #include <new>
 #include <utility>
 #include <vector>
@@ -838,6 +839,8 @@ struct adacomp_server {
     int validate = 0;
     int mode = 0;
     int rule = 0;                 // 0: per-parameter staleness (Eq. 3); 1: the update's staleness i - j for every entry
+    // resident blocks per SM of every (kernel, shared memory size) launched so far: asked once, not per launch
+    mutable std::map<std::pair<const void*, size_t>, int> blocks_per_sm;
 };
 
 namespace {
@@ -851,16 +854,31 @@ size_t carve_server(adacomp_server_t* s, void* base, uint64_t n_params, uint64_t
     return c.used;
 }
 
+// How many blocks of `kernel` with `smem` bytes of dynamic shared memory stay resident per SM; the first time a
+// (kernel, size) pair is seen the kernel is also allowed `max_smem` bytes.
+template <typename Kernel>
+int resident_blocks(const adacomp_server_t* s, Kernel kernel, int threads, size_t smem, size_t max_smem, int* per_sm) {
+    const auto key = std::make_pair(reinterpret_cast<const void*>(kernel), smem);
+    const auto it = s->blocks_per_sm.find(key);
+    if (it != s->blocks_per_sm.end()) { *per_sm = it->second; return ADACOMP_OK; }
+    ADACOMP_CUDA(cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(max_smem)));
+    int n = 1;
+    ADACOMP_CUDA(cudaOccupancyMaxActiveBlocksPerMultiprocessor(&n, kernel, threads, smem));
+    if (n < 1) n = 1;
+    try { s->blocks_per_sm[key] = n; } catch (...) { return ADACOMP_ERR_ALLOC; }
+    *per_sm = n;
+    return ADACOMP_OK;
+}
+
 // Launches k_apply_warps<R, kPre, kExtra> over all ranges of R parameters with as many blocks as stay resident.
 template <uint32_t R, bool kPre, bool kExtra>
 int launch_apply_warps_as(const adacomp_server_t* s, const ServerParams& sp, const BatchDesc& d, const uint32_t* d_idx,
                           const float* d_val, float lr, uint32_t* d_sigma_out, cudaStream_t st) {
     const size_t smem = wp_smem_bytes(R, d.n_updates, kPre);
     const uint32_t n_ranges = static_cast<uint32_t>((s->n_params + R - 1) / R);
-    ADACOMP_CUDA(cudaFuncSetAttribute(k_apply_warps<R, kPre, kExtra>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                      static_cast<int>(wp_smem_bytes(R, kMaxBatch, kPre))));
     int per_sm = 1;
-    ADACOMP_CUDA(cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, k_apply_warps<R, kPre, kExtra>, kWpThreads, smem));
+    const int rc = resident_blocks(s, k_apply_warps<R, kPre, kExtra>, kWpThreads, smem, wp_smem_bytes(R, kMaxBatch, kPre), &per_sm);
+    if (rc != ADACOMP_OK) return rc;
     unsigned grid = static_cast<unsigned>(s->n_sms) * static_cast<unsigned>(per_sm > 0 ? per_sm : 1);
     const unsigned most_blocks = (n_ranges + kWpWarps - 1) / kWpWarps;
     if (grid > most_blocks) grid = most_blocks;
@@ -885,10 +903,9 @@ template <uint32_t R, bool kPre, bool kExtra>
 int launch_apply_merged_as(const adacomp_server_t* s, const ServerParams& sp, const BatchDesc& d, uint64_t pairs,
                            const uint32_t* d_idx, const float* d_val, float lr, uint32_t* d_sigma_out, cudaStream_t st) {
     const size_t smem = mg_smem_bytes(R, d.n_updates, kPre);
-    ADACOMP_CUDA(cudaFuncSetAttribute(k_apply_merged<R, kPre, kExtra>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                      static_cast<int>(mg_smem_bytes(R, kMaxBatch, kPre))));
     int per_sm = 1;
-    ADACOMP_CUDA(cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, k_apply_merged<R, kPre, kExtra>, kMgThreads, smem));
+    const int rc = resident_blocks(s, k_apply_merged<R, kPre, kExtra>, kMgThreads, smem, mg_smem_bytes(R, kMaxBatch, kPre), &per_sm);
+    if (rc != ADACOMP_OK) return rc;
     const uint64_t warps = static_cast<uint64_t>(s->n_sms) * static_cast<uint64_t>(per_sm > 0 ? per_sm : 1) * kMgWarps;
     uint64_t range = R;
     if (R == 0) {
