@@ -128,7 +128,7 @@ __device__ __forceinline__ uint32_t first_at_or_above(const uint32_t* __restrict
 // ---------------------------------------------------------------------------------------------
 // Several updates per launch, one WARP per range of parameters, no block barrier in the loop.  A
 // warp owns a run of ranges of R consecutive parameters and a slice of shared memory: Theta and
-// the heads of the range (two buffers: the next range's arrive while this one is worked on), a
+// the heads of the range (two buffers where R <= 256: the next range's arrive while this one is worked on), a
 // mask per parameter (bit b: update b of the launch changed it) and, per update, a stage with
 // the update's next 32 pairs from its cursor.  All of that is brought in by asynchronous copies
 // issued a range ahead, so that no load is waited for in the common case.
@@ -149,8 +149,13 @@ constexpr int kWpThreads = 128;
 constexpr uint32_t kWpWarps = kWpThreads / 32;
 constexpr uint32_t kWpGroups = 4;              // groups of asynchronous copies per range
 
+// Ranges of up to 256 parameters keep two buffers of Theta and heads (the next range arrives while this one is
+// worked on); longer ranges keep one, which lets more warps stay resident, and fetch the next range from L2
+// between two ranges.
+__host__ __device__ constexpr uint32_t wp_buffers(uint32_t range) { return range <= 256 ? 2u : 1u; }
 __host__ __device__ inline size_t wp_warp_words(uint32_t range, uint32_t n_updates, bool pre) {
-    return 32 + (pre ? 96 : 64) * static_cast<size_t>(n_updates) + (pre ? 6 : 5) * static_cast<size_t>(range);
+    return 32 + (pre ? 96 : 64) * static_cast<size_t>(n_updates) +
+           (2 * wp_buffers(range) + (pre ? 2 : 1)) * static_cast<size_t>(range);
 }
 __host__ __device__ inline size_t wp_smem_bytes(uint32_t range, uint32_t n_updates, bool pre) {
     return 64 * 4 + kWpWarps * wp_warp_words(range, n_updates, pre) * 4;
@@ -174,15 +179,16 @@ k_apply_warps(const ServerParams sp, const BatchDesc d, const uint32_t* __restri
               float lr, uint32_t* sigma_out, uint32_t n_ranges) {
     extern __shared__ __align__(16) unsigned char s_wp[];
     static_assert(R % 64 == 0 && R >= 128, "16-byte pieces, whole warps");
+    constexpr uint32_t kBuffers = wp_buffers(R);
     float* s_alpha = reinterpret_cast<float*>(s_wp);                            // [64] alpha / sigma for the small counts
     const uint32_t B = d.n_updates;
     const uint32_t tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     uint32_t* s_cur = reinterpret_cast<uint32_t*>(s_wp) + 64 + warp * wp_warp_words(R, B, kPre);   // [32] cursor of every update
     uint32_t* s_k = s_cur + 32;                                                 // [B][32] staged indices
     float* s_v = reinterpret_cast<float*>(s_k + 32 * B);                        // [B][32] staged values
-    float* s_theta = s_v + 32 * B;                                              // [2][R] Theta of the range
-    uint32_t* s_head = reinterpret_cast<uint32_t*>(s_theta) + 2 * R;            // [2][R] latest change of the parameter
-    uint32_t* s_mask = s_head + 2 * R;                                          // [R] updates of this launch that changed it
+    float* s_theta = s_v + 32 * B;                                              // [kBuffers][R] Theta of the range
+    uint32_t* s_head = reinterpret_cast<uint32_t*>(s_theta) + kBuffers * R;     // [kBuffers][R] latest change of the parameter
+    uint32_t* s_mask = s_head + kBuffers * R;                                          // [R] updates of this launch that changed it
     uint32_t* s_head0 = s_mask + R;                                             // [R] head when the launch began (kPre)
     uint32_t* s_hops = s_head0 + R;                                             // [B][32] chain entries inside the window before the launch (kPre)
 
@@ -236,21 +242,31 @@ k_apply_warps(const ServerParams sp, const BatchDesc d, const uint32_t* __restri
     for (uint32_t b = 0; b < B; ++b) refill(b, s_cur[b]);
     sweep_in(r_lo, 0);
 #pragma unroll
-    for (uint32_t g = 0; g < kWpGroups; ++g) copy_async_commit();   // the first holds everything, the others are empty
+    for (uint32_t g = 0; g < kWpGroups + (kBuffers == 1 ? 1 : 0); ++g) copy_async_commit();   // the first holds everything, the others are empty
 
     const uint32_t per_group = (B + kWpGroups - 1) / kWpGroups;     // <= 8
     for (uint32_t r = r_lo; r < r_hi; ++r) {
-        const uint32_t p = (r - r_lo) & 1u;
+        const uint32_t p = kBuffers == 2 ? (r - r_lo) & 1u : 0u;
         const uint32_t lo = r * R, hi = range_end(r);
         float* th = s_theta + p * R;
         uint32_t* hd = s_head + p * R;
-        if (r + 1 < r_hi) sweep_in(r + 1, p ^ 1u);
+        if (kBuffers == 2) {
+            if (r + 1 < r_hi) sweep_in(r + 1, p ^ 1u);          // lands while this range is worked on
+        } else if (r + 1 < r_hi && lane * 32 < 2 * R) {         // one buffer: the next range's lines go to L2 for now
+            const uint32_t o = (lane * 32) % R;
+            if (static_cast<uint64_t>(r + 1) * R + o < sp.n_params)
+                prefetch_l2((lane * 32 < R ? reinterpret_cast<const uint32_t*>(sp.theta) : sp.head) + (r + 1) * R + o);
+        }
 #pragma unroll
         for (uint32_t o = lane * 4; o < R; o += 128) *reinterpret_cast<uint4*>(s_mask + o) = make_uint4(0, 0, 0, 0);
         // ---- the updates in arrival order
 #pragma unroll 1
         for (uint32_t g = 0; g < kWpGroups; ++g) {
-            copy_async_wait<kWpGroups - 1>();                   // what was issued a range ago for this group has landed
+            // what was issued a range ago for this group has landed (with one buffer every range ends with a group of
+            // its own, the next range's Theta and heads, which the first group waits for)
+            if (kBuffers == 2) copy_async_wait<kWpGroups - 1>();
+            else if (g == 0) copy_async_wait<0>();
+            else copy_async_wait<kWpGroups>();
             __syncwarp();
             if (kPre && g == 0) {
 #pragma unroll
@@ -382,6 +398,10 @@ k_apply_warps(const ServerParams sp, const BatchDesc d, const uint32_t* __restri
                 if (lo + o < hi && s_mask[o]) { sp.theta[lo + o] = th[o]; sp.head[lo + o] = hd[o]; }
         }
         __syncwarp();
+        if (kBuffers == 1) {
+            if (r + 1 < r_hi) sweep_in(r + 1, 0);
+            copy_async_commit();
+        }
     }
     copy_async_wait<0>();
     __syncwarp();
