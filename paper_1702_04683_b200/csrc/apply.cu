@@ -425,7 +425,7 @@ k_apply_warps(const ServerParams sp, const BatchDesc d, const uint32_t* __restri
 //           memory: Eq. 3 is the walk along the parameter's chain while it stays inside the window
 //           (pairs of this launch applied earlier are on the chain already), Eq. 5, Eq. 4, and the
 //           pair becomes the head.  Loads of Theta, heads and links go to L2 (no L1 line survives
-//           a change by another lane).  The host sizes the ranges to about 128 pairs.
+//           a change by another lane).  The host sizes the ranges to about 48 pairs.
 //   R > 0   ranges of R parameters whose Theta, heads and change masks live in the warp's shared
 //           memory, as in k_apply_warps (asynchronous copies a range ahead, Eq. 3 inside the launch
 //           from the mask, written back where changed): for launches that touch most 32-byte
@@ -918,7 +918,7 @@ int launch_apply_warps(const adacomp_server_t* s, const ServerParams& sp, const 
 }
 
 // Launches k_apply_merged<R, kPre, kExtra>.  R = 0: only the named parameters are touched, ranges sized so that
-// one holds about 128 pairs of the launch; R > 0: ranges of R parameters, swept through shared memory.
+// one holds about 48 pairs of the launch; R > 0: ranges of R parameters, swept through shared memory.
 template <uint32_t R, bool kPre, bool kExtra>
 int launch_apply_merged_as(const adacomp_server_t* s, const ServerParams& sp, const BatchDesc& d, uint64_t pairs,
                            const uint32_t* d_idx, const float* d_val, float lr, uint32_t* d_sigma_out, cudaStream_t st) {
@@ -929,9 +929,9 @@ int launch_apply_merged_as(const adacomp_server_t* s, const ServerParams& sp, co
     const uint64_t warps = static_cast<uint64_t>(s->n_sms) * static_cast<uint64_t>(per_sm > 0 ? per_sm : 1) * kMgWarps;
     uint64_t range = R;
     if (R == 0) {
-        // a range should hold about 128 pairs (some 8 per update, so that a stage of 32 lasts a few ranges), and
-        // every warp should get at least two ranges
-        double want = 128.0 * static_cast<double>(s->n_params) / static_cast<double>(pairs);
+        // a range should hold about 48 pairs (a few per update, so that a stage of 32 lasts several ranges; measured:
+        // 32 to 64 do equally well, 128 and more are slower), and every warp should get at least two ranges
+        double want = 48.0 * static_cast<double>(s->n_params) / static_cast<double>(pairs);
         const double balance = static_cast<double>(s->n_params) / (2.0 * static_cast<double>(warps));
         if (want > balance) want = balance;
         range = want < 32.0 ? 32 : static_cast<uint64_t>(want) / 32 * 32;
