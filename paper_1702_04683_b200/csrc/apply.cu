@@ -128,7 +128,7 @@ __device__ __forceinline__ uint32_t first_at_or_above(const uint32_t* __restrict
 // ---------------------------------------------------------------------------------------------
 // Several updates per launch, one WARP per range of parameters, no block barrier in the loop.  A
 // warp owns a run of ranges of R consecutive parameters and a slice of shared memory: Theta and
-// the heads of the range (two buffers where R <= 256: the next range's arrive while this one is worked on), a
+// the heads of the range (with two buffers the next range's arrive while this one is worked on), a
 // mask per parameter (bit b: update b of the launch changed it) and, per update, a stage with
 // the update's next 32 pairs from its cursor.  All of that is brought in by asynchronous copies
 // issued a range ahead, so that no load is waited for in the common case.
@@ -149,16 +149,15 @@ constexpr int kWpThreads = 128;
 constexpr uint32_t kWpWarps = kWpThreads / 32;
 constexpr uint32_t kWpGroups = 4;              // groups of asynchronous copies per range
 
-// Ranges of up to 256 parameters keep two buffers of Theta and heads (the next range arrives while this one is
-// worked on); longer ranges keep one, which lets more warps stay resident, and fetch the next range from L2
-// between two ranges.
-__host__ __device__ constexpr uint32_t wp_buffers(uint32_t range) { return range <= 256 ? 2u : 1u; }
-__host__ __device__ inline size_t wp_warp_words(uint32_t range, uint32_t n_updates, bool pre) {
-    return 32 + (pre ? 96 : 64) * static_cast<size_t>(n_updates) +
-           (2 * wp_buffers(range) + (pre ? 2 : 1)) * static_cast<size_t>(range);
+// `buffers` of Theta and heads per warp: with two the next range arrives while this one is worked on; with one
+// more warps stay resident and the next range is fetched (from L2, where a prefetch put it) between two ranges.
+// Measured: one is better for ranges longer than 256 parameters when a launch holds more than 8 updates (their
+// stages are what fills shared memory then), two otherwise.
+__host__ __device__ inline size_t wp_warp_words(uint32_t range, uint32_t n_updates, bool pre, uint32_t buffers) {
+    return 32 + (pre ? 96 : 64) * static_cast<size_t>(n_updates) + (2 * buffers + (pre ? 2 : 1)) * static_cast<size_t>(range);
 }
-__host__ __device__ inline size_t wp_smem_bytes(uint32_t range, uint32_t n_updates, bool pre) {
-    return 64 * 4 + kWpWarps * wp_warp_words(range, n_updates, pre) * 4;
+__host__ __device__ inline size_t wp_smem_bytes(uint32_t range, uint32_t n_updates, bool pre, uint32_t buffers) {
+    return 64 * 4 + kWpWarps * wp_warp_words(range, n_updates, pre, buffers) * 4;
 }
 
 __device__ __forceinline__ uint32_t smem_address(const void* p) { return static_cast<uint32_t>(__cvta_generic_to_shared(p)); }
@@ -173,17 +172,16 @@ __device__ __forceinline__ void copy_async_commit() { asm volatile("cp.async.com
 template <int kPending>
 __device__ __forceinline__ void copy_async_wait() { asm volatile("cp.async.wait_group %0;" ::"n"(kPending) : "memory"); }
 
-template <uint32_t R, bool kPre, bool kExtra>
+template <uint32_t R, uint32_t kBuffers, bool kPre, bool kExtra>
 __global__ void __launch_bounds__(kWpThreads)
 k_apply_warps(const ServerParams sp, const BatchDesc d, const uint32_t* __restrict__ idx, const float* __restrict__ val,
               float lr, uint32_t* sigma_out, uint32_t n_ranges) {
     extern __shared__ __align__(16) unsigned char s_wp[];
     static_assert(R % 64 == 0 && R >= 128, "16-byte pieces, whole warps");
-    constexpr uint32_t kBuffers = wp_buffers(R);
     float* s_alpha = reinterpret_cast<float*>(s_wp);                            // [64] alpha / sigma for the small counts
     const uint32_t B = d.n_updates;
     const uint32_t tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-    uint32_t* s_cur = reinterpret_cast<uint32_t*>(s_wp) + 64 + warp * wp_warp_words(R, B, kPre);   // [32] cursor of every update
+    uint32_t* s_cur = reinterpret_cast<uint32_t*>(s_wp) + 64 + warp * wp_warp_words(R, B, kPre, kBuffers);   // [32] cursor of every update
     uint32_t* s_k = s_cur + 32;                                                 // [B][32] staged indices
     float* s_v = reinterpret_cast<float*>(s_k + 32 * B);                        // [B][32] staged values
     float* s_theta = s_v + 32 * B;                                              // [kBuffers][R] Theta of the range
@@ -890,31 +888,41 @@ int resident_blocks(const adacomp_server_t* s, Kernel kernel, int threads, size_
     return ADACOMP_OK;
 }
 
-// Launches k_apply_warps<R, kPre, kExtra> over all ranges of R parameters with as many blocks as stay resident.
-template <uint32_t R, bool kPre, bool kExtra>
+// Launches k_apply_warps<R, kBuffers, kPre, kExtra> over all ranges of R parameters with as many blocks as stay resident.
+template <uint32_t R, uint32_t kBuffers, bool kPre, bool kExtra>
 int launch_apply_warps_as(const adacomp_server_t* s, const ServerParams& sp, const BatchDesc& d, const uint32_t* d_idx,
                           const float* d_val, float lr, uint32_t* d_sigma_out, cudaStream_t st) {
-    const size_t smem = wp_smem_bytes(R, d.n_updates, kPre);
+    const size_t smem = wp_smem_bytes(R, d.n_updates, kPre, kBuffers);
     const uint32_t n_ranges = static_cast<uint32_t>((s->n_params + R - 1) / R);
     int per_sm = 1;
-    const int rc = resident_blocks(s, k_apply_warps<R, kPre, kExtra>, kWpThreads, smem, wp_smem_bytes(R, kMaxBatch, kPre), &per_sm);
+    const int rc = resident_blocks(s, k_apply_warps<R, kBuffers, kPre, kExtra>, kWpThreads, smem,
+                                   wp_smem_bytes(R, kMaxBatch, kPre, kBuffers), &per_sm);
     if (rc != ADACOMP_OK) return rc;
     unsigned grid = static_cast<unsigned>(s->n_sms) * static_cast<unsigned>(per_sm > 0 ? per_sm : 1);
     const unsigned most_blocks = (n_ranges + kWpWarps - 1) / kWpWarps;
     if (grid > most_blocks) grid = most_blocks;
-    k_apply_warps<R, kPre, kExtra><<<grid, kWpThreads, smem, st>>>(sp, d, d_idx, d_val, lr, d_sigma_out, n_ranges);
+    k_apply_warps<R, kBuffers, kPre, kExtra><<<grid, kWpThreads, smem, st>>>(sp, d, d_idx, d_val, lr, d_sigma_out, n_ranges);
     ADACOMP_LAUNCH_CHECK();
     return ADACOMP_OK;
+}
+
+template <uint32_t R, uint32_t kBuffers>
+int launch_apply_warps_with(const adacomp_server_t* s, const ServerParams& sp, const BatchDesc& d, const uint32_t* d_idx,
+                            const float* d_val, float lr, uint32_t* d_sigma_out, cudaStream_t st) {
+    const bool pre = d.pre_mask != 0, extra = d_sigma_out != nullptr || sp.validate != 0;
+    if (pre) return extra ? launch_apply_warps_as<R, kBuffers, true, true>(s, sp, d, d_idx, d_val, lr, d_sigma_out, st)
+                          : launch_apply_warps_as<R, kBuffers, true, false>(s, sp, d, d_idx, d_val, lr, d_sigma_out, st);
+    return extra ? launch_apply_warps_as<R, kBuffers, false, true>(s, sp, d, d_idx, d_val, lr, d_sigma_out, st)
+                 : launch_apply_warps_as<R, kBuffers, false, false>(s, sp, d, d_idx, d_val, lr, d_sigma_out, st);
 }
 
 template <uint32_t R>
 int launch_apply_warps(const adacomp_server_t* s, const ServerParams& sp, const BatchDesc& d, const uint32_t* d_idx,
                        const float* d_val, float lr, uint32_t* d_sigma_out, cudaStream_t st) {
-    const bool pre = d.pre_mask != 0, extra = d_sigma_out != nullptr || sp.validate != 0;
-    if (pre) return extra ? launch_apply_warps_as<R, true, true>(s, sp, d, d_idx, d_val, lr, d_sigma_out, st)
-                          : launch_apply_warps_as<R, true, false>(s, sp, d, d_idx, d_val, lr, d_sigma_out, st);
-    return extra ? launch_apply_warps_as<R, false, true>(s, sp, d, d_idx, d_val, lr, d_sigma_out, st)
-                 : launch_apply_warps_as<R, false, false>(s, sp, d, d_idx, d_val, lr, d_sigma_out, st);
+    if constexpr (R > 256) {
+        if (d.n_updates > 8) return launch_apply_warps_with<R, 1>(s, sp, d, d_idx, d_val, lr, d_sigma_out, st);
+    }
+    return launch_apply_warps_with<R, 2>(s, sp, d, d_idx, d_val, lr, d_sigma_out, st);
 }
 
 // Launches k_apply_merged<R, kPre, kExtra>.  R = 0: only the named parameters are touched, ranges sized so that
