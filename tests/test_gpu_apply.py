@@ -264,6 +264,37 @@ def test_forty_updates_without_staleness_counts(binding, mode, density):
     assert np.array_equal(bits(theta), bits(ref.theta()))
 
 
+@pytest.mark.parametrize("mode", MODES)
+def test_every_update_names_the_same_parameters(binding, mode):
+    """Forty updates that all name the same 300 parameters (plus a few of their own): inside a launch
+    every parameter is changed by every update, so the order of the updates per parameter is all
+    that keeps the result right.  Staleness counts and parameters bit for bit."""
+    P = 50_000
+    rng = np.random.default_rng(77)
+    theta = torch.from_numpy(rng.standard_normal(P).astype(np.float32)).to(DEV)
+    ref = oracle.Server(theta.cpu().numpy())
+    srv = binding.Server(theta, history_pairs=1 << 18, max_window_updates=64)
+    srv.set_mode(mode)
+    common = np.sort(rng.choice(P, 300, replace=False))
+    ts = 0
+    for call in range(2):
+        ups = [np.unique(np.concatenate([common, rng.choice(P, 20, replace=False)])).astype(np.uint32) for _ in range(40)]
+        vals = [rng.standard_normal(a.size).astype(np.float32) for a in ups]
+        begin = np.concatenate([[0], np.cumsum([a.size for a in ups])[:-1]]).astype(np.uint64)
+        count = np.array([a.size for a in ups], np.uint32)
+        pull = np.array([max(0, ts + b - int(rng.integers(0, 45))) for b in range(40)], np.uint64)
+        idx, val = i32(np.concatenate(ups)), torch.from_numpy(np.concatenate(vals)).to(DEV)
+        sigma = torch.full_like(idx, -1)
+        srv.apply(idx, val, begin, count, pull, 0.05, sigma_out=sigma)
+        s = u32(sigma)
+        for b in range(40):
+            want = ref.apply(ups[b], vals[b], int(pull[b]), 0.05)
+            assert np.array_equal(s[int(begin[b]):int(begin[b]) + ups[b].size], want), f"call {call} update {b}"
+        ts += 40
+    assert srv.last_error() == 0 and srv.timestamp == ts == ref.timestamp
+    assert np.array_equal(bits(theta), bits(ref.theta()))
+
+
 def test_window_and_capacity_errors_leave_the_server_unchanged(binding):
     theta = torch.zeros(100, device=DEV)
     srv = binding.Server(theta, history_pairs=40, max_window_updates=8)     # ring of 64 pairs
