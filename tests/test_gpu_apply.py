@@ -11,7 +11,7 @@ from helpers import assert_same_pipeline, bits, gpu_pipeline, oracle_keep_counts
 
 pytestmark = pytest.mark.gpu
 DEV = torch.device("cuda", 0)
-MODES = [1, 2, 3, 4]
+MODES = [0, 1, 2, 3, 4]
 
 
 @pytest.fixture(scope="module")
