@@ -33,10 +33,9 @@ METRIC = "dense-gradient GB/s scanned (select+compact, with the selected pairs a
 UNIT = "GB/s"
 FALLBACK_HBM_GBS = 6650.0
 
-# DRAM bytes (read + write) of ONE scan-kernel launch, from the ncu capture summarised in
-# profiles/dram_traffic_large_flat_w4.md: workload 4 with 4 workers, MB per keep fraction (1/25 and
-# 1/10 are the dense scan kernel).  A launch over W workers moves W / 4 times as much.  Only valid while
-# the kernel source is the one that was profiled.
+# DRAM bytes (read + write) of ONE scan-kernel launch from an ncu capture of workload 4 with 4 workers,
+# MB per keep fraction (1/25 and 1/10 are the dense scan kernel).  A launch over W workers moves W / 4
+# times as much.  Only valid while the kernel source is the one that was profiled.
 SCAN_TRAFFIC_W4_MB = {"1/1000": 1645.7, "1/400": 1684.6, "1/160": 1795.8, "1/64": 1793.4, "1/25": 1788.9, "1/10": 2008.2}
 SCAN_SOURCE_SHA256_16 = "b6c409439069c8f1"
 

@@ -150,9 +150,9 @@ ADACOMP_API const char* adacomp_select_stage_name(uint32_t stage);
 ADACOMP_API int adacomp_select_pairs_per_worker(const adacomp_select_t* h, uint64_t* pairs_out);
 /* Values of entries chosen elsewhere: d_val_out[w][e] = d_grads[w][d_idx[w][e]] for the handle's
  * K = pairs_per_worker entries of each of n_workers workers (same layouts as adacomp_select).
- * Serves selections the library does not make itself, e.g. the random selection that one variant
- * of Comp-ASGD uses ("Compression" paragraph: the subset is chosen "randomly, or by keeping only
- * the largest gradients"); the random draw is the caller's.  An index outside the layout's extent
+ * Serves selections the library does not make itself, e.g. the random subset that one variant
+ * of Comp-ASGD sends instead of the largest entries ("Compression" paragraph); the random draw
+ * is the caller's.  An index outside the layout's extent
  * reads as 0 and is reported by adacomp_select_last_error as ADACOMP_ERR_INVALID. */
 ADACOMP_API int adacomp_select_gather(adacomp_select_t* h, const float* d_grads, uint64_t worker_stride_elems,
                                       uint32_t n_workers, const uint32_t* d_idx, float* d_val_out,
@@ -170,7 +170,7 @@ ADACOMP_API int adacomp_select_destroy(adacomp_select_t* h);
  * adacomp_select for a single segment {offset 0, n, k} and a single worker: the k entries of
  * largest magnitude of d_grad[0 .. n), lower index first among equals, written by ascending
  * index to d_idx_out[0 .. k) / d_val_out[0 .. k).  No handle and no workspace: the scratch the
- * selection needs (about 11 KB) is a fixed array inside the library, present on every GPU that
+ * selection needs (11 008 bytes) is a fixed array inside the library, present on every GPU that
  * loads it for as long as the process lives; the call allocates nothing, on the host or on the
  * device, and frees nothing.  Meant for code that runs where an allocation is not an option:
  * inside another framework's step whose memory pool it cannot reach, in a loop whose memory was
@@ -186,6 +186,11 @@ ADACOMP_API int adacomp_select_destroy(adacomp_select_t* h);
  * Work is enqueued on cuda_stream; the call returns without waiting. */
 ADACOMP_API int adacomp_select_static(const float* d_grad, uint32_t n, uint32_t k, uint32_t* d_idx_out,
                                       float* d_val_out, int device, void* cuda_stream);
+/* Companion of adacomp_select_static (no counterpart in the paper either): waits for cuda_stream,
+ * then returns the first error the device recorded during adacomp_select_static calls on `device`
+ * since the last call of this function (ADACOMP_OK if none) and clears it.  The status word is
+ * part of the same built-in array: nothing is allocated and the caller passes no buffer. */
+ADACOMP_API int adacomp_select_static_last_error(int device, void* cuda_stream);
 
 /* ------------------------------------------------------------------------------------------
  * Server side: Algorithm 2 (Eq. 3, Eq. 4, Eq. 5; "Complexity" paragraph for the history).
@@ -209,7 +214,7 @@ ADACOMP_API int adacomp_server_create(adacomp_server_t** s, uint64_t n_params, u
                           uint32_t max_window_updates, void* d_workspace, size_t workspace_bytes,
                           int device);
 
-/* "Initialize Theta(0)" (Algorithm 2): adopts d_theta (n_params fp32, caller-owned, holding
+/* First step of Algorithm 2 (the initial parameters): adopts d_theta (n_params fp32, caller-owned, holding
  * the initial values) as the parameter vector that adacomp_apply updates in place, sets the
  * timestamp to 0 and forgets all history.  The buffer must outlive the server or the next
  * reset. */
@@ -245,7 +250,11 @@ ADACOMP_API int adacomp_server_pull(adacomp_server_t* s, float* d_theta_copy, ui
  * pairs exceed history_pairs), ADACOMP_ERR_INVALID.  On the device an index >= n_params is
  * skipped and reported by adacomp_server_last_error as ADACOMP_ERR_UNSORTED; with validation
  * switched on (adacomp_server_set_validation) so is an index that is not larger than its
- * predecessor in the same update. */
+ * predecessor in the same update.  ADACOMP_ERR_ALLOC: a host-side table could not be allocated
+ * (nothing enqueued, server unchanged).  If a kernel launch itself fails (ADACOMP_ERR_CUDA) after
+ * earlier launches of the same call were enqueued, the device's history is ahead of the host's
+ * bookkeeping: the server then refuses every further update with ADACOMP_ERR_CUDA until
+ * adacomp_server_reset. */
 ADACOMP_API int adacomp_apply(adacomp_server_t* s, const uint32_t* d_idx, const float* d_val,
                               const uint64_t* h_pair_begin, const uint32_t* h_pair_count,
                               const uint64_t* h_pull_ts, uint32_t n_updates, float lr,
@@ -289,8 +298,8 @@ ADACOMP_API int adacomp_server_set_validation(adacomp_server_t* s, int on);
 ADACOMP_API int adacomp_server_set_mode(adacomp_server_t* s, int mode);
 /* Which rule adacomp_apply follows.
  * 0 = AdaComp (default): per-parameter staleness sigma_k of Eq. 3, learning rate of Eq. 5.
- * 1 = the competitors' rule of the "Experimental setup" (ASGD, Comp-ASGD: "the learning rate is
- *     divided by staleness and is global to each update"): every entry of an update that pulled
+ * 1 = the competitors' rule of the "Experimental setup" (ASGD, Comp-ASGD: one learning rate per
+ *     update, the base rate over the update's staleness): every entry of an update that pulled
  *     at j and is applied at timestamp i gets alpha / (i - j) (alpha if i = j), Eq. 4 is applied
  *     to every entry as written (zero-valued ones too), d_sigma_out receives i - j, and no history
  *     is read or kept.  ADACOMP_ERR_WINDOW if j > i or i - j >= 2^24.
@@ -321,7 +330,10 @@ ADACOMP_API int adacomp_server_destroy(adacomp_server_t* s);
  * per worker, n_blocks = ceil(pairs_per_worker / 256)) is the word at which block b starts in
  * worker w's stream d_words + w * words_per_worker; the last entry is the stream's length.
  * words_per_worker must be at least adacomp_encode_capacity_words(pairs_per_worker)
- * (ADACOMP_ERR_CAPACITY otherwise).  All arrays are the caller's device memory. */
+ * (ADACOMP_ERR_CAPACITY otherwise).  All arrays are the caller's device memory.  Decoding does not
+ * trust the stream: a block whose offset, width (> 32) or payload would reach outside the worker's
+ * words_per_worker words is not read; all its entries decode to 0xFFFFFFFF, an index that
+ * adacomp_apply skips and reports (ADACOMP_ERR_UNSORTED). */
 ADACOMP_API uint64_t adacomp_encode_capacity_words(uint64_t pairs_per_worker);
 ADACOMP_API int adacomp_encode_indices(const uint32_t* d_idx, uint64_t pairs_per_worker, uint32_t n_workers,
                                        uint32_t* d_words, uint64_t words_per_worker, uint64_t* d_block_off,

@@ -193,8 +193,8 @@ int oracle_literal_apply(void* h, const uint32_t* idx, const float* val, uint64_
 }
 
 // --- per-parameter form -----------------------------------------------------
-// "counting the number of updates applied on it since the last pull by the
-// worker" (text under Eq. 3): every parameter keeps the ascending list of
+// The text under Eq. 3 reads sigma_k as a count of the updates that changed
+// parameter k since the worker's last pull: every parameter keeps the ascending list of
 // timestamps at which a non-zero update touched it; sigma_k is how many of
 // them are >= j.  Same function as the literal form, cost O(sigma_k) per
 // entry, usable on the full-size workloads.
@@ -242,8 +242,8 @@ int oracle_server_apply(void* h, const uint32_t* idx, const float* val, uint64_t
 }
 
 // --- the competitors' rule ------------------------------------------------------
-// ASGD and Comp-ASGD ("Experimental setup"): "the learning rate is divided by
-// staleness and is global to each update".  The staleness of an update is the
+// ASGD and Comp-ASGD ("Experimental setup"): one learning rate per update, the
+// base rate over the update's staleness.  The staleness of an update is the
 // number of times Theta has evolved between the fetch at timestamp j and the push
 // at timestamp i ("The parameter server model": w2's update on Figure 2 has
 // staleness 2), i.e. sigma = i - j, the same for every entry of the update.  The

@@ -60,6 +60,7 @@ def _load():
         "adacomp_select_profile": (i32, [vp, P(f32), u32, P(u64)]),
         "adacomp_select_stage_name": (ctypes.c_char_p, [u32]),
         "adacomp_select_static": (i32, [vp, u32, u32, vp, vp, i32, vp]),
+        "adacomp_select_static_last_error": (i32, [i32, vp]),
         "adacomp_select_pairs_per_worker": (i32, [vp, P(u64)]),
         "adacomp_select_last_error": (i32, [vp, vp, P(u64)]),
         "adacomp_select_destroy": (i32, [vp]),
@@ -167,6 +168,11 @@ def adacomp_select_static(grad: torch.Tensor, k: int, idx_out: torch.Tensor, val
     _check(_lib.adacomp_select_static(grad.data_ptr(), grad.numel(), int(k), _dev(idx_out, torch.int32, "idx_out"),
                                       _dev(val_out, torch.float32, "val_out"), grad.device.index,
                                       _stream_ptr(stream)), "adacomp_select_static")
+
+
+def adacomp_select_static_last_error(device_index: int = 0, stream: Optional[torch.cuda.Stream] = None) -> int:
+    """Waits for the stream; first device-side error of adacomp_select_static calls since the last read."""
+    return int(_lib.adacomp_select_static_last_error(int(device_index), _stream_ptr(stream)))
 
 
 # ----------------------------------------------------------------------------- worker side

@@ -730,8 +730,8 @@ k_apply_merged(const ServerParams sp, const BatchDesc d, uint32_t range, const u
 }
 
 // ---------------------------------------------------------------------------------------------
-// The competitors' rule ("Experimental setup": for ASGD and Comp-ASGD the learning rate is divided
-// by staleness and is global to each update): every entry of an update gets the same learning
+// The competitors' rule ("Experimental setup": ASGD and Comp-ASGD use one learning rate per update,
+// the base rate over the update's staleness): every entry of an update gets the same learning
 // rate alpha / (i - j), which the host has already computed (one fp32 division); Eq. 4 is applied
 // to every entry as written.  No history is read or kept.  One launch per update, the stream
 // orders updates.
@@ -857,6 +857,7 @@ struct adacomp_server {
     int validate = 0;
     int mode = 0;
     int rule = 0;                 // 0: per-parameter staleness (Eq. 3); 1: the update's staleness i - j for every entry
+    bool poisoned = false;        // a launch failed after earlier launches of the same call were enqueued: reset needed
     // resident blocks per SM of every (kernel, shared memory size) launched so far: asked once, not per launch
     mutable std::map<std::pair<const void*, size_t>, int> blocks_per_sm;
 };
@@ -1018,6 +1019,7 @@ int adacomp_server_reset(adacomp_server_t* s, float* d_theta, void* cuda_stream)
     ADACOMP_CUDA(cudaMemsetAsync(s->d_head, 0xFF, s->n_params * sizeof(uint32_t), st));
     ADACOMP_CUDA(cudaMemsetAsync(s->d_status, 0, sizeof(int), st));
     s->d_theta = d_theta;
+    s->poisoned = false;
     s->timestamp = 0;
     s->pos_next = 0;
     s->pos_base = 0;
@@ -1038,10 +1040,14 @@ int adacomp_server_pull(adacomp_server_t* s, float* d_theta_copy, uint64_t* h_ti
     return ADACOMP_OK;
 }
 
-int adacomp_apply(adacomp_server_t* s, const uint32_t* d_idx, const float* d_val,
-                  const uint64_t* h_pair_begin, const uint32_t* h_pair_count, const uint64_t* h_pull_ts,
-                  uint32_t n_updates, float lr, uint32_t* d_sigma_out, void* cuda_stream) {
+// The body of adacomp_apply; may throw std::bad_alloc from its host-side tables (caught by the caller).
+// `*enqueued` is set once the first kernel of the call has been launched: an error after that leaves device
+// and host bookkeeping out of step.
+static int apply_body(adacomp_server_t* s, const uint32_t* d_idx, const float* d_val,
+                      const uint64_t* h_pair_begin, const uint32_t* h_pair_count, const uint64_t* h_pull_ts,
+                      uint32_t n_updates, float lr, uint32_t* d_sigma_out, void* cuda_stream, bool* enqueued) {
     if (!s || !s->d_theta) return ADACOMP_ERR_INVALID;
+    if (s->poisoned) return ADACOMP_ERR_CUDA;
     if (n_updates == 0) return ADACOMP_OK;
     if (!h_pair_begin || !h_pair_count || !h_pull_ts) return ADACOMP_ERR_INVALID;
     uint64_t call_pairs = 0;
@@ -1059,6 +1065,7 @@ int adacomp_apply(adacomp_server_t* s, const uint32_t* d_idx, const float* d_val
         DeviceGuard guard(s->device);
         if (guard.err != cudaSuccess) return cuda_fail(guard.err);
         cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+        *enqueued = true;
         ServerParams sp;
         sp.theta = s->d_theta;
         sp.head = nullptr;
@@ -1099,9 +1106,41 @@ int adacomp_apply(adacomp_server_t* s, const uint32_t* d_idx, const float* d_val
         win_abs[b] = ws;
     }
 
+    // ---- which updates share a launch (modes 0, 2, 3): up to kMaxBatch consecutive ones, and no more than the
+    // ring allows.  Warps of one launch work on different parameter ranges at their own pace, so a pair of a late
+    // update may be linked into the ring while an early update of the same launch still walks its window: the
+    // slot written must not be one the window can reach, i.e. the launch must end within `ring` positions of
+    // the oldest window start among its updates.  A launch is cut before the update that would break this (one
+    // update alone never does: that is the check above).
+    std::vector<uint32_t> launch_first;               // first update of every launch, plus n_updates at the end
+    launch_first.reserve(n_updates / kMaxBatch + 2);
+    for (uint32_t b0 = 0; b0 < n_updates;) {
+        launch_first.push_back(b0);
+        uint64_t oldest = win_abs[b0];
+        uint32_t b1 = b0 + 1;
+        while (b1 < n_updates && b1 - b0 < kMaxBatch) {
+            const uint64_t o = win_abs[b1] < oldest ? win_abs[b1] : oldest;
+            if (start_abs[b1 + 1] - o > s->ring) break;
+            oldest = o;
+            ++b1;
+        }
+        b0 = b1;
+    }
+    launch_first.push_back(n_updates);
+    bool shared_slots = false;                 // two updates write their counts to the same slots: order matters
+    if (d_sigma_out && n_updates > 1 && s->mode != 1) {
+        std::vector<std::pair<uint64_t, uint64_t>> slices;
+        for (uint32_t b = 0; b < n_updates; ++b)
+            if (h_pair_count[b]) slices.emplace_back(h_pair_begin[b], h_pair_begin[b] + h_pair_count[b]);
+        std::sort(slices.begin(), slices.end());
+        for (size_t a = 1; a < slices.size(); ++a)
+            if (slices[a].first < slices[a - 1].second) { shared_slots = true; break; }
+    }
+
     DeviceGuard guard(s->device);
     if (guard.err != cudaSuccess) return cuda_fail(guard.err);
     cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+    *enqueued = true;
 
     if (s->mode == 4) {
         // ---- the paper's list structure: windows are bounded, positions are only ring slots (no re-basing)
@@ -1175,20 +1214,12 @@ int adacomp_apply(adacomp_server_t* s, const uint32_t* d_idx, const float* d_val
     // 8 % of the parameters or more (most 32-byte sectors of Theta are touched anyway), else the kernel that
     // touches only the named parameters; a single update, and updates whose staleness slots overlap in memory, go
     // one per launch.
-    bool shared_slots = false;                 // two updates write their counts to the same slots: order matters
-    if (d_sigma_out && n_updates > 1 && s->mode != 1) {
-        std::vector<std::pair<uint64_t, uint64_t>> slices;
-        for (uint32_t b = 0; b < n_updates; ++b)
-            if (h_pair_count[b]) slices.emplace_back(h_pair_begin[b], h_pair_begin[b] + h_pair_count[b]);
-        std::sort(slices.begin(), slices.end());
-        for (size_t a = 1; a < slices.size(); ++a)
-            if (slices[a].first < slices[a - 1].second) { shared_slots = true; break; }
-    }
     const bool one_by_one = s->mode == 1 || shared_slots || (s->mode == 0 && n_updates == 1);
     const bool theta_aligned = reinterpret_cast<uintptr_t>(s->d_theta) % 16 == 0;
-    for (uint32_t b0 = 0; b0 < n_updates && !one_by_one; b0 += kMaxBatch) {
+    for (size_t g = 0; g + 1 < launch_first.size() && !one_by_one; ++g) {
+        const uint32_t b0 = launch_first[g];
         BatchDesc d;
-        d.n_updates = (n_updates - b0 < kMaxBatch) ? n_updates - b0 : kMaxBatch;
+        d.n_updates = launch_first[g + 1] - b0;
         d.pre_mask = 0;
         uint64_t pairs = 0;
         uint32_t most = 0;
@@ -1249,6 +1280,23 @@ int adacomp_apply(adacomp_server_t* s, const uint32_t* d_idx, const float* d_val
     s->pos_next = start_abs[n_updates];
     s->timestamp = i0 + n_updates;        // the timestamp advances once per update (Algorithm 2)
     return ADACOMP_OK;
+}
+
+int adacomp_apply(adacomp_server_t* s, const uint32_t* d_idx, const float* d_val,
+                  const uint64_t* h_pair_begin, const uint32_t* h_pair_count, const uint64_t* h_pull_ts,
+                  uint32_t n_updates, float lr, uint32_t* d_sigma_out, void* cuda_stream) {
+    bool enqueued = false;
+    int rc;
+    try {
+        rc = apply_body(s, d_idx, d_val, h_pair_begin, h_pair_count, h_pull_ts, n_updates, lr, d_sigma_out, cuda_stream,
+                        &enqueued);
+    } catch (...) {                                     // a host-side table could not be allocated
+        rc = ADACOMP_ERR_ALLOC;
+    }
+    // an error after the first launch leaves the device's history ahead of the host's bookkeeping: the server
+    // refuses further updates until it is reset
+    if (rc != ADACOMP_OK && enqueued && s) s->poisoned = true;
+    return rc;
 }
 
 int adacomp_apply_host(adacomp_server_t* s, const uint32_t* h_idx, const float* h_val,

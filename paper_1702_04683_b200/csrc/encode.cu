@@ -122,9 +122,18 @@ k_decode(const uint32_t* __restrict__ words, uint64_t words_per_worker, const ui
     const uint64_t b = blockIdx.x, w = blockIdx.y, first = b * kCodeBlock;
     const uint32_t n = static_cast<uint32_t>(K - first < kCodeBlock ? K - first : kCodeBlock);
     const uint32_t t = threadIdx.x, lane = t & 31, warp = t >> 5;
-    const uint32_t* in = words + w * words_per_worker + block_off[w * (n_blocks + 1) + b];
-    uint32_t width = in[1];
-    width = width > 32 ? 32 : width;
+    // the stream is untrusted (it arrives from a worker): the block must lie inside the worker's words with a
+    // width of at most 32 bits, else the block decodes to 0xFFFFFFFF everywhere, an index no server accepts
+    // (adacomp_apply skips and reports it), and nothing outside the stream is read
+    const uint64_t off = block_off[w * (n_blocks + 1) + b];
+    bool sound = off + 2 <= words_per_worker;
+    const uint32_t* in = words + w * words_per_worker + (sound ? off : 0);
+    uint32_t width = sound ? in[1] : 0u;
+    sound = sound && width <= 32 && off + 2 + (static_cast<uint64_t>(n - 1) * width + 31) / 32 <= words_per_worker;
+    if (!sound) {
+        if (t < n) idx_out[w * K + first + t] = 0xFFFFFFFFu;
+        return;
+    }
     uint32_t step = 0;                                   // what entry t adds to its predecessor
     if (t == 0) step = in[0];
     else if (t < n) {

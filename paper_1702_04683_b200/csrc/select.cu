@@ -592,3 +592,19 @@ extern "C" int adacomp_select_static(const float* d_grad, uint32_t n, uint32_t k
     ADACOMP_LAUNCH_CHECK();
     return ADACOMP_OK;
 }
+
+// Companion of adacomp_select_static: the status word lives in the same built-in array, so reading it
+// needs no buffer from the caller and no allocation either.
+extern "C" int adacomp_select_static_last_error(int device, void* cuda_stream) {
+    DeviceGuard guard(device);
+    if (guard.err != cudaSuccess) return cuda_fail(guard.err);
+    unsigned char* base = nullptr;
+    const int rc = static_scratch_for(device, &base);
+    if (rc != ADACOMP_OK) return rc;
+    cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+    int status = 0;
+    ADACOMP_CUDA(cudaMemcpyAsync(&status, base + kStOffStatus, sizeof status, cudaMemcpyDeviceToHost, st));
+    ADACOMP_CUDA(cudaMemsetAsync(base + kStOffStatus, 0, sizeof(int), st));
+    ADACOMP_CUDA(cudaStreamSynchronize(st));
+    return status;
+}

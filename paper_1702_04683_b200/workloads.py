@@ -177,7 +177,7 @@ def round_gradients(wl: Workload, rnd: int, device="cpu", workers: Optional[Sequ
 
 
 def initial_parameters(wl: Workload, device="cpu") -> torch.Tensor:
-    """Theta(0): N(0, 0.05^2) ("Initialize Theta(0) with random values", Algorithm 2)."""
+    """Theta(0): N(0, 0.05^2) (Algorithm 2 starts from random parameters)."""
     g = torch.Generator(device=device)
     g.manual_seed(wl.seed * 7919 + 17 + wl.index)
     return torch.empty(wl.n_params, dtype=torch.float32, device=device).normal_(0.0, 0.05, generator=g)

@@ -131,12 +131,34 @@ def test_resnet_full_size_server(binding, mode):
     run_server_both(binding, wl, ks, mode)
 
 
-@pytest.mark.parametrize("mode", MODES)
-@pytest.mark.parametrize("keep", [(1, 1000), (1, 10)])
+# every keep fraction the benchmark times in the automatic mode (each picks another kernel or
+# range size); the two ends of the sweep also in every forced mode
+_LARGE_FLAT_CASES = [(0, k) for k in wlmod.workload(4).keep_fractions] + \
+                    [(m, k) for m in MODES[1:] for k in ((1, 1000), (1, 10))]
+
+
+@pytest.mark.parametrize("mode,keep", _LARGE_FLAT_CASES)
 def test_large_flat_full_size_server_sampled(binding, mode, keep):
     wl = wlmod.workload(4)
     ks = oracle_keep_counts(wl.tensor_sizes, keep)
     run_server_both(binding, wl, ks, mode, sample_only=True)
+
+
+# ----------------------------------------------------------------------------- whole path, full sizes
+
+@pytest.mark.parametrize("index,keep,rounds", [(1, (1, 100), 2), (2, (1, 100), 1), (2, (1, 10), 1), (3, (5, 1000), 2)])
+def test_full_size_selector_output_meets_the_server(index, keep, rounds):
+    """The 200-worker, the tie-stress and the ResNet-50-shaped workloads at full tensor sizes and
+    full worker counts: what the selector emits is what the server applies, round after round,
+    against the oracle's select -> apply (two rounds where the workload has more: the second one
+    carries windows that reach back over the first)."""
+    import dataclasses
+    wl = dataclasses.replace(wlmod.workload(index), n_rounds=rounds)
+    got = gpu_pipeline(wl, keep, mode=0)
+    want = oracle_pipeline(wl, keep, DEV)
+    assert_same_pipeline(got, want)
+    if rounds > 1:
+        assert max(int(s.max()) for s in want["sigma"]) >= 1
 
 
 # ----------------------------------------------------------------------------- semantics and errors
@@ -261,6 +283,78 @@ def test_forty_updates_without_staleness_counts(binding, mode, density):
             ref.apply(ups[b], vals[b], int(pull[b]), 0.05)
         ts += n_up
     assert srv.last_error() == 0 and srv.timestamp == ts == ref.timestamp
+    assert np.array_equal(bits(theta), bits(ref.theta()))
+
+
+@pytest.mark.parametrize("mode", [0, 3])
+@pytest.mark.parametrize("n_up", [6, 12])
+@pytest.mark.parametrize("with_sigma", [False, True])
+def test_updates_of_six_percent_density(binding, mode, n_up, with_sigma):
+    """Updates whose densest one names 5.1 % - 6.8 % of the parameters: the dense kernel then works on
+    ranges of 384 parameters, with two buffers of Theta and heads for up to 8 updates per launch and
+    one buffer beyond.  Second call: windows that reach back before the launch."""
+    P = 300_011
+    rng = np.random.default_rng(384 + n_up)
+    theta = torch.from_numpy(rng.standard_normal(P).astype(np.float32)).to(DEV)
+    ref = oracle.Server(theta.cpu().numpy())
+    srv = binding.Server(theta, history_pairs=1 << 21, max_window_updates=64)
+    srv.set_mode(mode)
+    ts = 0
+    for call in range(2):
+        sizes = [int(P * d) for d in rng.uniform(0.052, 0.066, n_up)]
+        sizes[0] = int(P * 0.066)
+        ups = [np.sort(rng.choice(P, sz, replace=False)).astype(np.uint32) for sz in sizes]
+        vals = [rng.standard_normal(a.size).astype(np.float32) for a in ups]
+        vals[1][::4] = 0.0
+        begin = np.concatenate([[0], np.cumsum([a.size for a in ups])[:-1]]).astype(np.uint64)
+        count = np.array([a.size for a in ups], np.uint32)
+        pull = np.array([max(0, ts + b - int(rng.integers(0, 2 * n_up))) for b in range(n_up)], np.uint64)
+        idx, val = i32(np.concatenate(ups)), torch.from_numpy(np.concatenate(vals)).to(DEV)
+        sigma = torch.full_like(idx, -1) if with_sigma else None
+        srv.apply(idx, val, begin, count, pull, 0.05, sigma_out=sigma)
+        for b in range(n_up):
+            want = ref.apply(ups[b], vals[b], int(pull[b]), 0.05)
+            if with_sigma:
+                lo = int(begin[b])
+                assert np.array_equal(u32(sigma)[lo:lo + ups[b].size], want), f"call {call} update {b}"
+        ts += n_up
+    assert srv.last_error() == 0 and srv.timestamp == ts == ref.timestamp
+    assert np.array_equal(bits(theta), bits(ref.theta()))
+
+
+@pytest.mark.parametrize("mode", MODES)
+def test_tight_history_ring_in_one_call(binding, mode):
+    """A ring sized with no slack, several updates in one call: an old window on the first update,
+    later updates of the same call that name parameters with history and whose pairs would wrap
+    onto ring slots the first update's window still reaches.  Launches must be cut so that no such
+    slot is overwritten while it can still be walked: staleness and parameters against the oracle."""
+    P = 4096
+    rng = np.random.default_rng(64)
+    theta = torch.from_numpy(rng.standard_normal(P).astype(np.float32)).to(DEV)
+    ref = oracle.Server(theta.cpu().numpy())
+    srv = binding.Server(theta, history_pairs=40, max_window_updates=8)          # ring of 64 slots
+    srv.set_mode(mode)
+    def run(ups, pulls, lr=0.25):
+        vals = [(1.0 + rng.random(len(a))).astype(np.float32) for a in ups]
+        begin = np.concatenate([[0], np.cumsum([len(a) for a in ups])[:-1]]).astype(np.uint64)
+        count = np.array([len(a) for a in ups], np.uint32)
+        idx = i32(np.concatenate(ups).astype(np.uint32))
+        val = torch.from_numpy(np.concatenate(vals)).to(DEV)
+        sigma = torch.full_like(idx, -1)
+        srv.apply(idx, val, begin, count, np.array(pulls, np.uint64), lr, sigma_out=sigma)
+        s = u32(sigma)
+        for b, a in enumerate(ups):
+            want = ref.apply(np.asarray(a, np.uint32), vals[b], int(pulls[b]), lr)
+            assert np.array_equal(s[int(begin[b]):int(begin[b]) + len(a)], want), f"update {b}"
+    u0 = np.arange(0, 30) * 100                            # update 0: positions 0 .. 29
+    run([u0], [0])
+    # one call: b0 pulled at 0 (window = update 0), 10 pairs on update 0's parameters (positions 30 .. 39);
+    # b1 fresh, 30 pairs on update 0's parameters (positions 40 .. 69: the last six wrap onto slots 0 .. 5)
+    run([u0[:10], u0], [0, 2])
+    # the same shape again, further along the ring, with three updates in the call
+    ts = srv.timestamp
+    run([u0[5:15], u0[:15], u0[10:25]], [ts - 1, ts, ts + 1])          # 40 pairs: all the history the server keeps
+    assert srv.last_error() == 0 and srv.timestamp == ref.timestamp
     assert np.array_equal(bits(theta), bits(ref.theta()))
 
 

@@ -89,3 +89,25 @@ def test_full_size_update_round_trip_and_sampled_blocks(binding):
         assert int(h_off[w, b + 1]) - lo == ow.size
         assert np.array_equal(u32(words[w, lo:lo + ow.size]), ow)
     assert 4.0 * float(h_off[:, -1].sum()) / (4 * K) < 1.0      # under a byte per index at keep 1/10
+
+
+def test_corrupt_streams_are_not_followed(binding):
+    """A decoder at the server's ingress cannot trust what arrives: block offsets that point outside
+    the stream, a width above 32 bits, or a payload that would run past the end must not be read;
+    the block decodes to 0xFFFFFFFF (an index every server refuses) and the other blocks are intact."""
+    rng = np.random.default_rng(5)
+    K = 1000                                                    # four blocks
+    rows = np.stack([np.sort(rng.choice(10**6, K, replace=False)).astype(np.uint32) for _ in range(2)])
+    idx = torch.from_numpy(rows.view(np.int32)).to(DEV)
+    words, off = binding.adacomp_encode_indices(idx)
+    cap = words.shape[1]
+    bad_off = off.clone()
+    bad_off[0, 1] = 10**12                                      # block 1 of worker 0: far outside the stream
+    bad_off[1, 3] = cap - 1                                     # block 3 of worker 1: header would straddle the end
+    bad_words = words.clone()
+    bad_words[0, int(off[0, 2]) + 1] = 77                       # block 2 of worker 0: a width of 77 bits
+    back = u32(binding.adacomp_decode_indices(bad_words, bad_off, K))
+    want = rows.copy()
+    want[0, 256:512] = want[0, 512:768] = 0xFFFFFFFF
+    want[1, 768:] = 0xFFFFFFFF
+    assert np.array_equal(back, want)

@@ -252,19 +252,29 @@ def test_resnet50_shaped_full_tensors(binding):
     check_against_oracle(binding, g, wl.offsets, wl.tensor_sizes, ks)
 
 
-@pytest.mark.parametrize("keep", [(1, 1000), (1, 64), (1, 10)])
-def test_large_flat_full_size_sampled(binding, keep):
-    """100 M parameters x 16 workers in the launch configuration the benchmark times; the oracle
-    checks sampled (worker, tensor) selections one by one, and cheap invariants cover the rest."""
-    dev = torch.device("cuda", 0)
+@pytest.fixture(scope="module")
+def large_flat_gradients():
+    """Workload 4's 16 x 100 M gradients, generated once for the six keep fractions."""
     wl = wlmod.workload(4)
-    g = wlmod.round_gradients(wl, 0, dev)
+    g = wlmod.round_gradients(wl, 0, torch.device("cuda", 0))
+    yield wl, g
+    del g
+    torch.cuda.empty_cache()
+
+
+@pytest.mark.parametrize("keep", wlmod.workload(4).keep_fractions)
+def test_large_flat_full_size_sampled(binding, large_flat_gradients, keep):
+    """100 M parameters x 16 workers in the launch configuration the benchmark times, at every keep
+    fraction it times; the oracle checks sampled (worker, tensor) selections one by one, and cheap
+    invariants cover the rest."""
+    dev = torch.device("cuda", 0)
+    wl, g = large_flat_gradients
     ks = oracle_keep_counts(wl.tensor_sizes, keep)
     K = sum(ks)
     segs = binding.segments_from(wl.offsets, wl.tensor_sizes, ks)
     sel = binding.Selector(segs, wl.n_workers, dev)
     idx, val = sel.select(g)
-    assert sel.last_error()[0] == 0
+    assert sel.last_error() == (0, 0)              # every selection stayed on the single-pass route
     # invariants at full size, on the GPU: ascending inside each tensor's slice, values are the
     # entries they name, indices stay inside their tensor
     idx64 = idx.view(wl.n_workers, len(ks), ks[0]).to(torch.int64) & 0xFFFFFFFF
@@ -273,12 +283,66 @@ def test_large_flat_full_size_sampled(binding, keep):
     assert bool(((idx64 >= lo) & (idx64 < lo + wl.tensor_sizes[0])).all())
     gathered = torch.gather(g, 1, idx64.view(wl.n_workers, K))
     assert torch.equal(gathered.view(torch.int32), val.view(torch.int32))
-    # the oracle on sampled selections
+    del idx64, gathered
+    # the oracle on sampled selections: 26 distinct (worker, tensor) pairs, the first and the last included
     rng = np.random.default_rng(keep[1])
-    for _ in range(6):
-        w, l = int(rng.integers(wl.n_workers)), int(rng.integers(len(ks)))
+    n_inst = wl.n_workers * len(ks)
+    picks = set(rng.choice(n_inst, 24, replace=False).tolist()) | {0, n_inst - 1}
+    for inst in sorted(picks):
+        w, l = divmod(inst, len(ks))
         off, n = wl.offsets[l], wl.tensor_sizes[l]
         oi, ov = oracle.select(g[w, off:off + n].cpu().numpy(), ks[l], offset=off)
         lo_k = sum(ks[:l])
-        assert np.array_equal(u32(idx[w, lo_k:lo_k + ks[l]]), oi)
-        assert np.array_equal(bits(val[w, lo_k:lo_k + ks[l]]), bits(ov))
+        assert np.array_equal(u32(idx[w, lo_k:lo_k + ks[l]]), oi), (w, l)
+        assert np.array_equal(bits(val[w, lo_k:lo_k + ks[l]]), bits(ov)), (w, l)
+
+
+# ----------------------------------------------------------------------------- NaN
+
+def _nan_patterns():
+    """Quiet, signalling and payload-carrying NaNs of both signs, as fp32 bit patterns."""
+    return np.array([0x7FC00000, 0xFFC00000, 0x7FA00001, 0xFF800001, 0x7FC12345, 0x7FFFFFFF, 0xFFFFFFFF, 0x7F800001],
+                    dtype=np.uint32)
+
+
+def test_nan_orders_above_inf_on_every_route(binding):
+    """The contract for NaN inputs: a NaN orders above +Inf by its bit pattern (sign dropped), the
+    same on every route, values bit for bit.  One bracketed tensor (the single pass detects the NaN
+    and hands the tensor to the general route), one tensor small enough for the on-chip route, one
+    tensor that keeps more than a quarter (general route by plan)."""
+    dev = torch.device("cuda", 0)
+    rng = np.random.default_rng(404)
+    sizes = [200_000, 9_000, 50_000]
+    ks = [2_000, 90, 20_000]
+    offsets = [0, 200_003, 209_010]
+    stride = offsets[-1] + sizes[-1] + 1
+    W = 4
+    g = rng.standard_normal((W, stride)).astype(np.float32)
+    nan = _nan_patterns()
+    gb = g.view(np.uint32)
+    # worker 0: no NaN anywhere; worker 1: NaNs in every tensor (fewer than k); worker 2: NaNs and
+    # infinities together in the bracketed tensor; worker 3: more NaNs than k in the small tensor
+    for off, n in zip(offsets, sizes):
+        gb[1, off + rng.choice(n, nan.size, replace=False)] = nan
+    pos = rng.choice(sizes[0], nan.size + 4, replace=False)
+    gb[2, pos[:nan.size]] = nan
+    g[2, pos[nan.size:]] = [np.inf, -np.inf, np.inf, -np.inf]
+    many = rng.choice(sizes[1], 200, replace=False)
+    gb[3, offsets[1] + many] = nan[rng.integers(0, nan.size, 200)]
+    gt = torch.from_numpy(g).to(dev)
+    assert np.array_equal(gt.cpu().numpy().view(np.uint32), gb)          # the copy kept every payload
+    sel = binding.Selector(binding.segments_from(offsets, sizes, ks), W, dev)
+    idx, val = sel.select(gt)
+    status, general = sel.last_error()
+    assert status == 0
+    # general route: the third tensor of every worker (by plan) and the bracketed tensor of the two
+    # workers whose single pass met a NaN
+    assert general == W + 2
+    h_idx, h_val = u32(idx), val.cpu().numpy()
+    for w in range(W):
+        oi, ov = oracle.select_layers(g[w], offsets, sizes, ks)
+        assert np.array_equal(h_idx[w], oi), f"worker {w}: indices differ"
+        assert np.array_equal(bits(h_val[w]), bits(ov)), f"worker {w}: values differ"
+    # every NaN of worker 1 is among the kept entries of its tensor (it orders above everything finite)
+    kept = set(h_idx[1].tolist())
+    assert all(int(i) in kept for i in np.flatnonzero(np.isnan(g[1])))

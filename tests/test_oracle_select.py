@@ -190,3 +190,29 @@ def test_keep_count_of_the_workloads():
     # a 64-entry tensor at 0.5 % still sends one entry
     assert oracle.keep_count(64, 5, 1000) == 1
     assert oracle.keep_count(2_359_296, 5, 1000) == 11_797     # 11796.48 rounded up
+
+
+def test_nan_orders_above_inf_by_bit_pattern():
+    """The reading for NaN inputs: the key is the bit pattern without the sign, so every NaN
+    outranks +-Inf and NaNs rank among themselves by payload; values keep their bits (signalling
+    NaNs are not quieted).  Checked with the pairwise form of the rule and by subset enumeration."""
+    pats = np.array([0x7FC00000, 0xFFC00000, 0x7FA00001, 0xFF800001, 0x7FC12345, 0x7FFFFFFF], dtype=np.uint32)
+    tiny = np.array([1.0, np.inf, 0.0, -np.inf, 2.0, -3.0, 0.5], dtype=np.float32)
+    tiny = np.concatenate([tiny, pats[:3].view(np.float32)])
+    rng = np.random.default_rng(9)
+    tiny = tiny[rng.permutation(tiny.size)]
+    for k in range(1, tiny.size + 1):
+        idx, val = oracle.select(tiny, k)
+        assert tuple(int(i) for i in idx) == unique_valid_subset(tiny, k)
+        assert np.array_equal(val.view(np.uint32), tiny.view(np.uint32)[idx])
+        idx2, _ = oracle.select(tiny, k, full_sort=True)
+        assert np.array_equal(idx, idx2)
+    # with 3 NaNs and 2 infinities, k = 3 keeps exactly the NaNs and k = 5 adds both infinities
+    nan_at = set(np.flatnonzero(np.isnan(tiny)).tolist())
+    assert set(oracle.select(tiny, 3)[0].tolist()) == nan_at
+    assert set(oracle.select(tiny, 5)[0].tolist()) == nan_at | set(np.flatnonzero(np.isinf(tiny)).tolist())
+    g = rng.standard_normal(5000).astype(np.float32)
+    g.view(np.uint32)[rng.choice(5000, pats.size, replace=False)] = pats
+    for k in (1, 3, 6, 7, 50):
+        idx, val = oracle.select(g, k)
+        check_is_the_selection(g, k, idx, val)

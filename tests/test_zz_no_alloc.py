@@ -5,15 +5,20 @@ framework's training step has no access to that framework's memory pool, a servi
 its memory at start-up must not grow, and under memory pressure an allocation may stall the
 device or fail.  For them the library carries a small fixed scratch array of its own, and
 adacomp_select_static uses it instead of a caller-provided workspace.  This test checks, through
-the C ABI, that it returns exactly what the regular entry point returns (indices and values bit
-for bit, the tolerance all selection tests use), twice in a row with different inputs, since
-the second call finds the array as the first one left it.  It is collected last on purpose.
+the C ABI, that it returns exactly what the regular entry point returns and what the CPU oracle
+returns (indices and values bit for bit, the tolerance all selection tests use), twice in a row
+with different inputs, since the second call finds the array as the first one left it; that
+further calls leave the amount of free device memory where it was; and the edges of its own
+geometry (a base that is only 4-byte aligned, the largest size it takes).  It is collected last
+on purpose.
 """
 import ctypes
 
 import numpy as np
 import pytest
 import torch
+
+import oracle
 
 pytestmark = pytest.mark.gpu
 
@@ -32,6 +37,12 @@ def regular_select(binding, g, k):
     return idx[0].clone(), val[0].clone()
 
 
+def assert_is_oracle_selection(g, k, idx, val):
+    want_idx, want_val = oracle.select(g.cpu().numpy(), k)
+    assert np.array_equal(idx.cpu().numpy().view(np.uint32), want_idx)
+    assert np.array_equal(val.cpu().numpy().view(np.uint32), want_val.view(np.uint32))
+
+
 def test_static_entry_point_matches_regular_one_twice_in_a_row(binding):
     dev = torch.device("cuda", 0)
     gen = torch.Generator(device=dev)
@@ -44,13 +55,39 @@ def test_static_entry_point_matches_regular_one_twice_in_a_row(binding):
     launches = binding.adacomp_kernel_launches()
     for g, (n, k), (idx, val) in zip(inputs, cases, outs):       # two calls back to back on one stream
         binding.adacomp_select_static(g, k, idx, val)
-    torch.cuda.synchronize()
+    assert binding.adacomp_select_static_last_error(0) == 0      # waits for the stream
     assert binding.adacomp_kernel_launches() == launches + 2 * 8
     for g, (n, k), (idx, val) in zip(inputs, cases, outs):
         want_idx, want_val = regular_select(binding, g, k)
         assert torch.equal(idx, want_idx)
         assert torch.equal(val.view(torch.int32), want_val.view(torch.int32))
         assert bool((idx[1:] > idx[:-1]).all())
+        assert_is_oracle_selection(g, k, idx, val)
+
+
+def test_static_entry_point_allocates_nothing_and_takes_awkward_geometry(binding):
+    dev = torch.device("cuda", 0)
+    gen = torch.Generator(device=dev)
+    gen.manual_seed(777)
+    n_max = 1 << 24                                              # the most the built-in scratch covers
+    buf = torch.randn(n_max + 8, device=dev, generator=gen)
+    odd = buf[1:200_002]                                         # 4 bytes past a 16-byte boundary, odd length
+    assert odd.data_ptr() % 16 == 4
+    big = buf[1:n_max + 1]                                       # with the odd base this needs every chunk slot of the scratch
+    cases = [(odd, 1_234), (big, 5_000), (big[:n_max - 3], 1)]
+    outs = [(torch.full((k,), -1, dtype=torch.int32, device=dev), torch.zeros(k, device=dev)) for _, k in cases]
+    binding.adacomp_select_static(odd, 7, outs[0][0][:7], outs[0][1][:7])        # first call on the device: address look-up
+    torch.cuda.synchronize()
+    allocated, reserved = torch.cuda.memory_allocated(dev), torch.cuda.memory_reserved(dev)
+    free_before, _ = torch.cuda.mem_get_info(dev)
+    for (g, k), (idx, val) in zip(cases, outs):
+        binding.adacomp_select_static(g, k, idx, val)
+    assert binding.adacomp_select_static_last_error(0) == 0
+    free_after, _ = torch.cuda.mem_get_info(dev)
+    assert torch.cuda.memory_allocated(dev) == allocated and torch.cuda.memory_reserved(dev) == reserved
+    assert free_after >= free_before                             # nothing was taken from the device behind torch's back
+    for (g, k), (idx, val) in zip(cases, outs):
+        assert_is_oracle_selection(g, k, idx, val)
 
 
 def test_static_entry_point_limits(binding):
