@@ -128,9 +128,9 @@ ADACOMP_API int adacomp_select_host(adacomp_select_t* h, const float* h_grads, u
 
 /* Chooses how selections are computed; the results are identical.
  * 0 = automatic: tensors of at least 32768 entries with k <= n/4 take the bracketed route (a
- *     sample brackets the threshold, then the gradient is read once); tensors of up to 16384
- *     entries are selected whole in shared memory (read once); instances whose bracket turns out
- *     wrong (or that hold a NaN), and all other tensors, take the general route;
+ *     sample brackets the threshold, then the gradient is read once); shorter tensors are
+ *     selected whole in shared memory (read once); instances whose bracket turns out wrong (or
+ *     that hold a NaN), and longer tensors with k > n/4, take the general route;
  * 1 = general route for everything (multi-pass radix select; reads the gradient five times). */
 ADACOMP_API int adacomp_select_set_route(adacomp_select_t* h, int route);
 
@@ -138,8 +138,8 @@ ADACOMP_API int adacomp_select_set_route(adacomp_select_t* h, int route);
  * around each of its kernels (a few microseconds of host work per call, no synchronisation).
  * adacomp_select_profile waits for the calls made since profiling was switched on and writes
  * the mean device time per call of each stage, in milliseconds, to h_ms_out[0 .. n_stages),
- * n_stages = 10 (0 for a stage that never ran), and the number of calls to *h_calls_out (may be
- * NULL).  Switching profiling on (again) starts a fresh measurement.
+ * n_stages = the number of stages adacomp_select_stage_name knows (0 for a stage that never ran),
+ * and the number of calls to *h_calls_out (may be NULL).  Switching profiling on (again) starts a fresh measurement.
  * adacomp_select_stage_name names a stage ("bracket_scan", ...; "" beyond the last). */
 ADACOMP_API int adacomp_select_set_profiling(adacomp_select_t* h, int on);
 ADACOMP_API int adacomp_select_profile(adacomp_select_t* h, float* h_ms_out, uint32_t n_stages,

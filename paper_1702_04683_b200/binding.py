@@ -283,10 +283,13 @@ class Selector:
 
     def profile(self) -> dict:
         """Mean device milliseconds per kernel and call since profiling was switched on."""
-        ms = (ctypes.c_float * 10)()
+        n = 0
+        while _lib.adacomp_select_stage_name(n):
+            n += 1
+        ms = (ctypes.c_float * n)()
         calls = ctypes.c_uint64(0)
-        _check(_lib.adacomp_select_profile(self._h, ms, 10, ctypes.byref(calls)), "adacomp_select_profile")
-        out = {_lib.adacomp_select_stage_name(i).decode(): float(ms[i]) for i in range(10)}
+        _check(_lib.adacomp_select_profile(self._h, ms, n, ctypes.byref(calls)), "adacomp_select_profile")
+        out = {_lib.adacomp_select_stage_name(i).decode(): float(ms[i]) for i in range(n)}
         out["calls"] = int(calls.value)
         return out
 

@@ -10,11 +10,11 @@
 using namespace adacomp;
 
 namespace {
-constexpr int kSelectStages = 10;
+constexpr int kSelectStages = 11;
 constexpr int kProfileRing = 32;
 const char* const kStageNames[kSelectStages] = {
     "bracket_sample", "bracket_scan", "bracket_resolve", "bracket_emit", "general_plan",
-    "general_hist0", "general_hist1", "general_hist2", "general_count", "general_write"};
+    "general_hist0", "general_hist1", "general_hist2", "general_count", "general_write", "fallback_solo"};
 }  // namespace
 
 struct adacomp_select {
@@ -74,7 +74,7 @@ void plan_bracket(Layer& L, Layout* out) {
     L.sample = L.n_spans = L.span_base = L.cand_cap = L.win_cap = 0;
     L.cand_base = L.win_base = 0;
     if (L.n < kBracketMinN || L.n > kBracketMaxN || L.k == 0 || static_cast<uint64_t>(L.k) * 4 > L.n) {
-        if (L.k > 0 && L.n <= kSampleMax) {                    // small enough for the keys to sit in shared memory whole
+        if (L.k > 0 && L.n <= kSmallMax) {                     // small enough for the keys to sit in shared memory whole
             L.bracket = kRouteSmall;
             if (L.n > out->max_sample) out->max_sample = L.n;
         }
@@ -245,7 +245,7 @@ int adacomp_select_create(adacomp_select_t** h, const adacomp_segment_t* h_segs,
         e = cudaMemcpy(s->d_items, lay.items.data(), lay.items.size() * sizeof(uint2), cudaMemcpyHostToDevice);
     if (e == cudaSuccess)
         e = cudaFuncSetAttribute(k_bracket_sample, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                 static_cast<int>(kSampleMax * sizeof(uint32_t)));
+                                 static_cast<int>(kSmallMax * sizeof(uint32_t)));
     if (e == cudaSuccess)
         e = cudaFuncSetAttribute(k_bracket_scan, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                  static_cast<int>(kScanSmemPerWarp * (kThreads / 32)));
@@ -344,12 +344,22 @@ int adacomp_select(adacomp_select_t* h, const float* d_grads, uint64_t worker_st
     }
     ADACOMP_CUDA(mark(4));
 
-    // general route for whatever is flagged for it (tensors not on the bracketed route, and
-    // instances whose bracket missed); the kernels find an empty list otherwise
+    if (bracketed && h->all_bracketed) {
+        // every tensor is on a single-pass route: only instances whose bracket missed are left, which is
+        // rare, so one launch in which a block works such an instance off alone replaces the six below
+        unsigned solo = static_cast<unsigned>(h->n_sms) * 2;
+        if (solo > n_inst) solo = n_inst;
+        ADACOMP_CUDA(mark(10));
+        k_fallback_solo<<<solo, kBig, 0, st>>>(p);
+        ADACOMP_LAUNCH_CHECK();
+        ADACOMP_CUDA(mark(11));
+        return ADACOMP_OK;
+    }
+
+    // general route for whatever is flagged for it (tensors not on a single-pass route, and
+    // instances whose bracket missed)
     const uint64_t total_slots = static_cast<uint64_t>(h->slots_per_worker) * n_workers;
-    // when every tensor is on the bracketed route the general kernels almost always find an empty
-    // list: keep their grid small then (a rare miss still gets one block per SM and chunk)
-    uint64_t grid64 = static_cast<uint64_t>(h->n_sms) * (bracketed && h->all_bracketed ? 1 : 8);
+    uint64_t grid64 = static_cast<uint64_t>(h->n_sms) * 8;
     if (grid64 > total_slots) grid64 = total_slots;
     if (grid64 == 0) grid64 = 1;
     const unsigned grid = static_cast<unsigned>(grid64);

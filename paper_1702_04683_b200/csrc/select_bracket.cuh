@@ -37,6 +37,7 @@ constexpr uint32_t kMaxSpans = 4096;                  // spans whose counters th
 constexpr uint32_t kBracketMaxN = 0xFFFF0000u;        // shifted 32-bit coordinates must not wrap
 constexpr uint32_t kBracketMinN = 32768;
 constexpr uint32_t kSampleMax = 16384;
+constexpr uint32_t kSmallMax = kBracketMinN - 1;         // longest tensor whose keys are selected whole in shared memory
 constexpr uint32_t kSampleMin = 2048;
 constexpr float kBracketZ = 5.0f;                     // half-width of the bracket in sample standard deviations
 constexpr uint32_t kGatherMax = 1024;
@@ -60,6 +61,16 @@ __host__ __device__ inline void bracket_ranks(uint32_t n, uint32_t k, uint32_t m
 __device__ __forceinline__ uint32_t hash32(uint32_t x) {
     x ^= x >> 16; x *= 0x7feb352du; x ^= x >> 15; x *= 0x846ca68bu; x ^= x >> 16;
     return x;
+}
+
+// hist[bin] += 1 for every lane with `on`, one shared-memory atomic per distinct bin of the warp: lanes
+// that hold the same bin are found with a match and the lowest of them adds their number.  Magnitudes
+// of real gradients crowd into a handful of exponent values, so without this the lanes of a warp
+// would queue up on the same few counters.  All 32 lanes must call.
+__device__ __forceinline__ void hist_add_aggregated(uint32_t* hist, uint32_t bin, bool on) {
+    const uint32_t peers = __match_any_sync(0xFFFFFFFFu, on ? bin : 0xFFFFFFFFu);
+    const uint32_t lane = threadIdx.x & 31;
+    if (on && (peers & ((1u << lane) - 1u)) == 0) atomicAdd(&hist[bin], __popc(peers));
 }
 
 // Descending walk over a 2048-bin histogram in shared memory: the bucket holding the rem-th
@@ -94,10 +105,12 @@ __device__ uint32_t smem_kth_largest(const uint32_t* keys, uint32_t m, uint32_t 
         const int nb = pass == 0 ? 2048 : 1024;
         for (int b = threadIdx.x; b < 2048; b += kBig) hist[b] = 0;
         __syncthreads();
-        for (uint32_t i = threadIdx.x; i < m; i += kBig) {
-            const uint32_t key = keys[i];
-            const bool match = pass == 0 || (key >> (shift + 10)) == (prefix >> (shift + 10));
-            if (match) atomicAdd(&hist[(key >> shift) & (nb - 1)], 1u);
+        for (uint32_t i0 = 0; i0 < m; i0 += kBig) {
+            const uint32_t i = i0 + threadIdx.x;
+            const uint32_t key = i < m ? keys[i] : 0u;
+            const bool match = i < m && (pass == 0 || (key >> (shift + 10)) == (prefix >> (shift + 10)));
+            if (pass == 0) hist_add_aggregated(hist, (key >> shift) & (nb - 1), match);   // every key counts: crowded bins
+            else if (match) atomicAdd(&hist[(key >> shift) & (nb - 1)], 1u);
         }
         __syncthreads();
         uint32_t b, above, cnt;
@@ -121,6 +134,7 @@ __global__ void __launch_bounds__(kBig) k_bracket_sample(SelectParams p, int gen
     const Layer L = p.layers[l];
     Inst* st = &p.inst[inst];
     const bool bracket = L.bracket && !general_only;
+    if (inst == 0 && threadIdx.x == 0) p.list_len[0] = 0;        // selections that took the general route: none so far
     if (threadIdx.x == 0) {
         st->prefix = 0; st->k_rem = L.k; st->n_gt = 0;
         st->flags = bracket ? 0u : (L.k > 0 ? kInstGeneral : 0u);
@@ -930,6 +944,105 @@ __global__ void __launch_bounds__(kThreads) k_bracket_emit(SelectParams p) {
             }
             off += __popc(b);
         }
+    }
+}
+
+// ---------------------------------------------------------------------------------------------
+// The general route done by ONE block per instance, for layouts whose tensors are all on a single-pass
+// route: only instances whose bracket missed (or that hold a NaN) are flagged then, which is rare, so
+// one launch that usually finds nothing replaces the general route's six.  A block takes the flagged
+// instances blockIdx.x, blockIdx.x + gridDim.x, ... and does for each what the general route does:
+// three digit passes over bits [30:20], [19:10], [9:0] of the keys give the exact k-th largest key T,
+// then one more pass writes, in index order, every entry with key > T and the r lowest-index entries
+// with key == T (a block walks its tensor front to back, so the running counts are simply carried
+// along: no count pass).  Four reads of the tensor, the later ones mostly from L2.
+__global__ void __launch_bounds__(kBig) k_fallback_solo(SelectParams p) {
+    __shared__ uint32_t s_hist[2048];
+    __shared__ uint32_t s_warp[33];
+    __shared__ uint32_t s_bc[3];
+    const uint32_t n_inst = p.n_workers * p.n_layers;
+    for (uint32_t inst = blockIdx.x; inst < n_inst; inst += gridDim.x) {
+        Inst* st = &p.inst[inst];
+        if (!(__ldcg(&st->flags) & kInstGeneral)) continue;      // the same for every thread of the block
+        const uint32_t w = inst / p.n_layers, l = inst - w * p.n_layers;
+        const Layer L = p.layers[l];
+        if (L.k == 0) continue;
+        const float* first = p.grads + static_cast<uint64_t>(w) * p.stride + L.offset;
+        const uint32_t mis = static_cast<uint32_t>((reinterpret_cast<uintptr_t>(first) >> 2) & 3u);
+        const float4* vec = reinterpret_cast<const float4*>(first - mis);
+        const uint64_t n_shift = static_cast<uint64_t>(L.n) + mis, nvec = (n_shift + 3) >> 2;
+        uint32_t prefix = 0, rem = L.k;
+        if (L.k < L.n) {
+#pragma unroll 1
+            for (int pass = 0; pass < 3; ++pass) {
+                const int shift = pass == 0 ? 20 : (pass == 1 ? 10 : 0);
+                const uint32_t nb = pass == 0 ? 2048u : 1024u;
+                for (int b = threadIdx.x; b < 2048; b += kBig) s_hist[b] = 0;
+                __syncthreads();
+                for (uint64_t base = 0; base < nvec; base += kBig) {
+                    const uint64_t v = base + threadIdx.x;
+                    float4 x = make_float4(0.f, 0.f, 0.f, 0.f);
+                    if (v < nvec) x = __ldg(&vec[v]);
+                    const float xs[4] = {x.x, x.y, x.z, x.w};
+#pragma unroll
+                    for (int q = 0; q < 4; ++q) {
+                        const uint64_t e = v * 4 + q;
+                        const uint32_t key = magnitude_key(xs[q]);
+                        const bool on = e >= mis && e < n_shift &&
+                                        (pass == 0 || (key >> (shift + 10)) == (prefix >> (shift + 10)));
+                        const uint32_t bin = (key >> shift) & (nb - 1u);
+                        if (pass == 0) hist_add_aggregated(s_hist, bin, on);      // every entry counts: crowded bins
+                        else if (on) atomicAdd(&s_hist[bin], 1u);                 // few entries match the prefix
+                    }
+                }
+                __syncthreads();
+                uint32_t b, above, cnt;
+                block_pick_bucket(s_hist, rem, &b, &above, &cnt, s_warp, s_bc);   // unused upper bins are zero
+                prefix |= b << shift;
+                rem -= above;
+            }
+        }
+        // k = n: prefix = 0 and rem = n keep every entry (all keys are >= 0)
+        const uint32_t T = prefix, r = rem;
+        uint32_t gt_base = 0, eq_base = 0;
+        uint32_t* idx_out = p.idx_out + static_cast<uint64_t>(w) * p.K + L.out_offset;
+        float* val_out = p.val_out + static_cast<uint64_t>(w) * p.K + L.out_offset;
+        for (uint64_t base = 0; base < nvec; base += kBig) {
+            const uint64_t v = base + threadIdx.x;
+            float xs[4] = {0.f, 0.f, 0.f, 0.f};
+            uint32_t gtm = 0, eqm = 0;
+            if (v < nvec) {
+                const float4 x = __ldg(&vec[v]);
+                xs[0] = x.x; xs[1] = x.y; xs[2] = x.z; xs[3] = x.w;
+#pragma unroll
+                for (int q = 0; q < 4; ++q) {
+                    const uint64_t e = v * 4 + q;
+                    const uint32_t key = magnitude_key(xs[q]);
+                    const bool ok = e >= mis && e < n_shift;
+                    gtm |= (ok && key > T) ? (1u << q) : 0u;
+                    eqm |= (ok && key == T) ? (1u << q) : 0u;
+                }
+            }
+            // a tile holds 4096 entries: both counts fit 16 bits only up to 4095, so they are scanned apart
+            uint32_t tot_gt, tot_eq;
+            uint32_t gt_before = gt_base + block_exclusive_scan_t<kBig>(__popc(gtm), &tot_gt, s_warp);
+            uint32_t eq_before = eq_base + block_exclusive_scan_t<kBig>(__popc(eqm), &tot_eq, s_warp);
+#pragma unroll
+            for (int q = 0; q < 4; ++q) {
+                const bool is_gt = (gtm >> q) & 1u, is_eq = (eqm >> q) & 1u;
+                if (is_gt || (is_eq && eq_before < r)) {
+                    const uint32_t pos = gt_before + (eq_before < r ? eq_before : r);
+                    idx_out[pos] = static_cast<uint32_t>(L.offset + (v * 4 + q - mis));
+                    val_out[pos] = xs[q];
+                }
+                gt_before += is_gt ? 1u : 0u;
+                eq_before += is_eq ? 1u : 0u;
+            }
+            gt_base += tot_gt;
+            eq_base += tot_eq;
+        }
+        if (threadIdx.x == 0) atomicAdd(&p.list_len[0], 1u);       // reported as "took the general route"
+        __syncthreads();
     }
 }
 

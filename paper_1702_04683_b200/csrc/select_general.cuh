@@ -281,16 +281,23 @@ __global__ void __launch_bounds__(kThreads) k_general_hist(SelectParams p) {
         __syncthreads();
         for (uint32_t i = 0; i < cv.iters; ++i) {
             const uint64_t v = cv.vec_begin + static_cast<uint64_t>(i) * kThreads + threadIdx.x;
-            if (v < cv.nvec) {
-                const float4 x = __ldg(&cv.vec[v]);
-                const float xs[4] = {x.x, x.y, x.z, x.w};
-                const uint64_t e0 = v * 4;
+            float4 x = make_float4(0.f, 0.f, 0.f, 0.f);
+            if (v < cv.nvec) x = __ldg(&cv.vec[v]);
+            const float xs[4] = {x.x, x.y, x.z, x.w};
+            const uint64_t e0 = v * 4;
 #pragma unroll
-                for (int q = 0; q < 4; ++q) {
-                    const uint64_t e = e0 + q;
-                    const uint32_t key = magnitude_key(xs[q]);
-                    if (e >= cv.mis && e < cv.n_shift && Digit<PASS>::match(key, prefix))
-                        atomicAdd(&sh[Digit<PASS>::of(key)], 1u);
+            for (int q = 0; q < 4; ++q) {
+                const uint64_t e = e0 + q;
+                const uint32_t key = magnitude_key(xs[q]);
+                const bool on = v < cv.nvec && e >= cv.mis && e < cv.n_shift && Digit<PASS>::match(key, prefix);
+                if (PASS == 0) {
+                    // every entry counts and magnitudes crowd into a few exponent values: lanes of the warp that
+                    // hold the same digit are found with a match and the lowest of them adds their number
+                    const uint32_t digit = Digit<PASS>::of(key);
+                    const uint32_t peers = __match_any_sync(0xFFFFFFFFu, on ? digit : 0xFFFFFFFFu);
+                    if (on && (peers & ((1u << (threadIdx.x & 31)) - 1u)) == 0) atomicAdd(&sh[digit], __popc(peers));
+                } else if (on) {
+                    atomicAdd(&sh[Digit<PASS>::of(key)], 1u);                  // few entries match the prefix
                 }
             }
         }
