@@ -11,6 +11,7 @@ using namespace adacomp;
 
 namespace {
 constexpr int kSelectStages = 11;
+constexpr uint64_t kDefaultWaveBytes = 40ull << 20;      // candidate + window lists one wave may write (a third of L2)
 constexpr int kProfileRing = 32;
 const char* const kStageNames[kSelectStages] = {
     "bracket_sample", "bracket_scan", "bracket_resolve", "bracket_emit", "general_plan",
@@ -43,11 +44,18 @@ struct adacomp_select {
     uint32_t* d_win_idx = nullptr;
     uint2* d_sub_tab = nullptr;
     uint32_t* d_span_off = nullptr;
-    // optional stage timing: events around every kernel of the last call
-    // optional stage timing: a ring of event sets, one per call, folded into sums when reused or read
+    // waves: the single-pass route works through the (worker, tensor) instances in runs whose candidate and
+    // window lists fit the part of L2 set aside for them, so that the kernels after the scan read them from L2
+    std::vector<uint32_t> sparse_before, dense_before, all_before;   // [tensor]: work items of earlier tensors, per item list
+    std::vector<uint64_t> list_bytes;                                // [tensor]: expected bytes of both lists
+    std::vector<uint32_t> wave_first;                                // scratch of a call: first instance of every wave
+    uint64_t wave_bytes = 0;                                         // 0: default
+    // optional stage timing: a ring of event lists, one per call (a stage may be launched several times per
+    // call, once per wave), folded into sums when reused or read
     bool profiling = false;
-    cudaEvent_t ev[kProfileRing][kSelectStages + 1] = {};
-    bool ev_recorded[kProfileRing][kSelectStages + 1] = {};
+    struct Span { int stage; cudaEvent_t a, b; };
+    std::vector<Span> spans[kProfileRing];
+    size_t spans_used[kProfileRing] = {};
     bool ring_used[kProfileRing] = {};
     int ring_next = 0;
     double stage_ms_sum[kSelectStages] = {};
@@ -58,8 +66,10 @@ namespace {
 
 struct Layout {
     std::vector<Layer> layers;
-    std::vector<uint2> items;          // scan / emit work items: sparse-scan tensors first, then dense-scan ones
-    std::vector<uint2> dense_items;
+    std::vector<uint2> items;          // work items (tensor, first span): sparse-scan tensors, then dense-scan ones, then all by tensor
+    std::vector<uint2> dense_items, all_items;
+    std::vector<uint32_t> sparse_before, dense_before, all_before;
+    std::vector<uint64_t> list_bytes;
     uint64_t extent = 0, K = 0;
     uint64_t cand_stride = 0, win_stride = 0, span_stride = 0;
     uint32_t slots_per_worker = 0, max_sample = 0, n_items_sparse = 0;
@@ -104,6 +114,7 @@ void plan_bracket(Layer& L, Layout* out) {
     L.win_cap = static_cast<uint32_t>(win);
     L.cand_base = out->cand_stride;
     L.win_base = out->win_stride;
+    out->list_bytes.back() = static_cast<uint64_t>(8.0 * n * (lo_frac + win_frac));   // what the scan is expected to write
     out->span_stride += n_spans;
     out->cand_stride += (L.cand_cap + 63) & ~63ull;
     out->win_stride += (L.win_cap + 63) & ~63ull;
@@ -131,13 +142,23 @@ int build_layout(const adacomp_segment_t* segs, uint32_t n_segs, uint32_t max_wo
         slots += L.n_slots;
         K += s.k;
         end_prev = s.offset + s.n;
+        out->sparse_before.push_back(static_cast<uint32_t>(out->items.size()));
+        out->dense_before.push_back(static_cast<uint32_t>(out->dense_items.size()));
+        out->all_before.push_back(static_cast<uint32_t>(out->all_items.size()));
+        out->list_bytes.push_back(0);
         plan_bracket(L, out);
         if (L.bracket == kRouteSmall) out->any_small = true;
-        for (uint32_t s0 = 0; L.bracket && s0 < L.n_spans; s0 += kSpansPerBlock)
+        for (uint32_t s0 = 0; L.bracket && s0 < L.n_spans; s0 += kSpansPerBlock) {
             (L.bracket == 2 ? out->dense_items : out->items).push_back(make_uint2(l, s0));
+            out->all_items.push_back(make_uint2(l, s0));
+        }
     }
+    out->sparse_before.push_back(static_cast<uint32_t>(out->items.size()));
+    out->dense_before.push_back(static_cast<uint32_t>(out->dense_items.size()));
+    out->all_before.push_back(static_cast<uint32_t>(out->all_items.size()));
     out->n_items_sparse = static_cast<uint32_t>(out->items.size());
     out->items.insert(out->items.end(), out->dense_items.begin(), out->dense_items.end());
+    out->items.insert(out->items.end(), out->all_items.begin(), out->all_items.end());
     if (K > kMaxIndex || slots * max_workers > 0x7FFFFFFFull ||
         static_cast<uint64_t>(n_segs) * max_workers > 0x7FFFFFFFull ||
         out->span_stride * max_workers > 0x7FFFFFFFull || out->items.size() > 0x7FFFFFFFull)
@@ -171,21 +192,45 @@ size_t carve(adacomp_select_t* h, void* base, const Layout& lay, uint32_t max_wo
     return c.used;
 }
 
-// Adds the stage times of one finished (or finishing: waits for it) event set to the sums.
+// Adds the stage times of one finished (or finishing: waits for it) call to the sums.
 cudaError_t fold_profile_slot(adacomp_select_t* h, int slot) {
     if (!h->ring_used[slot]) return cudaSuccess;
-    for (int i = 0; i < kSelectStages; ++i) {
-        if (!h->ev_recorded[slot][i] || !h->ev_recorded[slot][i + 1]) continue;
-        cudaError_t e = cudaEventSynchronize(h->ev[slot][i + 1]);
+    for (size_t i = 0; i < h->spans_used[slot]; ++i) {
+        const adacomp_select::Span& sp = h->spans[slot][i];
+        cudaError_t e = cudaEventSynchronize(sp.b);
         if (e != cudaSuccess) return e;
         float ms = 0.f;
-        e = cudaEventElapsedTime(&ms, h->ev[slot][i], h->ev[slot][i + 1]);
+        e = cudaEventElapsedTime(&ms, sp.a, sp.b);
         if (e != cudaSuccess) return e;
-        h->stage_ms_sum[i] += ms;
+        h->stage_ms_sum[sp.stage] += ms;
     }
+    h->spans_used[slot] = 0;
     h->ring_used[slot] = false;
     h->profiled_calls += 1;
     return cudaSuccess;
+}
+
+// Cuts the instances [0, n_workers x tensors) of a call into waves: runs of consecutive instances whose
+// expected candidate and window lists together stay within `budget` bytes (at least one instance each).
+void plan_waves(adacomp_select_t* h, uint32_t n_workers, uint64_t budget) {
+    h->wave_first.clear();
+    h->wave_first.push_back(0);
+    const uint32_t L = h->n_layers;
+    uint64_t per_worker = 0;
+    for (uint32_t l = 0; l < L; ++l) per_worker += h->list_bytes[l];
+    if (per_worker * n_workers > budget) {
+        uint64_t in_wave = 0;
+        for (uint32_t w = 0; w < n_workers; ++w)
+            for (uint32_t l = 0; l < L; ++l) {
+                const uint64_t b = h->list_bytes[l];
+                if (in_wave && in_wave + b > budget) {
+                    h->wave_first.push_back(w * L + l);
+                    in_wave = 0;
+                }
+                in_wave += b;
+            }
+    }
+    h->wave_first.push_back(n_workers * L);
 }
 
 }  // namespace
@@ -221,7 +266,12 @@ int adacomp_select_create(adacomp_select_t** h, const adacomp_segment_t* h_segs,
     s->slots_per_worker = lay.slots_per_worker;
     s->extent = lay.extent;
     s->K = lay.K;
-    s->n_items = static_cast<uint32_t>(lay.items.size());
+    s->n_items = static_cast<uint32_t>(lay.all_items.size());
+    s->sparse_before = lay.sparse_before;
+    s->dense_before = lay.dense_before;
+    s->all_before = lay.all_before;
+    s->list_bytes = lay.list_bytes;
+    s->wave_first.reserve(static_cast<size_t>(n_segs) * max_workers + 2);
     s->n_items_sparse = lay.n_items_sparse;
     s->all_bracketed = true;
     for (const Layer& L : lay.layers)
@@ -255,6 +305,12 @@ int adacomp_select_create(adacomp_select_t** h, const adacomp_segment_t* h_segs,
     if (e == cudaSuccess) e = cudaDeviceSynchronize();
     if (e != cudaSuccess) { delete s; return cuda_fail(e); }
     *h = s;
+    return ADACOMP_OK;
+}
+
+int adacomp_select_set_wave_bytes(adacomp_select_t* h, uint64_t bytes) {
+    if (!h) return ADACOMP_ERR_INVALID;
+    h->wave_bytes = bytes;
     return ADACOMP_OK;
 }
 
@@ -305,54 +361,84 @@ int adacomp_select(adacomp_select_t* h, const float* d_grads, uint64_t worker_st
     const unsigned n_inst = n_workers * h->n_layers;
     const bool bracketed = h->route == 0 && (h->n_items > 0 || h->any_small);
     int slot = 0;
-    if (h->profiling) {                                   // take the next event set of the ring
+    if (h->profiling) {                                   // take the next event list of the ring
         slot = h->ring_next;
         h->ring_next = (h->ring_next + 1) % kProfileRing;
         ADACOMP_CUDA(fold_profile_slot(h, slot));         // its previous user finished long ago
-        for (int i = 0; i <= kSelectStages; ++i) h->ev_recorded[slot][i] = false;
         h->ring_used[slot] = true;
     }
-    // mark(i): the boundary before stage i (and after stage i - 1)
-    auto mark = [&](int i) -> cudaError_t {
+    // begin(stage) ... end(): CUDA events around one launch (only while profiling)
+    auto begin = [&](int stage) -> cudaError_t {
         if (!h->profiling) return cudaSuccess;
-        h->ev_recorded[slot][i] = true;
-        return cudaEventRecord(h->ev[slot][i], st);
+        std::vector<adacomp_select::Span>& v = h->spans[slot];
+        if (h->spans_used[slot] == v.size()) {
+            adacomp_select::Span sp = {stage, nullptr, nullptr};
+            cudaError_t e = cudaEventCreate(&sp.a);
+            if (e == cudaSuccess) e = cudaEventCreate(&sp.b);
+            if (e != cudaSuccess) return e;
+            try { v.push_back(sp); } catch (...) { return cudaErrorMemoryAllocation; }
+        }
+        v[h->spans_used[slot]].stage = stage;
+        return cudaEventRecord(v[h->spans_used[slot]].a, st);
     };
-    ADACOMP_CUDA(mark(0));
+    auto end = [&]() -> cudaError_t {
+        if (!h->profiling) return cudaSuccess;
+        return cudaEventRecord(h->spans[slot][h->spans_used[slot]++].b, st);
+    };
 
-    // bracketed route: sample -> single pass -> resolve -> emit
+    // single-pass routes: sample (and the tensors that are selected on chip), then per wave the one pass over
+    // the gradient, the exact threshold, and the ordered write
+    ADACOMP_CUDA(begin(0));
     k_bracket_sample<<<n_inst, kBig, bracketed ? h->max_sample * sizeof(uint32_t) : 0, st>>>(p, bracketed ? 0 : 1);
     ADACOMP_LAUNCH_CHECK();
-    ADACOMP_CUDA(mark(1));
+    ADACOMP_CUDA(end());
     if (bracketed && h->n_items > 0) {
-        const dim3 grid(h->n_items, n_workers);
-        if (h->n_items_sparse) {
-            k_bracket_scan<<<dim3(h->n_items_sparse, n_workers), kThreads, kScanSmemPerWarp * (kThreads / 32), st>>>(p, 0u);
+        const uint32_t L = h->n_layers;
+        const uint32_t n_sparse = h->sparse_before[L], n_dense = h->dense_before[L], n_all = h->all_before[L];
+        plan_waves(h, n_workers, h->wave_bytes ? h->wave_bytes : kDefaultWaveBytes);
+        for (size_t v = 0; v + 1 < h->wave_first.size(); ++v) {
+            const uint32_t i0 = h->wave_first[v], i1 = h->wave_first[v + 1];
+            const uint32_t w0 = i0 / L, l0 = i0 - w0 * L, w1 = i1 / L, l1 = i1 - w1 * L;
+            // work items of a list are numbered worker by worker, tensor by tensor: a wave is a range of them
+            auto range = [&](const std::vector<uint32_t>& before, uint32_t per_worker, uint32_t* first) -> uint32_t {
+                *first = w0 * per_worker + before[l0];
+                return w1 * per_worker + before[l1] - *first;
+            };
+            uint32_t first = 0, count = range(h->sparse_before, n_sparse, &first);
+            ADACOMP_CUDA(begin(1));
+            if (count) {
+                k_bracket_scan<<<count, kThreads, kScanSmemPerWarp * (kThreads / 32), st>>>(p, 0u, n_sparse, first);
+                ADACOMP_LAUNCH_CHECK();
+            }
+            count = range(h->dense_before, n_dense, &first);
+            if (count) {
+                k_bracket_scan_dense<<<count, kThreads, kDenseSmemPerWarp * (kThreads / 32), st>>>(p, n_sparse, n_dense, first);
+                ADACOMP_LAUNCH_CHECK();
+            }
+            ADACOMP_CUDA(end());
+            ADACOMP_CUDA(begin(2));
+            k_bracket_resolve<<<i1 - i0, kBig, 0, st>>>(p, i0);
             ADACOMP_LAUNCH_CHECK();
+            ADACOMP_CUDA(end());
+            count = range(h->all_before, n_all, &first);
+            ADACOMP_CUDA(begin(3));
+            if (count) {
+                k_bracket_emit<<<count, kThreads, 0, st>>>(p, n_sparse + n_dense, n_all, first);
+                ADACOMP_LAUNCH_CHECK();
+            }
+            ADACOMP_CUDA(end());
         }
-        if (h->n_items > h->n_items_sparse) {
-            k_bracket_scan_dense<<<dim3(h->n_items - h->n_items_sparse, n_workers), kThreads,
-                                   kDenseSmemPerWarp * (kThreads / 32), st>>>(p, h->n_items_sparse);
-            ADACOMP_LAUNCH_CHECK();
-        }
-        ADACOMP_CUDA(mark(2));
-        k_bracket_resolve<<<n_inst, kBig, 0, st>>>(p);
-        ADACOMP_LAUNCH_CHECK();
-        ADACOMP_CUDA(mark(3));
-        k_bracket_emit<<<grid, kThreads, 0, st>>>(p);
-        ADACOMP_LAUNCH_CHECK();
     }
-    ADACOMP_CUDA(mark(4));
 
     if (bracketed && h->all_bracketed) {
         // every tensor is on a single-pass route: only instances whose bracket missed are left, which is
         // rare, so one launch in which a block works such an instance off alone replaces the six below
         unsigned solo = static_cast<unsigned>(h->n_sms) * 2;
         if (solo > n_inst) solo = n_inst;
-        ADACOMP_CUDA(mark(10));
+        ADACOMP_CUDA(begin(10));
         k_fallback_solo<<<solo, kBig, 0, st>>>(p);
         ADACOMP_LAUNCH_CHECK();
-        ADACOMP_CUDA(mark(11));
+        ADACOMP_CUDA(end());
         return ADACOMP_OK;
     }
 
@@ -363,24 +449,30 @@ int adacomp_select(adacomp_select_t* h, const float* d_grads, uint64_t worker_st
     if (grid64 > total_slots) grid64 = total_slots;
     if (grid64 == 0) grid64 = 1;
     const unsigned grid = static_cast<unsigned>(grid64);
+    ADACOMP_CUDA(begin(4));
     k_general_plan<<<1, kThreads, 0, st>>>(p);
     ADACOMP_LAUNCH_CHECK();
-    ADACOMP_CUDA(mark(5));
+    ADACOMP_CUDA(end());
+    ADACOMP_CUDA(begin(5));
     k_general_hist<0><<<grid, kThreads, 0, st>>>(p);
     ADACOMP_LAUNCH_CHECK();
-    ADACOMP_CUDA(mark(6));
+    ADACOMP_CUDA(end());
+    ADACOMP_CUDA(begin(6));
     k_general_hist<1><<<grid, kThreads, 0, st>>>(p);
     ADACOMP_LAUNCH_CHECK();
-    ADACOMP_CUDA(mark(7));
+    ADACOMP_CUDA(end());
+    ADACOMP_CUDA(begin(7));
     k_general_hist<2><<<grid, kThreads, 0, st>>>(p);
     ADACOMP_LAUNCH_CHECK();
-    ADACOMP_CUDA(mark(8));
+    ADACOMP_CUDA(end());
+    ADACOMP_CUDA(begin(8));
     k_general_count<<<grid, kThreads, 0, st>>>(p);
     ADACOMP_LAUNCH_CHECK();
-    ADACOMP_CUDA(mark(9));
+    ADACOMP_CUDA(end());
+    ADACOMP_CUDA(begin(9));
     k_general_write<<<grid, kThreads, 0, st>>>(p);
     ADACOMP_LAUNCH_CHECK();
-    ADACOMP_CUDA(mark(10));
+    ADACOMP_CUDA(end());
     return ADACOMP_OK;
 }
 
@@ -388,9 +480,6 @@ int adacomp_select_set_profiling(adacomp_select_t* h, int on) {
     if (!h) return ADACOMP_ERR_INVALID;
     DeviceGuard guard(h->device);
     if (guard.err != cudaSuccess) return cuda_fail(guard.err);
-    if (on && !h->ev[0][0])
-        for (int r = 0; r < kProfileRing; ++r)
-            for (int i = 0; i <= kSelectStages; ++i) ADACOMP_CUDA(cudaEventCreate(&h->ev[r][i]));
     for (int r = 0; r < kProfileRing; ++r) ADACOMP_CUDA(fold_profile_slot(h, r));
     for (int i = 0; i < kSelectStages; ++i) h->stage_ms_sum[i] = 0.0;      // a fresh measurement starts here
     h->profiled_calls = 0;
@@ -399,7 +488,7 @@ int adacomp_select_set_profiling(adacomp_select_t* h, int on) {
 }
 
 int adacomp_select_profile(adacomp_select_t* h, float* h_ms_out, uint32_t n_stages, uint64_t* h_calls_out) {
-    if (!h || !h_ms_out || n_stages != kSelectStages || !h->ev[0][0]) return ADACOMP_ERR_INVALID;
+    if (!h || !h_ms_out || n_stages != kSelectStages) return ADACOMP_ERR_INVALID;
     DeviceGuard guard(h->device);
     if (guard.err != cudaSuccess) return cuda_fail(guard.err);
     for (int r = 0; r < kProfileRing; ++r) ADACOMP_CUDA(fold_profile_slot(h, r));
@@ -476,10 +565,10 @@ int adacomp_select_gather(adacomp_select_t* h, const float* d_grads, uint64_t wo
 }
 
 int adacomp_select_destroy(adacomp_select_t* h) {
-    if (h && h->ev[0][0]) {
+    if (h) {
         DeviceGuard guard(h->device);
         for (int r = 0; r < kProfileRing; ++r)
-            for (int i = 0; i <= kSelectStages; ++i) cudaEventDestroy(h->ev[r][i]);
+            for (const adacomp_select::Span& sp : h->spans[r]) { cudaEventDestroy(sp.a); cudaEventDestroy(sp.b); }
     }
     delete h;
     return ADACOMP_OK;

@@ -47,6 +47,20 @@ constexpr uint32_t kRouteSmall = 3u;                  // Layer::bracket of a ten
 constexpr uint32_t kInstBracket = 2u;                 // bracket valid, scan/emit act on the instance
 constexpr uint32_t kInstOverflow = 4u;                // a candidate or window list ran out of room
 
+// The dense gradient is read once and never again: its lines are marked to leave L2 first, so that what the
+// scan writes for the kernels that follow (candidate and window lists) is still in L2 when they read it.
+__device__ __forceinline__ uint64_t l2_policy_evict_first() {
+    uint64_t pol;
+    asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(pol));
+    return pol;
+}
+__device__ __forceinline__ float4 load_once(const float4* ptr, uint64_t pol) {
+    float4 r;
+    asm volatile("ld.global.nc.L2::cache_hint.v4.f32 {%0, %1, %2, %3}, [%4], %5;"
+                 : "=f"(r.x), "=f"(r.y), "=f"(r.z), "=f"(r.w) : "l"(ptr), "l"(pol));
+    return r;
+}
+
 // Sample ranks (1 = largest) whose keys bracket the k-th largest of n entries, from a sample of m.
 __host__ __device__ inline void bracket_ranks(uint32_t n, uint32_t k, uint32_t m, uint32_t* r_hi, uint32_t* r_lo) {
     const float p = static_cast<float>(k) / static_cast<float>(n);
@@ -285,10 +299,13 @@ __device__ __forceinline__ bool load_hits(const float4& x, float tlo_f) {
     return !(m4 < tlo_f);
 }
 
-__global__ void __launch_bounds__(kThreads, 4) k_bracket_scan(SelectParams p, uint32_t item_base) {
+__global__ void __launch_bounds__(kThreads, 4) k_bracket_scan(SelectParams p, uint32_t item_base, uint32_t per_worker,
+                                                              uint32_t g_first) {
     extern __shared__ __align__(16) unsigned char s_scan[];
-    const uint2 item = p.items[item_base + blockIdx.x];
-    const uint32_t l = item.x, w = blockIdx.y;
+    const uint32_t g = g_first + blockIdx.x, w = g / per_worker;       // work items are numbered worker by worker
+    const uint2 item = p.items[item_base + (g - w * per_worker)];
+    const uint32_t l = item.x;
+    const uint64_t once = l2_policy_evict_first();
     const Layer L = p.layers[l];
     Inst* st = &p.inst[w * p.n_layers + l];
     if (!(__ldcg(&st->flags) & kInstBracket)) return;
@@ -326,7 +343,7 @@ __global__ void __launch_bounds__(kThreads, 4) k_bracket_scan(SelectParams p, ui
     if (ss0 >= in_lo && ss0 < in_hi) {
         const float4* ptr = vec + ss0 * (kSubElems / 4) + lane;
 #pragma unroll
-        for (int i = 0; i < 8; ++i) x[i] = __ldg(ptr + i * 32);
+        for (int i = 0; i < 8; ++i) x[i] = load_once(ptr + i * 32, once);
         loaded = true;
     }
     bool saw_nan = false;
@@ -351,7 +368,7 @@ __global__ void __launch_bounds__(kThreads, 4) k_bracket_scan(SelectParams p, ui
                     h = load_hits(y, tlo_f);
                 } else {                                       // a piece at the tensor's ends: checked load, blank outside
                     const uint32_t v = ss * (kSubElems / 4) + i * 32 + lane;
-                    y = (v < nvec) ? __ldg(&vec[v]) : make_float4(0.f, 0.f, 0.f, 0.f);
+                    y = (v < nvec) ? load_once(&vec[v], once) : make_float4(0.f, 0.f, 0.f, 0.f);
                     float* ys = reinterpret_cast<float*>(&y);
 #pragma unroll
                     for (int c4 = 0; c4 < 4; ++c4)
@@ -363,7 +380,7 @@ __global__ void __launch_bounds__(kThreads, 4) k_bracket_scan(SelectParams p, ui
                     if (h) q[qn + __popc(b & lt)] = static_cast<uint16_t>(j * 256 + i * 32 + lane);
                     qn += __popc(b);
                 }
-                if (next_inside) x[i] = __ldg(nptr + i * 32);
+                if (next_inside) x[i] = load_once(nptr + i * 32, once);
             }
             loaded = next_inside;
         }
@@ -377,7 +394,7 @@ __global__ void __launch_bounds__(kThreads, 4) k_bracket_scan(SelectParams p, ui
             const uint32_t ent = q[t];
             const uint32_t pj = ent >> 8;
             const uint32_t v = (ss0 + kStep * pj) * (kSubElems / 4) + (ent & 255u);
-            const float4 y = (v < nvec) ? __ldg(&vec[v]) : make_float4(0.f, 0.f, 0.f, 0.f);
+            const float4 y = (v < nvec) ? load_once(&vec[v], once) : make_float4(0.f, 0.f, 0.f, 0.f);
             const float ys[4] = {y.x, y.y, y.z, y.w};
             uint32_t nc = 0, nw = 0;
 #pragma unroll
@@ -441,7 +458,7 @@ __global__ void __launch_bounds__(kThreads, 4) k_bracket_scan(SelectParams p, ui
             const uint32_t tot32 = __shfl_sync(0xFFFFFFFFu, sc, 31);
             if (nc) {
                 uint32_t r = (sc - cnt) & 0xFFFFu, wr = (sc - cnt) >> 16;
-                const float4 y = __ldg(&vec[v]);                 // queued loads lie inside the vector range
+                const float4 y = load_once(&vec[v], once);       // queued loads lie inside the vector range
                 const float ys[4] = {y.x, y.y, y.z, y.w};
 #pragma unroll
                 for (int c4 = 0; c4 < 4; ++c4) {
@@ -559,10 +576,13 @@ __device__ __forceinline__ void dense_place(const float4& x, float t, uint32_t& 
         : "memory");
 }
 
-__global__ void __launch_bounds__(kThreads, 4) k_bracket_scan_dense(SelectParams p, uint32_t item_base) {
+__global__ void __launch_bounds__(kThreads, 4) k_bracket_scan_dense(SelectParams p, uint32_t item_base, uint32_t per_worker,
+                                                                    uint32_t g_first) {
     extern __shared__ __align__(16) unsigned char s_scan[];
-    const uint2 item = p.items[item_base + blockIdx.x];
-    const uint32_t l = item.x, w = blockIdx.y;
+    const uint32_t g = g_first + blockIdx.x, w = g / per_worker;       // work items are numbered worker by worker
+    const uint2 item = p.items[item_base + (g - w * per_worker)];
+    const uint32_t l = item.x;
+    const uint64_t once = l2_policy_evict_first();
     const Layer L = p.layers[l];
     Inst* st = &p.inst[w * p.n_layers + l];
     if (!(__ldcg(&st->flags) & kInstBracket)) return;
@@ -672,7 +692,7 @@ __global__ void __launch_bounds__(kThreads, 4) k_bracket_scan_dense(SelectParams
 #pragma unroll
             for (int i = 0; i < 8; ++i) {
                 const uint32_t v = vec0 + i * 32 + lane;
-                x[i] = (inside || v < nvec) ? __ldg(&vec[v]) : make_float4(0.f, 0.f, 0.f, 0.f);
+                x[i] = (inside || v < nvec) ? load_once(&vec[v], once) : make_float4(0.f, 0.f, 0.f, 0.f);
             }
         }
         // ---- count and place, the lane's loads 0-3 first, then 4-7: the first half of the registers
@@ -721,7 +741,7 @@ __global__ void __launch_bounds__(kThreads, 4) k_bracket_scan_dense(SelectParams
             }
             if (next_inside) {                                 // these registers are free: the next piece's loads
 #pragma unroll
-                for (int i = 4 * h; i < 4 * h + 4; ++i) x[i] = __ldg(nptr + i * 32);
+                for (int i = 4 * h; i < 4 * h + 4; ++i) x[i] = load_once(nptr + i * 32, once);
             }
         }
         have_x = next_inside;
@@ -736,7 +756,7 @@ __global__ void __launch_bounds__(kThreads, 4) k_bracket_scan_dense(SelectParams
 
 // ---------------------------------------------------------------------------------------------
 // One block per instance: exact threshold inside the window, per-span output offsets.
-__global__ void __launch_bounds__(kBig) k_bracket_resolve(SelectParams p) {
+__global__ void __launch_bounds__(kBig) k_bracket_resolve(SelectParams p, uint32_t inst_first) {
     __shared__ uint32_t s_hist[2048];
     __shared__ uint32_t s_sel[kMaxSpans];
     __shared__ unsigned long long s_g[kGatherMax];
@@ -745,7 +765,7 @@ __global__ void __launch_bounds__(kBig) k_bracket_resolve(SelectParams p) {
     __shared__ uint32_t s_cnt;
     __shared__ unsigned long long s_cstar;
     __shared__ uint32_t s_carry;
-    const uint32_t inst = blockIdx.x;
+    const uint32_t inst = inst_first + blockIdx.x;
     const uint32_t w = inst / p.n_layers, l = inst - w * p.n_layers;
     const Layer L = p.layers[l];
     Inst* st = &p.inst[inst];
@@ -875,9 +895,11 @@ __global__ void __launch_bounds__(kBig) k_bracket_resolve(SelectParams p) {
 // ---------------------------------------------------------------------------------------------
 // grid = (scan items, workers); one warp per span: walk the candidates of its 8 pieces in index
 // order, keep those at or above the exact threshold, write them out contiguously.
-__global__ void __launch_bounds__(kThreads) k_bracket_emit(SelectParams p) {
-    const uint2 item = p.items[blockIdx.x];
-    const uint32_t l = item.x, w = blockIdx.y;
+__global__ void __launch_bounds__(kThreads) k_bracket_emit(SelectParams p, uint32_t item_base, uint32_t per_worker,
+                                                          uint32_t g_first) {
+    const uint32_t g = g_first + blockIdx.x, w = g / per_worker;       // work items are numbered worker by worker
+    const uint2 item = p.items[item_base + (g - w * per_worker)];
+    const uint32_t l = item.x;
     const Layer L = p.layers[l];
     const Inst* st = &p.inst[w * p.n_layers + l];
     if (!(__ldcg(&st->flags) & kInstBracket)) return;
@@ -939,8 +961,8 @@ __global__ void __launch_bounds__(kThreads) k_bracket_emit(SelectParams p) {
             const uint32_t b = __ballot_sync(0xFFFFFFFFu, keep);
             if (keep) {
                 const uint32_t pos = off + __popc(b & lt);
-                idx_out[pos] = glob + e[u];
-                val_out[pos] = v[u];
+                __stcs(&idx_out[pos], glob + e[u]);              // written once, read by another kernel much later
+                __stcs(&val_out[pos], v[u]);
             }
             off += __popc(b);
         }
