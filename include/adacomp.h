@@ -137,8 +137,8 @@ ADACOMP_API int adacomp_select_set_route(adacomp_select_t* h, int route);
 /* Tuning.  On the single-pass route the selections of one call are worked through in waves: runs of
  * consecutive (worker, tensor) selections whose intermediate lists (what the one pass over the gradient
  * keeps for the exact-threshold and write kernels) are expected to stay within `bytes`, so that those
- * kernels find the lists in L2 instead of DRAM.  0 = the default (40 MiB, a third of a B200's L2);
- * a value larger than everything a call writes gives one wave.  Results do not depend on it. */
+ * kernels find the lists in L2 instead of DRAM.  0 = the default: one wave per call (measured best:
+ * shorter waves leave the GPU underused between their kernels).  Results do not depend on it. */
 ADACOMP_API int adacomp_select_set_wave_bytes(adacomp_select_t* h, uint64_t bytes);
 
 /* Stage timing.  With profiling on, every adacomp_select call records CUDA events on its stream

@@ -11,7 +11,6 @@ using namespace adacomp;
 
 namespace {
 constexpr int kSelectStages = 11;
-constexpr uint64_t kDefaultWaveBytes = 40ull << 20;      // candidate + window lists one wave may write (a third of L2)
 constexpr int kProfileRing = 32;
 const char* const kStageNames[kSelectStages] = {
     "bracket_sample", "bracket_scan", "bracket_resolve", "bracket_emit", "general_plan",
@@ -395,7 +394,7 @@ int adacomp_select(adacomp_select_t* h, const float* d_grads, uint64_t worker_st
     if (bracketed && h->n_items > 0) {
         const uint32_t L = h->n_layers;
         const uint32_t n_sparse = h->sparse_before[L], n_dense = h->dense_before[L], n_all = h->all_before[L];
-        plan_waves(h, n_workers, h->wave_bytes ? h->wave_bytes : kDefaultWaveBytes);
+        plan_waves(h, n_workers, h->wave_bytes ? h->wave_bytes : ~0ull);
         for (size_t v = 0; v + 1 < h->wave_first.size(); ++v) {
             const uint32_t i0 = h->wave_first[v], i1 = h->wave_first[v + 1];
             const uint32_t w0 = i0 / L, l0 = i0 - w0 * L, w1 = i1 / L, l1 = i1 - w1 * L;

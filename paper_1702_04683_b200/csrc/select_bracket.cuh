@@ -119,12 +119,10 @@ __device__ uint32_t smem_kth_largest(const uint32_t* keys, uint32_t m, uint32_t 
         const int nb = pass == 0 ? 2048 : 1024;
         for (int b = threadIdx.x; b < 2048; b += kBig) hist[b] = 0;
         __syncthreads();
-        for (uint32_t i0 = 0; i0 < m; i0 += kBig) {
-            const uint32_t i = i0 + threadIdx.x;
-            const uint32_t key = i < m ? keys[i] : 0u;
-            const bool match = i < m && (pass == 0 || (key >> (shift + 10)) == (prefix >> (shift + 10)));
-            if (pass == 0) hist_add_aggregated(hist, (key >> shift) & (nb - 1), match);   // every key counts: crowded bins
-            else if (match) atomicAdd(&hist[(key >> shift) & (nb - 1)], 1u);
+        for (uint32_t i = threadIdx.x; i < m; i += kBig) {
+            const uint32_t key = keys[i];
+            const bool match = pass == 0 || (key >> (shift + 10)) == (prefix >> (shift + 10));
+            if (match) atomicAdd(&hist[(key >> shift) & (nb - 1)], 1u);
         }
         __syncthreads();
         uint32_t b, above, cnt;
@@ -343,7 +341,7 @@ __global__ void __launch_bounds__(kThreads, 4) k_bracket_scan(SelectParams p, ui
     if (ss0 >= in_lo && ss0 < in_hi) {
         const float4* ptr = vec + ss0 * (kSubElems / 4) + lane;
 #pragma unroll
-        for (int i = 0; i < 8; ++i) x[i] = load_once(ptr + i * 32, once);
+        for (int i = 0; i < 8; ++i) x[i] = __ldg(ptr + i * 32);
         loaded = true;
     }
     bool saw_nan = false;
@@ -368,7 +366,7 @@ __global__ void __launch_bounds__(kThreads, 4) k_bracket_scan(SelectParams p, ui
                     h = load_hits(y, tlo_f);
                 } else {                                       // a piece at the tensor's ends: checked load, blank outside
                     const uint32_t v = ss * (kSubElems / 4) + i * 32 + lane;
-                    y = (v < nvec) ? load_once(&vec[v], once) : make_float4(0.f, 0.f, 0.f, 0.f);
+                    y = (v < nvec) ? __ldg(&vec[v]) : make_float4(0.f, 0.f, 0.f, 0.f);
                     float* ys = reinterpret_cast<float*>(&y);
 #pragma unroll
                     for (int c4 = 0; c4 < 4; ++c4)
@@ -380,7 +378,7 @@ __global__ void __launch_bounds__(kThreads, 4) k_bracket_scan(SelectParams p, ui
                     if (h) q[qn + __popc(b & lt)] = static_cast<uint16_t>(j * 256 + i * 32 + lane);
                     qn += __popc(b);
                 }
-                if (next_inside) x[i] = load_once(nptr + i * 32, once);
+                if (next_inside) x[i] = __ldg(nptr + i * 32);
             }
             loaded = next_inside;
         }
@@ -394,7 +392,7 @@ __global__ void __launch_bounds__(kThreads, 4) k_bracket_scan(SelectParams p, ui
             const uint32_t ent = q[t];
             const uint32_t pj = ent >> 8;
             const uint32_t v = (ss0 + kStep * pj) * (kSubElems / 4) + (ent & 255u);
-            const float4 y = (v < nvec) ? load_once(&vec[v], once) : make_float4(0.f, 0.f, 0.f, 0.f);
+            const float4 y = (v < nvec) ? __ldg(&vec[v]) : make_float4(0.f, 0.f, 0.f, 0.f);
             const float ys[4] = {y.x, y.y, y.z, y.w};
             uint32_t nc = 0, nw = 0;
 #pragma unroll
@@ -788,25 +786,34 @@ __global__ void __launch_bounds__(kBig) k_bracket_resolve(SelectParams p, uint32
 
     // composite of a window entry = (key - t_lo) << 32 | ~index: larger = kept first (larger key,
     // then lower index)
-    // calls fn(composite, shifted index) for every window entry; four entries per thread are
-    // fetched before any is used, so their loads overlap
+    // calls fn(composite, shifted index) for every window entry; eight entries per thread are
+    // fetched before any is used, so their loads overlap (a pass over the list is bound by their latency)
     auto for_each_window = [&](auto fn) {
-        for (uint32_t i0 = threadIdx.x; i0 < n_win; i0 += kBig * 4) {
-            uint32_t key[4], idx[4];
+        constexpr int kAhead = 8;
+        for (uint32_t i0 = threadIdx.x; i0 < n_win; i0 += kBig * kAhead) {
+            uint32_t key[kAhead], idx[kAhead];
 #pragma unroll
-            for (int u = 0; u < 4; ++u) {
+            for (int u = 0; u < kAhead; ++u) {
                 const uint32_t i = i0 + u * kBig;
                 key[u] = i < n_win ? __ldcg(&win_key[i]) : 0u;
                 idx[u] = i < n_win ? __ldcg(&win_idx[i]) : 0u;
             }
 #pragma unroll
-            for (int u = 0; u < 4; ++u)
+            for (int u = 0; u < kAhead; ++u)
                 if (i0 + u * kBig < n_win)
                     fn((static_cast<unsigned long long>(key[u] - t_lo) << 32) |
                            static_cast<unsigned long long>(0xFFFFFFFFu - idx[u]),
                        idx[u]);
         }
     };
+    // kept window entries per span: counted in shared memory, or for very long tensors in the table
+    // that receives the spans' output offsets anyway.  The pass that collects the last undecided entries
+    // also counts the entries it sees above them, so the list is not read again once the threshold is known.
+    uint32_t* sel = L.n_spans <= kMaxSpans ? s_sel : span_off;
+    for (uint32_t s = threadIdx.x; s < L.n_spans; s += kBig) sel[s] = 0;
+    if (threadIdx.x == 0) s_carry = 0;
+    __syncthreads();
+    bool failed = false;
 
     unsigned long long cstar = ~0ull;                 // keep window entries with composite >= cstar
     if (need > 0) {
@@ -818,21 +825,26 @@ __global__ void __launch_bounds__(kBig) k_bracket_resolve(SelectParams p, uint32
             if (count <= kGatherMax) {                // few left: gather them and rank by brute force
                 if (threadIdx.x == 0) s_cnt = 0;
                 __syncthreads();
-                for_each_window([&](unsigned long long c, uint32_t) {
-                    if ((c >> hi_shift) == prefix) s_g[atomicAdd(&s_cnt, 1u)] = c;
+                for_each_window([&](unsigned long long c, uint32_t idx) {
+                    const unsigned long long top = c >> hi_shift;
+                    if (top == prefix) s_g[atomicAdd(&s_cnt, 1u)] = c;
+                    else if (top > prefix) atomicAdd(&sel[idx / kSpanElems], 1u);   // above the undecided ones: kept
                 });
                 __syncthreads();
+                unsigned long long mine = 0;
                 if (threadIdx.x < count) {
-                    const unsigned long long mine = s_g[threadIdx.x];
+                    mine = s_g[threadIdx.x];
                     uint32_t larger = 0;
                     for (uint32_t u = 0; u < count; ++u) larger += s_g[u] > mine ? 1u : 0u;
                     if (larger == rem - 1) s_cstar = mine;
                 }
                 __syncthreads();
                 cstar = s_cstar;
+                if (threadIdx.x < count && mine >= cstar)     // the kept ones among the collected entries
+                    atomicAdd(&sel[(0xFFFFFFFFu - static_cast<uint32_t>(mine)) / kSpanElems], 1u);
                 break;
             }
-            if (hi_shift == 0) { cstar = prefix; break; }     // cannot happen: composites are distinct
+            if (hi_shift == 0) { failed = true; break; }      // cannot happen: composites are distinct
             const int bits = hi_shift < 11 ? hi_shift : 11;
             const int new_shift = hi_shift - bits;
             for (int b = threadIdx.x; b < 2048; b += kBig) s_hist[b] = 0;
@@ -849,17 +861,6 @@ __global__ void __launch_bounds__(kBig) k_bracket_resolve(SelectParams p, uint32
             count = cnt;
             hi_shift = new_shift;
         }
-    }
-    // kept window entries per span: counted in shared memory, or for very long tensors in the table
-    // that receives the spans' output offsets anyway
-    uint32_t* sel = L.n_spans <= kMaxSpans ? s_sel : span_off;
-    for (uint32_t s = threadIdx.x; s < L.n_spans; s += kBig) sel[s] = 0;
-    if (threadIdx.x == 0) s_carry = 0;
-    __syncthreads();
-    if (need > 0) {
-        for_each_window([&](unsigned long long c, uint32_t idx) {
-            if (c >= cstar) atomicAdd(&sel[idx / kSpanElems], 1u);
-        });
     }
     __syncthreads();
     // exclusive prefix of kept entries over the spans
@@ -880,7 +881,7 @@ __global__ void __launch_bounds__(kBig) k_bracket_resolve(SelectParams p, uint32
         __syncthreads();
     }
     if (threadIdx.x == 0) {
-        if (s_carry != L.k) {
+        if (failed || s_carry != L.k) {
             st->flags = kInstGeneral;                 // defensive: counts must add up to k
         } else if (need > 0) {
             st->T = t_lo + static_cast<uint32_t>(cstar >> 32);
