@@ -49,7 +49,7 @@ def build(force: bool = False, verbose: bool = False) -> str:
     if not force and not is_stale():
         return LIB
     tmp = LIB + ".tmp.%d" % os.getpid()
-    cmd = [_nvcc(), *NVCC_FLAGS, "-I", INCLUDE, "-I", CSRC]
+    cmd = [_nvcc(), *NVCC_FLAGS, *os.environ.get("ADACOMP_NVCC_FLAGS", "").split(), "-I", INCLUDE, "-I", CSRC]
     if verbose:
         cmd += ["-Xptxas", "-v"]
     cmd += ["-o", tmp, *sources()]

@@ -9,6 +9,10 @@
 
 using namespace adacomp;
 
+#ifndef ADACOMP_DENSE_FROM
+#define ADACOMP_DENSE_FROM 0.03          // measured cross-over of the two scan kernels (build-time tunable)
+#endif
+
 namespace {
 constexpr int kSelectStages = 11;
 constexpr int kProfileRing = 32;
@@ -104,8 +108,8 @@ void plan_bracket(Layer& L, Layout* out) {
     double win = n * win_frac * (1.0 + 6.0 / std::sqrt(static_cast<double>(r_lo + 1 - r_hi))) + 2048.0;
     if (cand > n) cand = n;
     if (win > n) win = n;
-    // tensors whose candidates will be about a tenth of the entries or more take the dense scan kernel
-    L.bracket = lo_frac >= 0.03 ? 2 : 1;
+    // tensors whose candidates will be this fraction of the entries or more take the dense scan kernel
+    L.bracket = lo_frac >= ADACOMP_DENSE_FROM ? 2 : 1;
     L.sample = m;
     L.n_spans = n_spans;
     L.span_base = static_cast<uint32_t>(out->span_stride);

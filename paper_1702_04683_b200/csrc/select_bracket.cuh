@@ -495,92 +495,84 @@ __global__ void __launch_bounds__(kThreads, 4) k_bracket_scan(SelectParams p, ui
 // ---------------------------------------------------------------------------------------------
 // The same pass for tensors whose candidates are dense (a percent of the entries or more), where
 // nearly every load holds a candidate and queueing loads would only add work.  Same
-// decomposition (8 warps x 8 pieces of 1024 entries per block, warps on their own).  Per piece:
-//   count    the four components of each of the lane's loads are tested and counted, one byte per
-//            load (a compare and a predicated add per entry), and a byte-packed warp scan turns
-//            the counts into every candidate's place in index order (load, lane, component);
-//   place    a second sweep over the registers stores every candidate, value and position in one
-//            8-byte entry, at its place on a shared-memory stage behind the candidates of the
-//            pieces staged before (a compare, a predicated store and a predicated step of the
-//            address per entry: no branch).
-//   Both run for the lane's loads 0-3, whose registers are then refilled with the next piece,
-//   and again for loads 4-7.
-// Flush, once the stage could not take another piece and after the last one, while the next
-// piece's loads are in flight: a first pass with one lane per staged candidate counts the window
+// decomposition (8 warps x 8 pieces of 1024 entries per block, warps on their own), but the pieces
+// do not travel through registers: each warp keeps a ring of two 4 KB buffers in shared memory that
+// bulk asynchronous copies (cp.async.bulk, completion on an mbarrier of the warp's own) fill a piece
+// ahead, so loading costs the warp one instruction per piece.  Per piece:
+//   mask     lane L reads ITS 32 consecutive entries of the piece (eight 16-byte reads, the order of
+//            the eight rotated by the lane so that the banks are spread) and builds a 32-bit mask of
+//            its candidates: a compare and a predicated OR per entry; entries outside the tensor (the
+//            first and the last piece) are cleared from the mask, so no piece needs a path of its own;
+//   rank     population counts and one warp scan give every lane the place of its first candidate
+//            in index order (lane after lane: a lane's entries are consecutive);
+//   place    each lane walks the set bits of its mask and moves value and position, one 8-byte
+//            entry per candidate, from the piece's buffer to its place on a shared-memory stage
+//            behind the candidates staged before: work in proportion to the candidates, not to
+//            the entries.
+// Flush, when the stage cannot take the piece just counted and after the last one, while the next
+// piece's copy is in flight: a first pass with one lane per staged candidate counts the window
 // entries (those not above t_hi; also per piece, for the table) and looks for NaN; two atomics
 // reserve room in the candidate and the window list; a second pass writes both lists with
 // coalesced stores, window entries ranked by ballot.
-constexpr uint32_t kDenseStage = 768;                          // candidates the stage holds
-constexpr uint32_t kDensePiece = 512;                          // most candidates one piece (of 1024 entries) may bring
-constexpr size_t kDenseSmemPerWarp = kDenseStage * 8 + 64;
+constexpr uint32_t kDenseStage = 640;                          // candidates the stage holds; a piece that brings more is "crowded"
+constexpr uint32_t kDenseRing = 2;                             // piece buffers per warp
+constexpr uint32_t kPieceBytes = kSubElems * 4;
+constexpr size_t kDenseSmemPerWarp = kDenseRing * kPieceBytes + kDenseStage * 8 + 64 + 16;
+static_assert(kDenseSmemPerWarp % 16 == 0, "the warps' slices stay 16-byte aligned");
+constexpr uint32_t kWaitSpins = 1u << 20;                      // bounded wait for a bulk copy (each try suspends for a while)
 
-// cnt += kUnit for each of the four components with |x| >= t or unordered
-template <uint32_t kUnit>
-__device__ __forceinline__ void dense_count(const float4& x, float t, uint32_t& cnt) {
+__device__ __forceinline__ void mbar_init(uint32_t mbar, uint32_t count) {
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(mbar), "r"(count) : "memory");
+}
+__device__ __forceinline__ void mbar_expect_tx(uint32_t mbar, uint32_t bytes) {
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(mbar), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait(uint32_t mbar, uint32_t parity) {
+    uint32_t ok;
+    asm volatile(
+        "{\n\t"
+        ".reg .pred p;\n\t"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t"
+        "}"
+        : "=r"(ok) : "r"(mbar), "r"(parity) : "memory");
+    return ok != 0;
+}
+// bytes: a multiple of 16; both addresses 16-byte aligned.  No multicast: the copy lands in this block only.
+__device__ __forceinline__ void bulk_load(uint32_t smem_dst, const void* gmem_src, uint32_t bytes, uint32_t mbar) {
+    asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+                 ::"r"(smem_dst), "l"(gmem_src), "r"(bytes), "r"(mbar) : "memory");
+}
+
+// mask |= kBit << c for each of the four components c with |x| >= t or unordered
+template <uint32_t kBit>
+__device__ __forceinline__ void mask_or(const float4& x, float t, uint32_t& mask) {
     asm("{\n\t"
         ".reg .pred p;\n\t"
         ".reg .f32 a;\n\t"
         "abs.f32 a, %1;\n\t"
         "setp.geu.f32 p, a, %5;\n\t"
-        "@p add.u32 %0, %0, %6;\n\t"
+        "@p or.b32 %0, %0, %6;\n\t"
         "abs.f32 a, %2;\n\t"
         "setp.geu.f32 p, a, %5;\n\t"
-        "@p add.u32 %0, %0, %6;\n\t"
+        "@p or.b32 %0, %0, %7;\n\t"
         "abs.f32 a, %3;\n\t"
         "setp.geu.f32 p, a, %5;\n\t"
-        "@p add.u32 %0, %0, %6;\n\t"
+        "@p or.b32 %0, %0, %8;\n\t"
         "abs.f32 a, %4;\n\t"
         "setp.geu.f32 p, a, %5;\n\t"
-        "@p add.u32 %0, %0, %6;\n\t"
+        "@p or.b32 %0, %0, %9;\n\t"
         "}"
-        : "+r"(cnt)
-        : "f"(x.x), "f"(x.y), "f"(x.z), "f"(x.w), "f"(t), "n"(kUnit));
+        : "+r"(mask)
+        : "f"(x.x), "f"(x.y), "f"(x.z), "f"(x.w), "f"(t), "n"(kBit), "n"(kBit << 1), "n"(kBit << 2), "n"(kBit << 3));
 }
 
-// for each of the four components with |x| >= t or unordered: { stage[a] = (x, e); a += 8; ++e regardless }
-// a: shared-memory byte address of the next free stage entry of this lane's run; e0: position of x.x
-__device__ __forceinline__ void dense_place(const float4& x, float t, uint32_t& a, uint32_t e0) {
-    asm volatile(
-        "{\n\t"
-        ".reg .pred p;\n\t"
-        ".reg .f32 m;\n\t"
-        ".reg .b32 v, e;\n\t"
-        "abs.f32 m, %1;\n\t"
-        "setp.geu.f32 p, m, %5;\n\t"
-        "mov.b32 v, %1;\n\t"
-        "@p st.shared.v2.b32 [%0], {v, %6};\n\t"
-        "@p add.u32 %0, %0, 8;\n\t"
-        "abs.f32 m, %2;\n\t"
-        "setp.geu.f32 p, m, %5;\n\t"
-        "mov.b32 v, %2;\n\t"
-        "add.u32 e, %6, 1;\n\t"
-        "@p st.shared.v2.b32 [%0], {v, e};\n\t"
-        "@p add.u32 %0, %0, 8;\n\t"
-        "abs.f32 m, %3;\n\t"
-        "setp.geu.f32 p, m, %5;\n\t"
-        "mov.b32 v, %3;\n\t"
-        "add.u32 e, %6, 2;\n\t"
-        "@p st.shared.v2.b32 [%0], {v, e};\n\t"
-        "@p add.u32 %0, %0, 8;\n\t"
-        "abs.f32 m, %4;\n\t"
-        "setp.geu.f32 p, m, %5;\n\t"
-        "mov.b32 v, %4;\n\t"
-        "add.u32 e, %6, 3;\n\t"
-        "@p st.shared.v2.b32 [%0], {v, e};\n\t"
-        "@p add.u32 %0, %0, 8;\n\t"
-        "}"
-        : "+r"(a)
-        : "f"(x.x), "f"(x.y), "f"(x.z), "f"(x.w), "f"(t), "r"(e0)
-        : "memory");
-}
-
-__global__ void __launch_bounds__(kThreads, 4) k_bracket_scan_dense(SelectParams p, uint32_t item_base, uint32_t per_worker,
+__global__ void __launch_bounds__(kThreads, 2) k_bracket_scan_dense(SelectParams p, uint32_t item_base, uint32_t per_worker,
                                                                     uint32_t g_first) {
     extern __shared__ __align__(16) unsigned char s_scan[];
     const uint32_t g = g_first + blockIdx.x, w = g / per_worker;       // work items are numbered worker by worker
     const uint2 item = p.items[item_base + (g - w * per_worker)];
     const uint32_t l = item.x;
-    const uint64_t once = l2_policy_evict_first();
     const Layer L = p.layers[l];
     Inst* st = &p.inst[w * p.n_layers + l];
     if (!(__ldcg(&st->flags) & kInstBracket)) return;
@@ -598,19 +590,40 @@ __global__ void __launch_bounds__(kThreads, 4) k_bracket_scan_dense(SelectParams
     const uint32_t ss_end = min(item.y + kSpansPerBlock, L.n_spans) * kSubsPerSpan;
     const uint32_t ss0 = item.y * kSubsPerSpan + warp;
     if (ss0 >= ss_end) return;
-    const uint32_t in_lo = mis ? 1u : 0u, in_hi = n_shift / kSubElems;
     unsigned char* mine = s_scan + warp * kDenseSmemPerWarp;
-    uint2* stage = reinterpret_cast<uint2*>(mine);                                            // [kDenseStage] (value bits, shifted position)
-    uint32_t* s_tc = reinterpret_cast<uint32_t*>(mine + kDenseStage * 8);                      // [8] candidates per piece
+    uint2* stage = reinterpret_cast<uint2*>(mine + kDenseRing * kPieceBytes);                   // [kDenseStage] (value bits, shifted position)
+    uint32_t* s_tc = reinterpret_cast<uint32_t*>(mine + kDenseRing * kPieceBytes + kDenseStage * 8);   // [8] candidates per piece
     uint32_t* s_tw = s_tc + kBatch;                                                           // [8] window entries per piece
+    const uint32_t ring_base = static_cast<uint32_t>(__cvta_generic_to_shared(mine));
     const uint32_t stage_base = static_cast<uint32_t>(__cvta_generic_to_shared(stage));
+    const uint32_t mbar_base = stage_base + kDenseStage * 8 + 64;                             // [kDenseRing] one mbarrier per buffer
     uint32_t* cand_idx = p.cand_idx + static_cast<uint64_t>(w) * p.cand_stride + L.cand_base;
     float* cand_val = p.cand_val + static_cast<uint64_t>(w) * p.cand_stride + L.cand_base;
     uint32_t* win_key = p.win_key + static_cast<uint64_t>(w) * p.win_stride + L.win_base;
     uint32_t* win_idx = p.win_idx + static_cast<uint64_t>(w) * p.win_stride + L.win_base;
     uint2* sub_tab = p.sub_tab + (static_cast<uint64_t>(w) * p.span_stride + L.span_base) * kSubsPerSpan;
 
-    bool saw_nan = false, lost = false;                        // lost: something did not fit
+    // this warp's pieces: ss0 + kStep * j, j < n_mine; every one of them overlaps the tensor
+    uint32_t n_mine = 0;
+    while (n_mine < kBatch && ss0 + kStep * n_mine < ss_end && (ss0 + kStep * n_mine) * (kSubElems / 4) < nvec) ++n_mine;
+    if (n_mine == 0) return;
+    // the copy of piece j into buffer j % kDenseRing: the 16-byte groups of the piece that overlap the tensor
+    auto fetch = [&](uint32_t j) {
+        const uint32_t vec0 = (ss0 + kStep * j) * (kSubElems / 4);
+        const uint32_t groups = nvec - vec0 < kSubElems / 4 ? nvec - vec0 : kSubElems / 4;
+        const uint32_t mbar = mbar_base + 8u * (j % kDenseRing);
+        mbar_expect_tx(mbar, groups * 16u);
+        bulk_load(ring_base + (j % kDenseRing) * kPieceBytes, vec + vec0, groups * 16u, mbar);
+    };
+    if (lane == 0) {
+#pragma unroll
+        for (uint32_t r = 0; r < kDenseRing; ++r) mbar_init(mbar_base + 8u * r, 1u);
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        for (uint32_t j = 0; j < kDenseRing && j < n_mine; ++j) fetch(j);
+    }
+    __syncwarp();
+
+    bool saw_nan = false, lost = false;                        // lost: something did not fit, or a copy never arrived
     uint32_t staged = 0, j_first = 0;                          // candidates on the stage; first piece they belong to
     // everything staged since the last flush (pieces j_first .. j_end - 1) goes to the lists
     auto flush = [&](uint32_t j_end) {
@@ -678,77 +691,92 @@ __global__ void __launch_bounds__(kThreads, 4) k_bracket_scan_dense(SelectParams
         j_first = j_end;
     };
 
-    float4 x[8];
-    bool have_x = false;                                       // x already holds the piece about to be compacted
+    const uint32_t lane_base = lane * 128u, rot = (lane & 7u) << 4;   // the lane's 128 bytes of a buffer; its rotation of the 16-byte groups
 #pragma unroll 1
-    for (uint32_t j = 0; j < kBatch; ++j) {
-        const uint32_t ss = ss0 + kStep * j, next = ss + kStep;
-        if (ss >= ss_end) break;
-        const bool inside = ss >= in_lo && ss < in_hi;
-        const uint32_t vec0 = ss * (kSubElems / 4);
-        if (!have_x) {
-#pragma unroll
-            for (int i = 0; i < 8; ++i) {
-                const uint32_t v = vec0 + i * 32 + lane;
-                x[i] = (inside || v < nvec) ? load_once(&vec[v], once) : make_float4(0.f, 0.f, 0.f, 0.f);
+    for (uint32_t j = 0; j < n_mine; ++j) {
+        const uint32_t ss = ss0 + kStep * j;
+        const uint32_t buf = ring_base + (j % kDenseRing) * kPieceBytes;
+        {   // the copy of this piece has landed (bounded wait: a copy that never arrives must not hang the GPU)
+            const uint32_t mbar = mbar_base + 8u * (j % kDenseRing), parity = (j / kDenseRing) & 1u;
+            uint32_t spins = 0;
+            while (!mbar_try_wait(mbar, parity) && ++spins <= kWaitSpins) {}
+            if (__any_sync(0xFFFFFFFFu, spins > kWaitSpins)) {
+                // give up on the instance (the general route redoes it), but not before the copies still
+                // under way have had a second, equally bounded, chance to land: the block must not end under them
+                lost = true;
+                record_error(p.status, ADACOMP_ERR_TIMEOUT);
+                for (uint32_t jj = j; jj < n_mine && jj < j + kDenseRing; ++jj) {
+                    spins = 0;
+                    while (!mbar_try_wait(mbar_base + 8u * (jj % kDenseRing), (jj / kDenseRing) & 1u) && ++spins <= kWaitSpins) {}
+                }
+                break;
             }
         }
-        // ---- count and place, the lane's loads 0-3 first, then 4-7: the first half of the registers
-        // is refilled with the next piece while the second half is still being worked on
-        const bool next_inside = (j + 1 < kBatch) && next < ss_end && next >= in_lo && next < in_hi;
-        const float4* nptr = vec + (next_inside ? next : ss) * (kSubElems / 4) + lane;
-        const uint32_t e_lane = ss * kSubElems + lane * 4;    // shifted position of the lane's first entry of load 0
-        uint32_t tc = 0;
-        bool crowded = false;                                  // more candidates than a piece may bring
+        // ---- mask of the lane's candidates among its 32 consecutive entries
+        const uint32_t e_lane = ss * kSubElems + lane * 32u;   // shifted position of the lane's first entry
+        uint32_t mask = 0;
+        {
+            float4 q[8];
 #pragma unroll
-        for (int h = 0; h < 2; ++h) {
-            if (!inside) {                                     // first / last piece: blank what lies outside (t_lo > 0)
+            for (int i = 0; i < 8; ++i)                        // group i ^ (lane & 7) first: the eight lanes of a quarter warp hit distinct banks
+                asm volatile("ld.shared.v4.f32 {%0, %1, %2, %3}, [%4];"
+                             : "=f"(q[i].x), "=f"(q[i].y), "=f"(q[i].z), "=f"(q[i].w)
+                             : "r"(buf + lane_base + ((static_cast<uint32_t>(i) << 4) ^ rot)));
+            // q[i] holds group i ^ (lane & 7), i.e. entries 4 * (i ^ (lane & 7)) ..: the bits are put where they belong below
+            uint32_t raw = 0;                                  // bit 4 i + c: component c of q[i]
+            mask_or<1u << 0>(q[0], tlo_f, raw);  mask_or<1u << 4>(q[1], tlo_f, raw);
+            mask_or<1u << 8>(q[2], tlo_f, raw);  mask_or<1u << 12>(q[3], tlo_f, raw);
+            mask_or<1u << 16>(q[4], tlo_f, raw); mask_or<1u << 20>(q[5], tlo_f, raw);
+            mask_or<1u << 24>(q[6], tlo_f, raw); mask_or<1u << 28>(q[7], tlo_f, raw);
+            // nibble i of raw is group i ^ r of the lane (r = lane & 7): nibble g of mask = nibble g ^ r of raw.
+            // XOR with r permutes the nibbles in three steps, one per bit of r: swap neighbours, pairs, halves.
+            const uint32_t r = lane & 7u;
+            uint32_t m = raw;
+            if (r & 1u) m = ((m & 0x0F0F0F0Fu) << 4) | ((m >> 4) & 0x0F0F0F0Fu);
+            if (r & 2u) m = ((m & 0x00FF00FFu) << 8) | ((m >> 8) & 0x00FF00FFu);
+            if (r & 4u) m = (m << 16) | (m >> 16);
+            mask = m;
+        }
+        {   // entries before the tensor's first or at / after its end do not count
+            const uint32_t lo_cut = mis > e_lane ? mis - e_lane : 0u;                       // <= 3
+            const uint32_t hi_cut = n_shift > e_lane ? (n_shift - e_lane < 32u ? n_shift - e_lane : 32u) : 0u;
+            const uint32_t keep = (hi_cut == 32u ? 0xFFFFFFFFu : (1u << hi_cut) - 1u) & ~((1u << lo_cut) - 1u);
+            mask &= keep;
+        }
+        // ---- rank: where the lane's first candidate goes
+        const uint32_t cnt = __popc(mask);
+        uint32_t inc = cnt;
 #pragma unroll
-                for (int i = 4 * h; i < 4 * h + 4; ++i) {
-                    float xs[4] = {x[i].x, x[i].y, x[i].z, x[i].w};
-                    const uint32_t e0 = (vec0 + i * 32 + lane) * 4;
-#pragma unroll
-                    for (int q = 0; q < 4; ++q)
-                        if (e0 + q < mis || e0 + q >= n_shift) xs[q] = 0.f;
-                    x[i] = make_float4(xs[0], xs[1], xs[2], xs[3]);
+        for (int d = 1; d < 32; d <<= 1) {
+            const uint32_t y = __shfl_up_sync(0xFFFFFFFFu, inc, d);
+            if (lane >= static_cast<uint32_t>(d)) inc += y;
+        }
+        uint32_t tc = __shfl_sync(0xFFFFFFFFu, inc, 31);
+        if (staged + tc > kDenseStage) flush(j);               // make room first (pieces before this one)
+        if (tc > kDenseStage) { lost = true; tc = 0; }         // a crowded piece: the instance goes to the general route
+        if (tc) {
+            // ---- place: walk the set bits, value and position from the piece's buffer to the stage
+            uint32_t o = stage_base + 8u * (staged + inc - cnt);
+            uint32_t m = mask;
+            const uint32_t turns = __reduce_max_sync(0xFFFFFFFFu, cnt);
+#pragma unroll 1
+            for (uint32_t t = 0; t < turns; ++t) {
+                if (m) {
+                    const uint32_t b = __ffs(m) - 1u;
+                    m &= m - 1u;
+                    uint32_t v;
+                    asm volatile("ld.shared.b32 %0, [%1];" : "=r"(v) : "r"(buf + lane_base + (b << 2)));   // the buffer holds the piece as it is in memory
+                    asm volatile("st.shared.v2.b32 [%0], {%1, %2};" ::"r"(o), "r"(v), "r"(e_lane + b) : "memory");
+                    o += 8u;
                 }
-            }
-            uint32_t cnt = 0;                                  // candidates per load of this lane, one byte each
-            dense_count<1u>(x[4 * h], tlo_f, cnt);
-            dense_count<1u << 8>(x[4 * h + 1], tlo_f, cnt);
-            dense_count<1u << 16>(x[4 * h + 2], tlo_f, cnt);
-            dense_count<1u << 24>(x[4 * h + 3], tlo_f, cnt);
-            uint32_t inc = cnt;                                // a load holds at most 128 candidates: no byte overflows
-#pragma unroll
-            for (int d = 1; d < 32; d <<= 1) {
-                const uint32_t y = __shfl_up_sync(0xFFFFFFFFu, inc, d);
-                if (lane >= static_cast<uint32_t>(d)) inc += y;
-            }
-            const uint32_t tot = __shfl_sync(0xFFFFFFFFu, inc, 31), pre = inc - cnt;
-            const uint32_t sum = (tot & 0x00FF00FFu) + ((tot >> 8) & 0x00FF00FFu);
-            uint32_t load_off = staged + tc;                   // behind what is staged, the first half's candidates first
-            tc += (sum & 0xFFFFu) + (sum >> 16);
-            crowded = tc > kDensePiece;                        // (a half brings at most 512: the first one always fits)
-            if (!crowded) {
-#pragma unroll
-                for (int i = 4 * h; i < 4 * h + 4; ++i) {
-                    uint32_t a = stage_base + 8u * (load_off + ((pre >> ((i & 3) * 8)) & 255u));
-                    dense_place(x[i], tlo_f, a, e_lane + i * 128);
-                    load_off += (tot >> ((i & 3) * 8)) & 255u;
-                }
-            }
-            if (next_inside) {                                 // these registers are free: the next piece's loads
-#pragma unroll
-                for (int i = 4 * h; i < 4 * h + 4; ++i) x[i] = load_once(nptr + i * 32, once);
             }
         }
-        have_x = next_inside;
-        if (crowded) { lost = true; tc = 0; }
         if (lane == 0) s_tc[j] = tc;
         staged += tc;
-        __syncwarp();
-        if (staged + kDensePiece > kDenseStage || j + 1 == kBatch || next >= ss_end) flush(j + 1);
+        __syncwarp();                                          // the buffer has been read by every lane, the stage written
+        if (lane == 0 && j + kDenseRing < n_mine) fetch(j + kDenseRing);
     }
+    flush(n_mine);
     if (saw_nan || lost) atomicOr(&st->flags, kInstOverflow);
 }
 
