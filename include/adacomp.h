@@ -134,13 +134,6 @@ ADACOMP_API int adacomp_select_host(adacomp_select_t* h, const float* h_grads, u
  * 1 = general route for everything (multi-pass radix select; reads the gradient five times). */
 ADACOMP_API int adacomp_select_set_route(adacomp_select_t* h, int route);
 
-/* Tuning.  On the single-pass route the selections of one call are worked through in waves: runs of
- * consecutive (worker, tensor) selections whose intermediate lists (what the one pass over the gradient
- * keeps for the exact-threshold and write kernels) are expected to stay within `bytes`, so that those
- * kernels find the lists in L2 instead of DRAM.  0 = the default: one wave per call (measured best:
- * shorter waves leave the GPU underused between their kernels).  Results do not depend on it. */
-ADACOMP_API int adacomp_select_set_wave_bytes(adacomp_select_t* h, uint64_t bytes);
-
 /* Stage timing.  With profiling on, every adacomp_select call records CUDA events on its stream
  * around each of its kernels (a few microseconds of host work per call, no synchronisation).
  * adacomp_select_profile waits for the calls made since profiling was switched on and writes

@@ -56,7 +56,6 @@ def _load():
         "adacomp_select": (i32, [vp, vp, u64, u32, vp, vp, vp]),
         "adacomp_select_host": (i32, [vp, vp, u64, u32, vp, vp, vp, vp, vp, vp]),
         "adacomp_select_set_route": (i32, [vp, i32]),
-        "adacomp_select_set_wave_bytes": (i32, [vp, u64]),
         "adacomp_select_set_profiling": (i32, [vp, i32]),
         "adacomp_select_profile": (i32, [vp, P(f32), u32, P(u64)]),
         "adacomp_select_stage_name": (ctypes.c_char_p, [u32]),
@@ -278,10 +277,6 @@ class Selector:
     def set_route(self, route: int):
         """0 = automatic (bracketed single pass where eligible), 1 = general route only."""
         _check(_lib.adacomp_select_set_route(self._h, int(route)), "adacomp_select_set_route")
-
-    def set_wave_bytes(self, nbytes: int):
-        """Bytes of intermediate lists one wave of the single-pass route may write (0 = default)."""
-        _check(_lib.adacomp_select_set_wave_bytes(self._h, int(nbytes)), "adacomp_select_set_wave_bytes")
 
     def set_profiling(self, on: bool):
         _check(_lib.adacomp_select_set_profiling(self._h, int(on)), "adacomp_select_set_profiling")

@@ -9,10 +9,6 @@
 
 using namespace adacomp;
 
-#ifndef ADACOMP_DENSE_FROM
-#define ADACOMP_DENSE_FROM 0.03          // measured cross-over of the two scan kernels (build-time tunable)
-#endif
-
 namespace {
 constexpr int kSelectStages = 11;
 constexpr int kProfileRing = 32;
@@ -27,7 +23,7 @@ struct adacomp_select {
     int route = 0;         // 0 = automatic, 1 = general route for everything
     bool all_bracketed = false;   // every tensor with k > 0 is eligible for the bracketed route
     bool any_small = false;       // some tensor is selected whole in shared memory by the sample kernel
-    uint32_t n_layers = 0, max_workers = 0, slots_per_worker = 0, n_items = 0, n_items_sparse = 0, max_sample = 0;
+    uint32_t n_layers = 0, max_workers = 0, slots_per_worker = 0, n_items = 0, max_sample = 0;
     uint64_t extent = 0;   // one past the last entry any segment covers
     uint64_t K = 0;        // pairs per worker
     uint64_t cand_stride = 0, win_stride = 0, span_stride = 0;
@@ -47,14 +43,7 @@ struct adacomp_select {
     uint32_t* d_win_idx = nullptr;
     uint2* d_sub_tab = nullptr;
     uint32_t* d_span_off = nullptr;
-    // waves: the single-pass route works through the (worker, tensor) instances in runs whose candidate and
-    // window lists fit the part of L2 set aside for them, so that the kernels after the scan read them from L2
-    std::vector<uint32_t> sparse_before, dense_before, all_before;   // [tensor]: work items of earlier tensors, per item list
-    std::vector<uint64_t> list_bytes;                                // [tensor]: expected bytes of both lists
-    std::vector<uint32_t> wave_first;                                // scratch of a call: first instance of every wave
-    uint64_t wave_bytes = 0;                                         // 0: default
-    // optional stage timing: a ring of event lists, one per call (a stage may be launched several times per
-    // call, once per wave), folded into sums when reused or read
+    // optional stage timing: a ring of event lists, one per call, folded into sums when reused or read
     bool profiling = false;
     struct Span { int stage; cudaEvent_t a, b; };
     std::vector<Span> spans[kProfileRing];
@@ -69,13 +58,10 @@ namespace {
 
 struct Layout {
     std::vector<Layer> layers;
-    std::vector<uint2> items;          // work items (tensor, first span): sparse-scan tensors, then dense-scan ones, then all by tensor
-    std::vector<uint2> dense_items, all_items;
-    std::vector<uint32_t> sparse_before, dense_before, all_before;
-    std::vector<uint64_t> list_bytes;
+    std::vector<uint2> items;          // scan / emit work items: (tensor, first span)
     uint64_t extent = 0, K = 0;
     uint64_t cand_stride = 0, win_stride = 0, span_stride = 0;
-    uint32_t slots_per_worker = 0, max_sample = 0, n_items_sparse = 0;
+    uint32_t slots_per_worker = 0, max_sample = 0;
     bool any_small = false;            // some tensor is selected whole in shared memory by the sample kernel
 };
 
@@ -108,8 +94,7 @@ void plan_bracket(Layer& L, Layout* out) {
     double win = n * win_frac * (1.0 + 6.0 / std::sqrt(static_cast<double>(r_lo + 1 - r_hi))) + 2048.0;
     if (cand > n) cand = n;
     if (win > n) win = n;
-    // tensors whose candidates will be this fraction of the entries or more take the dense scan kernel
-    L.bracket = lo_frac >= ADACOMP_DENSE_FROM ? 2 : 1;
+    L.bracket = 1;
     L.sample = m;
     L.n_spans = n_spans;
     L.span_base = static_cast<uint32_t>(out->span_stride);
@@ -117,7 +102,6 @@ void plan_bracket(Layer& L, Layout* out) {
     L.win_cap = static_cast<uint32_t>(win);
     L.cand_base = out->cand_stride;
     L.win_base = out->win_stride;
-    out->list_bytes.back() = static_cast<uint64_t>(8.0 * n * (lo_frac + win_frac));   // what the scan is expected to write
     out->span_stride += n_spans;
     out->cand_stride += (L.cand_cap + 63) & ~63ull;
     out->win_stride += (L.win_cap + 63) & ~63ull;
@@ -145,23 +129,10 @@ int build_layout(const adacomp_segment_t* segs, uint32_t n_segs, uint32_t max_wo
         slots += L.n_slots;
         K += s.k;
         end_prev = s.offset + s.n;
-        out->sparse_before.push_back(static_cast<uint32_t>(out->items.size()));
-        out->dense_before.push_back(static_cast<uint32_t>(out->dense_items.size()));
-        out->all_before.push_back(static_cast<uint32_t>(out->all_items.size()));
-        out->list_bytes.push_back(0);
         plan_bracket(L, out);
         if (L.bracket == kRouteSmall) out->any_small = true;
-        for (uint32_t s0 = 0; L.bracket && s0 < L.n_spans; s0 += kSpansPerBlock) {
-            (L.bracket == 2 ? out->dense_items : out->items).push_back(make_uint2(l, s0));
-            out->all_items.push_back(make_uint2(l, s0));
-        }
+        for (uint32_t s0 = 0; L.bracket == 1 && s0 < L.n_spans; s0 += kSpansPerBlock) out->items.push_back(make_uint2(l, s0));
     }
-    out->sparse_before.push_back(static_cast<uint32_t>(out->items.size()));
-    out->dense_before.push_back(static_cast<uint32_t>(out->dense_items.size()));
-    out->all_before.push_back(static_cast<uint32_t>(out->all_items.size()));
-    out->n_items_sparse = static_cast<uint32_t>(out->items.size());
-    out->items.insert(out->items.end(), out->dense_items.begin(), out->dense_items.end());
-    out->items.insert(out->items.end(), out->all_items.begin(), out->all_items.end());
     if (K > kMaxIndex || slots * max_workers > 0x7FFFFFFFull ||
         static_cast<uint64_t>(n_segs) * max_workers > 0x7FFFFFFFull ||
         out->span_stride * max_workers > 0x7FFFFFFFull || out->items.size() > 0x7FFFFFFFull)
@@ -213,29 +184,6 @@ cudaError_t fold_profile_slot(adacomp_select_t* h, int slot) {
     return cudaSuccess;
 }
 
-// Cuts the instances [0, n_workers x tensors) of a call into waves: runs of consecutive instances whose
-// expected candidate and window lists together stay within `budget` bytes (at least one instance each).
-void plan_waves(adacomp_select_t* h, uint32_t n_workers, uint64_t budget) {
-    h->wave_first.clear();
-    h->wave_first.push_back(0);
-    const uint32_t L = h->n_layers;
-    uint64_t per_worker = 0;
-    for (uint32_t l = 0; l < L; ++l) per_worker += h->list_bytes[l];
-    if (per_worker * n_workers > budget) {
-        uint64_t in_wave = 0;
-        for (uint32_t w = 0; w < n_workers; ++w)
-            for (uint32_t l = 0; l < L; ++l) {
-                const uint64_t b = h->list_bytes[l];
-                if (in_wave && in_wave + b > budget) {
-                    h->wave_first.push_back(w * L + l);
-                    in_wave = 0;
-                }
-                in_wave += b;
-            }
-    }
-    h->wave_first.push_back(n_workers * L);
-}
-
 }  // namespace
 
 extern "C" {
@@ -269,13 +217,7 @@ int adacomp_select_create(adacomp_select_t** h, const adacomp_segment_t* h_segs,
     s->slots_per_worker = lay.slots_per_worker;
     s->extent = lay.extent;
     s->K = lay.K;
-    s->n_items = static_cast<uint32_t>(lay.all_items.size());
-    s->sparse_before = lay.sparse_before;
-    s->dense_before = lay.dense_before;
-    s->all_before = lay.all_before;
-    s->list_bytes = lay.list_bytes;
-    s->wave_first.reserve(static_cast<size_t>(n_segs) * max_workers + 2);
-    s->n_items_sparse = lay.n_items_sparse;
+    s->n_items = static_cast<uint32_t>(lay.items.size());
     s->all_bracketed = true;
     for (const Layer& L : lay.layers)
         if (L.k > 0 && !L.bracket) s->all_bracketed = false;
@@ -301,19 +243,10 @@ int adacomp_select_create(adacomp_select_t** h, const adacomp_segment_t* h_segs,
                                  static_cast<int>(kSmallMax * sizeof(uint32_t)));
     if (e == cudaSuccess)
         e = cudaFuncSetAttribute(k_bracket_scan, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                 static_cast<int>(kScanSmemPerWarp * (kThreads / 32)));
-    if (e == cudaSuccess)
-        e = cudaFuncSetAttribute(k_bracket_scan_dense, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                  static_cast<int>(kDenseSmemPerWarp * (kThreads / 32)));
     if (e == cudaSuccess) e = cudaDeviceSynchronize();
     if (e != cudaSuccess) { delete s; return cuda_fail(e); }
     *h = s;
-    return ADACOMP_OK;
-}
-
-int adacomp_select_set_wave_bytes(adacomp_select_t* h, uint64_t bytes) {
-    if (!h) return ADACOMP_ERR_INVALID;
-    h->wave_bytes = bytes;
     return ADACOMP_OK;
 }
 
@@ -389,48 +322,26 @@ int adacomp_select(adacomp_select_t* h, const float* d_grads, uint64_t worker_st
         return cudaEventRecord(h->spans[slot][h->spans_used[slot]++].b, st);
     };
 
-    // single-pass routes: sample (and the tensors that are selected on chip), then per wave the one pass over
-    // the gradient, the exact threshold, and the ordered write
+    // single-pass routes: sample (and the tensors that are selected on chip), the one pass over the gradient,
+    // the exact threshold, the ordered write
     ADACOMP_CUDA(begin(0));
     k_bracket_sample<<<n_inst, kBig, bracketed ? h->max_sample * sizeof(uint32_t) : 0, st>>>(p, bracketed ? 0 : 1);
     ADACOMP_LAUNCH_CHECK();
     ADACOMP_CUDA(end());
     if (bracketed && h->n_items > 0) {
-        const uint32_t L = h->n_layers;
-        const uint32_t n_sparse = h->sparse_before[L], n_dense = h->dense_before[L], n_all = h->all_before[L];
-        plan_waves(h, n_workers, h->wave_bytes ? h->wave_bytes : ~0ull);
-        for (size_t v = 0; v + 1 < h->wave_first.size(); ++v) {
-            const uint32_t i0 = h->wave_first[v], i1 = h->wave_first[v + 1];
-            const uint32_t w0 = i0 / L, l0 = i0 - w0 * L, w1 = i1 / L, l1 = i1 - w1 * L;
-            // work items of a list are numbered worker by worker, tensor by tensor: a wave is a range of them
-            auto range = [&](const std::vector<uint32_t>& before, uint32_t per_worker, uint32_t* first) -> uint32_t {
-                *first = w0 * per_worker + before[l0];
-                return w1 * per_worker + before[l1] - *first;
-            };
-            uint32_t first = 0, count = range(h->sparse_before, n_sparse, &first);
-            ADACOMP_CUDA(begin(1));
-            if (count) {
-                k_bracket_scan<<<count, kThreads, kScanSmemPerWarp * (kThreads / 32), st>>>(p, 0u, n_sparse, first);
-                ADACOMP_LAUNCH_CHECK();
-            }
-            count = range(h->dense_before, n_dense, &first);
-            if (count) {
-                k_bracket_scan_dense<<<count, kThreads, kDenseSmemPerWarp * (kThreads / 32), st>>>(p, n_sparse, n_dense, first);
-                ADACOMP_LAUNCH_CHECK();
-            }
-            ADACOMP_CUDA(end());
-            ADACOMP_CUDA(begin(2));
-            k_bracket_resolve<<<i1 - i0, kBig, 0, st>>>(p, i0);
-            ADACOMP_LAUNCH_CHECK();
-            ADACOMP_CUDA(end());
-            count = range(h->all_before, n_all, &first);
-            ADACOMP_CUDA(begin(3));
-            if (count) {
-                k_bracket_emit<<<count, kThreads, 0, st>>>(p, n_sparse + n_dense, n_all, first);
-                ADACOMP_LAUNCH_CHECK();
-            }
-            ADACOMP_CUDA(end());
-        }
+        const dim3 grid(h->n_items, n_workers);
+        ADACOMP_CUDA(begin(1));
+        k_bracket_scan<<<grid, kThreads, kDenseSmemPerWarp * (kThreads / 32), st>>>(p);
+        ADACOMP_LAUNCH_CHECK();
+        ADACOMP_CUDA(end());
+        ADACOMP_CUDA(begin(2));
+        k_bracket_resolve<<<n_inst, kBig, 0, st>>>(p);
+        ADACOMP_LAUNCH_CHECK();
+        ADACOMP_CUDA(end());
+        ADACOMP_CUDA(begin(3));
+        k_bracket_emit<<<grid, kThreads, 0, st>>>(p);
+        ADACOMP_LAUNCH_CHECK();
+        ADACOMP_CUDA(end());
     }
 
     if (bracketed && h->all_bracketed) {

@@ -5,15 +5,13 @@
 //   k_bracket_sample   per (worker, tensor): read a stratified sample, take two of its order
 //                      statistics t_lo <= t_hi chosen so that, with overwhelming probability,
 //                      #{key > t_hi} <= k <= #{key >= t_lo};
-//   k_bracket_scan     the single pass over the gradient (k_bracket_scan_dense for tensors where
-//                      a tenth or more of the entries are candidates).  Every warp works on its
-//                      own: it streams 1024-entry pieces, reserves room with one 64-bit atomic
-//                      per round of up to 8 pieces and appends, in index order, the entries with
-//                      key >= t_lo ("candidates", about 1.1-2.5 k of them per tensor) to the
-//                      instance's candidate list; candidates with key <= t_hi (the "window",
-//                      where the threshold must lie) also go to a small unordered list; a table
-//                      records where each piece put its candidates and how many of them are
-//                      above the window;
+//   k_bracket_scan     the single pass over the gradient.  Every warp works on its own: its pieces of
+//                      1024 entries arrive in shared memory by bulk asynchronous copies, every lane masks
+//                      its 32 consecutive entries, and the entries with key >= t_lo ("candidates", about
+//                      1.1-2.5 k of them per tensor) are appended, in index order, to the instance's
+//                      candidate list; candidates with key <= t_hi (the "window", where the threshold
+//                      must lie) also go to a small unordered list; a table records where each piece put
+//                      its candidates and how many of them are above the window;
 //   k_bracket_resolve  per instance: verify the bracket with the exact counts, find the exact
 //                      threshold inside the window (radix select on (key, index) composites,
 //                      finished by brute force once few entries remain), count the kept window
@@ -46,20 +44,6 @@ constexpr int kBig = 1024;                            // threads of the per-inst
 constexpr uint32_t kRouteSmall = 3u;                  // Layer::bracket of a tensor that is selected whole in shared memory
 constexpr uint32_t kInstBracket = 2u;                 // bracket valid, scan/emit act on the instance
 constexpr uint32_t kInstOverflow = 4u;                // a candidate or window list ran out of room
-
-// The dense gradient is read once and never again: its lines are marked to leave L2 first, so that what the
-// scan writes for the kernels that follow (candidate and window lists) is still in L2 when they read it.
-__device__ __forceinline__ uint64_t l2_policy_evict_first() {
-    uint64_t pol;
-    asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(pol));
-    return pol;
-}
-__device__ __forceinline__ float4 load_once(const float4* ptr, uint64_t pol) {
-    float4 r;
-    asm volatile("ld.global.nc.L2::cache_hint.v4.f32 {%0, %1, %2, %3}, [%4], %5;"
-                 : "=f"(r.x), "=f"(r.y), "=f"(r.z), "=f"(r.w) : "l"(ptr), "l"(pol));
-    return r;
-}
 
 // Sample ranks (1 = largest) whose keys bracket the k-th largest of n entries, from a sample of m.
 __host__ __device__ inline void bracket_ranks(uint32_t n, uint32_t k, uint32_t m, uint32_t* r_hi, uint32_t* r_lo) {
@@ -260,249 +244,18 @@ __global__ void __launch_bounds__(kBig) k_bracket_sample(SelectParams p, int gen
 }
 
 // ---------------------------------------------------------------------------------------------
-// max(a, b) that returns NaN if either input is NaN (fmaxf would drop the NaN).
-__device__ __forceinline__ float max_nan(float a, float b) {
-    float r;
-    asm("max.NaN.f32 %0, %1, %2;" : "=f"(r) : "f"(a), "f"(b));
-    return r;
-}
-
-// The single pass over the gradient.  grid = (scan items, workers); an item is up to
-// kSpansPerBlock consecutive spans of one tensor = 64 pieces of 1024 entries, and each of the 8
-// warps of a block takes 8 of them (round robin), entirely on its own: no block-level barrier.
-// A warp reads a piece with 8 coalesced float4 loads per lane, so index order is (piece, load,
-// lane, component).
-//   Streaming.  The four magnitudes of a load are reduced to their maximum and compared once
-//   with t_lo (for non-NaN data |x| >= t as floats is the integer test on the key; a NaN
-//   propagates through the maximum and counts as a hit).  One ballot per load tells the warp
-//   whether any lane hit; the loads that hit are queued (their position only, 2 bytes) in the
-//   warp's slice of shared memory, in index order.  As soon as a load has been tested its
-//   registers are refilled with the same load of the warp's next piece, so a warp always has
-//   4 KB in flight.
-//   Tail, once per round (a round ends after 8 pieces, or earlier once ~100 loads are queued, so
-//   that what the tail fetches again is still in L1 / L2), with work proportional to the queued
-//   loads and every lane busy.  Pass A fetches the queued loads again, classifies their entries
-//   (candidate: key >= t_lo; window: also key <= t_hi; bounds-checked) and counts per piece.  One
-//   64-bit atomic then reserves room in both lists for the whole round.  Pass B ranks the queue
-//   with warp scans, stages candidates and window entries in shared memory and copies them out
-//   with coalesced stores; 8 lanes write the pieces' table entries.
-// The first and last piece of a tensor use checked loads.  A NaN hands the instance to the
-// general route, which works on bit patterns only.
-constexpr uint32_t kScanQueue = 768;                           // queued loads per warp and round
-constexpr uint32_t kScanStage = 128;                           // entries staged per copy step (32 loads x 4)
-constexpr size_t kScanSmemPerWarp = kScanQueue * 3 + 32 + kScanStage * 16;
-
-__device__ __forceinline__ bool load_hits(const float4& x, float tlo_f) {
-    const float m4 = max_nan(max_nan(fabsf(x.x), fabsf(x.y)), max_nan(fabsf(x.z), fabsf(x.w)));
-    return !(m4 < tlo_f);
-}
-
-__global__ void __launch_bounds__(kThreads, 4) k_bracket_scan(SelectParams p, uint32_t item_base, uint32_t per_worker,
-                                                              uint32_t g_first) {
-    extern __shared__ __align__(16) unsigned char s_scan[];
-    const uint32_t g = g_first + blockIdx.x, w = g / per_worker;       // work items are numbered worker by worker
-    const uint2 item = p.items[item_base + (g - w * per_worker)];
-    const uint32_t l = item.x;
-    const uint64_t once = l2_policy_evict_first();
-    const Layer L = p.layers[l];
-    Inst* st = &p.inst[w * p.n_layers + l];
-    if (!(__ldcg(&st->flags) & kInstBracket)) return;
-    const uint32_t t_hi = __ldcg(&st->t_hi);
-    const float tlo_f = __uint_as_float(__ldcg(&st->t_lo)), thi_f = __uint_as_float(t_hi);
-    const float* first = p.grads + static_cast<uint64_t>(w) * p.stride + L.offset;
-    const uint32_t mis = static_cast<uint32_t>((reinterpret_cast<uintptr_t>(first) >> 2) & 3u);
-    const float4* vec = reinterpret_cast<const float4*>(first - mis);
-    const uint32_t n_shift = L.n + mis;                        // n <= kBracketMaxN on this route
-    const uint32_t nvec = (n_shift + 3) >> 2;
-    const uint32_t lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-    const uint32_t lt = (1u << lane) - 1u;
-    constexpr uint32_t kStep = kThreads / 32;                  // pieces between two pieces of one warp
-    constexpr uint32_t kBatch = kSpansPerBlock * kSubsPerSpan / kStep;   // pieces per warp: 8
-    const uint32_t ss_end = min(item.y + kSpansPerBlock, L.n_spans) * kSubsPerSpan;
-    const uint32_t ss0 = item.y * kSubsPerSpan + warp;         // this warp's pieces: ss0 + kStep * j
-    if (ss0 >= ss_end) return;
-    // pieces [in_lo, in_hi) lie entirely inside the tensor: no bounds checks needed
-    const uint32_t in_lo = mis ? 1u : 0u, in_hi = n_shift / kSubElems;
-    unsigned char* mine = s_scan + warp * kScanSmemPerWarp;
-    uint32_t* stage_idx = reinterpret_cast<uint32_t*>(mine);                        // [kScanStage]
-    float* stage_val = reinterpret_cast<float*>(mine + kScanStage * 4);             // [kScanStage]
-    uint32_t* stage_widx = reinterpret_cast<uint32_t*>(mine + kScanStage * 8);      // [kScanStage]
-    uint32_t* stage_wkey = reinterpret_cast<uint32_t*>(mine + kScanStage * 12);     // [kScanStage]
-    uint32_t* s_cnt = reinterpret_cast<uint32_t*>(mine + kScanStage * 16);          // [8] per piece: cand | win << 16
-    uint16_t* q = reinterpret_cast<uint16_t*>(mine + kScanStage * 16 + 32);         // queued load: j * 256 + i * 32 + lane
-    unsigned char* info = mine + kScanStage * 16 + 32 + kScanQueue * 2;             // candidate nibble | window nibble << 4
-    uint32_t* cand_idx = p.cand_idx + static_cast<uint64_t>(w) * p.cand_stride + L.cand_base;
-    float* cand_val = p.cand_val + static_cast<uint64_t>(w) * p.cand_stride + L.cand_base;
-    uint32_t* win_key = p.win_key + static_cast<uint64_t>(w) * p.win_stride + L.win_base;
-    uint32_t* win_idx = p.win_idx + static_cast<uint64_t>(w) * p.win_stride + L.win_base;
-
-    float4 x[8];
-    bool loaded = false;                                       // x holds the piece about to be tested
-    if (ss0 >= in_lo && ss0 < in_hi) {
-        const float4* ptr = vec + ss0 * (kSubElems / 4) + lane;
-#pragma unroll
-        for (int i = 0; i < 8; ++i) x[i] = __ldg(ptr + i * 32);
-        loaded = true;
-    }
-    bool saw_nan = false;
-    uint32_t j = 0;
-    while (j < kBatch && ss0 + kStep * j < ss_end) {
-        // ================= one round: stream pieces until the queue could overflow
-        uint32_t qn = 0;                                       // queued loads (warp-uniform)
-        if (lane < kBatch) s_cnt[lane] = 0;
-        __syncwarp();
-#pragma unroll 1
-        for (; j < kBatch && qn + 256 <= kScanQueue && qn < 96; ++j) {
-            const uint32_t ss = ss0 + kStep * j, next = ss + kStep;
-            if (ss >= ss_end) break;
-            const bool next_inside = (j + 1 < kBatch) && next < ss_end && next >= in_lo && next < in_hi;
-            const float4* nptr = vec + (next_inside ? next : ss0) * (kSubElems / 4) + lane;   // ss0: any valid address
-#pragma unroll
-            for (int i = 0; i < 8; ++i) {
-                float4 y;
-                bool h;
-                if (loaded) {
-                    y = x[i];
-                    h = load_hits(y, tlo_f);
-                } else {                                       // a piece at the tensor's ends: checked load, blank outside
-                    const uint32_t v = ss * (kSubElems / 4) + i * 32 + lane;
-                    y = (v < nvec) ? __ldg(&vec[v]) : make_float4(0.f, 0.f, 0.f, 0.f);
-                    float* ys = reinterpret_cast<float*>(&y);
-#pragma unroll
-                    for (int c4 = 0; c4 < 4; ++c4)
-                        if (v * 4 + c4 < mis || v * 4 + c4 >= n_shift) ys[c4] = 0.f;    // t_lo > 0: never a candidate
-                    h = load_hits(y, tlo_f);
-                }
-                const uint32_t b = __ballot_sync(0xFFFFFFFFu, h);
-                if (b) {                                       // queue the loads that hit; they are classified in the tail
-                    if (h) q[qn + __popc(b & lt)] = static_cast<uint16_t>(j * 256 + i * 32 + lane);
-                    qn += __popc(b);
-                }
-                if (next_inside) x[i] = __ldg(nptr + i * 32);
-            }
-            loaded = next_inside;
-        }
-        __syncwarp();
-        if (!qn) continue;                                     // the table entries stay (0, 0)
-
-        // ================= tail, pass A: fetch the queued loads again (an L1 / L2 hit: the round is
-        // short), classify their entries with every lane busy, count per piece
-        #pragma unroll 1
-        for (uint32_t t = lane; t < qn; t += 32) {
-            const uint32_t ent = q[t];
-            const uint32_t pj = ent >> 8;
-            const uint32_t v = (ss0 + kStep * pj) * (kSubElems / 4) + (ent & 255u);
-            const float4 y = (v < nvec) ? __ldg(&vec[v]) : make_float4(0.f, 0.f, 0.f, 0.f);
-            const float ys[4] = {y.x, y.y, y.z, y.w};
-            uint32_t nc = 0, nw = 0;
-#pragma unroll
-            for (int c4 = 0; c4 < 4; ++c4) {
-                const uint32_t e = v * 4 + c4;
-                const float a = fabsf(ys[c4]);
-                const bool cand = (e >= mis && e < n_shift) && !(a < tlo_f);
-                saw_nan |= cand && (a != a);
-                if (cand) nc |= 1u << c4;
-                if (cand && !(a > thi_f)) nw |= 1u << c4;
-            }
-            info[t] = static_cast<unsigned char>(nc | (nw << 4));
-            if (nc) atomicAdd(&s_cnt[pj], __popc(nc) | (__popc(nw) << 16));
-        }
-        __syncwarp();
-
-        // ================= tail: reserve once for the round, then rank and write
-        const uint32_t mycnt = lane < kBatch ? s_cnt[lane] : 0u;
-        uint32_t inc = mycnt;
-#pragma unroll
-        for (int d = 1; d < static_cast<int>(kBatch); d <<= 1) {
-            const uint32_t y = __shfl_up_sync(0xFFFFFFFFu, inc, d);
-            if (lane >= static_cast<uint32_t>(d)) inc += y;
-        }
-        const uint32_t tot = __shfl_sync(0xFFFFFFFFu, inc, kBatch - 1);
-        const uint32_t total_c = tot & 0xFFFFu, total_w = tot >> 16;
-        if (!total_c) continue;
-        unsigned long long old = 0;
-        if (lane == 0)
-            old = atomicAdd(reinterpret_cast<unsigned long long*>(&st->cand_count),
-                            static_cast<unsigned long long>(total_c) | (static_cast<unsigned long long>(total_w) << 32));
-        old = __shfl_sync(0xFFFFFFFFu, old, 0);
-        const uint32_t cb = static_cast<uint32_t>(old), wb = static_cast<uint32_t>(old >> 32);
-        if ((static_cast<uint64_t>(cb) + total_c > L.cand_cap) || (static_cast<uint64_t>(wb) + total_w > L.win_cap)) {
-            if (lane == 0) atomicOr(&st->flags, kInstOverflow);
-            continue;
-        }
-        if (lane < kBatch && (mycnt & 0xFFFFu)) {
-            const uint32_t tc = mycnt & 0xFFFFu, tw = mycnt >> 16;
-            p.sub_tab[(static_cast<uint64_t>(w) * p.span_stride + L.span_base) * kSubsPerSpan + ss0 + kStep * lane] =
-                make_uint2(cb + ((inc - mycnt) & 0xFFFFu), tc | ((tc - tw) << 16));
-        }
-        uint32_t run = cb, wrun = wb;
-        #pragma unroll 1
-        for (uint32_t t0 = 0; t0 < qn; t0 += 32) {
-            const uint32_t t = t0 + lane;
-            uint32_t nc = 0, nw = 0, v = 0;
-            if (t < qn) {
-                const uint32_t ent = q[t], inf = info[t];
-                nc = inf & 15u;
-                nw = inf >> 4;
-                v = (ss0 + kStep * (ent >> 8)) * (kSubElems / 4) + (ent & 255u);
-            }
-            const uint32_t cnt = __popc(nc) | (__popc(nw) << 16);
-            uint32_t sc = cnt;
-#pragma unroll
-            for (int d = 1; d < 32; d <<= 1) {
-                const uint32_t y = __shfl_up_sync(0xFFFFFFFFu, sc, d);
-                if (lane >= static_cast<uint32_t>(d)) sc += y;
-            }
-            const uint32_t tot32 = __shfl_sync(0xFFFFFFFFu, sc, 31);
-            if (nc) {
-                uint32_t r = (sc - cnt) & 0xFFFFu, wr = (sc - cnt) >> 16;
-                const float4 y = load_once(&vec[v], once);       // queued loads lie inside the vector range
-                const float ys[4] = {y.x, y.y, y.z, y.w};
-#pragma unroll
-                for (int c4 = 0; c4 < 4; ++c4) {
-                    if ((nc >> c4) & 1u) {
-                        stage_idx[r] = v * 4 + c4;               // shifted coordinate inside the tensor
-                        stage_val[r] = ys[c4];
-                        ++r;
-                        if ((nw >> c4) & 1u) {
-                            stage_widx[wr] = v * 4 + c4;
-                            stage_wkey[wr] = magnitude_key(ys[c4]);
-                            ++wr;
-                        }
-                    }
-                }
-            }
-            __syncwarp();
-            const uint32_t n_c = tot32 & 0xFFFFu, n_w = tot32 >> 16;
-            #pragma unroll 1
-            for (uint32_t r = lane; r < n_c; r += 32) {
-                cand_idx[run + r] = stage_idx[r];
-                cand_val[run + r] = stage_val[r];
-            }
-            #pragma unroll 1
-            for (uint32_t r = lane; r < n_w; r += 32) {
-                win_idx[wrun + r] = stage_widx[r];
-                win_key[wrun + r] = stage_wkey[r];
-            }
-            __syncwarp();
-            run += n_c;
-            wrun += n_w;
-        }
-    }
-    if (saw_nan) atomicOr(&st->flags, kInstOverflow);
-}
-
-// ---------------------------------------------------------------------------------------------
-// The same pass for tensors whose candidates are dense (a percent of the entries or more), where
-// nearly every load holds a candidate and queueing loads would only add work.  Same
-// decomposition (8 warps x 8 pieces of 1024 entries per block, warps on their own), but the pieces
-// do not travel through registers: each warp keeps a ring of two 4 KB buffers in shared memory that
-// bulk asynchronous copies (cp.async.bulk, completion on an mbarrier of the warp's own) fill a piece
-// ahead, so loading costs the warp one instruction per piece.  Per piece:
+// The single pass over the gradient.  A work item is up to kSpansPerBlock consecutive spans of one
+// tensor = 64 pieces of 1024 entries, and each of the 8 warps of a block takes 8 of them (round robin),
+// entirely on its own: no block-level barrier.  The pieces do not travel through registers: each warp
+// keeps a ring of two 4 KB buffers in shared memory that bulk asynchronous copies (cp.async.bulk,
+// completion on an mbarrier of the warp's own) fill a piece ahead, so loading costs the warp one
+// instruction per piece.  Per piece:
 //   mask     lane L reads ITS 32 consecutive entries of the piece (eight 16-byte reads, the order of
 //            the eight rotated by the lane so that the banks are spread) and builds a 32-bit mask of
-//            its candidates: a compare and a predicated OR per entry; entries outside the tensor (the
-//            first and the last piece) are cleared from the mask, so no piece needs a path of its own;
+//            its candidates (key >= t_lo; for non-NaN data |x| >= t as floats is the integer test on
+//            the key, and a NaN counts as a candidate): a compare and a predicated OR per entry;
+//            entries outside the tensor (the first and the last piece) are cleared from the mask, so
+//            no piece needs a path of its own;
 //   rank     population counts and one warp scan give every lane the place of its first candidate
 //            in index order (lane after lane: a lane's entries are consecutive);
 //   place    each lane walks the set bits of its mask and moves value and position, one 8-byte
@@ -513,8 +266,12 @@ __global__ void __launch_bounds__(kThreads, 4) k_bracket_scan(SelectParams p, ui
 // piece's copy is in flight: a first pass with one lane per staged candidate counts the window
 // entries (those not above t_hi; also per piece, for the table) and looks for NaN; two atomics
 // reserve room in the candidate and the window list; a second pass writes both lists with
-// coalesced stores, window entries ranked by ballot.
-constexpr uint32_t kDenseStage = 640;                          // candidates the stage holds; a piece that brings more is "crowded"
+// coalesced stores, window entries ranked by ballot.  A piece with more candidates than the stage
+// holds (a stretch of large entries) goes to the lists directly, each lane writing its own.
+// Candidates stay in index order inside a piece; the table records, per piece, where its candidates
+// are in the list, how many, and how many of them lie above the window.  A NaN hands the instance to
+// the general route, which works on bit patterns only.
+constexpr uint32_t kDenseStage = 640;                          // candidates the stage holds; a piece that brings more is written directly
 constexpr uint32_t kDenseRing = 2;                             // piece buffers per warp
 constexpr uint32_t kPieceBytes = kSubElems * 4;
 constexpr size_t kDenseSmemPerWarp = kDenseRing * kPieceBytes + kDenseStage * 8 + 64 + 16;
@@ -567,12 +324,10 @@ __device__ __forceinline__ void mask_or(const float4& x, float t, uint32_t& mask
         : "f"(x.x), "f"(x.y), "f"(x.z), "f"(x.w), "f"(t), "n"(kBit), "n"(kBit << 1), "n"(kBit << 2), "n"(kBit << 3));
 }
 
-__global__ void __launch_bounds__(kThreads, 2) k_bracket_scan_dense(SelectParams p, uint32_t item_base, uint32_t per_worker,
-                                                                    uint32_t g_first) {
+__global__ void __launch_bounds__(kThreads, 2) k_bracket_scan(SelectParams p) {
     extern __shared__ __align__(16) unsigned char s_scan[];
-    const uint32_t g = g_first + blockIdx.x, w = g / per_worker;       // work items are numbered worker by worker
-    const uint2 item = p.items[item_base + (g - w * per_worker)];
-    const uint32_t l = item.x;
+    const uint2 item = p.items[blockIdx.x];
+    const uint32_t l = item.x, w = blockIdx.y;
     const Layer L = p.layers[l];
     Inst* st = &p.inst[w * p.n_layers + l];
     if (!(__ldcg(&st->flags) & kInstBracket)) return;
@@ -753,7 +508,48 @@ __global__ void __launch_bounds__(kThreads, 2) k_bracket_scan_dense(SelectParams
         }
         uint32_t tc = __shfl_sync(0xFFFFFFFFu, inc, 31);
         if (staged + tc > kDenseStage) flush(j);               // make room first (pieces before this one)
-        if (tc > kDenseStage) { lost = true; tc = 0; }         // a crowded piece: the instance goes to the general route
+        if (tc > kDenseStage) {
+            // ---- a crowded piece does not fit the stage: its candidates go to the lists directly, every lane
+            // its own run (rare: a stretch in which most entries are large)
+            uint32_t wcnt = 0;
+            for (uint32_t m = mask; m; m &= m - 1u) {
+                const float a = fabsf(*reinterpret_cast<const float*>(mine + (j % kDenseRing) * kPieceBytes + lane_base + ((__ffs(m) - 1u) << 2)));
+                saw_nan |= a != a;
+                wcnt += !(a > thi_f) ? 1u : 0u;
+            }
+            uint32_t winc = wcnt;
+#pragma unroll
+            for (int d = 1; d < 32; d <<= 1) {
+                const uint32_t y = __shfl_up_sync(0xFFFFFFFFu, winc, d);
+                if (lane >= static_cast<uint32_t>(d)) winc += y;
+            }
+            const uint32_t tw = __shfl_sync(0xFFFFFFFFu, winc, 31);
+            uint32_t old_c = 0, old_w = 0;
+            if (lane == 0) {
+                old_c = atomicAdd(&st->cand_count, tc);
+                if (tw) old_w = atomicAdd(&st->win_count, tw);
+            }
+            const uint32_t cb = __shfl_sync(0xFFFFFFFFu, old_c, 0), wb = __shfl_sync(0xFFFFFFFFu, old_w, 0);
+            if (lane == 0) sub_tab[ss] = make_uint2(cb, tc | ((tc - tw) << 16));
+            if (static_cast<uint64_t>(cb) + tc > L.cand_cap || static_cast<uint64_t>(wb) + tw > L.win_cap) {
+                lost = true;
+            } else {
+                uint32_t o = cb + inc - cnt, wo = wb + winc - wcnt;
+                for (uint32_t m = mask; m; m &= m - 1u) {
+                    const uint32_t b = __ffs(m) - 1u;
+                    const float v = *reinterpret_cast<const float*>(mine + (j % kDenseRing) * kPieceBytes + lane_base + (b << 2));
+                    cand_idx[o] = e_lane + b;
+                    cand_val[o] = v;
+                    ++o;
+                    if (!(fabsf(v) > thi_f)) {
+                        win_idx[wo] = e_lane + b;
+                        win_key[wo] = magnitude_key(v);
+                        ++wo;
+                    }
+                }
+            }
+            tc = 0;                                            // nothing of this piece is on the stage or in a later flush
+        }
         if (tc) {
             // ---- place: walk the set bits, value and position from the piece's buffer to the stage
             uint32_t o = stage_base + 8u * (staged + inc - cnt);
@@ -782,7 +578,7 @@ __global__ void __launch_bounds__(kThreads, 2) k_bracket_scan_dense(SelectParams
 
 // ---------------------------------------------------------------------------------------------
 // One block per instance: exact threshold inside the window, per-span output offsets.
-__global__ void __launch_bounds__(kBig) k_bracket_resolve(SelectParams p, uint32_t inst_first) {
+__global__ void __launch_bounds__(kBig) k_bracket_resolve(SelectParams p) {
     __shared__ uint32_t s_hist[2048];
     __shared__ uint32_t s_sel[kMaxSpans];
     __shared__ unsigned long long s_g[kGatherMax];
@@ -791,7 +587,7 @@ __global__ void __launch_bounds__(kBig) k_bracket_resolve(SelectParams p, uint32
     __shared__ uint32_t s_cnt;
     __shared__ unsigned long long s_cstar;
     __shared__ uint32_t s_carry;
-    const uint32_t inst = inst_first + blockIdx.x;
+    const uint32_t inst = blockIdx.x;
     const uint32_t w = inst / p.n_layers, l = inst - w * p.n_layers;
     const Layer L = p.layers[l];
     Inst* st = &p.inst[inst];
@@ -924,11 +720,9 @@ __global__ void __launch_bounds__(kBig) k_bracket_resolve(SelectParams p, uint32
 // ---------------------------------------------------------------------------------------------
 // grid = (scan items, workers); one warp per span: walk the candidates of its 8 pieces in index
 // order, keep those at or above the exact threshold, write them out contiguously.
-__global__ void __launch_bounds__(kThreads) k_bracket_emit(SelectParams p, uint32_t item_base, uint32_t per_worker,
-                                                          uint32_t g_first) {
-    const uint32_t g = g_first + blockIdx.x, w = g / per_worker;       // work items are numbered worker by worker
-    const uint2 item = p.items[item_base + (g - w * per_worker)];
-    const uint32_t l = item.x;
+__global__ void __launch_bounds__(kThreads) k_bracket_emit(SelectParams p) {
+    const uint2 item = p.items[blockIdx.x];
+    const uint32_t l = item.x, w = blockIdx.y;
     const Layer L = p.layers[l];
     const Inst* st = &p.inst[w * p.n_layers + l];
     if (!(__ldcg(&st->flags) & kInstBracket)) return;
