@@ -134,6 +134,12 @@ ADACOMP_API int adacomp_select_host(adacomp_select_t* h, const float* h_grads, u
  * 1 = general route for everything (multi-pass radix select; reads the gradient five times). */
 ADACOMP_API int adacomp_select_set_route(adacomp_select_t* h, int route);
 
+/* How the handle's layout is mapped on this device: h_info_out[0] = tensors on the cluster route (large
+ * tensors selected by one thread-block cluster each, everything between the one pass over the gradient and
+ * the ordered write kept in the cluster's shared memory), [1] = blocks per cluster, [2] = buffers per warp
+ * in its ring of bulk copies, [3] = clusters the device keeps resident.  All 0 if no tensor is on that route. */
+ADACOMP_API int adacomp_select_route_info(const adacomp_select_t* h, uint32_t* h_info_out);
+
 /* Stage timing.  With profiling on, every adacomp_select call records CUDA events on its stream
  * around each of its kernels (a few microseconds of host work per call, no synchronisation).
  * adacomp_select_profile waits for the calls made since profiling was switched on and writes

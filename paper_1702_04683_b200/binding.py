@@ -56,6 +56,7 @@ def _load():
         "adacomp_select": (i32, [vp, vp, u64, u32, vp, vp, vp]),
         "adacomp_select_host": (i32, [vp, vp, u64, u32, vp, vp, vp, vp, vp, vp]),
         "adacomp_select_set_route": (i32, [vp, i32]),
+        "adacomp_select_route_info": (i32, [vp, P(u32)]),
         "adacomp_select_set_profiling": (i32, [vp, i32]),
         "adacomp_select_profile": (i32, [vp, P(f32), u32, P(u64)]),
         "adacomp_select_stage_name": (ctypes.c_char_p, [u32]),
@@ -277,6 +278,13 @@ class Selector:
     def set_route(self, route: int):
         """0 = automatic (bracketed single pass where eligible), 1 = general route only."""
         _check(_lib.adacomp_select_set_route(self._h, int(route)), "adacomp_select_set_route")
+
+    def route_info(self) -> dict:
+        """Tensors on the cluster route and the cluster shape chosen on this device."""
+        info = (ctypes.c_uint32 * 4)()
+        _check(_lib.adacomp_select_route_info(self._h, info), "adacomp_select_route_info")
+        return {"cluster_tensors": int(info[0]), "blocks_per_cluster": int(info[1]), "ring_slots": int(info[2]),
+                "resident_clusters": int(info[3])}
 
     def set_profiling(self, on: bool):
         _check(_lib.adacomp_select_set_profiling(self._h, int(on)), "adacomp_select_set_profiling")

@@ -5,7 +5,7 @@
 #include <new>
 #include <vector>
 
-#include "select_bracket.cuh"
+#include "select_cluster.cuh"
 
 using namespace adacomp;
 
@@ -23,6 +23,11 @@ struct adacomp_select {
     int route = 0;         // 0 = automatic, 1 = general route for everything
     bool all_bracketed = false;   // every tensor with k > 0 is eligible for the bracketed route
     bool any_small = false;       // some tensor is selected whole in shared memory by the sample kernel
+    // cluster route: large tensors selected by one thread-block cluster each, everything between the pass and the write on chip
+    uint32_t n_cl = 0;            // tensors on the cluster route
+    uint32_t cl_ctas = 0, cl_ring = 0, cl_qmax = 0, cl_smem = 0;   // blocks per cluster, ring slots per warp, most pieces per block, shared memory per block
+    int cl_active = 0;            // clusters the device keeps resident
+    uint32_t* d_cl_layers = nullptr;
     uint32_t n_layers = 0, max_workers = 0, slots_per_worker = 0, n_items = 0, max_sample = 0;
     uint64_t extent = 0;   // one past the last entry any segment covers
     uint64_t K = 0;        // pairs per worker
@@ -59,6 +64,7 @@ namespace {
 struct Layout {
     std::vector<Layer> layers;
     std::vector<uint2> items;          // scan / emit work items: (tensor, first span)
+    std::vector<double> cand_frac;     // [tensor] expected fraction of candidates (0: not on a bracketed route)
     uint64_t extent = 0, K = 0;
     uint64_t cand_stride = 0, win_stride = 0, span_stride = 0;
     uint32_t slots_per_worker = 0, max_sample = 0;
@@ -95,6 +101,7 @@ void plan_bracket(Layer& L, Layout* out) {
     if (cand > n) cand = n;
     if (win > n) win = n;
     L.bracket = 1;
+    out->cand_frac.back() = lo_frac;
     L.sample = m;
     L.n_spans = n_spans;
     L.span_base = static_cast<uint32_t>(out->span_stride);
@@ -106,6 +113,80 @@ void plan_bracket(Layer& L, Layout* out) {
     out->cand_stride += (L.cand_cap + 63) & ~63ull;
     out->win_stride += (L.win_cap + 63) & ~63ull;
     if (m > out->max_sample) out->max_sample = m;
+}
+
+// Work items of the list route's scan and emit kernels: the tensors whose Layer::bracket is 1.
+void build_items(Layout* out) {
+    out->items.clear();
+    for (uint32_t l = 0; l < out->layers.size(); ++l) {
+        const Layer& L = out->layers[l];
+        for (uint32_t s0 = 0; L.bracket == 1 && s0 < L.n_spans; s0 += kSpansPerBlock) out->items.push_back(make_uint2(l, s0));
+    }
+}
+
+// Chooses the tensors of the cluster route on this device: bracketed tensors of at least kClMinN entries whose
+// expected candidates (with a margin) fit the value stores of a cluster.  Clusters of 8 blocks if every such
+// tensor fits them, else of 16 where the device takes clusters of that size; what fits neither stays on the
+// list route.  Fills h->cl_* and re-labels the chosen layers; returns their indices.
+std::vector<uint32_t> plan_cluster_route(adacomp_select_t* h, Layout* lay, int device) {
+    std::vector<uint32_t> chosen;
+    int smem_optin = 0;
+    if (cudaDeviceGetAttribute(&smem_optin, cudaDevAttrMaxSharedMemoryPerBlockOptin, device) != cudaSuccess || smem_optin < 160 * 1024)
+        return chosen;
+    std::vector<uint32_t> large;
+    for (uint32_t l = 0; l < lay->layers.size(); ++l)
+        if (lay->layers[l].bracket == 1 && lay->layers[l].n >= kClMinN) large.push_back(l);
+    if (large.empty()) return chosen;
+    auto pieces_of = [&](uint32_t l) { return (lay->layers[l].n + 3u + kClPiece - 1u) / kClPiece; };
+    // does tensor l fit clusters of C blocks with `ring` ring slots per warp when no block holds more than q_max pieces?
+    auto fits = [&](uint32_t l, uint32_t C, uint32_t ring, uint32_t q_max) {
+        const ClusterLayout y = cluster_layout(ring, q_max, static_cast<uint32_t>(smem_optin));
+        const double per_block = lay->layers[l].n * lay->cand_frac[l] / C;
+        return per_block * 1.12 + 1024.0 <= static_cast<double>(y.vals_cap);
+    };
+    // how many clusters of C blocks stay resident (0: the device does not take them)
+    auto resident = [&](uint32_t C) -> int {
+        if (cudaFuncSetAttribute(k_select_cluster, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_optin) != cudaSuccess) return 0;
+        if (C > 8 && cudaFuncSetAttribute(k_select_cluster, cudaFuncAttributeNonPortableClusterSizeAllowed, 1) != cudaSuccess) return 0;
+        cudaLaunchConfig_t cfg = {};
+        cfg.gridDim = dim3(C);
+        cfg.blockDim = dim3(kClThreads);
+        cfg.dynamicSmemBytes = static_cast<size_t>(smem_optin);
+        cudaLaunchAttribute at[1];
+        at[0].id = cudaLaunchAttributeClusterDimension;
+        at[0].val.clusterDim.x = C;
+        at[0].val.clusterDim.y = 1;
+        at[0].val.clusterDim.z = 1;
+        cfg.attrs = at;
+        cfg.numAttrs = 1;
+        int n = 0;
+        if (cudaOccupancyMaxActiveClusters(&n, k_select_cluster, &cfg) != cudaSuccess) { cudaGetLastError(); return 0; }
+        return n;
+    };
+    uint32_t best_C = 0, best_ring = 0, best_q = 0;
+    std::vector<uint32_t> best_set;
+    for (uint32_t C : {8u, 16u}) {
+        uint32_t q_max = 0;
+        for (uint32_t l : large) q_max = std::max(q_max, (pieces_of(l) + C - 1) / C);
+        for (uint32_t ring : {3u, 2u}) {
+            if (!cluster_layout_ok(ring, q_max)) continue;
+            std::vector<uint32_t> set;
+            for (uint32_t l : large) if (fits(l, C, ring, q_max)) set.push_back(l);
+            if (set.size() > best_set.size()) { best_set = set; best_C = C; best_ring = ring; best_q = q_max; }
+        }
+        if (best_set.size() == large.size()) break;        // everything fits: no need for larger clusters
+    }
+    if (best_set.empty()) return chosen;
+    const int n_resident = resident(best_C);
+    if (n_resident < 1) return chosen;
+    h->cl_ctas = best_C;
+    h->cl_ring = best_ring;
+    h->cl_qmax = best_q;
+    h->cl_smem = static_cast<uint32_t>(smem_optin);
+    h->cl_active = n_resident;
+    for (uint32_t l : best_set) lay->layers[l].bracket = kRouteCluster;
+    build_items(lay);
+    return best_set;
 }
 
 int build_layout(const adacomp_segment_t* segs, uint32_t n_segs, uint32_t max_workers, Layout* out) {
@@ -129,10 +210,11 @@ int build_layout(const adacomp_segment_t* segs, uint32_t n_segs, uint32_t max_wo
         slots += L.n_slots;
         K += s.k;
         end_prev = s.offset + s.n;
+        out->cand_frac.push_back(0.0);
         plan_bracket(L, out);
         if (L.bracket == kRouteSmall) out->any_small = true;
-        for (uint32_t s0 = 0; L.bracket == 1 && s0 < L.n_spans; s0 += kSpansPerBlock) out->items.push_back(make_uint2(l, s0));
     }
+    build_items(out);
     if (K > kMaxIndex || slots * max_workers > 0x7FFFFFFFull ||
         static_cast<uint64_t>(n_segs) * max_workers > 0x7FFFFFFFull ||
         out->span_stride * max_workers > 0x7FFFFFFFull || out->items.size() > 0x7FFFFFFFull)
@@ -163,6 +245,7 @@ size_t carve(adacomp_select_t* h, void* base, const Layout& lay, uint32_t max_wo
     h->d_win_idx = c.take<uint32_t>(lay.win_stride * W);
     h->d_sub_tab = c.take<uint2>(lay.span_stride * W * kSubsPerSpan + 1);
     h->d_span_off = c.take<uint32_t>(lay.span_stride * W + 1);
+    h->d_cl_layers = c.take<uint32_t>(lay.layers.size());
     return c.used;
 }
 
@@ -229,6 +312,14 @@ int adacomp_select_create(adacomp_select_t** h, const adacomp_segment_t* h_segs,
     DeviceGuard guard(device);
     cudaError_t e = guard.err;
     if (e == cudaSuccess) e = cudaDeviceGetAttribute(&s->n_sms, cudaDevAttrMultiProcessorCount, device);
+    std::vector<uint32_t> cl_layers;
+    if (e == cudaSuccess) {
+        try { cl_layers = plan_cluster_route(s, &lay, device); } catch (...) { delete s; return ADACOMP_ERR_ALLOC; }
+        s->n_cl = static_cast<uint32_t>(cl_layers.size());
+        s->n_items = static_cast<uint32_t>(lay.items.size());
+    }
+    if (e == cudaSuccess && !cl_layers.empty())
+        e = cudaMemcpy(s->d_cl_layers, cl_layers.data(), cl_layers.size() * sizeof(uint32_t), cudaMemcpyHostToDevice);
     // only the bookkeeping needs clearing; the candidate / window lists are write-before-read
     if (e == cudaSuccess) {
         const size_t head = reinterpret_cast<char*>(s->d_items) - static_cast<char*>(d_workspace);
@@ -247,6 +338,15 @@ int adacomp_select_create(adacomp_select_t** h, const adacomp_segment_t* h_segs,
     if (e == cudaSuccess) e = cudaDeviceSynchronize();
     if (e != cudaSuccess) { delete s; return cuda_fail(e); }
     *h = s;
+    return ADACOMP_OK;
+}
+
+int adacomp_select_route_info(const adacomp_select_t* h, uint32_t* h_info_out) {
+    if (!h || !h_info_out) return ADACOMP_ERR_INVALID;
+    h_info_out[0] = h->n_cl;
+    h_info_out[1] = h->cl_ctas;
+    h_info_out[2] = h->cl_ring;
+    h_info_out[3] = static_cast<uint32_t>(h->cl_active);
     return ADACOMP_OK;
 }
 
@@ -295,7 +395,7 @@ int adacomp_select(adacomp_select_t* h, const float* d_grads, uint64_t worker_st
     p.span_stride = h->span_stride;
 
     const unsigned n_inst = n_workers * h->n_layers;
-    const bool bracketed = h->route == 0 && (h->n_items > 0 || h->any_small);
+    const bool bracketed = h->route == 0 && (h->n_items > 0 || h->any_small || h->n_cl > 0);
     int slot = 0;
     if (h->profiling) {                                   // take the next event list of the ring
         slot = h->ring_next;
@@ -340,6 +440,29 @@ int adacomp_select(adacomp_select_t* h, const float* d_grads, uint64_t worker_st
         ADACOMP_CUDA(end());
         ADACOMP_CUDA(begin(3));
         k_bracket_emit<<<grid, kThreads, 0, st>>>(p);
+        ADACOMP_LAUNCH_CHECK();
+        ADACOMP_CUDA(end());
+    }
+
+    if (bracketed && h->n_cl > 0) {
+        // cluster route: persistent clusters, one (worker, tensor) instance at a time
+        const uint64_t n_ord = static_cast<uint64_t>(n_workers) * h->n_cl;
+        const uint32_t n_clusters = static_cast<uint32_t>(n_ord < static_cast<uint64_t>(h->cl_active) ? n_ord : h->cl_active);
+        cudaLaunchConfig_t cfg = {};
+        cfg.gridDim = dim3(n_clusters * h->cl_ctas);
+        cfg.blockDim = dim3(kClThreads);
+        cfg.dynamicSmemBytes = h->cl_smem;
+        cfg.stream = st;
+        cudaLaunchAttribute at[1];
+        at[0].id = cudaLaunchAttributeClusterDimension;
+        at[0].val.clusterDim.x = h->cl_ctas;
+        at[0].val.clusterDim.y = 1;
+        at[0].val.clusterDim.z = 1;
+        cfg.attrs = at;
+        cfg.numAttrs = 1;
+        ADACOMP_CUDA(begin(1));
+        ADACOMP_CUDA(cudaLaunchKernelEx(&cfg, k_select_cluster, p, static_cast<const uint32_t*>(h->d_cl_layers), h->n_cl, h->cl_ring,
+                                        h->cl_qmax, h->cl_smem));
         ADACOMP_LAUNCH_CHECK();
         ADACOMP_CUDA(end());
     }

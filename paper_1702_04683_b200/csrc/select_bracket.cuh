@@ -240,7 +240,8 @@ __global__ void __launch_bounds__(kBig) k_bracket_sample(SelectParams p, int gen
     // the scan compares magnitudes as floats and blanks padding with zeros: it needs a positive,
     // non-NaN lower bound
     const bool usable = t_lo != 0 && t_lo <= 0x7F800000u;
-    if (threadIdx.x == 0) { st->t_lo = t_lo; st->t_hi = t_hi; st->flags = usable ? kInstBracket : kInstGeneral; }
+    // a tensor on the cluster route (Layer::bracket == 2) is marked for the cluster kernel, the others for scan / resolve / emit
+    if (threadIdx.x == 0) { st->t_lo = t_lo; st->t_hi = t_hi; st->flags = usable ? (L.bracket == 2u ? 8u : kInstBracket) : kInstGeneral; }
 }
 
 // ---------------------------------------------------------------------------------------------
