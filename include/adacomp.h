@@ -131,13 +131,19 @@ ADACOMP_API int adacomp_select_host(adacomp_select_t* h, const float* h_grads, u
  *     sample brackets the threshold, then the gradient is read once); shorter tensors are
  *     selected whole in shared memory (read once); instances whose bracket turns out wrong (or
  *     that hold a NaN), and longer tensors with k > n/4, take the general route;
- * 1 = general route for everything (multi-pass radix select; reads the gradient five times). */
+ * 1 = general route for everything (multi-pass radix select; reads the gradient five times);
+ * 2 = as 0, but tensors of a million entries or more whose candidates fit take the cluster route: one
+ *     thread-block cluster per (worker, tensor) keeps masks and candidate values in its distributed
+ *     shared memory between the single pass and the ordered write, so DRAM sees the gradient once and
+ *     the output once and nothing else.  Measured slower than 0 on a B200 (its blocks can hold fewer
+ *     warps, and a cluster's steps run one after the other), hence not the default. */
 ADACOMP_API int adacomp_select_set_route(adacomp_select_t* h, int route);
 
 /* How the handle's layout is mapped on this device: h_info_out[0] = tensors on the cluster route (large
  * tensors selected by one thread-block cluster each, everything between the one pass over the gradient and
  * the ordered write kept in the cluster's shared memory), [1] = blocks per cluster, [2] = buffers per warp
- * in its ring of bulk copies, [3] = clusters the device keeps resident.  All 0 if no tensor is on that route. */
+ * in its ring of bulk copies + 256 x warps per block, [3] = clusters the device keeps resident.  All 0 if
+ * no tensor is on that route. */
 ADACOMP_API int adacomp_select_route_info(const adacomp_select_t* h, uint32_t* h_info_out);
 
 /* Stage timing.  With profiling on, every adacomp_select call records CUDA events on its stream

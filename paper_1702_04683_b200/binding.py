@@ -283,8 +283,8 @@ class Selector:
         """Tensors on the cluster route and the cluster shape chosen on this device."""
         info = (ctypes.c_uint32 * 4)()
         _check(_lib.adacomp_select_route_info(self._h, info), "adacomp_select_route_info")
-        return {"cluster_tensors": int(info[0]), "blocks_per_cluster": int(info[1]), "ring_slots": int(info[2]),
-                "resident_clusters": int(info[3])}
+        return {"cluster_tensors": int(info[0]), "blocks_per_cluster": int(info[1]), "ring_slots": int(info[2]) & 255,
+                "warps_per_block": int(info[2]) >> 8, "resident_clusters": int(info[3])}
 
     def set_profiling(self, on: bool):
         _check(_lib.adacomp_select_set_profiling(self._h, int(on)), "adacomp_select_set_profiling")

@@ -25,7 +25,7 @@ struct adacomp_select {
     bool any_small = false;       // some tensor is selected whole in shared memory by the sample kernel
     // cluster route: large tensors selected by one thread-block cluster each, everything between the pass and the write on chip
     uint32_t n_cl = 0;            // tensors on the cluster route
-    uint32_t cl_ctas = 0, cl_ring = 0, cl_qmax = 0, cl_smem = 0;   // blocks per cluster, ring slots per warp, most pieces per block, shared memory per block
+    uint32_t cl_ctas = 0, cl_warps = 0, cl_ring = 0, cl_qmax = 0, cl_smem = 0;   // blocks per cluster, warps per block, ring slots per warp, most pieces per block, shared memory per block
     int cl_active = 0;            // clusters the device keeps resident
     uint32_t* d_cl_layers = nullptr;
     uint32_t n_layers = 0, max_workers = 0, slots_per_worker = 0, n_items = 0, max_sample = 0;
@@ -76,6 +76,7 @@ struct Layout {
 // quantiles; exceeding them is not an error, it only sends the instance to the general route.
 void plan_bracket(Layer& L, Layout* out) {
     L.bracket = 0;
+    L.cluster = L.pad = 0;
     L.sample = L.n_spans = L.span_base = L.cand_cap = L.win_cap = 0;
     L.cand_base = L.win_base = 0;
     if (L.n < kBracketMinN || L.n > kBracketMaxN || L.k == 0 || static_cast<uint64_t>(L.k) * 4 > L.n) {
@@ -138,19 +139,19 @@ std::vector<uint32_t> plan_cluster_route(adacomp_select_t* h, Layout* lay, int d
         if (lay->layers[l].bracket == 1 && lay->layers[l].n >= kClMinN) large.push_back(l);
     if (large.empty()) return chosen;
     auto pieces_of = [&](uint32_t l) { return (lay->layers[l].n + 3u + kClPiece - 1u) / kClPiece; };
-    // does tensor l fit clusters of C blocks with `ring` ring slots per warp when no block holds more than q_max pieces?
-    auto fits = [&](uint32_t l, uint32_t C, uint32_t ring, uint32_t q_max) {
-        const ClusterLayout y = cluster_layout(ring, q_max, static_cast<uint32_t>(smem_optin));
+    // does tensor l fit clusters of C blocks of n_warps warps with `ring` ring slots per warp when no block holds more than q_max pieces?
+    auto fits = [&](uint32_t l, uint32_t C, uint32_t n_warps, uint32_t ring, uint32_t q_max) {
+        const ClusterLayout y = cluster_layout(n_warps, ring, q_max, static_cast<uint32_t>(smem_optin));
         const double per_block = lay->layers[l].n * lay->cand_frac[l] / C;
         return per_block * 1.12 + 1024.0 <= static_cast<double>(y.vals_cap);
     };
     // how many clusters of C blocks stay resident (0: the device does not take them)
-    auto resident = [&](uint32_t C) -> int {
+    auto resident = [&](uint32_t C, uint32_t n_warps) -> int {
         if (cudaFuncSetAttribute(k_select_cluster, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_optin) != cudaSuccess) return 0;
         if (C > 8 && cudaFuncSetAttribute(k_select_cluster, cudaFuncAttributeNonPortableClusterSizeAllowed, 1) != cudaSuccess) return 0;
         cudaLaunchConfig_t cfg = {};
         cfg.gridDim = dim3(C);
-        cfg.blockDim = dim3(kClThreads);
+        cfg.blockDim = dim3(n_warps * 32);
         cfg.dynamicSmemBytes = static_cast<size_t>(smem_optin);
         cudaLaunchAttribute at[1];
         at[0].id = cudaLaunchAttributeClusterDimension;
@@ -163,29 +164,31 @@ std::vector<uint32_t> plan_cluster_route(adacomp_select_t* h, Layout* lay, int d
         if (cudaOccupancyMaxActiveClusters(&n, k_select_cluster, &cfg) != cudaSuccess) { cudaGetLastError(); return 0; }
         return n;
     };
-    uint32_t best_C = 0, best_ring = 0, best_q = 0;
+    // block shapes in order of preference: more warps and more bytes in flight first, a larger value store last
+    const uint32_t shapes[4][2] = {{16, 2}, {12, 2}, {8, 3}, {8, 2}};
+    uint32_t best_C = 0, best_warps = 0, best_ring = 0, best_q = 0;
     std::vector<uint32_t> best_set;
     for (uint32_t C : {8u, 16u}) {
         uint32_t q_max = 0;
         for (uint32_t l : large) q_max = std::max(q_max, (pieces_of(l) + C - 1) / C);
-        for (uint32_t ring : {3u, 2u}) {
-            if (!cluster_layout_ok(ring, q_max)) continue;
+        for (const auto& shape : shapes) {
+            if (!cluster_layout_ok(shape[0], shape[1], q_max)) continue;
             std::vector<uint32_t> set;
-            for (uint32_t l : large) if (fits(l, C, ring, q_max)) set.push_back(l);
-            if (set.size() > best_set.size()) { best_set = set; best_C = C; best_ring = ring; best_q = q_max; }
+            for (uint32_t l : large) if (fits(l, C, shape[0], shape[1], q_max)) set.push_back(l);
+            if (set.size() > best_set.size()) { best_set = set; best_C = C; best_warps = shape[0]; best_ring = shape[1]; best_q = q_max; }
         }
         if (best_set.size() == large.size()) break;        // everything fits: no need for larger clusters
     }
     if (best_set.empty()) return chosen;
-    const int n_resident = resident(best_C);
+    const int n_resident = resident(best_C, best_warps);
     if (n_resident < 1) return chosen;
     h->cl_ctas = best_C;
+    h->cl_warps = best_warps;
     h->cl_ring = best_ring;
     h->cl_qmax = best_q;
     h->cl_smem = static_cast<uint32_t>(smem_optin);
     h->cl_active = n_resident;
-    for (uint32_t l : best_set) lay->layers[l].bracket = kRouteCluster;
-    build_items(lay);
+    for (uint32_t l : best_set) lay->layers[l].cluster = 1;
     return best_set;
 }
 
@@ -345,13 +348,13 @@ int adacomp_select_route_info(const adacomp_select_t* h, uint32_t* h_info_out) {
     if (!h || !h_info_out) return ADACOMP_ERR_INVALID;
     h_info_out[0] = h->n_cl;
     h_info_out[1] = h->cl_ctas;
-    h_info_out[2] = h->cl_ring;
+    h_info_out[2] = h->cl_ring | (h->cl_warps << 8);
     h_info_out[3] = static_cast<uint32_t>(h->cl_active);
     return ADACOMP_OK;
 }
 
 int adacomp_select_set_route(adacomp_select_t* h, int route) {
-    if (!h || route < 0 || route > 1) return ADACOMP_ERR_INVALID;
+    if (!h || route < 0 || route > 2) return ADACOMP_ERR_INVALID;
     h->route = route;
     return ADACOMP_OK;
 }
@@ -395,7 +398,8 @@ int adacomp_select(adacomp_select_t* h, const float* d_grads, uint64_t worker_st
     p.span_stride = h->span_stride;
 
     const unsigned n_inst = n_workers * h->n_layers;
-    const bool bracketed = h->route == 0 && (h->n_items > 0 || h->any_small || h->n_cl > 0);
+    const bool bracketed = h->route != 1 && (h->n_items > 0 || h->any_small);
+    const bool clusters = bracketed && h->route == 2 && h->n_cl > 0;
     int slot = 0;
     if (h->profiling) {                                   // take the next event list of the ring
         slot = h->ring_next;
@@ -425,7 +429,7 @@ int adacomp_select(adacomp_select_t* h, const float* d_grads, uint64_t worker_st
     // single-pass routes: sample (and the tensors that are selected on chip), the one pass over the gradient,
     // the exact threshold, the ordered write
     ADACOMP_CUDA(begin(0));
-    k_bracket_sample<<<n_inst, kBig, bracketed ? h->max_sample * sizeof(uint32_t) : 0, st>>>(p, bracketed ? 0 : 1);
+    k_bracket_sample<<<n_inst, kBig, bracketed ? h->max_sample * sizeof(uint32_t) : 0, st>>>(p, bracketed ? (clusters ? 2 : 0) : 1);
     ADACOMP_LAUNCH_CHECK();
     ADACOMP_CUDA(end());
     if (bracketed && h->n_items > 0) {
@@ -444,13 +448,13 @@ int adacomp_select(adacomp_select_t* h, const float* d_grads, uint64_t worker_st
         ADACOMP_CUDA(end());
     }
 
-    if (bracketed && h->n_cl > 0) {
+    if (clusters) {
         // cluster route: persistent clusters, one (worker, tensor) instance at a time
         const uint64_t n_ord = static_cast<uint64_t>(n_workers) * h->n_cl;
         const uint32_t n_clusters = static_cast<uint32_t>(n_ord < static_cast<uint64_t>(h->cl_active) ? n_ord : h->cl_active);
         cudaLaunchConfig_t cfg = {};
         cfg.gridDim = dim3(n_clusters * h->cl_ctas);
-        cfg.blockDim = dim3(kClThreads);
+        cfg.blockDim = dim3(h->cl_warps * 32);
         cfg.dynamicSmemBytes = h->cl_smem;
         cfg.stream = st;
         cudaLaunchAttribute at[1];

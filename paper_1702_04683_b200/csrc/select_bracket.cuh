@@ -129,7 +129,7 @@ __global__ void __launch_bounds__(kBig) k_bracket_sample(SelectParams p, int gen
     const uint32_t w = inst / p.n_layers, l = inst - w * p.n_layers;
     const Layer L = p.layers[l];
     Inst* st = &p.inst[inst];
-    const bool bracket = L.bracket && !general_only;
+    const bool bracket = L.bracket && general_only != 1;
     if (inst == 0 && threadIdx.x == 0) p.list_len[0] = 0;        // selections that took the general route: none so far
     if (threadIdx.x == 0) {
         st->prefix = 0; st->k_rem = L.k; st->n_gt = 0;
@@ -240,8 +240,13 @@ __global__ void __launch_bounds__(kBig) k_bracket_sample(SelectParams p, int gen
     // the scan compares magnitudes as floats and blanks padding with zeros: it needs a positive,
     // non-NaN lower bound
     const bool usable = t_lo != 0 && t_lo <= 0x7F800000u;
-    // a tensor on the cluster route (Layer::bracket == 2) is marked for the cluster kernel, the others for scan / resolve / emit
-    if (threadIdx.x == 0) { st->t_lo = t_lo; st->t_hi = t_hi; st->flags = usable ? (L.bracket == 2u ? 8u : kInstBracket) : kInstGeneral; }
+    // with the cluster route switched on (general_only == 2) the tensors that fit it are marked for the cluster kernel
+    // (flag 8), the others, as always, for scan / resolve / emit
+    if (threadIdx.x == 0) {
+        st->t_lo = t_lo;
+        st->t_hi = t_hi;
+        st->flags = usable ? (general_only == 2 && L.cluster ? 8u : kInstBracket) : kInstGeneral;
+    }
 }
 
 // ---------------------------------------------------------------------------------------------

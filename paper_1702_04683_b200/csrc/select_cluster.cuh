@@ -4,21 +4,23 @@
 // output once (8 bytes per kept entry): the algorithmic traffic of SELECT_GRAD, nothing else.
 //
 // A cluster of C blocks (8, or 16 where the device allows) takes one (worker, tensor) instance at a time;
-// block r owns a contiguous run of the tensor's 512-entry pieces.  Per instance:
-//   pass     every warp streams its pieces through a ring of 2 KB shared-memory buffers filled by bulk
-//            asynchronous copies (cp.async.bulk + an mbarrier per buffer, the warp's own).  A lane reads its 16
-//            consecutive entries, builds the mask of its candidates (key >= t_lo, the lower bracket
-//            bound from the sample kernel) and copies the candidates' VALUES, in index order, into the
-//            block's value store; the piece's 512-bit mask and where its values start are kept too.
-//            Positions are never stored: mask + order give them back.
+// block r owns a contiguous run of the tensor's 1024-entry pieces.  Per instance:
+//   pass     every warp streams its pieces through a ring of 4 KB shared-memory buffers filled by bulk
+//            asynchronous copies (cp.async.bulk + an mbarrier per buffer, the warp's own), exactly as the
+//            list route's scan kernel does.  A lane reads its 32 consecutive entries, builds the mask of
+//            its candidates (key >= t_lo, the lower bracket bound from the sample kernel) and copies the
+//            candidates' VALUES, in index order, into the block's value store; the piece's 1024-bit mask
+//            and where its values start are kept too.  Positions are never stored: mask + order give
+//            them back.
 //   select   the k-th largest candidate key, exactly: digit passes over the keys in the value stores
 //            (bins of the undecided key range, shared-memory histograms, summed over the cluster
 //            through distributed shared memory so that every block picks the same bin), two or three
 //            passes until the range is one key T; r = how many entries equal to T are kept.
-//   count    per piece the candidates above T and equal to T; prefix sums over the pieces of a block
-//            and, through one exchange, over the blocks give every piece its place in the output and
-//            the rank of its first tie (the r lowest-index ties are the ones kept).
-//   write    per piece, every lane walks its mask again and writes the kept (index, value) pairs.
+//   count    per piece (one thread each) the candidates above T and equal to T; prefix sums over the
+//            pieces of a block and, through one exchange, over the blocks give every piece its place in
+//            the output and the rank of its first tie (the r lowest-index ties are the ones kept).
+//   write    per piece (one thread each) a walk over the mask's set bits writes the kept (index, value)
+//            pairs.
 // Between the steps stands the cluster's hardware barrier; no block waits on a flag, and none leaves
 // while its shared memory may still be read.  If a store overflows, a NaN turns up, or fewer than k
 // candidates were seen (the bracket missed), the instance is handed to the general route untouched.
@@ -30,12 +32,10 @@
 
 namespace adacomp {
 
-constexpr int kClThreads = 512;
-constexpr uint32_t kClWarps = kClThreads / 32;
-constexpr uint32_t kClPiece = 512;                    // entries per piece: 16 per lane
+constexpr int kClMaxThreads = 512;                    // blocks run 8, 12 or 16 warps: more warps where the value store can be smaller
+constexpr uint32_t kClPiece = kSubElems;              // entries per piece: 32 per lane
 constexpr uint32_t kClPieceBytes = kClPiece * 4;
 constexpr uint32_t kClMaxCtas = 16;
-constexpr uint32_t kRouteCluster = 2u;                // Layer::bracket of a tensor on this route
 constexpr uint32_t kInstCluster = 8u;                 // bracket valid, the cluster kernel acts on the instance
 constexpr uint32_t kClMinN = 1u << 20;                // shorter tensors stay on the list route: the barriers would cost more than they save
 
@@ -45,48 +45,78 @@ struct ClusterLayout {
     uint32_t ring, mbar, bitmap, pinfo, misc, vals, vals_cap;      // vals_cap: values the store holds
     uint32_t hist, pcount, ppost;                                   // inside the ring
 };
-__host__ __device__ inline ClusterLayout cluster_layout(uint32_t ring_slots, uint32_t q_max, uint32_t total_bytes) {
+__host__ __device__ inline ClusterLayout cluster_layout(uint32_t n_warps, uint32_t ring_slots, uint32_t q_max, uint32_t total_bytes) {
     ClusterLayout y;
     y.ring = 0;
-    const uint32_t ring_bytes = kClWarps * ring_slots * kClPieceBytes;
+    const uint32_t ring_bytes = n_warps * ring_slots * kClPieceBytes;
     y.hist = 0;                                       // 2048 bins
     y.pcount = 8192;                                  // [q_max] (above T, equal to T)
-    y.ppost = 8192 + q_max * 8;                       // [q_max] (place in the output, rank of the first tie)
+    y.ppost = 8192 + q_max * 8;                       // [q_max] (above T before the piece, equal to T before it)
     y.mbar = ring_bytes;                              // [warps][ring_slots] mbarriers
-    y.bitmap = y.mbar + ((kClWarps * ring_slots * 8 + 15) & ~15u);   // [q_max][32] 16-bit masks
-    y.pinfo = y.bitmap + q_max * 64;                  // [q_max] first value | count << 22
+    y.bitmap = y.mbar + ((n_warps * ring_slots * 8 + 15) & ~15u);   // [q_max][32] 32-bit masks
+    y.pinfo = y.bitmap + q_max * 128;                 // [q_max] first value | count << 21
     y.misc = (y.pinfo + q_max * 4 + 15) & ~15u;       // counters, exchange slots, scan scratch
     y.vals = y.misc + 512;
     y.vals_cap = total_bytes > y.vals ? (total_bytes - y.vals) / 4 : 0;
-    if (y.vals_cap > (1u << 22) - 1) y.vals_cap = (1u << 22) - 1;
+    if (y.vals_cap > (1u << 21) - 1) y.vals_cap = (1u << 21) - 1;
     return y;
 }
 // the tables of the later steps must fit the ring
-__host__ __device__ inline bool cluster_layout_ok(uint32_t ring_slots, uint32_t q_max) {
-    return 8192 + q_max * 16 <= kClWarps * ring_slots * kClPieceBytes;
+__host__ __device__ inline bool cluster_layout_ok(uint32_t n_warps, uint32_t ring_slots, uint32_t q_max) {
+    return 8192 + q_max * 16 <= n_warps * ring_slots * kClPieceBytes;
 }
 
-// Descending walk over a 2048-bin histogram in shared memory with THREADS threads: the bin holding the
-// rem-th largest.  out[0] = bin, out[1] = entries above it, out[2] = its count, out[3] = 1 if found.
-template <int THREADS>
-__device__ __forceinline__ void block_pick_bin(const uint32_t* hist, uint32_t rem, uint32_t* out /*[4] shared*/, uint32_t* s_warp /*[33]*/) {
-    constexpr int M = 2048 / THREADS;
+// Block-wide exclusive prefix sum for a block of n_warps (<= 32) full warps.  s_warp needs 33 entries.
+__device__ __forceinline__ uint32_t block_exclusive_scan_rt(uint32_t v, uint32_t* total, uint32_t* s_warp, uint32_t n_warps) {
+    const uint32_t lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    uint32_t inc = v;
+#pragma unroll
+    for (int d = 1; d < 32; d <<= 1) {
+        const uint32_t y = __shfl_up_sync(0xFFFFFFFFu, inc, d);
+        if (lane >= static_cast<uint32_t>(d)) inc += y;
+    }
+    __syncthreads();
+    if (lane == 31) s_warp[warp] = inc;
+    __syncthreads();
+    if (warp == 0) {
+        const uint32_t t = lane < n_warps ? s_warp[lane] : 0u;
+        uint32_t winc = t;
+#pragma unroll
+        for (int d = 1; d < 32; d <<= 1) {
+            const uint32_t y = __shfl_up_sync(0xFFFFFFFFu, winc, d);
+            if (lane >= static_cast<uint32_t>(d)) winc += y;
+        }
+        if (lane < n_warps) s_warp[lane] = winc - t;
+        if (lane == 31) s_warp[32] = winc;
+    }
+    __syncthreads();
+    *total = s_warp[32];
+    return s_warp[warp] + inc - v;
+}
+
+// Descending walk over a 2048-bin histogram in shared memory by the first 256 threads of a block of n_warps warps
+// (8 bins each): the bin holding the rem-th largest.  out[0] = bin, out[1] = entries above it, out[2] = its count,
+// out[3] = 1 if found.  All threads call.
+__device__ __forceinline__ void block_pick_bin(const uint32_t* hist, uint32_t rem, uint32_t* out /*[4] shared*/, uint32_t* s_warp /*[33]*/,
+                                               uint32_t n_warps) {
+    constexpr int M = 8;
+    const bool mine = threadIdx.x < 2048 / M;
     const int top = 2047 - static_cast<int>(threadIdx.x) * M;
     uint32_t h[M], sum = 0;
 #pragma unroll
-    for (int q = 0; q < M; ++q) { h[q] = hist[top - q]; sum += h[q]; }
+    for (int q = 0; q < M; ++q) { h[q] = mine ? hist[top - q] : 0u; sum += h[q]; }
     if (threadIdx.x == 0) out[3] = 0;
     uint32_t total;
-    uint32_t above = block_exclusive_scan_t<THREADS>(sum, &total, s_warp);      // (barriers inside: out[3] = 0 is seen)
+    uint32_t above = block_exclusive_scan_rt(sum, &total, s_warp, n_warps);     // (barriers inside: out[3] = 0 is seen)
 #pragma unroll
     for (int q = 0; q < M; ++q) {
-        if (above < rem && rem <= above + h[q]) { out[0] = top - q; out[1] = above; out[2] = h[q]; out[3] = 1; }
+        if (mine && above < rem && rem <= above + h[q]) { out[0] = top - q; out[1] = above; out[2] = h[q]; out[3] = 1; }
         above += h[q];
     }
     __syncthreads();
 }
 
-__global__ void __launch_bounds__(kClThreads, 1)
+__global__ void __launch_bounds__(kClMaxThreads, 1)
 k_select_cluster(SelectParams p, const uint32_t* __restrict__ cl_layers, uint32_t n_cl, uint32_t ring_slots, uint32_t q_max,
                  uint32_t smem_bytes) {
     extern __shared__ __align__(16) unsigned char s_cl[];
@@ -95,8 +125,9 @@ k_select_cluster(SelectParams p, const uint32_t* __restrict__ cl_layers, uint32_
     const uint32_t C = cluster.num_blocks(), rank = cluster.block_rank();
     const uint32_t cluster_id = blockIdx.x / C, n_clusters = gridDim.x / C;
     const uint32_t lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-    const ClusterLayout Y = cluster_layout(ring_slots, q_max, smem_bytes);
-    uint16_t* s_bitmap = reinterpret_cast<uint16_t*>(s_cl + Y.bitmap);
+    const uint32_t n_threads = blockDim.x, n_warps = n_threads >> 5;
+    const ClusterLayout Y = cluster_layout(n_warps, ring_slots, q_max, smem_bytes);
+    uint32_t* s_bitmap = reinterpret_cast<uint32_t*>(s_cl + Y.bitmap);
     uint32_t* s_pinfo = reinterpret_cast<uint32_t*>(s_cl + Y.pinfo);
     uint32_t* s_vals = reinterpret_cast<uint32_t*>(s_cl + Y.vals);
     uint32_t* s_hist = reinterpret_cast<uint32_t*>(s_cl + Y.hist);
@@ -104,7 +135,7 @@ k_select_cluster(SelectParams p, const uint32_t* __restrict__ cl_layers, uint32_
     uint2* s_ppost = reinterpret_cast<uint2*>(s_cl + Y.ppost);
     uint32_t* s_misc = reinterpret_cast<uint32_t*>(s_cl + Y.misc);
     uint32_t* s_used = s_misc + 0;                    // values in the store
-    uint32_t* s_over = s_misc + 1;                    // != 0: the store overflowed, a NaN was seen, or a copy never arrived
+    uint32_t* s_over = s_misc + 1;                    // != 0: the store overflowed, or a copy never arrived
     uint32_t* s_above = s_misc + 2;                   // keys above the hinted range (first digit pass)
     uint32_t* s_nan = s_misc + 3;                     // != 0: a NaN among them
     uint32_t* s_x = s_misc + 4;                       // [4] what this block tells the others: used, over, above-T total, equal-T total
@@ -146,9 +177,9 @@ k_select_cluster(SelectParams p, const uint32_t* __restrict__ cl_layers, uint32_
 
         // ============================ pass: candidates' values into the block's store
         // (Q > q_max cannot happen with the host's choice of q_max; if it did the tables would not hold the pieces: nothing is read)
-        const uint32_t n_mine = (q_count > warp && !dead && Q <= q_max) ? (q_count - warp + kClWarps - 1) / kClWarps : 0u;
-        auto fetch = [&](uint32_t j) {               // lane 0: piece q0 + warp + kClWarps j into ring slot (fetched + j) % ring_slots
-            const uint32_t vec0 = (q0 + warp + kClWarps * j) * (kClPiece / 4);
+        const uint32_t n_mine = (q_count > warp && !dead && Q <= q_max) ? (q_count - warp + n_warps - 1) / n_warps : 0u;
+        auto fetch = [&](uint32_t j) {               // lane 0: piece q0 + warp + n_warps j into ring slot (fetched + j) % ring_slots
+            const uint32_t vec0 = (q0 + warp + n_warps * j) * (kClPiece / 4);
             const uint32_t groups = nvec - vec0 < kClPiece / 4 ? nvec - vec0 : kClPiece / 4;
             const uint32_t slot = (fetched + j) % ring_slots;
             mbar_expect_tx(mbar_base + 8u * slot, groups * 16u);
@@ -159,7 +190,7 @@ k_select_cluster(SelectParams p, const uint32_t* __restrict__ cl_layers, uint32_
             for (uint32_t j = 0; j < ring_slots && j < n_mine; ++j) fetch(j);
         }
         if (dead && q_count > warp && lane == 0) *s_over = 1u;
-        const uint32_t rot = (lane >> 1) & 3u;       // rotation of the lane's four 16-byte groups: a quarter warp hits distinct banks
+        const uint32_t lane_base = lane * 128u, rot = (lane & 7u) << 4;   // the lane's 128 bytes of a buffer; its rotation of the 16-byte groups
 #pragma unroll 1
         for (uint32_t j = 0; j < n_mine; ++j) {
             const uint32_t u = fetched + j, slot = u % ring_slots;
@@ -180,26 +211,30 @@ k_select_cluster(SelectParams p, const uint32_t* __restrict__ cl_layers, uint32_
                     break;
                 }
             }
-            const uint32_t lq = warp + kClWarps * j;                      // the piece's number inside the block
-            const uint32_t e_lane = (q0 + lq) * kClPiece + lane * 16u;    // shifted position of the lane's first entry
-            const uint32_t buf = ring_base + slot * kClPieceBytes, lane_base = lane * 64u;
+            const uint32_t lq = warp + n_warps * j;                       // the piece's number inside the block
+            const uint32_t e_lane = (q0 + lq) * kClPiece + lane * 32u;    // shifted position of the lane's first entry
+            const uint32_t buf = ring_base + slot * kClPieceBytes;
             uint32_t mask;
             {
-                float4 q[4];
+                float4 q[8];
 #pragma unroll
-                for (int i = 0; i < 4; ++i)
+                for (int i = 0; i < 8; ++i)                               // group i ^ (lane & 7) first: the eight lanes of a quarter warp hit distinct banks
                     asm volatile("ld.shared.v4.f32 {%0, %1, %2, %3}, [%4];"
                                  : "=f"(q[i].x), "=f"(q[i].y), "=f"(q[i].z), "=f"(q[i].w)
-                                 : "r"(buf + lane_base + ((static_cast<uint32_t>(i) ^ rot) << 4)));
-                uint32_t raw = 0;                                      // nibble i: group i ^ rot
+                                 : "r"(buf + lane_base + ((static_cast<uint32_t>(i) << 4) ^ rot)));
+                uint32_t raw = 0;                                         // nibble i: group i ^ (lane & 7)
                 mask_or<1u << 0>(q[0], tlo_f, raw);  mask_or<1u << 4>(q[1], tlo_f, raw);
                 mask_or<1u << 8>(q[2], tlo_f, raw);  mask_or<1u << 12>(q[3], tlo_f, raw);
-                uint32_t m = raw;                                      // nibble g of the mask = nibble g ^ rot of raw
-                if (rot & 1u) m = ((m & 0x0F0Fu) << 4) | ((m >> 4) & 0x0F0Fu);
-                if (rot & 2u) m = ((m & 0x00FFu) << 8) | (m >> 8);
+                mask_or<1u << 16>(q[4], tlo_f, raw); mask_or<1u << 20>(q[5], tlo_f, raw);
+                mask_or<1u << 24>(q[6], tlo_f, raw); mask_or<1u << 28>(q[7], tlo_f, raw);
+                const uint32_t r7 = lane & 7u;                            // nibble g of the mask = nibble g ^ r7 of raw
+                uint32_t m = raw;
+                if (r7 & 1u) m = ((m & 0x0F0F0F0Fu) << 4) | ((m >> 4) & 0x0F0F0F0Fu);
+                if (r7 & 2u) m = ((m & 0x00FF00FFu) << 8) | ((m >> 8) & 0x00FF00FFu);
+                if (r7 & 4u) m = (m << 16) | (m >> 16);
                 const uint32_t lo_cut = mis > e_lane ? mis - e_lane : 0u;                    // <= 3
-                const uint32_t hi_cut = n_shift > e_lane ? (n_shift - e_lane < 16u ? n_shift - e_lane : 16u) : 0u;
-                mask = m & ((1u << hi_cut) - 1u) & ~((1u << lo_cut) - 1u);
+                const uint32_t hi_cut = n_shift > e_lane ? (n_shift - e_lane < 32u ? n_shift - e_lane : 32u) : 0u;
+                mask = m & (hi_cut == 32u ? 0xFFFFFFFFu : (1u << hi_cut) - 1u) & ~((1u << lo_cut) - 1u);
             }
             const uint32_t cnt = __popc(mask);
             uint32_t inc = cnt;
@@ -213,9 +248,9 @@ k_select_cluster(SelectParams p, const uint32_t* __restrict__ cl_layers, uint32_
             if (lane == 0 && tc) off = atomicAdd(s_used, tc);            // room in the block's store
             off = __shfl_sync(0xFFFFFFFFu, off, 0);
             const bool fits = off + tc <= Y.vals_cap;
-            s_bitmap[lq * 32u + lane] = static_cast<uint16_t>(fits ? mask : 0u);
+            s_bitmap[lq * 32u + lane] = fits ? mask : 0u;
             if (lane == 0) {
-                s_pinfo[lq] = fits ? (off | (tc << 22)) : 0u;
+                s_pinfo[lq] = fits ? (off | (tc << 21)) : 0u;
                 if (!fits) *s_over = 1u;
             }
             if (tc && fits) {
@@ -261,11 +296,11 @@ k_select_cluster(SelectParams p, const uint32_t* __restrict__ cl_layers, uint32_
             for (int pass = 0; pass < 8 && !bad; ++pass) {
                 const uint32_t width = hi - lo + 1u;                   // >= 1
                 const uint32_t sh = width > 2048u ? (32u - __clz(width - 1u)) - 11u : 0u;
-                for (uint32_t b = threadIdx.x; b < 2048u; b += kClThreads) s_hist[b] = 0;
+                for (uint32_t b = threadIdx.x; b < 2048u; b += n_threads) s_hist[b] = 0;
                 if (threadIdx.x == 0) { *s_above = 0; *s_nan = 0; }
                 __syncthreads();
                 uint32_t above = 0, nan = 0;
-                for (uint32_t i = threadIdx.x; i < used; i += kClThreads) {
+                for (uint32_t i = threadIdx.x; i < used; i += n_threads) {
                     const uint32_t key = s_vals[i] & 0x7FFFFFFFu;
                     if (key >= lo && key <= hi) atomicAdd(&s_hist[(key - lo) >> sh], 1u);
                     else if (key > hi) { ++above; nan |= key > 0x7F800000u ? 1u : 0u; }
@@ -278,14 +313,20 @@ k_select_cluster(SelectParams p, const uint32_t* __restrict__ cl_layers, uint32_
                 }
                 __syncthreads();
                 cluster.sync();                                        // all shares counted
-                // this block's bins, summed over the cluster and handed to everyone; block 0 does the same for the count above
-                for (uint32_t t = threadIdx.x; t < 2048u / C; t += kClThreads) {
+                // this block's bins, summed over the cluster and handed to everyone (the loads of a bin's C shares are
+                // independent: they overlap); block 0 does the same for the count above
+                for (uint32_t t = threadIdx.x; t < 2048u / C; t += n_threads) {
                     const uint32_t bin = rank * (2048u / C) + t;
+                    uint32_t part[kClMaxCtas];
+#pragma unroll
+                    for (uint32_t b = 0; b < kClMaxCtas; ++b) part[b] = b < C ? cluster.map_shared_rank(s_hist, b)[bin] : 0u;
                     uint32_t sum = 0;
-                    for (uint32_t b = 0; b < C; ++b) sum += cluster.map_shared_rank(s_hist, b)[bin];
-                    for (uint32_t b = 0; b < C; ++b) cluster.map_shared_rank(s_hist, b)[bin] = sum;
+#pragma unroll
+                    for (uint32_t b = 0; b < kClMaxCtas; ++b) sum += part[b];
+#pragma unroll
+                    for (uint32_t b = 0; b < kClMaxCtas; ++b) if (b < C) cluster.map_shared_rank(s_hist, b)[bin] = sum;
                 }
-                if (hinted && rank == 0 && threadIdx.x == 0) {
+                if (hinted && rank == 0 && threadIdx.x == 32) {
                     uint32_t sum = 0, flag = 0;
                     for (uint32_t b = 0; b < C; ++b) {
                         sum += *cluster.map_shared_rank(s_above, b);
@@ -309,7 +350,7 @@ k_select_cluster(SelectParams p, const uint32_t* __restrict__ cl_layers, uint32_
                     rem -= a;
                     hinted = false;
                 }
-                block_pick_bin<kClThreads>(s_hist, rem, s_bc, s_warp);
+                block_pick_bin(s_hist, rem, s_bc, s_warp, n_warps);
                 if (!s_bc[3]) { bad = true; why = 4u; break; }         // cannot happen: the counts add up to >= rem
                 const uint32_t bin = s_bc[0];
                 rem -= s_bc[1];
@@ -328,29 +369,27 @@ k_select_cluster(SelectParams p, const uint32_t* __restrict__ cl_layers, uint32_
             continue;
         }
 
-        // ============================ count: per piece, candidates above T and equal to T
-        for (uint32_t lq = warp; lq < q_count; lq += kClWarps) {
-            const uint32_t info = s_pinfo[lq], off = info & 0x3FFFFFu, cnt = info >> 22;
+        // ============================ count: per piece (one thread each), candidates above T and equal to T
+        for (uint32_t lq = threadIdx.x; lq < q_count; lq += n_threads) {
+            const uint32_t info = s_pinfo[lq], off = info & 0x1FFFFFu, cnt = info >> 21;
             uint32_t gt = 0, eq = 0;
-            for (uint32_t i = lane; i < cnt; i += 32) {
+            for (uint32_t i = 0; i < cnt; ++i) {
                 const uint32_t key = s_vals[off + i] & 0x7FFFFFFFu;
                 gt += key > T ? 1u : 0u;
                 eq += key == T ? 1u : 0u;
             }
-            gt = __reduce_add_sync(0xFFFFFFFFu, gt);
-            eq = __reduce_add_sync(0xFFFFFFFFu, eq);
-            if (lane == 0) s_pcount[lq] = make_uint2(gt, eq);
+            s_pcount[lq] = make_uint2(gt, eq);
         }
         if (threadIdx.x == 0) { s_carry[0] = 0; s_carry[1] = 0; }
         __syncthreads();
         // exclusive prefixes over the block's pieces (kept for the write step in s_ppost: above-T before, equal-T before)
-        for (uint32_t base = 0; base < q_count; base += kClThreads) {
+        for (uint32_t base = 0; base < q_count; base += n_threads) {
             const uint32_t lq = base + threadIdx.x;
             uint2 c = make_uint2(0u, 0u);
             if (lq < q_count) c = s_pcount[lq];
             uint32_t tg, te;
-            const uint32_t eg = block_exclusive_scan_t<kClThreads>(c.x, &tg, s_warp);
-            const uint32_t ee = block_exclusive_scan_t<kClThreads>(c.y, &te, s_warp);
+            const uint32_t eg = block_exclusive_scan_rt(c.x, &tg, s_warp, n_warps);
+            const uint32_t ee = block_exclusive_scan_rt(c.y, &te, s_warp, n_warps);
             const uint32_t c0 = s_carry[0], c1 = s_carry[1];
             if (lq < q_count) s_ppost[lq] = make_uint2(c0 + eg, c1 + ee);
             __syncthreads();
@@ -378,59 +417,37 @@ k_select_cluster(SelectParams p, const uint32_t* __restrict__ cl_layers, uint32_
             continue;
         }
 
-        // ============================ write: the kept pairs, in index order
+        // ============================ write: the kept pairs, in index order; one thread walks one piece
         uint32_t* idx_out = p.idx_out + static_cast<uint64_t>(w) * p.K + L.out_offset;
         float* val_out = p.val_out + static_cast<uint64_t>(w) * p.K + L.out_offset;
         const uint32_t glob = static_cast<uint32_t>(L.offset) - mis;    // shifted position -> index in the gradient vector
-        for (uint32_t lq = warp; lq < q_count; lq += kClWarps) {
-            const uint32_t info = s_pinfo[lq], off = info & 0x3FFFFFu;
-            if ((info >> 22) == 0) continue;
+        for (uint32_t lq = threadIdx.x; lq < q_count; lq += n_threads) {
+            const uint32_t info = s_pinfo[lq];
+            if ((info >> 21) == 0) continue;
+            uint32_t at = info & 0x1FFFFFu;                             // the piece's next value in the store
             const uint2 post = s_ppost[lq];
-            const uint32_t eq_piece = eq_base + post.y;                 // ties before this piece
-            const uint32_t ties_before = r > eq_base ? (r - eq_base < post.y ? r - eq_base : post.y) : 0u;   // of them kept, inside this block
-            const uint32_t mask = s_bitmap[lq * 32u + lane];
-            const uint32_t cnt = __popc(mask);
-            uint32_t inc = cnt;
+            uint32_t tie_rank = eq_base + post.y;                       // global rank of the piece's first tie
+            const uint32_t ties_before = r > eq_base ? (r - eq_base < post.y ? r - eq_base : post.y) : 0u;   // kept ties before the piece, inside this block
+            uint32_t o = out_base + post.x + ties_before;               // the piece's first place in the output
+            const uint32_t e_piece = glob + (q0 + lq) * kClPiece;
+            const uint4* words = reinterpret_cast<const uint4*>(s_bitmap + lq * 32u);
+#pragma unroll 1
+            for (uint32_t g4 = 0; g4 < 8; ++g4) {                       // 4 lanes' masks at a time
+                const uint4 wv = words[g4];
+                const uint32_t wd[4] = {wv.x, wv.y, wv.z, wv.w};
 #pragma unroll
-            for (int d = 1; d < 32; d <<= 1) {
-                const uint32_t y = __shfl_up_sync(0xFFFFFFFFu, inc, d);
-                if (lane >= static_cast<uint32_t>(d)) inc += y;
-            }
-            const uint32_t my_first = off + inc - cnt;                  // the lane's first value in the store
-            // first walk: how many of the lane's candidates are above T, how many equal
-            uint32_t gt = 0, eq = 0;
-            for (uint32_t i = 0; i < cnt; ++i) {
-                const uint32_t key = s_vals[my_first + i] & 0x7FFFFFFFu;
-                gt += key > T ? 1u : 0u;
-                eq += key == T ? 1u : 0u;
-            }
-            uint32_t eq_inc = eq;
-#pragma unroll
-            for (int d = 1; d < 32; d <<= 1) {
-                const uint32_t y = __shfl_up_sync(0xFFFFFFFFu, eq_inc, d);
-                if (lane >= static_cast<uint32_t>(d)) eq_inc += y;
-            }
-            uint32_t tie_rank = eq_piece + eq_inc - eq;                 // global rank of the lane's first tie
-            const uint32_t ties_mine = r > tie_rank ? (r - tie_rank < eq ? r - tie_rank : eq) : 0u;
-            const uint32_t kept = gt + ties_mine;
-            uint32_t k_inc = kept;
-#pragma unroll
-            for (int d = 1; d < 32; d <<= 1) {
-                const uint32_t y = __shfl_up_sync(0xFFFFFFFFu, k_inc, d);
-                if (lane >= static_cast<uint32_t>(d)) k_inc += y;
-            }
-            uint32_t o = out_base + post.x + ties_before + k_inc - kept;   // the lane's first place in the output
-            // second walk: write what is kept
-            const uint32_t e_lane = (q0 + lq) * kClPiece + lane * 16u;
-            uint32_t at = my_first;
-            for (uint32_t m = mask; m; m &= m - 1u, ++at) {
-                const uint32_t bits = s_vals[at], key = bits & 0x7FFFFFFFu;
-                bool keep = key > T;
-                if (key == T) { keep = tie_rank < r; ++tie_rank; }
-                if (keep) {
-                    __stcs(&idx_out[o], glob + e_lane + (__ffs(m) - 1u));
-                    __stcs(&val_out[o], __uint_as_float(bits));
-                    ++o;
+                for (uint32_t c4 = 0; c4 < 4; ++c4) {
+                    const uint32_t e_word = e_piece + (g4 * 4u + c4) * 32u;
+                    for (uint32_t m = wd[c4]; m; m &= m - 1u, ++at) {
+                        const uint32_t bits = s_vals[at], key = bits & 0x7FFFFFFFu;
+                        bool keep = key > T;
+                        if (key == T) { keep = tie_rank < r; ++tie_rank; }
+                        if (keep) {
+                            __stcs(&idx_out[o], e_word + (__ffs(m) - 1u));
+                            __stcs(&val_out[o], __uint_as_float(bits));
+                            ++o;
+                        }
+                    }
                 }
             }
         }

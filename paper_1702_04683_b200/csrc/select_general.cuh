@@ -41,6 +41,8 @@ struct Layer {            // one tensor V_l / beta_l of the layout
     uint32_t win_cap;     // room in the window list
     uint64_t cand_base;   // first candidate slot inside a worker's candidate range
     uint64_t win_base;    // first window slot inside a worker's window range
+    uint32_t cluster;     // 1: large enough, and small enough, for the cluster route (select_cluster.cuh) on this device
+    uint32_t pad;
 };
 
 struct Inst {             // selection state of one (worker, tensor)

@@ -194,6 +194,39 @@ def test_dense_candidates_crowded_and_spread(binding):
         assert general <= 1                                            # at most the tied worker fell back
 
 
+@pytest.mark.parametrize("k", [1, 1_500, 75_000, 300_000])
+def test_cluster_route_on_large_tensors(binding, k):
+    """Route 2: tensors of a million entries or more are selected by one thread-block cluster each, which
+    keeps masks and candidate values on chip between the single pass and the ordered write.  Rows at odd
+    alignments, a crowded stretch (its block's store overflows: handed to the general route), a coarse grid
+    with thousands of ties at the threshold, a NaN (handed over), a shorter tensor beside the large one."""
+    dev = torch.device("cuda", 0)
+    n, n2 = 1_300_003, 200_000
+    gen = torch.Generator(device=dev)
+    gen.manual_seed(k)
+    g = torch.randn((5, n + n2 + 7), device=dev, generator=gen)[:, 3:n + n2 + 3]
+    g[1, :n] = torch.round(g[1, :n] * 8) / 8
+    g[2, 100_000:400_000] *= 1000.0
+    g[3, 777_777] = float("nan")
+    g[4, :n] *= torch.rand(n, device=dev, generator=gen) ** 4
+    k2 = 2_000
+    sel = binding.Selector(binding.segments_from([0, n], [n, n2], [k, k2]), 5, dev)
+    assert sel.route_info()["cluster_tensors"] == 1
+    sel.set_route(2)
+    idx, val = sel.select(g)
+    status, general = sel.last_error()
+    assert status == 0 and 1 <= general <= 3             # the NaN for sure; the crowded and the tied worker may join it
+    g_host = g.cpu().numpy()
+    for w in range(5):
+        oi, ov = oracle.select_layers(g_host[w], [0, n], [n, n2], [k, k2])
+        assert np.array_equal(u32(idx)[w], oi), w
+        assert np.array_equal(bits(val[w]), bits(ov)), w
+    sel.set_route(0)                                       # the same handle on the default route: same answer
+    idx0, val0 = sel.select(g)
+    assert sel.last_error()[0] == 0
+    assert torch.equal(idx, idx0) and torch.equal(val.view(torch.int32), val0.view(torch.int32))
+
+
 @pytest.mark.parametrize("n,k", [(32_768, 1), (32_768, 8192), (40_000, 400), (65_537, 700), (1 << 20, 1), (3_000_001, 30_001)])
 def test_bracket_route_sizes(binding, n, k):
     dev = torch.device("cuda", 0)
