@@ -128,36 +128,34 @@ __device__ __forceinline__ uint32_t first_at_or_above(const uint32_t* __restrict
 // ---------------------------------------------------------------------------------------------
 // Several updates per launch, one WARP per range of parameters, no block barrier in the loop.  A
 // warp owns a run of ranges of R consecutive parameters and a slice of shared memory: Theta and
-// the heads of the range (with two buffers the next range's arrive while this one is worked on), a
-// mask per parameter (bit b: update b of the launch changed it) and, per update, a stage with
-// the update's next 32 pairs from its cursor.  All of that is brought in by asynchronous copies
-// issued a range ahead, so that no load is waited for in the common case.
-// Per range the warp takes the updates ONE AFTER THE OTHER in arrival order.  The staged pairs
-// below the range's end are the update's pairs of this range (its index list is ascending), and
-// each lane applies one of them against shared memory exactly as Algorithm 2 states it: Eq. 3
-// inside the launch is a population count of the parameter's mask under the update's window bits,
-// the part of a window before the launch a chain walk from the head the parameter had when the
-// launch began; Eq. 5; Eq. 4; the pair is linked behind the head (one coalesced store to the ring
-// per update) and becomes the head.  The stage of an update that consumed pairs is refilled from
-// its new cursor; updates with no pair in the range are skipped four or eight at a time.  When all
-// 32 staged pairs lay in the range the update may have more there: they are fetched and applied
-// before the next update is looked at (the host sizes R so that this is rare).  At the end of
-// the range Theta and heads go back, 16 bytes per lane, where a parameter changed.  Updates are
-// applied in order per range, which is all Algorithm 2 needs: same results, bit for bit, as one
-// launch per update.  kExtra: staleness counts are written, or the lists are validated.
+// the heads of the range (two buffers: the next range's arrive by asynchronous copies while this
+// one is worked on) and a mask per parameter (bit b: update b of the launch changed it).  The
+// updates' pairs never pass through shared memory: every lane keeps, IN REGISTERS, one pair of
+// each update (lane t: the pair at the update's cursor + t), i.e. the warp holds the next 32 pairs
+// of all updates at once.  The loop over the updates is unrolled, so that "update b" is a fixed
+// set of registers and its descriptor (first pair, pair count, position, window bits) constant
+// operands of the instructions; a stage is refilled by plain loads right after it was used, a
+// whole range before it is needed again, so their latency is hidden by program order alone.
+// Per range the warp takes the updates ONE AFTER THE OTHER in arrival order.  The lanes whose
+// pair lies below the range's end hold the update's pairs of this range (its index list is
+// ascending), and each applies its pair against shared memory exactly as Algorithm 2 states it:
+// Eq. 3 inside the launch is a population count of the parameter's mask under the update's window
+// bits, the part of a window before the launch a chain walk from the head the parameter had when
+// the launch began; Eq. 5; Eq. 4; the pair is linked behind the head (one coalesced store to the
+// ring per update) and becomes the head.  When all 32 pairs lay in the range the update may have
+// more there: they are loaded and applied before the next update is looked at (the host sizes R so
+// that this is rare).  At the end of the range Theta and heads go back, 16 bytes per lane, where a
+// parameter changed.  Updates are applied in order per range, which is all Algorithm 2 needs:
+// same results, bit for bit, as one launch per update.  NB: updates the unrolled loop covers (16 or
+// 32).  kExtra: staleness counts are written, or the lists are validated.
 constexpr int kWpThreads = 128;
 constexpr uint32_t kWpWarps = kWpThreads / 32;
-constexpr uint32_t kWpGroups = 4;              // groups of asynchronous copies per range
 
-// `buffers` of Theta and heads per warp: with two the next range arrives while this one is worked on; with one
-// more warps stay resident and the next range is fetched (from L2, where a prefetch put it) between two ranges.
-// Measured: one is better for ranges longer than 256 parameters when a launch holds more than 8 updates (their
-// stages are what fills shared memory then), two otherwise.
-__host__ __device__ inline size_t wp_warp_words(uint32_t range, uint32_t n_updates, bool pre, uint32_t buffers) {
-    return 32 + (pre ? 96 : 64) * static_cast<size_t>(n_updates) + (2 * buffers + (pre ? 2 : 1)) * static_cast<size_t>(range);
+__host__ __device__ inline size_t wp_warp_words(uint32_t range, bool pre) {
+    return (pre ? 6 : 5) * static_cast<size_t>(range);          // Theta and heads twice, masks, (heads at the launch's start)
 }
-__host__ __device__ inline size_t wp_smem_bytes(uint32_t range, uint32_t n_updates, bool pre, uint32_t buffers) {
-    return 64 * 4 + kWpWarps * wp_warp_words(range, n_updates, pre, buffers) * 4;
+__host__ __device__ inline size_t wp_smem_bytes(uint32_t range, bool pre) {
+    return 64 * 4 + kWpWarps * wp_warp_words(range, pre) * 4;
 }
 
 __device__ __forceinline__ uint32_t smem_address(const void* p) { return static_cast<uint32_t>(__cvta_generic_to_shared(p)); }
@@ -172,23 +170,20 @@ __device__ __forceinline__ void copy_async_commit() { asm volatile("cp.async.com
 template <int kPending>
 __device__ __forceinline__ void copy_async_wait() { asm volatile("cp.async.wait_group %0;" ::"n"(kPending) : "memory"); }
 
-template <uint32_t R, uint32_t kBuffers, bool kPre, bool kExtra>
+template <uint32_t R, uint32_t NB, bool kPre, bool kExtra>
 __global__ void __launch_bounds__(kWpThreads)
 k_apply_warps(const ServerParams sp, const BatchDesc d, const uint32_t* __restrict__ idx, const float* __restrict__ val,
               float lr, uint32_t* sigma_out, uint32_t n_ranges) {
     extern __shared__ __align__(16) unsigned char s_wp[];
     static_assert(R % 64 == 0 && R >= 128, "16-byte pieces, whole warps");
+    static_assert(NB <= kMaxBatch, "one mask bit per update");
     float* s_alpha = reinterpret_cast<float*>(s_wp);                            // [64] alpha / sigma for the small counts
-    const uint32_t B = d.n_updates;
+    const uint32_t B = d.n_updates;                                             // <= NB
     const uint32_t tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-    uint32_t* s_cur = reinterpret_cast<uint32_t*>(s_wp) + 64 + warp * wp_warp_words(R, B, kPre, kBuffers);   // [32] cursor of every update
-    uint32_t* s_k = s_cur + 32;                                                 // [B][32] staged indices
-    float* s_v = reinterpret_cast<float*>(s_k + 32 * B);                        // [B][32] staged values
-    float* s_theta = s_v + 32 * B;                                              // [kBuffers][R] Theta of the range
-    uint32_t* s_head = reinterpret_cast<uint32_t*>(s_theta) + kBuffers * R;     // [kBuffers][R] latest change of the parameter
-    uint32_t* s_mask = s_head + kBuffers * R;                                          // [R] updates of this launch that changed it
+    float* s_theta = reinterpret_cast<float*>(s_wp) + 64 + warp * wp_warp_words(R, kPre);   // [2][R] Theta of the range
+    uint32_t* s_head = reinterpret_cast<uint32_t*>(s_theta) + 2 * R;            // [2][R] latest change of the parameter
+    uint32_t* s_mask = s_head + 2 * R;                                          // [R] updates of this launch that changed it
     uint32_t* s_head0 = s_mask + R;                                             // [R] head when the launch began (kPre)
-    uint32_t* s_hops = s_head0 + R;                                             // [B][32] chain entries inside the window before the launch (kPre)
 
     if (tid < kAlphaTable) s_alpha[tid] = tid ? __fdiv_rn(lr, static_cast<float>(tid)) : lr;   // Eq. 5 for the small counts, once
     __syncthreads();                                            // the only block barrier
@@ -197,22 +192,6 @@ k_apply_warps(const ServerParams sp, const BatchDesc d, const uint32_t* __restri
     const uint32_t r_hi = static_cast<uint32_t>(static_cast<uint64_t>(n_ranges) * (gw + 1) / n_gw);
     if (r_lo == r_hi) return;
 
-    constexpr bool kAhead = R <= 256;                           // dense updates: a stage is often used up within a range
-    const uint32_t a_k = smem_address(s_k + lane), a_v = smem_address(s_v + lane);
-    // the stage of update b takes its next 32 pairs from `cur` (kNone beyond the end of the list)
-    auto refill = [&](uint32_t b, uint32_t cur) {
-        const uint32_t t = cur + lane;
-        if (t < d.n_pairs[b]) {
-            copy_async_4(a_k + b * 128, idx + d.pair_begin[b] + t);
-            copy_async_4(a_v + b * 128, val + d.pair_begin[b] + t);
-            if (kAhead && t + 32 < d.n_pairs[b]) {              // the 32 pairs after these: wanted soon, or at once if all 32 lie in the range
-                prefetch_l2(idx + d.pair_begin[b] + t + 32);
-                prefetch_l2(val + d.pair_begin[b] + t + 32);
-            }
-        } else {
-            s_k[b * 32 + lane] = kNone;
-        }
-    };
     auto range_end = [&](uint32_t r) -> uint32_t {
         const uint64_t e = (static_cast<uint64_t>(r) + 1) * R;
         return e <= sp.n_params ? static_cast<uint32_t>(e) : static_cast<uint32_t>(sp.n_params);
@@ -234,152 +213,99 @@ k_apply_warps(const ServerParams sp, const BatchDesc d, const uint32_t* __restri
         }
     };
 
-    if (lane < B)                                               // cursor: first pair at or above the first owned parameter
-        s_cur[lane] = first_at_or_above(idx + d.pair_begin[lane], d.n_pairs[lane], static_cast<uint64_t>(r_lo) * R, sp.n_params);
-    __syncwarp();
-    for (uint32_t b = 0; b < B; ++b) refill(b, s_cur[b]);
-    sweep_in(r_lo, 0);
+    // ---- the registers that stand for the updates: cursor, and this lane's pair of the 32 at the cursor
+    uint32_t cur[NB], k[NB];
+    float v[NB];
+    {
+        uint32_t mine = 0;                                      // lane b: first pair of update b at or above the first owned parameter
+        if (lane < B) mine = first_at_or_above(idx + d.pair_begin[lane], d.n_pairs[lane], static_cast<uint64_t>(r_lo) * R, sp.n_params);
 #pragma unroll
-    for (uint32_t g = 0; g < kWpGroups + (kBuffers == 1 ? 1 : 0); ++g) copy_async_commit();   // the first holds everything, the others are empty
+        for (uint32_t b = 0; b < NB; ++b) cur[b] = __shfl_sync(0xFFFFFFFFu, mine, b & 31u);
+    }
+    // the lane's pair of update b at its cursor (kNone beyond the end of the list, and for updates the launch does not have)
+#define ADACOMP_WP_LOAD(b)                                                                    \
+    do {                                                                                      \
+        const uint32_t t_ = cur[b] + lane;                                                    \
+        k[b] = kNone;                                                                         \
+        v[b] = 0.f;                                                                           \
+        if ((b) < B && t_ < d.n_pairs[b]) {                                                   \
+            k[b] = __ldg(idx + d.pair_begin[b] + t_);                                         \
+            v[b] = __ldg(val + d.pair_begin[b] + t_);                                         \
+        }                                                                                     \
+    } while (0)
+#pragma unroll
+    for (uint32_t b = 0; b < NB; ++b) ADACOMP_WP_LOAD(b);
+    sweep_in(r_lo, 0);
+    copy_async_commit();
 
-    const uint32_t per_group = (B + kWpGroups - 1) / kWpGroups;     // <= 8
     for (uint32_t r = r_lo; r < r_hi; ++r) {
-        const uint32_t p = kBuffers == 2 ? (r - r_lo) & 1u : 0u;
+        const uint32_t p = (r - r_lo) & 1u;
         const uint32_t lo = r * R, hi = range_end(r);
         float* th = s_theta + p * R;
         uint32_t* hd = s_head + p * R;
-        if (kBuffers == 2) {
-            if (r + 1 < r_hi) sweep_in(r + 1, p ^ 1u);          // lands while this range is worked on
-        } else if (r + 1 < r_hi && lane * 32 < 2 * R) {         // one buffer: the next range's lines go to L2 for now
-            const uint32_t o = (lane * 32) % R;
-            if (static_cast<uint64_t>(r + 1) * R + o < sp.n_params)
-                prefetch_l2((lane * 32 < R ? reinterpret_cast<const uint32_t*>(sp.theta) : sp.head) + (r + 1) * R + o);
-        }
+        if (r + 1 < r_hi) sweep_in(r + 1, p ^ 1u);              // lands while this range is worked on
+        copy_async_commit();
 #pragma unroll
         for (uint32_t o = lane * 4; o < R; o += 128) *reinterpret_cast<uint4*>(s_mask + o) = make_uint4(0, 0, 0, 0);
-        // ---- the updates in arrival order
-#pragma unroll 1
-        for (uint32_t g = 0; g < kWpGroups; ++g) {
-            // what was issued a range ago for this group has landed (with one buffer every range ends with a group of
-            // its own, the next range's Theta and heads, which the first group waits for)
-            if (kBuffers == 2) copy_async_wait<kWpGroups - 1>();
-            else if (g == 0) copy_async_wait<0>();
-            else copy_async_wait<kWpGroups>();
+        copy_async_wait<1>();                                   // this range's Theta and heads have landed
+        __syncwarp();
+        if (kPre) {
+#pragma unroll
+            for (uint32_t o = lane * 4; o < R; o += 128)
+                *reinterpret_cast<uint4*>(s_head0 + o) = *reinterpret_cast<const uint4*>(hd + o);
             __syncwarp();
-            if (kPre && g == 0) {
+        }
+        // ---- the updates in arrival order
 #pragma unroll
-                for (uint32_t o = lane * 4; o < R; o += 128)
-                    *reinterpret_cast<uint4*>(s_head0 + o) = *reinterpret_cast<const uint4*>(hd + o);
-                __syncwarp();
-            }
-            const uint32_t b_first = g * per_group;
-            if (kPre) {
-                // Eq. 3 before the launch for the staged pairs of the group's updates: the walk from the head the
-                // parameter had when the launch began does not depend on the order inside the launch, so four
-                // updates' walks run side by side here instead of one after the other in the loop below
-                const uint32_t b_last = b_first + per_group < B ? b_first + per_group : B;
-#pragma unroll 1
-                for (uint32_t b0 = b_first; b0 < b_last; b0 += 4) {
-                    uint32_t q[4], ws[4], hp[4];
-#pragma unroll
-                    for (uint32_t u = 0; u < 4; ++u) {
-                        q[u] = kNone;
-                        ws[u] = 0;
-                        hp[u] = 0;
-                        if (b0 + u < b_last && ((d.pre_mask >> (b0 + u)) & 1u)) {
-                            const uint32_t k = s_k[(b0 + u) * 32 + lane];
-                            if (k >= lo && k < hi) {
-                                q[u] = s_head0[k - lo];
-                                ws[u] = d.win_start[b0 + u];
-                            }
-                        }
-                    }
-                    bool walking = true;
-                    while (walking) {
-                        walking = false;
-#pragma unroll
-                        for (uint32_t u = 0; u < 4; ++u) {
-                            if (q[u] != kNone && q[u] >= ws[u]) {
-                                if (++hp[u] > sp.max_window) { record_error(sp.status, ADACOMP_ERR_WINDOW); q[u] = kNone; }
-                                else q[u] = sp.prev[(q[u] + sp.ring_shift) & sp.ring_mask];
-                                walking = true;
-                            }
-                        }
-                    }
-#pragma unroll
-                    for (uint32_t u = 0; u < 4; ++u)
-                        if (b0 + u < b_last) s_hops[(b0 + u) * 32 + lane] = hp[u];
+        for (uint32_t b = 0; b < NB; ++b) {
+            if (b >= B) break;                                  // the same for every lane
+            uint32_t bal = __ballot_sync(0xFFFFFFFFu, k[b] < hi);
+            if (bal == 0) continue;                             // no pair of this update in the range
+            const uint32_t bits_b = d.win_bits[b], bit_b = 1u << b;
+            for (;;) {
+                const uint32_t kk = k[b];
+                if (kExtra && sp.validate) {
+                    uint32_t before = __shfl_up_sync(0xFFFFFFFFu, kk, 1);
+                    if (lane == 0) before = cur[b] > 0 ? idx[d.pair_begin[b] + cur[b] - 1] : 0u;
+                    if (kk < hi && cur[b] + lane > 0 && before >= kk) record_error(sp.status, ADACOMP_ERR_UNSORTED);
                 }
-                __syncwarp();
-            }
-            // which updates of the group have a pair in this range: lane t looks at the first staged index of update g * per_group + t
-            uint32_t first_k = kNone;
-            if (lane < per_group && b_first + lane < B) first_k = s_k[(b_first + lane) * 32];
-            uint32_t live = __ballot_sync(0xFFFFFFFFu, first_k < hi);
-#pragma unroll 1
-            while (live) {
-                const uint32_t b = b_first + __ffs(live) - 1;
-                live &= live - 1;
-                uint32_t k = s_k[b * 32 + lane];
-                float v = s_v[b * 32 + lane];
-                uint32_t cur = s_cur[b];
-                const uint32_t bits_b = d.win_bits[b], bit_b = 1u << b, pos_l = d.pos_start[b] + lane;
-                uint32_t bal = __ballot_sync(0xFFFFFFFFu, k < hi);
-                bool staged = true;                             // these 32 pairs come from the stage: their walks are done
-                for (;;) {
-                    if (kExtra && sp.validate) {
-                        uint32_t before = __shfl_up_sync(0xFFFFFFFFu, k, 1);
-                        if (lane == 0) before = cur > 0 ? idx[d.pair_begin[b] + cur - 1] : 0u;
-                        if (k < hi && cur + lane > 0 && before >= k) record_error(sp.status, ADACOMP_ERR_UNSORTED);
-                    }
-                    if (k < hi) {
-                        if (k >= lo) {
-                            const uint32_t kl = k - lo;
-                            const bool change = v != 0.0f;      // Eq. 3 counts changes: a zero entry is not one
-                            const uint32_t m = change ? atomicOr(&s_mask[kl], bit_b) : s_mask[kl];
-                            uint32_t sigma = __popc(m & bits_b);                                       // Eq. 3, inside the launch
-                            if (kPre && (d.pre_mask & bit_b)) {                                        // Eq. 3, before the launch
-                                if (staged) {
-                                    sigma += s_hops[b * 32 + lane];
-                                } else {
-                                    const uint32_t ws = d.win_start[b];
-                                    uint32_t q = s_head0[kl], hops = 0;
-                                    while (q != kNone && q >= ws) {
-                                        if (++hops > sp.max_window) { record_error(sp.status, ADACOMP_ERR_WINDOW); break; }
-                                        q = sp.prev[(q + sp.ring_shift) & sp.ring_mask];
-                                    }
-                                    sigma += hops;
-                                }
+                if (kk < hi) {
+                    if (kk >= lo) {
+                        const uint32_t kl = kk - lo;
+                        const float vv = v[b];
+                        const bool change = vv != 0.0f;         // Eq. 3 counts changes: a zero entry is not one
+                        const uint32_t m = s_mask[kl];           // lanes of one update hold distinct parameters: no atomics
+                        if (change) s_mask[kl] = m | bit_b;
+                        uint32_t sigma = __popc(m & bits_b);                                           // Eq. 3, inside the launch
+                        if (kPre && (d.pre_mask & bit_b)) {                                            // Eq. 3, before the launch
+                            const uint32_t ws = d.win_start[b];
+                            uint32_t q = s_head0[kl], hops = 0;
+                            while (q != kNone && q >= ws) {
+                                if (++hops > sp.max_window) { record_error(sp.status, ADACOMP_ERR_WINDOW); break; }
+                                q = sp.prev[(q + sp.ring_shift) & sp.ring_mask];
                             }
-                            if (kExtra && sigma_out) sigma_out[d.pair_begin[b] + cur + lane] = sigma;
-                            if (change) {
-                                const float alpha_k = sigma < kAlphaTable ? s_alpha[sigma] : __fdiv_rn(lr, static_cast<float>(sigma));   // Eq. 5
-                                th[kl] = __fsub_rn(th[kl], __fmul_rn(alpha_k, v));                     // Eq. 4
-                                const uint32_t pos = pos_l + cur;
-                                sp.prev[(pos + sp.ring_shift) & sp.ring_mask] = atomicExch(&hd[kl], pos);
-                            }
-                        } else {                                // an index before the range: the list was not ascending
-                            record_error(sp.status, ADACOMP_ERR_UNSORTED);
+                            sigma += hops;
                         }
+                        if (kExtra && sigma_out) sigma_out[d.pair_begin[b] + cur[b] + lane] = sigma;
+                        if (change) {
+                            const float alpha_k = sigma < kAlphaTable ? s_alpha[sigma] : __fdiv_rn(lr, static_cast<float>(sigma));   // Eq. 5
+                            th[kl] = __fsub_rn(th[kl], __fmul_rn(alpha_k, vv));                        // Eq. 4
+                            const uint32_t pos = d.pos_start[b] + cur[b] + lane;
+                            sp.prev[(pos + sp.ring_shift) & sp.ring_mask] = hd[kl];
+                            hd[kl] = pos;
+                        }
+                    } else {                                    // an index before the range: the list was not ascending
+                        record_error(sp.status, ADACOMP_ERR_UNSORTED);
                     }
-                    __syncwarp();                               // the next update sees this one's changes
-                    const uint32_t cnt = __popc(bal);
-                    cur += cnt;
-                    if (cnt < 32) break;
-                    const uint32_t t = cur + lane;              // the update may have more pairs in this range
-                    staged = false;
-                    k = kNone;
-                    if (t < d.n_pairs[b]) {
-                        k = idx[d.pair_begin[b] + t];
-                        v = val[d.pair_begin[b] + t];
-                    }
-                    bal = __ballot_sync(0xFFFFFFFFu, k < hi);
-                    if (bal == 0) break;
                 }
-                if (lane == 0) s_cur[b] = cur;
-                refill(b, cur);
+                __syncwarp();                                   // the next update sees this one's changes
+                const uint32_t cnt = __popc(bal);
+                cur[b] += cnt;
+                ADACOMP_WP_LOAD(b);                             // the next 32 pairs from the new cursor: wanted a range from now
+                if (cnt < 32) break;
+                bal = __ballot_sync(0xFFFFFFFFu, k[b] < hi);    // all 32 lay in the range: the update may have more there
+                if (bal == 0) break;
             }
-            copy_async_commit();
         }
         // ---- Theta and heads go back where a parameter changed
         if (hi - lo == R) {
@@ -396,15 +322,15 @@ k_apply_warps(const ServerParams sp, const BatchDesc d, const uint32_t* __restri
                 if (lo + o < hi && s_mask[o]) { sp.theta[lo + o] = th[o]; sp.head[lo + o] = hd[o]; }
         }
         __syncwarp();
-        if (kBuffers == 1) {
-            if (r + 1 < r_hi) sweep_in(r + 1, 0);
-            copy_async_commit();
-        }
     }
     copy_async_wait<0>();
-    __syncwarp();
     // whoever owns the last range sees what no range claimed: indices >= n_params
-    if (r_hi == n_ranges && lane < B && s_cur[lane] < d.n_pairs[lane]) record_error(sp.status, ADACOMP_ERR_UNSORTED);
+    if (r_hi == n_ranges) {
+#pragma unroll
+        for (uint32_t b = 0; b < NB; ++b)
+            if (b < B && cur[b] < d.n_pairs[b] && lane == 0) record_error(sp.status, ADACOMP_ERR_UNSORTED);
+    }
+#undef ADACOMP_WP_LOAD
 }
 
 // ---------------------------------------------------------------------------------------------
@@ -889,41 +815,40 @@ int resident_blocks(const adacomp_server_t* s, Kernel kernel, int threads, size_
     return ADACOMP_OK;
 }
 
-// Launches k_apply_warps<R, kBuffers, kPre, kExtra> over all ranges of R parameters with as many blocks as stay resident.
-template <uint32_t R, uint32_t kBuffers, bool kPre, bool kExtra>
+// Launches k_apply_warps<R, NB, kPre, kExtra> over all ranges of R parameters with as many blocks as stay resident.
+template <uint32_t R, uint32_t NB, bool kPre, bool kExtra>
 int launch_apply_warps_as(const adacomp_server_t* s, const ServerParams& sp, const BatchDesc& d, const uint32_t* d_idx,
                           const float* d_val, float lr, uint32_t* d_sigma_out, cudaStream_t st) {
-    const size_t smem = wp_smem_bytes(R, d.n_updates, kPre, kBuffers);
+    const size_t smem = wp_smem_bytes(R, kPre);
     const uint32_t n_ranges = static_cast<uint32_t>((s->n_params + R - 1) / R);
     int per_sm = 1;
-    const int rc = resident_blocks(s, k_apply_warps<R, kBuffers, kPre, kExtra>, kWpThreads, smem,
-                                   wp_smem_bytes(R, kMaxBatch, kPre, kBuffers), &per_sm);
+    const int rc = resident_blocks(s, k_apply_warps<R, NB, kPre, kExtra>, kWpThreads, smem, smem, &per_sm);
     if (rc != ADACOMP_OK) return rc;
     unsigned grid = static_cast<unsigned>(s->n_sms) * static_cast<unsigned>(per_sm > 0 ? per_sm : 1);
     const unsigned most_blocks = (n_ranges + kWpWarps - 1) / kWpWarps;
     if (grid > most_blocks) grid = most_blocks;
-    k_apply_warps<R, kBuffers, kPre, kExtra><<<grid, kWpThreads, smem, st>>>(sp, d, d_idx, d_val, lr, d_sigma_out, n_ranges);
+    k_apply_warps<R, NB, kPre, kExtra><<<grid, kWpThreads, smem, st>>>(sp, d, d_idx, d_val, lr, d_sigma_out, n_ranges);
     ADACOMP_LAUNCH_CHECK();
     return ADACOMP_OK;
 }
 
-template <uint32_t R, uint32_t kBuffers>
+template <uint32_t R, uint32_t NB>
 int launch_apply_warps_with(const adacomp_server_t* s, const ServerParams& sp, const BatchDesc& d, const uint32_t* d_idx,
                             const float* d_val, float lr, uint32_t* d_sigma_out, cudaStream_t st) {
     const bool pre = d.pre_mask != 0, extra = d_sigma_out != nullptr || sp.validate != 0;
-    if (pre) return extra ? launch_apply_warps_as<R, kBuffers, true, true>(s, sp, d, d_idx, d_val, lr, d_sigma_out, st)
-                          : launch_apply_warps_as<R, kBuffers, true, false>(s, sp, d, d_idx, d_val, lr, d_sigma_out, st);
-    return extra ? launch_apply_warps_as<R, kBuffers, false, true>(s, sp, d, d_idx, d_val, lr, d_sigma_out, st)
-                 : launch_apply_warps_as<R, kBuffers, false, false>(s, sp, d, d_idx, d_val, lr, d_sigma_out, st);
+    if (pre) return extra ? launch_apply_warps_as<R, NB, true, true>(s, sp, d, d_idx, d_val, lr, d_sigma_out, st)
+                          : launch_apply_warps_as<R, NB, true, false>(s, sp, d, d_idx, d_val, lr, d_sigma_out, st);
+    return extra ? launch_apply_warps_as<R, NB, false, true>(s, sp, d, d_idx, d_val, lr, d_sigma_out, st)
+                 : launch_apply_warps_as<R, NB, false, false>(s, sp, d, d_idx, d_val, lr, d_sigma_out, st);
 }
 
+// The unrolled loop over the updates comes in two lengths: launches of up to 16 updates keep 16 pairs per lane in
+// registers, longer ones 32.
 template <uint32_t R>
 int launch_apply_warps(const adacomp_server_t* s, const ServerParams& sp, const BatchDesc& d, const uint32_t* d_idx,
                        const float* d_val, float lr, uint32_t* d_sigma_out, cudaStream_t st) {
-    if constexpr (R > 256) {
-        if (d.n_updates > 8) return launch_apply_warps_with<R, 1>(s, sp, d, d_idx, d_val, lr, d_sigma_out, st);
-    }
-    return launch_apply_warps_with<R, 2>(s, sp, d, d_idx, d_val, lr, d_sigma_out, st);
+    if (d.n_updates <= 16) return launch_apply_warps_with<R, 16>(s, sp, d, d_idx, d_val, lr, d_sigma_out, st);
+    return launch_apply_warps_with<R, 32>(s, sp, d, d_idx, d_val, lr, d_sigma_out, st);
 }
 
 // Launches k_apply_merged<R, kPre, kExtra>.  R = 0: only the named parameters are touched, ranges sized so that
