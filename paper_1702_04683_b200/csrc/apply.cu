@@ -152,7 +152,7 @@ constexpr int kWpThreads = 128;
 constexpr uint32_t kWpWarps = kWpThreads / 32;
 
 __host__ __device__ inline size_t wp_warp_words(uint32_t range, bool pre) {
-    return (pre ? 6 : 5) * static_cast<size_t>(range);          // Theta and heads twice, masks, (heads at the launch's start)
+    return (pre ? 7 : 6) * static_cast<size_t>(range);          // Theta twice, (mask, head) records twice, (heads at the launch's start)
 }
 __host__ __device__ inline size_t wp_smem_bytes(uint32_t range, bool pre) {
     return 64 * 4 + kWpWarps * wp_warp_words(range, pre) * 4;
@@ -181,9 +181,11 @@ k_apply_warps(const ServerParams sp, const BatchDesc d, const uint32_t* __restri
     const uint32_t B = d.n_updates;                                             // <= NB
     const uint32_t tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     float* s_theta = reinterpret_cast<float*>(s_wp) + 64 + warp * wp_warp_words(R, kPre);   // [2][R] Theta of the range
-    uint32_t* s_head = reinterpret_cast<uint32_t*>(s_theta) + 2 * R;            // [2][R] latest change of the parameter
-    uint32_t* s_mask = s_head + 2 * R;                                          // [R] updates of this launch that changed it
-    uint32_t* s_head0 = s_mask + R;                                             // [R] head when the launch began (kPre)
+    // [2][R] per parameter ONE 8-byte record: .x = updates of this launch that changed it (mask), .y = its latest change
+    // (head).  A pair reads and writes both with one access each: the shared-memory pipe is what bounds this kernel, and
+    // lanes that fall on the same bank cost a pass each.
+    uint2* s_rec = reinterpret_cast<uint2*>(s_theta + 2 * R);
+    uint32_t* s_head0 = reinterpret_cast<uint32_t*>(s_rec + 2 * R);             // [R] head when the launch began (kPre)
 
     if (tid < kAlphaTable) s_alpha[tid] = tid ? __fdiv_rn(lr, static_cast<float>(tid)) : lr;   // Eq. 5 for the small counts, once
     __syncthreads();                                            // the only block barrier
@@ -201,14 +203,13 @@ k_apply_warps(const ServerParams sp, const BatchDesc d, const uint32_t* __restri
         const uint32_t lo = r * R, hi = range_end(r);
         if (hi - lo == R) {
 #pragma unroll
-            for (uint32_t o = lane * 4; o < R; o += 128) {
-                copy_async_16(smem_address(s_theta + p * R + o), sp.theta + lo + o);
-                copy_async_16(smem_address(s_head + p * R + o), sp.head + lo + o);
-            }
+            for (uint32_t o = lane * 4; o < R; o += 128) copy_async_16(smem_address(s_theta + p * R + o), sp.theta + lo + o);
+#pragma unroll
+            for (uint32_t o = lane; o < R; o += 32) copy_async_4(smem_address(&s_rec[p * R + o].y), sp.head + lo + o);
         } else {                                                // the last range may be short: plain loads
             for (uint32_t o = lane; o < R; o += 32) {
                 s_theta[p * R + o] = lo + o < hi ? sp.theta[lo + o] : 0.f;
-                s_head[p * R + o] = lo + o < hi ? sp.head[lo + o] : kNone;
+                s_rec[p * R + o].y = lo + o < hi ? sp.head[lo + o] : kNone;
             }
         }
     };
@@ -242,17 +243,16 @@ k_apply_warps(const ServerParams sp, const BatchDesc d, const uint32_t* __restri
         const uint32_t p = (r - r_lo) & 1u;
         const uint32_t lo = r * R, hi = range_end(r);
         float* th = s_theta + p * R;
-        uint32_t* hd = s_head + p * R;
+        uint2* rec = s_rec + p * R;
         if (r + 1 < r_hi) sweep_in(r + 1, p ^ 1u);              // lands while this range is worked on
         copy_async_commit();
 #pragma unroll
-        for (uint32_t o = lane * 4; o < R; o += 128) *reinterpret_cast<uint4*>(s_mask + o) = make_uint4(0, 0, 0, 0);
+        for (uint32_t o = lane; o < R; o += 32) rec[o].x = 0u;  // (the heads of this buffer were copied in a range ago: other bytes)
         copy_async_wait<1>();                                   // this range's Theta and heads have landed
         __syncwarp();
         if (kPre) {
 #pragma unroll
-            for (uint32_t o = lane * 4; o < R; o += 128)
-                *reinterpret_cast<uint4*>(s_head0 + o) = *reinterpret_cast<const uint4*>(hd + o);
+            for (uint32_t o = lane; o < R; o += 32) s_head0[o] = rec[o].y;
             __syncwarp();
         }
         // ---- the updates in arrival order
@@ -274,9 +274,8 @@ k_apply_warps(const ServerParams sp, const BatchDesc d, const uint32_t* __restri
                         const uint32_t kl = kk - lo;
                         const float vv = v[b];
                         const bool change = vv != 0.0f;         // Eq. 3 counts changes: a zero entry is not one
-                        const uint32_t m = s_mask[kl];           // lanes of one update hold distinct parameters: no atomics
-                        if (change) s_mask[kl] = m | bit_b;
-                        uint32_t sigma = __popc(m & bits_b);                                           // Eq. 3, inside the launch
+                        const uint2 mh = rec[kl];                // lanes of one update hold distinct parameters: no atomics
+                        uint32_t sigma = __popc(mh.x & bits_b);                                        // Eq. 3, inside the launch
                         if (kPre && (d.pre_mask & bit_b)) {                                            // Eq. 3, before the launch
                             const uint32_t ws = d.win_start[b];
                             uint32_t q = s_head0[kl], hops = 0;
@@ -291,8 +290,8 @@ k_apply_warps(const ServerParams sp, const BatchDesc d, const uint32_t* __restri
                             const float alpha_k = sigma < kAlphaTable ? s_alpha[sigma] : __fdiv_rn(lr, static_cast<float>(sigma));   // Eq. 5
                             th[kl] = __fsub_rn(th[kl], __fmul_rn(alpha_k, vv));                        // Eq. 4
                             const uint32_t pos = d.pos_start[b] + cur[b] + lane;
-                            sp.prev[(pos + sp.ring_shift) & sp.ring_mask] = hd[kl];
-                            hd[kl] = pos;
+                            sp.prev[(pos + sp.ring_shift) & sp.ring_mask] = mh.y;
+                            rec[kl] = make_uint2(mh.x | bit_b, pos);
                         }
                     } else {                                    // an index before the range: the list was not ascending
                         record_error(sp.status, ADACOMP_ERR_UNSORTED);
@@ -311,15 +310,15 @@ k_apply_warps(const ServerParams sp, const BatchDesc d, const uint32_t* __restri
         if (hi - lo == R) {
 #pragma unroll
             for (uint32_t o = lane * 4; o < R; o += 128) {
-                const uint4 m4 = *reinterpret_cast<const uint4*>(s_mask + o);
-                if (m4.x | m4.y | m4.z | m4.w) {
+                const uint4 a = *reinterpret_cast<const uint4*>(rec + o), c = *reinterpret_cast<const uint4*>(rec + o + 2);   // records o .. o + 3
+                if (a.x | a.z | c.x | c.z) {
                     *reinterpret_cast<float4*>(sp.theta + lo + o) = *reinterpret_cast<const float4*>(th + o);
-                    *reinterpret_cast<uint4*>(sp.head + lo + o) = *reinterpret_cast<const uint4*>(hd + o);
+                    *reinterpret_cast<uint4*>(sp.head + lo + o) = make_uint4(a.y, a.w, c.y, c.w);
                 }
             }
         } else {
             for (uint32_t o = lane; o < R; o += 32)
-                if (lo + o < hi && s_mask[o]) { sp.theta[lo + o] = th[o]; sp.head[lo + o] = hd[o]; }
+                if (lo + o < hi && rec[o].x) { sp.theta[lo + o] = th[o]; sp.head[lo + o] = rec[o].y; }
         }
         __syncwarp();
     }
