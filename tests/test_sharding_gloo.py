@@ -91,6 +91,81 @@ def test_two_rank_parameter_sharding_matches_one_server():
             assert np.array_equal(sig, full[sel])
 
 
+class OracleApplier:
+    """The oracle behind the interface of the library's server: lets ShardedServer run on CPU ranks."""
+
+    def __init__(self, theta):
+        self.srv = oracle.Server(theta)
+
+    @property
+    def timestamp(self):
+        return self.srv.timestamp
+
+    def apply(self, idx, val, begin, count, pull_ts, lr, sigma_out=None):
+        i, v = idx.numpy().view(np.uint32), val.numpy()
+        for b in range(len(begin)):
+            lo, n = int(begin[b]), int(count[b])
+            sig = self.srv.apply(i[lo:lo + n], v[lo:lo + n], int(pull_ts[b]), lr)
+            if sigma_out is not None:
+                sigma_out.numpy().view(np.uint32)[lo:lo + n] = sig
+
+
+def sharded_worker(rank, world, port, q):
+    os.environ.update(MASTER_ADDR="127.0.0.1", MASTER_PORT=str(port))
+    dist.init_process_group("gloo", rank=rank, world_size=world)
+    try:
+        wl, ks = scenario()
+        per_rank = wl.n_workers // world
+        ranges = sharding.parameter_ranges(wl.n_params, world)
+        lo, hi = ranges[rank]
+        theta0 = wlmod.initial_parameters(wl, "cpu")
+        shard = theta0[lo:hi].clone()
+        srv = sharding.ShardedServer(shard, wl.n_params, per_rank, history_pairs=1 << 16, max_window_updates=64,
+                                     applier=OracleApplier(shard.numpy()))
+        log = []
+        for r, rd in enumerate(wlmod.arrival_schedule(wl)):
+            idx_all, val_all = wlmod.synthetic_updates(wl, ks, r, "cpu", zero_fraction=0.05)    # int32 holding uint32 bits
+            mine = slice(rank * per_rank, (rank + 1) * per_rank)
+            sigma, begin, count = srv.step(idx_all[mine], val_all[mine], rd.order, rd.pull_ts, wl.lr, want_sigma=True)
+            for w in range(wl.n_workers):
+                log.append((r, w, sigma.numpy().view(np.uint32)[int(begin[w]):int(begin[w]) + int(count[w])].copy()))
+        q.put((rank, lo, hi, srv.applier.srv.theta(), srv.timestamp, log))
+    finally:
+        dist.destroy_process_group()
+
+
+def test_sharded_server_class_matches_one_server():
+    """The class a multi-GPU job uses (exchange, then the local apply in global arrival order), driven on
+    two CPU ranks with the oracle as the local applier: staleness counts and parameters of the shards
+    are those of one server that sees everything."""
+    world = 2
+    ctx = mp.get_context("spawn")
+    q = ctx.Queue()
+    port = free_port()
+    procs = [ctx.Process(target=sharded_worker, args=(r, world, port, q)) for r in range(world)]
+    for p in procs:
+        p.start()
+    results = sorted(q.get(timeout=180) for _ in range(world))
+    for p in procs:
+        p.join(timeout=60)
+        assert p.exitcode == 0
+    wl, ks = scenario()
+    ref = oracle.Server(wlmod.initial_parameters(wl, "cpu").numpy())
+    ref_sig = {}
+    for r, rd in enumerate(wlmod.arrival_schedule(wl)):
+        idx_all, val_all = wlmod.synthetic_updates(wl, ks, r, "cpu", zero_fraction=0.05)
+        for b, w in enumerate(rd.order.tolist()):
+            i32 = idx_all[w].numpy().view(np.uint32)
+            ref_sig[(r, w)] = (i32, ref.apply(i32, val_all[w].numpy(), int(rd.pull_ts[b]), wl.lr))
+    want = ref.theta()
+    for rank, lo, hi, theta, ts, log in results:
+        assert ts == ref.timestamp
+        assert np.array_equal(theta.view(np.uint32), want[lo:hi].view(np.uint32))
+        for r, w, sig in log:
+            i32, full = ref_sig[(r, w)]
+            assert np.array_equal(sig, full[(i32 >= lo) & (i32 < hi)])
+
+
 def test_ranges_and_slice_points():
     ranges = sharding.parameter_ranges(10_000, 4)
     assert ranges[0][0] == 0 and ranges[-1][1] == 10_000
