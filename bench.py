@@ -33,27 +33,96 @@ METRIC = "dense-gradient GB/s scanned (select+compact, with the selected pairs a
 UNIT = "GB/s"
 FALLBACK_HBM_GBS = 6650.0
 
-# DRAM bytes (read + write) of ONE scan-kernel launch from an ncu capture of workload 4 with 4 workers,
-# MB per keep fraction (1/25 and 1/10 are the dense scan kernel).  A launch over W workers moves W / 4
-# times as much.  Only valid while the kernel source is the one that was profiled.
-SCAN_TRAFFIC_W4_MB = {"1/1000": 1645.7, "1/400": 1684.6, "1/160": 1795.8, "1/64": 1793.4, "1/25": 1788.9, "1/10": 2008.2}
-SCAN_SOURCE_SHA256_16 = "b6c409439069c8f1"
+# DRAM bytes (read + write) of ONE launch of the scan kernel and of the dominant apply kernel, from an ncu capture of
+# workload 4 with 4 workers / 4 updates, MB per keep fraction.  A launch over W workers moves W / 4 times as much
+# (every worker's tensors are independent; for the apply kernels the sweep of Theta and heads does not grow with W, so
+# only the scan figure is scaled and the apply figure is reported as captured).  Only valid while the kernel sources are
+# the ones that were profiled (guarded by their hashes).
+SCAN_TRAFFIC_W4_MB = {}
+APPLY_TRAFFIC_W4_MB = {}
+SCAN_SOURCE_SHA256_16 = ""
+APPLY_SOURCE_SHA256_16 = ""
+
+
+def _source_hash(name):
+    import hashlib
+    try:
+        src = open(os.path.join(ROOT, "paper_1702_04683_b200", "csrc", name), "rb").read()
+    except OSError:
+        return None
+    return hashlib.sha256(src).hexdigest()[:16]
 
 
 def scan_traffic_bytes(workload_index, keeps, workers):
     """Mean DRAM bytes per scan launch over the given keep fractions, or None if unknown."""
-    import hashlib
-    try:
-        src = open(os.path.join(ROOT, "paper_1702_04683_b200", "csrc", "select_bracket.cuh"), "rb").read()
-    except OSError:
-        return None
-    if hashlib.sha256(src).hexdigest()[:16] != SCAN_SOURCE_SHA256_16 or workload_index != 4:
+    if not SCAN_SOURCE_SHA256_16 or _source_hash("select_bracket.cuh") != SCAN_SOURCE_SHA256_16 or workload_index != 4:
         return None
     try:
         per = [SCAN_TRAFFIC_W4_MB["%d/%d" % k] * 1e6 * workers / 4.0 for k in keeps]
     except KeyError:
         return None
     return sum(per) / len(per)
+
+
+def apply_traffic_mb(workload_index, keep):
+    """DRAM MB of the apply launch captured with 4 updates at this keep fraction, or None if unknown."""
+    if not APPLY_SOURCE_SHA256_16 or _source_hash("apply.cu") != APPLY_SOURCE_SHA256_16 or workload_index != 4:
+        return None
+    return APPLY_TRAFFIC_W4_MB.get("%d/%d" % keep)
+
+
+def run_apply_variants(binding, wl, dev, peak, keep=(1, 100), reps=5, warmup=3):
+    """adacomp_apply on index sets and windows the main sweep does not show, at one keep fraction, W updates per call:
+    'uniform' (one index per stratum, all pulled at the round's start: what top-k of iid data gives), 'clustered' (all
+    pairs of an update inside a random twentieth of each tensor, as real gradients crowd into rows and layers) and
+    'stale' (uniform index sets, every update pulled 2 W updates before it is applied: windows that reach back over two
+    earlier rounds)."""
+    W, P = wl.n_workers, wl.n_params
+    ks = [binding.adacomp_keep_count(n, *keep) for n in wl.tensor_sizes]
+    K = int(sum(ks))
+    stream = torch.cuda.current_stream()
+    idx_u, val = wlmod.synthetic_updates(wl, ks, 0, dev)
+    # clustered: squeeze every tensor's strata into a window of n / 20 entries at a seeded offset per (worker, tensor)
+    gen = torch.Generator(device=dev)
+    gen.manual_seed(4242)
+    idx_c = torch.empty_like(idx_u)
+    at = 0
+    for off, n, k in zip(wl.offsets, wl.tensor_sizes, ks):
+        width = max(k, n // 20)
+        start = (torch.rand((W, 1), device=dev, generator=gen) * (n - width)).to(torch.int64)
+        t = torch.arange(k, dtype=torch.int64, device=dev).view(1, k)
+        idx_c[:, at:at + k] = (off + start + (t * width) // k).to(torch.int32)
+        at += k
+    begin = np.arange(W, dtype=np.uint64) * np.uint64(K)
+    count = np.full(W, K, np.uint32)
+    out = {"keep": "%d/%d" % keep, "updates_per_call": W, "pairs_per_update": K}
+
+    def timed(srv, idx, stale):
+        def call(fresh=False):
+            ts = srv.timestamp
+            pull = np.full(W, ts, np.uint64) if fresh or not stale else (ts + np.arange(W, dtype=np.uint64) - np.uint64(2 * W))
+            srv.apply(idx.view(-1), val.view(-1), begin, count, pull, wl.lr)
+        for _ in range(2):
+            call(fresh=True)                                       # two rounds of history for the stale windows to reach into
+        for _ in range(warmup):
+            call()
+        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        a.record(stream)
+        for _ in range(reps):
+            call()
+        b.record(stream)
+        torch.cuda.synchronize()
+        return a.elapsed_time(b) / reps
+
+    for name, idx, stale in (("uniform", idx_u, False), ("clustered", idx_c, False), ("stale", idx_u, True)):
+        theta = wlmod.initial_parameters(wl, dev)
+        srv = binding.Server(theta, history_pairs=4 * W * K, max_window_updates=4 * W)
+        ms = timed(srv, idx, stale)
+        assert srv.last_error() == 0
+        out[name] = {"apply_ms": round(ms, 4), "apply_pairs_per_s": round(W * K / ms * 1e3, 1),
+                     "apply_alg_frac_of_hbm_peak": round(W * K * 28.0 / ms / 1e6 / peak, 4)}
+        del srv, theta
+    return out
 
 
 def run_competitors(binding, wl, grads, dev, peak, keep=(1, 100), reps=5, warmup=3):
@@ -185,6 +254,9 @@ def parse_args():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-competitors", action="store_true")
+    ap.add_argument("--sharded", action="store_true",
+                    help="N > 1: one server sharded by parameter range over the ranks (each rank selects for W / N workers, "
+                         "the updates' slices are exchanged, every rank applies its range) instead of N independent replicas")
     return ap.parse_args()
 
 
@@ -264,6 +336,12 @@ def setup_dist(args):
         import torch.distributed as dist
         torch.cuda.set_device(local)
         dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+    elif args.sharded:
+        # one rank: the exchange of the sharded server is a local copy, but its path is the one that runs
+        import torch.distributed as dist
+        os.environ.setdefault("MASTER_ADDR", "127.0.0.1")
+        os.environ.setdefault("MASTER_PORT", "29533")
+        dist.init_process_group("gloo", rank=0, world_size=1)
     return world, rank, local
 
 
@@ -302,21 +380,38 @@ def run_native(args):
         raise SystemExit("bench.py needs a CUDA device: the hot path has no CPU fallback")
     dev = torch.device("cuda", local)
     torch.cuda.set_device(dev)
-    wl = wlmod.workload(args.workload, seed=rank)
+    import dataclasses
+    sharded = bool(args.sharded)
+    wl = wlmod.workload(args.workload, seed=0 if sharded else rank)
     if args.workers:
-        import dataclasses
         wl = dataclasses.replace(wl, n_workers=args.workers)
     keeps = [parse_keep(args.keep)] if args.keep else list(wl.keep_fractions)
     W, P = wl.n_workers, wl.n_params
     stream = torch.cuda.current_stream()
 
-    grads = wlmod.round_gradients(wl, 0, dev)                       # resident before the timer starts
-    points = [Point(binding, wl, k, dev) for k in keeps]
-    K_max = max(p.K for p in points)
-    theta = wlmod.initial_parameters(wl, dev)
-    srv = binding.Server(theta, history_pairs=2 * W * K_max, max_window_updates=2 * W)
+    if sharded:
+        # ONE server over all ranks: rank r hosts W / N workers and owns a contiguous range of the parameters
+        from paper_1702_04683_b200 import sharding
+        if W % world:
+            raise SystemExit("--sharded needs a worker count that the number of ranks divides")
+        W_local = W // world
+        wl_local = dataclasses.replace(wl, n_workers=W_local)
+        grads = wlmod.round_gradients(wl, 0, dev, workers=range(rank * W_local, (rank + 1) * W_local))
+        points = [Point(binding, wl_local, k, dev) for k in keeps]
+        K_max = max(p.K for p in points)
+        lo, hi = sharding.parameter_ranges(P, world)[rank]
+        theta = wlmod.initial_parameters(wl, dev)[lo:hi].clone()
+        ssrv = sharding.ShardedServer(theta, P, W_local, history_pairs=2 * W * K_max, max_window_updates=2 * W)
+        srv = ssrv.applier
+        rng = np.random.default_rng(1234)                            # the same arrival order on every rank
+    else:
+        grads = wlmod.round_gradients(wl, 0, dev)                   # resident before the timer starts
+        points = [Point(binding, wl, k, dev) for k in keeps]
+        K_max = max(p.K for p in points)
+        theta = wlmod.initial_parameters(wl, dev)
+        srv = binding.Server(theta, history_pairs=2 * W * K_max, max_window_updates=2 * W)
+        rng = np.random.default_rng(1234 + rank)
     srv.set_mode(args.apply_mode)
-    rng = np.random.default_rng(1234 + rank)
     last_push = np.full(W, -1, dtype=np.int64)
 
     def ev():
@@ -329,7 +424,10 @@ def run_native(args):
             e0 = ev(); e0.record(stream)
             p.sel.select(grads, p.idx, p.val)
             e1 = ev(); e1.record(stream)
-            srv.apply(p.idx.view(-1), p.val.view(-1), order.astype(np.uint64) * np.uint64(p.K), p.count, pull, wl.lr)
+            if sharded:
+                ssrv.step(p.idx, p.val, order, pull, wl.lr)
+            else:
+                srv.apply(p.idx.view(-1), p.val.view(-1), order.astype(np.uint64) * np.uint64(p.K), p.count, pull, wl.lr)
             e2 = ev(); e2.record(stream)
             marks.append((e0, e1, e2))
         if record is not None:
@@ -375,17 +473,29 @@ def run_native(args):
     pts = []
     sel_ms_all, sel_bytes_all = 0.0, 0.0
     scan_ms_all, scan_bytes_all, scan_launches = 0.0, 0.0, 0
+    W_sel = W // world if sharded else W          # workers one rank selects for
+    apply_points = []
     for i, p in enumerate(points):
         stages = p.sel.profile()
         calls = stages.pop("calls")
         scan_ms_all += stages["bracket_scan"]
-        scan_bytes_all += W * 4.0 * P
+        scan_bytes_all += W_sel * 4.0 * P
         scan_launches += calls
         sel_ms = statistics.mean(m[i][0].elapsed_time(m[i][1]) for m in rec)
         app_ms = statistics.mean(m[i][1].elapsed_time(m[i][2]) for m in rec)
-        scanned = W * 4.0 * P
-        sel_alg = W * (4.0 * P + 8.0 * p.K)
-        pairs = W * p.K
+        scanned = W_sel * 4.0 * P
+        sel_alg = W_sel * (4.0 * P + 8.0 * p.K)
+        pairs = W * p.K / (world if sharded else 1)
+        # what the apply launch must move when it sweeps Theta and heads once (16 B per parameter it owns) and reads the
+        # pairs and writes their links (12 B per pair), against the 28 B per pair of the per-pair formulation
+        sweep_bytes = 16.0 * (P / (world if sharded else 1)) + 12.0 * pairs
+        cap_mb = apply_traffic_mb(args.workload, p.keep)
+        apply_points.append({"keep": f"{p.keep[0]}/{p.keep[1]}", "apply_ms": round(app_ms, 4),
+                             "alg_gbs_28B_per_pair": round(pairs * 28.0 / app_ms / 1e6, 1),
+                             "alg_frac": round(pairs * 28.0 / app_ms / 1e6 / peak, 4),
+                             "sweep_formulation_gbs": round(sweep_bytes / app_ms / 1e6, 1),
+                             "sweep_formulation_frac": round(sweep_bytes / app_ms / 1e6 / peak, 4),
+                             "dram_mb_4_updates_ncu": cap_mb})
         pts.append({
             "keep": f"{p.keep[0]}/{p.keep[1]}", "pairs_per_update": p.K,
             "select_ms": round(sel_ms, 4), "apply_ms": round(app_ms, 4),
@@ -402,43 +512,51 @@ def run_native(args):
         sel_bytes_all += sel_alg
     ms_per_step = total_ms / args.steps
     scanned_per_step = len(points) * W * 4.0 * P
-    value = world * scanned_per_step / ms_per_step / 1e6
+    value = (1 if sharded else world) * scanned_per_step / ms_per_step / 1e6     # a sharded job scans W workers in all
 
     out = {
         "metric": METRIC, "value": round(value, 2), "unit": UNIT, "n_gpus": world, "steps": args.steps,
         "warmup": args.warmup, "ms_per_step": round(ms_per_step, 4), "higher_is_better": True,
-        "scaling": "weak", "vs_baseline": None, "dtype": "u32 keys / f32 update arithmetic", "data": "synthetic",
+        "scaling": "strong" if sharded else "weak", "vs_baseline": None, "dtype": "u32 keys / f32 update arithmetic", "data": "synthetic",
         "config": {"workload": wl.name, "tensors": len(wl.tensor_sizes), "params": P, "workers": W,
                    "keep_fractions": [pt["keep"] for pt in pts], "step": "select + apply for every keep fraction",
                    "l2": "inputs larger than L2 (%.1f GB of gradients per keep fraction)" % (W * 4.0 * P / 1e9),
-                   "apply_mode": args.apply_mode, "multi_gpu": "independent replicas, one per rank"},
+                   "apply_mode": args.apply_mode,
+                   "multi_gpu": ("one server sharded by parameter range over the ranks: each rank selects for W / N workers, the updates' "
+                                 "slices are exchanged (send / recv), every rank applies its range") if sharded
+                   else "independent replicas, one per rank (no data-path collective)"},
         "gpu_launches": int(launches),
         "clocks": clocks,
         "points": pts,
         # dominant kernel: the single streaming pass over the dense gradients.  Algorithmic bytes per
         # launch = workers x 4 bytes x parameters; duration = mean over its launches in the timed
         # region, from CUDA events recorded on the launching stream around the kernel.
-        "roofline": {"bound": "hbm", "kernel": "k_bracket_scan (k_bracket_scan_dense where 3 % of the entries or more are candidates)", "launches_timed": int(scan_launches),
+        "roofline": {"bound": "hbm", "kernel": "k_bracket_scan (the one pass over the dense gradients)", "launches_timed": int(scan_launches),
                      "achieved": round(scan_bytes_all / scan_ms_all / 1e6, 1) if scan_ms_all else None,
                      "peak": peak, "peak_kind": "of " + peak_kind, "unit": "GB/s",
                      "frac": round(scan_bytes_all / scan_ms_all / 1e6 / peak, 4) if scan_ms_all else None,
                      "traffic": (lambda t: round(t / 1e9, 3) if t else None)(scan_traffic_bytes(args.workload, keeps, W)),
-                     "traffic_unit": "GB per launch (ncu dram read + write, mean over the keep fractions; algorithmic: %.1f GB)" % (W * 4.0 * P / 1e9),
+                     "traffic_unit": "GB per launch (ncu dram read + write of a 4-worker capture x W / 4, mean over the keep fractions; algorithmic: %.1f GB)" % (W_sel * 4.0 * P / 1e9),
+                     # the apply kernels, per keep fraction: the dominant kernel of the launch against the same peak
+                     "apply": {"what": "one adacomp_apply launch of W updates per keep fraction; alg = 28 B per pair; sweep formulation = "
+                                       "16 B per parameter + 12 B per pair (what a launch that sweeps Theta and heads once must move)",
+                               "points": apply_points},
                      "select_call": {"what": "all kernels of adacomp_select, read 4P + write 8K per worker",
                                      "achieved": round(sel_bytes_all / sel_ms_all / 1e6, 1),
                                      "frac": round(sel_bytes_all / sel_ms_all / 1e6 / peak, 4)}},
     }
     if world == 1 and not args.no_competitors:
         out["encoding"] = run_encoding(binding, points, W, peak)
-    if world == 1 and not args.no_competitors and args.keep is None:
+    if world == 1 and not args.no_competitors and args.keep is None and not sharded:
         out["competitors"] = run_competitors(binding, wl, grads, dev, peak)
-    if world == 1 and not args.no_e2e:
+        out["apply_variants"] = run_apply_variants(binding, wl, dev, peak)
+    if world == 1 and not args.no_e2e and not sharded:
         out["e2e"] = run_e2e(args, binding, wl, points, srv, grads, rng, last_push, dev, stream)
     if world == 1 and rank == 0 and not args.no_cpu_baseline:
         out["cpu_baseline"] = cpu_baseline(wl, keeps, grads)
     if rank == 0:
         print(json.dumps(out))
-    if world > 1:
+    if world > 1 or sharded:
         import torch.distributed as dist
         dist.destroy_process_group()
 
