@@ -22,6 +22,10 @@
 
 using namespace adacomp;
 
+#ifndef ADACOMP_THIN_PAIRS
+#define ADACOMP_THIN_PAIRS 5.0      // updates that bring at most this many pairs per 256 parameters count as thin (build-time tunable)
+#endif
+
 namespace {
 
 constexpr uint32_t kNone = 0xFFFFFFFFu;
@@ -1168,7 +1172,7 @@ static int apply_body(adacomp_server_t* s, const uint32_t* d_idx, const float* d
         const bool sweep = theta_aligned &&
                            (s->mode == 3 || (s->mode == 0 && static_cast<double>(pairs) >= 0.08 * static_cast<double>(s->n_params)));
         int rc;
-        if (sweep && dens * 256.0 <= 5.0) {
+        if (sweep && dens * 256.0 <= ADACOMP_THIN_PAIRS) {
             // thin updates (a handful of pairs per update and range): all updates' pairs of a range lined up and
             // applied 32 at a time against the range's slices in shared memory
             if (dens * 512.0 <= 4.0) rc = launch_apply_merged<512>(s, sp, d, pairs, d_idx, d_val, lr, d_sigma_out, st);
