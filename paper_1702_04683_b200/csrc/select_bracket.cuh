@@ -61,16 +61,6 @@ __device__ __forceinline__ uint32_t hash32(uint32_t x) {
     return x;
 }
 
-// hist[bin] += 1 for every lane with `on`, one shared-memory atomic per distinct bin of the warp: lanes
-// that hold the same bin are found with a match and the lowest of them adds their number.  Magnitudes
-// of real gradients crowd into a handful of exponent values, so without this the lanes of a warp
-// would queue up on the same few counters.  All 32 lanes must call.
-__device__ __forceinline__ void hist_add_aggregated(uint32_t* hist, uint32_t bin, bool on) {
-    const uint32_t peers = __match_any_sync(0xFFFFFFFFu, on ? bin : 0xFFFFFFFFu);
-    const uint32_t lane = threadIdx.x & 31;
-    if (on && (peers & ((1u << lane) - 1u)) == 0) atomicAdd(&hist[bin], __popc(peers));
-}
-
 // Descending walk over a 2048-bin histogram in shared memory: the bucket holding the rem-th
 // largest.  All kBig threads call; results are returned to all.
 __device__ __forceinline__ void block_pick_bucket(const uint32_t* hist, uint32_t rem, uint32_t* bucket,
@@ -842,8 +832,7 @@ __global__ void __launch_bounds__(kBig) k_fallback_solo(SelectParams p) {
                         const bool on = e >= mis && e < n_shift &&
                                         (pass == 0 || (key >> (shift + 10)) == (prefix >> (shift + 10)));
                         const uint32_t bin = (key >> shift) & (nb - 1u);
-                        if (pass == 0) hist_add_aggregated(s_hist, bin, on);      // every entry counts: crowded bins
-                        else if (on) atomicAdd(&s_hist[bin], 1u);                 // few entries match the prefix
+                        if (on) atomicAdd(&s_hist[bin], 1u);
                     }
                 }
                 __syncthreads();
