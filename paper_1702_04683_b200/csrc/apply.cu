@@ -37,6 +37,7 @@ struct ServerParams {
     uint32_t* head;
     uint32_t* prev;
     int* status;
+    const uint32_t* gate;    // see BatchDesc::gate_hi
     uint64_t n_params;
     uint32_t ring_mask;
     uint32_t ring_shift;     // (position base) mod ring size: slot = (pos32 + ring_shift) & ring_mask
@@ -97,7 +98,31 @@ struct BatchDesc {
     uint32_t win_bits[kMaxBatch];              // updates of this launch inside update b's window (bits below b)
     uint32_t pre_mask;                         // bit b: update b's window starts before the launch
     uint32_t n_updates;
+    uint32_t gate_lo, gate_hi;                 // gate_hi != 0: the launch does its work only if gate_lo <= *gate < gate_hi
 };
+
+// Two kernels may be enqueued for the same updates, of which a count taken on the device picks one.
+__device__ __forceinline__ bool gate_open(const ServerParams& sp, const BatchDesc& d) {
+    if (d.gate_hi == 0) return true;
+    const uint32_t v = *sp.gate;
+    return v >= d.gate_lo && v < d.gate_hi;
+}
+
+// How crowded the updates' index lists are where they crowd: 256 stretches of 32 consecutive pairs are looked at per
+// update (one block each), and the stretches that would put 16 pairs or more into 256 parameters are counted into
+// *gate.  Evenly spread thin updates have next to none of these; updates whose pairs sit in a small part of the
+// parameters have little else.
+constexpr uint32_t kProbeThreads = 256;
+__global__ void __launch_bounds__(kProbeThreads)
+k_apply_probe(const BatchDesc d, const uint32_t* __restrict__ idx, uint32_t* gate) {
+    const uint32_t n = d.n_pairs[blockIdx.x];
+    if (n < 64) return;
+    const uint32_t* list = idx + d.pair_begin[blockIdx.x];
+    const uint32_t e = static_cast<uint32_t>(static_cast<uint64_t>(n - 32) * threadIdx.x / kProbeThreads);
+    const uint32_t span = __ldg(list + e + 31) - __ldg(list + e);          // 31 gaps
+    const int crowded = __syncthreads_count(span < 31u * 256u / 16u);
+    if (threadIdx.x == 0 && crowded) atomicAdd(gate, static_cast<uint32_t>(crowded));
+}
 
 constexpr uint32_t kAlphaTable = 33;             // alpha / sigma kept ready for sigma < 33
 
@@ -181,6 +206,7 @@ k_apply_warps(const ServerParams sp, const BatchDesc d, const uint32_t* __restri
     extern __shared__ __align__(16) unsigned char s_wp[];
     static_assert(R % 64 == 0 && R >= 128, "16-byte pieces, whole warps");
     static_assert(NB <= kMaxBatch, "one mask bit per update");
+    if (!gate_open(sp, d)) return;
     float* s_alpha = reinterpret_cast<float*>(s_wp);                            // [64] alpha / sigma for the small counts
     const uint32_t B = d.n_updates;                                             // <= NB
     const uint32_t tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
@@ -376,6 +402,7 @@ k_apply_merged(const ServerParams sp, const BatchDesc d, uint32_t range, const u
     extern __shared__ __align__(16) unsigned char s_mg[];
     static_assert(R % 128 == 0, "16-byte pieces, whole warps");
     constexpr bool kSlices = R != 0;                            // Theta, heads and masks of the range in shared memory
+    if (!gate_open(sp, d)) return;
     if constexpr (kSlices) range = R;
     const uint32_t B = d.n_updates;
     const uint32_t lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
@@ -798,7 +825,7 @@ size_t carve_server(adacomp_server_t* s, void* base, uint64_t n_params, uint64_t
     s->d_head = c.take<uint32_t>(n_params);
     s->d_prev = c.take<uint32_t>(ring);
     s->d_changed = c.take<uint8_t>(ring);
-    s->d_status = c.take<int>(1);
+    s->d_status = c.take<int>(2);        // [0] the error word, [1] the count that picks between two enqueued kernels
     return c.used;
 }
 
@@ -1003,6 +1030,7 @@ static int apply_body(adacomp_server_t* s, const uint32_t* d_idx, const float* d
         sp.ring_mask = sp.ring_shift = 0;
         sp.max_window = s->max_window;
         sp.validate = s->validate;
+        sp.gate = nullptr;
         for (uint32_t b = 0; b < n_updates; ++b) {
             UpdateDesc u;
             u.pair_begin = h_pair_begin[b];
@@ -1084,6 +1112,7 @@ static int apply_body(adacomp_server_t* s, const uint32_t* d_idx, const float* d
         sp.ring_shift = 0;
         sp.max_window = s->max_window;
         sp.validate = s->validate;
+        sp.gate = nullptr;
         const uint64_t mask = s->ring - 1;
         for (uint32_t b = 0; b < n_updates; ++b) {
             const uint64_t i = i0 + b, j = h_pull_ts[b];
@@ -1136,6 +1165,7 @@ static int apply_body(adacomp_server_t* s, const uint32_t* d_idx, const float* d
     sp.ring_shift = static_cast<uint32_t>(s->pos_base & (s->ring - 1));
     sp.max_window = s->max_window;
     sp.validate = s->validate;
+    sp.gate = reinterpret_cast<const uint32_t*>(s->d_status + 1);
 
     // ---- launches.  One launch per update, or launches of up to kMaxBatch updates each: same results.
     // Automatic choice per launch: a dense sweep of Theta through shared memory when the launch's pairs number
@@ -1149,6 +1179,7 @@ static int apply_body(adacomp_server_t* s, const uint32_t* d_idx, const float* d
         BatchDesc d;
         d.n_updates = launch_first[g + 1] - b0;
         d.pre_mask = 0;
+        d.gate_lo = d.gate_hi = 0;
         uint64_t pairs = 0;
         uint32_t most = 0;
         const uint64_t ts0 = i0 + b0;
@@ -1175,6 +1206,23 @@ static int apply_body(adacomp_server_t* s, const uint32_t* d_idx, const float* d
         if (sweep && dens * 256.0 <= ADACOMP_THIN_PAIRS) {
             // thin updates (a handful of pairs per update and range): all updates' pairs of a range lined up and
             // applied 32 at a time against the range's slices in shared memory
+            // ... unless the pairs crowd into a small part of the parameters, where the ranges they fall into are
+            // as busy as a dense update's: a count taken on the device picks between the two kernels, both enqueued
+            uint32_t probed = 0;
+            for (uint32_t b = 0; b < d.n_updates; ++b) probed += d.n_pairs[b] >= 64 ? kProbeThreads : 0;
+            const uint32_t crowded_from = probed / 4;
+            if (crowded_from) {
+                uint32_t* gate = reinterpret_cast<uint32_t*>(s->d_status + 1);
+                ADACOMP_CUDA(cudaMemsetAsync(gate, 0, sizeof(uint32_t), st));
+                k_apply_probe<<<d.n_updates, kProbeThreads, 0, st>>>(d, d_idx, gate);
+                ADACOMP_LAUNCH_CHECK();
+                d.gate_lo = crowded_from;
+                d.gate_hi = 0xFFFFFFFFu;
+                rc = launch_apply_warps<128>(s, sp, d, d_idx, d_val, lr, d_sigma_out, st);
+                if (rc != ADACOMP_OK) return rc;
+                d.gate_lo = 0;
+                d.gate_hi = crowded_from;
+            }
             if (dens * 512.0 <= 4.0) rc = launch_apply_merged<512>(s, sp, d, pairs, d_idx, d_val, lr, d_sigma_out, st);
             else rc = launch_apply_merged<256>(s, sp, d, pairs, d_idx, d_val, lr, d_sigma_out, st);
         } else if (sweep) {

@@ -223,6 +223,39 @@ def test_clustered_and_uneven_updates(binding, mode):
     assert np.array_equal(bits(theta), bits(ref.theta()))
 
 
+@pytest.mark.parametrize("mode", [0, 3])
+@pytest.mark.parametrize("crowded", [12, 3, 0])
+def test_thin_updates_that_crowd_into_a_small_stretch(binding, mode, crowded):
+    """Updates thin by their pair counts (1 % of the parameters each) of which `crowded` draw their pairs from
+    one twentieth of the parameter vector and the rest from all of it: all, a few and none of them crowded,
+    which is what decides the kernel on the device."""
+    P, n_up, per = 2_000_000, 12, 20_000
+    rng = np.random.default_rng(400 + crowded)
+    theta = torch.from_numpy(rng.standard_normal(P).astype(np.float32)).to(DEV)
+    ref = oracle.Server(theta.cpu().numpy())
+    srv = binding.Server(theta, history_pairs=4 * n_up * per, max_window_updates=3 * n_up)
+    srv.set_mode(mode)
+    ts = 0
+    for call in range(3):
+        lo = int(rng.integers(0, P - P // 20))
+        ups = [np.sort(rng.choice(np.arange(lo, lo + P // 20) if b < crowded else P, per, replace=False)).astype(np.uint32)
+               for b in range(n_up)]
+        vals = [rng.standard_normal(per).astype(np.float32) for _ in ups]
+        begin = (np.arange(n_up) * per).astype(np.uint64)
+        count = np.full(n_up, per, np.uint32)
+        pull = np.array([max(0, ts + b - int(rng.integers(0, 2 * n_up))) for b in range(n_up)], np.uint64)
+        idx, val = i32(np.concatenate(ups)), torch.from_numpy(np.concatenate(vals)).to(DEV)
+        sigma = torch.full_like(idx, -1)
+        srv.apply(idx, val, begin, count, pull, 0.05, sigma_out=sigma)
+        s = u32(sigma)
+        for b in range(n_up):
+            want = ref.apply(ups[b], vals[b], int(pull[b]), 0.05)
+            assert np.array_equal(s[b * per:(b + 1) * per], want), f"call {call} update {b}"
+        ts += n_up
+    assert srv.last_error() == 0 and srv.timestamp == ts == ref.timestamp
+    assert np.array_equal(bits(theta), bits(ref.theta()))
+
+
 @pytest.mark.parametrize("mode", MODES)
 def test_parameters_on_an_odd_address_and_odd_count(binding, mode):
     """Theta as a view that starts 4 bytes past a 16-byte boundary, with a parameter count that is
