@@ -9,44 +9,53 @@
 //            little-endian bit string held in 32-bit words (none if w = 0).
 // block_off[b] is the word at which block b starts inside the worker's stream, block_off[n_blocks]
 // the stream's length.  Three kernels encode (measure every block, prefix-sum the sizes, pack), one
-// decodes; a block is one CUDA block of 256 threads, one entry per thread.
+// decodes; a block of the format is one warp's work, eight entries per lane.
 #include "common.cuh"
 
 using namespace adacomp;
 
 namespace {
 
-constexpr int kCodeBlock = 256;
+constexpr int kCodeBlock = 256;                 // entries per block of the format
+constexpr int kRows = kCodeBlock / 32;          // a warp holds a block as 8 rows of 32 entries, entry e = row * 32 + lane
+constexpr int kCodeWarps = 8;                   // blocks of the format per CUDA block, one warp each
+constexpr int kCodeThreads = kCodeWarps * 32;
 
-__device__ __forceinline__ uint32_t block_max_256(uint32_t v, uint32_t* s_red) {
-    v = __reduce_max_sync(0xFFFFFFFFu, v);
-    if ((threadIdx.x & 31) == 0) s_red[threadIdx.x >> 5] = v;
-    __syncthreads();
-    uint32_t m = s_red[0];
+// Block `b` of worker `w`, held by one warp: v[r] = entry r * 32 + lane (0 past the end), gap[r] its gap (0 for the
+// block's first entry and past the end).  Returns the block's width.  Every load is one coalesced row.
+__device__ __forceinline__ uint32_t load_block_gaps(const uint32_t* __restrict__ list, uint64_t first, uint32_t n,
+                                                    uint32_t lane, uint32_t (&v)[kRows], uint32_t (&gap)[kRows]) {
 #pragma unroll
-    for (int i = 1; i < kCodeBlock / 32; ++i) m = max(m, s_red[i]);
-    __syncthreads();
-    return m;
+    for (int r = 0; r < kRows; ++r) {
+        const uint32_t e = r * 32 + lane;
+        v[r] = e < n ? __ldg(list + first + e) : 0u;
+    }
+    uint32_t widest = 0;
+#pragma unroll
+    for (int r = 0; r < kRows; ++r) {
+        uint32_t before = __shfl_up_sync(0xFFFFFFFFu, v[r], 1);
+        if (r > 0) {
+            const uint32_t last_row = __shfl_sync(0xFFFFFFFFu, v[r - 1], 31);
+            if (lane == 0) before = last_row;
+        }
+        const uint32_t e = r * 32 + lane;
+        gap[r] = (e >= 1 && e < n) ? v[r] - before - 1u : 0u;
+        widest = max(widest, gap[r]);
+    }
+    widest = __reduce_max_sync(0xFFFFFFFFu, widest);
+    return widest ? 32u - static_cast<uint32_t>(__clz(widest)) : 0u;
 }
 
-// the gap of entry t of the block (0 for the block's first entry and past the end) and the block's width
-__device__ __forceinline__ uint32_t gap_and_width(const uint32_t* idx, uint64_t first, uint32_t n, uint32_t* s_red, uint32_t* width) {
-    const uint32_t t = threadIdx.x;
-    uint32_t gap = 0;
-    if (t >= 1 && t < n) gap = idx[first + t] - idx[first + t - 1] - 1u;
-    const uint32_t widest = block_max_256(gap, s_red);
-    *width = widest ? 32u - static_cast<uint32_t>(__clz(widest)) : 0u;
-    return gap;
-}
-
-__global__ void __launch_bounds__(kCodeBlock)
+__global__ void __launch_bounds__(kCodeThreads)
 k_encode_measure(const uint32_t* __restrict__ idx, uint64_t K, uint64_t n_blocks, uint64_t* __restrict__ block_off) {
-    __shared__ uint32_t s_red[kCodeBlock / 32];
-    const uint64_t b = blockIdx.x, w = blockIdx.y, first = b * kCodeBlock;
+    const uint32_t lane = threadIdx.x & 31;
+    const uint64_t b = static_cast<uint64_t>(blockIdx.x) * kCodeWarps + (threadIdx.x >> 5), w = blockIdx.y;
+    if (b >= n_blocks) return;
+    const uint64_t first = b * kCodeBlock;
     const uint32_t n = static_cast<uint32_t>(K - first < kCodeBlock ? K - first : kCodeBlock);
-    uint32_t width;
-    gap_and_width(idx + w * K, first, n, s_red, &width);
-    if (threadIdx.x == 0) {
+    uint32_t v[kRows], gap[kRows];
+    const uint32_t width = load_block_gaps(idx + w * K, first, n, lane, v, gap);
+    if (lane == 0) {
         block_off[w * (n_blocks + 1) + b + 1] = 2 + (static_cast<uint64_t>(n - 1) * width + 31) / 32;   // size, summed up next
         if (b == 0) block_off[w * (n_blocks + 1)] = 0;
     }
@@ -88,75 +97,96 @@ __global__ void __launch_bounds__(1024) k_encode_offsets(uint64_t* __restrict__ 
     }
 }
 
-__global__ void __launch_bounds__(kCodeBlock)
+__global__ void __launch_bounds__(kCodeThreads)
 k_encode_pack(const uint32_t* __restrict__ idx, uint64_t K, uint64_t n_blocks, const uint64_t* __restrict__ block_off,
               uint32_t* __restrict__ words, uint64_t words_per_worker) {
-    __shared__ uint32_t s_red[kCodeBlock / 32];
-    __shared__ uint32_t s_bits[kCodeBlock];
-    const uint64_t b = blockIdx.x, w = blockIdx.y, first = b * kCodeBlock;
+    __shared__ uint32_t s_bits[kCodeWarps][kCodeBlock];          // the payload of each warp's block
+    const uint32_t lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const uint64_t b = static_cast<uint64_t>(blockIdx.x) * kCodeWarps + warp, w = blockIdx.y;
+    if (b >= n_blocks) return;
+    const uint64_t first = b * kCodeBlock;
     const uint32_t n = static_cast<uint32_t>(K - first < kCodeBlock ? K - first : kCodeBlock);
-    const uint32_t t = threadIdx.x;
-    s_bits[t] = 0;
-    uint32_t width;
-    const uint32_t gap = gap_and_width(idx + w * K, first, n, s_red, &width);     // (its barriers also publish s_bits = 0)
+    uint32_t v[kRows], gap[kRows];
+    const uint32_t width = load_block_gaps(idx + w * K, first, n, lane, v, gap);
     uint32_t* out = words + w * words_per_worker + block_off[w * (n_blocks + 1) + b];
-    if (t == 0) {
-        out[0] = idx[w * K + first];
+    if (lane == 0) {
+        out[0] = v[0];
         out[1] = width;
     }
-    if (t >= 1 && t < n && width) {
-        const uint32_t pos = (t - 1) * width, word = pos >> 5, shift = pos & 31;
-        const unsigned long long spread = static_cast<unsigned long long>(gap) << shift;
-        atomicOr(&s_bits[word], static_cast<uint32_t>(spread));
-        if (shift + width > 32) atomicOr(&s_bits[word + 1], static_cast<uint32_t>(spread >> 32));
-    }
-    __syncthreads();
     const uint32_t payload = ((n - 1) * width + 31) / 32;
-    if (t < payload) out[2 + t] = s_bits[t];
+    if (!payload) return;
+    uint32_t* bits = s_bits[warp];
+#pragma unroll
+    for (int r = 0; r < kRows; ++r) bits[r * 32 + lane] = 0;
+    __syncwarp();
+#pragma unroll
+    for (int r = 0; r < kRows; ++r) {
+        const uint32_t e = r * 32 + lane;
+        if (e >= 1 && e < n) {
+            const uint32_t pos = (e - 1) * width, word = pos >> 5, shift = pos & 31;
+            const unsigned long long spread = static_cast<unsigned long long>(gap[r]) << shift;
+            atomicOr(&bits[word], static_cast<uint32_t>(spread));
+            if (shift + width > 32) atomicOr(&bits[word + 1], static_cast<uint32_t>(spread >> 32));
+        }
+    }
+    __syncwarp();
+    for (uint32_t t = lane; t < payload; t += 32) out[2 + t] = bits[t];
 }
 
-__global__ void __launch_bounds__(kCodeBlock)
+__global__ void __launch_bounds__(kCodeThreads)
 k_decode(const uint32_t* __restrict__ words, uint64_t words_per_worker, const uint64_t* __restrict__ block_off,
          uint64_t K, uint64_t n_blocks, uint32_t* __restrict__ idx_out) {
-    __shared__ uint32_t s_warp[kCodeBlock / 32];
-    const uint64_t b = blockIdx.x, w = blockIdx.y, first = b * kCodeBlock;
+    const uint32_t lane = threadIdx.x & 31;
+    const uint64_t b = static_cast<uint64_t>(blockIdx.x) * kCodeWarps + (threadIdx.x >> 5), w = blockIdx.y;
+    if (b >= n_blocks) return;
+    const uint64_t first = b * kCodeBlock;
     const uint32_t n = static_cast<uint32_t>(K - first < kCodeBlock ? K - first : kCodeBlock);
-    const uint32_t t = threadIdx.x, lane = t & 31, warp = t >> 5;
+    uint32_t* out = idx_out + w * K + first;
     // the stream is untrusted (it arrives from a worker): the block must lie inside the worker's words with a
     // width of at most 32 bits, else the block decodes to 0xFFFFFFFF everywhere, an index no server accepts
     // (adacomp_apply skips and reports it), and nothing outside the stream is read
     const uint64_t off = block_off[w * (n_blocks + 1) + b];
     bool sound = off + 2 <= words_per_worker;
     const uint32_t* in = words + w * words_per_worker + (sound ? off : 0);
-    uint32_t width = sound ? in[1] : 0u;
+    const uint32_t width = sound ? __ldg(in + 1) : 0u;
     sound = sound && width <= 32 && off + 2 + (static_cast<uint64_t>(n - 1) * width + 31) / 32 <= words_per_worker;
     if (!sound) {
-        if (t < n) idx_out[w * K + first + t] = 0xFFFFFFFFu;
+#pragma unroll
+        for (int r = 0; r < kRows; ++r)
+            if (r * 32 + lane < n) out[r * 32 + lane] = 0xFFFFFFFFu;
         return;
     }
-    uint32_t step = 0;                                   // what entry t adds to its predecessor
-    if (t == 0) step = in[0];
-    else if (t < n) {
-        uint32_t gap = 0;
-        if (width) {
-            const uint32_t pos = (t - 1) * width, word = pos >> 5, shift = pos & 31;
-            unsigned long long window = in[2 + word];
-            if (shift + width > 32) window |= static_cast<unsigned long long>(in[2 + word + 1]) << 32;
-            gap = static_cast<uint32_t>(window >> shift) & (width == 32 ? 0xFFFFFFFFu : ((1u << width) - 1u));
-        }
-        step = gap + 1u;
-    }
-    uint32_t v = step;                                   // running sum modulo 2^32: the index
+    const uint32_t keep = width == 32 ? 0xFFFFFFFFu : ((1u << width) - 1u);
+    uint32_t step[kRows];                                // what an entry adds to its predecessor
 #pragma unroll
-    for (int d = 1; d < 32; d <<= 1) {
-        const uint32_t y = __shfl_up_sync(0xFFFFFFFFu, v, d);
-        if (lane >= static_cast<uint32_t>(d)) v += y;
+    for (int r = 0; r < kRows; ++r) {
+        const uint32_t e = r * 32 + lane;
+        step[r] = 0;
+        if (e == 0) step[r] = __ldg(in);
+        else if (e < n) {
+            uint32_t gap = 0;
+            if (width) {
+                const uint32_t pos = (e - 1) * width, word = pos >> 5, shift = pos & 31;
+                unsigned long long window = __ldg(in + 2 + word);
+                if (shift + width > 32) window |= static_cast<unsigned long long>(__ldg(in + 2 + word + 1)) << 32;
+                gap = static_cast<uint32_t>(window >> shift) & keep;
+            }
+            step[r] = gap + 1u;
+        }
     }
-    if (lane == 31) s_warp[warp] = v;
-    __syncthreads();
-    uint32_t before = 0;
-    for (uint32_t i = 0; i < warp; ++i) before += s_warp[i];
-    if (t < n) idx_out[w * K + first + t] = before + v;
+    uint32_t carry = 0;                                  // running sum modulo 2^32: the index
+#pragma unroll
+    for (int r = 0; r < kRows; ++r) {
+        uint32_t v = step[r];
+#pragma unroll
+        for (int d = 1; d < 32; d <<= 1) {
+            const uint32_t y = __shfl_up_sync(0xFFFFFFFFu, v, d);
+            if (lane >= static_cast<uint32_t>(d)) v += y;
+        }
+        v += carry;
+        if (r * 32 + lane < n) out[r * 32 + lane] = v;
+        carry = __shfl_sync(0xFFFFFFFFu, v, 31);
+    }
 }
 
 }  // namespace
@@ -182,12 +212,12 @@ int adacomp_encode_indices(const uint32_t* d_idx, uint64_t pairs_per_worker, uin
         ADACOMP_CUDA(cudaMemsetAsync(d_block_off, 0, n_workers * sizeof(uint64_t), st));
         return ADACOMP_OK;
     }
-    const dim3 grid(static_cast<unsigned>(n_blocks), n_workers);
-    k_encode_measure<<<grid, kCodeBlock, 0, st>>>(d_idx, K, n_blocks, d_block_off);
+    const dim3 grid(static_cast<unsigned>((n_blocks + kCodeWarps - 1) / kCodeWarps), n_workers);
+    k_encode_measure<<<grid, kCodeThreads, 0, st>>>(d_idx, K, n_blocks, d_block_off);
     ADACOMP_LAUNCH_CHECK();
     k_encode_offsets<<<n_workers, 1024, 0, st>>>(d_block_off, n_blocks);
     ADACOMP_LAUNCH_CHECK();
-    k_encode_pack<<<grid, kCodeBlock, 0, st>>>(d_idx, K, n_blocks, d_block_off, d_words, words_per_worker);
+    k_encode_pack<<<grid, kCodeThreads, 0, st>>>(d_idx, K, n_blocks, d_block_off, d_words, words_per_worker);
     ADACOMP_LAUNCH_CHECK();
     return ADACOMP_OK;
 }
@@ -202,7 +232,8 @@ int adacomp_decode_indices(const uint32_t* d_words, uint64_t words_per_worker, c
     if (!d_words || !d_idx_out) return ADACOMP_ERR_INVALID;
     DeviceGuard guard(device);
     if (guard.err != cudaSuccess) return cuda_fail(guard.err);
-    k_decode<<<dim3(static_cast<unsigned>(n_blocks), n_workers), kCodeBlock, 0, static_cast<cudaStream_t>(cuda_stream)>>>(
+    k_decode<<<dim3(static_cast<unsigned>((n_blocks + kCodeWarps - 1) / kCodeWarps), n_workers), kCodeThreads, 0,
+               static_cast<cudaStream_t>(cuda_stream)>>>(
         d_words, words_per_worker, d_block_off, K, n_blocks, d_idx_out);
     ADACOMP_LAUNCH_CHECK();
     return ADACOMP_OK;
