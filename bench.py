@@ -33,13 +33,13 @@ METRIC = "dense-gradient GB/s scanned (select+compact, with the selected pairs a
 UNIT = "GB/s"
 FALLBACK_HBM_GBS = 6650.0
 
-# DRAM bytes (read + write) of ONE launch of the scan kernel and of the dominant apply kernel, from an ncu capture of
-# workload 4 with 4 workers / 4 updates, MB per keep fraction.  A launch over W workers moves W / 4 times as much
-# (every worker's tensors are independent; for the apply kernels the sweep of Theta and heads does not grow with W, so
-# only the scan figure is scaled and the apply figure is reported as captured).  Only valid while the kernel sources are
-# the ones that were profiled (guarded by their hashes).
+# DRAM bytes (read + write) of ONE launch of the scan kernel and of the apply kernel that does the work, from ncu
+# captures of workload 4, MB per keep fraction.  The scan kernel was captured with 4 of the 16 workers: a launch over W
+# workers moves W / 4 times as much (every worker's tensors are independent).  The apply kernel was captured with all 16
+# updates in the launch on tensors four times smaller: parameters and pairs, hence the traffic, are a quarter of a
+# full-size launch's.  Only valid while the kernel sources are the ones that were profiled (guarded by their hashes).
 SCAN_TRAFFIC_W4_MB = {}
-APPLY_TRAFFIC_W4_MB = {}
+APPLY_TRAFFIC_DIV4_MB = {}
 SCAN_SOURCE_SHA256_16 = ""
 APPLY_SOURCE_SHA256_16 = ""
 
@@ -65,10 +65,12 @@ def scan_traffic_bytes(workload_index, keeps, workers):
 
 
 def apply_traffic_mb(workload_index, keep):
-    """DRAM MB of the apply launch captured with 4 updates at this keep fraction, or None if unknown."""
+    """DRAM MB of a full-size apply launch at this keep fraction: 4 x the ncu capture of the 16-update launch on tensors
+    four times smaller (--divide 4; parameters and pairs, hence the traffic, scale together), or None if unknown."""
     if not APPLY_SOURCE_SHA256_16 or _source_hash("apply.cu") != APPLY_SOURCE_SHA256_16 or workload_index != 4:
         return None
-    return APPLY_TRAFFIC_W4_MB.get("%d/%d" % keep)
+    mb = APPLY_TRAFFIC_DIV4_MB.get("%d/%d" % keep)
+    return None if mb is None else round(4.0 * mb, 1)
 
 
 def run_apply_variants(binding, wl, dev, peak, keep=(1, 100), reps=5, warmup=3):
@@ -249,6 +251,9 @@ def parse_args():
     ap.add_argument("--workload", type=int, default=4)
     ap.add_argument("--keep", default=None, help="one keep fraction a/b instead of the workload's list")
     ap.add_argument("--workers", type=int, default=None, help="override the number of workers (smaller captures)")
+    ap.add_argument("--divide", type=int, default=None,
+                    help="every tensor this many times smaller, the number of workers kept (smaller captures of the "
+                         "kernels that take all workers' updates in one launch)")
     ap.add_argument("--e2e-steps", type=int, default=2)
     ap.add_argument("--apply-mode", type=int, default=0)
     ap.add_argument("--no-cpu-baseline", action="store_true")
@@ -385,6 +390,8 @@ def run_native(args):
     wl = wlmod.workload(args.workload, seed=0 if sharded else rank)
     if args.workers:
         wl = dataclasses.replace(wl, n_workers=args.workers)
+    if args.divide:
+        wl = wl.scaled(args.divide)
     keeps = [parse_keep(args.keep)] if args.keep else list(wl.keep_fractions)
     W, P = wl.n_workers, wl.n_params
     stream = torch.cuda.current_stream()
@@ -495,7 +502,7 @@ def run_native(args):
                              "alg_frac": round(pairs * 28.0 / app_ms / 1e6 / peak, 4),
                              "sweep_formulation_gbs": round(sweep_bytes / app_ms / 1e6, 1),
                              "sweep_formulation_frac": round(sweep_bytes / app_ms / 1e6 / peak, 4),
-                             "dram_mb_4_updates_ncu": cap_mb})
+                             "dram_mb_ncu_quarter_size_x4": cap_mb})
         pts.append({
             "keep": f"{p.keep[0]}/{p.keep[1]}", "pairs_per_update": p.K,
             "select_ms": round(sel_ms, 4), "apply_ms": round(app_ms, 4),

@@ -268,7 +268,7 @@ __global__ void __launch_bounds__(kBig) k_bracket_sample(SelectParams p, int gen
 // are in the list, how many, and how many of them lie above the window.  A NaN hands the instance to
 // the general route, which works on bit patterns only.
 constexpr uint32_t kDenseStage = 640;                          // candidates the stage holds; a piece that brings more is written directly
-constexpr uint32_t kDenseRing = 2;                             // piece buffers per warp
+constexpr uint32_t kDenseRing = 1;                             // piece buffers per warp
 constexpr uint32_t kPieceBytes = kSubElems * 4;
 constexpr size_t kDenseSmemPerWarp = kDenseRing * kPieceBytes + kDenseStage * 8 + 64 + 16;
 static_assert(kDenseSmemPerWarp % 16 == 0, "the warps' slices stay 16-byte aligned");
@@ -320,7 +320,7 @@ __device__ __forceinline__ void mask_or(const float4& x, float t, uint32_t& mask
         : "f"(x.x), "f"(x.y), "f"(x.z), "f"(x.w), "f"(t), "n"(kBit), "n"(kBit << 1), "n"(kBit << 2), "n"(kBit << 3));
 }
 
-__global__ void __launch_bounds__(kThreads, 2) k_bracket_scan(SelectParams p) {
+__global__ void __launch_bounds__(kThreads, 3) k_bracket_scan(SelectParams p) {
     extern __shared__ __align__(16) unsigned char s_scan[];
     const uint2 item = p.items[blockIdx.x];
     const uint32_t l = item.x, w = blockIdx.y;
@@ -365,6 +365,11 @@ __global__ void __launch_bounds__(kThreads, 2) k_bracket_scan(SelectParams p) {
         const uint32_t mbar = mbar_base + 8u * (j % kDenseRing);
         mbar_expect_tx(mbar, groups * 16u);
         bulk_load(ring_base + (j % kDenseRing) * kPieceBytes, vec + vec0, groups * 16u, mbar);
+        if (j + 1 < n_mine) {                                  // the piece after it: on its way to L2 meanwhile
+            const uint32_t v1 = (ss0 + kStep * (j + 1)) * (kSubElems / 4);
+            const uint32_t g1 = nvec - v1 < kSubElems / 4 ? nvec - v1 : kSubElems / 4;
+            asm volatile("cp.async.bulk.prefetch.L2.global [%0], %1;" ::"l"(vec + v1), "r"(g1 * 16u) : "memory");
+        }
     };
     if (lane == 0) {
 #pragma unroll
