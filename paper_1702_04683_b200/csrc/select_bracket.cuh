@@ -267,7 +267,7 @@ __global__ void __launch_bounds__(kBig) k_bracket_sample(SelectParams p, int gen
 // Candidates stay in index order inside a piece; the table records, per piece, where its candidates
 // are in the list, how many, and how many of them lie above the window.  A NaN hands the instance to
 // the general route, which works on bit patterns only.
-constexpr uint32_t kDenseStage = 640;                          // candidates the stage holds; a piece that brings more is written directly
+constexpr uint32_t kDenseStage = 352;                          // candidates the stage holds; a piece that brings more is written directly
 constexpr uint32_t kDenseRing = 1;                             // piece buffers per warp
 constexpr uint32_t kPieceBytes = kSubElems * 4;
 constexpr size_t kDenseSmemPerWarp = kDenseRing * kPieceBytes + kDenseStage * 8 + 64 + 16;
@@ -320,7 +320,7 @@ __device__ __forceinline__ void mask_or(const float4& x, float t, uint32_t& mask
         : "f"(x.x), "f"(x.y), "f"(x.z), "f"(x.w), "f"(t), "n"(kBit), "n"(kBit << 1), "n"(kBit << 2), "n"(kBit << 3));
 }
 
-__global__ void __launch_bounds__(kThreads, 3) k_bracket_scan(SelectParams p) {
+__global__ void __launch_bounds__(kThreads, 4) k_bracket_scan(SelectParams p) {
     extern __shared__ __align__(16) unsigned char s_scan[];
     const uint2 item = p.items[blockIdx.x];
     const uint32_t l = item.x, w = blockIdx.y;
