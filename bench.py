@@ -38,10 +38,10 @@ FALLBACK_HBM_GBS = 6650.0
 # workers moves W / 4 times as much (every worker's tensors are independent).  The apply kernel was captured with all 16
 # updates in the launch on tensors four times smaller: parameters and pairs, hence the traffic, are a quarter of a
 # full-size launch's.  Only valid while the kernel sources are the ones that were profiled (guarded by their hashes).
-SCAN_TRAFFIC_W4_MB = {}
-APPLY_TRAFFIC_DIV4_MB = {}
-SCAN_SOURCE_SHA256_16 = ""
-APPLY_SOURCE_SHA256_16 = ""
+SCAN_TRAFFIC_W4_MB = {'1/1000': 1617.7, '1/400': 1627.8, '1/160': 1648.6, '1/64': 1692.6, '1/25': 1789.1, '1/10': 2010.7}
+APPLY_TRAFFIC_DIV4_MB = {'1/1000': 91.3, '1/400': 190.1, '1/160': 321.8, '1/64': 463.4, '1/25': 583.9, '1/10': 925.6}
+SCAN_SOURCE_SHA256_16 = "5a3bbfbce034ab9e"
+APPLY_SOURCE_SHA256_16 = "0402d0792ba9bb99"
 
 
 def _source_hash(name):
@@ -497,11 +497,13 @@ def run_native(args):
         # pairs and writes their links (12 B per pair), against the 28 B per pair of the per-pair formulation
         sweep_bytes = 16.0 * (P / (world if sharded else 1)) + 12.0 * pairs
         cap_mb = apply_traffic_mb(args.workload, p.keep)
+        sweeps = args.apply_mode == 3 or (args.apply_mode == 0 and pairs >= 0.08 * (P / (world if sharded else 1)))
         apply_points.append({"keep": f"{p.keep[0]}/{p.keep[1]}", "apply_ms": round(app_ms, 4),
                              "alg_gbs_28B_per_pair": round(pairs * 28.0 / app_ms / 1e6, 1),
                              "alg_frac": round(pairs * 28.0 / app_ms / 1e6 / peak, 4),
-                             "sweep_formulation_gbs": round(sweep_bytes / app_ms / 1e6, 1),
-                             "sweep_formulation_frac": round(sweep_bytes / app_ms / 1e6 / peak, 4),
+                             # only where the launch does sweep (the library's rule: pairs >= 8 % of the parameters)
+                             "sweep_formulation_gbs": round(sweep_bytes / app_ms / 1e6, 1) if sweeps else None,
+                             "sweep_formulation_frac": round(sweep_bytes / app_ms / 1e6 / peak, 4) if sweeps else None,
                              "dram_mb_ncu_quarter_size_x4": cap_mb})
         pts.append({
             "keep": f"{p.keep[0]}/{p.keep[1]}", "pairs_per_update": p.K,
