@@ -40,7 +40,7 @@ FALLBACK_HBM_GBS = 6650.0
 # full-size launch's.  Only valid while the kernel sources are the ones that were profiled (guarded by their hashes).
 SCAN_TRAFFIC_W4_MB = {'1/1000': 1617.7, '1/400': 1627.8, '1/160': 1648.6, '1/64': 1692.6, '1/25': 1789.1, '1/10': 2010.7}
 APPLY_TRAFFIC_DIV4_MB = {'1/1000': 91.3, '1/400': 190.1, '1/160': 321.8, '1/64': 463.4, '1/25': 583.9, '1/10': 925.6}
-SCAN_SOURCE_SHA256_16 = "5a3bbfbce034ab9e"
+SCAN_SOURCE_SHA256_16 = "b3f19e7900b079fc"
 APPLY_SOURCE_SHA256_16 = "0402d0792ba9bb99"
 
 

@@ -19,7 +19,9 @@
 //   k_bracket_emit     per span (8 pieces), one warp: read its candidates, keep those at or above
 //                      the exact threshold, write them to the output in index order.
 // The result is exact whatever the sample looked like: if the exact counts contradict the
-// bracket, or a list overflows its capacity, the instance is handed to the general route.
+// bracket, a list overflows its capacity or a NaN is seen, the instance is flagged and redone
+// exactly: by k_fallback_solo (one block per flagged instance) when all tensors of the handle are on
+// this route or small enough to be selected whole in shared memory, else by the general route.
 // No kernel waits on another block; all cross-block traffic is atomics plus kernel boundaries.
 #pragma once
 
@@ -39,7 +41,8 @@ constexpr uint32_t kSmallMax = kBracketMinN - 1;         // longest tensor whose
 constexpr uint32_t kSampleMin = 2048;
 constexpr float kBracketZ = 5.0f;                     // half-width of the bracket in sample standard deviations
 constexpr uint32_t kGatherMax = 1024;
-constexpr int kBig = 1024;                            // threads of the per-instance kernels
+constexpr int kBig = 512;                             // threads of the per-instance kernels (measured: 1024 and 256 are slower
+                                                      // where a call has thousands of small tensors, equal elsewhere)
 
 constexpr uint32_t kRouteSmall = 3u;                  // Layer::bracket of a tensor that is selected whole in shared memory
 constexpr uint32_t kInstBracket = 2u;                 // bracket valid, scan/emit act on the instance
@@ -139,7 +142,8 @@ __global__ void __launch_bounds__(kBig) k_bracket_sample(SelectParams p, int gen
         // k-th largest key; with k = n every entry is kept (T = 0: all keys are above or equal)
         const uint32_t T = k < n ? smem_kth_largest(s_keys, n, k, s_hist, s_warp, s_bc) : 0u;
         const uint32_t lane = threadIdx.x & 31, warp = threadIdx.x >> 5, lt = (1u << lane) - 1u;
-        const uint32_t seg = (((n + 31) / 32) + 31) & ~31u;    // entries per warp, a multiple of 32
+        constexpr uint32_t kWarps = kBig / 32;
+        const uint32_t seg = (((n + kWarps - 1) / kWarps) + 31) & ~31u;    // entries per warp, a multiple of 32
         const uint32_t e0 = warp * seg < n ? warp * seg : n, e1 = e0 + seg < n ? e0 + seg : n;
         uint32_t gt = 0, eq = 0;
         for (uint32_t e = e0 + lane; e < e1; e += 32) {
@@ -155,7 +159,7 @@ __global__ void __launch_bounds__(kBig) k_bracket_sample(SelectParams p, int gen
         if (lane == 0) { s_hist[warp] = gt; s_hist[32 + warp] = eq; }
         __syncthreads();
         // every warp works out where all stretches begin: lane j stands for warp j's stretch
-        const uint32_t gt_j = s_hist[lane], eq_j = s_hist[32 + lane];
+        const uint32_t gt_j = lane < kWarps ? s_hist[lane] : 0u, eq_j = lane < kWarps ? s_hist[32 + lane] : 0u;
         uint32_t n_gt = gt_j, eq_inc = eq_j;
 #pragma unroll
         for (int d = 16; d; d >>= 1) n_gt += __shfl_xor_sync(0xFFFFFFFFu, n_gt, d);
@@ -242,10 +246,12 @@ __global__ void __launch_bounds__(kBig) k_bracket_sample(SelectParams p, int gen
 // ---------------------------------------------------------------------------------------------
 // The single pass over the gradient.  A work item is up to kSpansPerBlock consecutive spans of one
 // tensor = 64 pieces of 1024 entries, and each of the 8 warps of a block takes 8 of them (round robin),
-// entirely on its own: no block-level barrier.  The pieces do not travel through registers: each warp
-// keeps a ring of two 4 KB buffers in shared memory that bulk asynchronous copies (cp.async.bulk,
-// completion on an mbarrier of the warp's own) fill a piece ahead, so loading costs the warp one
-// instruction per piece.  Per piece:
+// entirely on its own: no block-level barrier.  The pieces do not travel through registers: a bulk
+// asynchronous copy (cp.async.bulk, completion on an mbarrier of the warp's own) brings a piece into the
+// warp's 4 KB buffer in shared memory while the piece after it is prefetched into L2, so loading costs the
+// warp two instructions per piece.  One buffer, not a ring: what the kernel needs to keep the memory
+// system and the issue slots busy is warps (7 KB of shared memory per warp leave room for four blocks,
+// 32 warps, per SM), and the other warps' work covers the wait for a copy that comes from L2.  Per piece:
 //   mask     lane L reads ITS 32 consecutive entries of the piece (eight 16-byte reads, the order of
 //            the eight rotated by the lane so that the banks are spread) and builds a 32-bit mask of
 //            its candidates (key >= t_lo; for non-NaN data |x| >= t as floats is the integer test on
@@ -259,7 +265,7 @@ __global__ void __launch_bounds__(kBig) k_bracket_sample(SelectParams p, int gen
 //            behind the candidates staged before: work in proportion to the candidates, not to
 //            the entries.
 // Flush, when the stage cannot take the piece just counted and after the last one, while the next
-// piece's copy is in flight: a first pass with one lane per staged candidate counts the window
+// piece is on its way to L2: a first pass with one lane per staged candidate counts the window
 // entries (those not above t_hi; also per piece, for the table) and looks for NaN; two atomics
 // reserve room in the candidate and the window list; a second pass writes both lists with
 // coalesced stores, window entries ranked by ballot.  A piece with more candidates than the stage
@@ -656,17 +662,16 @@ __global__ void __launch_bounds__(kBig) k_bracket_resolve(SelectParams p) {
                     else if (top > prefix) atomicAdd(&sel[idx / kSpanElems], 1u);   // above the undecided ones: kept
                 });
                 __syncthreads();
-                unsigned long long mine = 0;
-                if (threadIdx.x < count) {
-                    mine = s_g[threadIdx.x];
+                for (uint32_t t = threadIdx.x; t < count; t += kBig) {
+                    const unsigned long long mine = s_g[t];
                     uint32_t larger = 0;
                     for (uint32_t u = 0; u < count; ++u) larger += s_g[u] > mine ? 1u : 0u;
                     if (larger == rem - 1) s_cstar = mine;
                 }
                 __syncthreads();
                 cstar = s_cstar;
-                if (threadIdx.x < count && mine >= cstar)     // the kept ones among the collected entries
-                    atomicAdd(&sel[(0xFFFFFFFFu - static_cast<uint32_t>(mine)) / kSpanElems], 1u);
+                for (uint32_t t = threadIdx.x; t < count; t += kBig)      // the kept ones among the collected entries
+                    if (s_g[t] >= cstar) atomicAdd(&sel[(0xFFFFFFFFu - static_cast<uint32_t>(s_g[t])) / kSpanElems], 1u);
                 break;
             }
             if (hi_shift == 0) { failed = true; break; }      // cannot happen: composites are distinct

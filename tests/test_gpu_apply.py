@@ -510,6 +510,33 @@ def test_pull_returns_timestamp_and_copy(binding):
     assert int(s[0]) == 0 and fresh[2].item() == -1.0 and theta[2].item() == 1.0   # history was forgotten
 
 
+@pytest.mark.parametrize("n_workers,pad", [(5, 0), (11, 12), (16, 4)])
+def test_select_from_host_memory(binding, n_workers, pad):
+    """adacomp_select_host with several worker counts and a worker stride longer than the layout: the pairs that arrive in
+    host memory are the oracle's, and the device staging buffers hold the same."""
+    wl = wlmod.workload(0).scaled(16, n_workers=n_workers)
+    keep = (1, 100)
+    sel = binding.Selector(binding.make_segments(wl.tensor_sizes, keep), n_workers, DEV)
+    K, W, P = sel.pairs_per_worker, n_workers, wl.n_params
+    g = wlmod.round_gradients(wl, 0, "cpu")
+    h_g = torch.zeros((W, P + pad)).pin_memory()
+    h_g[:, :P] = g
+    d_g = torch.empty((W, P + pad), device=DEV)
+    d_idx = torch.empty((W, K), dtype=torch.int32, device=DEV)
+    d_val = torch.empty((W, K), device=DEV)
+    h_idx = torch.full((W, K), -1, dtype=torch.int32).pin_memory()
+    h_val = torch.zeros((W, K)).pin_memory()
+    for _ in range(2):
+        sel.select_host(h_g, d_g, d_idx, d_val, h_idx, h_val)
+    torch.cuda.current_stream().synchronize()
+    assert sel.last_error()[0] == 0
+    ks = oracle_keep_counts(wl.tensor_sizes, keep)
+    for w in range(W):
+        oi, ov = oracle.select_layers(g[w].numpy(), wl.offsets, wl.tensor_sizes, ks)
+        assert np.array_equal(h_idx[w].numpy().view(np.uint32), oi) and np.array_equal(bits(h_val[w]), bits(ov))
+    assert torch.equal(d_idx.cpu(), h_idx) and torch.equal(d_val.cpu().view(torch.int32), h_val.view(torch.int32))
+
+
 def test_host_entry_points(binding):
     wl = wlmod.workload(0).scaled(16)
     keep = (1, 100)
