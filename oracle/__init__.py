@@ -72,6 +72,10 @@ def lib():
             L.oracle_encode_indices.argtypes = [u32p, ctypes.c_uint64, u32p, u64p]
             L.oracle_decode_indices.restype = ctypes.c_int
             L.oracle_decode_indices.argtypes = [u32p, u64p, ctypes.c_uint64, u32p]
+            L.oracle_encode_values.restype = ctypes.c_uint64
+            L.oracle_encode_values.argtypes = [f32p, ctypes.c_uint64, u32p, u64p]
+            L.oracle_decode_values.restype = ctypes.c_int
+            L.oracle_decode_values.argtypes = [u32p, u64p, ctypes.c_uint64, f32p]
             L.oracle_parameter_trace.restype = ctypes.c_int
             L.oracle_parameter_trace.argtypes = [
                 ctypes.c_uint32, ctypes.c_float, u32p, f32p, u64p, u64p, ctypes.c_uint64, ctypes.c_uint64,
@@ -200,6 +204,26 @@ def decode_indices(words, block_off, n_pairs: int):
     block_off = np.ascontiguousarray(block_off, dtype=np.uint64)
     out = np.empty(n_pairs, dtype=np.uint32)
     if lib().oracle_decode_indices(_p(words, ctypes.c_uint32), _p(block_off, ctypes.c_uint64), n_pairs, _p(out, ctypes.c_uint32)) != 0:
+        raise ValueError("oracle decode: bad stream")
+    return out
+
+
+def encode_values(val):
+    """Lossless block-wise packing of fp32 values (sign, exponent relative to the block's smallest, mantissa)
+    -> (words uint32, block_off uint64[n_blocks + 1])."""
+    val = _f32(val)
+    n_blocks = (val.size + 255) // 256
+    words = np.empty(val.size + n_blocks, dtype=np.uint32)              # the most the format can take
+    off = np.empty(n_blocks + 1, dtype=np.uint64)
+    total = lib().oracle_encode_values(_p(val, ctypes.c_float), val.size, _p(words, ctypes.c_uint32), _p(off, ctypes.c_uint64))
+    return words[:int(total)].copy(), off
+
+
+def decode_values(words, block_off, n_pairs: int):
+    words = np.ascontiguousarray(words, dtype=np.uint32)
+    block_off = np.ascontiguousarray(block_off, dtype=np.uint64)
+    out = np.empty(n_pairs, dtype=np.float32)
+    if lib().oracle_decode_values(_p(words, ctypes.c_uint32), _p(block_off, ctypes.c_uint64), n_pairs, _p(out, ctypes.c_float)) != 0:
         raise ValueError("oracle decode: bad stream")
     return out
 

@@ -368,6 +368,74 @@ int oracle_decode_indices(const uint32_t* words, const uint64_t* block_off, uint
     return 0;
 }
 
+// --- value packing ----------------------------------------------------------------
+// The value half of the same open point (footnote of "Algorithm details"), lossless:
+// every fp32 bit pattern comes back as it went in, so Eq. 4 sees the same inputs.  The
+// values of an update are cut into blocks of 256 entries, as the indices are.  With
+// E(x) = the 8-bit exponent field of x (bits 30..23), a block is stored as
+//   word 0      e_min | w_e << 8: e_min the smallest E in the block, w_e the number of
+//               bits of the largest (E - e_min), 0..8,
+//   then        the n entries, 24 + w_e bits each, entry t at bit t * (24 + w_e) of a
+//               little-endian bit string held in 32-bit words; an entry is the 23 mantissa
+//               bits, above them (E - e_min) in w_e bits, above that the sign bit.
+// The largest magnitudes of a tensor lie within a few powers of two of each other, so
+// w_e is 2 or 3 and a value costs 26 or 27 bits instead of 32.
+uint64_t oracle_encode_values(const float* val, uint64_t n_pairs, uint32_t* words_out, uint64_t* block_off_out) {
+    uint64_t at = 0, n_blocks = (n_pairs + 255) / 256;
+    for (uint64_t b = 0; b < n_blocks; ++b) {
+        const uint64_t first = b * 256, n = std::min<uint64_t>(256, n_pairs - first);
+        block_off_out[b] = at;
+        uint32_t e_min = 255, e_max = 0;
+        for (uint64_t t = 0; t < n; ++t) {
+            uint32_t bits;
+            std::memcpy(&bits, &val[first + t], 4);
+            const uint32_t e = (bits >> 23) & 0xFFu;
+            e_min = std::min(e_min, e);
+            e_max = std::max(e_max, e);
+        }
+        const uint32_t w_e = bits_needed(e_max - e_min), width = 24 + w_e;
+        words_out[at++] = e_min | (w_e << 8);
+        const uint64_t payload = (n * width + 31) / 32;
+        for (uint64_t i = 0; i < payload; ++i) words_out[at + i] = 0;
+        for (uint64_t t = 0; t < n; ++t) {
+            uint32_t bits;
+            std::memcpy(&bits, &val[first + t], 4);
+            const uint64_t mantissa = bits & 0x7FFFFFu, e_rel = ((bits >> 23) & 0xFFu) - e_min, sign = bits >> 31;
+            const uint64_t entry = mantissa | (e_rel << 23) | (sign << (23 + w_e));
+            for (uint32_t bit = 0; bit < width; ++bit) {                          // bit by bit, as the format is defined
+                const uint64_t pos = t * width + bit;
+                if ((entry >> bit) & 1u) words_out[at + pos / 32] |= 1u << (pos % 32);
+            }
+        }
+        at += payload;
+    }
+    block_off_out[n_blocks] = at;
+    return at;
+}
+
+int oracle_decode_values(const uint32_t* words, const uint64_t* block_off, uint64_t n_pairs, float* val_out) {
+    const uint64_t n_blocks = (n_pairs + 255) / 256;
+    for (uint64_t b = 0; b < n_blocks; ++b) {
+        const uint64_t first = b * 256, n = std::min<uint64_t>(256, n_pairs - first), at = block_off[b];
+        const uint32_t e_min = words[at] & 0xFFu, w_e = (words[at] >> 8) & 0xFFu, width = 24 + w_e;
+        if (w_e > 8 || (words[at] >> 16) != 0) return -1;
+        for (uint64_t t = 0; t < n; ++t) {
+            uint64_t entry = 0;
+            for (uint32_t bit = 0; bit < width; ++bit) {
+                const uint64_t pos = t * width + bit;
+                entry |= static_cast<uint64_t>((words[at + 1 + pos / 32] >> (pos % 32)) & 1u) << bit;
+            }
+            const uint32_t mantissa = static_cast<uint32_t>(entry & 0x7FFFFFu);
+            const uint32_t e = e_min + static_cast<uint32_t>((entry >> 23) & ((1u << w_e) - 1u));
+            const uint32_t sign = static_cast<uint32_t>((entry >> (23 + w_e)) & 1u);
+            if (e > 255) return -1;
+            const uint32_t bits = mantissa | (e << 23) | (sign << 31);
+            std::memcpy(&val_out[first + t], &bits, 4);
+        }
+    }
+    return 0;
+}
+
 // --- one parameter at a time --------------------------------------------------
 // The history of a single parameter k through a whole sequence of updates,
 // computed the way the paper's complexity paragraph describes it: each update
