@@ -235,10 +235,27 @@ def run_encoding(binding, points, W, peak, reps=5, warmup=3):
         if not torch.equal(back, p.idx):
             raise SystemExit("index coding: the round trip changed an index")
         coded_words = float(off[:, -1].sum().item())
-        out.append({"keep": f"{p.keep[0]}/{p.keep[1]}", "bytes_per_pair": round(4.0 + 4.0 * coded_words / (W * p.K), 3),
-                    "plain_bytes_per_pair": 8.0, "encode_ms": round(enc_ms, 4), "decode_ms": round(dec_ms, 4),
-                    "encode_pairs_per_s": round(W * p.K / enc_ms * 1e3, 1), "decode_pairs_per_s": round(W * p.K / dec_ms * 1e3, 1)})
         del words, off, back
+        # the values, packed losslessly
+        vwords, voff = binding.adacomp_encode_values(p.val)
+        vcap = vwords.shape[1]
+        vback = torch.empty_like(p.val)
+        venc_ms = timed(lambda: binding._check(raw.adacomp_encode_values(p.val.data_ptr(), p.K, W, vwords.data_ptr(), vcap, voff.data_ptr(),
+                                                                         dev_index, int(stream.cuda_stream)), "encode values"))
+        vdec_ms = timed(lambda: binding._check(raw.adacomp_decode_values(vwords.data_ptr(), vcap, voff.data_ptr(), p.K, W, vback.data_ptr(),
+                                                                         dev_index, int(stream.cuda_stream)), "decode values"))
+        if not torch.equal(vback.view(torch.int32), p.val.view(torch.int32)):
+            raise SystemExit("value packing: the round trip changed a value")
+        value_words = float(voff[:, -1].sum().item())
+        idx_bytes, val_bytes = 4.0 * coded_words / (W * p.K), 4.0 * value_words / (W * p.K)
+        out.append({"keep": f"{p.keep[0]}/{p.keep[1]}", "plain_bytes_per_pair": 8.0,
+                    "bytes_per_pair": round(4.0 + idx_bytes, 3),                      # coded indices, plain values
+                    "bytes_per_pair_values_packed": round(idx_bytes + val_bytes, 3),  # coded indices, packed values
+                    "index_bytes": round(idx_bytes, 3), "value_bytes": round(val_bytes, 3),
+                    "encode_ms": round(enc_ms, 4), "decode_ms": round(dec_ms, 4),
+                    "encode_pairs_per_s": round(W * p.K / enc_ms * 1e3, 1), "decode_pairs_per_s": round(W * p.K / dec_ms * 1e3, 1),
+                    "values_encode_ms": round(venc_ms, 4), "values_decode_ms": round(vdec_ms, 4)})
+        del vwords, voff, vback
     return out
 
 

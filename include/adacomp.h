@@ -354,6 +354,30 @@ ADACOMP_API int adacomp_decode_indices(const uint32_t* d_words, uint64_t words_p
                                        const uint64_t* d_block_off, uint64_t pairs_per_worker,
                                        uint32_t n_workers, uint32_t* d_idx_out, int device, void* cuda_stream);
 
+/* ---- value packing ------------------------------------------------------------------------
+ * The value half of the same open point (footnote of "Algorithm details"), lossless: every fp32
+ * bit pattern comes back as it went in, so Eq. 4 sees the same inputs.  A worker's
+ * pairs_per_worker values are cut into blocks of 256 entries, like the indices.  With E(x) the
+ * 8-bit exponent field of x, a block is stored as: one word e_min | w_e << 8 (e_min the smallest
+ * E in the block, w_e the number of bits of the largest E - e_min, 0 .. 8); then the block's n
+ * entries, 24 + w_e bits each, entry t at bit t * (24 + w_e) of a little-endian bit string held in
+ * 32-bit words, an entry being the 23 mantissa bits, above them E - e_min in w_e bits, above
+ * that the sign.  (The largest magnitudes of a tensor lie within a few powers of two of each
+ * other: 26 or 27 bits a value.)  d_block_off and d_words are laid out as for the indices;
+ * words_per_worker must be at least adacomp_encode_values_capacity_words(pairs_per_worker)
+ * (ADACOMP_ERR_CAPACITY otherwise).  All arrays are the caller's device memory.  Decoding does not
+ * trust the stream: a block whose header has w_e > 8 or other bits set, or whose offset or
+ * payload would reach outside the worker's words_per_worker words, is not read; all its entries
+ * decode to +0.0, a value that changes no parameter, and so does an entry whose exponent would
+ * come out above 255. */
+ADACOMP_API uint64_t adacomp_encode_values_capacity_words(uint64_t pairs_per_worker);
+ADACOMP_API int adacomp_encode_values(const float* d_val, uint64_t pairs_per_worker, uint32_t n_workers,
+                                      uint32_t* d_words, uint64_t words_per_worker, uint64_t* d_block_off,
+                                      int device, void* cuda_stream);
+ADACOMP_API int adacomp_decode_values(const uint32_t* d_words, uint64_t words_per_worker,
+                                      const uint64_t* d_block_off, uint64_t pairs_per_worker,
+                                      uint32_t n_workers, float* d_val_out, int device, void* cuda_stream);
+
 #ifdef __cplusplus
 }
 #endif

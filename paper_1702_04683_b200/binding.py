@@ -77,6 +77,9 @@ def _load():
         "adacomp_encode_capacity_words": (u64, [u64]),
         "adacomp_encode_indices": (i32, [vp, u64, u32, vp, u64, vp, i32, vp]),
         "adacomp_decode_indices": (i32, [vp, u64, vp, u64, u32, vp, i32, vp]),
+        "adacomp_encode_values_capacity_words": (u64, [u64]),
+        "adacomp_encode_values": (i32, [vp, u64, u32, vp, u64, vp, i32, vp]),
+        "adacomp_decode_values": (i32, [vp, u64, vp, u64, u32, vp, i32, vp]),
         "adacomp_server_set_rule": (i32, [vp, i32]),
         "adacomp_apply_dense": (i32, [vp, vp, u64, f32, vp]),
         "adacomp_select_gather": (i32, [vp, vp, u64, u32, vp, vp, vp]),
@@ -203,6 +206,34 @@ def adacomp_decode_indices(words: torch.Tensor, block_off: torch.Tensor, pairs_p
     _check(_lib.adacomp_decode_indices(_dev(words, torch.int32, "words"), words.shape[1], _dev(block_off, torch.int64, "block_off"),
                                        int(pairs_per_worker), W, out.data_ptr(), words.device.index or 0, _stream_ptr(stream)),
            "adacomp_decode_indices")
+    return out
+
+
+def adacomp_encode_values_capacity_words(pairs_per_worker: int) -> int:
+    return int(_lib.adacomp_encode_values_capacity_words(int(pairs_per_worker)))
+
+
+def adacomp_encode_values(val: torch.Tensor, stream: Optional[torch.cuda.Stream] = None):
+    """val [W, K] float32 -> (words [W, capacity] int32, block_off [W, n_blocks + 1] int64): the lossless block-wise
+    packing of every worker's values."""
+    if val.dim() == 1:
+        val = val.unsqueeze(0)
+    W, K = val.shape
+    cap = adacomp_encode_values_capacity_words(K)
+    words = torch.empty((W, max(cap, 1)), dtype=torch.int32, device=val.device)
+    off = torch.empty((W, (K + 255) // 256 + 1), dtype=torch.int64, device=val.device)
+    _check(_lib.adacomp_encode_values(_dev(val, torch.float32, "val") if K else None, K, W, words.data_ptr(), words.shape[1],
+                                      off.data_ptr(), val.device.index or 0, _stream_ptr(stream)), "adacomp_encode_values")
+    return words, off
+
+
+def adacomp_decode_values(words: torch.Tensor, block_off: torch.Tensor, pairs_per_worker: int,
+                          stream: Optional[torch.cuda.Stream] = None) -> torch.Tensor:
+    W = words.shape[0]
+    out = torch.empty((W, pairs_per_worker), dtype=torch.float32, device=words.device)
+    _check(_lib.adacomp_decode_values(_dev(words, torch.int32, "words"), words.shape[1], _dev(block_off, torch.int64, "block_off"),
+                                      int(pairs_per_worker), W, out.data_ptr(), words.device.index or 0, _stream_ptr(stream)),
+           "adacomp_decode_values")
     return out
 
 

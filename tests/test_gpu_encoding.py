@@ -1,5 +1,5 @@
-"""Parity of the index coding (CUDA, through the C ABI) with the CPU oracle: the streams and the
-block offsets word for word, and the round trip."""
+"""Parity of the index coding and of the value packing (CUDA, through the C ABI) with the CPU oracle: the
+streams and the block offsets word for word, and the round trip."""
 import numpy as np
 import pytest
 import torch
@@ -111,3 +111,85 @@ def test_corrupt_streams_are_not_followed(binding):
     want[0, 256:512] = want[0, 512:768] = 0xFFFFFFFF
     want[1, 768:] = 0xFFFFFFFF
     assert np.array_equal(back, want)
+
+
+# ----------------------------------------------------------------------------- value packing
+
+def check_values(binding, val_rows):
+    """val_rows: [W, K] float32 numpy (any bit patterns).  Packs on the GPU, compares the stream and the block
+    offsets with the oracle word for word, unpacks again: every bit pattern must come back."""
+    rows = np.ascontiguousarray(val_rows, dtype=np.float32)
+    val = torch.from_numpy(rows.view(np.int32)).to(DEV).view(torch.float32)
+    W, K = val.shape
+    words, off = binding.adacomp_encode_values(val)
+    torch.cuda.synchronize()
+    h_words, h_off = words.cpu().numpy().view(np.uint32), off.cpu().numpy().astype(np.uint64)
+    total = 0
+    for w in range(W):
+        ow, oo = oracle.encode_values(rows[w])
+        assert np.array_equal(h_off[w], oo), f"worker {w}: block offsets differ"
+        assert np.array_equal(h_words[w, :ow.size], ow), f"worker {w}: stream differs"
+        total += ow.size
+    back = binding.adacomp_decode_values(words, off, K)
+    assert np.array_equal(back.view(torch.int32).cpu().numpy().view(np.uint32), rows.view(np.uint32))
+    return 4.0 * total / max(1, W * K)
+
+
+@pytest.mark.parametrize("K", [0, 1, 2, 255, 256, 257, 512, 70_001])
+@pytest.mark.parametrize("spread", [0.0, 2.0, 40.0])
+def test_values_around_the_block_boundaries(binding, K, spread):
+    rng = np.random.default_rng(K + int(spread))
+    rows = (rng.standard_normal((3, K)) * np.exp2(rng.uniform(-spread, spread, (3, K)))).astype(np.float32)
+    check_values(binding, rows)
+
+
+def test_every_kind_of_bit_pattern_is_packed_and_comes_back(binding):
+    pats = np.array([0x00000000, 0x80000000, 0x00000001, 0x807FFFFF, 0x00800000, 0x7F7FFFFF, 0xFF7FFFFF, 0x7F800000,
+                     0xFF800000, 0x7FC00000, 0xFFC12345, 0x7F800001, 0x3F800000, 0xBF800000], dtype=np.uint32)
+    assert check_values(binding, pats.view(np.float32)[None]) > 4.0          # all 8 exponent bits: 32 bits an entry + the header
+    rng = np.random.default_rng(9)
+    anything = rng.integers(0, 2**32, (2, 5000), dtype=np.uint64).astype(np.uint32)
+    check_values(binding, anything.view(np.float32))
+    same = np.full((1, 600), -0.375, np.float32)                              # one exponent: 24 bits an entry
+    assert check_values(binding, same) < 3.03
+    with pytest.raises(binding.AdacompError) as e:                            # stream capacity too small
+        v = torch.zeros((1, 1000), device=DEV)
+        small = torch.empty((1, 1000), dtype=torch.int32, device=DEV)
+        off = torch.empty((1, 5), dtype=torch.int64, device=DEV)
+        binding._check(binding.raw().adacomp_encode_values(v.data_ptr(), 1000, 1, small.data_ptr(), 1000, off.data_ptr(), 0, 0), "enc")
+    assert e.value.status == binding.ERR_CAPACITY
+
+
+@pytest.mark.parametrize("keep", [(1, 1000), (1, 100), (1, 10)])
+def test_selected_values_of_a_workload(binding, keep):
+    """What adacomp_select emits, packed: bytes per value against the 4 of the plain list, on Gaussian gradients
+    (the large flat workload, scaled down) and on the heavy-tailed tie-stress workload."""
+    wl = wlmod.workload(4).scaled(16, n_workers=3)
+    sel = binding.Selector(binding.make_segments(wl.tensor_sizes, keep), 3, DEV)
+    _, val = sel.select(wlmod.round_gradients(wl, 0, DEV))
+    assert check_values(binding, val.cpu().numpy()) < 3.4
+    wl = wlmod.workload(2)
+    sel = binding.Selector(binding.make_segments(wl.tensor_sizes, keep), 5, DEV)
+    _, val = sel.select(wlmod.round_gradients(wl, 0, DEV, workers=range(5)))
+    assert check_values(binding, val.cpu().numpy()) < 4.0
+
+
+def test_corrupt_value_streams_are_not_followed(binding):
+    """Block offsets that point outside the stream, a header no encoder writes, or a payload that would run past the
+    end must not be read: the block unpacks to +0.0 (a value that changes no parameter), the other blocks are intact."""
+    rng = np.random.default_rng(6)
+    K = 1000                                                    # four blocks
+    rows = rng.standard_normal((2, K)).astype(np.float32)
+    val = torch.from_numpy(rows).to(DEV)
+    words, off = binding.adacomp_encode_values(val)
+    cap = words.shape[1]
+    bad_off = off.clone()
+    bad_off[0, 1] = 10**12                                      # block 1 of worker 0: far outside the stream
+    bad_off[1, 3] = cap - 3                                     # block 3 of worker 1: its payload would run past the end
+    bad_words = words.clone()
+    bad_words[0, int(off[0, 2])] = 9 << 8                       # block 2 of worker 0: an exponent width of 9 bits
+    back = binding.adacomp_decode_values(bad_words, bad_off, K).cpu().numpy()
+    want = rows.copy()
+    want[0, 256:768] = 0.0
+    want[1, 768:] = 0.0
+    assert np.array_equal(back.view(np.uint32), want.view(np.uint32))
