@@ -38,8 +38,8 @@ FALLBACK_HBM_GBS = 6650.0
 # workers moves W / 4 times as much (every worker's tensors are independent).  The apply kernel was captured with all 16
 # updates in the launch on tensors four times smaller: parameters and pairs, hence the traffic, are a quarter of a
 # full-size launch's.  Only valid while the kernel sources are the ones that were profiled (guarded by their hashes).
-SCAN_TRAFFIC_W4_MB = {'1/1000': 1617.7, '1/400': 1627.8, '1/160': 1648.6, '1/64': 1692.6, '1/25': 1789.1, '1/10': 2010.7}
-APPLY_TRAFFIC_DIV4_MB = {'1/1000': 91.3, '1/400': 190.1, '1/160': 321.8, '1/64': 463.4, '1/25': 583.9, '1/10': 925.6}
+SCAN_TRAFFIC_W4_MB = {'1/1000': 1617.6, '1/400': 1628.4, '1/160': 1648.4, '1/64': 1695.6, '1/25': 1788.5, '1/10': 2010.7}
+APPLY_TRAFFIC_DIV4_MB = {'1/1000': 91.0, '1/400': 190.3, '1/160': 321.6, '1/64': 463.4, '1/25': 583.7, '1/10': 926.0}
 SCAN_SOURCE_SHA256_16 = "b3f19e7900b079fc"
 APPLY_SOURCE_SHA256_16 = "0402d0792ba9bb99"
 
