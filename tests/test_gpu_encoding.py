@@ -193,3 +193,27 @@ def test_corrupt_value_streams_are_not_followed(binding):
     want[0, 256:768] = 0.0
     want[1, 768:] = 0.0
     assert np.array_equal(back.view(np.uint32), want.view(np.uint32))
+
+
+def test_full_size_values_round_trip_and_sampled_blocks(binding):
+    """10^7 values per worker (the largest update of the benchmark, as the selector emits it for 4 workers): round
+    trip on the GPU bit for bit, the oracle on sampled blocks."""
+    wl = wlmod.workload(4)
+    import dataclasses
+    wl4 = dataclasses.replace(wl, n_workers=4)
+    sel = binding.Selector(binding.make_segments(wl.tensor_sizes, (1, 10)), 4, DEV)
+    _, val = sel.select(wlmod.round_gradients(wl4, 0, DEV))
+    K = val.shape[1]
+    words, off = binding.adacomp_encode_values(val)
+    back = binding.adacomp_decode_values(words, off, K)
+    assert torch.equal(back.view(torch.int32), val.view(torch.int32))
+    h_off = off.cpu().numpy()
+    rng = np.random.default_rng(4)
+    for _ in range(40):
+        w, b = int(rng.integers(4)), int(rng.integers((K + 255) // 256))
+        blk = val[w, 256 * b:256 * b + 256].cpu().numpy()
+        ow, _ = oracle.encode_values(blk)
+        lo = int(h_off[w, b])
+        assert int(h_off[w, b + 1]) - lo == ow.size
+        assert np.array_equal(u32(words[w, lo:lo + ow.size]), ow)
+    assert 4.0 * float(h_off[:, -1].sum()) / (4 * K) < 3.3      # 26 to 27 bits a value
