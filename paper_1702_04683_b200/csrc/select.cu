@@ -333,7 +333,10 @@ int adacomp_select_create(adacomp_select_t** h, const adacomp_segment_t* h_segs,
     if (e == cudaSuccess && !lay.items.empty())
         e = cudaMemcpy(s->d_items, lay.items.data(), lay.items.size() * sizeof(uint2), cudaMemcpyHostToDevice);
     if (e == cudaSuccess)
-        e = cudaFuncSetAttribute(k_bracket_sample, cudaFuncAttributeMaxDynamicSharedMemorySize,
+        e = cudaFuncSetAttribute(k_bracket_sample<kBigFew>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                 static_cast<int>(kSmallMax * sizeof(uint32_t)));
+    if (e == cudaSuccess)
+        e = cudaFuncSetAttribute(k_bracket_sample<kBigMany>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                  static_cast<int>(kSmallMax * sizeof(uint32_t)));
     if (e == cudaSuccess)
         e = cudaFuncSetAttribute(k_bracket_scan, cudaFuncAttributeMaxDynamicSharedMemorySize,
@@ -429,7 +432,12 @@ int adacomp_select(adacomp_select_t* h, const float* d_grads, uint64_t worker_st
     // single-pass routes: sample (and the tensors that are selected on chip), the one pass over the gradient,
     // the exact threshold, the ordered write
     ADACOMP_CUDA(begin(0));
-    k_bracket_sample<<<n_inst, kBig, bracketed ? h->max_sample * sizeof(uint32_t) : 0, st>>>(p, bracketed ? (clusters ? 2 : 0) : 1);
+    // per-instance kernels: smaller blocks when the instances are many (more of them resident, finer rounds)
+    const bool many = n_inst > 2u * static_cast<uint32_t>(h->n_sms);
+    const size_t sample_smem = bracketed ? h->max_sample * sizeof(uint32_t) : 0;
+    const int sample_mode = bracketed ? (clusters ? 2 : 0) : 1;
+    if (many) k_bracket_sample<kBigMany><<<n_inst, kBigMany, sample_smem, st>>>(p, sample_mode);
+    else k_bracket_sample<kBigFew><<<n_inst, kBigFew, sample_smem, st>>>(p, sample_mode);
     ADACOMP_LAUNCH_CHECK();
     ADACOMP_CUDA(end());
     if (bracketed && h->n_items > 0) {
@@ -439,7 +447,8 @@ int adacomp_select(adacomp_select_t* h, const float* d_grads, uint64_t worker_st
         ADACOMP_LAUNCH_CHECK();
         ADACOMP_CUDA(end());
         ADACOMP_CUDA(begin(2));
-        k_bracket_resolve<<<n_inst, kBig, 0, st>>>(p);
+        if (many) k_bracket_resolve<kBigMany><<<n_inst, kBigMany, 0, st>>>(p);
+        else k_bracket_resolve<kBigFew><<<n_inst, kBigFew, 0, st>>>(p);
         ADACOMP_LAUNCH_CHECK();
         ADACOMP_CUDA(end());
         ADACOMP_CUDA(begin(3));
@@ -477,7 +486,7 @@ int adacomp_select(adacomp_select_t* h, const float* d_grads, uint64_t worker_st
         unsigned solo = static_cast<unsigned>(h->n_sms) * 2;
         if (solo > n_inst) solo = n_inst;
         ADACOMP_CUDA(begin(10));
-        k_fallback_solo<<<solo, kBig, 0, st>>>(p);
+        k_fallback_solo<<<solo, kSoloThreads, 0, st>>>(p);
         ADACOMP_LAUNCH_CHECK();
         ADACOMP_CUDA(end());
         return ADACOMP_OK;
@@ -716,7 +725,7 @@ extern "C" int adacomp_select_static(const float* d_grad, uint32_t n, uint32_t k
     if (grid > L.n_slots) grid = L.n_slots;
     k_static_setup<<<1, kThreads, 0, st>>>(L);
     ADACOMP_LAUNCH_CHECK();
-    k_bracket_sample<<<1, kBig, 0, st>>>(p, 1);                 // general route only: resets the instance record
+    k_bracket_sample<kBigFew><<<1, kBigFew, 0, st>>>(p, 1);     // general route only: resets the instance record
     ADACOMP_LAUNCH_CHECK();
     k_general_plan<<<1, kThreads, 0, st>>>(p);
     ADACOMP_LAUNCH_CHECK();

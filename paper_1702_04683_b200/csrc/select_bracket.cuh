@@ -41,8 +41,13 @@ constexpr uint32_t kSmallMax = kBracketMinN - 1;         // longest tensor whose
 constexpr uint32_t kSampleMin = 2048;
 constexpr float kBracketZ = 5.0f;                     // half-width of the bracket in sample standard deviations
 constexpr uint32_t kGatherMax = 1024;
-constexpr int kBig = 512;                             // threads of the per-instance kernels (measured: 1024 and 256 are slower
-                                                      // where a call has thousands of small tensors, equal elsewhere)
+// Threads of the per-instance kernels (sample, resolve): a template parameter, chosen per call by the number of
+// instances.  Measured: with thousands of instances (the ResNet-50-shaped call has 5152) 512 threads are 9 % faster
+// over the whole call than 1024, with 400 instances 1 % faster, with 16 instances (one segment over a whole model of
+// 10^8 parameters) 10 % slower.
+constexpr int kBigFew = 1024;                         // calls with few instances
+constexpr int kBigMany = 512;                         // calls with many
+constexpr int kSoloThreads = 512;                     // the fallback kernel
 
 constexpr uint32_t kRouteSmall = 3u;                  // Layer::bracket of a tensor that is selected whole in shared memory
 constexpr uint32_t kInstBracket = 2u;                 // bracket valid, scan/emit act on the instance
@@ -65,17 +70,18 @@ __device__ __forceinline__ uint32_t hash32(uint32_t x) {
 }
 
 // Descending walk over a 2048-bin histogram in shared memory: the bucket holding the rem-th
-// largest.  All kBig threads call; results are returned to all.
+// largest.  All kT threads of the block call; results are returned to all.
+template <int kT>
 __device__ __forceinline__ void block_pick_bucket(const uint32_t* hist, uint32_t rem, uint32_t* bucket,
                                                   uint32_t* above_out, uint32_t* count_out,
                                                   uint32_t* s_warp /*[33]*/, uint32_t* s_bc /*[3]*/) {
-    constexpr int M = 2048 / kBig;
+    constexpr int M = 2048 / kT;
     const int top = 2047 - static_cast<int>(threadIdx.x) * M;
     uint32_t h[M], sum = 0;
 #pragma unroll
     for (int q = 0; q < M; ++q) { h[q] = hist[top - q]; sum += h[q]; }
     uint32_t total;
-    uint32_t above = block_exclusive_scan_t<kBig>(sum, &total, s_warp);
+    uint32_t above = block_exclusive_scan_t<kT>(sum, &total, s_warp);
 #pragma unroll
     for (int q = 0; q < M; ++q) {
         if (above < rem && rem <= above + h[q]) { s_bc[0] = top - q; s_bc[1] = above; s_bc[2] = h[q]; }
@@ -87,6 +93,7 @@ __device__ __forceinline__ void block_pick_bucket(const uint32_t* hist, uint32_t
 }
 
 // rank-th largest (1 = largest) of m keys in shared memory; three digit passes.
+template <int kT>
 __device__ uint32_t smem_kth_largest(const uint32_t* keys, uint32_t m, uint32_t rank, uint32_t* hist,
                                      uint32_t* s_warp, uint32_t* s_bc) {
     uint32_t prefix = 0, rem = rank;
@@ -94,16 +101,16 @@ __device__ uint32_t smem_kth_largest(const uint32_t* keys, uint32_t m, uint32_t 
     for (int pass = 0; pass < 3; ++pass) {
         const int shift = pass == 0 ? 20 : (pass == 1 ? 10 : 0);
         const int nb = pass == 0 ? 2048 : 1024;
-        for (int b = threadIdx.x; b < 2048; b += kBig) hist[b] = 0;
+        for (int b = threadIdx.x; b < 2048; b += kT) hist[b] = 0;
         __syncthreads();
-        for (uint32_t i = threadIdx.x; i < m; i += kBig) {
+        for (uint32_t i = threadIdx.x; i < m; i += kT) {
             const uint32_t key = keys[i];
             const bool match = pass == 0 || (key >> (shift + 10)) == (prefix >> (shift + 10));
             if (match) atomicAdd(&hist[(key >> shift) & (nb - 1)], 1u);
         }
         __syncthreads();
         uint32_t b, above, cnt;
-        block_pick_bucket(hist, rem, &b, &above, &cnt, s_warp, s_bc);   // unused upper bins are zero
+        block_pick_bucket<kT>(hist, rem, &b, &above, &cnt, s_warp, s_bc);   // unused upper bins are zero
         prefix |= b << shift;
         rem -= above;
     }
@@ -113,7 +120,8 @@ __device__ uint32_t smem_kth_largest(const uint32_t* keys, uint32_t m, uint32_t 
 // ---------------------------------------------------------------------------------------------
 // One block per (worker, tensor): reset the instance, and bracket its threshold if it is on
 // this route.  Dynamic shared memory: the sample keys.
-__global__ void __launch_bounds__(kBig) k_bracket_sample(SelectParams p, int general_only) {
+template <int kT>
+__global__ void __launch_bounds__(kT) k_bracket_sample(SelectParams p, int general_only) {
     extern __shared__ uint32_t s_keys[];
     __shared__ uint32_t s_hist[2048];
     __shared__ uint32_t s_warp[33];
@@ -137,12 +145,12 @@ __global__ void __launch_bounds__(kBig) k_bracket_sample(SelectParams p, int gen
         // digit passes over the keys on chip, then an ordered write (a warp per stretch of the tensor)
         const float* first = p.grads + static_cast<uint64_t>(w) * p.stride + L.offset;
         const uint32_t n = L.n, k = L.k;
-        for (uint32_t i = threadIdx.x; i < n; i += kBig) s_keys[i] = magnitude_key(first[i]);
+        for (uint32_t i = threadIdx.x; i < n; i += kT) s_keys[i] = magnitude_key(first[i]);
         __syncthreads();
         // k-th largest key; with k = n every entry is kept (T = 0: all keys are above or equal)
-        const uint32_t T = k < n ? smem_kth_largest(s_keys, n, k, s_hist, s_warp, s_bc) : 0u;
+        const uint32_t T = k < n ? smem_kth_largest<kT>(s_keys, n, k, s_hist, s_warp, s_bc) : 0u;
         const uint32_t lane = threadIdx.x & 31, warp = threadIdx.x >> 5, lt = (1u << lane) - 1u;
-        constexpr uint32_t kWarps = kBig / 32;
+        constexpr uint32_t kWarps = kT / 32;
         const uint32_t seg = (((n + kWarps - 1) / kWarps) + 31) & ~31u;    // entries per warp, a multiple of 32
         const uint32_t e0 = warp * seg < n ? warp * seg : n, e1 = e0 + seg < n ? e0 + seg : n;
         uint32_t gt = 0, eq = 0;
@@ -203,7 +211,7 @@ __global__ void __launch_bounds__(kBig) k_bracket_sample(SelectParams p, int gen
     }
     {   // the scan only writes the table entries of pieces that hold candidates
         uint2* sub_tab = p.sub_tab + (static_cast<uint64_t>(w) * p.span_stride + L.span_base) * kSubsPerSpan;
-        for (uint32_t t = threadIdx.x; t < L.n_spans * kSubsPerSpan; t += kBig) sub_tab[t] = make_uint2(0u, 0u);
+        for (uint32_t t = threadIdx.x; t < L.n_spans * kSubsPerSpan; t += kT) sub_tab[t] = make_uint2(0u, 0u);
     }
 
     const float* first = p.grads + static_cast<uint64_t>(w) * p.stride + L.offset;
@@ -212,7 +220,7 @@ __global__ void __launch_bounds__(kBig) k_bracket_sample(SelectParams p, int gen
     const uint32_t m = L.sample, n_chunks = m / 32, stratum = L.n / n_chunks;   // stratum >= 128
     // chunk j: 32 consecutive entries starting at a hashed position inside stratum j, moved up to
     // the next 32-byte boundary; always inside the tensor
-    for (uint32_t t = threadIdx.x; t < n_chunks * 8; t += kBig) {
+    for (uint32_t t = threadIdx.x; t < n_chunks * 8; t += kT) {
         const uint32_t j = t >> 3, part = t & 7;
         const uint32_t e = j * stratum + hash32(j * 2654435761u + l * 40503u + 977u) % (stratum - 40);
         const uint32_t s = (e + mis + 7) & ~7u;                  // shifted coordinate, multiple of 8
@@ -228,8 +236,8 @@ __global__ void __launch_bounds__(kBig) k_bracket_sample(SelectParams p, int gen
         if (threadIdx.x == 0) st->flags = kInstGeneral;
         return;
     }
-    const uint32_t t_lo = smem_kth_largest(s_keys, m, r_lo, s_hist, s_warp, s_bc);
-    uint32_t t_hi = r_hi ? smem_kth_largest(s_keys, m, r_hi, s_hist, s_warp, s_bc) : 0x7FFFFFFFu;
+    const uint32_t t_lo = smem_kth_largest<kT>(s_keys, m, r_lo, s_hist, s_warp, s_bc);
+    uint32_t t_hi = r_hi ? smem_kth_largest<kT>(s_keys, m, r_hi, s_hist, s_warp, s_bc) : 0x7FFFFFFFu;
     if (t_hi > 0x7F800000u) t_hi = 0x7FFFFFFFu;       // "no upper bound" (as a float: unordered)
     // the scan compares magnitudes as floats and blanks padding with zeros: it needs a positive,
     // non-NaN lower bound
@@ -585,7 +593,8 @@ __global__ void __launch_bounds__(kThreads, 4) k_bracket_scan(SelectParams p) {
 
 // ---------------------------------------------------------------------------------------------
 // One block per instance: exact threshold inside the window, per-span output offsets.
-__global__ void __launch_bounds__(kBig) k_bracket_resolve(SelectParams p) {
+template <int kT>
+__global__ void __launch_bounds__(kT) k_bracket_resolve(SelectParams p) {
     __shared__ uint32_t s_hist[2048];
     __shared__ uint32_t s_sel[kMaxSpans];
     __shared__ unsigned long long s_g[kGatherMax];
@@ -621,17 +630,17 @@ __global__ void __launch_bounds__(kBig) k_bracket_resolve(SelectParams p) {
     // fetched before any is used, so their loads overlap (a pass over the list is bound by their latency)
     auto for_each_window = [&](auto fn) {
         constexpr int kAhead = 8;
-        for (uint32_t i0 = threadIdx.x; i0 < n_win; i0 += kBig * kAhead) {
+        for (uint32_t i0 = threadIdx.x; i0 < n_win; i0 += kT * kAhead) {
             uint32_t key[kAhead], idx[kAhead];
 #pragma unroll
             for (int u = 0; u < kAhead; ++u) {
-                const uint32_t i = i0 + u * kBig;
+                const uint32_t i = i0 + u * kT;
                 key[u] = i < n_win ? __ldcg(&win_key[i]) : 0u;
                 idx[u] = i < n_win ? __ldcg(&win_idx[i]) : 0u;
             }
 #pragma unroll
             for (int u = 0; u < kAhead; ++u)
-                if (i0 + u * kBig < n_win)
+                if (i0 + u * kT < n_win)
                     fn((static_cast<unsigned long long>(key[u] - t_lo) << 32) |
                            static_cast<unsigned long long>(0xFFFFFFFFu - idx[u]),
                        idx[u]);
@@ -641,7 +650,7 @@ __global__ void __launch_bounds__(kBig) k_bracket_resolve(SelectParams p) {
     // that receives the spans' output offsets anyway.  The pass that collects the last undecided entries
     // also counts the entries it sees above them, so the list is not read again once the threshold is known.
     uint32_t* sel = L.n_spans <= kMaxSpans ? s_sel : span_off;
-    for (uint32_t s = threadIdx.x; s < L.n_spans; s += kBig) sel[s] = 0;
+    for (uint32_t s = threadIdx.x; s < L.n_spans; s += kT) sel[s] = 0;
     if (threadIdx.x == 0) s_carry = 0;
     __syncthreads();
     bool failed = false;
@@ -662,7 +671,7 @@ __global__ void __launch_bounds__(kBig) k_bracket_resolve(SelectParams p) {
                     else if (top > prefix) atomicAdd(&sel[idx / kSpanElems], 1u);   // above the undecided ones: kept
                 });
                 __syncthreads();
-                for (uint32_t t = threadIdx.x; t < count; t += kBig) {
+                for (uint32_t t = threadIdx.x; t < count; t += kT) {
                     const unsigned long long mine = s_g[t];
                     uint32_t larger = 0;
                     for (uint32_t u = 0; u < count; ++u) larger += s_g[u] > mine ? 1u : 0u;
@@ -670,14 +679,14 @@ __global__ void __launch_bounds__(kBig) k_bracket_resolve(SelectParams p) {
                 }
                 __syncthreads();
                 cstar = s_cstar;
-                for (uint32_t t = threadIdx.x; t < count; t += kBig)      // the kept ones among the collected entries
+                for (uint32_t t = threadIdx.x; t < count; t += kT)      // the kept ones among the collected entries
                     if (s_g[t] >= cstar) atomicAdd(&sel[(0xFFFFFFFFu - static_cast<uint32_t>(s_g[t])) / kSpanElems], 1u);
                 break;
             }
             if (hi_shift == 0) { failed = true; break; }      // cannot happen: composites are distinct
             const int bits = hi_shift < 11 ? hi_shift : 11;
             const int new_shift = hi_shift - bits;
-            for (int b = threadIdx.x; b < 2048; b += kBig) s_hist[b] = 0;
+            for (int b = threadIdx.x; b < 2048; b += kT) s_hist[b] = 0;
             __syncthreads();
             for_each_window([&](unsigned long long c, uint32_t) {
                 if ((c >> hi_shift) == prefix)
@@ -685,7 +694,7 @@ __global__ void __launch_bounds__(kBig) k_bracket_resolve(SelectParams p) {
             });
             __syncthreads();
             uint32_t b, above, cnt;
-            block_pick_bucket(s_hist, rem, &b, &above, &cnt, s_warp, s_bc);
+            block_pick_bucket<kT>(s_hist, rem, &b, &above, &cnt, s_warp, s_bc);
             prefix = (prefix << bits) | b;
             rem -= above;
             count = cnt;
@@ -694,7 +703,7 @@ __global__ void __launch_bounds__(kBig) k_bracket_resolve(SelectParams p) {
     }
     __syncthreads();
     // exclusive prefix of kept entries over the spans
-    for (uint32_t base = 0; base < L.n_spans; base += kBig) {
+    for (uint32_t base = 0; base < L.n_spans; base += kT) {
         const uint32_t s = base + threadIdx.x;
         uint32_t kept = 0;
         if (s < L.n_spans) {
@@ -703,7 +712,7 @@ __global__ void __launch_bounds__(kBig) k_bracket_resolve(SelectParams p) {
             for (uint32_t j = 0; j < kSubsPerSpan; ++j) kept += __ldcg(&sub_tab[s * kSubsPerSpan + j]).y >> 16;
         }
         uint32_t tot;
-        const uint32_t ex = block_exclusive_scan_t<kBig>(kept, &tot, s_warp);
+        const uint32_t ex = block_exclusive_scan_t<kT>(kept, &tot, s_warp);
         const uint32_t carry = s_carry;
         if (s < L.n_spans) span_off[s] = carry + ex;
         __syncthreads();
@@ -807,7 +816,7 @@ __global__ void __launch_bounds__(kThreads) k_bracket_emit(SelectParams p) {
 // then one more pass writes, in index order, every entry with key > T and the r lowest-index entries
 // with key == T (a block walks its tensor front to back, so the running counts are simply carried
 // along: no count pass).  Four reads of the tensor, the later ones mostly from L2.
-__global__ void __launch_bounds__(kBig) k_fallback_solo(SelectParams p) {
+__global__ void __launch_bounds__(kSoloThreads) k_fallback_solo(SelectParams p) {
     __shared__ uint32_t s_hist[2048];
     __shared__ uint32_t s_warp[33];
     __shared__ uint32_t s_bc[3];
@@ -828,9 +837,9 @@ __global__ void __launch_bounds__(kBig) k_fallback_solo(SelectParams p) {
             for (int pass = 0; pass < 3; ++pass) {
                 const int shift = pass == 0 ? 20 : (pass == 1 ? 10 : 0);
                 const uint32_t nb = pass == 0 ? 2048u : 1024u;
-                for (int b = threadIdx.x; b < 2048; b += kBig) s_hist[b] = 0;
+                for (int b = threadIdx.x; b < 2048; b += kSoloThreads) s_hist[b] = 0;
                 __syncthreads();
-                for (uint64_t base = 0; base < nvec; base += kBig) {
+                for (uint64_t base = 0; base < nvec; base += kSoloThreads) {
                     const uint64_t v = base + threadIdx.x;
                     float4 x = make_float4(0.f, 0.f, 0.f, 0.f);
                     if (v < nvec) x = __ldg(&vec[v]);
@@ -847,7 +856,7 @@ __global__ void __launch_bounds__(kBig) k_fallback_solo(SelectParams p) {
                 }
                 __syncthreads();
                 uint32_t b, above, cnt;
-                block_pick_bucket(s_hist, rem, &b, &above, &cnt, s_warp, s_bc);   // unused upper bins are zero
+                block_pick_bucket<kSoloThreads>(s_hist, rem, &b, &above, &cnt, s_warp, s_bc);   // unused upper bins are zero
                 prefix |= b << shift;
                 rem -= above;
             }
@@ -857,7 +866,7 @@ __global__ void __launch_bounds__(kBig) k_fallback_solo(SelectParams p) {
         uint32_t gt_base = 0, eq_base = 0;
         uint32_t* idx_out = p.idx_out + static_cast<uint64_t>(w) * p.K + L.out_offset;
         float* val_out = p.val_out + static_cast<uint64_t>(w) * p.K + L.out_offset;
-        for (uint64_t base = 0; base < nvec; base += kBig) {
+        for (uint64_t base = 0; base < nvec; base += kSoloThreads) {
             const uint64_t v = base + threadIdx.x;
             float xs[4] = {0.f, 0.f, 0.f, 0.f};
             uint32_t gtm = 0, eqm = 0;
@@ -875,8 +884,8 @@ __global__ void __launch_bounds__(kBig) k_fallback_solo(SelectParams p) {
             }
             // a tile holds 4096 entries: both counts fit 16 bits only up to 4095, so they are scanned apart
             uint32_t tot_gt, tot_eq;
-            uint32_t gt_before = gt_base + block_exclusive_scan_t<kBig>(__popc(gtm), &tot_gt, s_warp);
-            uint32_t eq_before = eq_base + block_exclusive_scan_t<kBig>(__popc(eqm), &tot_eq, s_warp);
+            uint32_t gt_before = gt_base + block_exclusive_scan_t<kSoloThreads>(__popc(gtm), &tot_gt, s_warp);
+            uint32_t eq_before = eq_base + block_exclusive_scan_t<kSoloThreads>(__popc(eqm), &tot_eq, s_warp);
 #pragma unroll
             for (int q = 0; q < 4; ++q) {
                 const bool is_gt = (gtm >> q) & 1u, is_eq = (eqm >> q) & 1u;
