@@ -305,7 +305,7 @@ __device__ __forceinline__ bool mbar_try_wait(uint32_t mbar, uint32_t parity) {
         : "=r"(ok) : "r"(mbar), "r"(parity) : "memory");
     return ok != 0;
 }
-// bytes: a multiple of 16; both addresses 16-byte aligned.  No multicast: the copy lands in this block only.
+// bytes: a multiple of 16; both addresses 16-byte aligned.  The copy lands in this block only (a plain bulk copy).
 __device__ __forceinline__ void bulk_load(uint32_t smem_dst, const void* gmem_src, uint32_t bytes, uint32_t mbar) {
     asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
                  ::"r"(smem_dst), "l"(gmem_src), "r"(bytes), "r"(mbar) : "memory");
