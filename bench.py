@@ -40,7 +40,7 @@ FALLBACK_HBM_GBS = 6650.0
 # full-size launch's.  Only valid while the kernel sources are the ones that were profiled (guarded by their hashes).
 SCAN_TRAFFIC_W4_MB = {'1/1000': 1617.6, '1/400': 1628.4, '1/160': 1648.4, '1/64': 1695.6, '1/25': 1788.5, '1/10': 2010.7}
 APPLY_TRAFFIC_DIV4_MB = {'1/1000': 91.0, '1/400': 190.3, '1/160': 321.6, '1/64': 463.4, '1/25': 583.7, '1/10': 926.0}
-SCAN_SOURCE_SHA256_16 = "ce1457ee33fe090e"
+SCAN_SOURCE_SHA256_16 = "fa86615eff0206da"
 APPLY_SOURCE_SHA256_16 = "0402d0792ba9bb99"
 
 

@@ -23,6 +23,7 @@ struct adacomp_select {
     int route = 0;         // 0 = automatic, 1 = general route for everything
     bool all_bracketed = false;   // every tensor with k > 0 is eligible for the bracketed route
     bool any_small = false;       // some tensor is selected whole in shared memory by the sample kernel
+    bool emit_thin = false;       // every tensor of the list route expects a handful of candidates per piece: a lane per piece writes them
     // cluster route: large tensors selected by one thread-block cluster each, everything between the pass and the write on chip
     uint32_t n_cl = 0;            // tensors on the cluster route
     uint32_t cl_ctas = 0, cl_warps = 0, cl_ring = 0, cl_qmax = 0, cl_smem = 0;   // blocks per cluster, warps per block, ring slots per warp, most pieces per block, shared memory per block
@@ -309,6 +310,12 @@ int adacomp_select_create(adacomp_select_t** h, const adacomp_segment_t* h_segs,
         if (L.k > 0 && !L.bracket) s->all_bracketed = false;
     s->max_sample = lay.max_sample;
     s->any_small = lay.any_small;
+    {   // at most about six candidates per 1024-entry piece everywhere: the thin form of the ordered write
+        double most = 0.0;
+        for (uint32_t l = 0; l < lay.layers.size(); ++l)
+            if (lay.layers[l].bracket == 1 && lay.cand_frac[l] > most) most = lay.cand_frac[l];
+        s->emit_thin = most > 0.0 && most * kSubElems <= 6.0;      // measured: at ten per piece the warp-per-span form is faster again
+    }
     s->cand_stride = lay.cand_stride;
     s->win_stride = lay.win_stride;
     s->span_stride = lay.span_stride;
@@ -452,7 +459,8 @@ int adacomp_select(adacomp_select_t* h, const float* d_grads, uint64_t worker_st
         ADACOMP_LAUNCH_CHECK();
         ADACOMP_CUDA(end());
         ADACOMP_CUDA(begin(3));
-        k_bracket_emit<<<grid, kThreads, 0, st>>>(p);
+        if (h->emit_thin) k_bracket_emit_thin<<<grid, kEmitThinThreads, 0, st>>>(p);
+        else k_bracket_emit<<<grid, kThreads, 0, st>>>(p);
         ADACOMP_LAUNCH_CHECK();
         ADACOMP_CUDA(end());
     }

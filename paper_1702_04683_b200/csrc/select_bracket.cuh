@@ -808,6 +808,75 @@ __global__ void __launch_bounds__(kThreads) k_bracket_emit(SelectParams p) {
 }
 
 // ---------------------------------------------------------------------------------------------
+// The same ordered write for calls whose tensors have a handful of candidates per piece (low keep fractions): there
+// the kernel above spends a warp, and its whole set-up, on a span with a dozen candidates, and is bound by instruction
+// issue.  Here a LANE takes a piece and a warp four spans: the lane reads its piece's table entry, walks the piece's
+// candidates once to count the kept ones (remembering which of the first 32), a scan over the eight lanes of a span
+// gives it its place behind the span's output offset, and it walks them again to write.  grid = (scan items,
+// workers), two warps per block.  Any data is handled, only not fast when pieces hold many candidates.
+constexpr int kEmitThinThreads = 64;
+__global__ void __launch_bounds__(kEmitThinThreads) k_bracket_emit_thin(SelectParams p) {
+    const uint2 item = p.items[blockIdx.x];
+    const uint32_t l = item.x, w = blockIdx.y;
+    const Layer L = p.layers[l];
+    const Inst* st = &p.inst[w * p.n_layers + l];
+    if (!(__ldcg(&st->flags) & kInstBracket)) return;
+    const uint32_t lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const uint32_t sub = lane & 7u;
+    const uint32_t s = item.y + warp * 4 + (lane >> 3);        // kSpansPerBlock = 8 spans per item: two warps, four spans each
+    static_assert(kSpansPerBlock == 8 && kSubsPerSpan == 8, "a lane per piece, eight lanes per span, two warps per item");
+    const bool valid = s < L.n_spans;
+    const uint32_t T = __ldcg(&st->T), cut = __ldcg(&st->cut);
+    const float* first = p.grads + static_cast<uint64_t>(w) * p.stride + L.offset;
+    const uint32_t mis = static_cast<uint32_t>((reinterpret_cast<uintptr_t>(first) >> 2) & 3u);
+    const uint32_t* cand_idx = p.cand_idx + static_cast<uint64_t>(w) * p.cand_stride + L.cand_base;
+    const float* cand_val = p.cand_val + static_cast<uint64_t>(w) * p.cand_stride + L.cand_base;
+    const uint64_t span_at = static_cast<uint64_t>(w) * p.span_stride + L.span_base + s;
+    uint2 tab = make_uint2(0, 0);
+    uint32_t off = 0;
+    if (valid) {
+        tab = __ldcg(&p.sub_tab[span_at * kSubsPerSpan + sub]);
+        off = __ldcg(&p.span_off[span_at]);
+    }
+    const uint32_t cnt = tab.y & 0xFFFFu, at = tab.x;
+    uint32_t kept = 0, keep_mask = 0;
+    for (uint32_t i = 0; i < cnt; ++i) {
+        const uint32_t e = __ldg(&cand_idx[at + i]);
+        const uint32_t key = magnitude_key(__ldg(&cand_val[at + i]));
+        const uint32_t k = (key > T || (key == T && e < cut)) ? 1u : 0u;
+        kept += k;
+        if (i < 32) keep_mask |= k << i;
+    }
+    uint32_t inc = kept;                                       // inclusive prefix over the 8 pieces of the span
+#pragma unroll
+    for (int d = 1; d < 8; d <<= 1) {
+        const uint32_t y = __shfl_up_sync(0xFFFFFFFFu, inc, d);
+        if (sub >= static_cast<uint32_t>(d)) inc += y;
+    }
+    if (!kept) return;
+    uint32_t pos = off + inc - kept;
+    uint32_t* idx_out = p.idx_out + static_cast<uint64_t>(w) * p.K + L.out_offset;
+    float* val_out = p.val_out + static_cast<uint64_t>(w) * p.K + L.out_offset;
+    const uint32_t glob = static_cast<uint32_t>(L.offset) - mis;        // shifted coordinate -> vector index
+    for (uint32_t i = 0; i < cnt; ++i) {
+        const uint32_t e = __ldg(&cand_idx[at + i]);
+        const float v = __ldg(&cand_val[at + i]);
+        bool keep;
+        if (i < 32) {
+            keep = (keep_mask >> i) & 1u;
+        } else {
+            const uint32_t key = magnitude_key(v);
+            keep = key > T || (key == T && e < cut);
+        }
+        if (keep) {
+            __stcs(&idx_out[pos], glob + e);
+            __stcs(&val_out[pos], v);
+            ++pos;
+        }
+    }
+}
+
+// ---------------------------------------------------------------------------------------------
 // The general route done by ONE block per instance, for layouts whose tensors are all on a single-pass
 // route: only instances whose bracket missed (or that hold a NaN) are flagged then, which is rare, so
 // one launch that usually finds nothing replaces the general route's six.  A block takes the flagged

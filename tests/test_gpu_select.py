@@ -194,6 +194,32 @@ def test_dense_candidates_crowded_and_spread(binding):
         assert general <= 1                                            # at most the tied worker fell back
 
 
+@pytest.mark.parametrize("k", [40, 1_500, 6_000])
+def test_low_keep_fractions_with_candidates_crowded_into_a_few_pieces(binding, k):
+    """Keep fractions of 1/37 500 to 1/250 pick the form of the ordered write in which a lane takes a piece: evenly
+    spread data (a few candidates per piece), a burst of large entries inside two pieces (far more than 32 candidates
+    in a piece), data concentrated near zero, a coarse grid with ties at every level, two tensors of different
+    lengths side by side, odd alignment."""
+    dev = torch.device("cuda", 0)
+    n, n2 = 1_500_001, 70_000
+    gen = torch.Generator(device=dev)
+    gen.manual_seed(100 + k)
+    g = torch.randn((4, n + n2 + 5), device=dev, generator=gen)[:, 1:n + n2 + 1]
+    g[1, 300_100:301_900] *= 50.0                                      # 1800 large entries in a row
+    g[2, :n] *= torch.rand(n, device=dev, generator=gen) ** 4          # heavy concentration near zero
+    g[3, :n] = torch.round(g[3, :n] * 4) / 4                           # coarse grid: many ties at every level
+    k2 = max(1, k // 20)
+    sel = binding.Selector(binding.segments_from([0, n], [n, n2], [k, k2]), 4, dev)
+    for _ in range(2):
+        idx, val = sel.select(g)
+    status, general = sel.last_error()
+    assert status == 0 and general <= 2                                 # at most the tied row's tensors fell back
+    for w in range(4):
+        oi, ov = oracle.select_layers(g[w].cpu().numpy(), [0, n], [n, n2], [k, k2])
+        assert np.array_equal(u32(idx[w]), oi), (k, w)
+        assert np.array_equal(bits(val[w]), bits(ov)), (k, w)
+
+
 @pytest.mark.parametrize("k", [1, 1_500, 75_000, 300_000])
 def test_cluster_route_on_large_tensors(binding, k):
     """Route 2: tensors of a million entries or more are selected by one thread-block cluster each, which
