@@ -466,7 +466,7 @@ def run_native(args):
     for _ in range(args.warmup):
         one_step(None)
     for p in points:
-        p.sel.set_profiling(True)      # CUDA events around every select kernel of the timed steps (no syncs)
+        p.sel.set_profiling(2)         # CUDA events around the scan kernel of every timed select call (no syncs)
     barrier()
     sampler = ClockSampler(local)
     if rank == 0:
@@ -488,6 +488,16 @@ def run_native(args):
         t = torch.tensor([total_ms], device=dev, dtype=torch.float64)
         dist.all_reduce(t, op=dist.ReduceOp.MAX)
         total_ms = float(t.item())
+    scan_profiles = [p.sel.profile() for p in points]        # the scan kernel, over the timed steps
+    # where the rest of a select call goes: two more steps, not timed, with events around every kernel
+    for p in points:
+        p.sel.set_profiling(1)
+    for _ in range(2):
+        one_step(None)
+    barrier()
+    stage_profiles = [p.sel.profile() for p in points]
+    for p in points:
+        p.sel.set_profiling(0)
     status = [p.sel.last_error()[0] for p in points] + [srv.last_error()]
     if any(status):
         raise SystemExit(f"device-side error recorded during the benchmark: {status}")
@@ -500,9 +510,11 @@ def run_native(args):
     W_sel = W // world if sharded else W          # workers one rank selects for
     apply_points = []
     for i, p in enumerate(points):
-        stages = p.sel.profile()
-        calls = stages.pop("calls")
-        scan_ms_all += stages["bracket_scan"]
+        calls = scan_profiles[i].pop("calls")
+        stages = stage_profiles[i]
+        stages.pop("calls")
+        scan_ms_timed = scan_profiles[i]["bracket_scan"]
+        scan_ms_all += scan_ms_timed
         scan_bytes_all += W_sel * 4.0 * P
         scan_launches += calls
         sel_ms = statistics.mean(m[i][0].elapsed_time(m[i][1]) for m in rec)
@@ -532,6 +544,8 @@ def run_native(args):
             "apply_updates_per_s": round(W / app_ms * 1e3, 1),
             "apply_alg_gbs_28B_per_pair": round(pairs * 28.0 / app_ms / 1e6, 1),
             "apply_alg_frac_of_hbm_peak": round(pairs * 28.0 / app_ms / 1e6 / peak, 4),
+            "scan_kernel_ms": round(scan_ms_timed, 4),                       # in the timed steps
+            # every kernel of the call, from two extra steps after the timed ones (events between the kernels lengthen a call)
             "select_stage_ms": {k: round(v, 4) for k, v in stages.items() if v > 0},
         })
         sel_ms_all += sel_ms

@@ -146,8 +146,10 @@ ADACOMP_API int adacomp_select_set_route(adacomp_select_t* h, int route);
  * no tensor is on that route. */
 ADACOMP_API int adacomp_select_route_info(const adacomp_select_t* h, uint32_t* h_info_out);
 
-/* Stage timing.  With profiling on, every adacomp_select call records CUDA events on its stream
- * around each of its kernels (a few microseconds of host work per call, no synchronisation).
+/* Stage timing.  With profiling on (on = 1), every adacomp_select call records CUDA events on its stream
+ * around each of its kernels (no synchronisation; the events between the kernels cost some ten
+ * microseconds per call on the device); on = 2 records them around the one pass over the gradient
+ * only (stage "bracket_scan"), which leaves the call's own duration practically untouched.
  * adacomp_select_profile waits for the calls made since profiling was switched on and writes
  * the mean device time per call of each stage, in milliseconds, to h_ms_out[0 .. n_stages),
  * n_stages = the number of stages adacomp_select_stage_name knows (0 for a stage that never ran),

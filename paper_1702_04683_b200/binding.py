@@ -317,7 +317,8 @@ class Selector:
         return {"cluster_tensors": int(info[0]), "blocks_per_cluster": int(info[1]), "ring_slots": int(info[2]) & 255,
                 "warps_per_block": int(info[2]) >> 8, "resident_clusters": int(info[3])}
 
-    def set_profiling(self, on: bool):
+    def set_profiling(self, on):
+        """False / 0: off; True / 1: CUDA events around every kernel; 2: around the pass over the gradient only."""
         _check(_lib.adacomp_select_set_profiling(self._h, int(on)), "adacomp_select_set_profiling")
 
     def profile(self) -> dict:

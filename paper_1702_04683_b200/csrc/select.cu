@@ -50,7 +50,7 @@ struct adacomp_select {
     uint2* d_sub_tab = nullptr;
     uint32_t* d_span_off = nullptr;
     // optional stage timing: a ring of event lists, one per call, folded into sums when reused or read
-    bool profiling = false;
+    int profiling = 0;            // 0 off, 1 events around every kernel, 2 around the pass over the gradient only
     struct Span { int stage; cudaEvent_t a, b; };
     std::vector<Span> spans[kProfileRing];
     size_t spans_used[kProfileRing] = {};
@@ -418,8 +418,10 @@ int adacomp_select(adacomp_select_t* h, const float* d_grads, uint64_t worker_st
         h->ring_used[slot] = true;
     }
     // begin(stage) ... end(): CUDA events around one launch (only while profiling)
+    bool recording = false;
     auto begin = [&](int stage) -> cudaError_t {
-        if (!h->profiling) return cudaSuccess;
+        recording = h->profiling == 1 || (h->profiling == 2 && stage == 1);
+        if (!recording) return cudaSuccess;
         std::vector<adacomp_select::Span>& v = h->spans[slot];
         if (h->spans_used[slot] == v.size()) {
             adacomp_select::Span sp = {stage, nullptr, nullptr};
@@ -432,7 +434,7 @@ int adacomp_select(adacomp_select_t* h, const float* d_grads, uint64_t worker_st
         return cudaEventRecord(v[h->spans_used[slot]].a, st);
     };
     auto end = [&]() -> cudaError_t {
-        if (!h->profiling) return cudaSuccess;
+        if (!recording) return cudaSuccess;
         return cudaEventRecord(h->spans[slot][h->spans_used[slot]++].b, st);
     };
 
@@ -541,7 +543,7 @@ int adacomp_select_set_profiling(adacomp_select_t* h, int on) {
     for (int r = 0; r < kProfileRing; ++r) ADACOMP_CUDA(fold_profile_slot(h, r));
     for (int i = 0; i < kSelectStages; ++i) h->stage_ms_sum[i] = 0.0;      // a fresh measurement starts here
     h->profiled_calls = 0;
-    h->profiling = on != 0;
+    h->profiling = on == 2 ? 2 : (on != 0 ? 1 : 0);
     return ADACOMP_OK;
 }
 
