@@ -405,3 +405,30 @@ def test_nan_orders_above_inf_on_every_route(binding):
     # every NaN of worker 1 is among the kept entries of its tensor (it orders above everything finite)
     kept = set(h_idx[1].tolist())
     assert all(int(i) in kept for i in np.flatnonzero(np.isnan(g[1])))
+
+
+def test_stage_timing_modes_leave_the_result_alone(binding):
+    """Events around every kernel (1), around the pass over the gradient only (2), or none (0): the same pairs come
+    out, the call count is the number of calls since the switch, and mode 2 reports that one stage only."""
+    dev = torch.device("cuda", 0)
+    n, k = 600_000, 3_000
+    gen = torch.Generator(device=dev)
+    gen.manual_seed(31)
+    g = torch.randn((3, n), device=dev, generator=gen)
+    sel = binding.Selector(binding.segments_from([0], [n], [k]), 3, dev)
+    want_idx, want_val = sel.select(g)
+    want_idx, want_val = want_idx.clone(), want_val.clone()
+    for mode, calls in ((1, 3), (2, 2), (0, 1)):
+        sel.set_profiling(mode)
+        for _ in range(calls):
+            idx, val = sel.select(g)
+        assert torch.equal(idx, want_idx) and torch.equal(val.view(torch.int32), want_val.view(torch.int32))
+        if mode:
+            prof = sel.profile()
+            assert prof.pop("calls") == calls
+            timed = {name for name, ms in prof.items() if ms > 0}
+            assert "bracket_scan" in timed
+            assert (timed == {"bracket_scan"}) == (mode == 2)
+    assert sel.last_error() == (0, 0)
+    oi, ov = oracle.select(g[1].cpu().numpy(), k)
+    assert np.array_equal(u32(want_idx[1]), oi) and np.array_equal(bits(want_val[1]), bits(ov))
