@@ -180,8 +180,11 @@ __device__ __forceinline__ uint32_t first_at_or_above(const uint32_t* __restrict
 constexpr int kWpThreads = 128;
 constexpr uint32_t kWpWarps = kWpThreads / 32;
 
+// Buffers for Theta and the records of a range: two (the next range arrives while this one is worked on), or one for
+// ranges of 512, where shared memory, not registers, decides how many warps an SM holds.
+__host__ __device__ constexpr uint32_t wp_bufs(uint32_t range) { return range >= 512 ? 1u : 2u; }
 __host__ __device__ inline size_t wp_warp_words(uint32_t range, bool pre) {
-    return (pre ? 7 : 6) * static_cast<size_t>(range);          // Theta twice, (mask, head) records twice, (heads at the launch's start)
+    return (3 * wp_bufs(range) + (pre ? 1 : 0)) * static_cast<size_t>(range);   // Theta, (mask, head) records, (heads at the launch's start)
 }
 __host__ __device__ inline size_t wp_smem_bytes(uint32_t range, bool pre) {
     return 64 * 4 + kWpWarps * wp_warp_words(range, pre) * 4;
@@ -214,8 +217,9 @@ k_apply_warps(const ServerParams sp, const BatchDesc d, const uint32_t* __restri
     // [2][R] per parameter ONE 8-byte record: .x = updates of this launch that changed it (mask), .y = its latest change
     // (head).  A pair reads and writes both with one access each: the shared-memory pipe is what bounds this kernel, and
     // lanes that fall on the same bank cost a pass each.
-    uint2* s_rec = reinterpret_cast<uint2*>(s_theta + 2 * R);
-    uint32_t* s_head0 = reinterpret_cast<uint32_t*>(s_rec + 2 * R);             // [R] head when the launch began (kPre)
+    constexpr uint32_t kBufs = wp_bufs(R);
+    uint2* s_rec = reinterpret_cast<uint2*>(s_theta + kBufs * R);
+    uint32_t* s_head0 = reinterpret_cast<uint32_t*>(s_rec + kBufs * R);         // [R] head when the launch began (kPre)
 
     if (tid < kAlphaTable) s_alpha[tid] = tid ? __fdiv_rn(lr, static_cast<float>(tid)) : lr;   // Eq. 5 for the small counts, once
     __syncthreads();                                            // the only block barrier
@@ -270,15 +274,20 @@ k_apply_warps(const ServerParams sp, const BatchDesc d, const uint32_t* __restri
     copy_async_commit();
 
     for (uint32_t r = r_lo; r < r_hi; ++r) {
-        const uint32_t p = (r - r_lo) & 1u;
+        const uint32_t p = kBufs == 2 ? (r - r_lo) & 1u : 0u;
         const uint32_t lo = r * R, hi = range_end(r);
         float* th = s_theta + p * R;
         uint2* rec = s_rec + p * R;
-        if (r + 1 < r_hi) sweep_in(r + 1, p ^ 1u);              // lands while this range is worked on
+        if (kBufs == 2) {
+            if (r + 1 < r_hi) sweep_in(r + 1, p ^ 1u);          // lands while this range is worked on
+        } else if (r != r_lo) {
+            sweep_in(r, 0);                                     // one buffer: free since the last range went back
+        }
         copy_async_commit();
 #pragma unroll
-        for (uint32_t o = lane; o < R; o += 32) rec[o].x = 0u;  // (the heads of this buffer were copied in a range ago: other bytes)
-        copy_async_wait<1>();                                   // this range's Theta and heads have landed
+        for (uint32_t o = lane; o < R; o += 32) rec[o].x = 0u;  // (the heads are copied into other bytes of the records)
+        if (kBufs == 2) copy_async_wait<1>();                   // this range's Theta and heads have landed
+        else copy_async_wait<0>();
         __syncwarp();
         if (kPre) {
 #pragma unroll
@@ -1232,7 +1241,7 @@ static int apply_body(adacomp_server_t* s, const uint32_t* d_idx, const float* d
                 d.gate_lo = 0;
                 d.gate_hi = crowded_from;
             }
-            if (dens * 512.0 <= 4.0) rc = launch_apply_merged<512>(s, sp, d, pairs, d_idx, d_val, lr, d_sigma_out, st);
+            if (dens * 512.0 <= 6.0) rc = launch_apply_merged<512>(s, sp, d, pairs, d_idx, d_val, lr, d_sigma_out, st);
             else rc = launch_apply_merged<256>(s, sp, d, pairs, d_idx, d_val, lr, d_sigma_out, st);
         } else if (sweep) {
             // range size: the densest update should bring about 26 pairs per range (mean of a uniformly spread
