@@ -38,10 +38,10 @@ FALLBACK_HBM_GBS = 6650.0
 # workers moves W / 4 times as much (every worker's tensors are independent).  The apply kernel was captured with all 16
 # updates in the launch on tensors four times smaller: parameters and pairs, hence the traffic, are a quarter of a
 # full-size launch's.  Only valid while the kernel sources are the ones that were profiled (guarded by their hashes).
-SCAN_TRAFFIC_W4_MB = {'1/1000': 1617.3, '1/400': 1628.2, '1/160': 1648.3, '1/64': 1693.1, '1/25': 1789.1, '1/10': 2010.9}
-APPLY_TRAFFIC_DIV4_MB = {'1/1000': 91.0, '1/400': 190.3, '1/160': 321.6, '1/64': 462.6, '1/25': 583.6, '1/10': 924.9}
+SCAN_TRAFFIC_W4_MB = {'1/1000': 1617.2, '1/400': 1627.7, '1/160': 1648.3, '1/64': 1691.3, '1/25': 1789.2, '1/10': 2010.6}
+APPLY_TRAFFIC_DIV4_MB = {'1/1000': 91.3, '1/400': 190.1, '1/160': 327.4, '1/64': 463.5, '1/25': 632.0, '1/10': 924.8}
 SCAN_SOURCE_SHA256_16 = "fa86615eff0206da"
-APPLY_SOURCE_SHA256_16 = "0402d0792ba9bb99"
+APPLY_SOURCE_SHA256_16 = "6dff16245f48ee38"
 
 
 def _source_hash(name):
